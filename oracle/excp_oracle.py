@@ -1,0 +1,513 @@
+"""CPU oracle for the ExCP per-tensor compression path (arXiv 2406.11257).
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain, single-threaded
+statement of what the CUDA library must compute.  It shares no code with the
+CUDA path and is never imported by it; only the tests, the smoke check and the
+benchmark's CPU-baseline leg may call it.
+
+What is written from the paper, and where the paper is silent:
+
+  * residual                 Section 3.1, Eq. (ckpt_res); Algorithm 1, step 1
+  * weight mask  (M2W)       Section 3.2, Eq. (rw)
+  * moment mask  (W2M)       Section 3.2, Eq. (ro)
+  * joint application        Algorithm 1, step 2 ("joint_prune")
+  * non-uniform quantisation Section 3.3 (K-means to 2^n - 1 centres, zero keeps
+                             one code) and Section 4.1 (n = 4, two codes per byte)
+  * reconstruction           Algorithm 2
+
+The paper does not say how the median, the mean, the K-means start, its
+iteration count, its arithmetic or the byte layout are to be taken.  The
+readings used here (all of them deterministic, so that the result is unique):
+
+  R1  median(W) in Eq. (rw) is the LOWER median (rank floor((n-1)/2)) of the
+      absolute values of either W_t (the letter of the text) or dW_t (the
+      quantity actually pruned); `median_source` selects.
+  R2  the mask of Eq. (rw) compares |dW(i)| * sqrt(m_t(i)) > alpha * median in
+      fp32 (the product form of |dW(i)| > alpha / sqrt(m_t(i)) * median, which
+      also settles m_t(i) = 0 as "pruned").
+  R3  mean(v_t) in Eq. (ro) is the mean of |v_t|, taken EXACTLY (as a rational
+      number) and rounded once to fp32, round-to-nearest-even.
+  R4  both Adam moments take the mask M_o (Appendix A prunes "the moments").
+  R5  K-means is Lloyd's algorithm in one dimension, per tensor and per stream
+      (dW, first moment, second moment), K = 2^bits - 1 centres:
+        start   the K equal-mass quantiles of a seeded, index-stratified sample
+                of at most 1024 surviving values;
+        assign  nearest centre, a point on a mid-point going to the lower
+                centre, the mid-point of two neighbours taken in fp64:
+                cluster(x) = #{ j : 2x > c_j + c_(j+1) }
+                (of coincident centres the first takes the points at or
+                below them, the last those above);
+        update  fixed-point mean (rule R-SUM below); a cluster without members
+                keeps its centre; centres are re-sorted ascending;
+        T fixed iterations, then one last assignment gives the codes 1..K.
+  R-SUM a sum that feeds a centre is taken in fixed point so that its value
+      cannot depend on the order of summation: with E = max(floor(log2(max|x|)),
+      -126) over the stream, Q(x) = rint(x * 2^(30-E)) (half-to-even), the sum
+      of Q in int64, mean = fp32( fp64(sum) / fp64(count) * 2^(E-30) ).
+  R6  byte layout: see `encode_record`.
+
+The paper calls Adam's first moment v_t and its second moment m_t; to stay clear
+of the clash with the usual letters the code below says `ea` (first moment,
+exp_avg) and `eas` (second moment, exp_avg_sq).
+
+Parity status: every function below is pinned by tests/test_oracle_pins.py
+(hand-computed example, brute force, exact rational arithmetic, invariants).
+"""
+from __future__ import annotations
+
+import math
+import struct
+from dataclasses import dataclass
+from fractions import Fraction
+
+import numpy as np
+
+MAGIC = 0x50435845  # "EXCP", little endian
+VERSION = 1
+SAMPLE_MAX = 1024
+HEADER_FIXED = 64
+
+MEDIAN_ABS_WEIGHT = 0
+MEDIAN_ABS_RESIDUAL = 1
+
+_M64 = (1 << 64) - 1
+
+
+@dataclass
+class Params:
+    """Hyper-parameters.  alpha, beta, bits: Section 4.1 (5e-5, 2.0, 4)."""
+    alpha: float = 5e-5
+    beta: float = 2.0
+    bits: int = 4
+    kmeans_iters: int = 10
+    seed: int = 0
+    median_source: int = MEDIAN_ABS_WEIGHT
+
+
+class InvalidInput(ValueError):
+    """A NaN, an infinity, or a negative second moment in the inputs."""
+
+
+class CorruptBlob(ValueError):
+    """The record does not parse."""
+
+
+# --------------------------------------------------------------------------
+# Section 3.1: residual
+# --------------------------------------------------------------------------
+def residual(w_t: np.ndarray, w_prev: np.ndarray) -> np.ndarray:
+    """dW_t = W_t - W^_(t-1), fp32 (Eq. ckpt_res; Algorithm 1, first step)."""
+    return np.subtract(w_t, w_prev, dtype=np.float32)
+
+
+# --------------------------------------------------------------------------
+# Section 3.2: statistics behind the two thresholds
+# --------------------------------------------------------------------------
+def lower_median_abs(x: np.ndarray) -> np.float32:
+    """Lower median of |x| (reading R1): the element of rank floor((n-1)/2)."""
+    n = x.size
+    if n == 0:
+        return np.float32(0.0)
+    a = np.abs(x.astype(np.float32, copy=False))
+    k = (n - 1) // 2
+    return np.float32(np.partition(a, k)[k])
+
+
+def round_ratio_to_f32(num: int, den: int) -> np.float32:
+    """The fp32 value nearest to num/den (num >= 0, den > 0), ties to even,
+    subnormals included; integer arithmetic only."""
+    if num < 0 or den <= 0:
+        raise ValueError("num >= 0 and den > 0 required")
+    if num == 0:
+        return np.float32(0.0)
+    e = num.bit_length() - den.bit_length()
+    # make 2^e <= num/den < 2^(e+1)
+    if e >= 0:
+        below = num < (den << e)
+    else:
+        below = (num << -e) < den
+    if below:
+        e -= 1
+    u = max(e - 23, -149)            # exponent of the last kept bit
+    if u >= 0:
+        n_, d_ = num, den << u
+    else:
+        n_, d_ = num << -u, den
+    m, r = divmod(n_, d_)
+    if 2 * r > d_ or (2 * r == d_ and (m & 1)):
+        m += 1
+    return np.float32(math.ldexp(m, u))
+
+
+def exact_sum_abs_units(x: np.ndarray) -> int:
+    """sum |x_i| as an integer count of 2^-149 (every fp32 is a multiple of it)."""
+    a = np.abs(x.astype(np.float32, copy=False)).ravel()
+    if a.size >= (1 << 29):
+        raise ValueError("tensor too large for the exact per-exponent sums")
+    bits = a.view(np.uint32)
+    e = (bits >> 23).astype(np.int64)
+    m = (bits & np.uint32(0x7FFFFF)).astype(np.int64)
+    m = np.where(e > 0, m | (1 << 23), m)
+    e1 = np.maximum(e, 1)            # subnormals share the exponent of 2^-126
+    total = 0
+    # 24-bit mantissas times fewer than 2^29 terms stay below 2^53: the
+    # float64 weights of bincount add without rounding.
+    per_exp = np.bincount(e1, weights=m.astype(np.float64), minlength=256)
+    for ee in range(1, 256):
+        s = int(per_exp[ee])
+        if s:
+            total += s << (ee - 1)   # value = m * 2^(ee-150) = m * 2^(ee-1) units
+    return total
+
+
+def exact_mean_abs(x: np.ndarray) -> np.float32:
+    """mean(|x|), exact then rounded once to fp32 (reading R3)."""
+    n = x.size
+    if n == 0:
+        return np.float32(0.0)
+    return round_ratio_to_f32(exact_sum_abs_units(x), n << 149)
+
+
+def validate_inputs(w_t, w_prev, ea, eas) -> None:
+    for a in (w_t, w_prev, ea, eas):
+        if not np.all(np.isfinite(a)):
+            raise InvalidInput("non-finite input")
+    if np.any(eas < 0):
+        raise InvalidInput("negative second moment")
+
+
+# --------------------------------------------------------------------------
+# Section 3.2: the two masks and their joint application
+# --------------------------------------------------------------------------
+def weight_mask(dw: np.ndarray, eas: np.ndarray, alpha, med) -> tuple[np.ndarray, np.float32]:
+    """M_w of Eq. (rw) in the product form of reading R2."""
+    thr_w = np.float32(np.float32(alpha) * np.float32(med))
+    lhs = np.abs(dw).astype(np.float32) * np.sqrt(eas.astype(np.float32))
+    return lhs > thr_w, thr_w
+
+
+def moment_mask(ea: np.ndarray, m_w: np.ndarray, beta, mean) -> tuple[np.ndarray, np.float32]:
+    """M_o of Eq. (ro): |first moment| above beta * mean AND the weight kept."""
+    thr_o = np.float32(np.float32(beta) * np.float32(mean))
+    return (np.abs(ea) > thr_o) & m_w, thr_o
+
+
+# --------------------------------------------------------------------------
+# Section 3.3: non-uniform quantisation (reading R5)
+# --------------------------------------------------------------------------
+def mix64(z: int) -> int:
+    """One step of the SplitMix64 generator (Steele, Lea, Flood 2014) from state z."""
+    z = (z + 0x9E3779B97F4A7C15) & _M64
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & _M64
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & _M64
+    return z ^ (z >> 31)
+
+
+def sample_hash(seed: int, tensor_index: int, stream: int, i: int) -> int:
+    h = mix64((seed + tensor_index) & _M64)
+    h = mix64((h + stream) & _M64)
+    return mix64((h + i) & _M64)
+
+
+def kmeans_start(s: np.ndarray, k: int, seed: int, tensor_index: int, stream: int) -> np.ndarray:
+    """K equal-mass quantiles of a seeded, index-stratified sample of s."""
+    nnz = s.size
+    c = np.zeros(k, dtype=np.float32)
+    if nnz == 0:
+        return c
+    m = min(nnz, SAMPLE_MAX)
+    picks = np.empty(m, dtype=np.float32)
+    for i in range(m):
+        lo = (i * nnz) // m
+        hi = ((i + 1) * nnz) // m
+        picks[i] = s[lo + sample_hash(seed, tensor_index, stream, i) % (hi - lo)]
+    picks.sort()
+    for j in range(k):
+        c[j] = picks[((2 * j + 1) * m) // (2 * k)]
+    return c
+
+
+def assign(s: np.ndarray, c: np.ndarray) -> np.ndarray:
+    """Nearest centre: the number of mid-points lying strictly below x."""
+    x2 = 2.0 * s.astype(np.float64)
+    idx = np.zeros(s.shape, dtype=np.int64)
+    for j in range(len(c) - 1):
+        idx += x2 > (np.float64(c[j]) + np.float64(c[j + 1]))
+    return idx
+
+
+def rsum_exponent(s: np.ndarray) -> int:
+    if s.size == 0:
+        return 0
+    mx = float(np.max(np.abs(s)))
+    if mx == 0.0:
+        return 0
+    return max(math.frexp(mx)[1] - 1, -126)
+
+
+def rsum_quantize(s: np.ndarray, e: int) -> np.ndarray:
+    return np.rint(np.ldexp(s.astype(np.float64), 30 - e)).astype(np.int64)
+
+
+def rsum_mean(qsum: int, count: int, e: int) -> np.float32:
+    return np.float32(math.ldexp(float(qsum) / float(count), e - 30))
+
+
+def lloyd(s: np.ndarray, c0: np.ndarray, iters: int) -> tuple[np.ndarray, np.ndarray]:
+    """T Lloyd iterations from c0, then the final assignment.
+    Returns (centres, cluster index per value)."""
+    c = c0.astype(np.float32).copy()
+    k = len(c)
+    if s.size == 0:
+        return c, np.zeros(0, dtype=np.int64)
+    e = rsum_exponent(s)
+    q = rsum_quantize(s, e)
+    for _ in range(iters):
+        idx = assign(s, c)
+        for j in range(k):
+            members = idx == j
+            cnt = int(np.count_nonzero(members))
+            if cnt:
+                c[j] = rsum_mean(int(q[members].sum(dtype=np.int64)), cnt, e)
+        c.sort()
+    return c, assign(s, c)
+
+
+# --------------------------------------------------------------------------
+# Byte layout (reading R6)
+# --------------------------------------------------------------------------
+def _align16(n: int) -> int:
+    return (n + 15) & ~15
+
+
+def header_bytes(k: int) -> int:
+    return _align16(HEADER_FIXED + 3 * 4 * k)
+
+
+def bitmap_bytes(numel: int) -> int:
+    return _align16(4 * ((numel + 31) // 32))
+
+
+def code_bytes(nnz: int, bits: int) -> int:
+    return _align16((nnz * bits + 7) // 8)
+
+
+def record_bytes(numel: int, nnz_w: int, nnz_o: int, bits: int) -> int:
+    k = (1 << bits) - 1
+    return (header_bytes(k) + 2 * bitmap_bytes(numel) + code_bytes(nnz_w, bits)
+            + 2 * code_bytes(nnz_o, bits))
+
+
+def pack_codes(codes: np.ndarray, bits: int) -> bytes:
+    """Code r sits at bit r*bits of the stream, low bits first (Section 4.1:
+    two 4-bit codes per byte)."""
+    per = 8 // bits
+    n = codes.size
+    padded = np.zeros(((n + per - 1) // per) * per, dtype=np.uint8)
+    padded[:n] = codes
+    out = np.zeros(padded.size // per, dtype=np.uint8)
+    for r in range(per):
+        out |= (padded[r::per] << np.uint8(r * bits)).astype(np.uint8)
+    raw = out.tobytes()
+    return raw + b"\0" * (code_bytes(n, bits) - len(raw))
+
+
+def unpack_codes(raw: bytes, nnz: int, bits: int) -> np.ndarray:
+    per = 8 // bits
+    b = np.frombuffer(raw, dtype=np.uint8)
+    out = np.zeros(b.size * per, dtype=np.uint8)
+    for r in range(per):
+        out[r::per] = (b >> np.uint8(r * bits)) & np.uint8((1 << bits) - 1)
+    return out[:nnz]
+
+
+def pack_bitmap(mask: np.ndarray) -> bytes:
+    """Bit k of 32-bit little-endian word w is element 32*w + k."""
+    raw = np.packbits(mask.astype(np.uint8), bitorder="little").tobytes()
+    return raw + b"\0" * (bitmap_bytes(mask.size) - len(raw))
+
+
+def unpack_bitmap(raw: bytes, numel: int) -> np.ndarray:
+    b = np.frombuffer(raw, dtype=np.uint8)
+    return np.unpackbits(b, bitorder="little")[:numel].astype(bool)
+
+
+def encode_record(numel, bits, m_w, m_o, c_w, c_ea, c_eas, codes_w, codes_ea, codes_eas) -> bytes:
+    """One tensor's record.  Little endian; every section starts on 16 bytes;
+    padding is zero.
+
+      0  u32 magic "EXCP"     4  u32 version (1)    8  u64 numel
+     16  u64 nnz_w           24  u64 nnz_o         32  u32 bits   36 u32 K
+     40  u32 header bytes    44  u32 zero          48  u64 record bytes
+     56  u64 zero
+     64  fp32 centres of dW [K], of the first moment [K], of the second [K]
+     ..  bitmap of M_w, bitmap of M_o       (u32 words, LSB = lowest index)
+     ..  codes of dW, of the first moment, of the second moment (survivors in
+         index order, `bits` each, value 1..K)
+    """
+    k = (1 << bits) - 1
+    nnz_w = int(np.count_nonzero(m_w))
+    nnz_o = int(np.count_nonzero(m_o))
+    hb = header_bytes(k)
+    total = record_bytes(numel, nnz_w, nnz_o, bits)
+    head = struct.pack("<IIQQQIIIIQQ", MAGIC, VERSION, numel, nnz_w, nnz_o, bits, k, hb, 0, total, 0)
+    head += np.asarray(c_w, dtype="<f4").tobytes()
+    head += np.asarray(c_ea, dtype="<f4").tobytes()
+    head += np.asarray(c_eas, dtype="<f4").tobytes()
+    head += b"\0" * (hb - len(head))
+    out = (head + pack_bitmap(m_w) + pack_bitmap(m_o) + pack_codes(codes_w, bits)
+           + pack_codes(codes_ea, bits) + pack_codes(codes_eas, bits))
+    assert len(out) == total
+    return out
+
+
+def parse_record(blob: bytes) -> dict:
+    if len(blob) < HEADER_FIXED:
+        raise CorruptBlob("short header")
+    (magic, version, numel, nnz_w, nnz_o, bits, k, hb, z0, total, z1) = struct.unpack_from(
+        "<IIQQQIIIIQQ", blob, 0)
+    if magic != MAGIC or version != VERSION:
+        raise CorruptBlob("magic/version")
+    if bits not in (2, 4, 8) or k != (1 << bits) - 1 or hb != header_bytes(k):
+        raise CorruptBlob("bits/K/header size")
+    if nnz_o > nnz_w or nnz_w > numel:
+        raise CorruptBlob("counts")
+    if total != record_bytes(numel, nnz_w, nnz_o, bits) or len(blob) < total:
+        raise CorruptBlob("record size")
+    cents = np.frombuffer(blob, dtype="<f4", count=3 * k, offset=HEADER_FIXED).reshape(3, k)
+    off = hb
+    bb = bitmap_bytes(numel)
+    m_w = unpack_bitmap(blob[off:off + bb], numel); off += bb
+    m_o = unpack_bitmap(blob[off:off + bb], numel); off += bb
+    if np.count_nonzero(m_w) != nnz_w or np.count_nonzero(m_o) != nnz_o:
+        raise CorruptBlob("bitmap population")
+    if np.any(m_o & ~m_w):
+        raise CorruptBlob("moment kept where the weight is pruned")
+    cw = code_bytes(nnz_w, bits)
+    co = code_bytes(nnz_o, bits)
+    codes_w = unpack_codes(blob[off:off + cw], nnz_w, bits); off += cw
+    codes_ea = unpack_codes(blob[off:off + co], nnz_o, bits); off += co
+    codes_eas = unpack_codes(blob[off:off + co], nnz_o, bits); off += co
+    for c in (codes_w, codes_ea, codes_eas):
+        if c.size and (c.min() < 1 or c.max() > k):
+            raise CorruptBlob("code out of range")
+    return dict(numel=numel, nnz_w=nnz_w, nnz_o=nnz_o, bits=bits, k=k, record_bytes=total,
+                c_w=cents[0].copy(), c_ea=cents[1].copy(), c_eas=cents[2].copy(),
+                m_w=m_w, m_o=m_o, codes_w=codes_w, codes_ea=codes_ea, codes_eas=codes_eas)
+
+
+# --------------------------------------------------------------------------
+# Algorithm 1 (without the archiver) and Algorithm 2
+# --------------------------------------------------------------------------
+def compress_tensor(w_t, w_prev, ea, eas, p: Params, tensor_index: int = 0):
+    """Algorithm 1 for one tensor, up to (not including) the archiver.
+    Returns (record bytes, dict of every intermediate)."""
+    w_t = np.ascontiguousarray(w_t, dtype=np.float32).ravel()
+    w_prev = np.ascontiguousarray(w_prev, dtype=np.float32).ravel()
+    ea = np.ascontiguousarray(ea, dtype=np.float32).ravel()
+    eas = np.ascontiguousarray(eas, dtype=np.float32).ravel()
+    n = w_t.size
+    if not (w_prev.size == ea.size == eas.size == n):
+        raise ValueError("size mismatch")
+    if p.bits not in (2, 4, 8):
+        raise ValueError("bits")
+    validate_inputs(w_t, w_prev, ea, eas)
+    k = (1 << p.bits) - 1
+
+    dw = residual(w_t, w_prev)                                        # Algorithm 1, step 1
+    src = w_t if p.median_source == MEDIAN_ABS_WEIGHT else dw
+    med = lower_median_abs(src)
+    mean = exact_mean_abs(ea)
+    m_w, thr_w = weight_mask(dw, eas, p.alpha, med)                   # Eq. (rw)
+    m_o, thr_o = moment_mask(ea, m_w, p.beta, mean)                   # Eq. (ro)
+    s_w, s_ea, s_eas = dw[m_w], ea[m_o], eas[m_o]                     # joint_prune
+
+    cents, codes = [], []
+    for stream, s in enumerate((s_w, s_ea, s_eas)):                   # quantize(.)
+        c0 = kmeans_start(s, k, p.seed, tensor_index, stream)
+        c, idx = lloyd(s, c0, p.kmeans_iters)
+        cents.append(c)
+        codes.append((idx + 1).astype(np.uint8))
+    blob = encode_record(n, p.bits, m_w, m_o, cents[0], cents[1], cents[2], *codes)
+    info = dict(numel=n, dw=dw, median=med, mean_abs_ea=mean, thr_w=thr_w, thr_o=thr_o,
+                m_w=m_w, m_o=m_o, nnz_w=int(m_w.sum()), nnz_o=int(m_o.sum()),
+                s_w=s_w, s_ea=s_ea, s_eas=s_eas, c_w=cents[0], c_ea=cents[1], c_eas=cents[2],
+                codes_w=codes[0], codes_ea=codes[1], codes_eas=codes[2])
+    return blob, info
+
+
+def decompress_tensor(blob: bytes, w_prev):
+    """Algorithm 2: codes -> centres, W^_t = W^_(t-1) + dW^Q*; pruned entries
+    keep W^_(t-1) unchanged and decode to 0 in both moments."""
+    r = parse_record(blob)
+    w_prev = np.ascontiguousarray(w_prev, dtype=np.float32).ravel()
+    if w_prev.size != r["numel"]:
+        raise ValueError("size mismatch")
+    w_hat = w_prev.copy()
+    kept = r["m_w"]
+    w_hat[kept] = w_prev[kept] + r["c_w"][r["codes_w"].astype(np.int64) - 1]
+    ea_hat = np.zeros(r["numel"], dtype=np.float32)
+    eas_hat = np.zeros(r["numel"], dtype=np.float32)
+    ea_hat[r["m_o"]] = r["c_ea"][r["codes_ea"].astype(np.int64) - 1]
+    eas_hat[r["m_o"]] = r["c_eas"][r["codes_eas"].astype(np.int64) - 1]
+    return w_hat, ea_hat, eas_hat
+
+
+def compress_checkpoint(tensors, p: Params):
+    """Algorithm 1 over a tensor list: records back to back; tensor i starts at
+    offsets[i] and uses i as its index in the K-means start."""
+    blobs, infos, offsets = [], [], [0]
+    for i, (w_t, w_prev, ea, eas) in enumerate(tensors):
+        b, info = compress_tensor(w_t, w_prev, ea, eas, p, tensor_index=i)
+        blobs.append(b)
+        infos.append(info)
+        offsets.append(offsets[-1] + len(b))
+    return b"".join(blobs), offsets, infos
+
+
+def decompress_checkpoint(blob: bytes, offsets, w_prev_list):
+    return [decompress_tensor(blob[offsets[i]:offsets[i + 1]], w_prev_list[i])
+            for i in range(len(w_prev_list))]
+
+
+# --------------------------------------------------------------------------
+# Brute-force helpers used only by the pins
+# --------------------------------------------------------------------------
+def brute_mean_abs(x) -> Fraction:
+    return sum((Fraction(abs(float(v))) for v in x), Fraction(0)) / len(x)
+
+
+def brute_nearest(x: float, c) -> int:
+    """argmin_j |x - c_j| in exact rational arithmetic, lowest index on ties."""
+    best, bj = None, 0
+    for j, cj in enumerate(c):
+        d = abs(Fraction(float(x)) - Fraction(float(cj)))
+        if best is None or d < best:
+            best, bj = d, j
+    return bj
+
+
+def optimal_kmeans_1d_sse(values, k: int) -> Fraction:
+    """Smallest within-cluster sum of squares over all partitions of the sorted
+    values into at most k contiguous groups (dynamic programme, exact)."""
+    v = sorted(Fraction(float(x)) for x in values)
+    n = len(v)
+
+    def cost(i, j):  # group v[i:j]
+        seg = v[i:j]
+        mu = sum(seg) / len(seg)
+        return sum((t - mu) ** 2 for t in seg)
+
+    dp = [[None] * (n + 1) for _ in range(k + 1)]
+    dp[0][0] = Fraction(0)
+    for g in range(1, k + 1):
+        for j in range(1, n + 1):
+            best = dp[g - 1][j] if g > 1 else None  # fewer groups also allowed
+            for i in range(g - 1, j):
+                if dp[g - 1][i] is None:
+                    continue
+                cand = dp[g - 1][i] + cost(i, j)
+                if best is None or cand < best:
+                    best = cand
+            dp[g][j] = best
+    return dp[k][n]
