@@ -1,0 +1,175 @@
+/*
+ * excp.h -- C ABI of the ExCP checkpoint-compression hot path for NVIDIA B200 (sm_100a).
+ *
+ * What the library computes (arXiv 2406.11257, "ExCP: Extreme LLM Checkpoint
+ * Compression via Weight-Momentum Joint Shrinking"):
+ *
+ *   compress   Algorithm 1 without its archiver step, per tensor:
+ *                dW = W_t - W^_(t-1)                       (Section 3.1, Eq. ckpt_res)
+ *                M_w(i) = [ |dW(i)| * sqrt(eas(i)) > alpha * median ]      (Section 3.2, Eq. rw)
+ *                M_o(i) = [ |ea(i)| > beta * mean(|ea|) ] and M_w(i)       (Section 3.2, Eq. ro)
+ *                joint application of M_w to dW and of M_o to BOTH moments (Algorithm 1, joint_prune)
+ *                K-means of the survivors to 2^bits - 1 centres per stream, codes 1..K,
+ *                packed `bits` per code (Section 3.3; Section 4.1: bits = 4, two per byte)
+ *   decompress Algorithm 2 without its un-archiver step:
+ *                dW^ = C_w[I_w], O^ = C_o[I_o], W^_t = W^_(t-1) + dW^
+ *
+ * Letters: the paper writes v_t for Adam's FIRST moment and m_t for its SECOND.  This header
+ * says `ea` (first moment, exp_avg) and `eas` (second moment, exp_avg_sq).
+ *
+ * Where the paper is silent the library fixes one reading so that the output is unique:
+ *   - the median is the lower median (rank floor((n-1)/2)) of |W_t| (EXCP_MEDIAN_ABS_WEIGHT, the
+ *     letter of Eq. rw) or of |dW| (EXCP_MEDIAN_ABS_RESIDUAL), per tensor;
+ *   - mean(|ea|) is the exact mean rounded once to fp32;
+ *   - K-means is Lloyd's algorithm per tensor and per stream (dW, ea, eas): start = the K
+ *     equal-mass quantiles of a seeded index-stratified sample of <= 1024 survivors; assignment
+ *     = number of mid-points (c_j + c_j+1)/2, taken in fp64, lying strictly below x; update =
+ *     fixed-point mean (values scaled by 2^(30-E), E = exponent of the stream's largest
+ *     magnitude, rounded half-to-even, summed in int64); empty clusters keep their centre;
+ *     centres re-sorted; `kmeans_iters` iterations, then the final assignment.
+ *
+ * Record layout of one tensor (little endian, every section on a 16-byte boundary, padding zero):
+ *     0 u32 magic "EXCP"   4 u32 version = 1     8 u64 numel
+ *    16 u64 nnz_w         24 u64 nnz_o          32 u32 bits      36 u32 K = 2^bits - 1
+ *    40 u32 header bytes  44 u32 0              48 u64 record bytes   56 u64 0
+ *    64 f32 centres of dW [K], of ea [K], of eas [K]; header padded to 16 bytes
+ *    .. bitmap of M_w, bitmap of M_o: u32 words, bit k of word w = element 32 w + k
+ *    .. codes of dW [nnz_w], of ea [nnz_o], of eas [nnz_o]: survivors in index order, `bits`
+ *       each, value 1..K, survivor r at bit r * bits of the section (low bits first)
+ * A checkpoint blob is the tensors' records back to back.
+ *
+ * Conventions for every call:
+ *   - "device" pointers are CUDA device memory on the handle's device, 16-byte aligned;
+ *     "host" pointers are ordinary host memory.  The library never frees or reallocates a
+ *     caller's buffer and never writes an input.
+ *   - All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = the
+ *     legacy default stream).  Calls that return sizes or statistics to the host
+ *     synchronise that stream once, at their end.
+ *   - The handle owns the scratch workspace; it is not thread-safe: one call at a time.
+ *   - Errors are return codes; nothing is thrown and nothing aborts.  After a non-OK
+ *     return the output buffers hold unspecified bytes.
+ */
+#ifndef EXCP_H_
+#define EXCP_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct excp_handle_s* excp_handle;
+
+typedef enum {
+    EXCP_OK = 0,
+    EXCP_ERR_INVALID_ARG = -1,      /* null / misaligned pointer, bad parameter, workspace too small for a tensor */
+    EXCP_ERR_UNSUPPORTED = -2,      /* a code width the kernels do not implement */
+    EXCP_ERR_BUFFER_TOO_SMALL = -3, /* blob_capacity below what the records need */
+    EXCP_ERR_CUDA = -4,             /* a CUDA runtime call failed; see excp_last_cuda_error */
+    EXCP_ERR_CORRUPT_BLOB = -5,     /* decompress: header, sizes, bitmap population or a code is inconsistent */
+    EXCP_ERR_NONFINITE_INPUT = -6,  /* compress: NaN or infinity in an input, or a negative second moment */
+    EXCP_ERR_TIMEOUT = -7           /* reserved: no kernel of this library waits on another */
+} excp_status;
+
+typedef enum {
+    EXCP_MEDIAN_ABS_WEIGHT = 0,     /* median(|W_t|): Eq. (rw) as printed */
+    EXCP_MEDIAN_ABS_RESIDUAL = 1    /* median(|dW_t|): the quantity the mask prunes */
+} excp_median_source;
+
+/* Hyper-parameters.  Section 4.1: alpha = 5e-5, beta = 2.0, bits = 4. */
+typedef struct {
+    float alpha;                    /* Eq. (rw) */
+    float beta;                     /* Eq. (ro) */
+    int bits;                       /* code width n; K = 2^n - 1 centres.  4 is implemented. */
+    int kmeans_iters;               /* Lloyd iterations before the final assignment (>= 0) */
+    unsigned long long seed;        /* seed of the K-means start sample */
+    int median_source;              /* excp_median_source */
+    unsigned flags;                 /* must be 0 */
+} excp_params;
+
+/* Per-tensor result, written to host memory. */
+typedef struct {
+    unsigned long long numel;
+    unsigned long long nnz_w;       /* population of M_w */
+    unsigned long long nnz_o;       /* population of M_o */
+    unsigned long long blob_bytes;  /* size of this tensor's record */
+    float median;                   /* the median entering Eq. (rw) */
+    float mean_abs_ea;              /* the mean entering Eq. (ro) */
+    float thr_w;                    /* alpha * median */
+    float thr_o;                    /* beta * mean */
+} excp_tensor_stats;
+
+/* Creates a handle on CUDA device `device` with a scratch workspace for `workspace_numel`
+ * elements (about 12.3 bytes each; tensors are processed in groups whose sizes, each rounded
+ * up to 4096, sum to at most this), so the largest single tensor must not exceed it.
+ * Allocates device and pinned host memory.  Returns EXCP_ERR_CUDA if the device or the
+ * memory cannot be had. */
+excp_status excp_create(excp_handle* out, int device, size_t workspace_numel);
+
+/* Frees everything the handle owns.  NULL is accepted. */
+excp_status excp_destroy(excp_handle h);
+
+/* Size in bytes of a record with the given counts (the layout above).  0 if bits is not 2, 4 or 8. */
+size_t excp_record_bytes(size_t numel, size_t nnz_w, size_t nnz_o, int bits);
+
+/* Worst-case record size for a tensor of `numel` elements (every element kept). */
+size_t excp_compress_bound(size_t numel, int bits);
+
+/* Static, NUL-terminated description of a status code. */
+const char* excp_status_string(excp_status s);
+
+/* The cudaError_t (as int) of the last failed CUDA call on this handle, 0 if none. */
+excp_status excp_last_cuda_error(excp_handle h, int* cuda_err);
+
+/* Algorithm 1 (up to the archiver) for one tensor.
+ *   w_t, w_prev, ea, eas  device, fp32[numel], read only.  w_prev is the LAST RECONSTRUCTED
+ *                         weight tensor W^_(t-1) (Section 3.4).
+ *   blob_out              device, blob_capacity bytes; receives the record.
+ *   blob_bytes_out        host; receives the record size.
+ *   stats_out             host, may be NULL.
+ * numel = 0 is legal and gives a header-only record.  The tensor counts as index 0 of a
+ * checkpoint for the K-means start.  Synchronises the stream. */
+excp_status excp_compress_tensor(excp_handle h, const excp_params* params,
+                                 const float* w_t, const float* w_prev, const float* ea, const float* eas,
+                                 size_t numel, void* blob_out, size_t blob_capacity,
+                                 size_t* blob_bytes_out, excp_tensor_stats* stats_out, void* cuda_stream);
+
+/* Algorithm 1 over a tensor list; tensor i uses i as its index in the K-means start.
+ *   w_t, w_prev, ea, eas  host arrays [num_tensors] of device pointers (fp32[numel[i]]).
+ *   numel                 host [num_tensors].
+ *   blob_out              device, blob_capacity bytes; records back to back.
+ *   tensor_offsets_out    host [num_tensors + 1]; record i is [offsets[i], offsets[i+1]).
+ *   stats_out             host [num_tensors], may be NULL.
+ * All tensors of a group run through each kernel together, so the number of launches does
+ * not grow with the tensor count.  Synchronises the stream. */
+excp_status excp_compress_checkpoint(excp_handle h, const excp_params* params, size_t num_tensors,
+                                     const float* const* w_t, const float* const* w_prev,
+                                     const float* const* ea, const float* const* eas,
+                                     const size_t* numel, void* blob_out, size_t blob_capacity,
+                                     size_t* tensor_offsets_out, excp_tensor_stats* stats_out,
+                                     void* cuda_stream);
+
+/* Algorithm 2 (after the un-archiver) for one tensor.
+ *   blob                  device, blob_bytes bytes, one record.
+ *   w_prev                device fp32[numel]: W^_(t-1).
+ *   w_out, ea_out, eas_out device fp32[numel].  w_out may be the same buffer as w_prev
+ *                         (in-place update); no other overlap is allowed.
+ * Pruned weights keep w_prev bit for bit; pruned moments decode to 0.
+ * Synchronises the stream; returns EXCP_ERR_CORRUPT_BLOB if the record is inconsistent
+ * (every read stays inside [blob, blob + blob_bytes) even then). */
+excp_status excp_decompress_tensor(excp_handle h, const void* blob, size_t blob_bytes,
+                                   const float* w_prev, size_t numel,
+                                   float* w_out, float* ea_out, float* eas_out, void* cuda_stream);
+
+/* Algorithm 2 over a tensor list (the loop body of Algorithm 3).
+ *   blob                  device; tensor_offsets host [num_tensors + 1] as returned by compress.
+ *   w_prev, w_out, ea_out, eas_out  host arrays [num_tensors] of device pointers. */
+excp_status excp_decompress_checkpoint(excp_handle h, const void* blob, const size_t* tensor_offsets,
+                                       size_t num_tensors, const float* const* w_prev, const size_t* numel,
+                                       float* const* w_out, float* const* ea_out, float* const* eas_out,
+                                       void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EXCP_H_ */

@@ -1,0 +1,187 @@
+"""ctypes binding of libexcp.so (include/excp.h).  Argument marshalling only:
+every step of compression and decompression runs in the library's CUDA kernels.
+PyTorch supplies device memory and the stream.  There is no CPU fallback: if
+the library cannot be loaded the import of this module's handle fails loudly."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+from . import build as _build
+
+MEDIAN_ABS_WEIGHT = 0
+MEDIAN_ABS_RESIDUAL = 1
+
+STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED", -3: "BUFFER_TOO_SMALL", -4: "CUDA",
+          -5: "CORRUPT_BLOB", -6: "NONFINITE_INPUT", -7: "TIMEOUT"}
+
+EXPORTS = ["excp_create", "excp_destroy", "excp_record_bytes", "excp_compress_bound",
+           "excp_status_string", "excp_last_cuda_error", "excp_compress_tensor",
+           "excp_compress_checkpoint", "excp_decompress_tensor", "excp_decompress_checkpoint"]
+
+
+class ExcpError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        super().__init__(f"{what}: EXCP_ERR_{STATUS.get(status, status)}")
+        self.status = status
+
+
+class CParams(C.Structure):
+    _fields_ = [("alpha", C.c_float), ("beta", C.c_float), ("bits", C.c_int), ("kmeans_iters", C.c_int),
+                ("seed", C.c_ulonglong), ("median_source", C.c_int), ("flags", C.c_uint)]
+
+
+class CStats(C.Structure):
+    _fields_ = [("numel", C.c_ulonglong), ("nnz_w", C.c_ulonglong), ("nnz_o", C.c_ulonglong),
+                ("blob_bytes", C.c_ulonglong), ("median", C.c_float), ("mean_abs_ea", C.c_float),
+                ("thr_w", C.c_float), ("thr_o", C.c_float)]
+
+
+@dataclass
+class Params:
+    alpha: float = 5e-5
+    beta: float = 2.0
+    bits: int = 4
+    kmeans_iters: int = 10
+    seed: int = 0
+    median_source: int = MEDIAN_ABS_WEIGHT
+
+    def to_c(self) -> CParams:
+        return CParams(self.alpha, self.beta, self.bits, self.kmeans_iters, self.seed, self.median_source, 0)
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """Loads (building first if the sources are newer) libexcp.so and declares the prototypes."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.build()
+    lib = C.CDLL(path)
+    vp, sz = C.c_void_p, C.c_size_t
+    lib.excp_create.argtypes = [C.POINTER(vp), C.c_int, sz]
+    lib.excp_destroy.argtypes = [vp]
+    lib.excp_record_bytes.argtypes = [sz, sz, sz, C.c_int]
+    lib.excp_record_bytes.restype = sz
+    lib.excp_compress_bound.argtypes = [sz, C.c_int]
+    lib.excp_compress_bound.restype = sz
+    lib.excp_status_string.argtypes = [C.c_int]
+    lib.excp_status_string.restype = C.c_char_p
+    lib.excp_last_cuda_error.argtypes = [vp, C.POINTER(C.c_int)]
+    lib.excp_compress_tensor.argtypes = [vp, C.POINTER(CParams), vp, vp, vp, vp, sz, vp, sz,
+                                         C.POINTER(sz), C.POINTER(CStats), vp]
+    lib.excp_compress_checkpoint.argtypes = [vp, C.POINTER(CParams), sz, C.POINTER(vp), C.POINTER(vp),
+                                             C.POINTER(vp), C.POINTER(vp), C.POINTER(sz), vp, sz,
+                                             C.POINTER(sz), C.POINTER(CStats), vp]
+    lib.excp_decompress_tensor.argtypes = [vp, vp, sz, vp, sz, vp, vp, vp, vp]
+    lib.excp_decompress_checkpoint.argtypes = [vp, vp, C.POINTER(sz), sz, C.POINTER(vp), C.POINTER(sz),
+                                               C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), vp]
+    for name in EXPORTS:
+        if getattr(lib, name).restype is C.c_int:
+            getattr(lib, name).restype = C.c_int
+    _lib = lib
+    return lib
+
+
+def _ptr(t: torch.Tensor | None) -> int:
+    return 0 if t is None or t.numel() == 0 else t.data_ptr()
+
+
+def _check_f32_cuda(*ts: torch.Tensor) -> None:
+    for t in ts:
+        if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+            raise TypeError("expected contiguous float32 CUDA tensors")
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def record_bytes(numel: int, nnz_w: int, nnz_o: int, bits: int = 4) -> int:
+    return load_library().excp_record_bytes(numel, nnz_w, nnz_o, bits)
+
+
+def compress_bound(numel: int, bits: int = 4) -> int:
+    return load_library().excp_compress_bound(numel, bits)
+
+
+class Handle:
+    """Owns the library's scratch workspace on one device (excp_create / excp_destroy)."""
+
+    def __init__(self, workspace_numel: int, device: int | None = None):
+        self.lib = load_library()
+        self.device = torch.cuda.current_device() if device is None else device
+        self._h = C.c_void_p()
+        st = self.lib.excp_create(C.byref(self._h), self.device, workspace_numel)
+        if st != 0:
+            raise ExcpError(st, "excp_create")
+
+    def close(self) -> None:
+        if self._h:
+            self.lib.excp_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def last_cuda_error(self) -> int:
+        e = C.c_int(0)
+        self.lib.excp_last_cuda_error(self._h, C.byref(e))
+        return e.value
+
+    # ---- Algorithm 1 -----------------------------------------------------
+    def compress_tensor(self, p: Params, w_t, w_prev, ea, eas, blob_out: torch.Tensor):
+        """excp_compress_tensor.  Returns (record bytes, stats)."""
+        _check_f32_cuda(w_t, w_prev, ea, eas)
+        cp, nbytes, stats = p.to_c(), C.c_size_t(0), CStats()
+        st = self.lib.excp_compress_tensor(self._h, C.byref(cp), _ptr(w_t), _ptr(w_prev), _ptr(ea), _ptr(eas),
+                                           w_t.numel(), blob_out.data_ptr(), blob_out.numel() * blob_out.element_size(),
+                                           C.byref(nbytes), C.byref(stats), _stream())
+        if st != 0:
+            raise ExcpError(st, "excp_compress_tensor")
+        return nbytes.value, stats
+
+    def compress_checkpoint(self, p: Params, tensors, blob_out: torch.Tensor, want_stats: bool = True):
+        """excp_compress_checkpoint over a list of (w_t, w_prev, ea, eas).
+        Returns (offsets list of len n+1, list of stats or None)."""
+        n = len(tensors)
+        for q in tensors:
+            _check_f32_cuda(*q)
+        arr = lambda k: (C.c_void_p * n)(*[_ptr(q[k]) for q in tensors])
+        numel = (C.c_size_t * n)(*[q[0].numel() for q in tensors])
+        offs = (C.c_size_t * (n + 1))()
+        stats = (CStats * n)() if want_stats else None
+        cp = p.to_c()
+        st = self.lib.excp_compress_checkpoint(self._h, C.byref(cp), n, arr(0), arr(1), arr(2), arr(3), numel,
+                                               blob_out.data_ptr(), blob_out.numel() * blob_out.element_size(),
+                                               offs, stats, _stream())
+        if st != 0:
+            raise ExcpError(st, "excp_compress_checkpoint")
+        return list(offs), (list(stats) if want_stats else None)
+
+    # ---- Algorithm 2 -----------------------------------------------------
+    def decompress_tensor(self, blob: torch.Tensor, blob_bytes: int, w_prev, w_out, ea_out, eas_out) -> None:
+        _check_f32_cuda(w_prev, w_out, ea_out, eas_out)
+        st = self.lib.excp_decompress_tensor(self._h, blob.data_ptr(), blob_bytes, _ptr(w_prev), w_prev.numel(),
+                                             _ptr(w_out), _ptr(ea_out), _ptr(eas_out), _stream())
+        if st != 0:
+            raise ExcpError(st, "excp_decompress_tensor")
+
+    def decompress_checkpoint(self, blob: torch.Tensor, offsets, w_prev, w_out, ea_out, eas_out) -> None:
+        n = len(w_prev)
+        _check_f32_cuda(*w_prev, *w_out, *ea_out, *eas_out)
+        arr = lambda ts: (C.c_void_p * n)(*[_ptr(t) for t in ts])
+        numel = (C.c_size_t * n)(*[t.numel() for t in w_prev])
+        offs = (C.c_size_t * (n + 1))(*offsets)
+        st = self.lib.excp_decompress_checkpoint(self._h, blob.data_ptr(), offs, n, arr(w_prev), numel,
+                                                 arr(w_out), arr(ea_out), arr(eas_out), _stream())
+        if st != 0:
+            raise ExcpError(st, "excp_decompress_checkpoint")

@@ -1,0 +1,344 @@
+// The C ABI of include/excp.h: handle, argument checks, grouping of the tensor
+// list, and the order of the kernel launches.  No arithmetic of the method
+// lives here.
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/excp.h"
+#include "excp_common.cuh"
+
+using namespace excp;
+
+struct excp_handle_s {
+    int device = 0;
+    int sms = 0;
+    size_t cap_tiles = 0;
+    Workspace ws{};
+    TensorState* d_state = nullptr;      // MAX_GROUP_TENSORS
+    DecState* d_dstate = nullptr;        // MAX_GROUP_TENSORS
+    CallState* d_call = nullptr;
+    void* d_desc = nullptr;              // TensorDesc[] or DecDesc[] of the whole call
+    TensorResult* d_results = nullptr;
+    void* h_desc = nullptr;              // pinned
+    TensorResult* h_results = nullptr;   // pinned
+    CallState* h_call = nullptr;         // pinned
+    size_t tensor_cap = 0;               // entries the per-call arrays hold
+    int last_cuda_error = 0;
+};
+
+namespace {
+
+constexpr size_t DESC_BYTES = sizeof(TensorDesc) > sizeof(DecDesc) ? sizeof(TensorDesc) : sizeof(DecDesc);
+constexpr unsigned long long MAX_NUMEL = 1ull << 31;
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+        if (prev != dev) ok = cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() {
+        int now = -1;
+        if (prev >= 0 && cudaGetDevice(&now) == cudaSuccess && now != prev) cudaSetDevice(prev);
+    }
+};
+
+bool check(excp_handle h, cudaError_t e) {
+    if (e == cudaSuccess) return true;
+    h->last_cuda_error = (int)e;
+    return false;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+void free_call_arrays(excp_handle h) {
+    if (h->d_desc) cudaFree(h->d_desc);
+    if (h->d_results) cudaFree(h->d_results);
+    if (h->h_desc) cudaFreeHost(h->h_desc);
+    if (h->h_results) cudaFreeHost(h->h_results);
+    h->d_desc = nullptr; h->d_results = nullptr; h->h_desc = nullptr; h->h_results = nullptr;
+    h->tensor_cap = 0;
+}
+
+bool ensure_call_arrays(excp_handle h, size_t n) {
+    if (n <= h->tensor_cap) return true;
+    free_call_arrays(h);
+    size_t cap = 4096;
+    while (cap < n) cap *= 2;
+    if (!check(h, cudaMalloc(&h->d_desc, cap * DESC_BYTES))) return false;
+    if (!check(h, cudaMalloc(reinterpret_cast<void**>(&h->d_results), cap * sizeof(TensorResult)))) return false;
+    if (!check(h, cudaMallocHost(&h->h_desc, cap * DESC_BYTES))) return false;
+    if (!check(h, cudaMallocHost(reinterpret_cast<void**>(&h->h_results), cap * sizeof(TensorResult)))) return false;
+    h->tensor_cap = cap;
+    return true;
+}
+
+struct Group { size_t first, count; u32 tiles; };
+
+// Consecutive tensors whose tiles fit the workspace (and the per-group state).
+bool make_groups(excp_handle h, const size_t* numel, size_t n, std::vector<Group>& out) {
+    Group g{0, 0, 0};
+    for (size_t i = 0; i < n; ++i) {
+        if (numel[i] > MAX_NUMEL) return false;
+        const size_t t = (numel[i] + TILE - 1) / TILE;
+        if (t > h->cap_tiles) return false;
+        if (g.count && (g.tiles + t > h->cap_tiles || g.count >= (size_t)MAX_GROUP_TENSORS)) {
+            out.push_back(g);
+            g = Group{i, 0, 0};
+        }
+        g.tiles += (u32)t;
+        ++g.count;
+    }
+    if (g.count) out.push_back(g);
+    return true;
+}
+
+excp_status status_from_flags(u32 flags) {
+    if (flags & FLAG_INTERNAL) return EXCP_ERR_CUDA;
+    if (flags & FLAG_NONFINITE) return EXCP_ERR_NONFINITE_INPUT;
+    if (flags & FLAG_CORRUPT) return EXCP_ERR_CORRUPT_BLOB;
+    if (flags & FLAG_BLOB_FULL) return EXCP_ERR_BUFFER_TOO_SMALL;
+    return EXCP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+excp_status excp_create(excp_handle* out, int device, size_t workspace_numel) {
+    if (!out) return EXCP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (workspace_numel == 0 || workspace_numel > (1ull << 40)) return EXCP_ERR_INVALID_ARG;
+    excp_handle h = new (std::nothrow) excp_handle_s();
+    if (!h) return EXCP_ERR_CUDA;
+    h->device = device;
+    DeviceGuard guard(device);
+    cudaDeviceProp prop;
+    bool ok = guard.ok && check(h, cudaGetDeviceProperties(&prop, device));
+    if (ok) {
+        h->sms = prop.multiProcessorCount;
+        h->cap_tiles = (workspace_numel + TILE - 1) / TILE;
+        const size_t elems = h->cap_tiles * (size_t)TILE;
+        for (int k = 0; k < 3 && ok; ++k)
+            ok = check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.surv[k]), elems * sizeof(float)));
+        ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.bm_w), elems / 8));
+        ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.bm_o), elems / 8));
+        ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.tile_cnt_w), h->cap_tiles * 4));
+        ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.tile_cnt_o), h->cap_tiles * 4));
+        ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.tile_off_w), h->cap_tiles * 4));
+        ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.tile_off_o), h->cap_tiles * 4));
+        ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->d_state), MAX_GROUP_TENSORS * sizeof(TensorState)));
+        ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->d_dstate), MAX_GROUP_TENSORS * sizeof(DecState)));
+        ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->d_call), sizeof(CallState)));
+        ok = ok && check(h, cudaMallocHost(reinterpret_cast<void**>(&h->h_call), sizeof(CallState)));
+        ok = ok && ensure_call_arrays(h, 1);
+    }
+    if (!ok) {
+        excp_destroy(h);
+        return EXCP_ERR_CUDA;
+    }
+    *out = h;
+    return EXCP_OK;
+}
+
+excp_status excp_destroy(excp_handle h) {
+    if (!h) return EXCP_OK;
+    DeviceGuard guard(h->device);
+    for (int k = 0; k < 3; ++k) if (h->ws.surv[k]) cudaFree(h->ws.surv[k]);
+    if (h->ws.bm_w) cudaFree(h->ws.bm_w);
+    if (h->ws.bm_o) cudaFree(h->ws.bm_o);
+    if (h->ws.tile_cnt_w) cudaFree(h->ws.tile_cnt_w);
+    if (h->ws.tile_cnt_o) cudaFree(h->ws.tile_cnt_o);
+    if (h->ws.tile_off_w) cudaFree(h->ws.tile_off_w);
+    if (h->ws.tile_off_o) cudaFree(h->ws.tile_off_o);
+    if (h->d_state) cudaFree(h->d_state);
+    if (h->d_dstate) cudaFree(h->d_dstate);
+    if (h->d_call) cudaFree(h->d_call);
+    if (h->h_call) cudaFreeHost(h->h_call);
+    free_call_arrays(h);
+    delete h;
+    return EXCP_OK;
+}
+
+size_t excp_record_bytes(size_t numel, size_t nnz_w, size_t nnz_o, int bits) {
+    if (bits != 2 && bits != 4 && bits != 8) return 0;
+    return (size_t)record_bytes(numel, nnz_w, nnz_o, bits);
+}
+
+size_t excp_compress_bound(size_t numel, int bits) { return excp_record_bytes(numel, numel, numel, bits); }
+
+const char* excp_status_string(excp_status s) {
+    switch (s) {
+        case EXCP_OK: return "ok";
+        case EXCP_ERR_INVALID_ARG: return "invalid argument";
+        case EXCP_ERR_UNSUPPORTED: return "unsupported code width";
+        case EXCP_ERR_BUFFER_TOO_SMALL: return "output buffer too small";
+        case EXCP_ERR_CUDA: return "CUDA error";
+        case EXCP_ERR_CORRUPT_BLOB: return "corrupt record";
+        case EXCP_ERR_NONFINITE_INPUT: return "non-finite input or negative second moment";
+        case EXCP_ERR_TIMEOUT: return "timeout";
+    }
+    return "unknown status";
+}
+
+excp_status excp_last_cuda_error(excp_handle h, int* cuda_err) {
+    if (!h || !cuda_err) return EXCP_ERR_INVALID_ARG;
+    *cuda_err = h->last_cuda_error;
+    return EXCP_OK;
+}
+
+excp_status excp_compress_checkpoint(excp_handle h, const excp_params* params, size_t num_tensors,
+                                     const float* const* w_t, const float* const* w_prev,
+                                     const float* const* ea, const float* const* eas,
+                                     const size_t* numel, void* blob_out, size_t blob_capacity,
+                                     size_t* tensor_offsets_out, excp_tensor_stats* stats_out,
+                                     void* cuda_stream) {
+    if (!h || !params || !tensor_offsets_out) return EXCP_ERR_INVALID_ARG;
+    if (num_tensors && (!w_t || !w_prev || !ea || !eas || !numel)) return EXCP_ERR_INVALID_ARG;
+    if (!blob_out || !aligned16(blob_out)) return EXCP_ERR_INVALID_ARG;
+    if (params->bits == 2 || params->bits == 8) return EXCP_ERR_UNSUPPORTED;
+    if (params->bits != 4 || params->kmeans_iters < 0 || params->flags != 0 ||
+        (params->median_source != 0 && params->median_source != 1) ||
+        !(params->alpha >= 0.f) || !(params->beta >= 0.f) || std::isinf(params->alpha) ||
+        std::isinf(params->beta))
+        return EXCP_ERR_INVALID_ARG;
+    for (size_t i = 0; i < num_tensors; ++i) {
+        if (numel[i] == 0) continue;
+        if (!w_t[i] || !w_prev[i] || !ea[i] || !eas[i]) return EXCP_ERR_INVALID_ARG;
+        if (!aligned16(w_t[i]) || !aligned16(w_prev[i]) || !aligned16(ea[i]) || !aligned16(eas[i]))
+            return EXCP_ERR_INVALID_ARG;
+    }
+    tensor_offsets_out[0] = 0;
+    if (num_tensors == 0) return EXCP_OK;
+
+    std::vector<Group> groups;
+    if (!make_groups(h, numel, num_tensors, groups)) return EXCP_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return EXCP_ERR_CUDA;
+    if (!ensure_call_arrays(h, num_tensors)) return EXCP_ERR_CUDA;
+
+    TensorDesc* hd = static_cast<TensorDesc*>(h->h_desc);
+    for (const Group& g : groups) {
+        u32 tile = 0;
+        for (size_t i = g.first; i < g.first + g.count; ++i) {
+            TensorDesc& d = hd[i];
+            d.w_t = w_t[i]; d.w_prev = w_prev[i]; d.ea = ea[i]; d.eas = eas[i];
+            d.numel = numel[i];
+            d.tensor_index = i;
+            d.tile_begin = tile;
+            d.num_tiles = (u32)((numel[i] + TILE - 1) / TILE);
+            tile += d.num_tiles;
+        }
+    }
+    Params p;
+    p.alpha = params->alpha; p.beta = params->beta; p.bits = params->bits;
+    p.kmeans_iters = params->kmeans_iters; p.seed = params->seed; p.median_source = params->median_source;
+
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    LaunchCfg cfg{h->sms, stream};
+    TensorDesc* dd = static_cast<TensorDesc*>(h->d_desc);
+    bool ok = check(h, cudaMemsetAsync(h->d_call, 0, sizeof(CallState), stream));
+    ok = ok && check(h, cudaMemcpyAsync(dd, hd, num_tensors * sizeof(TensorDesc), cudaMemcpyHostToDevice, stream));
+    for (size_t gi = 0; ok && gi < groups.size(); ++gi) {
+        const Group& g = groups[gi];
+        const int nt = (int)g.count;
+        ok = check(h, cudaMemsetAsync(h->d_state, 0, nt * sizeof(TensorState), stream));
+        if (!ok) break;
+        launch_stats(cfg, dd + g.first, h->d_state, nt, g.tiles, h->ws, p);
+        launch_mask_compact(cfg, dd + g.first, h->d_state, nt, g.tiles, h->ws, p, h->d_call, blob_capacity);
+        launch_kmeans(cfg, dd + g.first, h->d_state, nt, g.tiles, h->ws, p);
+        launch_pack(cfg, dd + g.first, h->d_state, nt, g.tiles, h->ws, p,
+                    static_cast<unsigned char*>(blob_out), h->d_call, h->d_results + g.first);
+        ok = check(h, cudaGetLastError());
+    }
+    ok = ok && check(h, cudaMemcpyAsync(h->h_results, h->d_results, num_tensors * sizeof(TensorResult),
+                                        cudaMemcpyDeviceToHost, stream));
+    ok = ok && check(h, cudaMemcpyAsync(h->h_call, h->d_call, sizeof(CallState), cudaMemcpyDeviceToHost, stream));
+    if (!check(h, cudaStreamSynchronize(stream)) || !ok) return EXCP_ERR_CUDA;
+
+    for (size_t i = 0; i < num_tensors; ++i) {
+        const TensorResult& r = h->h_results[i];
+        tensor_offsets_out[i] = (size_t)r.blob_off;
+        tensor_offsets_out[i + 1] = (size_t)(r.blob_off + r.blob_bytes);
+        if (stats_out) {
+            excp_tensor_stats& s = stats_out[i];
+            s.numel = numel[i]; s.nnz_w = r.nnz_w; s.nnz_o = r.nnz_o; s.blob_bytes = r.blob_bytes;
+            s.median = r.median; s.mean_abs_ea = r.mean_abs_ea; s.thr_w = r.thr_w; s.thr_o = r.thr_o;
+        }
+    }
+    return status_from_flags(h->h_call->flags);
+}
+
+excp_status excp_compress_tensor(excp_handle h, const excp_params* params,
+                                 const float* w_t, const float* w_prev, const float* ea, const float* eas,
+                                 size_t numel, void* blob_out, size_t blob_capacity,
+                                 size_t* blob_bytes_out, excp_tensor_stats* stats_out, void* cuda_stream) {
+    if (!blob_bytes_out) return EXCP_ERR_INVALID_ARG;
+    size_t offs[2] = {0, 0};
+    const excp_status s = excp_compress_checkpoint(h, params, 1, &w_t, &w_prev, &ea, &eas, &numel, blob_out,
+                                                   blob_capacity, offs, stats_out, cuda_stream);
+    *blob_bytes_out = offs[1] - offs[0];
+    return s;
+}
+
+excp_status excp_decompress_checkpoint(excp_handle h, const void* blob, const size_t* tensor_offsets,
+                                       size_t num_tensors, const float* const* w_prev, const size_t* numel,
+                                       float* const* w_out, float* const* ea_out, float* const* eas_out,
+                                       void* cuda_stream) {
+    if (!h || !blob || !tensor_offsets || !aligned16(blob)) return EXCP_ERR_INVALID_ARG;
+    if (num_tensors == 0) return EXCP_OK;
+    if (!w_prev || !numel || !w_out || !ea_out || !eas_out) return EXCP_ERR_INVALID_ARG;
+    for (size_t i = 0; i < num_tensors; ++i) {
+        if (tensor_offsets[i + 1] < tensor_offsets[i] || (tensor_offsets[i] & 15u)) return EXCP_ERR_INVALID_ARG;
+        if (numel[i] == 0) continue;
+        if (!w_prev[i] || !w_out[i] || !ea_out[i] || !eas_out[i]) return EXCP_ERR_INVALID_ARG;
+        if (!aligned16(w_prev[i]) || !aligned16(w_out[i]) || !aligned16(ea_out[i]) || !aligned16(eas_out[i]))
+            return EXCP_ERR_INVALID_ARG;
+    }
+    std::vector<Group> groups;
+    if (!make_groups(h, numel, num_tensors, groups)) return EXCP_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return EXCP_ERR_CUDA;
+    if (!ensure_call_arrays(h, num_tensors)) return EXCP_ERR_CUDA;
+
+    DecDesc* hd = static_cast<DecDesc*>(h->h_desc);
+    const unsigned char* base = static_cast<const unsigned char*>(blob);
+    for (const Group& g : groups) {
+        u32 tile = 0;
+        for (size_t i = g.first; i < g.first + g.count; ++i) {
+            DecDesc& d = hd[i];
+            d.rec = base + tensor_offsets[i];
+            d.rec_avail = tensor_offsets[i + 1] - tensor_offsets[i];
+            d.w_prev = w_prev[i]; d.w_out = w_out[i]; d.ea_out = ea_out[i]; d.eas_out = eas_out[i];
+            d.numel = numel[i];
+            d.tile_begin = tile;
+            d.num_tiles = (u32)((numel[i] + TILE - 1) / TILE);
+            tile += d.num_tiles;
+        }
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    LaunchCfg cfg{h->sms, stream};
+    DecDesc* dd = static_cast<DecDesc*>(h->d_desc);
+    bool ok = check(h, cudaMemsetAsync(h->d_call, 0, sizeof(CallState), stream));
+    ok = ok && check(h, cudaMemcpyAsync(dd, hd, num_tensors * sizeof(DecDesc), cudaMemcpyHostToDevice, stream));
+    for (size_t gi = 0; ok && gi < groups.size(); ++gi) {
+        const Group& g = groups[gi];
+        launch_decode(cfg, dd + g.first, h->d_dstate, (int)g.count, g.tiles, h->ws, h->d_call);
+        ok = check(h, cudaGetLastError());
+    }
+    ok = ok && check(h, cudaMemcpyAsync(h->h_call, h->d_call, sizeof(CallState), cudaMemcpyDeviceToHost, stream));
+    if (!check(h, cudaStreamSynchronize(stream)) || !ok) return EXCP_ERR_CUDA;
+    return status_from_flags(h->h_call->flags);
+}
+
+excp_status excp_decompress_tensor(excp_handle h, const void* blob, size_t blob_bytes,
+                                   const float* w_prev, size_t numel,
+                                   float* w_out, float* ea_out, float* eas_out, void* cuda_stream) {
+    const size_t offs[2] = {0, blob_bytes};
+    return excp_decompress_checkpoint(h, blob, offs, 1, &w_prev, &numel, &w_out, &ea_out, &eas_out, cuda_stream);
+}
+
+}  // extern "C"

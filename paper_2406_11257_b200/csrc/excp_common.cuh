@@ -1,0 +1,241 @@
+// Shared declarations of the ExCP kernels: tile geometry, per-tensor device
+// records, small device helpers, and the launch wrappers each .cu file exports.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace excp {
+
+typedef unsigned long long u64;
+typedef long long s64;
+typedef unsigned int u32;
+
+// A tile is the unit of work of every sweep: 4096 consecutive elements of one
+// tensor = 256 threads x 4 rounds x one float4.  Tiles never span tensors, so a
+// tile's 128 bitmap words and its survivor segment belong to exactly one tensor.
+constexpr int TILE = 4096;
+constexpr int TPB = 256;
+constexpr int TILE_WORDS = TILE / 32;
+constexpr int ROUNDS = TILE / (TPB * 4);         // 4
+constexpr int CHUNKS = ROUNDS * (TPB / 32);      // 32 warp-chunks of 128 elements per tile
+
+constexpr int HIST1_BITS = 13;                   // first radix-select level: top 13 of 31 key bits
+constexpr int HIST1_BINS = 1 << HIST1_BITS;
+constexpr int HIST1_SHIFT = 31 - HIST1_BITS;     // 18 bits left for the in-bin select
+constexpr int KMAX = 15;                         // centres at 4 bits
+constexpr int KPAD = 16;
+constexpr int SAMPLE_MAX = 1024;                 // K-means start sample
+constexpr int MAX_GROUP_TENSORS = 1024;
+
+constexpr u32 FLAG_NONFINITE = 1u;               // NaN/Inf input or negative second moment
+constexpr u32 FLAG_BLOB_FULL = 2u;               // records do not fit blob_capacity
+constexpr u32 FLAG_CORRUPT = 4u;                 // decompress: inconsistent record
+constexpr u32 FLAG_INTERNAL = 8u;                // a self-check failed (candidate count mismatch)
+
+constexpr u32 MAGIC = 0x50435845u;
+constexpr u32 VERSION = 1u;
+constexpr int HEADER_FIXED = 64;
+
+struct TensorDesc {              // built on the host, one per tensor of a group
+    const float* w_t;
+    const float* w_prev;
+    const float* ea;
+    const float* eas;
+    u64 numel;
+    u64 tensor_index;            // position in the checkpoint (enters the start sample)
+    u32 tile_begin;              // first tile of this tensor within the group
+    u32 num_tiles;
+};
+
+struct StreamState {             // K-means state of one stream (0 = dW, 1 = ea, 2 = eas)
+    float cent[KPAD];            // centres, ascending; [15] unused
+    float thr[KPAD];             // thr[j] = largest fp32 <= (c_j + c_j+1)/2; +inf from K-1 on
+    s64 acc_sum[KPAD];           // fixed-point sums of the current pass
+    u64 acc_cnt[KPAD];
+    u32 maxkey;                  // max |x| bit pattern over the survivors
+    int e;                       // fixed-point exponent E
+    float scale1, scale2;        // 2^(30-E) split in two exact factors
+};
+
+struct TensorState {             // device scratch, zeroed per group
+    u32 hist1[HIST1_BINS];
+    u64 sum_lo[256];             // exact sum of |ea|: low/high halves of warp partial sums,
+    u64 sum_hi[256];             //   indexed by the partial sum's exponent
+    u64 sum_low[256];            // mantissa sums of the rare elements far below a warp's maximum
+    u32 bin1;
+    u32 rank_in_bin;
+    u32 bin_count;
+    u32 cand_count;
+    u32 flags;
+    u32 median_bits;
+    float mean_abs_ea;
+    float thr_w, thr_o;
+    u32 nnz_w, nnz_o;
+    u32 pad_;
+    u64 blob_off;                // start of this tensor's record in the blob
+    u64 blob_bytes;
+    StreamState s[3];
+};
+
+struct TensorResult {            // copied back to the host at the end of a call
+    u64 nnz_w, nnz_o, blob_off, blob_bytes;
+    float median, mean_abs_ea, thr_w, thr_o;
+};
+
+struct CallState {               // one per handle, device resident
+    u64 blob_cursor;             // running end of the records written so far
+    u32 flags;                   // OR of every tensor's flags
+    u32 pad_;
+};
+
+struct Workspace {               // device arrays sized for cap_tiles tiles
+    float* surv[3];              // survivors, each tile's compacted at the tile's own start
+    u32* bm_w;                   // bitmaps, TILE_WORDS words per tile
+    u32* bm_o;
+    u32* tile_cnt_w;             // survivors per tile
+    u32* tile_cnt_o;
+    u32* tile_off_w;             // exclusive prefix of the counts within the tensor
+    u32* tile_off_o;
+};
+
+struct Params {
+    float alpha, beta;
+    int bits, kmeans_iters;
+    u64 seed;
+    int median_source;
+};
+
+struct DecDesc {                 // decompress: one per tensor of a group
+    const unsigned char* rec;    // start of the record
+    u64 rec_avail;               // bytes the caller says belong to it
+    const float* w_prev;
+    float* w_out;
+    float* ea_out;
+    float* eas_out;
+    u64 numel;
+    u32 tile_begin;
+    u32 num_tiles;
+};
+
+struct DecState {                // decompress scratch per tensor
+    u32 valid;
+    u32 bits;
+    u32 nnz_w, nnz_o;
+    u64 off_bm_w, off_bm_o, off_codes[3];
+    float cent[3][KPAD];
+};
+
+// ---- layout arithmetic (host and device) ----------------------------------
+__host__ __device__ inline u64 align16(u64 n) { return (n + 15ull) & ~15ull; }
+__host__ __device__ inline u64 header_bytes(int k) { return align16(HEADER_FIXED + 12ull * k); }
+__host__ __device__ inline u64 bitmap_bytes(u64 numel) { return align16(4ull * ((numel + 31) / 32)); }
+__host__ __device__ inline u64 code_bytes(u64 nnz, int bits) { return align16((nnz * bits + 7) / 8); }
+__host__ __device__ inline u64 record_bytes(u64 numel, u64 nnz_w, u64 nnz_o, int bits) {
+    return header_bytes((1 << bits) - 1) + 2 * bitmap_bytes(numel) + code_bytes(nnz_w, bits) +
+           2 * code_bytes(nnz_o, bits);
+}
+
+// ---- device helpers ---------------------------------------------------------
+#ifdef __CUDACC__
+// Tensor that owns group tile `tile` (descs are in tile order).
+__device__ inline int find_tensor(const TensorDesc* __restrict__ descs, int n, u32 tile) {
+    int lo = 0, hi = n - 1;
+    while (lo < hi) {
+        int mid = (lo + hi + 1) >> 1;
+        if (descs[mid].tile_begin <= tile) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+__device__ inline int find_tensor(const DecDesc* __restrict__ descs, int n, u32 tile) {
+    int lo = 0, hi = n - 1;
+    while (lo < hi) {
+        int mid = (lo + hi + 1) >> 1;
+        if (descs[mid].tile_begin <= tile) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+// Four consecutive elements starting at i0 (a multiple of 4).  Elements at or
+// past n read as 0 and are reported through the return value (count valid).
+__device__ inline int load4(const float* __restrict__ p, u64 i0, u64 n, float v[4]) {
+    if (i0 + 4 <= n) {
+        float4 t = __ldcs(reinterpret_cast<const float4*>(p + i0));
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+        return 4;
+    }
+    int c = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        if (i0 + k < n) { v[k] = __ldcs(p + i0 + k); c = k + 1; } else v[k] = 0.f;
+    }
+    return c;
+}
+
+// Contiguous share of [0, total) for block b of g.
+__device__ inline void block_range(u32 total, u32& lo, u32& hi) {
+    lo = (u32)(((u64)total * blockIdx.x) / gridDim.x);
+    hi = (u32)(((u64)total * (blockIdx.x + 1)) / gridDim.x);
+}
+
+__device__ inline u64 warp_sum_u64(u64 v) {
+#pragma unroll
+    for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Exclusive prefix of the per-tile survivor counts of the tiles [tb, tb + ntl)
+// (one tensor), written to tile_off_*; totals returned to every thread.
+// Called by a whole block of TPB threads.
+__device__ inline void scan_tile_counts(u32 tb, u32 ntl, const Workspace& ws, u32& tot_w, u32& tot_o) {
+    __shared__ u32 wtot[2][TPB / 32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    u32 carry_w = 0, carry_o = 0;
+    for (u32 b0 = 0; b0 < ntl; b0 += TPB) {
+        const u32 i = b0 + tid;
+        const u32 cw = i < ntl ? ws.tile_cnt_w[tb + i] : 0u;
+        const u32 co = i < ntl ? ws.tile_cnt_o[tb + i] : 0u;
+        u32 iw = cw, io = co;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            u32 x = __shfl_up_sync(0xffffffffu, iw, o);
+            u32 y = __shfl_up_sync(0xffffffffu, io, o);
+            if (lane >= o) { iw += x; io += y; }
+        }
+        if (lane == 31) { wtot[0][warp] = iw; wtot[1][warp] = io; }
+        __syncthreads();
+        u32 bw = 0, bo = 0, tw = 0, to = 0;
+#pragma unroll
+        for (int w = 0; w < TPB / 32; ++w) {
+            if (w < warp) { bw += wtot[0][w]; bo += wtot[1][w]; }
+            tw += wtot[0][w]; to += wtot[1][w];
+        }
+        if (i < ntl) {
+            ws.tile_off_w[tb + i] = carry_w + bw + iw - cw;
+            ws.tile_off_o[tb + i] = carry_o + bo + io - co;
+        }
+        carry_w += tw; carry_o += to;
+        __syncthreads();
+    }
+    tot_w = carry_w; tot_o = carry_o;
+}
+#endif
+
+// ---- launch wrappers --------------------------------------------------------
+struct LaunchCfg {
+    int sms;
+    cudaStream_t stream;
+};
+
+void launch_stats(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
+                  const Workspace& ws, const Params& p);
+void launch_mask_compact(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
+                         const Workspace& ws, const Params& p, CallState* call, u64 blob_capacity);
+void launch_kmeans(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
+                   const Workspace& ws, const Params& p);
+void launch_pack(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
+                 const Workspace& ws, const Params& p, unsigned char* blob, CallState* call,
+                 TensorResult* results);
+void launch_decode(const LaunchCfg&, const DecDesc* descs, DecState* st, int nt, u32 tiles,
+                   const Workspace& ws, CallState* call);
+
+}  // namespace excp
