@@ -1,0 +1,389 @@
+#!/usr/bin/env python
+"""Benchmark of the ExCP compression hot path.
+
+One "step" = one excp_compress_checkpoint call over the whole tensor list of the
+workload (all stages: statistics, masks + compaction, K-means, packing), inputs
+resident in HBM.  `value` = parameters compressed per second over all ranks.
+Beside it: per-stage CUDA-event times and the roofline of the dominant kernel,
+the decompress rate, the end-to-end rate through the host-buffer entry point
+(host->device and device->host copies inside the timed region), and the CPU
+oracle timed on a bounded sample of the same workload.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--config llama-7b|pythia-1.4b|pythia-410m|tiny] [--median residual|weight]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+os.environ.setdefault("PYTORCH_CUDA_ALLOC_CONF", "expandable_segments:True")
+
+METRIC = "compress params/s and GB/s of (W,W_prev,m,v) read at 7B shape; % of HBM peak"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="llama-7b")
+    ap.add_argument("--median", default="residual", choices=["residual", "weight"])
+    ap.add_argument("--kmeans-iters", type=int, default=10)
+    ap.add_argument("--workspace-numel", type=int, default=1_200_000_000)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-decompress", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--max-tensors", type=int, default=None, help="debug: only the first tensors of the list")
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi sampling of SM clock and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "200", "-i", str(self.index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        clocks, reasons, mx = [], set(), None
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                clocks.append(float(parts[1])); mx = float(parts[2])
+            except ValueError:
+                continue
+            for name, v in zip(names, parts[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        self.f.close()
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        if clocks:
+            out.update(sm_mhz=statistics.median(clocks), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(clocks))
+        return out
+
+
+def mem_available_gb() -> float:
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable"):
+                return int(line.split()[1]) / 1e6
+    except Exception:
+        pass
+    return 0.0
+
+
+def oracle_sample(args, shapes, seed):
+    """The oracle, as it stands, on one mid-sized tensor of the workload.  Returns (params/s, description)."""
+    import torch
+    from oracle import excp_oracle as orc
+    from paper_2406_11257_b200 import synth
+    cand = [(i, n) for i, (_, n) in enumerate(shapes) if n <= 17_000_000]
+    idx, numel = max(cand, key=lambda t: t[1])
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    q = [t.cpu().numpy() for t in synth.make_quad(numel, seed, idx, device=dev)]
+    p = orc.Params(kmeans_iters=args.kmeans_iters, median_source=1 if args.median == "residual" else 0)
+    torch.set_num_threads(1)
+    t0 = time.perf_counter()
+    orc.compress_tensor(*q, p, tensor_index=idx)
+    dt = time.perf_counter() - t0
+    return numel / dt, f"tensor {idx} ({shapes[idx][0]}, {numel} params) of the workload, {dt:.1f} s", numel, dt
+
+
+def run_reference(args):
+    """The CPU oracle as the reference arm: each step compresses a bounded sample of the workload."""
+    from paper_2406_11257_b200 import synth
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    shapes = synth.tensor_list(synth.CONFIG_SHAPES[args.config])
+    cand = [(i, n) for i, (_, n) in enumerate(shapes) if n <= 4_500_000] or [(0, shapes[0][1])]
+    idx, numel = max(cand, key=lambda t: t[1])
+    import torch
+    from oracle import excp_oracle as orc
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    q = [t.cpu().numpy() for t in synth.make_quad(numel, 0, idx, device=dev)]
+    p = orc.Params(kmeans_iters=args.kmeans_iters, median_source=1 if args.median == "residual" else 0)
+    torch.set_num_threads(1)
+    for _ in range(args.warmup):
+        orc.compress_tensor(*q, p, tensor_index=idx)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        orc.compress_tensor(*q, p, tensor_index=idx)
+    dt = time.perf_counter() - t0
+    value = numel * args.steps / dt
+    sample = f"tensor {idx} ({shapes[idx][0]}, {numel} params) of the workload per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "params/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{args.config} shaped checkpoint pair, median of |{'dW' if args.median == 'residual' else 'W'}|",
+                   "kmeans_iters": args.kmeans_iters, "bits": 4},
+        "cpu_baseline": {"value": value, "unit": "params/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "params/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2406_11257_b200 import binding, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the compression path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    shape = synth.CONFIG_SHAPES[args.config]
+    shapes = synth.tensor_list(shape)
+    if args.max_tensors:
+        shapes = shapes[:args.max_tensors]
+    n_tot = sum(n for _, n in shapes)
+    seed = 1000 + rank                                    # every rank compresses its own checkpoint
+    quads = [synth.make_quad(n, seed, i, device=dev) for i, (_, n) in enumerate(shapes)]
+    torch.cuda.synchronize()
+
+    ws_numel = min(args.workspace_numel, n_tot + 4096 * len(shapes))
+    ws_numel = max(ws_numel, max(n for _, n in shapes))
+    h = binding.Handle(workspace_numel=ws_numel)
+    p = binding.Params(kmeans_iters=args.kmeans_iters,
+                       median_source=binding.MEDIAN_ABS_RESIDUAL if args.median == "residual" else binding.MEDIAN_ABS_WEIGHT)
+    bound = sum(binding.compress_bound(n) for _, n in shapes)
+    cap = min(bound, int(0.80 * n_tot) + 1024 * len(shapes) + (1 << 20))
+    blob = torch.empty(cap, dtype=torch.uint8, device=dev)
+
+    h.profile_enable(True)
+    offs = stats = None
+    for _ in range(max(args.warmup, 0)):
+        offs, stats = h.compress_checkpoint(p, quads, blob)
+    stage_ms = {}
+    launches = 0
+    sampler = ClockSampler(local)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(); torch.cuda.synchronize()
+    sampler.start()
+    ev0.record()
+    for _ in range(args.steps):
+        offs, stats = h.compress_checkpoint(p, quads, blob)
+        ms, l = h.profile_read()
+        launches += l
+        for k, v in ms.items():
+            stage_ms[k] = stage_ms.get(k, 0.0) + v
+    ev1.record()
+    torch.cuda.synchronize(); barrier()
+    clocks = sampler.stop()
+    elapsed_ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / args.steps
+    value = world * n_tot / (ms_per_step * 1e-3)
+
+    nnz_w = sum(s.nnz_w for s in stats)
+    nnz_o = sum(s.nnz_o for s in stats)
+    blob_bytes = offs[-1]
+    f_w, f_o = nnz_w / n_tot, nnz_o / n_tot
+    T = args.kmeans_iters
+    src_b = 8 if args.median == "residual" else 4
+    # bytes each stage must move once (its inputs read once, its outputs written once)
+    stage_bytes = {
+        "stats1": (src_b + 4) * n_tot,
+        "stats2": src_b * n_tot,
+        "mask_compact": 16 * n_tot + n_tot / 4 + 4 * nnz_w + 8 * nnz_o,
+        "lloyd_dw": T * 4 * nnz_w, "lloyd_ea": T * 4 * nnz_o, "lloyd_eas": T * 4 * nnz_o,
+        "pack_codes": 4.5 * (nnz_w + 2 * nnz_o),
+        "copy_bitmaps": n_tot / 2,
+    }
+    # what the method itself must move (one statistics sweep, not two)
+    algo_bytes = sum(v for k, v in stage_bytes.items() if k != "stats2")
+    peak, peak_kind = measured_peak()
+    per_step = {k: v / args.steps for k, v in stage_ms.items()}
+    dom = max((k for k in stage_bytes), key=lambda k: per_step.get(k, 0.0))
+    dom_ms = per_step[dom]
+    dom_gbs = stage_bytes[dom] / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
+    groups_note = f"{launches // args.steps} launches per step"
+    stages = {k: {"ms": round(per_step.get(k, 0.0), 4),
+                  "gbs": round(stage_bytes[k] / (per_step[k] * 1e-3) / 1e9, 1) if k in stage_bytes and per_step.get(k, 0) > 0 else None}
+              for k in per_step if per_step[k] > 0}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": "params/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{shape.name} checkpoint pair ({len(shapes)} tensors, {n_tot} params, fp32 W_t, W_prev, ea, eas), "
+                               f"median of |{'dW' if args.median == 'residual' else 'W_t'}|, alpha 5e-5, beta 2.0",
+                   "bits": 4, "kmeans_iters": T, "l2": "inputs larger than L2 (no flush needed)" if 16 * n_tot > 4e8 else "inputs fit L2",
+                   "workspace_numel": ws_numel, "per_rank": "each rank compresses its own checkpoint; no collective"},
+        "input_gbs": 16 * value / 1e9,
+        "algorithmic_bytes_per_param": algo_bytes / n_tot,
+        "algorithmic_gbs": algo_bytes / n_tot * value / world / 1e9,
+        "hbm_frac_of_measured": algo_bytes / n_tot * value / world / 1e9 / peak,
+        "hbm_frac_of_nominal_8TBs": algo_bytes / n_tot * value / world / 1e9 / NOMINAL_HBM_GBS,
+        "survivors": {"f_w": f_w, "f_o": f_o},
+        "compression": {"blob_bytes": blob_bytes, "ratio_vs_12B_per_param": 12 * n_tot / blob_bytes},
+        "stages": stages,
+        "roofline": {"bound": "hbm", "kernel": dom, "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": dom_gbs / peak, "peak_kind": peak_kind, "traffic": None,
+                     "algorithmic_bytes_per_step": stage_bytes[dom], "ms_per_step": dom_ms, "note": groups_note},
+        "clocks": clocks,
+        "gpu_launches": launches,
+    }
+
+    # ---- decompress (Algorithm 2) on the records just written ---------------
+    if not args.no_decompress:
+        h.profile_enable(False)
+        chunk_cap = ws_numel
+        out_w = torch.empty(chunk_cap, dtype=torch.float32, device=dev)
+        out_a = torch.empty(chunk_cap, dtype=torch.float32, device=dev)
+        out_s = torch.empty(chunk_cap, dtype=torch.float32, device=dev)
+        chunks, cur, used = [], [], 0
+        for i, (_, n) in enumerate(shapes):
+            n4 = (n + 3) // 4 * 4
+            if cur and used + n4 > chunk_cap:
+                chunks.append(cur); cur, used = [], 0
+            cur.append((i, used, n)); used += n4
+        if cur:
+            chunks.append(cur)
+
+        def decompress_all():
+            for ch in chunks:
+                i0, i1 = ch[0][0], ch[-1][0] + 1
+                wp = [quads[i][1] for i, _, _ in ch]
+                h.decompress_checkpoint(blob[offs[i0]:], [o - offs[i0] for o in offs[i0:i1 + 1]], wp,
+                                        [out_w[o:o + n] for _, o, n in ch], [out_a[o:o + n] for _, o, n in ch],
+                                        [out_s[o:o + n] for _, o, n in ch])
+        decompress_all()
+        torch.cuda.synchronize()
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0.record()
+        for _ in range(args.steps):
+            decompress_all()
+        d1.record(); torch.cuda.synchronize()
+        dms = d0.elapsed_time(d1) / args.steps
+        dec_bytes = n_tot / 4 + 0.5 * (nnz_w + 2 * nnz_o) + 4 * n_tot + 12 * n_tot
+        out["decompress"] = {"value": n_tot / (dms * 1e-3), "unit": "params/s", "ms_per_step": dms,
+                             "algorithmic_gbs": dec_bytes / (dms * 1e-3) / 1e9,
+                             "hbm_frac_of_measured": dec_bytes / (dms * 1e-3) / 1e9 / peak,
+                             "calls_per_step": len(chunks)}
+        del out_w, out_a, out_s
+
+    # ---- end to end through the host-buffer entry point ----------------------
+    if not args.no_e2e:
+        need_gb = 16 * n_tot / 1e9
+        sub = list(range(len(shapes)))
+        if mem_available_gb() < 1.4 * need_gb + 8:
+            budget, acc, sub = 0.45 * mem_available_gb() * 1e9, 0, []
+            for i, (_, n) in enumerate(shapes):
+                if acc + 16 * n > budget:
+                    break
+                sub.append(i); acc += 16 * n
+        n_sub = sum(shapes[i][1] for i in sub)
+        hq = []
+        for i in sub:
+            hq.append(tuple(torch.empty(shapes[i][1], dtype=torch.float32, pin_memory=True) for _ in range(4)))
+            for dst, src in zip(hq[-1], quads[i]):
+                dst.copy_(src)
+        hblob = torch.empty(min(cap, int(0.80 * n_sub) + 1024 * len(sub) + (1 << 20)), dtype=torch.uint8, pin_memory=True)
+        e2e_ws = min(ws_numel, max(160_000_000, max(shapes[i][1] for i in sub)))
+        h2 = binding.Handle(workspace_numel=e2e_ws)
+        hoffs, _ = h2.compress_checkpoint_host(p, hq, hblob, want_stats=False)       # warm-up (allocates the staging)
+        barrier(); torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.e2e_steps):
+            hoffs, _ = h2.compress_checkpoint_host(p, hq, hblob, want_stats=False)
+        e1.record(); torch.cuda.synchronize(); barrier()
+        ems = e0.elapsed_time(e1) / args.e2e_steps
+        if world > 1:
+            t = torch.tensor([ems], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ems = float(t.item())
+        out["e2e"] = {"value": world * n_sub / (ems * 1e-3), "unit": "params/s", "h2d_bytes_per_step": 16 * n_sub,
+                      "d2h_bytes_per_step": hoffs[-1], "ms_per_step": ems, "steps": args.e2e_steps,
+                      "sample": "whole workload" if len(sub) == len(shapes) else f"first {len(sub)} tensors ({n_sub} params): host memory",
+                      "h2d_gbs": 16 * n_sub / (ems * 1e-3) / 1e9}
+        h2.close()
+        del hq, hblob
+
+    # ---- the oracle on the host cores (rank 0, one GPU only) -----------------
+    if not args.no_cpu and rank == 0 and world == 1:
+        v, desc, _, _ = oracle_sample(args, shapes, seed)
+        out["cpu_baseline"] = {"value": v, "unit": "params/s", "cores": 1, "kind": "oracle", "sample": desc}
+
+    h.close()
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

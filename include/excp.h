@@ -149,6 +149,23 @@ excp_status excp_compress_checkpoint(excp_handle h, const excp_params* params, s
                                      size_t* tensor_offsets_out, excp_tensor_stats* stats_out,
                                      void* cuda_stream);
 
+/* excp_compress_checkpoint for a checkpoint that lives in HOST memory (the usual case: the
+ * compression runs beside training, Section 3.4, on a copy of the states).
+ *   w_t, w_prev, ea, eas  host arrays [num_tensors] of HOST pointers (fp32[numel[i]]); page-locked
+ *                         memory is needed for the copies to overlap the kernels.
+ *   blob_out              HOST, blob_capacity bytes; receives the records back to back.
+ * The tensor list is cut into the same groups as in excp_compress_checkpoint; while the kernels
+ * of one group run on `cuda_stream`, the inputs of the next are copied to a second device
+ * staging slot on a copy stream of the handle and the finished records are copied back on
+ * another.  The first call allocates the staging (32 bytes per workspace element plus two record
+ * buffers).  Records and offsets are identical to excp_compress_checkpoint's.  Synchronises. */
+excp_status excp_compress_checkpoint_host(excp_handle h, const excp_params* params, size_t num_tensors,
+                                          const float* const* w_t, const float* const* w_prev,
+                                          const float* const* ea, const float* const* eas,
+                                          const size_t* numel, void* blob_out, size_t blob_capacity,
+                                          size_t* tensor_offsets_out, excp_tensor_stats* stats_out,
+                                          void* cuda_stream);
+
 /* Algorithm 2 (after the un-archiver) for one tensor.
  *   blob                  device, blob_bytes bytes, one record.
  *   w_prev                device fp32[numel]: W^_(t-1).
@@ -168,6 +185,20 @@ excp_status excp_decompress_checkpoint(excp_handle h, const void* blob, const si
                                        size_t num_tensors, const float* const* w_prev, const size_t* numel,
                                        float* const* w_out, float* const* ea_out, float* const* eas_out,
                                        void* cuda_stream);
+
+/* Per-stage timing of the last compress/decompress call (no counterpart in the paper; the
+ * stages are this library's kernels).  With timing enabled each call records CUDA events on
+ * its stream between stages and, after its final synchronisation, sums the elapsed times per
+ * stage.  The launch counter is kept whether or not timing is enabled.
+ *   excp_profile_enable       turns event recording on (non-zero) or off; creates the events once.
+ *   excp_profile_stage_count  number of stages; excp_profile_stage_name gives each a static name.
+ *   excp_profile_read         stage_ms_out: host double[stage_count], milliseconds per stage of the
+ *                             last call (may be NULL); launches_out: kernels launched by the last
+ *                             call (may be NULL). */
+excp_status excp_profile_enable(excp_handle h, int enable);
+int excp_profile_stage_count(void);
+const char* excp_profile_stage_name(int stage);
+excp_status excp_profile_read(excp_handle h, double* stage_ms_out, unsigned long long* launches_out);
 
 #ifdef __cplusplus
 }

@@ -20,7 +20,8 @@ STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED", -3: "BUFFER_TOO_SMALL",
 
 EXPORTS = ["excp_create", "excp_destroy", "excp_record_bytes", "excp_compress_bound",
            "excp_status_string", "excp_last_cuda_error", "excp_compress_tensor",
-           "excp_compress_checkpoint", "excp_decompress_tensor", "excp_decompress_checkpoint"]
+           "excp_compress_checkpoint", "excp_compress_checkpoint_host", "excp_decompress_tensor", "excp_decompress_checkpoint",
+           "excp_profile_enable", "excp_profile_stage_count", "excp_profile_stage_name", "excp_profile_read"]
 
 
 class ExcpError(RuntimeError):
@@ -78,9 +79,15 @@ def load_library() -> C.CDLL:
     lib.excp_compress_checkpoint.argtypes = [vp, C.POINTER(CParams), sz, C.POINTER(vp), C.POINTER(vp),
                                              C.POINTER(vp), C.POINTER(vp), C.POINTER(sz), vp, sz,
                                              C.POINTER(sz), C.POINTER(CStats), vp]
+    lib.excp_compress_checkpoint_host.argtypes = lib.excp_compress_checkpoint.argtypes
     lib.excp_decompress_tensor.argtypes = [vp, vp, sz, vp, sz, vp, vp, vp, vp]
     lib.excp_decompress_checkpoint.argtypes = [vp, vp, C.POINTER(sz), sz, C.POINTER(vp), C.POINTER(sz),
                                                C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), vp]
+    lib.excp_profile_enable.argtypes = [vp, C.c_int]
+    lib.excp_profile_stage_count.argtypes = []
+    lib.excp_profile_stage_name.argtypes = [C.c_int]
+    lib.excp_profile_stage_name.restype = C.c_char_p
+    lib.excp_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_ulonglong)]
     for name in EXPORTS:
         if getattr(lib, name).restype is C.c_int:
             getattr(lib, name).restype = C.c_int
@@ -137,6 +144,19 @@ class Handle:
         self.lib.excp_last_cuda_error(self._h, C.byref(e))
         return e.value
 
+    def profile_enable(self, on: bool = True) -> None:
+        st = self.lib.excp_profile_enable(self._h, int(on))
+        if st != 0:
+            raise ExcpError(st, "excp_profile_enable")
+
+    def profile_read(self):
+        """(dict stage name -> ms of the last call, kernel launches of the last call)."""
+        n = self.lib.excp_profile_stage_count()
+        ms = (C.c_double * n)()
+        launches = C.c_ulonglong(0)
+        self.lib.excp_profile_read(self._h, ms, C.byref(launches))
+        return {self.lib.excp_profile_stage_name(i).decode(): ms[i] for i in range(n)}, launches.value
+
     # ---- Algorithm 1 -----------------------------------------------------
     def compress_tensor(self, p: Params, w_t, w_prev, ea, eas, blob_out: torch.Tensor):
         """excp_compress_tensor.  Returns (record bytes, stats)."""
@@ -165,6 +185,28 @@ class Handle:
                                                offs, stats, _stream())
         if st != 0:
             raise ExcpError(st, "excp_compress_checkpoint")
+        return list(offs), (list(stats) if want_stats else None)
+
+    def compress_checkpoint_host(self, p: Params, tensors, blob_out: torch.Tensor, want_stats: bool = True):
+        """excp_compress_checkpoint_host: `tensors` and `blob_out` are HOST tensors
+        (page-locked for the copies to overlap the kernels)."""
+        n = len(tensors)
+        for q in tensors:
+            for t in q:
+                if t.is_cuda or t.dtype != torch.float32 or not t.is_contiguous():
+                    raise TypeError("expected contiguous float32 host tensors")
+        if blob_out.is_cuda:
+            raise TypeError("blob_out must be a host tensor")
+        arr = lambda k: (C.c_void_p * n)(*[_ptr(q[k]) for q in tensors])
+        numel = (C.c_size_t * n)(*[q[0].numel() for q in tensors])
+        offs = (C.c_size_t * (n + 1))()
+        stats = (CStats * n)() if want_stats else None
+        cp = p.to_c()
+        st = self.lib.excp_compress_checkpoint_host(self._h, C.byref(cp), n, arr(0), arr(1), arr(2), arr(3), numel,
+                                                    blob_out.data_ptr(), blob_out.numel() * blob_out.element_size(),
+                                                    offs, stats, _stream())
+        if st != 0:
+            raise ExcpError(st, "excp_compress_checkpoint_host")
         return list(offs), (list(stats) if want_stats else None)
 
     # ---- Algorithm 2 -----------------------------------------------------

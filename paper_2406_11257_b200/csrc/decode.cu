@@ -200,11 +200,13 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
 void launch_decode(const LaunchCfg& cfg, const DecDesc* descs, DecState* st, int nt, u32 tiles,
                    const Workspace& ws, CallState* call) {
     dec_validate_kernel<<<nt, 64, 0, cfg.stream>>>(descs, st, call);
-    if (!tiles) return;
+    if (!tiles) { prof_mark(cfg, ST_DEC_PREP, 1); return; }
     dec_popcount_kernel<<<(tiles + TPB / 32 - 1) / (TPB / 32), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws);
     dec_scan_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, ws, call);
+    prof_mark(cfg, ST_DEC_PREP, 3);
     const u32 grid = min(tiles, (u32)cfg.sms * 4u);
     decode_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, call);
+    prof_mark(cfg, ST_DECODE, 1);
 }
 
 }  // namespace excp

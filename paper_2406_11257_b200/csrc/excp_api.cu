@@ -11,6 +11,41 @@
 
 using namespace excp;
 
+namespace excp {
+// Launch counter and optional CUDA-event timing of the stages of one call.
+struct Profiler {
+    bool enabled = false;
+    std::vector<cudaEvent_t> ev;
+    std::vector<int> stage;
+    size_t used = 0;
+    double ms[ST_COUNT] = {};
+    unsigned long long launches = 0;
+    void begin(cudaStream_t s) {
+        used = 0;
+        launches = 0;
+        for (double& m : ms) m = 0.0;
+        if (enabled && !ev.empty()) cudaEventRecord(ev[0], s);
+    }
+    void finish() {   // after the stream has been synchronised
+        if (!enabled) return;
+        for (size_t i = 1; i <= used; ++i) {
+            float t = 0.f;
+            if (cudaEventElapsedTime(&t, ev[i - 1], ev[i]) == cudaSuccess) ms[stage[i]] += t;
+        }
+    }
+};
+void prof_mark(const LaunchCfg& cfg, int stage, int launches) {
+    Profiler* p = cfg.prof;
+    if (!p) return;
+    p->launches += (unsigned long long)launches;
+    if (p->enabled && p->used + 1 < p->ev.size()) {
+        ++p->used;
+        p->stage[p->used] = stage;
+        cudaEventRecord(p->ev[p->used], cfg.stream);
+    }
+}
+}  // namespace excp
+
 struct excp_handle_s {
     int device = 0;
     int sms = 0;
@@ -26,6 +61,13 @@ struct excp_handle_s {
     CallState* h_call = nullptr;         // pinned
     size_t tensor_cap = 0;               // entries the per-call arrays hold
     int last_cuda_error = 0;
+    Profiler prof;
+    // host-buffer path: two staging slots (inputs + records), its own copy streams
+    float* stage[2][4] = {};
+    unsigned char* stage_blob[2] = {};
+    size_t stage_blob_bytes = 0;
+    cudaStream_t s_h2d = nullptr, s_d2h = nullptr;
+    cudaEvent_t ev_h2d[2] = {}, ev_compute[2] = {}, ev_d2h[2] = {};
 };
 
 namespace {
@@ -96,6 +138,67 @@ bool make_groups(excp_handle h, const size_t* numel, size_t n, std::vector<Group
     return true;
 }
 
+excp_status validate_params(const excp_params* params) {
+    if (!params) return EXCP_ERR_INVALID_ARG;
+    if (params->bits == 2 || params->bits == 8) return EXCP_ERR_UNSUPPORTED;
+    if (params->bits != 4 || params->kmeans_iters < 0 || params->flags != 0 ||
+        (params->median_source != 0 && params->median_source != 1) ||
+        !(params->alpha >= 0.f) || !(params->beta >= 0.f) || std::isinf(params->alpha) ||
+        std::isinf(params->beta))
+        return EXCP_ERR_INVALID_ARG;
+    return EXCP_OK;
+}
+
+Params to_params(const excp_params* params) {
+    Params p;
+    p.alpha = params->alpha; p.beta = params->beta; p.bits = params->bits;
+    p.kmeans_iters = params->kmeans_iters; p.seed = params->seed; p.median_source = params->median_source;
+    return p;
+}
+
+// All kernels of one group, in order.
+bool run_group(excp_handle h, const LaunchCfg& cfg, const TensorDesc* descs, int nt, u32 tiles, const Params& p,
+               unsigned char* blob, u64 blob_capacity, TensorResult* results) {
+    if (!check(h, cudaMemsetAsync(h->d_state, 0, nt * sizeof(TensorState), cfg.stream))) return false;
+    launch_stats(cfg, descs, h->d_state, nt, tiles, h->ws, p);
+    launch_mask_compact(cfg, descs, h->d_state, nt, tiles, h->ws, p, h->d_call, blob_capacity);
+    launch_kmeans(cfg, descs, h->d_state, nt, tiles, h->ws, p);
+    launch_pack(cfg, descs, h->d_state, nt, tiles, h->ws, p, blob, h->d_call, results);
+    return check(h, cudaGetLastError());
+}
+
+void fill_outputs(excp_handle h, size_t first, size_t count, const size_t* numel, size_t base,
+                  size_t* tensor_offsets_out, excp_tensor_stats* stats_out) {
+    for (size_t i = first; i < first + count; ++i) {
+        const TensorResult& r = h->h_results[i];
+        tensor_offsets_out[i] = base + (size_t)r.blob_off;
+        tensor_offsets_out[i + 1] = base + (size_t)(r.blob_off + r.blob_bytes);
+        if (stats_out) {
+            excp_tensor_stats& s = stats_out[i];
+            s.numel = numel[i]; s.nnz_w = r.nnz_w; s.nnz_o = r.nnz_o; s.blob_bytes = r.blob_bytes;
+            s.median = r.median; s.mean_abs_ea = r.mean_abs_ea; s.thr_w = r.thr_w; s.thr_o = r.thr_o;
+        }
+    }
+}
+
+bool ensure_host_path(excp_handle h) {
+    if (h->s_h2d) return true;
+    const size_t elems = h->cap_tiles * (size_t)TILE;
+    h->stage_blob_bytes = (size_t)record_bytes(elems, elems, elems, 4) + (size_t)MAX_GROUP_TENSORS * 512;
+    bool ok = true;
+    for (int k = 0; k < 2 && ok; ++k) {
+        for (int j = 0; j < 4 && ok; ++j)
+            ok = check(h, cudaMalloc(reinterpret_cast<void**>(&h->stage[k][j]), elems * sizeof(float)));
+        ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->stage_blob[k]), h->stage_blob_bytes));
+        ok = ok && check(h, cudaEventCreateWithFlags(&h->ev_h2d[k], cudaEventDisableTiming));
+        ok = ok && check(h, cudaEventCreateWithFlags(&h->ev_compute[k], cudaEventDisableTiming));
+        ok = ok && check(h, cudaEventCreateWithFlags(&h->ev_d2h[k], cudaEventDisableTiming));
+    }
+    ok = ok && check(h, cudaStreamCreateWithFlags(&h->s_d2h, cudaStreamNonBlocking));
+    ok = ok && check(h, cudaStreamCreateWithFlags(&h->s_h2d, cudaStreamNonBlocking));
+    return ok;
+}
+
 excp_status status_from_flags(u32 flags) {
     if (flags & FLAG_INTERNAL) return EXCP_ERR_CUDA;
     if (flags & FLAG_NONFINITE) return EXCP_ERR_NONFINITE_INPUT;
@@ -159,6 +262,16 @@ excp_status excp_destroy(excp_handle h) {
     if (h->d_call) cudaFree(h->d_call);
     if (h->h_call) cudaFreeHost(h->h_call);
     free_call_arrays(h);
+    for (int k = 0; k < 2; ++k) {
+        for (int j = 0; j < 4; ++j) if (h->stage[k][j]) cudaFree(h->stage[k][j]);
+        if (h->stage_blob[k]) cudaFree(h->stage_blob[k]);
+        if (h->ev_h2d[k]) cudaEventDestroy(h->ev_h2d[k]);
+        if (h->ev_compute[k]) cudaEventDestroy(h->ev_compute[k]);
+        if (h->ev_d2h[k]) cudaEventDestroy(h->ev_d2h[k]);
+    }
+    if (h->s_h2d) cudaStreamDestroy(h->s_h2d);
+    if (h->s_d2h) cudaStreamDestroy(h->s_d2h);
+    for (cudaEvent_t e : h->prof.ev) cudaEventDestroy(e);
     delete h;
     return EXCP_OK;
 }
@@ -199,12 +312,8 @@ excp_status excp_compress_checkpoint(excp_handle h, const excp_params* params, s
     if (!h || !params || !tensor_offsets_out) return EXCP_ERR_INVALID_ARG;
     if (num_tensors && (!w_t || !w_prev || !ea || !eas || !numel)) return EXCP_ERR_INVALID_ARG;
     if (!blob_out || !aligned16(blob_out)) return EXCP_ERR_INVALID_ARG;
-    if (params->bits == 2 || params->bits == 8) return EXCP_ERR_UNSUPPORTED;
-    if (params->bits != 4 || params->kmeans_iters < 0 || params->flags != 0 ||
-        (params->median_source != 0 && params->median_source != 1) ||
-        !(params->alpha >= 0.f) || !(params->beta >= 0.f) || std::isinf(params->alpha) ||
-        std::isinf(params->beta))
-        return EXCP_ERR_INVALID_ARG;
+    const excp_status ps = validate_params(params);
+    if (ps != EXCP_OK) return ps;
     for (size_t i = 0; i < num_tensors; ++i) {
         if (numel[i] == 0) continue;
         if (!w_t[i] || !w_prev[i] || !ea[i] || !eas[i]) return EXCP_ERR_INVALID_ARG;
@@ -233,43 +342,124 @@ excp_status excp_compress_checkpoint(excp_handle h, const excp_params* params, s
             tile += d.num_tiles;
         }
     }
-    Params p;
-    p.alpha = params->alpha; p.beta = params->beta; p.bits = params->bits;
-    p.kmeans_iters = params->kmeans_iters; p.seed = params->seed; p.median_source = params->median_source;
-
+    const Params p = to_params(params);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    LaunchCfg cfg{h->sms, stream};
+    LaunchCfg cfg{h->sms, stream, &h->prof};
+    h->prof.begin(stream);
     TensorDesc* dd = static_cast<TensorDesc*>(h->d_desc);
     bool ok = check(h, cudaMemsetAsync(h->d_call, 0, sizeof(CallState), stream));
     ok = ok && check(h, cudaMemcpyAsync(dd, hd, num_tensors * sizeof(TensorDesc), cudaMemcpyHostToDevice, stream));
     for (size_t gi = 0; ok && gi < groups.size(); ++gi) {
         const Group& g = groups[gi];
-        const int nt = (int)g.count;
-        ok = check(h, cudaMemsetAsync(h->d_state, 0, nt * sizeof(TensorState), stream));
-        if (!ok) break;
-        launch_stats(cfg, dd + g.first, h->d_state, nt, g.tiles, h->ws, p);
-        launch_mask_compact(cfg, dd + g.first, h->d_state, nt, g.tiles, h->ws, p, h->d_call, blob_capacity);
-        launch_kmeans(cfg, dd + g.first, h->d_state, nt, g.tiles, h->ws, p);
-        launch_pack(cfg, dd + g.first, h->d_state, nt, g.tiles, h->ws, p,
-                    static_cast<unsigned char*>(blob_out), h->d_call, h->d_results + g.first);
-        ok = check(h, cudaGetLastError());
+        ok = run_group(h, cfg, dd + g.first, (int)g.count, g.tiles, p, static_cast<unsigned char*>(blob_out),
+                       blob_capacity, h->d_results + g.first);
     }
     ok = ok && check(h, cudaMemcpyAsync(h->h_results, h->d_results, num_tensors * sizeof(TensorResult),
                                         cudaMemcpyDeviceToHost, stream));
     ok = ok && check(h, cudaMemcpyAsync(h->h_call, h->d_call, sizeof(CallState), cudaMemcpyDeviceToHost, stream));
     if (!check(h, cudaStreamSynchronize(stream)) || !ok) return EXCP_ERR_CUDA;
+    h->prof.finish();
+    fill_outputs(h, 0, num_tensors, numel, 0, tensor_offsets_out, stats_out);
+    return status_from_flags(h->h_call->flags);
+}
 
-    for (size_t i = 0; i < num_tensors; ++i) {
-        const TensorResult& r = h->h_results[i];
-        tensor_offsets_out[i] = (size_t)r.blob_off;
-        tensor_offsets_out[i + 1] = (size_t)(r.blob_off + r.blob_bytes);
-        if (stats_out) {
-            excp_tensor_stats& s = stats_out[i];
-            s.numel = numel[i]; s.nnz_w = r.nnz_w; s.nnz_o = r.nnz_o; s.blob_bytes = r.blob_bytes;
-            s.median = r.median; s.mean_abs_ea = r.mean_abs_ea; s.thr_w = r.thr_w; s.thr_o = r.thr_o;
+excp_status excp_compress_checkpoint_host(excp_handle h, const excp_params* params, size_t num_tensors,
+                                          const float* const* w_t, const float* const* w_prev,
+                                          const float* const* ea, const float* const* eas,
+                                          const size_t* numel, void* blob_out, size_t blob_capacity,
+                                          size_t* tensor_offsets_out, excp_tensor_stats* stats_out,
+                                          void* cuda_stream) {
+    if (!h || !params || !tensor_offsets_out || !blob_out) return EXCP_ERR_INVALID_ARG;
+    if (num_tensors && (!w_t || !w_prev || !ea || !eas || !numel)) return EXCP_ERR_INVALID_ARG;
+    const excp_status ps = validate_params(params);
+    if (ps != EXCP_OK) return ps;
+    for (size_t i = 0; i < num_tensors; ++i)
+        if (numel[i] && (!w_t[i] || !w_prev[i] || !ea[i] || !eas[i])) return EXCP_ERR_INVALID_ARG;
+    tensor_offsets_out[0] = 0;
+    if (num_tensors == 0) return EXCP_OK;
+
+    std::vector<Group> groups;
+    if (!make_groups(h, numel, num_tensors, groups)) return EXCP_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return EXCP_ERR_CUDA;
+    if (!ensure_call_arrays(h, num_tensors) || !ensure_host_path(h)) return EXCP_ERR_CUDA;
+
+    TensorDesc* hd = static_cast<TensorDesc*>(h->h_desc);
+    for (size_t gi = 0; gi < groups.size(); ++gi) {
+        const Group& g = groups[gi];
+        const int slot = (int)(gi & 1);
+        u32 tile = 0;
+        for (size_t i = g.first; i < g.first + g.count; ++i) {
+            TensorDesc& d = hd[i];
+            const size_t off = (size_t)tile * TILE;
+            d.w_t = h->stage[slot][0] + off; d.w_prev = h->stage[slot][1] + off;
+            d.ea = h->stage[slot][2] + off; d.eas = h->stage[slot][3] + off;
+            d.numel = numel[i];
+            d.tensor_index = i;
+            d.tile_begin = tile;
+            d.num_tiles = (u32)((numel[i] + TILE - 1) / TILE);
+            tile += d.num_tiles;
         }
     }
-    return status_from_flags(h->h_call->flags);
+    const Params p = to_params(params);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    LaunchCfg cfg{h->sms, stream, &h->prof};
+    h->prof.begin(stream);
+    TensorDesc* dd = static_cast<TensorDesc*>(h->d_desc);
+    bool ok = check(h, cudaMemsetAsync(h->d_call, 0, sizeof(CallState), stream));
+    ok = ok && check(h, cudaMemcpyAsync(dd, hd, num_tensors * sizeof(TensorDesc), cudaMemcpyHostToDevice, stream));
+
+    // copies of group g into its slot; the slot is free once group g-2 has been computed
+    auto issue_h2d = [&](size_t gi) {
+        const Group& g = groups[gi];
+        const int slot = (int)(gi & 1);
+        bool k = true;
+        if (gi >= 2) k = check(h, cudaStreamWaitEvent(h->s_h2d, h->ev_compute[slot], 0));
+        const float* const* src[4] = {w_t, w_prev, ea, eas};
+        for (size_t i = g.first; k && i < g.first + g.count; ++i) {
+            if (!numel[i]) continue;
+            const size_t off = (size_t)hd[i].tile_begin * TILE;
+            for (int j = 0; k && j < 4; ++j)
+                k = check(h, cudaMemcpyAsync(h->stage[slot][j] + off, src[j][i], numel[i] * sizeof(float),
+                                             cudaMemcpyHostToDevice, h->s_h2d));
+        }
+        return k && check(h, cudaEventRecord(h->ev_h2d[slot], h->s_h2d));
+    };
+
+    size_t host_off = 0;
+    u32 flags = 0;
+    ok = ok && issue_h2d(0);
+    for (size_t gi = 0; ok && gi < groups.size(); ++gi) {
+        const Group& g = groups[gi];
+        const int slot = (int)(gi & 1);
+        if (gi + 1 < groups.size()) ok = issue_h2d(gi + 1);
+        ok = ok && check(h, cudaStreamWaitEvent(stream, h->ev_h2d[slot], 0));
+        if (gi >= 2) ok = ok && check(h, cudaStreamWaitEvent(stream, h->ev_d2h[slot], 0));
+        ok = ok && check(h, cudaMemsetAsync(&h->d_call->blob_cursor, 0, sizeof(u64), stream));
+        ok = ok && run_group(h, cfg, dd + g.first, (int)g.count, g.tiles, p, h->stage_blob[slot],
+                             h->stage_blob_bytes, h->d_results + g.first);
+        ok = ok && check(h, cudaMemcpyAsync(h->h_results + g.first, h->d_results + g.first,
+                                            g.count * sizeof(TensorResult), cudaMemcpyDeviceToHost, stream));
+        ok = ok && check(h, cudaMemcpyAsync(h->h_call, h->d_call, sizeof(CallState), cudaMemcpyDeviceToHost, stream));
+        ok = ok && check(h, cudaEventRecord(h->ev_compute[slot], stream));
+        ok = ok && check(h, cudaEventSynchronize(h->ev_compute[slot]));
+        if (!ok) break;
+        const size_t bytes = (size_t)h->h_call->blob_cursor;
+        flags |= h->h_call->flags;
+        if (host_off + bytes > blob_capacity) { flags |= FLAG_BLOB_FULL; break; }
+        ok = check(h, cudaStreamWaitEvent(h->s_d2h, h->ev_compute[slot], 0));
+        ok = ok && check(h, cudaMemcpyAsync(static_cast<unsigned char*>(blob_out) + host_off, h->stage_blob[slot],
+                                            bytes, cudaMemcpyDeviceToHost, h->s_d2h));
+        ok = ok && check(h, cudaEventRecord(h->ev_d2h[slot], h->s_d2h));
+        fill_outputs(h, g.first, g.count, numel, host_off, tensor_offsets_out, stats_out);
+        host_off += bytes;
+    }
+    const bool s1 = check(h, cudaStreamSynchronize(h->s_h2d));
+    const bool s2 = check(h, cudaStreamSynchronize(h->s_d2h));
+    const bool s3 = check(h, cudaStreamSynchronize(stream));
+    if (!ok || !s1 || !s2 || !s3) return EXCP_ERR_CUDA;
+    h->prof.finish();
+    return status_from_flags(flags);
 }
 
 excp_status excp_compress_tensor(excp_handle h, const excp_params* params,
@@ -320,7 +510,8 @@ excp_status excp_decompress_checkpoint(excp_handle h, const void* blob, const si
         }
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    LaunchCfg cfg{h->sms, stream};
+    LaunchCfg cfg{h->sms, stream, &h->prof};
+    h->prof.begin(stream);
     DecDesc* dd = static_cast<DecDesc*>(h->d_desc);
     bool ok = check(h, cudaMemsetAsync(h->d_call, 0, sizeof(CallState), stream));
     ok = ok && check(h, cudaMemcpyAsync(dd, hd, num_tensors * sizeof(DecDesc), cudaMemcpyHostToDevice, stream));
@@ -331,7 +522,37 @@ excp_status excp_decompress_checkpoint(excp_handle h, const void* blob, const si
     }
     ok = ok && check(h, cudaMemcpyAsync(h->h_call, h->d_call, sizeof(CallState), cudaMemcpyDeviceToHost, stream));
     if (!check(h, cudaStreamSynchronize(stream)) || !ok) return EXCP_ERR_CUDA;
+    h->prof.finish();
     return status_from_flags(h->h_call->flags);
+}
+
+excp_status excp_profile_enable(excp_handle h, int enable) {
+    if (!h) return EXCP_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (enable && h->prof.ev.empty()) {
+        h->prof.ev.resize(8192);
+        h->prof.stage.assign(8192, 0);
+        for (cudaEvent_t& e : h->prof.ev)
+            if (!check(h, cudaEventCreate(&e))) return EXCP_ERR_CUDA;
+    }
+    h->prof.enabled = enable != 0;
+    return EXCP_OK;
+}
+
+int excp_profile_stage_count(void) { return ST_COUNT; }
+
+const char* excp_profile_stage_name(int stage) {
+    static const char* names[ST_COUNT] = {
+        "stats1", "stats2", "mask_compact", "scan_layout", "kmeans_start", "lloyd_dw", "lloyd_ea",
+        "lloyd_eas", "kmeans_update", "header_edges", "pack_codes", "copy_bitmaps", "dec_prep", "decode"};
+    return stage >= 0 && stage < ST_COUNT ? names[stage] : "";
+}
+
+excp_status excp_profile_read(excp_handle h, double* stage_ms_out, unsigned long long* launches_out) {
+    if (!h) return EXCP_ERR_INVALID_ARG;
+    if (stage_ms_out) for (int i = 0; i < ST_COUNT; ++i) stage_ms_out[i] = h->prof.ms[i];
+    if (launches_out) *launches_out = h->prof.launches;
+    return EXCP_OK;
 }
 
 excp_status excp_decompress_tensor(excp_handle h, const void* blob, size_t blob_bytes,

@@ -221,10 +221,21 @@ __device__ inline void scan_tile_counts(u32 tb, u32 ntl, const Workspace& ws, u3
 #endif
 
 // ---- launch wrappers --------------------------------------------------------
+enum Stage {                       // for the optional per-stage event timing
+    ST_STATS1 = 0, ST_STATS2, ST_MASK_COMPACT, ST_SCAN_LAYOUT, ST_KMEANS_START, ST_LLOYD_W, ST_LLOYD_EA,
+    ST_LLOYD_EAS, ST_KMEANS_UPDATE, ST_HEADER_EDGES, ST_PACK_CODES, ST_COPY_BITMAPS, ST_DEC_PREP,
+    ST_DECODE, ST_COUNT
+};
+
+struct Profiler;
 struct LaunchCfg {
     int sms;
     cudaStream_t stream;
+    Profiler* prof;
 };
+// Counts `launches` kernel launches; with timing enabled also records an event
+// that closes stage `stage` (implemented beside the handle).
+void prof_mark(const LaunchCfg& cfg, int stage, int launches);
 
 void launch_stats(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                   const Workspace& ws, const Params& p);

@@ -188,13 +188,18 @@ __global__ void __launch_bounds__(96) kmeans_update_kernel(TensorState* __restri
 void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                    const Workspace& ws, const Params& p) {
     kmeans_start_kernel<<<dim3(nt, 3), SAMPLE_MAX, 0, cfg.stream>>>(descs, st, ws, p.seed);
+    prof_mark(cfg, ST_KMEANS_START, 1);
     if (!tiles) return;
     const u32 grid = min(tiles, (u32)cfg.sms * 4u);
     for (int it = 0; it < p.kmeans_iters; ++it) {
         lloyd_pass_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws.surv[0], ws.tile_cnt_w, 0);
+        prof_mark(cfg, ST_LLOYD_W, 1);
         lloyd_pass_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws.surv[1], ws.tile_cnt_o, 1);
+        prof_mark(cfg, ST_LLOYD_EA, 1);
         lloyd_pass_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws.surv[2], ws.tile_cnt_o, 2);
+        prof_mark(cfg, ST_LLOYD_EAS, 1);
         kmeans_update_kernel<<<nt, 96, 0, cfg.stream>>>(st);
+        prof_mark(cfg, ST_KMEANS_UPDATE, 1);
     }
 }
 

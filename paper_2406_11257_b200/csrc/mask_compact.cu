@@ -207,9 +207,11 @@ void launch_mask_compact(const LaunchCfg& cfg, const TensorDesc* descs, TensorSt
     if (tiles) {
         const u32 grid = min(tiles, (u32)cfg.sms * 4u);
         mask_compact_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, call);
+        prof_mark(cfg, ST_MASK_COMPACT, 1);
     }
     tile_scan_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, ws);
     layout_kernel<<<1, MAX_GROUP_TENSORS, 0, cfg.stream>>>(descs, st, nt, p.bits, call, blob_capacity);
+    prof_mark(cfg, ST_SCAN_LAYOUT, 2);
 }
 
 }  // namespace excp

@@ -181,8 +181,9 @@ void launch_pack(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st,
                  const Workspace& ws, const Params& p, unsigned char* blob, CallState* call,
                  TensorResult* results) {
     header_kernel<<<nt, 64, 0, cfg.stream>>>(descs, st, blob, call, results);
-    if (!tiles) return;
+    if (!tiles) { prof_mark(cfg, ST_HEADER_EDGES, 1); return; }
     clear_edges_kernel<<<(tiles + TPB - 1) / TPB, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, blob, call);
+    prof_mark(cfg, ST_HEADER_EDGES, 2);
     const u32 grid = min(tiles, (u32)cfg.sms * 8u);
     pack_codes_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws.surv[0], ws.tile_cnt_w,
                                                      ws.tile_off_w, 0, blob, call);
@@ -190,9 +191,11 @@ void launch_pack(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st,
                                                      ws.tile_off_o, 1, blob, call);
     pack_codes_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws.surv[2], ws.tile_cnt_o,
                                                      ws.tile_off_o, 2, blob, call);
+    prof_mark(cfg, ST_PACK_CODES, 3);
     const u64 quads = (u64)tiles * (TILE_WORDS / 4);
     copy_bitmaps_kernel<<<(u32)((quads + TPB - 1) / TPB), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws,
                                                                                blob, call);
+    prof_mark(cfg, ST_COPY_BITMAPS, 1);
 }
 
 }  // namespace excp

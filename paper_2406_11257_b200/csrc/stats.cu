@@ -331,11 +331,13 @@ void launch_stats(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st
         stats1_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, resid);
     }
     stats1_finish_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st);
+    prof_mark(cfg, ST_STATS1, tiles ? 2 : 1);
     if (tiles) {
         const u32 grid = min(tiles, (u32)cfg.sms * 8u);
         stats2_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, resid);
     }
     stats2_finish_kernel<<<nt, 1024, 0, cfg.stream>>>(descs, st, ws, p.alpha, p.beta);
+    prof_mark(cfg, ST_STATS2, tiles ? 2 : 1);
 }
 
 }  // namespace excp

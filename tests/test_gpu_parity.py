@@ -303,3 +303,39 @@ def test_corrupt_records_are_refused_without_faulting(handle):
         handle.decompress_tensor(blob, nbytes - 16, dq[1], *outs)
     assert e.value.status == -5
     handle.decompress_tensor(blob, nbytes, dq[1], *outs)     # the intact record still decodes
+
+
+# ----------------------------------------------------------------- host path
+def test_host_buffer_path_gives_the_same_records(handle):
+    sizes = [5000, 0, 70000, 1, 4096, 130000, 33, 8192, 99999, 64000]
+    quads = [rand_quad_np(n, 1000 + i) for i, n in enumerate(sizes)]
+    dquads = to_dev(quads)
+    p = binding.Params(median_source=binding.MEDIAN_ABS_RESIDUAL, seed=8)
+    blob, offs, stats = gpu_compress(handle, p, dquads)
+    small = binding.Handle(workspace_numel=140_000)          # several groups: both staging slots reused
+    try:
+        hquads = [tuple(torch.as_tensor(a).pin_memory() for a in q) for q in quads]
+        hblob = torch.full((offs[-1] + 64,), 0xCD, dtype=torch.uint8).pin_memory()
+        for _ in range(2):
+            hoffs, hstats = small.compress_checkpoint_host(p, hquads, hblob)
+            assert hoffs == offs
+            assert bytes(hblob[:offs[-1]].numpy()) == blob[:offs[-1]].cpu().numpy().tobytes()
+            assert [s.nnz_w for s in hstats] == [s.nnz_w for s in stats]
+        with pytest.raises(binding.ExcpError) as e:
+            small.compress_checkpoint_host(p, hquads, hblob[:offs[-1] - 16])
+        assert e.value.status == -3
+    finally:
+        small.close()
+
+
+def test_profile_counts_launches_and_times_stages(handle):
+    dq = [synth.make_quad(200_000, 3, 0, device=DEV)]
+    blob = torch.empty(binding.compress_bound(200_000), dtype=torch.uint8, device=DEV)
+    handle.profile_enable(True)
+    try:
+        handle.compress_tensor(binding.Params(median_source=1, kmeans_iters=10), *dq[0], blob)
+        ms, launches = handle.profile_read()
+        assert launches == 4 + 1 + 2 + 1 + 10 * 4 + 2 + 3 + 1
+        assert ms["mask_compact"] > 0 and ms["lloyd_dw"] > 0 and ms["decode"] == 0
+    finally:
+        handle.profile_enable(False)
