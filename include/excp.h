@@ -68,7 +68,7 @@ typedef enum {
     EXCP_ERR_CUDA = -4,             /* a CUDA runtime call failed; see excp_last_cuda_error */
     EXCP_ERR_CORRUPT_BLOB = -5,     /* decompress: header, sizes, bitmap population or a code is inconsistent */
     EXCP_ERR_NONFINITE_INPUT = -6,  /* compress: NaN or infinity in an input, or a negative second moment */
-    EXCP_ERR_TIMEOUT = -7           /* reserved: no kernel of this library waits on another */
+    EXCP_ERR_TIMEOUT = -7           /* a bounded wait on an asynchronous copy ran out (no kernel waits on another kernel) */
 } excp_status;
 
 typedef enum {

@@ -162,7 +162,7 @@ bool run_group(excp_handle h, const LaunchCfg& cfg, const TensorDesc* descs, int
     if (!check(h, cudaMemsetAsync(h->d_state, 0, nt * sizeof(TensorState), cfg.stream))) return false;
     launch_stats(cfg, descs, h->d_state, nt, tiles, h->ws, p);
     launch_mask_compact(cfg, descs, h->d_state, nt, tiles, h->ws, p, h->d_call, blob_capacity);
-    launch_kmeans(cfg, descs, h->d_state, nt, tiles, h->ws, p);
+    launch_kmeans(cfg, descs, h->d_state, nt, tiles, h->ws, p, h->d_call);
     launch_pack(cfg, descs, h->d_state, nt, tiles, h->ws, p, blob, h->d_call, results);
     return check(h, cudaGetLastError());
 }
@@ -200,6 +200,7 @@ bool ensure_host_path(excp_handle h) {
 }
 
 excp_status status_from_flags(u32 flags) {
+    if (flags & FLAG_TIMEOUT) return EXCP_ERR_TIMEOUT;
     if (flags & FLAG_INTERNAL) return EXCP_ERR_CUDA;
     if (flags & FLAG_NONFINITE) return EXCP_ERR_NONFINITE_INPUT;
     if (flags & FLAG_CORRUPT) return EXCP_ERR_CORRUPT_BLOB;

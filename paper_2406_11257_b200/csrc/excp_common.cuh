@@ -31,6 +31,7 @@ constexpr u32 FLAG_NONFINITE = 1u;               // NaN/Inf input or negative se
 constexpr u32 FLAG_BLOB_FULL = 2u;               // records do not fit blob_capacity
 constexpr u32 FLAG_CORRUPT = 4u;                 // decompress: inconsistent record
 constexpr u32 FLAG_INTERNAL = 8u;                // a self-check failed (candidate count mismatch)
+constexpr u32 FLAG_TIMEOUT = 16u;                // a bounded wait on an asynchronous copy ran out
 
 constexpr u32 MAGIC = 0x50435845u;
 constexpr u32 VERSION = 1u;
@@ -242,7 +243,7 @@ void launch_stats(const LaunchCfg&, const TensorDesc* descs, TensorState* st, in
 void launch_mask_compact(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                          const Workspace& ws, const Params& p, CallState* call, u64 blob_capacity);
 void launch_kmeans(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
-                   const Workspace& ws, const Params& p);
+                   const Workspace& ws, const Params& p, CallState* call);
 void launch_pack(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                  const Workspace& ws, const Params& p, unsigned char* blob, CallState* call,
                  TensorResult* results);

@@ -12,6 +12,7 @@
 //   update   mean = fp32(fp64(sum)/fp64(count) * 2^(E-30)); empty clusters keep
 //            their centre; centres re-sorted; new thresholds
 #include "excp_common.cuh"
+#include "tma.cuh"
 
 namespace excp {
 
@@ -82,76 +83,155 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
 }
 
 // One Lloyd sweep of one stream over every tile of the group.
-__global__ void __launch_bounds__(TPB) lloyd_pass_kernel(const TensorDesc* __restrict__ descs,
-                                                         TensorState* __restrict__ st, int nt, u32 tiles,
-                                                         const float* __restrict__ surv,
-                                                         const u32* __restrict__ tile_cnt, int stream) {
-    __shared__ u64 acc[KPAD][TPB];       // [cluster][thread]: bank = thread, conflict free
-    __shared__ float thr[KPAD];
-    __shared__ s64 red_sum[8][KPAD];
-    __shared__ u32 red_cnt[8][KPAD];
+//
+// Every warp works alone on a contiguous run of tiles: lane 0 streams the tiles'
+// survivor segments into the warp's own ring of shared-memory stages with bulk
+// asynchronous copies (512 values per copy, four in flight), the warp consumes
+// them as float4, and nothing in the sweep synchronises the block.
+constexpr int LCH = 512;             // values per staged chunk
+constexpr int LST = 4;               // stages per warp
+constexpr int LWARPS = TPB / 32;
+
+struct LloydSmem {
+    float buf[LWARPS][LST][LCH];
+    u64 acc[KMAX][TPB];              // [cluster][thread]: a private cell per thread, bank = thread
+    u64 bar[LWARPS][LST];
+    float thr[LWARPS][KPAD];         // each warp's copy of its tensor's thresholds
+};
+
+__global__ void __launch_bounds__(TPB, 2) lloyd_pass_kernel(const TensorDesc* __restrict__ descs,
+                                                            TensorState* __restrict__ st, int nt, u32 tiles,
+                                                            const float* __restrict__ surv,
+                                                            const u32* __restrict__ tile_cnt, int stream,
+                                                            CallState* call) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    LloydSmem& sm = *reinterpret_cast<LloydSmem*>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 #pragma unroll
-    for (int j = 0; j < KPAD; ++j) acc[j][tid] = 0;
-    u32 lo, hi;
-    block_range(tiles, lo, hi);
-    int cur = -1;
-    u32 tb = 0, ntl = 0;
-    float s1 = 0.f, s2 = 0.f;
-    int since = 0;
+    for (int j = 0; j < KMAX; ++j) sm.acc[j][tid] = 0;
+    if (lane == 0) {
+        for (int s = 0; s < LST; ++s) mbar_init(&sm.bar[warp][s], 1);
+        mbar_fence_init();
+    }
+    __syncwarp();
 
-    auto flush = [&](int t) {
-        // per-thread cells -> block totals -> one integer atomic per cluster
+    const u32 gw = blockIdx.x * LWARPS + warp, nw = gridDim.x * LWARPS;
+    const u32 wlo = (u32)(((u64)tiles * gw) / nw), whi = (u32)(((u64)tiles * (gw + 1)) / nw);
+    u32 g_issue = 0, g_cons = 0;     // chunks issued / consumed so far: stage = g % LST, phase = (g / LST) & 1
+    int cur = -1;
+    u32 tb = 0, ntl = 0, since = 0;
+    float t3 = 0.f, t7 = 0.f, t11 = 0.f;
+    float s1 = 0.f, s2 = 0.f;
+    const char* const thr_row = reinterpret_cast<const char*>(sm.thr[warp]);
+    char* const cell0 = reinterpret_cast<char*>(&sm.acc[0][tid]);
+
+    auto flush = [&](int tns) {      // this warp's cells -> one integer atomic per cluster
 #pragma unroll
         for (int j = 0; j < KMAX; ++j) {
-            const s64 v = (s64)acc[j][tid];
-            acc[j][tid] = 0;
+            const s64 v = (s64)sm.acc[j][tid];
+            sm.acc[j][tid] = 0;
             s64 c = (v + (1ll << 47)) >> 48;          // count sits above a 48-bit signed sum
-            s64 sm = v - (c << 48);
+            s64 q = v - (c << 48);
 #pragma unroll
             for (int o = 16; o; o >>= 1) {
                 c += __shfl_xor_sync(0xffffffffu, c, o);
-                sm += __shfl_xor_sync(0xffffffffu, sm, o);
+                q += __shfl_xor_sync(0xffffffffu, q, o);
             }
-            if (lane == 0) { red_sum[warp][j] = sm; red_cnt[warp][j] = (u32)c; }
-        }
-        __syncthreads();
-        if (tid < KMAX) {
-            s64 sm = 0; u64 c = 0;
-#pragma unroll
-            for (int w = 0; w < 8; ++w) { sm += red_sum[w][tid]; c += red_cnt[w][tid]; }
-            if (c) {
-                atomicAdd(reinterpret_cast<u64*>(&st[t].s[stream].acc_sum[tid]), (u64)sm);
-                atomicAdd(&st[t].s[stream].acc_cnt[tid], c);
+            if (lane == 0 && c) {
+                atomicAdd(reinterpret_cast<u64*>(&st[tns].s[stream].acc_sum[j]), (u64)q);
+                atomicAdd(&st[tns].s[stream].acc_cnt[j], (u64)c);
             }
         }
-        __syncthreads();
         since = 0;
     };
 
-    for (u32 tile = lo; tile < hi; ++tile) {
-        if (cur < 0 || tile >= tb + ntl) {
-            if (cur >= 0) flush(cur);
-            cur = find_tensor(descs, nt, tile);
-            tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
-            const StreamState& s = st[cur].s[stream];
-            __syncthreads();
-            if (tid < KPAD) thr[tid] = s.thr[tid];
-            s1 = s.scale1; s2 = s.scale2;
-            __syncthreads();
+    for (u32 w0 = wlo; w0 < whi; w0 += 32) {
+        const u32 wn = min(32u, whi - w0);
+        const u32 mycnt = (u32)lane < wn ? tile_cnt[w0 + lane] : 0u;
+        u32 it = 0, ic = 0;          // issue cursor: tile within the window, value offset in its segment
+        u32 ct = 0, cc = 0;          // consume cursor
+        while (it < wn && __shfl_sync(0xffffffffu, mycnt, it) == 0) ++it;
+        while (ct < wn && __shfl_sync(0xffffffffu, mycnt, ct) == 0) ++ct;
+        while (ct < wn) {
+            while (it < wn && g_issue - g_cons < (u32)LST) {
+                const u32 c = __shfl_sync(0xffffffffu, mycnt, it);
+                const u32 nel = min((u32)LCH, c - ic);
+                if (lane == 0) {
+                    const u32 bytes = ((nel + 3u) & ~3u) * 4u;
+                    u64* bar = &sm.bar[warp][g_issue % LST];
+                    mbar_arrive_expect_tx(bar, bytes);
+                    bulk_g2s(sm.buf[warp][g_issue % LST], surv + (u64)(w0 + it) * TILE + ic, bytes, bar);
+                }
+                ++g_issue;
+                ic += LCH;
+                if (ic >= c) {
+                    ic = 0; ++it;
+                    while (it < wn && __shfl_sync(0xffffffffu, mycnt, it) == 0) ++it;
+                }
+            }
+            const u32 tile = w0 + ct;
+            if (cur < 0 || tile >= tb + ntl) {
+                if (cur >= 0) flush(cur);
+                cur = find_tensor(descs, nt, tile);
+                tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
+                const StreamState& ss = st[cur].s[stream];
+                __syncwarp();
+                if (lane < KPAD) sm.thr[warp][lane] = ss.thr[lane];
+                __syncwarp();
+                t3 = sm.thr[warp][3]; t7 = sm.thr[warp][7]; t11 = sm.thr[warp][11];
+                s1 = ss.scale1; s2 = ss.scale2;
+            }
+            const u32 c = __shfl_sync(0xffffffffu, mycnt, ct);
+            const u32 nel = min((u32)LCH, c - cc);
+            const u32 stage = g_cons % LST;
+            if (!mbar_wait_warp(&sm.bar[warp][stage], (g_cons / LST) & 1u)) {
+                if (lane == 0) atomicOr(&call->flags, FLAG_TIMEOUT);
+                return;
+            }
+            const float4* b4 = reinterpret_cast<const float4*>(sm.buf[warp][stage]);
+            // cluster = number of thresholds below x: two levels from registers, two from the
+            // warp's threshold row in shared memory (index kept pre-scaled by 4 bytes)
+            auto find = [&](float x) -> u32 {
+                u32 p = x > t7 ? 32u : 0u;
+                p += (x > (p ? t11 : t3)) ? 16u : 0u;
+                p += (x > *reinterpret_cast<const float*>(thr_row + p + 4)) ? 8u : 0u;
+                p += (x > *reinterpret_cast<const float*>(thr_row + p)) ? 4u : 0u;
+                return p;
+            };
+            auto add = [&](u32 p, float x) {
+                const int q = __float2int_rn(__fmul_rn(__fmul_rn(x, s1), s2));
+                u64* cell = reinterpret_cast<u64*>(cell0 + p * (TPB * 2u));
+                *cell = (u64)((s64)*cell + (s64)q) + (1ull << 48);
+            };
+            if (nel == (u32)LCH) {
+                // all searches of a batch first (they only read), then the read-modify-writes
+#pragma unroll
+                for (int k = 0; k < LCH / 128; k += 2) {
+                    const float4 u4 = b4[lane + 32 * k], v4 = b4[lane + 32 * (k + 1)];
+                    const u32 p0 = find(u4.x), p1 = find(u4.y), p2 = find(u4.z), p3 = find(u4.w);
+                    const u32 p4 = find(v4.x), p5 = find(v4.y), p6 = find(v4.z), p7 = find(v4.w);
+                    add(p0, u4.x); add(p1, u4.y); add(p2, u4.z); add(p3, u4.w);
+                    add(p4, v4.x); add(p5, v4.y); add(p6, v4.z); add(p7, v4.w);
+                }
+            } else {
+                for (u32 f = lane; 4 * f < nel; f += 32) {
+                    const float4 v4 = b4[f];
+                    const u32 p0 = find(v4.x), p1 = find(v4.y), p2 = find(v4.z), p3 = find(v4.w);
+                    add(p0, v4.x);
+                    if (4 * f + 1 < nel) add(p1, v4.y);
+                    if (4 * f + 2 < nel) add(p2, v4.z);
+                    if (4 * f + 3 < nel) add(p3, v4.w);
+                }
+            }
+            __syncwarp();            // every lane is done with the stage before it is refilled
+            ++g_cons;
+            cc += LCH;
+            if (cc >= c) {
+                cc = 0; ++ct;
+                while (ct < wn && __shfl_sync(0xffffffffu, mycnt, ct) == 0) ++ct;
+            }
+            if (++since >= 1024) flush(cur);
         }
-        const u32 cnt = tile_cnt[tile];
-        const float* data = surv + (u64)tile * TILE;
-        for (u32 i = tid; i < cnt; i += TPB) {
-            const float x = data[i];
-            int p = (x > thr[7]) ? 8 : 0;
-            p += (x > thr[p + 3]) ? 4 : 0;
-            p += (x > thr[p + 1]) ? 2 : 0;
-            p += (x > thr[p]) ? 1 : 0;
-            const int q = __float2int_rn(__fmul_rn(__fmul_rn(x, s1), s2));
-            acc[p][tid] += (u64)((s64)q + (1ll << 48));
-        }
-        if (++since >= 1024) flush(cur);
     }
     if (cur >= 0) flush(cur);
 }
@@ -186,17 +266,19 @@ __global__ void __launch_bounds__(96) kmeans_update_kernel(TensorState* __restri
 }
 
 void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
-                   const Workspace& ws, const Params& p) {
+                   const Workspace& ws, const Params& p, CallState* call) {
     kmeans_start_kernel<<<dim3(nt, 3), SAMPLE_MAX, 0, cfg.stream>>>(descs, st, ws, p.seed);
     prof_mark(cfg, ST_KMEANS_START, 1);
     if (!tiles) return;
-    const u32 grid = min(tiles, (u32)cfg.sms * 4u);
+    const u32 grid = min((tiles + LWARPS - 1) / LWARPS, (u32)cfg.sms * 2u);
+    const size_t smem = sizeof(LloydSmem);
+    cudaFuncSetAttribute(lloyd_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     for (int it = 0; it < p.kmeans_iters; ++it) {
-        lloyd_pass_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws.surv[0], ws.tile_cnt_w, 0);
+        lloyd_pass_kernel<<<grid, TPB, smem, cfg.stream>>>(descs, st, nt, tiles, ws.surv[0], ws.tile_cnt_w, 0, call);
         prof_mark(cfg, ST_LLOYD_W, 1);
-        lloyd_pass_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws.surv[1], ws.tile_cnt_o, 1);
+        lloyd_pass_kernel<<<grid, TPB, smem, cfg.stream>>>(descs, st, nt, tiles, ws.surv[1], ws.tile_cnt_o, 1, call);
         prof_mark(cfg, ST_LLOYD_EA, 1);
-        lloyd_pass_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws.surv[2], ws.tile_cnt_o, 2);
+        lloyd_pass_kernel<<<grid, TPB, smem, cfg.stream>>>(descs, st, nt, tiles, ws.surv[2], ws.tile_cnt_o, 2, call);
         prof_mark(cfg, ST_LLOYD_EAS, 1);
         kmeans_update_kernel<<<nt, 96, 0, cfg.stream>>>(st);
         prof_mark(cfg, ST_KMEANS_UPDATE, 1);
