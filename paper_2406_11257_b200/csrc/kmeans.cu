@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
 // asynchronous copies (512 values per copy, four in flight), the warp consumes
 // them as float4, and nothing in the sweep synchronises the block.
 constexpr int LCH = 512;             // values per staged chunk
-constexpr int LST = 4;               // stages per warp
+constexpr int LST = 2;               // stages per warp
 constexpr int LWARPS = TPB / 32;
 
 struct LloydSmem {
@@ -99,7 +99,7 @@ struct LloydSmem {
     float thr[LWARPS][KPAD];         // each warp's copy of its tensor's thresholds
 };
 
-__global__ void __launch_bounds__(TPB, 2) lloyd_pass_kernel(const TensorDesc* __restrict__ descs,
+__global__ void __launch_bounds__(TPB, 3) lloyd_pass_kernel(const TensorDesc* __restrict__ descs,
                                                             TensorState* __restrict__ st, int nt, u32 tiles,
                                                             const float* __restrict__ surv,
                                                             const u32* __restrict__ tile_cnt, int stream,
@@ -270,7 +270,7 @@ void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* s
     kmeans_start_kernel<<<dim3(nt, 3), SAMPLE_MAX, 0, cfg.stream>>>(descs, st, ws, p.seed);
     prof_mark(cfg, ST_KMEANS_START, 1);
     if (!tiles) return;
-    const u32 grid = min((tiles + LWARPS - 1) / LWARPS, (u32)cfg.sms * 2u);
+    const u32 grid = min((tiles + LWARPS - 1) / LWARPS, (u32)cfg.sms * 3u);
     const size_t smem = sizeof(LloydSmem);
     cudaFuncSetAttribute(lloyd_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     for (int it = 0; it < p.kmeans_iters; ++it) {

@@ -8,6 +8,7 @@
 // count beside it.  No block waits for another; the tensor-wide offsets come
 // from a small scan afterwards and are only needed when the codes are packed.
 #include "excp_common.cuh"
+#include "warp_ring.cuh"
 
 namespace excp {
 
@@ -18,21 +19,39 @@ __device__ inline u32 spread8(u32 b) {   // bit i of an 8-bit value -> bit 4 i
     return b;
 }
 
-__global__ void __launch_bounds__(TPB) mask_compact_kernel(const TensorDesc* __restrict__ descs,
-                                                           TensorState* __restrict__ st, int nt,
-                                                           u32 tiles, Workspace ws, CallState* call) {
-    __shared__ u32 cnt_w[2][CHUNKS], cnt_o[2][CHUNKS];
+constexpr int MCH = 256;             // values per stream per staged chunk
+constexpr int MST = 3;               // chunks in flight per warp
+constexpr int MWARPS = TPB / 32;
+
+struct MaskSmem {
+    float buf[MWARPS][MST][4][MCH];
+    unsigned long long bar[MWARPS][MST];
+};
+
+// Every warp owns a contiguous run of tiles and walks it alone: 256-value chunks of the four
+// streams arrive in its ring of stages, a tile's survivor offset is a running count in the
+// warp, and nothing in the sweep synchronises the block.
+__global__ void __launch_bounds__(TPB, 2) mask_compact_kernel(const TensorDesc* __restrict__ descs,
+                                                              TensorState* __restrict__ st, int nt,
+                                                              u32 tiles, Workspace ws, CallState* call) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    MaskSmem& sm = *reinterpret_cast<MaskSmem*>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const u32 lt = (1u << lane) - 1u;
-    u32 lo, hi;
-    block_range(tiles, lo, hi);
-    int cur = -1;
-    u32 tb = 0, ntl = 0;
-    u64 n = 0;
-    const float *w_t = nullptr, *w_prev = nullptr, *ea = nullptr, *eas = nullptr;
+    WarpRing<4, MCH, MST> ring;
+    ring.init(&sm.buf[warp][0][0][0], sm.bar[warp], lane);
+
+    const u32 gw = blockIdx.x * MWARPS + warp, nw = gridDim.x * MWARPS;
+    const u32 wlo = (u32)(((u64)tiles * gw) / nw), whi = (u32)(((u64)tiles * (gw + 1)) / nw);
+    DenseCursor<MCH> ic, cc;
+    ic.start(wlo); cc.start(wlo);
+    const float* ip[4] = {nullptr, nullptr, nullptr, nullptr};      // issue side: the tensor's streams
+    const float* cp[4] = {nullptr, nullptr, nullptr, nullptr};      // consume side
     float thr_w = 0.f, thr_o = 0.f;
+    u32 rw = 0, ro = 0;               // survivors of the current tile so far (warp uniform)
     u32 mk0 = 0, mk1 = 0, mk2 = 0;    // running max |x| patterns of the survivors
     u32 bad = 0;
+    int prev = -1;
 
     auto flush_max = [&](int t) {
         mk0 = __reduce_max_sync(0xffffffffu, mk0);
@@ -46,104 +65,102 @@ __global__ void __launch_bounds__(TPB) mask_compact_kernel(const TensorDesc* __r
         mk0 = mk1 = mk2 = 0;
     };
 
-    int par = 0;
-    for (u32 tile = lo; tile < hi; ++tile, par ^= 1) {
-        if (cur < 0 || tile >= tb + ntl) {
-            if (cur >= 0) flush_max(cur);
-            cur = find_tensor(descs, nt, tile);
-            tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles; n = descs[cur].numel;
-            w_t = descs[cur].w_t; w_prev = descs[cur].w_prev; ea = descs[cur].ea; eas = descs[cur].eas;
-            thr_w = st[cur].thr_w; thr_o = st[cur].thr_o;
+    while (cc.tile < whi) {
+        while (ic.tile < whi && ring.can_issue()) {
+            if (ic.locate(descs, nt)) {
+                ip[0] = descs[ic.tns].w_t; ip[1] = descs[ic.tns].w_prev;
+                ip[2] = descs[ic.tns].ea; ip[3] = descs[ic.tns].eas;
+            }
+            const u64 e0 = ic.elem0();
+            const float* src[4] = {ip[0] + e0, ip[1] + e0, ip[2] + e0, ip[3] + e0};
+            ring.issue(lane, src, ic.valid() & ~3u);
+            ic.next();
         }
-        const u64 base = (u64)(tile - tb) * TILE;
-        float dwv[4 * ROUNDS], eav[4 * ROUNDS], easv[4 * ROUNDS];
-        u32 mw = 0, mo = 0;                 // this thread's 16 mask bits
-        u32 prew[ROUNDS], preo[ROUNDS];     // survivors before this lane within its chunk
-#pragma unroll
-        for (int r = 0; r < ROUNDS; ++r) {
-            const u64 i0 = base + (u64)r * (TPB * 4) + (u64)tid * 4;
-            float a[4], b[4], e[4], v[4];
-            load4(w_t, i0, n, a);
-            load4(w_prev, i0, n, b);
-            load4(ea, i0, n, e);
-            load4(eas, i0, n, v);
-            u32 bw[4], bo[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const u32 vb = __float_as_uint(v[k]);
-                bad |= ((__float_as_uint(a[k]) & 0x7fffffffu) >= 0x7f800000u) |
-                       ((__float_as_uint(b[k]) & 0x7fffffffu) >= 0x7f800000u) |
-                       ((__float_as_uint(e[k]) & 0x7fffffffu) >= 0x7f800000u) |
-                       ((vb & 0x7fffffffu) >= 0x7f800000u) | (vb > 0x80000000u);
-                const float dw = __fsub_rn(a[k], b[k]);
-                const float lhs = __fmul_rn(fabsf(dw), __fsqrt_rn(v[k]));
-                const bool kw = lhs > thr_w;                       // elements past numel: 0 > thr is false
-                const bool ko = kw && (fabsf(e[k]) > thr_o);
-                bw[k] = __ballot_sync(0xffffffffu, kw);
-                bo[k] = __ballot_sync(0xffffffffu, ko);
-                dwv[r * 4 + k] = dw; eav[r * 4 + k] = e[k]; easv[r * 4 + k] = v[k];
-                mw |= (u32)kw << (r * 4 + k);
-                mo |= (u32)ko << (r * 4 + k);
-            }
-            prew[r] = __popc(bw[0] & lt) + __popc(bw[1] & lt) + __popc(bw[2] & lt) + __popc(bw[3] & lt);
-            preo[r] = __popc(bo[0] & lt) + __popc(bo[1] & lt) + __popc(bo[2] & lt) + __popc(bo[3] & lt);
-            const int chunk = r * (TPB / 32) + warp;
-            if (lane < 4) {   // lane j assembles bitmap word j of this 128-element chunk
-                const int sh = 8 * lane;
-                const u32 ww = spread8((bw[0] >> sh) & 0xffu) | (spread8((bw[1] >> sh) & 0xffu) << 1) |
-                               (spread8((bw[2] >> sh) & 0xffu) << 2) | (spread8((bw[3] >> sh) & 0xffu) << 3);
-                const u32 wo = spread8((bo[0] >> sh) & 0xffu) | (spread8((bo[1] >> sh) & 0xffu) << 1) |
-                               (spread8((bo[2] >> sh) & 0xffu) << 2) | (spread8((bo[3] >> sh) & 0xffu) << 3);
-                const u64 wi = (u64)tile * TILE_WORDS + chunk * 4 + lane;
-                ws.bm_w[wi] = ww;
-                ws.bm_o[wi] = wo;
-            }
-            if (lane == 0) {
-                cnt_w[par][chunk] = __popc(bw[0]) + __popc(bw[1]) + __popc(bw[2]) + __popc(bw[3]);
-                cnt_o[par][chunk] = __popc(bo[0]) + __popc(bo[1]) + __popc(bo[2]) + __popc(bo[3]);
-            }
+        if (cc.locate(descs, nt)) {
+            if (prev >= 0) flush_max(prev);
+            prev = cc.tns;
+            cp[0] = descs[cc.tns].w_t; cp[1] = descs[cc.tns].w_prev;
+            cp[2] = descs[cc.tns].ea; cp[3] = descs[cc.tns].eas;
+            thr_w = st[cc.tns].thr_w; thr_o = st[cc.tns].thr_o;
         }
-        __syncthreads();
-        if (warp == 0) {      // exclusive prefix over the 32 chunks, in element order
-            u32 cw = cnt_w[par][lane], co = cnt_o[par][lane];
-            u32 iw = cw, io = co;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                u32 x = __shfl_up_sync(0xffffffffu, iw, o);
-                u32 y = __shfl_up_sync(0xffffffffu, io, o);
-                if (lane >= o) { iw += x; io += y; }
-            }
-            cnt_w[par][lane] = iw - cw;
-            cnt_o[par][lane] = io - co;
-            if (lane == 31) { ws.tile_cnt_w[tile] = iw; ws.tile_cnt_o[tile] = io; }
+        const u32 valid = cc.valid(), nbulk = valid & ~3u;
+        const u64 e0 = cc.elem0();
+        if (!ring.wait()) {
+            if (lane == 0) atomicOr(&call->flags, FLAG_TIMEOUT);
+            return;
         }
-        __syncthreads();
-        float* sw = ws.surv[0] + (u64)tile * TILE;
-        float* sea = ws.surv[1] + (u64)tile * TILE;
-        float* seas = ws.surv[2] + (u64)tile * TILE;
+        if (cc.chunk == 0) { rw = 0; ro = 0; }
+        const float* stg = ring.stage();
+        float* sw = ws.surv[0] + (u64)cc.tile * TILE;
+        float* sea = ws.surv[1] + (u64)cc.tile * TILE;
+        float* seas = ws.surv[2] + (u64)cc.tile * TILE;
 #pragma unroll
-        for (int r = 0; r < ROUNDS; ++r) {
-            const int chunk = r * (TPB / 32) + warp;
-            u32 pw = cnt_w[par][chunk] + prew[r];
-            u32 po = cnt_o[par][chunk] + preo[r];
+        for (int step = 0; step < MCH / 128; ++step) {
+            if ((u32)step * 128u < valid) {
+                const u32 o = step * 128 + lane * 4;
+                float a[4], b[4], e[4], v[4];
+                fetch4(stg, cp[0] + e0, o, nbulk, valid, a);
+                fetch4(stg + MCH, cp[1] + e0, o, nbulk, valid, b);
+                fetch4(stg + 2 * MCH, cp[2] + e0, o, nbulk, valid, e);
+                fetch4(stg + 3 * MCH, cp[3] + e0, o, nbulk, valid, v);
+                u32 bw[4], bo[4];
+                float dwv[4];
+                u32 mw = 0, mo = 0;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int j = r * 4 + k;
-                if ((mw >> j) & 1u) {
-                    sw[pw++] = dwv[j];
-                    mk0 = max(mk0, __float_as_uint(dwv[j]) & 0x7fffffffu);
+                for (int k = 0; k < 4; ++k) {
+                    const u32 vb = __float_as_uint(v[k]);
+                    bad |= ((__float_as_uint(a[k]) & 0x7fffffffu) >= 0x7f800000u) |
+                           ((__float_as_uint(b[k]) & 0x7fffffffu) >= 0x7f800000u) |
+                           ((__float_as_uint(e[k]) & 0x7fffffffu) >= 0x7f800000u) |
+                           ((vb & 0x7fffffffu) >= 0x7f800000u) | (vb > 0x80000000u);
+                    const float dw = __fsub_rn(a[k], b[k]);                      // Eq. (ckpt_res)
+                    const float lhs = __fmul_rn(fabsf(dw), __fsqrt_rn(v[k]));
+                    const bool kw = lhs > thr_w;                                 // Eq. (rw); past numel: 0 > thr is false
+                    const bool ko = kw && (fabsf(e[k]) > thr_o);                 // Eq. (ro)
+                    bw[k] = __ballot_sync(0xffffffffu, kw);
+                    bo[k] = __ballot_sync(0xffffffffu, ko);
+                    dwv[k] = dw;
+                    mw |= (u32)kw << k;
+                    mo |= (u32)ko << k;
                 }
-                if ((mo >> j) & 1u) {
-                    sea[po] = eav[j];
-                    seas[po] = easv[j];
-                    ++po;
-                    mk1 = max(mk1, __float_as_uint(eav[j]) & 0x7fffffffu);
-                    mk2 = max(mk2, __float_as_uint(easv[j]) & 0x7fffffffu);
+                if (lane < 4) {   // lane j assembles bitmap word j of these 128 values
+                    const int sh = 8 * lane;
+                    const u32 ww = spread8((bw[0] >> sh) & 0xffu) | (spread8((bw[1] >> sh) & 0xffu) << 1) |
+                                   (spread8((bw[2] >> sh) & 0xffu) << 2) | (spread8((bw[3] >> sh) & 0xffu) << 3);
+                    const u32 wo = spread8((bo[0] >> sh) & 0xffu) | (spread8((bo[1] >> sh) & 0xffu) << 1) |
+                                   (spread8((bo[2] >> sh) & 0xffu) << 2) | (spread8((bo[3] >> sh) & 0xffu) << 3);
+                    const u64 wi = (u64)cc.tile * TILE_WORDS + cc.chunk * (MCH / 32) + step * 4 + lane;
+                    ws.bm_w[wi] = ww;
+                    ws.bm_o[wi] = wo;
+                }
+                u32 pw = rw + __popc(bw[0] & lt) + __popc(bw[1] & lt) + __popc(bw[2] & lt) + __popc(bw[3] & lt);
+                u32 po = ro + __popc(bo[0] & lt) + __popc(bo[1] & lt) + __popc(bo[2] & lt) + __popc(bo[3] & lt);
+                rw += __popc(bw[0]) + __popc(bw[1]) + __popc(bw[2]) + __popc(bw[3]);
+                ro += __popc(bo[0]) + __popc(bo[1]) + __popc(bo[2]) + __popc(bo[3]);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    if ((mw >> k) & 1u) {
+                        sw[pw++] = dwv[k];
+                        mk0 = max(mk0, __float_as_uint(dwv[k]) & 0x7fffffffu);
+                    }
+                    if ((mo >> k) & 1u) {
+                        sea[po] = e[k];
+                        seas[po] = v[k];
+                        ++po;
+                        mk1 = max(mk1, __float_as_uint(e[k]) & 0x7fffffffu);
+                        mk2 = max(mk2, __float_as_uint(v[k]) & 0x7fffffffu);
+                    }
                 }
             }
         }
+        ring.release();
+        if (cc.chunk == DenseCursor<MCH>::CHUNKS_PER_TILE - 1 && lane == 0) {
+            ws.tile_cnt_w[cc.tile] = rw;
+            ws.tile_cnt_o[cc.tile] = ro;
+        }
+        cc.next();
     }
-    if (cur >= 0) flush_max(cur);
+    if (prev >= 0) flush_max(prev);
     if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(&call->flags, FLAG_NONFINITE);
 }
 
@@ -205,8 +222,9 @@ __global__ void __launch_bounds__(MAX_GROUP_TENSORS) layout_kernel(const TensorD
 void launch_mask_compact(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                          const Workspace& ws, const Params& p, CallState* call, u64 blob_capacity) {
     if (tiles) {
-        const u32 grid = min(tiles, (u32)cfg.sms * 4u);
-        mask_compact_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, call);
+        const u32 grid = min((tiles + MWARPS - 1) / MWARPS, (u32)cfg.sms * 2u);
+        cudaFuncSetAttribute(mask_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(MaskSmem));
+        mask_compact_kernel<<<grid, TPB, sizeof(MaskSmem), cfg.stream>>>(descs, st, nt, tiles, ws, call);
         prof_mark(cfg, ST_MASK_COMPACT, 1);
     }
     tile_scan_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, ws);

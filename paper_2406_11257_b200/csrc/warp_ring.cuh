@@ -1,0 +1,104 @@
+// A warp's private ring of shared-memory stages fed by bulk asynchronous copies,
+// and the cursor with which a warp walks the dense chunks of its run of tiles.
+//
+// The dense sweeps (statistics, mask + compaction, decode) are all built the same
+// way: every warp owns a contiguous run of tiles, lane 0 keeps NS x CH values per
+// stage in flight for the chunks ahead, the warp consumes chunk after chunk, and no
+// warp ever waits for another one.
+#pragma once
+#include "excp_common.cuh"
+#include "tma.cuh"
+
+namespace excp {
+
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+template <int NS, int CH, int ST>
+struct WarpRing {
+    static constexpr int STAGE_FLOATS = NS * CH;
+    float* buf;                    // ST stages of NS streams of CH values
+    unsigned long long* bar;       // one barrier per stage
+    u32 issued, consumed;          // chunks so far: stage = n % ST, phase = (n / ST) & 1
+
+    __device__ void init(float* b, unsigned long long* r, int lane) {
+        buf = b; bar = r; issued = 0; consumed = 0;
+        if (lane == 0) {
+            for (int s = 0; s < ST; ++s) mbar_init(&bar[s], 1);
+            mbar_fence_init();
+        }
+        __syncwarp();
+    }
+    __device__ bool can_issue() const { return issued - consumed < (u32)ST; }
+
+    // Starts the copies of one chunk: `nbulk` values (a multiple of 4, possibly 0) from each
+    // non-null source.  Called by the whole warp; lane 0 talks to the copy engine.
+    __device__ void issue(int lane, const float* const (&src)[NS], u32 nbulk) {
+        if (lane == 0) {
+            unsigned long long* b = &bar[issued % ST];
+            float* dst = buf + (issued % ST) * STAGE_FLOATS;
+            u32 n = 0;
+#pragma unroll
+            for (int k = 0; k < NS; ++k) n += src[k] != nullptr;
+            if (nbulk && n) {
+                mbar_arrive_expect_tx(b, n * nbulk * 4u);
+#pragma unroll
+                for (int k = 0; k < NS; ++k)
+                    if (src[k]) bulk_g2s(dst + k * CH, src[k], nbulk * 4u, b);
+            } else {
+                mbar_arrive(b);
+            }
+        }
+        ++issued;
+    }
+    // Blocks (bounded) until the oldest chunk in flight has landed.
+    __device__ bool wait() { return mbar_wait_warp(&bar[consumed % ST], (consumed / ST) & 1u); }
+    __device__ const float* stage() const { return buf + (consumed % ST) * STAGE_FLOATS; }
+    // Every lane is done reading the stage: it may be refilled.
+    __device__ void release() { __syncwarp(); ++consumed; }
+};
+
+// Position of a warp inside its run of tiles, in chunks of CH values.
+template <int CH>
+struct DenseCursor {
+    static constexpr u32 CHUNKS_PER_TILE = TILE / CH;
+    u32 tile, chunk;
+    int tns;                       // tensor owning `tile` (-1: not looked up yet)
+    u32 tb, ntl;                   // that tensor's tile range
+    u64 numel;
+
+    __device__ void start(u32 t) { tile = t; chunk = 0; tns = -1; tb = 0; ntl = 0; numel = 0; }
+    // Looks the tensor up when the tile has left the current one; true if it changed.
+    template <typename Desc>
+    __device__ bool locate(const Desc* __restrict__ descs, int nt) {
+        if (tns >= 0 && tile < tb + ntl) return false;
+        tns = find_tensor(descs, nt, tile);
+        tb = descs[tns].tile_begin; ntl = descs[tns].num_tiles; numel = descs[tns].numel;
+        return true;
+    }
+    __device__ u64 elem0() const { return (u64)(tile - tb) * TILE + (u64)chunk * CH; }   // within the tensor
+    __device__ u32 valid() const {                                                      // values of this chunk
+        const u64 e0 = elem0();
+        return e0 >= numel ? 0u : (u32)min((u64)CH, numel - e0);
+    }
+    __device__ void next() { if (++chunk == CHUNKS_PER_TILE) { chunk = 0; ++tile; } }
+};
+
+// Four consecutive values at offset o (a multiple of 4) of a chunk: from the stage where the
+// bulk copy brought them, from global memory for the ragged last values of a tensor, 0 past it.
+__device__ __forceinline__ void fetch4(const float* __restrict__ st, const float* __restrict__ g, u32 o,
+                                       u32 nbulk, u32 valid, float out[4]) {
+    if (o + 4 <= nbulk) {
+        const float4 t = *reinterpret_cast<const float4*>(st + o);
+        out[0] = t.x; out[1] = t.y; out[2] = t.z; out[3] = t.w;
+    } else {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const u32 i = o + k;
+            out[k] = i < nbulk ? st[i] : (i < valid ? __ldg(g + i) : 0.f);
+        }
+    }
+}
+
+}  // namespace excp
