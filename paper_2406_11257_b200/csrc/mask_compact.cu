@@ -2,7 +2,7 @@
 //   dW = W_t - W^_(t-1)                                   Eq. (ckpt_res)
 //   M_w = [ |dW| * sqrt(eas) > alpha * median ]           Eq. (rw), product form
 //   M_o = [ |ea| > beta * mean ] and M_w                  Eq. (ro)
-// and, fused with it, the bitmaps (warp ballots re-ordered to element order)
+// and, fused with it, the bitmaps (each warp ballot is one bitmap word)
 // and the compaction of the survivors: each tile's survivors are written, in
 // index order, at the start of the tile's own 4096-element segment, with the
 // count beside it.  No block waits for another; the tensor-wide offsets come
@@ -12,16 +12,10 @@
 
 namespace excp {
 
-__device__ inline u32 spread8(u32 b) {   // bit i of an 8-bit value -> bit 4 i
-    b = (b | (b << 12)) & 0x000F000Fu;
-    b = (b | (b << 6)) & 0x03030303u;
-    b = (b | (b << 3)) & 0x11111111u;
-    return b;
-}
-
-constexpr int MCH = 256;             // values per stream per staged chunk
-constexpr int MST = 3;               // chunks in flight per warp
-constexpr int MWARPS = TPB / 32;
+constexpr int MCH = 512;             // values per stream per staged chunk
+constexpr int MST = 2;               // chunks in flight per warp
+constexpr int MWARPS = 7;            // 7 warps x 16 KB of stages: two blocks per SM
+constexpr int MTPB = MWARPS * 32;
 
 struct MaskSmem {
     float buf[MWARPS][MST][4][MCH];
@@ -31,7 +25,7 @@ struct MaskSmem {
 // Every warp owns a contiguous run of tiles and walks it alone: 256-value chunks of the four
 // streams arrive in its ring of stages, a tile's survivor offset is a running count in the
 // warp, and nothing in the sweep synchronises the block.
-__global__ void __launch_bounds__(TPB, 2) mask_compact_kernel(const TensorDesc* __restrict__ descs,
+__global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc* __restrict__ descs,
                                                               TensorState* __restrict__ st, int nt,
                                                               u32 tiles, Workspace ws, CallState* call) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -43,31 +37,32 @@ __global__ void __launch_bounds__(TPB, 2) mask_compact_kernel(const TensorDesc* 
 
     const u32 gw = blockIdx.x * MWARPS + warp, nw = gridDim.x * MWARPS;
     const u32 wlo = (u32)(((u64)tiles * gw) / nw), whi = (u32)(((u64)tiles * (gw + 1)) / nw);
-    DenseCursor<MCH> ic, cc;
+    TileWalk<MCH> ic, cc;
     ic.start(wlo); cc.start(wlo);
     const float* ip[4] = {nullptr, nullptr, nullptr, nullptr};      // issue side: the tensor's streams
     const float* cp[4] = {nullptr, nullptr, nullptr, nullptr};      // consume side
     float thr_w = 0.f, thr_o = 0.f;
     u32 rw = 0, ro = 0;               // survivors of the current tile so far (warp uniform)
-    u32 mk0 = 0, mk1 = 0, mk2 = 0;    // running max |x| patterns of the survivors
-    u32 bad = 0;
+    float mk0 = 0.f, mk1 = 0.f, mk2 = 0.f;   // running max magnitudes of the survivors
+    float nanacc = 0.f;                      // turns NaN once any input is NaN or infinite
+    float minv = 0.f;                        // goes negative with a negative second moment
     int prev = -1;
 
-    auto flush_max = [&](int t) {
-        mk0 = __reduce_max_sync(0xffffffffu, mk0);
-        mk1 = __reduce_max_sync(0xffffffffu, mk1);
-        mk2 = __reduce_max_sync(0xffffffffu, mk2);
+    auto flush_max = [&](int t) {            // non-negative floats order like their bit patterns
+        const u32 m0 = __reduce_max_sync(0xffffffffu, __float_as_uint(mk0));
+        const u32 m1 = __reduce_max_sync(0xffffffffu, __float_as_uint(mk1));
+        const u32 m2 = __reduce_max_sync(0xffffffffu, __float_as_uint(mk2));
         if (lane == 0) {
-            if (mk0) atomicMax(&st[t].s[0].maxkey, mk0);
-            if (mk1) atomicMax(&st[t].s[1].maxkey, mk1);
-            if (mk2) atomicMax(&st[t].s[2].maxkey, mk2);
+            if (m0) atomicMax(&st[t].s[0].maxkey, m0);
+            if (m1) atomicMax(&st[t].s[1].maxkey, m1);
+            if (m2) atomicMax(&st[t].s[2].maxkey, m2);
         }
-        mk0 = mk1 = mk2 = 0;
+        mk0 = mk1 = mk2 = 0.f;
     };
 
     while (cc.tile < whi) {
         while (ic.tile < whi && ring.can_issue()) {
-            if (ic.locate(descs, nt)) {
+            if (ic.chunk == 0 && ic.enter_tile(descs, nt)) {
                 ip[0] = descs[ic.tns].w_t; ip[1] = descs[ic.tns].w_prev;
                 ip[2] = descs[ic.tns].ea; ip[3] = descs[ic.tns].eas;
             }
@@ -76,7 +71,7 @@ __global__ void __launch_bounds__(TPB, 2) mask_compact_kernel(const TensorDesc* 
             ring.issue(lane, src, ic.valid() & ~3u);
             ic.next();
         }
-        if (cc.locate(descs, nt)) {
+        if (cc.chunk == 0 && cc.enter_tile(descs, nt)) {
             if (prev >= 0) flush_max(prev);
             prev = cc.tns;
             cp[0] = descs[cc.tns].w_t; cp[1] = descs[cc.tns].w_prev;
@@ -94,73 +89,70 @@ __global__ void __launch_bounds__(TPB, 2) mask_compact_kernel(const TensorDesc* 
         float* sw = ws.surv[0] + (u64)cc.tile * TILE;
         float* sea = ws.surv[1] + (u64)cc.tile * TILE;
         float* seas = ws.surv[2] + (u64)cc.tile * TILE;
+        // Lane l takes values l, l+32, l+64, l+96 of each run of 128, so that a ballot IS a
+        // bitmap word and the survivors of one ballot go to consecutive addresses.
 #pragma unroll
         for (int step = 0; step < MCH / 128; ++step) {
             if ((u32)step * 128u < valid) {
-                const u32 o = step * 128 + lane * 4;
-                float a[4], b[4], e[4], v[4];
-                fetch4(stg, cp[0] + e0, o, nbulk, valid, a);
-                fetch4(stg + MCH, cp[1] + e0, o, nbulk, valid, b);
-                fetch4(stg + 2 * MCH, cp[2] + e0, o, nbulk, valid, e);
-                fetch4(stg + 3 * MCH, cp[3] + e0, o, nbulk, valid, v);
                 u32 bw[4], bo[4];
-                float dwv[4];
-                u32 mw = 0, mo = 0;
+                float dwv[4], eav[4], easv[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    const u32 vb = __float_as_uint(v[k]);
-                    bad |= ((__float_as_uint(a[k]) & 0x7fffffffu) >= 0x7f800000u) |
-                           ((__float_as_uint(b[k]) & 0x7fffffffu) >= 0x7f800000u) |
-                           ((__float_as_uint(e[k]) & 0x7fffffffu) >= 0x7f800000u) |
-                           ((vb & 0x7fffffffu) >= 0x7f800000u) | (vb > 0x80000000u);
-                    const float dw = __fsub_rn(a[k], b[k]);                      // Eq. (ckpt_res)
-                    const float lhs = __fmul_rn(fabsf(dw), __fsqrt_rn(v[k]));
+                    const u32 i = step * 128 + k * 32 + lane;
+                    float a, b, e, v;
+                    if (i < nbulk) {
+                        a = stg[i]; b = stg[MCH + i]; e = stg[2 * MCH + i]; v = stg[3 * MCH + i];
+                    } else if (i < valid) {          // ragged last values of a tensor
+                        a = __ldg(cp[0] + e0 + i); b = __ldg(cp[1] + e0 + i);
+                        e = __ldg(cp[2] + e0 + i); v = __ldg(cp[3] + e0 + i);
+                    } else {
+                        a = b = e = v = 0.f;
+                    }
+                    nanacc = __fmaf_rn(a, 0.f, nanacc);       // inf * 0 and NaN * 0 are NaN
+                    nanacc = __fmaf_rn(b, 0.f, nanacc);
+                    nanacc = __fmaf_rn(e, 0.f, nanacc);
+                    nanacc = __fmaf_rn(v, 0.f, nanacc);
+                    minv = fminf(minv, v);
+                    const float dw = __fsub_rn(a, b);                            // Eq. (ckpt_res)
+                    const float lhs = __fmul_rn(fabsf(dw), __fsqrt_rn(v));
                     const bool kw = lhs > thr_w;                                 // Eq. (rw); past numel: 0 > thr is false
-                    const bool ko = kw && (fabsf(e[k]) > thr_o);                 // Eq. (ro)
+                    const bool ko = kw && (fabsf(e) > thr_o);                    // Eq. (ro)
                     bw[k] = __ballot_sync(0xffffffffu, kw);
                     bo[k] = __ballot_sync(0xffffffffu, ko);
-                    dwv[k] = dw;
-                    mw |= (u32)kw << k;
-                    mo |= (u32)ko << k;
+                    dwv[k] = dw; eav[k] = e; easv[k] = v;
                 }
-                if (lane < 4) {   // lane j assembles bitmap word j of these 128 values
-                    const int sh = 8 * lane;
-                    const u32 ww = spread8((bw[0] >> sh) & 0xffu) | (spread8((bw[1] >> sh) & 0xffu) << 1) |
-                                   (spread8((bw[2] >> sh) & 0xffu) << 2) | (spread8((bw[3] >> sh) & 0xffu) << 3);
-                    const u32 wo = spread8((bo[0] >> sh) & 0xffu) | (spread8((bo[1] >> sh) & 0xffu) << 1) |
-                                   (spread8((bo[2] >> sh) & 0xffu) << 2) | (spread8((bo[3] >> sh) & 0xffu) << 3);
+                if (lane < 4) {
                     const u64 wi = (u64)cc.tile * TILE_WORDS + cc.chunk * (MCH / 32) + step * 4 + lane;
-                    ws.bm_w[wi] = ww;
-                    ws.bm_o[wi] = wo;
+                    ws.bm_w[wi] = lane == 0 ? bw[0] : lane == 1 ? bw[1] : lane == 2 ? bw[2] : bw[3];
+                    ws.bm_o[wi] = lane == 0 ? bo[0] : lane == 1 ? bo[1] : lane == 2 ? bo[2] : bo[3];
                 }
-                u32 pw = rw + __popc(bw[0] & lt) + __popc(bw[1] & lt) + __popc(bw[2] & lt) + __popc(bw[3] & lt);
-                u32 po = ro + __popc(bo[0] & lt) + __popc(bo[1] & lt) + __popc(bo[2] & lt) + __popc(bo[3] & lt);
-                rw += __popc(bw[0]) + __popc(bw[1]) + __popc(bw[2]) + __popc(bw[3]);
-                ro += __popc(bo[0]) + __popc(bo[1]) + __popc(bo[2]) + __popc(bo[3]);
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    if ((mw >> k) & 1u) {
-                        sw[pw++] = dwv[k];
-                        mk0 = max(mk0, __float_as_uint(dwv[k]) & 0x7fffffffu);
+                    if ((bw[k] >> lane) & 1u) {
+                        sw[rw + __popc(bw[k] & lt)] = dwv[k];
+                        mk0 = fmaxf(mk0, fabsf(dwv[k]));
                     }
-                    if ((mo >> k) & 1u) {
-                        sea[po] = e[k];
-                        seas[po] = v[k];
-                        ++po;
-                        mk1 = max(mk1, __float_as_uint(e[k]) & 0x7fffffffu);
-                        mk2 = max(mk2, __float_as_uint(v[k]) & 0x7fffffffu);
+                    if ((bo[k] >> lane) & 1u) {
+                        const u32 po = ro + __popc(bo[k] & lt);
+                        sea[po] = eav[k];
+                        seas[po] = easv[k];
+                        mk1 = fmaxf(mk1, fabsf(eav[k]));
+                        mk2 = fmaxf(mk2, easv[k]);
                     }
+                    rw += __popc(bw[k]);
+                    ro += __popc(bo[k]);
                 }
             }
         }
         ring.release();
-        if (cc.chunk == DenseCursor<MCH>::CHUNKS_PER_TILE - 1 && lane == 0) {
+        if (cc.chunk == TileWalk<MCH>::CHUNKS_PER_TILE - 1 && lane == 0) {
             ws.tile_cnt_w[cc.tile] = rw;
             ws.tile_cnt_o[cc.tile] = ro;
         }
         cc.next();
     }
     if (prev >= 0) flush_max(prev);
+    const bool bad = (nanacc != nanacc) || (minv < 0.f);
     if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(&call->flags, FLAG_NONFINITE);
 }
 
@@ -224,7 +216,7 @@ void launch_mask_compact(const LaunchCfg& cfg, const TensorDesc* descs, TensorSt
     if (tiles) {
         const u32 grid = min((tiles + MWARPS - 1) / MWARPS, (u32)cfg.sms * 2u);
         cudaFuncSetAttribute(mask_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(MaskSmem));
-        mask_compact_kernel<<<grid, TPB, sizeof(MaskSmem), cfg.stream>>>(descs, st, nt, tiles, ws, call);
+        mask_compact_kernel<<<grid, MTPB, sizeof(MaskSmem), cfg.stream>>>(descs, st, nt, tiles, ws, call);
         prof_mark(cfg, ST_MASK_COMPACT, 1);
     }
     tile_scan_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, ws);

@@ -20,24 +20,24 @@ struct WarpRing {
     static constexpr int STAGE_FLOATS = NS * CH;
     float* buf;                    // ST stages of NS streams of CH values
     unsigned long long* bar;       // one barrier per stage
-    u32 issued, consumed;          // chunks so far: stage = n % ST, phase = (n / ST) & 1
+    u32 i_stage, c_stage, c_phase, inflight;
 
     __device__ void init(float* b, unsigned long long* r, int lane) {
-        buf = b; bar = r; issued = 0; consumed = 0;
+        buf = b; bar = r; i_stage = 0; c_stage = 0; c_phase = 0; inflight = 0;
         if (lane == 0) {
             for (int s = 0; s < ST; ++s) mbar_init(&bar[s], 1);
             mbar_fence_init();
         }
         __syncwarp();
     }
-    __device__ bool can_issue() const { return issued - consumed < (u32)ST; }
+    __device__ bool can_issue() const { return inflight < (u32)ST; }
 
     // Starts the copies of one chunk: `nbulk` values (a multiple of 4, possibly 0) from each
     // non-null source.  Called by the whole warp; lane 0 talks to the copy engine.
     __device__ void issue(int lane, const float* const (&src)[NS], u32 nbulk) {
         if (lane == 0) {
-            unsigned long long* b = &bar[issued % ST];
-            float* dst = buf + (issued % ST) * STAGE_FLOATS;
+            unsigned long long* b = &bar[i_stage];
+            float* dst = buf + i_stage * STAGE_FLOATS;
             u32 n = 0;
 #pragma unroll
             for (int k = 0; k < NS; ++k) n += src[k] != nullptr;
@@ -50,38 +50,50 @@ struct WarpRing {
                 mbar_arrive(b);
             }
         }
-        ++issued;
+        i_stage = i_stage + 1 == (u32)ST ? 0u : i_stage + 1;
+        ++inflight;
     }
     // Blocks (bounded) until the oldest chunk in flight has landed.
-    __device__ bool wait() { return mbar_wait_warp(&bar[consumed % ST], (consumed / ST) & 1u); }
-    __device__ const float* stage() const { return buf + (consumed % ST) * STAGE_FLOATS; }
+    __device__ bool wait() { return mbar_wait_warp(&bar[c_stage], c_phase); }
+    __device__ const float* stage() const { return buf + c_stage * STAGE_FLOATS; }
     // Every lane is done reading the stage: it may be refilled.
-    __device__ void release() { __syncwarp(); ++consumed; }
+    __device__ void release() {
+        __syncwarp();
+        if (++c_stage == (u32)ST) { c_stage = 0; c_phase ^= 1u; }
+        --inflight;
+    }
 };
 
-// Position of a warp inside its run of tiles, in chunks of CH values.
+// A warp's position inside its run of tiles, in chunks of CH values.  The tensor is looked
+// up once per tile (enter_tile); chunk arithmetic stays in 32 bits.
 template <int CH>
-struct DenseCursor {
+struct TileWalk {
     static constexpr u32 CHUNKS_PER_TILE = TILE / CH;
     u32 tile, chunk;
-    int tns;                       // tensor owning `tile` (-1: not looked up yet)
+    u32 tv;                        // values of this tile that exist (0..TILE)
+    int tns;                       // tensor owning `tile` (-1: none yet)
     u32 tb, ntl;                   // that tensor's tile range
-    u64 numel;
+    u64 numel, toff;               // its size; offset of this tile's first value in it
 
-    __device__ void start(u32 t) { tile = t; chunk = 0; tns = -1; tb = 0; ntl = 0; numel = 0; }
-    // Looks the tensor up when the tile has left the current one; true if it changed.
+    __device__ void start(u32 t) { tile = t; chunk = 0; tv = 0; tns = -1; tb = 0; ntl = 0; numel = 0; toff = 0; }
+    // Call at the first chunk of every tile; true if the tensor changed.
     template <typename Desc>
-    __device__ bool locate(const Desc* __restrict__ descs, int nt) {
-        if (tns >= 0 && tile < tb + ntl) return false;
-        tns = find_tensor(descs, nt, tile);
-        tb = descs[tns].tile_begin; ntl = descs[tns].num_tiles; numel = descs[tns].numel;
-        return true;
+    __device__ bool enter_tile(const Desc* __restrict__ descs, int nt) {
+        bool changed = false;
+        if (tns < 0 || tile >= tb + ntl) {
+            tns = find_tensor(descs, nt, tile);
+            tb = descs[tns].tile_begin; ntl = descs[tns].num_tiles; numel = descs[tns].numel;
+            changed = true;
+        }
+        toff = (u64)(tile - tb) * TILE;
+        tv = toff >= numel ? 0u : (u32)min((u64)TILE, numel - toff);
+        return changed;
     }
-    __device__ u64 elem0() const { return (u64)(tile - tb) * TILE + (u64)chunk * CH; }   // within the tensor
-    __device__ u32 valid() const {                                                      // values of this chunk
-        const u64 e0 = elem0();
-        return e0 >= numel ? 0u : (u32)min((u64)CH, numel - e0);
+    __device__ u32 valid() const {                      // values of this chunk that exist
+        const u32 o = chunk * CH;
+        return tv > o ? min((u32)CH, tv - o) : 0u;
     }
+    __device__ u64 elem0() const { return toff + chunk * CH; }
     __device__ void next() { if (++chunk == CHUNKS_PER_TILE) { chunk = 0; ++tile; } }
 };
 
