@@ -250,7 +250,7 @@ def run_ours(args):
         "stats1": (src_b + 4) * n_tot,
         "stats2": src_b * n_tot,
         "mask_compact": 16 * n_tot + n_tot / 4 + 4 * nnz_w + 8 * nnz_o,
-        "lloyd_dw": T * 4 * nnz_w, "lloyd_ea": T * 4 * nnz_o, "lloyd_eas": T * 4 * nnz_o,
+        "lloyd_dw": T * 4 * nnz_w, "lloyd_moments": T * 8 * nnz_o,
         "pack_codes": 4.5 * (nnz_w + 2 * nnz_o),
         "copy_bitmaps": n_tot / 2,
     }

@@ -544,8 +544,8 @@ int excp_profile_stage_count(void) { return ST_COUNT; }
 
 const char* excp_profile_stage_name(int stage) {
     static const char* names[ST_COUNT] = {
-        "stats1", "stats2", "mask_compact", "scan_layout", "kmeans_start", "lloyd_dw", "lloyd_ea",
-        "lloyd_eas", "kmeans_update", "header_edges", "pack_codes", "copy_bitmaps", "dec_prep", "decode"};
+        "stats1", "stats2", "mask_compact", "scan_layout", "kmeans_start", "lloyd_dw", "lloyd_moments",
+        "unused", "kmeans_update", "header_edges", "pack_codes", "copy_bitmaps", "dec_prep", "decode"};
     return stage >= 0 && stage < ST_COUNT ? names[stage] : "";
 }
 

@@ -12,7 +12,7 @@
 //   update   mean = fp32(fp64(sum)/fp64(count) * 2^(E-30)); empty clusters keep
 //            their centre; centres re-sorted; new thresholds
 #include "excp_common.cuh"
-#include "tma.cuh"
+#include "seg_ring.cuh"
 
 namespace excp {
 
@@ -82,154 +82,133 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
     if (tid < 32) set_thresholds(s, tid);
 }
 
-// One Lloyd sweep of one stream over every tile of the group.
+// One Lloyd sweep over every tile of the group: NS = 1 for the dW stream, NS = 2 for the two
+// moment streams together (they share the mask M_o, hence their tile counts).
 //
-// Every warp works alone on a contiguous run of tiles: lane 0 streams the tiles'
-// survivor segments into the warp's own ring of shared-memory stages with bulk
-// asynchronous copies (512 values per copy, four in flight), the warp consumes
-// them as float4, and nothing in the sweep synchronises the block.
-constexpr int LCH = 512;             // values per staged chunk
+// Every warp works alone on a contiguous run of tiles: lane 0 streams the tiles' survivor
+// segments into the warp's own ring of shared-memory stages with bulk asynchronous copies,
+// the warp consumes them as float4, and nothing in the sweep synchronises the block.
 constexpr int LST = 2;               // stages per warp
 constexpr int LWARPS = TPB / 32;
 
+template <int NS, int CH>
 struct LloydSmem {
-    float buf[LWARPS][LST][LCH];
-    u64 acc[KMAX][TPB];              // [cluster][thread]: a private cell per thread, bank = thread
-    u64 bar[LWARPS][LST];
-    float thr[LWARPS][KPAD];         // each warp's copy of its tensor's thresholds
+    float buf[LWARPS][LST][NS][CH];
+    u64 acc[NS][KMAX][TPB];          // [stream][cluster][thread]: a private cell per thread, bank = thread
+    unsigned long long bar[LWARPS][LST];
+    float thr[LWARPS][NS][KPAD];     // each warp's copy of its tensor's thresholds
 };
 
-__global__ void __launch_bounds__(TPB, 3) lloyd_pass_kernel(const TensorDesc* __restrict__ descs,
-                                                            TensorState* __restrict__ st, int nt, u32 tiles,
-                                                            const float* __restrict__ surv,
-                                                            const u32* __restrict__ tile_cnt, int stream,
-                                                            CallState* call) {
+template <int NS, int CH>
+__global__ void __launch_bounds__(TPB, NS == 1 ? 3 : 2)
+lloyd_pass_kernel(const TensorDesc* __restrict__ descs, TensorState* __restrict__ st, int nt, u32 tiles,
+                  Workspace ws, int stream0, CallState* call) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    LloydSmem& sm = *reinterpret_cast<LloydSmem*>(smem_raw);
+    LloydSmem<NS, CH>& sm = *reinterpret_cast<LloydSmem<NS, CH>*>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 #pragma unroll
-    for (int j = 0; j < KMAX; ++j) sm.acc[j][tid] = 0;
-    if (lane == 0) {
-        for (int s = 0; s < LST; ++s) mbar_init(&sm.bar[warp][s], 1);
-        mbar_fence_init();
-    }
-    __syncwarp();
+    for (int k = 0; k < NS; ++k)
+#pragma unroll
+        for (int j = 0; j < KMAX; ++j) sm.acc[k][j][tid] = 0;
 
     const u32 gw = blockIdx.x * LWARPS + warp, nw = gridDim.x * LWARPS;
     const u32 wlo = (u32)(((u64)tiles * gw) / nw), whi = (u32)(((u64)tiles * (gw + 1)) / nw);
-    u32 g_issue = 0, g_cons = 0;     // chunks issued / consumed so far: stage = g % LST, phase = (g / LST) & 1
+    SegRing<NS, CH, LST> ring;
+    ring.init(&sm.buf[warp][0][0][0], sm.bar[warp], lane, wlo, whi);
+    const u32* tile_cnt = stream0 == 0 ? ws.tile_cnt_w : ws.tile_cnt_o;
+    const float* surv[NS];
+#pragma unroll
+    for (int k = 0; k < NS; ++k) surv[k] = ws.surv[stream0 + k];
+
     int cur = -1;
     u32 tb = 0, ntl = 0, since = 0;
-    float t3 = 0.f, t7 = 0.f, t11 = 0.f;
-    float s1 = 0.f, s2 = 0.f;
-    const char* const thr_row = reinterpret_cast<const char*>(sm.thr[warp]);
-    char* const cell0 = reinterpret_cast<char*>(&sm.acc[0][tid]);
+    float t3[NS], t7[NS], t11[NS], s1[NS], s2[NS];
+#pragma unroll
+    for (int k = 0; k < NS; ++k) t3[k] = t7[k] = t11[k] = s1[k] = s2[k] = 0.f;
+    char* const cell0 = reinterpret_cast<char*>(&sm.acc[0][0][tid]);
 
     auto flush = [&](int tns) {      // this warp's cells -> one integer atomic per cluster
 #pragma unroll
-        for (int j = 0; j < KMAX; ++j) {
-            const s64 v = (s64)sm.acc[j][tid];
-            sm.acc[j][tid] = 0;
-            s64 c = (v + (1ll << 47)) >> 48;          // count sits above a 48-bit signed sum
-            s64 q = v - (c << 48);
+        for (int k = 0; k < NS; ++k) {
 #pragma unroll
-            for (int o = 16; o; o >>= 1) {
-                c += __shfl_xor_sync(0xffffffffu, c, o);
-                q += __shfl_xor_sync(0xffffffffu, q, o);
-            }
-            if (lane == 0 && c) {
-                atomicAdd(reinterpret_cast<u64*>(&st[tns].s[stream].acc_sum[j]), (u64)q);
-                atomicAdd(&st[tns].s[stream].acc_cnt[j], (u64)c);
+            for (int j = 0; j < KMAX; ++j) {
+                const s64 v = (s64)sm.acc[k][j][tid];
+                sm.acc[k][j][tid] = 0;
+                s64 c = (v + (1ll << 47)) >> 48;          // count sits above a 48-bit signed sum
+                s64 q = v - (c << 48);
+#pragma unroll
+                for (int o = 16; o; o >>= 1) {
+                    c += __shfl_xor_sync(0xffffffffu, c, o);
+                    q += __shfl_xor_sync(0xffffffffu, q, o);
+                }
+                if (lane == 0 && c) {
+                    atomicAdd(reinterpret_cast<u64*>(&st[tns].s[stream0 + k].acc_sum[j]), (u64)q);
+                    atomicAdd(&st[tns].s[stream0 + k].acc_cnt[j], (u64)c);
+                }
             }
         }
         since = 0;
     };
 
-    for (u32 w0 = wlo; w0 < whi; w0 += 32) {
-        const u32 wn = min(32u, whi - w0);
-        const u32 mycnt = (u32)lane < wn ? tile_cnt[w0 + lane] : 0u;
-        u32 it = 0, ic = 0;          // issue cursor: tile within the window, value offset in its segment
-        u32 ct = 0, cc = 0;          // consume cursor
-        while (it < wn && __shfl_sync(0xffffffffu, mycnt, it) == 0) ++it;
-        while (ct < wn && __shfl_sync(0xffffffffu, mycnt, ct) == 0) ++ct;
-        while (ct < wn) {
-            while (it < wn && g_issue - g_cons < (u32)LST) {
-                const u32 c = __shfl_sync(0xffffffffu, mycnt, it);
-                const u32 nel = min((u32)LCH, c - ic);
-                if (lane == 0) {
-                    const u32 bytes = ((nel + 3u) & ~3u) * 4u;
-                    u64* bar = &sm.bar[warp][g_issue % LST];
-                    mbar_arrive_expect_tx(bar, bytes);
-                    bulk_g2s(sm.buf[warp][g_issue % LST], surv + (u64)(w0 + it) * TILE + ic, bytes, bar);
-                }
-                ++g_issue;
-                ic += LCH;
-                if (ic >= c) {
-                    ic = 0; ++it;
-                    while (it < wn && __shfl_sync(0xffffffffu, mycnt, it) == 0) ++it;
-                }
-            }
-            const u32 tile = w0 + ct;
+    for (bool first = true; ring.next_window(tile_cnt, lane, first); first = false) {
+        while (ring.have()) {
+            ring.issue_ahead(lane, surv);
+            const u32 tile = ring.tile();
             if (cur < 0 || tile >= tb + ntl) {
                 if (cur >= 0) flush(cur);
                 cur = find_tensor(descs, nt, tile);
                 tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
-                const StreamState& ss = st[cur].s[stream];
                 __syncwarp();
-                if (lane < KPAD) sm.thr[warp][lane] = ss.thr[lane];
+#pragma unroll
+                for (int k = 0; k < NS; ++k) {
+                    const StreamState& ss = st[cur].s[stream0 + k];
+                    if (lane < KPAD) sm.thr[warp][k][lane] = ss.thr[lane];
+                    s1[k] = ss.scale1; s2[k] = ss.scale2;
+                }
                 __syncwarp();
-                t3 = sm.thr[warp][3]; t7 = sm.thr[warp][7]; t11 = sm.thr[warp][11];
-                s1 = ss.scale1; s2 = ss.scale2;
+#pragma unroll
+                for (int k = 0; k < NS; ++k) {
+                    t3[k] = sm.thr[warp][k][3]; t7[k] = sm.thr[warp][k][7]; t11[k] = sm.thr[warp][k][11];
+                }
             }
-            const u32 c = __shfl_sync(0xffffffffu, mycnt, ct);
-            const u32 nel = min((u32)LCH, c - cc);
-            const u32 stage = g_cons % LST;
-            if (!mbar_wait_warp(&sm.bar[warp][stage], (g_cons / LST) & 1u)) {
+            const u32 nel = ring.nel();
+            if (!ring.wait()) {
                 if (lane == 0) atomicOr(&call->flags, FLAG_TIMEOUT);
                 return;
             }
-            const float4* b4 = reinterpret_cast<const float4*>(sm.buf[warp][stage]);
-            // cluster = number of thresholds below x: two levels from registers, two from the
-            // warp's threshold row in shared memory (index kept pre-scaled by 4 bytes)
-            auto find = [&](float x) -> u32 {
-                u32 p = x > t7 ? 32u : 0u;
-                p += (x > (p ? t11 : t3)) ? 16u : 0u;
-                p += (x > *reinterpret_cast<const float*>(thr_row + p + 4)) ? 8u : 0u;
-                p += (x > *reinterpret_cast<const float*>(thr_row + p)) ? 4u : 0u;
-                return p;
-            };
-            auto add = [&](u32 p, float x) {
-                const int q = __float2int_rn(__fmul_rn(__fmul_rn(x, s1), s2));
-                u64* cell = reinterpret_cast<u64*>(cell0 + p * (TPB * 2u));
-                *cell = (u64)((s64)*cell + (s64)q) + (1ull << 48);
-            };
-            if (nel == (u32)LCH) {
-                // all searches of a batch first (they only read), then the read-modify-writes
 #pragma unroll
-                for (int k = 0; k < LCH / 128; k += 2) {
-                    const float4 u4 = b4[lane + 32 * k], v4 = b4[lane + 32 * (k + 1)];
-                    const u32 p0 = find(u4.x), p1 = find(u4.y), p2 = find(u4.z), p3 = find(u4.w);
-                    const u32 p4 = find(v4.x), p5 = find(v4.y), p6 = find(v4.z), p7 = find(v4.w);
-                    add(p0, u4.x); add(p1, u4.y); add(p2, u4.z); add(p3, u4.w);
-                    add(p4, v4.x); add(p5, v4.y); add(p6, v4.z); add(p7, v4.w);
-                }
-            } else {
-                for (u32 f = lane; 4 * f < nel; f += 32) {
-                    const float4 v4 = b4[f];
-                    const u32 p0 = find(v4.x), p1 = find(v4.y), p2 = find(v4.z), p3 = find(v4.w);
-                    add(p0, v4.x);
-                    if (4 * f + 1 < nel) add(p1, v4.y);
-                    if (4 * f + 2 < nel) add(p2, v4.z);
-                    if (4 * f + 3 < nel) add(p3, v4.w);
+            for (int k = 0; k < NS; ++k) {
+                const float4* b4 = reinterpret_cast<const float4*>(ring.stage() + k * CH);
+                const char* thr_row = reinterpret_cast<const char*>(sm.thr[warp][k]);
+                char* const cells = cell0 + k * (KMAX * TPB * 8);
+                auto find = [&](float x) { return find_cluster4(x, t3[k], t7[k], t11[k], thr_row); };
+                auto add = [&](u32 p, float x) {
+                    const int q = __float2int_rn(__fmul_rn(__fmul_rn(x, s1[k]), s2[k]));
+                    u64* cell = reinterpret_cast<u64*>(cells + p * (TPB * 2u));
+                    *cell = (u64)((s64)*cell + (s64)q) + (1ull << 48);
+                };
+                if (nel == (u32)CH) {
+                    // all searches of a batch first (they only read), then the read-modify-writes
+#pragma unroll
+                    for (int f = 0; f < CH / 128; f += 2) {
+                        const float4 u4 = b4[lane + 32 * f], v4 = b4[lane + 32 * (f + 1)];
+                        const u32 p0 = find(u4.x), p1 = find(u4.y), p2 = find(u4.z), p3 = find(u4.w);
+                        const u32 p4 = find(v4.x), p5 = find(v4.y), p6 = find(v4.z), p7 = find(v4.w);
+                        add(p0, u4.x); add(p1, u4.y); add(p2, u4.z); add(p3, u4.w);
+                        add(p4, v4.x); add(p5, v4.y); add(p6, v4.z); add(p7, v4.w);
+                    }
+                } else {
+                    for (u32 f = lane; 4 * f < nel; f += 32) {
+                        const float4 v4 = b4[f];
+                        const u32 p0 = find(v4.x), p1 = find(v4.y), p2 = find(v4.z), p3 = find(v4.w);
+                        add(p0, v4.x);
+                        if (4 * f + 1 < nel) add(p1, v4.y);
+                        if (4 * f + 2 < nel) add(p2, v4.z);
+                        if (4 * f + 3 < nel) add(p3, v4.w);
+                    }
                 }
             }
-            __syncwarp();            // every lane is done with the stage before it is refilled
-            ++g_cons;
-            cc += LCH;
-            if (cc >= c) {
-                cc = 0; ++ct;
-                while (ct < wn && __shfl_sync(0xffffffffu, mycnt, ct) == 0) ++ct;
-            }
+            ring.advance();
             if (++since >= 1024) flush(cur);
         }
     }
@@ -270,16 +249,16 @@ void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* s
     kmeans_start_kernel<<<dim3(nt, 3), SAMPLE_MAX, 0, cfg.stream>>>(descs, st, ws, p.seed);
     prof_mark(cfg, ST_KMEANS_START, 1);
     if (!tiles) return;
-    const u32 grid = min((tiles + LWARPS - 1) / LWARPS, (u32)cfg.sms * 3u);
-    const size_t smem = sizeof(LloydSmem);
-    cudaFuncSetAttribute(lloyd_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const u32 grid1 = min((tiles + LWARPS - 1) / LWARPS, (u32)cfg.sms * 3u);
+    const u32 grid2 = min((tiles + LWARPS - 1) / LWARPS, (u32)cfg.sms * 2u);
+    const size_t smem1 = sizeof(LloydSmem<1, 512>), smem2 = sizeof(LloydSmem<2, 256>);
+    cudaFuncSetAttribute(lloyd_pass_kernel<1, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1);
+    cudaFuncSetAttribute(lloyd_pass_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
     for (int it = 0; it < p.kmeans_iters; ++it) {
-        lloyd_pass_kernel<<<grid, TPB, smem, cfg.stream>>>(descs, st, nt, tiles, ws.surv[0], ws.tile_cnt_w, 0, call);
+        lloyd_pass_kernel<1, 512><<<grid1, TPB, smem1, cfg.stream>>>(descs, st, nt, tiles, ws, 0, call);
         prof_mark(cfg, ST_LLOYD_W, 1);
-        lloyd_pass_kernel<<<grid, TPB, smem, cfg.stream>>>(descs, st, nt, tiles, ws.surv[1], ws.tile_cnt_o, 1, call);
+        lloyd_pass_kernel<2, 256><<<grid2, TPB, smem2, cfg.stream>>>(descs, st, nt, tiles, ws, 1, call);
         prof_mark(cfg, ST_LLOYD_EA, 1);
-        lloyd_pass_kernel<<<grid, TPB, smem, cfg.stream>>>(descs, st, nt, tiles, ws.surv[2], ws.tile_cnt_o, 2, call);
-        prof_mark(cfg, ST_LLOYD_EAS, 1);
         kmeans_update_kernel<<<nt, 96, 0, cfg.stream>>>(st);
         prof_mark(cfg, ST_KMEANS_UPDATE, 1);
     }

@@ -6,6 +6,7 @@
 // last 32-bit code word of a tile may be shared with its neighbours: those words
 // are cleared beforehand and OR-ed into; interior words are stored whole.
 #include "excp_common.cuh"
+#include "seg_ring.cuh"
 
 namespace excp {
 
@@ -99,57 +100,115 @@ __global__ void __launch_bounds__(TPB) clear_edges_kernel(const TensorDesc* __re
     }
 }
 
-// Final assignment + packing of one stream.
+// Final assignment + packing: NS = 1 for dW, NS = 2 for the two moment streams together.
+// A warp owns a run of tiles and streams their survivor segments through its ring of stages
+// (see seg_ring.cuh).  Within a tile the survivors form rows of 8 (one 32-bit word of codes in
+// the tile's own alignment); the tile starts at an arbitrary rank of the tensor, so every
+// output word is two neighbouring rows funnel-shifted by the rank's offset in its word.
+constexpr int PST = 2;
+constexpr int PWARPS = TPB / 32;
+
+template <int NS, int CH>
+struct PackSmem {
+    float buf[PWARPS][PST][NS][CH];
+    unsigned long long bar[PWARPS][PST];
+    float thr[PWARPS][NS][KPAD];
+    u32 rows[PWARPS][NS][CH / 8 + 2];   // [0] = last row of the previous chunk, then this chunk's rows
+};
+
+template <int NS, int CH>
 __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __restrict__ descs,
                                                          const TensorState* __restrict__ st, int nt,
-                                                         u32 tiles, const float* __restrict__ surv,
-                                                         const u32* __restrict__ tile_cnt,
-                                                         const u32* __restrict__ tile_off, int stream,
-                                                         unsigned char* blob, const CallState* call) {
-    __shared__ float thr[KPAD];
-    __shared__ unsigned char code[TILE];
+                                                         u32 tiles, Workspace ws, int stream0,
+                                                         unsigned char* blob, CallState* call) {
+    __shared__ __align__(128) PackSmem<NS, CH> sm;
     if (call->flags & FLAG_BLOB_FULL) return;
-    const int tid = threadIdx.x;
-    u32 lo, hi;
-    block_range(tiles, lo, hi);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const u32 gw = blockIdx.x * PWARPS + warp, nw = gridDim.x * PWARPS;
+    const u32 wlo = (u32)(((u64)tiles * gw) / nw), whi = (u32)(((u64)tiles * (gw + 1)) / nw);
+    SegRing<NS, CH, PST> ring;
+    ring.init(&sm.buf[warp][0][0][0], sm.bar[warp], lane, wlo, whi);
+    const u32* tile_cnt = stream0 == 0 ? ws.tile_cnt_w : ws.tile_cnt_o;
+    const u32* tile_off = stream0 == 0 ? ws.tile_off_w : ws.tile_off_o;
+    const float* surv[NS];
+#pragma unroll
+    for (int k = 0; k < NS; ++k) surv[k] = ws.surv[stream0 + k];
+    constexpr u32 ROWS = CH / 8;
+
     int cur = -1;
     u32 tb = 0, ntl = 0;
-    u32* words = nullptr;
-    for (u32 tile = lo; tile < hi; ++tile) {
-        if (cur < 0 || tile >= tb + ntl) {
-            cur = find_tensor(descs, nt, tile);
-            tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
-            const TensorState& s = st[cur];
-            const Sections sec = sections_of(descs[cur].numel, s.nnz_w, s.nnz_o);
-            words = reinterpret_cast<u32*>(blob + s.blob_off + sec.codes[stream]);
-            __syncthreads();
-            if (tid < KPAD) thr[tid] = s.s[stream].thr[tid];
-        }
-        __syncthreads();                       // thr ready; previous tile's codes consumed
-        const u32 cnt = tile_cnt[tile];
-        if (cnt == 0) continue;
-        const u32 off = tile_off[tile];
-        const float* data = surv + (u64)tile * TILE;
-        for (u32 i = tid; i < cnt; i += TPB) {
-            const float x = data[i];
-            int p = (x > thr[7]) ? 8 : 0;
-            p += (x > thr[p + 3]) ? 4 : 0;
-            p += (x > thr[p + 1]) ? 2 : 0;
-            p += (x > thr[p]) ? 1 : 0;
-            code[i] = (unsigned char)(p + 1);
-        }
-        __syncthreads();
-        const u32 w0 = off / PER_WORD, w1 = (off + cnt - 1) / PER_WORD;
-        for (u32 w = w0 + tid; w <= w1; w += TPB) {
-            u32 v = 0;
-            const s64 first = (s64)w * PER_WORD - (s64)off;      // local index of the word's code 0
+    u32* words[NS];
+    float t3[NS], t7[NS], t11[NS];
 #pragma unroll
-            for (int k = 0; k < PER_WORD; ++k) {
-                const s64 i = first + k;
-                if (i >= 0 && i < (s64)cnt) v |= (u32)code[i] << (BITS * k);
+    for (int k = 0; k < NS; ++k) { words[k] = nullptr; t3[k] = t7[k] = t11[k] = 0.f; }
+    u32 carry[NS];                       // last row of the previous chunk of the same tile
+#pragma unroll
+    for (int k = 0; k < NS; ++k) carry[k] = 0;
+
+    for (bool first = true; ring.next_window(tile_cnt, lane, first); first = false) {
+        while (ring.have()) {
+            ring.issue_ahead(lane, surv);
+            const u32 tile = ring.tile();
+            if (cur < 0 || tile >= tb + ntl) {
+                cur = find_tensor(descs, nt, tile);
+                tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
+                const TensorState& s = st[cur];
+                const Sections sec = sections_of(descs[cur].numel, s.nnz_w, s.nnz_o);
+                __syncwarp();
+#pragma unroll
+                for (int k = 0; k < NS; ++k) {
+                    words[k] = reinterpret_cast<u32*>(blob + s.blob_off + sec.codes[stream0 + k]);
+                    if (lane < KPAD) sm.thr[warp][k][lane] = s.s[stream0 + k].thr[lane];
+                }
+                __syncwarp();
+#pragma unroll
+                for (int k = 0; k < NS; ++k) {
+                    t3[k] = sm.thr[warp][k][3]; t7[k] = sm.thr[warp][k][7]; t11[k] = sm.thr[warp][k][11];
+                }
             }
-            if (first >= 0 && first + PER_WORD <= (s64)cnt) words[w] = v;
-            else atomicOr(&words[w], v);
+            const u32 cnt = ring.tile_cnt_cur(), off = ring.off(), nel = ring.nel();
+            const u32 t0 = tile_off[tile];                 // tensor-wide rank of the tile's first survivor
+            if (!ring.wait()) {
+                if (lane == 0) atomicOr(&call->flags, FLAG_TIMEOUT);
+                return;
+            }
+            const u32 nrows = (nel + 7) / 8;               // rows of this chunk
+            const u32 sh = (t0 & 7u) * BITS;               // a row's shift inside the tensor's words
+            const u32 wbase = t0 / 8 + off / 8;            // output word of this chunk's first row
+            const bool last_chunk = off + nel == cnt;
+#pragma unroll
+            for (int k = 0; k < NS; ++k) {
+                if (off == 0) carry[k] = 0;
+                const float* data = ring.stage() + k * CH;
+                const char* thr_row = reinterpret_cast<const char*>(sm.thr[warp][k]);
+                u32* rows = sm.rows[warp][k];
+                if (lane == 0) rows[0] = carry[k];
+                for (u32 r = lane; r < nrows; r += 32) {   // 8 codes -> one word in the tile's alignment
+                    const float4 u4 = *reinterpret_cast<const float4*>(data + 8 * r);
+                    const float4 v4 = *reinterpret_cast<const float4*>(data + 8 * r + 4);
+                    const float xs[8] = {u4.x, u4.y, u4.z, u4.w, v4.x, v4.y, v4.z, v4.w};
+                    u32 w = 0;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const u32 code = find_cluster4(xs[i], t3[k], t7[k], t11[k], thr_row) / 4 + 1;
+                        if (8 * r + i < nel) w |= code << (BITS * i);
+                    }
+                    rows[1 + r] = w;
+                }
+                if (lane == 0) rows[1 + nrows] = 0;
+                __syncwarp();
+                carry[k] = rows[nrows];                    // the chunk's last row (for the next chunk)
+                // output word m of the chunk = row m shifted up | row m-1 shifted down
+                const u32 nout = nrows + ((last_chunk && sh) ? 1u : 0u);
+                for (u32 m = lane; m < nout; m += 32) {
+                    const u32 v = (rows[1 + m] << sh) | (sh ? rows[m] >> (32 - sh) : 0u);
+                    const u64 g0 = (u64)(wbase + m) * 8;   // ranks the word covers: [g0, g0 + 8)
+                    if (g0 >= t0 && g0 + 8 <= (u64)t0 + cnt) words[k][wbase + m] = v;
+                    else if (v) atomicOr(&words[k][wbase + m], v);
+                }
+                __syncwarp();
+            }
+            ring.advance();
         }
     }
 }
@@ -184,14 +243,10 @@ void launch_pack(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st,
     if (!tiles) { prof_mark(cfg, ST_HEADER_EDGES, 1); return; }
     clear_edges_kernel<<<(tiles + TPB - 1) / TPB, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, blob, call);
     prof_mark(cfg, ST_HEADER_EDGES, 2);
-    const u32 grid = min(tiles, (u32)cfg.sms * 8u);
-    pack_codes_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws.surv[0], ws.tile_cnt_w,
-                                                     ws.tile_off_w, 0, blob, call);
-    pack_codes_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws.surv[1], ws.tile_cnt_o,
-                                                     ws.tile_off_o, 1, blob, call);
-    pack_codes_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws.surv[2], ws.tile_cnt_o,
-                                                     ws.tile_off_o, 2, blob, call);
-    prof_mark(cfg, ST_PACK_CODES, 3);
+    const u32 grid = min((tiles + PWARPS - 1) / PWARPS, (u32)cfg.sms * 4u);
+    pack_codes_kernel<1, 512><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 0, blob, call);
+    pack_codes_kernel<2, 256><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 1, blob, call);
+    prof_mark(cfg, ST_PACK_CODES, 2);
     const u64 quads = (u64)tiles * (TILE_WORDS / 4);
     copy_bitmaps_kernel<<<(u32)((quads + TPB - 1) / TPB), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws,
                                                                                blob, call);
