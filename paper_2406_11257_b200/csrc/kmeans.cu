@@ -6,8 +6,8 @@
 //            fp64 mid-point of centres j and j+1 (so the comparison is exactly
 //            "2x > c_j + c_j+1" in fp64); a 4-step binary search, no distances
 //   sums     Q(x) = rint(x * 2^(30-E)) in int32, accumulated as integers: each
-//            thread owns a private row of 16 shared-memory cells (count in the
-//            top 16 bits, sum below), so there are no atomics in the sweep and
+//            thread owns a private row of 15 shared-memory cells (48-bit sum above
+//            a 16-bit count), so there are no atomics in the sweep and
 //            the result is independent of the order of summation
 //   update   mean = fp32(fp64(sum)/fp64(count) * 2^(E-30)); empty clusters keep
 //            their centre; centres re-sorted; new thresholds
@@ -28,7 +28,7 @@ __device__ inline void set_thresholds(StreamState& s, int lane) {
     if (lane < KPAD) {
         float t = __uint_as_float(0x7f800000u);
         if (lane < KMAX - 1)
-            t = __double2float_rd(((double)s.cent[lane] + (double)s.cent[lane + 1]) * 0.5);
+            t = __double2float_rd(((double)s.cent[lane] + (double)s.cent[lane + 1]) * 0.5) + 0.f;   // -0 -> +0
         s.thr[lane] = t;
     }
 }
@@ -134,8 +134,8 @@ lloyd_pass_kernel(const TensorDesc* __restrict__ descs, TensorState* __restrict_
             for (int j = 0; j < KMAX; ++j) {
                 const s64 v = (s64)sm.acc[k][j][tid];
                 sm.acc[k][j][tid] = 0;
-                s64 c = (v + (1ll << 47)) >> 48;          // count sits above a 48-bit signed sum
-                s64 q = v - (c << 48);
+                s64 c, q;
+                cell_split((u64)v, q, c);
 #pragma unroll
                 for (int o = 16; o; o >>= 1) {
                     c += __shfl_xor_sync(0xffffffffu, c, o);
@@ -184,8 +184,7 @@ lloyd_pass_kernel(const TensorDesc* __restrict__ descs, TensorState* __restrict_
                 auto find = [&](float x) { return find_cluster4(x, t3[k], t7[k], t11[k], thr_row); };
                 auto add = [&](u32 p, float x) {
                     const int q = __float2int_rn(__fmul_rn(__fmul_rn(x, s1[k]), s2[k]));
-                    u64* cell = reinterpret_cast<u64*>(cells + p * (TPB * 2u));
-                    *cell = (u64)((s64)*cell + (s64)q) + (1ull << 48);
+                    cell_add(reinterpret_cast<u64*>(cells + p * (TPB * 2u)), q);
                 };
                 if (nel == (u32)CH) {
                     // all searches of a batch first (they only read), then the read-modify-writes

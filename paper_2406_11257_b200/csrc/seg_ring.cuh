@@ -17,39 +17,44 @@ struct SegRing {
     float* buf;
     unsigned long long* bar;
     u32 whi;                       // end of the warp's run of tiles
-    u32 w0, wn;                    // current window of up to 32 tiles
-    u32 mycnt;                     // count of tile w0 + lane
-    u32 it, ic;                    // issue cursor: tile within the window, value offset in its segment
-    u32 ct, cc;                    // consume cursor
+    u32 w0;                        // first tile of the current window of 32
+    u32 mycnt;                     // count of tile w0 + lane (0 past the run)
+    u32 nz;                        // lanes whose tile has survivors
+    u32 it, i_cnt, ic;             // issue cursor: tile in the window (32 = done), its count, value offset
+    u32 ct, c_cnt, cc;             // consume cursor
     u32 i_stage, c_stage, c_phase, inflight;
 
     __device__ void init(float* b, unsigned long long* r, int lane, u32 wlo, u32 whi_) {
-        buf = b; bar = r; whi = whi_; w0 = wlo; wn = 0;
+        buf = b; bar = r; whi = whi_; w0 = wlo;
         i_stage = c_stage = c_phase = inflight = 0;
+        it = ct = 32; i_cnt = c_cnt = ic = cc = 0; mycnt = 0; nz = 0;
         if (lane == 0) {
             for (int s = 0; s < ST; ++s) mbar_init(&bar[s], 1);
             mbar_fence_init();
         }
         __syncwarp();
     }
-    __device__ u32 cnt_of(u32 i) const { return __shfl_sync(0xffffffffu, mycnt, i); }
+    // first non-empty tile of the window after position i (i = -1: from the start); 32 if none
+    __device__ u32 next_tile(int i) const {
+        const u32 m = i >= 31 ? 0u : nz & (0xffffffffu << (i + 1));
+        return m ? (u32)__ffs((int)m) - 1u : 32u;
+    }
     // Loads the next window; false when the run is finished.  `first` on the first call.
     __device__ bool next_window(const u32* __restrict__ tile_cnt, int lane, bool first) {
         if (!first) w0 += 32;
         if (w0 >= whi) return false;
-        wn = min(32u, whi - w0);
-        mycnt = (u32)lane < wn ? tile_cnt[w0 + lane] : 0u;
-        it = ic = ct = cc = 0;
-        while (it < wn && cnt_of(it) == 0) ++it;
-        ct = it;
+        mycnt = w0 + lane < whi ? tile_cnt[w0 + lane] : 0u;
+        nz = __ballot_sync(0xffffffffu, mycnt != 0);
+        it = ct = next_tile(-1);
+        i_cnt = c_cnt = it < 32 ? __shfl_sync(0xffffffffu, mycnt, it) : 0u;
+        ic = cc = 0;
         return true;
     }
-    __device__ bool have() const { return ct < wn; }
+    __device__ bool have() const { return ct < 32; }
     __device__ void issue_ahead(int lane, const float* const (&surv)[NS]) {
-        while (it < wn && inflight < (u32)ST) {
-            const u32 c = cnt_of(it);
-            const u32 nel = min((u32)CH, c - ic);
+        while (it < 32 && inflight < (u32)ST) {
             if (lane == 0) {
+                const u32 nel = min((u32)CH, i_cnt - ic);
                 const u32 bytes = ((nel + 3u) & ~3u) * 4u;       // stays inside the tile's segment
                 unsigned long long* b = &bar[i_stage];
                 float* dst = buf + i_stage * STAGE_FLOATS;
@@ -61,40 +66,59 @@ struct SegRing {
             i_stage = i_stage + 1 == (u32)ST ? 0u : i_stage + 1;
             ++inflight;
             ic += CH;
-            if (ic >= c) {
-                ic = 0; ++it;
-                while (it < wn && cnt_of(it) == 0) ++it;
+            if (ic >= i_cnt) {
+                ic = 0;
+                it = next_tile((int)it);
+                i_cnt = it < 32 ? __shfl_sync(0xffffffffu, mycnt, it) : 0u;
             }
         }
     }
     __device__ u32 tile() const { return w0 + ct; }
-    __device__ u32 tile_cnt_cur() const { return cnt_of(ct); }
+    __device__ u32 tile_cnt_cur() const { return c_cnt; }
     __device__ u32 off() const { return cc; }                                   // first value of the chunk in its segment
-    __device__ u32 nel() const { return min((u32)CH, cnt_of(ct) - cc); }         // values in the chunk
+    __device__ u32 nel() const { return min((u32)CH, c_cnt - cc); }              // values in the chunk
     __device__ bool wait() { return mbar_wait_warp(&bar[c_stage], c_phase); }
     __device__ const float* stage() const { return buf + c_stage * STAGE_FLOATS; }
     __device__ void advance() {
         __syncwarp();                                   // every lane is done with the stage
         if (++c_stage == (u32)ST) { c_stage = 0; c_phase ^= 1u; }
         --inflight;
-        const u32 c = cnt_of(ct);
         cc += CH;
-        if (cc >= c) {
-            cc = 0; ++ct;
-            while (ct < wn && cnt_of(ct) == 0) ++ct;
+        if (cc >= c_cnt) {
+            cc = 0;
+            ct = next_tile((int)ct);
+            c_cnt = ct < 32 ? __shfl_sync(0xffffffffu, mycnt, ct) : 0u;
         }
     }
 };
 
 // Cluster of x = number of thresholds strictly below it.  thr_row: 16 fp32 thresholds
-// (ascending, +inf from the 15th on) in shared memory; t3, t7, t11 are copies in registers.
-// Returns 4 * cluster.
+// (ascending, +inf from the 15th on, none of them -0) in shared memory; t3, t7, t11 are copies
+// in registers.  Returns 4 * cluster.
+// "x > t" is read off the sign of t - x: with gradual underflow the difference of two distinct
+// floats is never rounded to zero, and t - x = +0 when they are equal.  This keeps the search
+// on the floating-point and multiply-add pipes.
+__device__ __forceinline__ u32 gt_bit(float t, float x) { return __float_as_uint(__fsub_rn(t, x)) >> 31; }
+
 __device__ __forceinline__ u32 find_cluster4(float x, float t3, float t7, float t11, const char* thr_row) {
     u32 p = x > t7 ? 32u : 0u;
     p += (x > (p ? t11 : t3)) ? 16u : 0u;
     p += (x > *reinterpret_cast<const float*>(thr_row + p + 4)) ? 8u : 0u;
     p += (x > *reinterpret_cast<const float*>(thr_row + p)) ? 4u : 0u;
     return p;
+}
+
+// cell += q * 2^16 + 1: a 48-bit signed sum above a 16-bit count (at most 65535 additions
+// between two flushes).
+__device__ __forceinline__ void cell_add(u64* cell, int q) {
+    u64 v;
+    asm("mad.wide.s32 %0, %1, 65536, %2;" : "=l"(v) : "r"(q), "l"(*cell));
+    const u32 lo = (u32)v + 1u;            // the count field cannot carry out of the low word
+    *cell = (v & 0xffffffff00000000ull) | lo;
+}
+__device__ __forceinline__ void cell_split(u64 v, s64& sum, s64& cnt) {
+    cnt = (s64)(v & 0xffffull);
+    sum = (s64)v >> 16;
 }
 
 }  // namespace excp
