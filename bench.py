@@ -246,16 +246,21 @@ def run_ours(args):
     T = args.kmeans_iters
     src_b = 8 if args.median == "residual" else 4
     # bytes each stage must move once (its inputs read once, its outputs written once)
+    surv = nnz_w + 2 * nnz_o
     stage_bytes = {
         "stats1": (src_b + 4) * n_tot,
         "stats2": src_b * n_tot,
-        "mask_compact": 16 * n_tot + n_tot / 4 + 4 * nnz_w + 8 * nnz_o,
-        "lloyd_dw": T * 4 * nnz_w, "lloyd_moments": T * 8 * nnz_o,
-        "pack_codes": 4.5 * (nnz_w + 2 * nnz_o),
+        "mask_compact": 16 * n_tot + n_tot / 4 + 4 * surv,
+        "bucket_ids": 5 * surv,                     # survivors read, one bucket byte each written
+        "bucket_scatter": 10 * surv,                # bucket bytes read twice, survivors read and written
+        "bucket_scan": T * 4 * surv * 14 / 256,     # about 14 of 256 buckets per iteration
+        "pack_codes": 4.5 * surv,
         "copy_bitmaps": n_tot / 2,
     }
-    # what the method itself must move (one statistics sweep, not two)
-    algo_bytes = sum(v for k, v in stage_bytes.items() if k != "stats2")
+    moved_bytes = sum(stage_bytes.values())         # what these kernels must move by design
+    # what the method moves when every Lloyd iteration sweeps the survivors (one statistics sweep,
+    # one mask sweep, T + 1 sweeps of the survivors, the codes)
+    algo_bytes = ((src_b + 4) + 16 + 0.25) * n_tot + 4 * surv + (T + 1) * 4 * surv + 0.5 * surv
     peak, peak_kind = measured_peak()
     per_step = {k: v / args.steps for k, v in stage_ms.items()}
     dom = max((k for k in stage_bytes), key=lambda k: per_step.get(k, 0.0))
@@ -276,6 +281,9 @@ def run_ours(args):
                    "workspace_numel": ws_numel, "per_rank": "each rank compresses its own checkpoint; no collective"},
         "input_gbs": 16 * value / 1e9,
         "algorithmic_bytes_per_param": algo_bytes / n_tot,
+        "moved_bytes_per_param": moved_bytes / n_tot,
+        "moved_gbs": moved_bytes / n_tot * value / world / 1e9,
+        "moved_frac_of_measured": moved_bytes / n_tot * value / world / 1e9 / peak,
         "algorithmic_gbs": algo_bytes / n_tot * value / world / 1e9,
         "hbm_frac_of_measured": algo_bytes / n_tot * value / world / 1e9 / peak,
         "hbm_frac_of_nominal_8TBs": algo_bytes / n_tot * value / world / 1e9 / NOMINAL_HBM_GBS,

@@ -46,6 +46,8 @@ struct TensorDesc {              // built on the host, one per tensor of a group
     u64 tensor_index;            // position in the checkpoint (enters the start sample)
     u32 tile_begin;              // first tile of this tensor within the group
     u32 num_tiles;
+    u32 scan_first;              // first work item of this tensor in the bucket-scan grid
+    u32 scan_n;                  // work items (splits) this tensor has there
 };
 
 struct StreamState {             // K-means state of one stream (0 = dW, 1 = ea, 2 = eas)
@@ -89,7 +91,28 @@ struct CallState {               // one per handle, device resident
     u32 pad_;
 };
 
+constexpr int NBKT = 256;         // value buckets per tensor and stream for the K-means iterations
+
+struct BucketStream {            // one stream's buckets: bucket b holds bnd[b-1] < x <= bnd[b]
+    float bnd[NBKT];             // upper bounds, ascending; bnd[255] = +inf
+    u32 cnt[NBKT];               // survivors per bucket
+    s64 sum[NBKT];               // their fixed-point sums
+    u32 off[NBKT + 1];           // exclusive prefix of cnt = start of each bucket in the bucketed copy
+    u32 pad_;
+    s64 sumpre[NBKT + 1];        // exclusive prefix of sum
+    u32 cursor[NBKT];            // next free slot of each bucket while scattering
+    u32 bstar[KPAD];             // bucket that holds threshold j
+    u64 part_cnt[KPAD];          // survivors <= threshold j inside that bucket
+    s64 part_sum[KPAD];          // and their fixed-point sum
+};
+struct BucketState {
+    BucketStream s[3];
+};
+
 struct Workspace {               // device arrays sized for cap_tiles tiles
+    float* bkt[3];               // survivors again, grouped by value bucket (order inside a bucket is arbitrary)
+    unsigned char* ids[3];       // bucket of each survivor, at the survivor's place in surv[]
+    BucketState* bst;            // per tensor of the group
     float* surv[3];              // survivors, each tile's compacted at the tile's own start
     u32* bm_w;                   // bitmaps, TILE_WORDS words per tile
     u32* bm_o;
@@ -223,8 +246,8 @@ __device__ inline void scan_tile_counts(u32 tb, u32 ntl, const Workspace& ws, u3
 
 // ---- launch wrappers --------------------------------------------------------
 enum Stage {                       // for the optional per-stage event timing
-    ST_STATS1 = 0, ST_STATS2, ST_MASK_COMPACT, ST_SCAN_LAYOUT, ST_KMEANS_START, ST_LLOYD_W, ST_LLOYD_EA,
-    ST_LLOYD_EAS, ST_KMEANS_UPDATE, ST_HEADER_EDGES, ST_PACK_CODES, ST_COPY_BITMAPS, ST_DEC_PREP,
+    ST_STATS1 = 0, ST_STATS2, ST_MASK_COMPACT, ST_SCAN_LAYOUT, ST_KMEANS_START, ST_BUCKET_IDS, ST_BUCKET_SCATTER,
+    ST_BUCKET_SCAN, ST_KMEANS_UPDATE, ST_HEADER_EDGES, ST_PACK_CODES, ST_COPY_BITMAPS, ST_DEC_PREP,
     ST_DECODE, ST_COUNT
 };
 
@@ -243,7 +266,7 @@ void launch_stats(const LaunchCfg&, const TensorDesc* descs, TensorState* st, in
 void launch_mask_compact(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                          const Workspace& ws, const Params& p, CallState* call, u64 blob_capacity);
 void launch_kmeans(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
-                   const Workspace& ws, const Params& p, CallState* call);
+                   u32 scan_items, const Workspace& ws, const Params& p, CallState* call);
 void launch_pack(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                  const Workspace& ws, const Params& p, unsigned char* blob, CallState* call,
                  TensorResult* results);

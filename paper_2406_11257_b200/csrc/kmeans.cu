@@ -4,13 +4,25 @@
 //   start    K equal-mass quantiles of a seeded, index-stratified sample
 //   assign   cluster(x) = #{ j : x > thr_j },  thr_j = largest fp32 not above the
 //            fp64 mid-point of centres j and j+1 (so the comparison is exactly
-//            "2x > c_j + c_j+1" in fp64); a 4-step binary search, no distances
-//   sums     Q(x) = rint(x * 2^(30-E)) in int32, accumulated as integers: each
-//            thread owns a private row of 15 shared-memory cells (48-bit sum above
-//            a 16-bit count), so there are no atomics in the sweep and
-//            the result is independent of the order of summation
+//            "2x > c_j + c_j+1" in fp64)
+//   sums     Q(x) = rint(x * 2^(30-E)) in int32, summed as integers, so that the
+//            result is independent of the order of summation
 //   update   mean = fp32(fp64(sum)/fp64(count) * 2^(E-30)); empty clusters keep
 //            their centre; centres re-sorted; new thresholds
+//
+// The iterations do not sweep the survivors.  Because the clusters are intervals
+// and the sums are integers, the survivors are first grouped ONCE into 256 value
+// buckets (bounds taken from the sorted start sample, so the buckets hold about
+// the same number each) with each bucket's count and sum.  An iteration then
+// needs, per threshold, only the bucket the threshold falls into: buckets below
+// it count whole, and the one bucket is scanned.  That is about 14/256 of the
+// data per iteration, and the sums are exactly those of a full sweep.
+//
+//   bucket_ids      sweep: bucket of every survivor (8-step search), counts
+//   bucket_offsets  prefix of the counts -> where each bucket starts
+//   bucket_scatter  sweep: survivors into their buckets, bucket sums
+//   bucket_prefix   prefix of the sums; first plan
+//   per iteration:  bucket_scan (the 14 threshold buckets), bucket_update
 #include "excp_common.cuh"
 #include "seg_ring.cuh"
 
@@ -44,9 +56,10 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
     const u32 tb = descs[t].tile_begin, ntl = descs[t].num_tiles;
     const u32* toff = (stream == 0 ? ws.tile_off_w : ws.tile_off_o) + tb;
     const float* data = ws.surv[stream] + (u64)tb * TILE;
-    if (tid < KPAD) { s.acc_sum[tid] = 0; s.acc_cnt[tid] = 0; }
+    BucketStream& bk = ws.bst[t].s[stream];
     if (nnz == 0) {
         if (tid < KPAD) { s.cent[tid] = 0.f; s.thr[tid] = __uint_as_float(0x7f800000u); }
+        if (tid < NBKT) bk.bnd[tid] = __uint_as_float(0x7f800000u);
         return;
     }
     const u32 m = min(nnz, (u32)SAMPLE_MAX);
@@ -78,79 +91,70 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
         }
     }
     if (tid < KPAD) s.cent[tid] = tid < KMAX ? smp[((2 * tid + 1) * m) / (2 * KMAX)] : 0.f;
+    // bucket bounds: every (m/256)-th sample value; any ascending values would do, these
+    // make the buckets about equally full
+    if (tid < NBKT) bk.bnd[tid] = tid < NBKT - 1 ? smp[((u32)(tid + 1) * m) / NBKT] : __uint_as_float(0x7f800000u);
     __syncthreads();
     if (tid < 32) set_thresholds(s, tid);
 }
 
-// One Lloyd sweep over every tile of the group: NS = 1 for the dW stream, NS = 2 for the two
-// moment streams together (they share the mask M_o, hence their tile counts).
-//
-// Every warp works alone on a contiguous run of tiles: lane 0 streams the tiles' survivor
-// segments into the warp's own ring of shared-memory stages with bulk asynchronous copies,
-// the warp consumes them as float4, and nothing in the sweep synchronises the block.
-constexpr int LST = 2;               // stages per warp
-constexpr int LWARPS = TPB / 32;
+
+// ---------------------------------------------------------------------------
+// Buckets.  bucket(x) = number of bounds strictly below x (bounds ascending, the last +inf),
+// so bucket b holds bnd[b-1] < x <= bnd[b].
+__device__ __forceinline__ u32 find_bucket(float x, const float* bnd) {
+    u32 b = 0;
+#pragma unroll
+    for (int step = NBKT / 2; step; step >>= 1) b += (x > bnd[b + step - 1]) ? (u32)step : 0u;
+    return b;
+}
+
+constexpr int BWARPS = TPB / 32;
+constexpr int BST = 2;               // stages per warp
 
 template <int NS, int CH>
-struct LloydSmem {
-    float buf[LWARPS][LST][NS][CH];
-    u64 acc[NS][KMAX][TPB];          // [stream][cluster][thread]: a private cell per thread, bank = thread
-    unsigned long long bar[LWARPS][LST];
-    float thr[LWARPS][NS][KPAD];     // each warp's copy of its tensor's thresholds
+struct BucketIdsSmem {
+    float buf[BWARPS][BST][NS][CH];
+    unsigned long long bar[BWARPS][BST];
+    float bnd[BWARPS][NS][NBKT];     // each warp's copy of its tensor's bounds
+    u32 hist[BWARPS][NS][NBKT];      // each warp's counts since its last flush
 };
 
+// Sweep 1 of the grouping: the bucket of every survivor (one byte, stored at the survivor's
+// own place) and the survivors per bucket.  NS = 1: dW; NS = 2: both moment streams.
 template <int NS, int CH>
-__global__ void __launch_bounds__(TPB, NS == 1 ? 3 : 2)
-lloyd_pass_kernel(const TensorDesc* __restrict__ descs, TensorState* __restrict__ st, int nt, u32 tiles,
-                  Workspace ws, int stream0, CallState* call) {
+__global__ void __launch_bounds__(TPB) bucket_ids_kernel(const TensorDesc* __restrict__ descs, int nt, u32 tiles,
+                                                         Workspace ws, int stream0, CallState* call) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    LloydSmem<NS, CH>& sm = *reinterpret_cast<LloydSmem<NS, CH>*>(smem_raw);
+    BucketIdsSmem<NS, CH>& sm = *reinterpret_cast<BucketIdsSmem<NS, CH>*>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-#pragma unroll
-    for (int k = 0; k < NS; ++k)
-#pragma unroll
-        for (int j = 0; j < KMAX; ++j) sm.acc[k][j][tid] = 0;
-
-    const u32 gw = blockIdx.x * LWARPS + warp, nw = gridDim.x * LWARPS;
+    const u32 gw = blockIdx.x * BWARPS + warp, nw = gridDim.x * BWARPS;
     const u32 wlo = (u32)(((u64)tiles * gw) / nw), whi = (u32)(((u64)tiles * (gw + 1)) / nw);
-    SegRing<NS, CH, LST> ring;
+    SegRing<NS, CH, BST> ring;
     ring.init(&sm.buf[warp][0][0][0], sm.bar[warp], lane, wlo, whi);
     const u32* tile_cnt = stream0 == 0 ? ws.tile_cnt_w : ws.tile_cnt_o;
     const float* surv[NS];
 #pragma unroll
-    for (int k = 0; k < NS; ++k) surv[k] = ws.surv[stream0 + k];
-
+    for (int k = 0; k < NS; ++k) {
+        surv[k] = ws.surv[stream0 + k];
+        for (int b = lane; b < NBKT; b += 32) sm.hist[warp][k][b] = 0;
+    }
+    __syncwarp();
     int cur = -1;
-    u32 tb = 0, ntl = 0, since = 0;
-    float t3[NS], t7[NS], t11[NS], s1[NS], s2[NS];
-#pragma unroll
-    for (int k = 0; k < NS; ++k) t3[k] = t7[k] = t11[k] = s1[k] = s2[k] = 0.f;
-    char* const cell0 = reinterpret_cast<char*>(&sm.acc[0][0][tid]);
+    u32 tb = 0, ntl = 0;
 
-    auto flush = [&](int tns) {      // this warp's cells -> one integer atomic per cluster
+    auto flush = [&](int tns) {
+        __syncwarp();
 #pragma unroll
-        for (int k = 0; k < NS; ++k) {
-#pragma unroll
-            for (int j = 0; j < KMAX; ++j) {
-                const s64 v = (s64)sm.acc[k][j][tid];
-                sm.acc[k][j][tid] = 0;
-                s64 c, q;
-                cell_split((u64)v, q, c);
-#pragma unroll
-                for (int o = 16; o; o >>= 1) {
-                    c += __shfl_xor_sync(0xffffffffu, c, o);
-                    q += __shfl_xor_sync(0xffffffffu, q, o);
-                }
-                if (lane == 0 && c) {
-                    atomicAdd(reinterpret_cast<u64*>(&st[tns].s[stream0 + k].acc_sum[j]), (u64)q);
-                    atomicAdd(&st[tns].s[stream0 + k].acc_cnt[j], (u64)c);
-                }
+        for (int k = 0; k < NS; ++k)
+            for (int b = lane; b < NBKT; b += 32) {
+                const u32 c = sm.hist[warp][k][b];
+                if (c) { atomicAdd(&ws.bst[tns].s[stream0 + k].cnt[b], c); sm.hist[warp][k][b] = 0; }
             }
-        }
-        since = 0;
+        __syncwarp();
     };
 
-    for (bool first = true; ring.next_window(tile_cnt, lane, first); first = false) {
+    while (ring.next_window(tile_cnt, lane, whi)) {
         while (ring.have()) {
             ring.issue_ahead(lane, surv);
             const u32 tile = ring.tile();
@@ -158,78 +162,282 @@ lloyd_pass_kernel(const TensorDesc* __restrict__ descs, TensorState* __restrict_
                 if (cur >= 0) flush(cur);
                 cur = find_tensor(descs, nt, tile);
                 tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
-                __syncwarp();
 #pragma unroll
-                for (int k = 0; k < NS; ++k) {
-                    const StreamState& ss = st[cur].s[stream0 + k];
-                    if (lane < KPAD) sm.thr[warp][k][lane] = ss.thr[lane];
-                    s1[k] = ss.scale1; s2[k] = ss.scale2;
-                }
+                for (int k = 0; k < NS; ++k)
+                    for (int b = lane; b < NBKT; b += 32) sm.bnd[warp][k][b] = ws.bst[cur].s[stream0 + k].bnd[b];
                 __syncwarp();
-#pragma unroll
-                for (int k = 0; k < NS; ++k) {
-                    t3[k] = sm.thr[warp][k][3]; t7[k] = sm.thr[warp][k][7]; t11[k] = sm.thr[warp][k][11];
-                }
             }
-            const u32 nel = ring.nel();
+            const u32 nel = ring.nel(), off = ring.off();
             if (!ring.wait()) {
                 if (lane == 0) atomicOr(&call->flags, FLAG_TIMEOUT);
                 return;
             }
 #pragma unroll
             for (int k = 0; k < NS; ++k) {
-                const float4* b4 = reinterpret_cast<const float4*>(ring.stage() + k * CH);
-                const char* thr_row = reinterpret_cast<const char*>(sm.thr[warp][k]);
-                char* const cells = cell0 + k * (KMAX * TPB * 8);
-                auto find = [&](float x) { return find_cluster4(x, t3[k], t7[k], t11[k], thr_row); };
-                auto add = [&](u32 p, float x) {
-                    const int q = __float2int_rn(__fmul_rn(__fmul_rn(x, s1[k]), s2[k]));
-                    cell_add(reinterpret_cast<u64*>(cells + p * (TPB * 2u)), q);
-                };
-                if (nel == (u32)CH) {
-                    // all searches of a batch first (they only read), then the read-modify-writes
-#pragma unroll
-                    for (int f = 0; f < CH / 128; f += 2) {
-                        const float4 u4 = b4[lane + 32 * f], v4 = b4[lane + 32 * (f + 1)];
-                        const u32 p0 = find(u4.x), p1 = find(u4.y), p2 = find(u4.z), p3 = find(u4.w);
-                        const u32 p4 = find(v4.x), p5 = find(v4.y), p6 = find(v4.z), p7 = find(v4.w);
-                        add(p0, u4.x); add(p1, u4.y); add(p2, u4.z); add(p3, u4.w);
-                        add(p4, v4.x); add(p5, v4.y); add(p6, v4.z); add(p7, v4.w);
-                    }
-                } else {
-                    for (u32 f = lane; 4 * f < nel; f += 32) {
-                        const float4 v4 = b4[f];
-                        const u32 p0 = find(v4.x), p1 = find(v4.y), p2 = find(v4.z), p3 = find(v4.w);
-                        add(p0, v4.x);
-                        if (4 * f + 1 < nel) add(p1, v4.y);
-                        if (4 * f + 2 < nel) add(p2, v4.z);
-                        if (4 * f + 3 < nel) add(p3, v4.w);
-                    }
+                const float* data = ring.stage() + k * CH;
+                const float* bnd = sm.bnd[warp][k];
+                u32* hist = sm.hist[warp][k];
+                unsigned char* idp = ws.ids[stream0 + k] + (u64)tile * TILE + off;
+                for (u32 f = lane; 4 * f < nel; f += 32) {
+                    const float4 v = *reinterpret_cast<const float4*>(data + 4 * f);
+                    const u32 b0 = find_bucket(v.x, bnd), b1 = find_bucket(v.y, bnd);
+                    const u32 b2 = find_bucket(v.z, bnd), b3 = find_bucket(v.w, bnd);
+                    *reinterpret_cast<u32*>(idp + 4 * f) = b0 | (b1 << 8) | (b2 << 16) | (b3 << 24);
+                    atomicAdd(&hist[b0], 1u);
+                    if (4 * f + 1 < nel) atomicAdd(&hist[b1], 1u);
+                    if (4 * f + 2 < nel) atomicAdd(&hist[b2], 1u);
+                    if (4 * f + 3 < nel) atomicAdd(&hist[b3], 1u);
                 }
             }
             ring.advance();
-            if (++since >= 1024) flush(cur);
         }
     }
     if (cur >= 0) flush(cur);
 }
 
-// New centres from the sums of the finished sweep; one block per tensor, one
-// warp per stream.
-__global__ void __launch_bounds__(96) kmeans_update_kernel(TensorState* __restrict__ st) {
+// Where each bucket starts in the bucketed copy (exclusive prefix of the counts).
+__global__ void __launch_bounds__(NBKT) bucket_offsets_kernel(Workspace ws) {
+    __shared__ u32 wtot[NBKT / 32];
+    BucketStream& bk = ws.bst[blockIdx.x].s[blockIdx.y];
+    const int b = threadIdx.x, lane = b & 31, warp = b >> 5;
+    const u32 c = bk.cnt[b];
+    u32 incl = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const u32 v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) wtot[warp] = incl;
+    __syncthreads();
+    u32 base = 0;
+    for (int w = 0; w < warp; ++w) base += wtot[w];
+    bk.off[b] = base + incl - c;
+    bk.cursor[b] = base + incl - c;
+    if (b == NBKT - 1) bk.off[NBKT] = base + incl;
+}
+
+template <int NS, int CH>
+struct ScatterSmem {
+    float buf[BWARPS][BST][NS][CH];
+    unsigned long long bar[BWARPS][BST];
+    u32 pos[BWARPS][NS][NBKT];       // counts of the window, then the next free slot of each bucket
+    u32 slo[BWARPS][NS][NBKT];       // low and high 16-bit halves of the window's fixed-point sums
+    int shi[BWARPS][NS][NBKT];
+};
+
+// Sweep 2 of the grouping: survivors into their buckets, and each bucket's fixed-point sum.
+// A warp takes windows of at most 16 tiles of one tensor: it counts the window's survivors per
+// bucket (from the bucket bytes), reserves room in every bucket with one integer atomic per
+// bucket, and then streams the values through its ring into place.  (A window has at most
+// 65536 survivors, which keeps the 32-bit halves of the sums from overflowing.)
+template <int NS, int CH>
+__global__ void __launch_bounds__(TPB) bucket_scatter_kernel(const TensorDesc* __restrict__ descs,
+                                                             const TensorState* __restrict__ st, int nt,
+                                                             u32 tiles, Workspace ws, int stream0,
+                                                             CallState* call) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    ScatterSmem<NS, CH>& sm = *reinterpret_cast<ScatterSmem<NS, CH>*>(smem_raw);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const u32 gw = blockIdx.x * BWARPS + warp, nw = gridDim.x * BWARPS;
+    const u32 wlo = (u32)(((u64)tiles * gw) / nw), whi = (u32)(((u64)tiles * (gw + 1)) / nw);
+    SegRing<NS, CH, BST> ring;
+    ring.init(&sm.buf[warp][0][0][0], sm.bar[warp], lane, wlo, whi);
+    const u32* tile_cnt = stream0 == 0 ? ws.tile_cnt_w : ws.tile_cnt_o;
+    const float* surv[NS];
+#pragma unroll
+    for (int k = 0; k < NS; ++k) surv[k] = ws.surv[stream0 + k];
+    int cur = -1;
+    u32 tb = 0, ntl = 0;
+    float s1[NS], s2[NS];
+#pragma unroll
+    for (int k = 0; k < NS; ++k) s1[k] = s2[k] = 0.f;
+
+    for (;;) {
+        const u32 first = ring.next_start();
+        if (first >= whi) break;
+        if (cur < 0 || first >= tb + ntl) {
+            cur = find_tensor(descs, nt, first);
+            tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
+#pragma unroll
+            for (int k = 0; k < NS; ++k) { s1[k] = st[cur].s[stream0 + k].scale1; s2[k] = st[cur].s[stream0 + k].scale2; }
+        }
+        if (!ring.next_window(tile_cnt, lane, min(tb + ntl, first + 16u))) break;
+#pragma unroll
+        for (int k = 0; k < NS; ++k)
+            for (int b = lane; b < NBKT; b += 32) { sm.pos[warp][k][b] = 0; sm.slo[warp][k][b] = 0; sm.shi[warp][k][b] = 0; }
+        __syncwarp();
+        // survivors of the window per bucket
+        for (u32 i = 0; i < ring.wn; ++i) {
+            const u32 c = ring.cnt_of(i);
+#pragma unroll
+            for (int k = 0; k < NS; ++k) {
+                const unsigned char* idp = ws.ids[stream0 + k] + (u64)(ring.w0 + i) * TILE;
+                for (u32 j = lane * 4; j < c; j += 128) {
+                    const u32 w = *reinterpret_cast<const u32*>(idp + j);
+                    atomicAdd(&sm.pos[warp][k][w & 255u], 1u);
+                    if (j + 1 < c) atomicAdd(&sm.pos[warp][k][(w >> 8) & 255u], 1u);
+                    if (j + 2 < c) atomicAdd(&sm.pos[warp][k][(w >> 16) & 255u], 1u);
+                    if (j + 3 < c) atomicAdd(&sm.pos[warp][k][w >> 24], 1u);
+                }
+            }
+        }
+        __syncwarp();
+        // room for them: one integer atomic per bucket and stream
+#pragma unroll
+        for (int k = 0; k < NS; ++k)
+            for (int b = lane; b < NBKT; b += 32) {
+                const u32 c = sm.pos[warp][k][b];
+                sm.pos[warp][k][b] = c ? atomicAdd(&ws.bst[cur].s[stream0 + k].cursor[b], c) : 0u;
+            }
+        __syncwarp();
+        while (ring.have()) {
+            ring.issue_ahead(lane, surv);
+            const u32 tile = ring.tile(), nel = ring.nel(), off = ring.off();
+            if (!ring.wait()) {
+                if (lane == 0) atomicOr(&call->flags, FLAG_TIMEOUT);
+                return;
+            }
+#pragma unroll
+            for (int k = 0; k < NS; ++k) {
+                const float* data = ring.stage() + k * CH;
+                const unsigned char* idp = ws.ids[stream0 + k] + (u64)tile * TILE + off;
+                float* dst = ws.bkt[stream0 + k] + (u64)tb * TILE;
+                for (u32 f = lane; 4 * f < nel; f += 32) {
+                    const float4 v = *reinterpret_cast<const float4*>(data + 4 * f);
+                    const u32 w = *reinterpret_cast<const u32*>(idp + 4 * f);
+                    const float xs[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        if (4 * f + e < nel) {
+                            const u32 b = (w >> (8 * e)) & 255u;
+                            dst[atomicAdd(&sm.pos[warp][k][b], 1u)] = xs[e];
+                            const int q = __float2int_rn(__fmul_rn(__fmul_rn(xs[e], s1[k]), s2[k]));
+                            atomicAdd(&sm.slo[warp][k][b], (u32)q & 0xffffu);
+                            atomicAdd(&sm.shi[warp][k][b], q >> 16);
+                        }
+                    }
+                }
+            }
+            ring.advance();
+        }
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < NS; ++k)
+            for (int b = lane; b < NBKT; b += 32) {
+                const s64 s = (s64)sm.shi[warp][k][b] * 65536 + (s64)sm.slo[warp][k][b];
+                if (s) atomicAdd(reinterpret_cast<u64*>(&ws.bst[cur].s[stream0 + k].sum[b]), (u64)s);
+            }
+        __syncwarp();
+    }
+}
+
+// The bucket each threshold falls into; the partial sums of the coming scan start at zero.
+// Lanes 0..13 of one warp.
+__device__ inline void plan_scan(const StreamState& s, BucketStream& bk, int lane) {
+    if (lane < KMAX - 1) {
+        bk.bstar[lane] = find_bucket(s.thr[lane], bk.bnd);
+        bk.part_cnt[lane] = 0;
+        bk.part_sum[lane] = 0;
+    }
+}
+
+// Exclusive prefix of the bucket sums; plan of the first iteration.  Grid (tensors, 3).
+__global__ void __launch_bounds__(NBKT) bucket_prefix_kernel(const TensorState* __restrict__ st, Workspace ws) {
+    __shared__ s64 wtot[NBKT / 32];
+    BucketStream& bk = ws.bst[blockIdx.x].s[blockIdx.y];
+    const int b = threadIdx.x, lane = b & 31, warp = b >> 5;
+    const s64 c = bk.sum[b];
+    s64 incl = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const s64 v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) wtot[warp] = incl;
+    __syncthreads();
+    s64 base = 0;
+    for (int w = 0; w < warp; ++w) base += wtot[w];
+    bk.sumpre[b] = base + incl - c;
+    if (b == NBKT - 1) bk.sumpre[NBKT] = base + incl;
+    if (warp == 0) plan_scan(st[blockIdx.x].s[blockIdx.y], bk, lane);
+}
+
+// One iteration's data pass: for threshold j of a stream, the survivors of its bucket that lie
+// at or below it.  Grid (work items, 3 * 14): a tensor has scan_n items that split each bucket.
+__global__ void __launch_bounds__(TPB) bucket_scan_kernel(const TensorDesc* __restrict__ descs,
+                                                          const TensorState* __restrict__ st, int nt,
+                                                          Workspace ws) {
+    __shared__ s64 rsum[TPB / 32];
+    __shared__ u32 rcnt[TPB / 32];
+    int lo = 0, hi = nt - 1;                       // tensor that owns this work item
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (descs[mid].scan_first <= blockIdx.x) lo = mid; else hi = mid - 1;
+    }
+    const int t = lo, k = blockIdx.y / (KMAX - 1), j = blockIdx.y % (KMAX - 1);
+    const u32 split = blockIdx.x - descs[t].scan_first, nsplit = descs[t].scan_n;
+    BucketStream& bk = ws.bst[t].s[k];
+    const u32 b = bk.bstar[j];
+    const u32 b_lo = bk.off[b], n = bk.off[b + 1] - b_lo;
+    if (n == 0) return;
+    const u32 a = b_lo + (u32)(((u64)n * split) / nsplit), e = b_lo + (u32)(((u64)n * (split + 1)) / nsplit);
+    const StreamState& ss = st[t].s[k];
+    const float thr = ss.thr[j], s1 = ss.scale1, s2 = ss.scale2;
+    const float* data = ws.bkt[k] + (u64)descs[t].tile_begin * TILE;
+    u32 cnt = 0;
+    s64 sum = 0;
+    for (u32 i = a + threadIdx.x; i < e; i += TPB) {
+        const float x = data[i];
+        if (!(x > thr)) {
+            ++cnt;
+            sum += __float2int_rn(__fmul_rn(__fmul_rn(x, s1), s2));
+        }
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    cnt = __reduce_add_sync(0xffffffffu, cnt);
+#pragma unroll
+    for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if (lane == 0) { rcnt[warp] = cnt; rsum[warp] = sum; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        u64 c = 0; s64 s = 0;
+        for (int w = 0; w < TPB / 32; ++w) { c += rcnt[w]; s += rsum[w]; }
+        if (c) {
+            atomicAdd(&bk.part_cnt[j], c);
+            atomicAdd(reinterpret_cast<u64*>(&bk.part_sum[j]), (u64)s);
+        }
+    }
+}
+
+// New centres from the finished scan; one block per tensor, one warp per stream.
+// L_j = survivors at or below threshold j = whole buckets below its bucket + the scanned part;
+// cluster k has L_k - L_(k-1) members (L_-1 = 0, L_14 = all), and its sum likewise.
+__global__ void __launch_bounds__(96) bucket_update_kernel(TensorState* __restrict__ st, Workspace ws) {
     const int t = blockIdx.x, stream = threadIdx.x >> 5, lane = threadIdx.x & 31;
     StreamState& s = st[t].s[stream];
+    BucketStream& bk = ws.bst[t].s[stream];
+    u64 L = 0;
+    s64 S = 0;
+    if (lane < KMAX - 1) {
+        const u32 b = bk.bstar[lane];
+        L = (u64)bk.off[b] + bk.part_cnt[lane];
+        S = bk.sumpre[b] + bk.part_sum[lane];
+    } else if (lane == KMAX - 1) {
+        L = bk.off[NBKT];
+        S = bk.sumpre[NBKT];
+    }
+    const u64 Lp = __shfl_up_sync(0xffffffffu, L, 1);
+    const s64 Sp = __shfl_up_sync(0xffffffffu, S, 1);
+    const u64 n = lane == 0 ? L : L - Lp;
+    const s64 sum = lane == 0 ? S : S - Sp;
     float c = __uint_as_float(0x7f800000u);
     if (lane < KMAX) {
         c = s.cent[lane];
-        const u64 n = s.acc_cnt[lane];
         if (n) {
-            const double mean = __ll2double_rn(s.acc_sum[lane]) / __ull2double_rn(n);
+            const double mean = __ll2double_rn(sum) / __ull2double_rn(n);
             const double scale = __longlong_as_double((s64)(s.e - 30 + 1023) << 52);
             c = __double2float_rn(mean * scale);
         }
-        s.acc_sum[lane] = 0;
-        s.acc_cnt[lane] = 0;
     }
     // sort ascending: rank of each centre among the 15 (ties by lane)
     int rank = 0;
@@ -241,24 +449,38 @@ __global__ void __launch_bounds__(96) kmeans_update_kernel(TensorState* __restri
     if (lane < KMAX) s.cent[rank] = c;
     __syncwarp();
     set_thresholds(s, lane);
+    __syncwarp();
+    plan_scan(s, bk, lane);
 }
 
 void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
-                   const Workspace& ws, const Params& p, CallState* call) {
+                   u32 scan_items, const Workspace& ws, const Params& p, CallState* call) {
     kmeans_start_kernel<<<dim3(nt, 3), SAMPLE_MAX, 0, cfg.stream>>>(descs, st, ws, p.seed);
     prof_mark(cfg, ST_KMEANS_START, 1);
-    if (!tiles) return;
-    const u32 grid1 = min((tiles + LWARPS - 1) / LWARPS, (u32)cfg.sms * 3u);
-    const u32 grid2 = min((tiles + LWARPS - 1) / LWARPS, (u32)cfg.sms * 2u);
-    const size_t smem1 = sizeof(LloydSmem<1, 512>), smem2 = sizeof(LloydSmem<2, 256>);
-    cudaFuncSetAttribute(lloyd_pass_kernel<1, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1);
-    cudaFuncSetAttribute(lloyd_pass_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
+    if (!tiles || p.kmeans_iters == 0) return;
+    const u32 grid = min((tiles + BWARPS - 1) / BWARPS, (u32)cfg.sms * 3u);
+    {
+        const size_t m1 = sizeof(BucketIdsSmem<1, 512>), m2 = sizeof(BucketIdsSmem<2, 256>);
+        cudaFuncSetAttribute(bucket_ids_kernel<1, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m1);
+        cudaFuncSetAttribute(bucket_ids_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m2);
+        bucket_ids_kernel<1, 512><<<grid, TPB, m1, cfg.stream>>>(descs, nt, tiles, ws, 0, call);
+        bucket_ids_kernel<2, 256><<<grid, TPB, m2, cfg.stream>>>(descs, nt, tiles, ws, 1, call);
+        prof_mark(cfg, ST_BUCKET_IDS, 2);
+    }
+    bucket_offsets_kernel<<<dim3(nt, 3), NBKT, 0, cfg.stream>>>(ws);
+    {
+        const size_t m1 = sizeof(ScatterSmem<1, 512>), m2 = sizeof(ScatterSmem<2, 256>);
+        cudaFuncSetAttribute(bucket_scatter_kernel<1, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m1);
+        cudaFuncSetAttribute(bucket_scatter_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m2);
+        bucket_scatter_kernel<1, 512><<<grid, TPB, m1, cfg.stream>>>(descs, st, nt, tiles, ws, 0, call);
+        bucket_scatter_kernel<2, 256><<<grid, TPB, m2, cfg.stream>>>(descs, st, nt, tiles, ws, 1, call);
+    }
+    bucket_prefix_kernel<<<dim3(nt, 3), NBKT, 0, cfg.stream>>>(st, ws);
+    prof_mark(cfg, ST_BUCKET_SCATTER, 4);
     for (int it = 0; it < p.kmeans_iters; ++it) {
-        lloyd_pass_kernel<1, 512><<<grid1, TPB, smem1, cfg.stream>>>(descs, st, nt, tiles, ws, 0, call);
-        prof_mark(cfg, ST_LLOYD_W, 1);
-        lloyd_pass_kernel<2, 256><<<grid2, TPB, smem2, cfg.stream>>>(descs, st, nt, tiles, ws, 1, call);
-        prof_mark(cfg, ST_LLOYD_EA, 1);
-        kmeans_update_kernel<<<nt, 96, 0, cfg.stream>>>(st);
+        bucket_scan_kernel<<<dim3(scan_items, 3 * (KMAX - 1)), TPB, 0, cfg.stream>>>(descs, st, nt, ws);
+        prof_mark(cfg, ST_BUCKET_SCAN, 1);
+        bucket_update_kernel<<<nt, 96, 0, cfg.stream>>>(st, ws);
         prof_mark(cfg, ST_KMEANS_UPDATE, 1);
     }
 }

@@ -133,7 +133,6 @@ __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __res
     const float* surv[NS];
 #pragma unroll
     for (int k = 0; k < NS; ++k) surv[k] = ws.surv[stream0 + k];
-    constexpr u32 ROWS = CH / 8;
 
     int cur = -1;
     u32 tb = 0, ntl = 0;
@@ -145,7 +144,7 @@ __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __res
 #pragma unroll
     for (int k = 0; k < NS; ++k) carry[k] = 0;
 
-    for (bool first = true; ring.next_window(tile_cnt, lane, first); first = false) {
+    while (ring.next_window(tile_cnt, lane, whi)) {
         while (ring.have()) {
             ring.issue_ahead(lane, surv);
             const u32 tile = ring.tile();

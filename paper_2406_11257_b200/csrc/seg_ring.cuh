@@ -17,7 +17,7 @@ struct SegRing {
     float* buf;
     unsigned long long* bar;
     u32 whi;                       // end of the warp's run of tiles
-    u32 w0;                        // first tile of the current window of 32
+    u32 w0, wn;                    // current window: tiles [w0, w0 + wn), wn <= 32
     u32 mycnt;                     // count of tile w0 + lane (0 past the run)
     u32 nz;                        // lanes whose tile has survivors
     u32 it, i_cnt, ic;             // issue cursor: tile in the window (32 = done), its count, value offset
@@ -25,7 +25,7 @@ struct SegRing {
     u32 i_stage, c_stage, c_phase, inflight;
 
     __device__ void init(float* b, unsigned long long* r, int lane, u32 wlo, u32 whi_) {
-        buf = b; bar = r; whi = whi_; w0 = wlo;
+        buf = b; bar = r; whi = whi_; w0 = wlo; wn = 0;
         i_stage = c_stage = c_phase = inflight = 0;
         it = ct = 32; i_cnt = c_cnt = ic = cc = 0; mycnt = 0; nz = 0;
         if (lane == 0) {
@@ -39,11 +39,15 @@ struct SegRing {
         const u32 m = i >= 31 ? 0u : nz & (0xffffffffu << (i + 1));
         return m ? (u32)__ffs((int)m) - 1u : 32u;
     }
-    // Loads the next window; false when the run is finished.  `first` on the first call.
-    __device__ bool next_window(const u32* __restrict__ tile_cnt, int lane, bool first) {
-        if (!first) w0 += 32;
-        if (w0 >= whi) return false;
-        mycnt = w0 + lane < whi ? tile_cnt[w0 + lane] : 0u;
+    __device__ u32 next_start() const { return w0 + wn; }
+    __device__ u32 cnt_of(u32 i) const { return __shfl_sync(0xffffffffu, mycnt, i); }   // tile i of the window
+    // Loads the next window, which ends before `limit` (and before the end of the run, and after
+    // at most 32 tiles); false when the run is finished.
+    __device__ bool next_window(const u32* __restrict__ tile_cnt, int lane, u32 limit) {
+        w0 += wn;
+        if (w0 >= whi) { wn = 0; return false; }
+        wn = min(32u, min(limit, whi) - w0);
+        mycnt = (u32)lane < wn ? tile_cnt[w0 + lane] : 0u;
         nz = __ballot_sync(0xffffffffu, mycnt != 0);
         it = ct = next_tile(-1);
         i_cnt = c_cnt = it < 32 ? __shfl_sync(0xffffffffu, mycnt, it) : 0u;
