@@ -251,8 +251,8 @@ def run_ours(args):
         "stats1": (src_b + 4) * n_tot,
         "stats2": src_b * n_tot,
         "mask_compact": 16 * n_tot + n_tot / 4 + 4 * surv,
-        "bucket_ids": 5 * surv,                     # survivors read, one bucket byte each written
-        "bucket_scatter": 10 * surv,                # bucket bytes read twice, survivors read and written
+        "bucket_ids": 4 * surv,                     # survivors read once to count them per bucket
+        "bucket_scatter": 8 * surv,                 # survivors read and written into their buckets
         "bucket_scan": T * 4 * surv * 14 / 256,     # about 14 of 256 buckets per iteration
         "pack_codes": 4.5 * surv,
         "copy_bitmaps": n_tot / 2,

@@ -237,7 +237,6 @@ excp_status excp_create(excp_handle* out, int device, size_t workspace_numel) {
         for (int k = 0; k < 3 && ok; ++k) {
             ok = check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.surv[k]), elems * sizeof(float)));
             ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.bkt[k]), elems * sizeof(float)));
-            ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.ids[k]), elems));
         }
         ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.bst), MAX_GROUP_TENSORS * sizeof(BucketState)));
         ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.bm_w), elems / 8));
@@ -266,7 +265,6 @@ excp_status excp_destroy(excp_handle h) {
     for (int k = 0; k < 3; ++k) {
         if (h->ws.surv[k]) cudaFree(h->ws.surv[k]);
         if (h->ws.bkt[k]) cudaFree(h->ws.bkt[k]);
-        if (h->ws.ids[k]) cudaFree(h->ws.ids[k]);
     }
     if (h->ws.bst) cudaFree(h->ws.bst);
     if (h->ws.bm_w) cudaFree(h->ws.bm_w);

@@ -93,8 +93,15 @@ struct CallState {               // one per handle, device resident
 
 constexpr int NBKT = 256;         // value buckets per tensor and stream for the K-means iterations
 
-struct BucketStream {            // one stream's buckets: bucket b holds bnd[b-1] < x <= bnd[b]
-    float bnd[NBKT];             // upper bounds, ascending; bnd[255] = +inf
+struct BucketFn {                // a monotone map of fp32 values to 0..255 (see bucket_of)
+    u32 lo;                      // magnitude bit pattern mapped to the first step
+    u32 shift;                   // magnitude bit patterns per step = 2^shift
+    u32 sgn;                     // 1: 128 steps per sign; 0: 256 steps, non-negative values
+    u32 pad_;
+};
+
+struct BucketStream {            // one stream's buckets
+    BucketFn fn;
     u32 cnt[NBKT];               // survivors per bucket
     s64 sum[NBKT];               // their fixed-point sums
     u32 off[NBKT + 1];           // exclusive prefix of cnt = start of each bucket in the bucketed copy
@@ -111,7 +118,6 @@ struct BucketState {
 
 struct Workspace {               // device arrays sized for cap_tiles tiles
     float* bkt[3];               // survivors again, grouped by value bucket (order inside a bucket is arbitrary)
-    unsigned char* ids[3];       // bucket of each survivor, at the survivor's place in surv[]
     BucketState* bst;            // per tensor of the group
     float* surv[3];              // survivors, each tile's compacted at the tile's own start
     u32* bm_w;                   // bitmaps, TILE_WORDS words per tile
@@ -161,6 +167,19 @@ __host__ __device__ inline u64 record_bytes(u64 numel, u64 nnz_w, u64 nnz_o, int
 
 // ---- device helpers ---------------------------------------------------------
 #ifdef __CUDACC__
+// Bucket of a value: steps of equal width in the bit pattern of |x| (so roughly logarithmic
+// in |x|), clamped at both ends, negative values mirrored below the positive ones.  All that
+// the K-means iterations need of it is that it never decreases when x grows.
+__device__ __forceinline__ u32 bucket_of(float x, const BucketFn& f) {
+    const u32 bits = __float_as_uint(x), a = bits & 0x7fffffffu;
+    u32 m = a > f.lo ? (a - f.lo) >> f.shift : 0u;
+    if (f.sgn) {
+        m = min(m, (u32)NBKT / 2 - 1);
+        return (bits >> 31) ? NBKT / 2 - 1 - m : NBKT / 2 + m;
+    }
+    return min(m, (u32)NBKT - 1);
+}
+
 // Tensor that owns group tile `tile` (descs are in tile order).
 __device__ inline int find_tensor(const TensorDesc* __restrict__ descs, int n, u32 tile) {
     int lo = 0, hi = n - 1;

@@ -12,13 +12,13 @@
 //
 // The iterations do not sweep the survivors.  Because the clusters are intervals
 // and the sums are integers, the survivors are first grouped ONCE into 256 value
-// buckets (bounds taken from the sorted start sample, so the buckets hold about
-// the same number each) with each bucket's count and sum.  An iteration then
+// buckets (a cheap monotone function of the value, scaled to the range of the
+// start sample) with each bucket's count and sum.  An iteration then
 // needs, per threshold, only the bucket the threshold falls into: buckets below
-// it count whole, and the one bucket is scanned.  That is about 14/256 of the
+// it count whole, and the one bucket is scanned.  That is a small part of the
 // data per iteration, and the sums are exactly those of a full sweep.
 //
-//   bucket_ids      sweep: bucket of every survivor (8-step search), counts
+//   bucket_count    sweep: survivors per bucket
 //   bucket_offsets  prefix of the counts -> where each bucket starts
 //   bucket_scatter  sweep: survivors into their buckets, bucket sums
 //   bucket_prefix   prefix of the sums; first plan
@@ -50,6 +50,7 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
                                                                   TensorState* __restrict__ st,
                                                                   Workspace ws, u64 seed) {
     __shared__ float smp[SAMPLE_MAX];
+    __shared__ u32 amin, amax;                        // smallest / largest magnitude pattern in the sample
     const int t = blockIdx.x, stream = blockIdx.y, tid = threadIdx.x;
     StreamState& s = st[t].s[stream];
     const u32 nnz = stream == 0 ? st[t].nnz_w : st[t].nnz_o;
@@ -59,7 +60,7 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
     BucketStream& bk = ws.bst[t].s[stream];
     if (nnz == 0) {
         if (tid < KPAD) { s.cent[tid] = 0.f; s.thr[tid] = __uint_as_float(0x7f800000u); }
-        if (tid < NBKT) bk.bnd[tid] = __uint_as_float(0x7f800000u);
+        if (tid == 0) { bk.fn.lo = 0; bk.fn.shift = 0; bk.fn.sgn = stream != 2; }
         return;
     }
     const u32 m = min(nnz, (u32)SAMPLE_MAX);
@@ -78,7 +79,12 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
         v = data[(u64)a * TILE + (r - toff[a])];
     }
     smp[tid] = v;
+    if (tid == 0) { amin = 0x7fffffffu; amax = 0u; }
     __syncthreads();
+    if ((u32)tid < m) {
+        atomicMin(&amin, __float_as_uint(v) & 0x7fffffffu);
+        atomicMax(&amax, __float_as_uint(v) & 0x7fffffffu);
+    }
     for (int k = 2; k <= SAMPLE_MAX; k <<= 1) {       // bitonic sort, ascending
         for (int j = k >> 1; j > 0; j >>= 1) {
             const int p = tid ^ j;
@@ -91,42 +97,36 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
         }
     }
     if (tid < KPAD) s.cent[tid] = tid < KMAX ? smp[((2 * tid + 1) * m) / (2 * KMAX)] : 0.f;
-    // bucket bounds: every (m/256)-th sample value; any ascending values would do, these
-    // make the buckets about equally full
-    if (tid < NBKT) bk.bnd[tid] = tid < NBKT - 1 ? smp[((u32)(tid + 1) * m) / NBKT] : __uint_as_float(0x7f800000u);
+    // bucket function: its steps span the magnitudes seen in the sample (any monotone map
+    // would give the same centres; this one spreads these survivors over the 256 buckets)
+    if (tid == 0) {
+        const u32 d = amax - amin;
+        const int half_bits = stream != 2 ? 7 : 8;            // log2 of the steps per sign
+        const int len = 32 - __clz(d);                        // d < 2^len
+        bk.fn.lo = amin; bk.fn.shift = len > half_bits ? len - half_bits : 0; bk.fn.sgn = stream != 2;
+    }
     __syncthreads();
     if (tid < 32) set_thresholds(s, tid);
 }
 
 
 // ---------------------------------------------------------------------------
-// Buckets.  bucket(x) = number of bounds strictly below x (bounds ascending, the last +inf),
-// so bucket b holds bnd[b-1] < x <= bnd[b].
-__device__ __forceinline__ u32 find_bucket(float x, const float* bnd) {
-    u32 b = 0;
-#pragma unroll
-    for (int step = NBKT / 2; step; step >>= 1) b += (x > bnd[b + step - 1]) ? (u32)step : 0u;
-    return b;
-}
-
 constexpr int BWARPS = TPB / 32;
 constexpr int BST = 2;               // stages per warp
 
 template <int NS, int CH>
-struct BucketIdsSmem {
+struct BucketCountSmem {
     float buf[BWARPS][BST][NS][CH];
     unsigned long long bar[BWARPS][BST];
-    float bnd[BWARPS][NS][NBKT];     // each warp's copy of its tensor's bounds
     u32 hist[BWARPS][NS][NBKT];      // each warp's counts since its last flush
 };
 
-// Sweep 1 of the grouping: the bucket of every survivor (one byte, stored at the survivor's
-// own place) and the survivors per bucket.  NS = 1: dW; NS = 2: both moment streams.
+// Sweep 1 of the grouping: survivors per bucket.  NS = 1: dW; NS = 2: both moment streams.
 template <int NS, int CH>
-__global__ void __launch_bounds__(TPB) bucket_ids_kernel(const TensorDesc* __restrict__ descs, int nt, u32 tiles,
-                                                         Workspace ws, int stream0, CallState* call) {
+__global__ void __launch_bounds__(TPB) bucket_count_kernel(const TensorDesc* __restrict__ descs, int nt, u32 tiles,
+                                                           Workspace ws, int stream0, CallState* call) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    BucketIdsSmem<NS, CH>& sm = *reinterpret_cast<BucketIdsSmem<NS, CH>*>(smem_raw);
+    BucketCountSmem<NS, CH>& sm = *reinterpret_cast<BucketCountSmem<NS, CH>*>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const u32 gw = blockIdx.x * BWARPS + warp, nw = gridDim.x * BWARPS;
     const u32 wlo = (u32)(((u64)tiles * gw) / nw), whi = (u32)(((u64)tiles * (gw + 1)) / nw);
@@ -134,9 +134,11 @@ __global__ void __launch_bounds__(TPB) bucket_ids_kernel(const TensorDesc* __res
     ring.init(&sm.buf[warp][0][0][0], sm.bar[warp], lane, wlo, whi);
     const u32* tile_cnt = stream0 == 0 ? ws.tile_cnt_w : ws.tile_cnt_o;
     const float* surv[NS];
+    BucketFn fn[NS];
 #pragma unroll
     for (int k = 0; k < NS; ++k) {
         surv[k] = ws.surv[stream0 + k];
+        fn[k] = BucketFn{0, 0, 0, 0};
         for (int b = lane; b < NBKT; b += 32) sm.hist[warp][k][b] = 0;
     }
     __syncwarp();
@@ -163,11 +165,9 @@ __global__ void __launch_bounds__(TPB) bucket_ids_kernel(const TensorDesc* __res
                 cur = find_tensor(descs, nt, tile);
                 tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
 #pragma unroll
-                for (int k = 0; k < NS; ++k)
-                    for (int b = lane; b < NBKT; b += 32) sm.bnd[warp][k][b] = ws.bst[cur].s[stream0 + k].bnd[b];
-                __syncwarp();
+                for (int k = 0; k < NS; ++k) fn[k] = ws.bst[cur].s[stream0 + k].fn;
             }
-            const u32 nel = ring.nel(), off = ring.off();
+            const u32 nel = ring.nel();
             if (!ring.wait()) {
                 if (lane == 0) atomicOr(&call->flags, FLAG_TIMEOUT);
                 return;
@@ -175,18 +175,13 @@ __global__ void __launch_bounds__(TPB) bucket_ids_kernel(const TensorDesc* __res
 #pragma unroll
             for (int k = 0; k < NS; ++k) {
                 const float* data = ring.stage() + k * CH;
-                const float* bnd = sm.bnd[warp][k];
                 u32* hist = sm.hist[warp][k];
-                unsigned char* idp = ws.ids[stream0 + k] + (u64)tile * TILE + off;
                 for (u32 f = lane; 4 * f < nel; f += 32) {
                     const float4 v = *reinterpret_cast<const float4*>(data + 4 * f);
-                    const u32 b0 = find_bucket(v.x, bnd), b1 = find_bucket(v.y, bnd);
-                    const u32 b2 = find_bucket(v.z, bnd), b3 = find_bucket(v.w, bnd);
-                    *reinterpret_cast<u32*>(idp + 4 * f) = b0 | (b1 << 8) | (b2 << 16) | (b3 << 24);
-                    atomicAdd(&hist[b0], 1u);
-                    if (4 * f + 1 < nel) atomicAdd(&hist[b1], 1u);
-                    if (4 * f + 2 < nel) atomicAdd(&hist[b2], 1u);
-                    if (4 * f + 3 < nel) atomicAdd(&hist[b3], 1u);
+                    atomicAdd(&hist[bucket_of(v.x, fn[k])], 1u);
+                    if (4 * f + 1 < nel) atomicAdd(&hist[bucket_of(v.y, fn[k])], 1u);
+                    if (4 * f + 2 < nel) atomicAdd(&hist[bucket_of(v.z, fn[k])], 1u);
+                    if (4 * f + 3 < nel) atomicAdd(&hist[bucket_of(v.w, fn[k])], 1u);
                 }
             }
             ring.advance();
@@ -216,118 +211,116 @@ __global__ void __launch_bounds__(NBKT) bucket_offsets_kernel(Workspace ws) {
     if (b == NBKT - 1) bk.off[NBKT] = base + incl;
 }
 
-template <int NS, int CH>
+constexpr int SCAP = 12288;          // survivors staged per window of tiles
+
 struct ScatterSmem {
-    float buf[BWARPS][BST][NS][CH];
-    unsigned long long bar[BWARPS][BST];
-    u32 pos[BWARPS][NS][NBKT];       // counts of the window, then the next free slot of each bucket
-    u32 slo[BWARPS][NS][NBKT];       // low and high 16-bit halves of the window's fixed-point sums
-    int shi[BWARPS][NS][NBKT];
+    float val[SCAP];                 // the window's survivors sorted by bucket
+    unsigned char bid[SCAP];         // and their buckets
+    u32 cnt[NBKT];                   // survivors of the window per bucket
+    u32 loff[NBKT];                  // start of each bucket in val[]
+    u32 lcur[NBKT];                  // next free place of each bucket in val[]
+    u32 gbase[NBKT];                 // room reserved for the bucket in the bucketed copy
+    u32 slo[NBKT];                   // low and high 16-bit halves of the window's fixed-point sums
+    int shi[NBKT];
+    u32 pre[33];                     // survivors before tile i of the window
+    u32 wtot[TPB / 32];
+    u32 wn;                          // tiles in the window
 };
 
 // Sweep 2 of the grouping: survivors into their buckets, and each bucket's fixed-point sum.
-// A warp takes windows of at most 16 tiles of one tensor: it counts the window's survivors per
-// bucket (from the bucket bytes), reserves room in every bucket with one integer atomic per
-// bucket, and then streams the values through its ring into place.  (A window has at most
-// 65536 survivors, which keeps the 32-bit halves of the sums from overflowing.)
-template <int NS, int CH>
-__global__ void __launch_bounds__(TPB) bucket_scatter_kernel(const TensorDesc* __restrict__ descs,
-                                                             const TensorState* __restrict__ st, int nt,
-                                                             u32 tiles, Workspace ws, int stream0,
-                                                             CallState* call) {
+// A block takes windows of tiles of one tensor holding at most SCAP survivors: it counts them
+// per bucket, reserves room in every bucket of the bucketed copy with one integer atomic,
+// sorts the window by bucket in shared memory and writes each bucket's run with consecutive
+// threads (one 4-byte store per survivor straight to its bucket would be bound by the number
+// of write requests, not by bytes).
+__global__ void __launch_bounds__(TPB, 3) bucket_scatter_kernel(const TensorDesc* __restrict__ descs,
+                                                                const TensorState* __restrict__ st, int nt,
+                                                                u32 tiles, Workspace ws, int stream) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    ScatterSmem<NS, CH>& sm = *reinterpret_cast<ScatterSmem<NS, CH>*>(smem_raw);
+    ScatterSmem& sm = *reinterpret_cast<ScatterSmem*>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const u32 gw = blockIdx.x * BWARPS + warp, nw = gridDim.x * BWARPS;
-    const u32 wlo = (u32)(((u64)tiles * gw) / nw), whi = (u32)(((u64)tiles * (gw + 1)) / nw);
-    SegRing<NS, CH, BST> ring;
-    ring.init(&sm.buf[warp][0][0][0], sm.bar[warp], lane, wlo, whi);
-    const u32* tile_cnt = stream0 == 0 ? ws.tile_cnt_w : ws.tile_cnt_o;
-    const float* surv[NS];
-#pragma unroll
-    for (int k = 0; k < NS; ++k) surv[k] = ws.surv[stream0 + k];
+    u32 lo, hi;
+    block_range(tiles, lo, hi);
+    const u32* tile_cnt = stream == 0 ? ws.tile_cnt_w : ws.tile_cnt_o;
+    const float* surv = ws.surv[stream];
     int cur = -1;
     u32 tb = 0, ntl = 0;
-    float s1[NS], s2[NS];
-#pragma unroll
-    for (int k = 0; k < NS; ++k) s1[k] = s2[k] = 0.f;
-
-    for (;;) {
-        const u32 first = ring.next_start();
-        if (first >= whi) break;
-        if (cur < 0 || first >= tb + ntl) {
-            cur = find_tensor(descs, nt, first);
+    BucketFn fn = BucketFn{0, 0, 0, 0};
+    float s1 = 0.f, s2 = 0.f;
+    u32 tile = lo;
+    while (tile < hi) {
+        if (cur < 0 || tile >= tb + ntl) {
+            cur = find_tensor(descs, nt, tile);
             tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
-#pragma unroll
-            for (int k = 0; k < NS; ++k) { s1[k] = st[cur].s[stream0 + k].scale1; s2[k] = st[cur].s[stream0 + k].scale2; }
+            fn = ws.bst[cur].s[stream].fn;
+            s1 = st[cur].s[stream].scale1; s2 = st[cur].s[stream].scale2;
         }
-        if (!ring.next_window(tile_cnt, lane, min(tb + ntl, first + 16u))) break;
+        const u32 wend = min(hi, tb + ntl);
+        if (warp == 0) {              // the window: leading tiles whose survivors fit the stage
+            const u32 c = tile + lane < wend ? tile_cnt[tile + lane] : 0u;
+            u32 incl = c;
 #pragma unroll
-        for (int k = 0; k < NS; ++k)
-            for (int b = lane; b < NBKT; b += 32) { sm.pos[warp][k][b] = 0; sm.slo[warp][k][b] = 0; sm.shi[warp][k][b] = 0; }
-        __syncwarp();
-        // survivors of the window per bucket
-        for (u32 i = 0; i < ring.wn; ++i) {
-            const u32 c = ring.cnt_of(i);
+            for (int o = 1; o < 32; o <<= 1) {
+                const u32 v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            const u32 ok = __ballot_sync(0xffffffffu, tile + lane < wend && incl <= (u32)SCAP);
+            sm.pre[lane] = incl - c;
+            if (lane == 31) sm.pre[32] = incl;
+            if (lane == 0) sm.wn = ok == 0xffffffffu ? 32u : (u32)__ffs((int)~ok) - 1u;
+        }
+        sm.cnt[tid] = 0; sm.slo[tid] = 0; sm.shi[tid] = 0;
+        __syncthreads();
+        const u32 wn = sm.wn, total = sm.pre[wn];
+        if (total) {
+            for (u32 i = 0; i < wn; ++i) {
+                const u32 c = sm.pre[i + 1] - sm.pre[i];
+                const float* data = surv + (u64)(tile + i) * TILE;
+                for (u32 e = tid; e < c; e += TPB) atomicAdd(&sm.cnt[bucket_of(data[e], fn)], 1u);
+            }
+            __syncthreads();
+            {                          // exclusive prefix of the counts; room in the bucketed copy
+                const u32 c = sm.cnt[tid];
+                u32 incl = c;
 #pragma unroll
-            for (int k = 0; k < NS; ++k) {
-                const unsigned char* idp = ws.ids[stream0 + k] + (u64)(ring.w0 + i) * TILE;
-                for (u32 j = lane * 4; j < c; j += 128) {
-                    const u32 w = *reinterpret_cast<const u32*>(idp + j);
-                    atomicAdd(&sm.pos[warp][k][w & 255u], 1u);
-                    if (j + 1 < c) atomicAdd(&sm.pos[warp][k][(w >> 8) & 255u], 1u);
-                    if (j + 2 < c) atomicAdd(&sm.pos[warp][k][(w >> 16) & 255u], 1u);
-                    if (j + 3 < c) atomicAdd(&sm.pos[warp][k][w >> 24], 1u);
+                for (int o = 1; o < 32; o <<= 1) {
+                    const u32 v = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += v;
+                }
+                if (lane == 31) sm.wtot[warp] = incl;
+                __syncthreads();
+                u32 base = 0;
+                for (int w = 0; w < warp; ++w) base += sm.wtot[w];
+                sm.loff[tid] = base + incl - c;
+                sm.lcur[tid] = base + incl - c;
+                sm.gbase[tid] = c ? atomicAdd(&ws.bst[cur].s[stream].cursor[tid], c) : 0u;
+            }
+            __syncthreads();
+            for (u32 i = 0; i < wn; ++i) {
+                const u32 c = sm.pre[i + 1] - sm.pre[i];
+                const float* data = surv + (u64)(tile + i) * TILE;
+                for (u32 e = tid; e < c; e += TPB) {
+                    const float x = data[e];
+                    const u32 b = bucket_of(x, fn);
+                    const u32 r = atomicAdd(&sm.lcur[b], 1u);
+                    sm.val[r] = x;
+                    sm.bid[r] = (unsigned char)b;
+                    const int q = __float2int_rn(__fmul_rn(__fmul_rn(x, s1), s2));
+                    atomicAdd(&sm.slo[b], (u32)q & 0xffffu);
+                    atomicAdd(&sm.shi[b], q >> 16);
                 }
             }
+            __syncthreads();
+            float* dst = ws.bkt[stream] + (u64)tb * TILE;
+            for (u32 i = tid; i < total; i += TPB) {
+                const u32 b = sm.bid[i];
+                dst[sm.gbase[b] + (i - sm.loff[b])] = sm.val[i];
+            }
+            const s64 sum = (s64)sm.shi[tid] * 65536 + (s64)sm.slo[tid];
+            if (sum) atomicAdd(reinterpret_cast<u64*>(&ws.bst[cur].s[stream].sum[tid]), (u64)sum);
         }
-        __syncwarp();
-        // room for them: one integer atomic per bucket and stream
-#pragma unroll
-        for (int k = 0; k < NS; ++k)
-            for (int b = lane; b < NBKT; b += 32) {
-                const u32 c = sm.pos[warp][k][b];
-                sm.pos[warp][k][b] = c ? atomicAdd(&ws.bst[cur].s[stream0 + k].cursor[b], c) : 0u;
-            }
-        __syncwarp();
-        while (ring.have()) {
-            ring.issue_ahead(lane, surv);
-            const u32 tile = ring.tile(), nel = ring.nel(), off = ring.off();
-            if (!ring.wait()) {
-                if (lane == 0) atomicOr(&call->flags, FLAG_TIMEOUT);
-                return;
-            }
-#pragma unroll
-            for (int k = 0; k < NS; ++k) {
-                const float* data = ring.stage() + k * CH;
-                const unsigned char* idp = ws.ids[stream0 + k] + (u64)tile * TILE + off;
-                float* dst = ws.bkt[stream0 + k] + (u64)tb * TILE;
-                for (u32 f = lane; 4 * f < nel; f += 32) {
-                    const float4 v = *reinterpret_cast<const float4*>(data + 4 * f);
-                    const u32 w = *reinterpret_cast<const u32*>(idp + 4 * f);
-                    const float xs[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        if (4 * f + e < nel) {
-                            const u32 b = (w >> (8 * e)) & 255u;
-                            dst[atomicAdd(&sm.pos[warp][k][b], 1u)] = xs[e];
-                            const int q = __float2int_rn(__fmul_rn(__fmul_rn(xs[e], s1[k]), s2[k]));
-                            atomicAdd(&sm.slo[warp][k][b], (u32)q & 0xffffu);
-                            atomicAdd(&sm.shi[warp][k][b], q >> 16);
-                        }
-                    }
-                }
-            }
-            ring.advance();
-        }
-        __syncwarp();
-#pragma unroll
-        for (int k = 0; k < NS; ++k)
-            for (int b = lane; b < NBKT; b += 32) {
-                const s64 s = (s64)sm.shi[warp][k][b] * 65536 + (s64)sm.slo[warp][k][b];
-                if (s) atomicAdd(reinterpret_cast<u64*>(&ws.bst[cur].s[stream0 + k].sum[b]), (u64)s);
-            }
-        __syncwarp();
+        tile += wn;
+        __syncthreads();
     }
 }
 
@@ -335,7 +328,7 @@ __global__ void __launch_bounds__(TPB) bucket_scatter_kernel(const TensorDesc* _
 // Lanes 0..13 of one warp.
 __device__ inline void plan_scan(const StreamState& s, BucketStream& bk, int lane) {
     if (lane < KMAX - 1) {
-        bk.bstar[lane] = find_bucket(s.thr[lane], bk.bnd);
+        bk.bstar[lane] = bucket_of(s.thr[lane], bk.fn);
         bk.part_cnt[lane] = 0;
         bk.part_sum[lane] = 0;
     }
@@ -460,23 +453,22 @@ void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* s
     if (!tiles || p.kmeans_iters == 0) return;
     const u32 grid = min((tiles + BWARPS - 1) / BWARPS, (u32)cfg.sms * 3u);
     {
-        const size_t m1 = sizeof(BucketIdsSmem<1, 512>), m2 = sizeof(BucketIdsSmem<2, 256>);
-        cudaFuncSetAttribute(bucket_ids_kernel<1, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m1);
-        cudaFuncSetAttribute(bucket_ids_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m2);
-        bucket_ids_kernel<1, 512><<<grid, TPB, m1, cfg.stream>>>(descs, nt, tiles, ws, 0, call);
-        bucket_ids_kernel<2, 256><<<grid, TPB, m2, cfg.stream>>>(descs, nt, tiles, ws, 1, call);
+        const size_t m1 = sizeof(BucketCountSmem<1, 512>), m2 = sizeof(BucketCountSmem<2, 256>);
+        cudaFuncSetAttribute(bucket_count_kernel<1, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m1);
+        cudaFuncSetAttribute(bucket_count_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m2);
+        bucket_count_kernel<1, 512><<<grid, TPB, m1, cfg.stream>>>(descs, nt, tiles, ws, 0, call);
+        bucket_count_kernel<2, 256><<<grid, TPB, m2, cfg.stream>>>(descs, nt, tiles, ws, 1, call);
         prof_mark(cfg, ST_BUCKET_IDS, 2);
     }
     bucket_offsets_kernel<<<dim3(nt, 3), NBKT, 0, cfg.stream>>>(ws);
     {
-        const size_t m1 = sizeof(ScatterSmem<1, 512>), m2 = sizeof(ScatterSmem<2, 256>);
-        cudaFuncSetAttribute(bucket_scatter_kernel<1, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m1);
-        cudaFuncSetAttribute(bucket_scatter_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m2);
-        bucket_scatter_kernel<1, 512><<<grid, TPB, m1, cfg.stream>>>(descs, st, nt, tiles, ws, 0, call);
-        bucket_scatter_kernel<2, 256><<<grid, TPB, m2, cfg.stream>>>(descs, st, nt, tiles, ws, 1, call);
+        const u32 sgrid = min(tiles, (u32)cfg.sms * 3u);
+        cudaFuncSetAttribute(bucket_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ScatterSmem));
+        for (int k = 0; k < 3; ++k)
+            bucket_scatter_kernel<<<sgrid, TPB, sizeof(ScatterSmem), cfg.stream>>>(descs, st, nt, tiles, ws, k);
     }
     bucket_prefix_kernel<<<dim3(nt, 3), NBKT, 0, cfg.stream>>>(st, ws);
-    prof_mark(cfg, ST_BUCKET_SCATTER, 4);
+    prof_mark(cfg, ST_BUCKET_SCATTER, 5);
     for (int it = 0; it < p.kmeans_iters; ++it) {
         bucket_scan_kernel<<<dim3(scan_items, 3 * (KMAX - 1)), TPB, 0, cfg.stream>>>(descs, st, nt, ws);
         prof_mark(cfg, ST_BUCKET_SCAN, 1);
