@@ -186,6 +186,32 @@ excp_status excp_decompress_checkpoint(excp_handle h, const void* blob, const si
                                        float* const* w_out, float* const* ea_out, float* const* eas_out,
                                        void* cuda_stream);
 
+/* excp_decompress_tensor for callers that cannot allocate memory (the paper has no counterpart:
+ * this is a property of the library, not of the method).
+ *
+ * It takes no handle and calls no allocating routine.  The little scratch memory that decoding
+ * needs (survivor counts and offsets per 4096-element tile, the parsed header, an error flag) is
+ * a fixed array inside the library's device image, which every GPU that loads the library holds
+ * until the process ends (about 65 KB).  It is meant for restore paths that run where memory
+ * cannot be requested: on a device that the training framework's own allocator has already
+ * reserved in full, so that cudaMalloc fails, or where the device-wide synchronisation that
+ * cudaMalloc / cudaFree imply must not happen because other streams are busy.
+ *
+ *   - Runs on the CURRENT device; all pointers are device memory of that device, 16-byte aligned.
+ *     Arguments and results are those of excp_decompress_tensor (w_out may be w_prev).
+ *   - numel may not exceed EXCP_NOALLOC_MAX_NUMEL; larger tensors return EXCP_ERR_INVALID_ARG
+ *     before anything is launched (use a handle for those).
+ *   - The first call on a device looks up the array's device address; make that first call
+ *     before any stream capture begins.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; each
+ *     call clears what it needs cleared.  Calls that overlap on the GPU (two streams, two
+ *     threads) race on it: issue them one after the other.
+ *   - Synchronises the stream; returns EXCP_ERR_CORRUPT_BLOB like excp_decompress_tensor. */
+#define EXCP_NOALLOC_MAX_NUMEL (1u << 24)
+excp_status excp_decompress_tensor_noalloc(const void* blob, size_t blob_bytes, const float* w_prev,
+                                           size_t numel, float* w_out, float* ea_out, float* eas_out,
+                                           void* cuda_stream);
+
 /* Per-stage timing of the last compress/decompress call (no counterpart in the paper; the
  * stages are this library's kernels).  With timing enabled each call records CUDA events on
  * its stream between stages and, after its final synchronisation, sums the elapsed times per

@@ -21,7 +21,7 @@ STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED", -3: "BUFFER_TOO_SMALL",
 EXPORTS = ["excp_create", "excp_destroy", "excp_record_bytes", "excp_compress_bound",
            "excp_status_string", "excp_last_cuda_error", "excp_compress_tensor",
            "excp_compress_checkpoint", "excp_compress_checkpoint_host", "excp_decompress_tensor", "excp_decompress_checkpoint",
-           "excp_profile_enable", "excp_profile_stage_count", "excp_profile_stage_name", "excp_profile_read"]
+           "excp_decompress_tensor_noalloc", "excp_profile_enable", "excp_profile_stage_count", "excp_profile_stage_name", "excp_profile_read"]
 
 
 class ExcpError(RuntimeError):
@@ -83,6 +83,7 @@ def load_library() -> C.CDLL:
     lib.excp_decompress_tensor.argtypes = [vp, vp, sz, vp, sz, vp, vp, vp, vp]
     lib.excp_decompress_checkpoint.argtypes = [vp, vp, C.POINTER(sz), sz, C.POINTER(vp), C.POINTER(sz),
                                                C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), vp]
+    lib.excp_decompress_tensor_noalloc.argtypes = [vp, sz, vp, sz, vp, vp, vp, vp]
     lib.excp_profile_enable.argtypes = [vp, C.c_int]
     lib.excp_profile_stage_count.argtypes = []
     lib.excp_profile_stage_name.argtypes = [C.c_int]
@@ -115,6 +116,22 @@ def record_bytes(numel: int, nnz_w: int, nnz_o: int, bits: int = 4) -> int:
 
 def compress_bound(numel: int, bits: int = 4) -> int:
     return load_library().excp_compress_bound(numel, bits)
+
+
+NOALLOC_MAX_NUMEL = 1 << 24
+
+
+def decompress_tensor_noalloc(blob: torch.Tensor, blob_bytes: int, w_prev, w_out, ea_out, eas_out) -> None:
+    """excp_decompress_tensor_noalloc: decode one record on the current device without a handle
+    and without any allocation by the library (for restore paths that cannot allocate: the
+    device is fully reserved by the framework's allocator, or cudaMalloc's device-wide
+    synchronisation is not acceptable).  Tensors of more than NOALLOC_MAX_NUMEL elements are
+    refused; calls must not overlap on the GPU."""
+    _check_f32_cuda(w_prev, w_out, ea_out, eas_out)
+    st = load_library().excp_decompress_tensor_noalloc(blob.data_ptr(), blob_bytes, _ptr(w_prev), w_prev.numel(),
+                                                       _ptr(w_out), _ptr(ea_out), _ptr(eas_out), _stream())
+    if st != 0:
+        raise ExcpError(st, "excp_decompress_tensor_noalloc")
 
 
 class Handle:

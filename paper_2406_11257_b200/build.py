@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libexcp.so")
-SOURCES = ["stats.cu", "mask_compact.cu", "kmeans.cu", "pack.cu", "decode.cu", "excp_api.cu"]
+SOURCES = ["stats.cu", "mask_compact.cu", "kmeans.cu", "pack.cu", "decode.cu", "excp_api.cu", "excp_noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-fmad=false", "-Xcompiler", "-fPIC", "-cudart", "static"]
 
