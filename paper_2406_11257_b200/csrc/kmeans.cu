@@ -211,24 +211,23 @@ __global__ void __launch_bounds__(NBKT) bucket_offsets_kernel(Workspace ws) {
     if (b == NBKT - 1) bk.off[NBKT] = base + incl;
 }
 
-constexpr int SCAP = 12288;          // survivors staged per window of tiles
+constexpr int SPT = 32;               // survivors a thread holds per window
+constexpr int SCAP = SPT * TPB;       // survivors staged per window of tiles (8192)
 
 struct ScatterSmem {
     float val[SCAP];                 // the window's survivors sorted by bucket
     unsigned char bid[SCAP];         // and their buckets
     u32 cnt[NBKT];                   // survivors of the window per bucket
-    u32 loff[NBKT];                  // start of each bucket in val[]
     u32 lcur[NBKT];                  // next free place of each bucket in val[]
-    u32 gbase[NBKT];                 // room reserved for the bucket in the bucketed copy
-    u32 slo[NBKT];                   // low and high 16-bit halves of the window's fixed-point sums
-    int shi[NBKT];
+    u32 delta[NBKT];                 // place in the bucketed copy minus place in val[], per bucket
     u32 pre[33];                     // survivors before tile i of the window
     u32 wtot[TPB / 32];
     u32 wn;                          // tiles in the window
 };
 
-// Sweep 2 of the grouping: survivors into their buckets, and each bucket's fixed-point sum.
-// A block takes windows of tiles of one tensor holding at most SCAP survivors: it counts them
+// Sweep 2 of the grouping: survivors into their buckets.
+// A block takes windows of tiles of one tensor holding at most SCAP survivors.  Every thread
+// loads its 32 survivors of the window at once (they stay in registers), the block counts them
 // per bucket, reserves room in every bucket of the bucketed copy with one integer atomic,
 // sorts the window by bucket in shared memory and writes each bucket's run with consecutive
 // threads (one 4-byte store per survivor straight to its bucket would be bound by the number
@@ -246,14 +245,12 @@ __global__ void __launch_bounds__(TPB, 3) bucket_scatter_kernel(const TensorDesc
     int cur = -1;
     u32 tb = 0, ntl = 0;
     BucketFn fn = BucketFn{0, 0, 0, 0};
-    float s1 = 0.f, s2 = 0.f;
     u32 tile = lo;
     while (tile < hi) {
         if (cur < 0 || tile >= tb + ntl) {
             cur = find_tensor(descs, nt, tile);
             tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
             fn = ws.bst[cur].s[stream].fn;
-            s1 = st[cur].s[stream].scale1; s2 = st[cur].s[stream].scale2;
         }
         const u32 wend = min(hi, tb + ntl);
         if (warp == 0) {              // the window: leading tiles whose survivors fit the stage
@@ -269,14 +266,29 @@ __global__ void __launch_bounds__(TPB, 3) bucket_scatter_kernel(const TensorDesc
             if (lane == 31) sm.pre[32] = incl;
             if (lane == 0) sm.wn = ok == 0xffffffffu ? 32u : (u32)__ffs((int)~ok) - 1u;
         }
-        sm.cnt[tid] = 0; sm.slo[tid] = 0; sm.shi[tid] = 0;
+        sm.cnt[tid] = 0;
         __syncthreads();
         const u32 wn = sm.wn, total = sm.pre[wn];
         if (total) {
-            for (u32 i = 0; i < wn; ++i) {
-                const u32 c = sm.pre[i + 1] - sm.pre[i];
-                const float* data = surv + (u64)(tile + i) * TILE;
-                for (u32 e = tid; e < c; e += TPB) atomicAdd(&sm.cnt[bucket_of(data[e], fn)], 1u);
+            // this thread's survivors: window ranks tid, tid + 256, ...  (tile found by walking pre[])
+            float x[SPT];
+            u32 ti = 0;
+#pragma unroll
+            for (int k = 0; k < SPT; ++k) {
+                const u32 idx = k * TPB + tid;
+                x[k] = 0.f;
+                if (idx < total) {
+                    while (idx >= sm.pre[ti + 1]) ++ti;
+                    x[k] = surv[(u64)(tile + ti) * TILE + (idx - sm.pre[ti])];
+                }
+            }
+            u32 bk[SPT / 4];            // the buckets of x[], one byte each
+#pragma unroll
+            for (int k = 0; k < SPT; ++k) {
+                const u32 b = bucket_of(x[k], fn);
+                if ((k & 3) == 0) bk[k / 4] = 0;
+                bk[k / 4] |= b << (8 * (k & 3));
+                if (k * TPB + tid < total) atomicAdd(&sm.cnt[b], 1u);
             }
             __syncthreads();
             {                          // exclusive prefix of the counts; room in the bucketed copy
@@ -291,33 +303,23 @@ __global__ void __launch_bounds__(TPB, 3) bucket_scatter_kernel(const TensorDesc
                 __syncthreads();
                 u32 base = 0;
                 for (int w = 0; w < warp; ++w) base += sm.wtot[w];
-                sm.loff[tid] = base + incl - c;
                 sm.lcur[tid] = base + incl - c;
-                sm.gbase[tid] = c ? atomicAdd(&ws.bst[cur].s[stream].cursor[tid], c) : 0u;
+                const u32 g = c ? atomicAdd(&ws.bst[cur].s[stream].cursor[tid], c) : 0u;
+                sm.delta[tid] = g - (base + incl - c);
             }
             __syncthreads();
-            for (u32 i = 0; i < wn; ++i) {
-                const u32 c = sm.pre[i + 1] - sm.pre[i];
-                const float* data = surv + (u64)(tile + i) * TILE;
-                for (u32 e = tid; e < c; e += TPB) {
-                    const float x = data[e];
-                    const u32 b = bucket_of(x, fn);
+#pragma unroll
+            for (int k = 0; k < SPT; ++k) {
+                if (k * TPB + tid < total) {
+                    const u32 b = (bk[k / 4] >> (8 * (k & 3))) & 255u;
                     const u32 r = atomicAdd(&sm.lcur[b], 1u);
-                    sm.val[r] = x;
+                    sm.val[r] = x[k];
                     sm.bid[r] = (unsigned char)b;
-                    const int q = __float2int_rn(__fmul_rn(__fmul_rn(x, s1), s2));
-                    atomicAdd(&sm.slo[b], (u32)q & 0xffffu);
-                    atomicAdd(&sm.shi[b], q >> 16);
                 }
             }
             __syncthreads();
             float* dst = ws.bkt[stream] + (u64)tb * TILE;
-            for (u32 i = tid; i < total; i += TPB) {
-                const u32 b = sm.bid[i];
-                dst[sm.gbase[b] + (i - sm.loff[b])] = sm.val[i];
-            }
-            const s64 sum = (s64)sm.shi[tid] * 65536 + (s64)sm.slo[tid];
-            if (sum) atomicAdd(reinterpret_cast<u64*>(&ws.bst[cur].s[stream].sum[tid]), (u64)sum);
+            for (u32 i = tid; i < total; i += TPB) dst[i + sm.delta[sm.bid[i]]] = sm.val[i];
         }
         tile += wn;
         __syncthreads();
@@ -331,6 +333,35 @@ __device__ inline void plan_scan(const StreamState& s, BucketStream& bk, int lan
         bk.bstar[lane] = bucket_of(s.thr[lane], bk.fn);
         bk.part_cnt[lane] = 0;
         bk.part_sum[lane] = 0;
+    }
+}
+
+// Fixed-point sum of every bucket, read off the bucketed copy (each bucket is contiguous there).
+// Grid (NBKT / 8, tensors * 3): a block takes eight neighbouring buckets.
+__global__ void __launch_bounds__(TPB) bucket_sum_kernel(const TensorDesc* __restrict__ descs,
+                                                         const TensorState* __restrict__ st, Workspace ws) {
+    __shared__ s64 rsum[TPB / 32];
+    const int t = blockIdx.y / 3, k = blockIdx.y % 3;
+    BucketStream& bk = ws.bst[t].s[k];
+    const float s1 = st[t].s[k].scale1, s2 = st[t].s[k].scale2;
+    const float* data = ws.bkt[k] + (u64)descs[t].tile_begin * TILE;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int b = blockIdx.x * 8; b < blockIdx.x * 8 + 8; ++b) {
+        const u32 r0 = bk.off[b], r1 = bk.off[b + 1];
+        if (r0 == r1) continue;
+        s64 sum = 0;
+        for (u32 i = r0 + threadIdx.x; i < r1; i += TPB)
+            sum += __float2int_rn(__fmul_rn(__fmul_rn(data[i], s1), s2));
+#pragma unroll
+        for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if (lane == 0) rsum[warp] = sum;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            s64 tot = 0;
+            for (int w = 0; w < TPB / 32; ++w) tot += rsum[w];
+            bk.sum[b] = tot;
+        }
+        __syncthreads();
     }
 }
 
@@ -467,8 +498,9 @@ void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* s
         for (int k = 0; k < 3; ++k)
             bucket_scatter_kernel<<<sgrid, TPB, sizeof(ScatterSmem), cfg.stream>>>(descs, st, nt, tiles, ws, k);
     }
+    bucket_sum_kernel<<<dim3(NBKT / 8, nt * 3), TPB, 0, cfg.stream>>>(descs, st, ws);
     bucket_prefix_kernel<<<dim3(nt, 3), NBKT, 0, cfg.stream>>>(st, ws);
-    prof_mark(cfg, ST_BUCKET_SCATTER, 5);
+    prof_mark(cfg, ST_BUCKET_SCATTER, 6);
     for (int it = 0; it < p.kmeans_iters; ++it) {
         bucket_scan_kernel<<<dim3(scan_items, 3 * (KMAX - 1)), TPB, 0, cfg.stream>>>(descs, st, nt, ws);
         prof_mark(cfg, ST_BUCKET_SCAN, 1);
