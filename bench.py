@@ -253,6 +253,7 @@ def run_ours(args):
         "mask_compact": 16 * n_tot + n_tot / 4 + 4 * surv,
         "bucket_ids": 4 * surv,                     # survivors read once to count them per bucket
         "bucket_scatter": 8 * surv,                 # survivors read and written into their buckets
+        "bucket_sum": 4 * surv,                     # the bucketed copy read once for the bucket sums
         "bucket_scan": T * 4 * surv * 14 / 256,     # about 14 of 256 buckets per iteration
         "pack_codes": 4.5 * surv,
         "copy_bitmaps": n_tot / 2,

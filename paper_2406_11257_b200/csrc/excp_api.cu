@@ -566,7 +566,7 @@ int excp_profile_stage_count(void) { return ST_COUNT; }
 const char* excp_profile_stage_name(int stage) {
     static const char* names[ST_COUNT] = {
         "stats1", "stats2", "mask_compact", "scan_layout", "kmeans_start", "bucket_ids", "bucket_scatter",
-        "bucket_scan", "kmeans_update", "header_edges", "pack_codes", "copy_bitmaps", "dec_prep", "decode"};
+        "bucket_scan", "kmeans_update", "header_edges", "pack_codes", "copy_bitmaps", "dec_prep", "decode", "bucket_sum"};
     return stage >= 0 && stage < ST_COUNT ? names[stage] : "";
 }
 

@@ -267,7 +267,7 @@ __device__ inline void scan_tile_counts(u32 tb, u32 ntl, const Workspace& ws, u3
 enum Stage {                       // for the optional per-stage event timing
     ST_STATS1 = 0, ST_STATS2, ST_MASK_COMPACT, ST_SCAN_LAYOUT, ST_KMEANS_START, ST_BUCKET_IDS, ST_BUCKET_SCATTER,
     ST_BUCKET_SCAN, ST_KMEANS_UPDATE, ST_HEADER_EDGES, ST_PACK_CODES, ST_COPY_BITMAPS, ST_DEC_PREP,
-    ST_DECODE, ST_COUNT
+    ST_DECODE, ST_BUCKET_SUM, ST_COUNT
 };
 
 struct Profiler;

@@ -337,31 +337,35 @@ __device__ inline void plan_scan(const StreamState& s, BucketStream& bk, int lan
 }
 
 // Fixed-point sum of every bucket, read off the bucketed copy (each bucket is contiguous there).
-// Grid (NBKT / 8, tensors * 3): a block takes eight neighbouring buckets.
+// Grid (NBKT, tensors * 3): one block per bucket.
 __global__ void __launch_bounds__(TPB) bucket_sum_kernel(const TensorDesc* __restrict__ descs,
                                                          const TensorState* __restrict__ st, Workspace ws) {
     __shared__ s64 rsum[TPB / 32];
-    const int t = blockIdx.y / 3, k = blockIdx.y % 3;
+    const int t = blockIdx.y / 3, k = blockIdx.y % 3, b = blockIdx.x;
     BucketStream& bk = ws.bst[t].s[k];
+    const u32 r0 = bk.off[b], r1 = bk.off[b + 1];
+    if (r0 == r1) return;
     const float s1 = st[t].s[k].scale1, s2 = st[t].s[k].scale2;
     const float* data = ws.bkt[k] + (u64)descs[t].tile_begin * TILE;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int b = blockIdx.x * 8; b < blockIdx.x * 8 + 8; ++b) {
-        const u32 r0 = bk.off[b], r1 = bk.off[b + 1];
-        if (r0 == r1) continue;
-        s64 sum = 0;
-        for (u32 i = r0 + threadIdx.x; i < r1; i += TPB)
-            sum += __float2int_rn(__fmul_rn(__fmul_rn(data[i], s1), s2));
+    s64 sum = 0;
+    u32 i = r0 + threadIdx.x;
+    for (; i + 7 * TPB < r1; i += 8 * TPB) {               // eight independent loads in flight
+        float x[8];
 #pragma unroll
-        for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-        if (lane == 0) rsum[warp] = sum;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            s64 tot = 0;
-            for (int w = 0; w < TPB / 32; ++w) tot += rsum[w];
-            bk.sum[b] = tot;
-        }
-        __syncthreads();
+        for (int j = 0; j < 8; ++j) x[j] = __ldcs(data + i + j * TPB);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) sum += __float2int_rn(__fmul_rn(__fmul_rn(x[j], s1), s2));
+    }
+    for (; i < r1; i += TPB) sum += __float2int_rn(__fmul_rn(__fmul_rn(__ldcs(data + i), s1), s2));
+#pragma unroll
+    for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if (lane == 0) rsum[warp] = sum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        s64 tot = 0;
+        for (int w = 0; w < TPB / 32; ++w) tot += rsum[w];
+        bk.sum[b] = tot;
     }
 }
 
@@ -498,9 +502,10 @@ void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* s
         for (int k = 0; k < 3; ++k)
             bucket_scatter_kernel<<<sgrid, TPB, sizeof(ScatterSmem), cfg.stream>>>(descs, st, nt, tiles, ws, k);
     }
-    bucket_sum_kernel<<<dim3(NBKT / 8, nt * 3), TPB, 0, cfg.stream>>>(descs, st, ws);
+    prof_mark(cfg, ST_BUCKET_SCATTER, 4);
+    bucket_sum_kernel<<<dim3(NBKT, nt * 3), TPB, 0, cfg.stream>>>(descs, st, ws);
     bucket_prefix_kernel<<<dim3(nt, 3), NBKT, 0, cfg.stream>>>(st, ws);
-    prof_mark(cfg, ST_BUCKET_SCATTER, 6);
+    prof_mark(cfg, ST_BUCKET_SUM, 2);
     for (int it = 0; it < p.kmeans_iters; ++it) {
         bucket_scan_kernel<<<dim3(scan_items, 3 * (KMAX - 1)), TPB, 0, cfg.stream>>>(descs, st, nt, ws);
         prof_mark(cfg, ST_BUCKET_SCAN, 1);
