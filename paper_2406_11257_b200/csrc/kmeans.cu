@@ -414,8 +414,20 @@ __global__ void __launch_bounds__(TPB) bucket_scan_kernel(const TensorDesc* __re
     const float* data = ws.bkt[k] + (u64)descs[t].tile_begin * TILE;
     u32 cnt = 0;
     s64 sum = 0;
-    for (u32 i = a + threadIdx.x; i < e; i += TPB) {
-        const float x = data[i];
+    u32 i = a + threadIdx.x;
+    for (; i + 7 * TPB < e; i += 8 * TPB) {                 // eight independent loads in flight
+        float x[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) x[j] = __ldcs(data + i + j * TPB);
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if (!(x[j] > thr)) {
+                ++cnt;
+                sum += __float2int_rn(__fmul_rn(__fmul_rn(x[j], s1), s2));
+            }
+    }
+    for (; i < e; i += TPB) {
+        const float x = __ldcs(data + i);
         if (!(x > thr)) {
             ++cnt;
             sum += __float2int_rn(__fmul_rn(__fmul_rn(x, s1), s2));
