@@ -30,6 +30,9 @@ os.environ.setdefault("PYTORCH_CUDA_ALLOC_CONF", "expandable_segments:True")
 
 METRIC = "compress params/s and GB/s of (W,W_prev,m,v) read at 7B shape; % of HBM peak"
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read + dram__bytes_write per parameter from the ncu captures summarised under
+# profiles/ (small case, scaled by parameters); only for kernels unchanged since the capture
+NCU_DRAM_BYTES_PER_PARAM = {"mask_compact": (1.027877e9 + 169.177856e6) / 64108544}
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -292,7 +295,8 @@ def run_ours(args):
         "compression": {"blob_bytes": blob_bytes, "ratio_vs_12B_per_param": 12 * n_tot / blob_bytes},
         "stages": stages,
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": dom_gbs / peak, "peak_kind": peak_kind, "traffic": None,
+                     "frac": dom_gbs / peak, "peak_kind": peak_kind,
+                     "traffic": NCU_DRAM_BYTES_PER_PARAM[dom] * n_tot if dom in NCU_DRAM_BYTES_PER_PARAM else None,
                      "algorithmic_bytes_per_step": stage_bytes[dom], "ms_per_step": dom_ms, "note": groups_note},
         "clocks": clocks,
         "gpu_launches": launches,
