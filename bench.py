@@ -252,7 +252,6 @@ def run_ours(args):
     surv = nnz_w + 2 * nnz_o
     stage_bytes = {
         "stats1": (src_b + 4) * n_tot,
-        "stats2": src_b * n_tot,
         "mask_compact": 16 * n_tot + n_tot / 4 + 4 * surv,
         "bucket_ids": 4 * surv,                     # survivors read once to count them per bucket
         "bucket_scatter": 8 * surv,                 # survivors read and written into their buckets

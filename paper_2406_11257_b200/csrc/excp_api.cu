@@ -168,7 +168,7 @@ bool run_group(excp_handle h, const LaunchCfg& cfg, const TensorDesc* descs, int
                const Params& p, unsigned char* blob, u64 blob_capacity, TensorResult* results) {
     if (!check(h, cudaMemsetAsync(h->d_state, 0, nt * sizeof(TensorState), cfg.stream))) return false;
     if (!check(h, cudaMemsetAsync(h->ws.bst, 0, nt * sizeof(BucketState), cfg.stream))) return false;
-    launch_stats(cfg, descs, h->d_state, nt, tiles, h->ws, p);
+    launch_stats(cfg, descs, h->d_state, nt, tiles, h->ws, p, h->d_call);
     launch_mask_compact(cfg, descs, h->d_state, nt, tiles, h->ws, p, h->d_call, blob_capacity);
     launch_kmeans(cfg, descs, h->d_state, nt, tiles, scan_items, h->ws, p, h->d_call);
     launch_pack(cfg, descs, h->d_state, nt, tiles, h->ws, p, blob, h->d_call, results);

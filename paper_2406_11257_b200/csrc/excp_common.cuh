@@ -74,6 +74,10 @@ struct TensorState {             // device scratch, zeroed per group
     float mean_abs_ea;
     float thr_w, thr_o;
     u32 nnz_w, nnz_o;
+    u32 lo_key, hi_key;          // bracket of magnitude patterns that should hold the median (from a sample)
+    u32 count_below;             // elements below the bracket
+    u32 med_done;                // the sample was the whole tensor: median already known
+    u32 need_hist;               // the bracket missed the median: take the histogram path
     u32 pad_;
     u64 blob_off;                // start of this tensor's record in the blob
     u64 blob_bytes;
@@ -281,7 +285,7 @@ struct LaunchCfg {
 void prof_mark(const LaunchCfg& cfg, int stage, int launches);
 
 void launch_stats(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
-                  const Workspace& ws, const Params& p);
+                  const Workspace& ws, const Params& p, CallState* call);
 void launch_mask_compact(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                          const Workspace& ws, const Params& p, CallState* call, u64 blob_capacity);
 void launch_kmeans(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,

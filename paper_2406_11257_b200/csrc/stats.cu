@@ -1,17 +1,23 @@
 // Per-tensor statistics behind the two thresholds of Section 3.2:
-//   the lower median of |W_t| or |dW_t| (Eq. rw) by a radix select on fp32 bit
-//   patterns, and the exact mean of |ea| (Eq. ro) by integer accumulation.
+//   the lower median of |W_t| or |dW_t| (Eq. rw), an exact order statistic found on
+//   fp32 bit patterns, and the exact mean of |ea| (Eq. ro) by integer accumulation.
 //
-// Sweep 1 (stats1): histogram of the top 13 key bits (per-block in shared
-//   memory, merged with integer atomics) + exact fixed-point sum of |ea|.
-// finish1:          pick the bin holding the median rank; turn the sum tables
-//   into the correctly rounded mean (multi-word integer arithmetic).
-// Sweep 2 (stats2): gather the keys of that bin (about 1 % of the tensor).
-// finish2:          select inside the candidates (two 9-bit levels); thresholds.
+// One sweep over the data is the rule:
+//   median_sample  65536 evenly spaced elements per tensor; two order statistics of the sample
+//                  bracket the median (a tensor no larger than the sample is settled here)
+//   stats_sweep    counts the elements below the bracket, gathers the keys inside it (about
+//                  2.5 % of the tensor), and accumulates the exact sum of |ea|
+//   stats_finish   selects the median among the gathered keys; the correctly rounded mean
+//                  (multi-word integer arithmetic); both thresholds
+// If the bracket misses the median (the sample misrepresents the tensor), that tensor takes
+// the histogram path -- two more sweeps: a histogram of the top 13 key bits, then a gather of
+// the median's bin and a select inside it.  Its kernels are always launched and return at
+// once for tensors that do not need them.
 //
 // Every reduction is over integers, so the result does not depend on the
 // order in which blocks or warps run.
 #include "excp_common.cuh"
+#include "warp_ring.cuh"
 
 namespace excp {
 
@@ -59,34 +65,22 @@ __device__ void find_rank_block(const u32* hist, u32 k, u32& bin, u32& rank_in, 
 }
 
 // ---------------------------------------------------------------------------
-// Sweep 1.
-__global__ void __launch_bounds__(TPB) stats1_kernel(const TensorDesc* __restrict__ descs,
-                                                     TensorState* __restrict__ st, int nt, u32 tiles,
-                                                     int residual_median) {
+// Histogram path, sweep 1: top 13 key bits, per block in shared memory, merged with integer
+// atomics.  Only tensors flagged need_hist.
+__global__ void __launch_bounds__(TPB) hist1_kernel(const TensorDesc* __restrict__ descs,
+                                                    TensorState* __restrict__ st, int nt, u32 tiles,
+                                                    int residual_median) {
     __shared__ u32 hist[HIST1_BINS];
-    const int tid = threadIdx.x, lane = tid & 31;
+    const int tid = threadIdx.x;
     for (int i = tid; i < HIST1_BINS; i += TPB) hist[i] = 0;
     __syncthreads();
-
     u32 lo, hi;
     block_range(tiles, lo, hi);
     int cur = -1;
     u32 tb = 0, ntl = 0;
     u64 n = 0;
-    const float *w_t = nullptr, *w_prev = nullptr, *ea = nullptr;
-    u64 acc = 0;          // this thread's share of sum |ea|, unit 2^(ecur-174)
-    int ecur = 1;         // biased exponent the unit is tied to (warp uniform)
-    int since = 0;
-
-    auto flush_acc = [&](int t) {
-        u64 s = warp_sum_u64(acc);
-        if (lane == 0 && s) {
-            atomicAdd(&st[t].sum_lo[ecur], s & 0xffffffffull);
-            atomicAdd(&st[t].sum_hi[ecur], s >> 32);
-        }
-        acc = 0;
-        since = 0;
-    };
+    bool active = false;
+    const float *w_t = nullptr, *w_prev = nullptr;
     auto flush_hist = [&](int t) {
         __syncthreads();
         for (int i = tid; i < HIST1_BINS; i += TPB) {
@@ -95,54 +89,33 @@ __global__ void __launch_bounds__(TPB) stats1_kernel(const TensorDesc* __restric
         }
         __syncthreads();
     };
-
     for (u32 tile = lo; tile < hi; ++tile) {
         if (cur < 0 || tile >= tb + ntl) {
-            if (cur >= 0) { flush_hist(cur); flush_acc(cur); }
-            ecur = 1;
+            if (cur >= 0 && active) flush_hist(cur);
             cur = find_tensor(descs, nt, tile);
             tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles; n = descs[cur].numel;
-            w_t = descs[cur].w_t; w_prev = descs[cur].w_prev; ea = descs[cur].ea;
+            w_t = descs[cur].w_t; w_prev = descs[cur].w_prev;
+            active = st[cur].need_hist != 0;
+            if (!active) tile = tb + ntl - 1;          // nothing to do for this tensor
         }
+        if (!active) continue;
         const u64 base = (u64)(tile - tb) * TILE;
-        u32 ke[4 * ROUNDS];
-        u32 kmax = 0;
 #pragma unroll
         for (int r = 0; r < ROUNDS; ++r) {
             const u64 i0 = base + (u64)r * (TPB * 4) + (u64)tid * 4;
-            float a[4], b[4], e[4];
+            float a[4], b[4];
             const int nv = load4(w_t, i0, n, a);
             if (residual_median) {
                 load4(w_prev, i0, n, b);
 #pragma unroll
                 for (int k = 0; k < 4; ++k) a[k] = __fsub_rn(a[k], b[k]);
             }
-            load4(ea, i0, n, e);
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
+            for (int k = 0; k < 4; ++k)
                 if (k < nv) atomicAdd(&hist[(__float_as_uint(a[k]) & 0x7fffffffu) >> HIST1_SHIFT], 1u);
-                const u32 kk = __float_as_uint(e[k]) & 0x7fffffffu;
-                ke[r * 4 + k] = kk;
-                kmax = max(kmax, kk);
-            }
         }
-        // exact sum of |ea|: integer mantissas shifted to a common unit tied to
-        // the largest exponent this warp has met
-        const int emax = max((int)(__reduce_max_sync(0xffffffffu, kmax) >> 23), 1);
-        if (emax > ecur) { flush_acc(cur); ecur = emax; }
-#pragma unroll
-        for (int j = 0; j < 4 * ROUNDS; ++j) {
-            const u32 kk = ke[j];
-            const int e = (int)(kk >> 23);
-            const u32 m = (kk & 0x7fffffu) | (e ? 0x800000u : 0u);
-            const int e1 = max(e, 1);
-            const int sh = e1 - ecur + 24;
-            if (sh >= 0) acc += (u64)m << sh;
-            else if (m) atomicAdd(&st[cur].sum_low[e1], (u64)m);
-        }
-        if (++since >= 32) flush_acc(cur);
     }
-    if (cur >= 0) { flush_hist(cur); flush_acc(cur); }
+    if (cur >= 0 && active) flush_hist(cur);
 }
 
 // ---------------------------------------------------------------------------
@@ -198,34 +171,25 @@ __device__ static float exact_mean_from_tables(const u64* lo, const u64* hi, con
     return __uint_as_float((u32)((u + 150) << 23) + m - 0x800000u);
 }
 
-__global__ void __launch_bounds__(TPB) stats1_finish_kernel(const TensorDesc* __restrict__ descs,
-                                                            TensorState* __restrict__ st) {
+// Histogram path: the bin that holds the median rank.  One block per flagged tensor.
+__global__ void __launch_bounds__(TPB) hist1_finish_kernel(const TensorDesc* __restrict__ descs,
+                                                           TensorState* __restrict__ st) {
     __shared__ u32 hist[HIST1_BINS];
-    __shared__ u64 tab[3][256];
     const int t = blockIdx.x, tid = threadIdx.x;
     TensorState& s = st[t];
+    if (!s.need_hist) return;
     const u64 n = descs[t].numel;
-    if (n == 0) {
-        if (tid == 0) { s.bin1 = 0; s.rank_in_bin = 0; s.bin_count = 0; s.mean_abs_ea = 0.f; }
-        return;
-    }
     for (int i = tid; i < HIST1_BINS; i += TPB) hist[i] = s.hist1[i];
-    tab[0][tid] = s.sum_lo[tid];
-    tab[1][tid] = s.sum_hi[tid];
-    tab[2][tid] = s.sum_low[tid];
     __syncthreads();
     u32 bin, rank_in, cnt;
     find_rank_block<HIST1_BINS>(hist, (u32)((n - 1) / 2), bin, rank_in, cnt);
-    if (tid == 0) {
-        s.bin1 = bin; s.rank_in_bin = rank_in; s.bin_count = cnt;
-        s.mean_abs_ea = exact_mean_from_tables(tab[0], tab[1], tab[2], n);
-    }
+    if (tid == 0) { s.bin1 = bin; s.rank_in_bin = rank_in; s.bin_count = cnt; s.cand_count = 0; }
 }
 
 // ---------------------------------------------------------------------------
-// Sweep 2: keys of the selected bin -> candidate list (kept in the tensor's own
-// survivor segment, which the mask sweep overwrites afterwards).
-__global__ void __launch_bounds__(TPB) stats2_kernel(const TensorDesc* __restrict__ descs,
+// Histogram path, sweep 2: keys of the selected bin -> candidate list (kept in the tensor's own
+// survivor segment, which the mask sweep overwrites afterwards).  Only flagged tensors.
+__global__ void __launch_bounds__(TPB) hist2_kernel(const TensorDesc* __restrict__ descs,
                                                      TensorState* __restrict__ st, int nt, u32 tiles,
                                                      Workspace ws, int residual_median) {
     const int tid = threadIdx.x, lane = tid & 31;
@@ -234,6 +198,7 @@ __global__ void __launch_bounds__(TPB) stats2_kernel(const TensorDesc* __restric
     int cur = -1;
     u32 tb = 0, ntl = 0, bin1 = 0;
     u64 n = 0;
+    bool active = false;
     const float *w_t = nullptr, *w_prev = nullptr;
     u32* cand = nullptr;
     for (u32 tile = lo; tile < hi; ++tile) {
@@ -243,7 +208,10 @@ __global__ void __launch_bounds__(TPB) stats2_kernel(const TensorDesc* __restric
             w_t = descs[cur].w_t; w_prev = descs[cur].w_prev;
             bin1 = st[cur].bin1;
             cand = reinterpret_cast<u32*>(ws.surv[0] + (u64)tb * TILE);
+            active = st[cur].need_hist != 0;
+            if (!active) tile = tb + ntl - 1;          // nothing to do for this tensor
         }
+        if (!active) continue;
         const u64 base = (u64)(tile - tb) * TILE;
 #pragma unroll
         for (int r = 0; r < ROUNDS; ++r) {
@@ -280,22 +248,14 @@ __global__ void __launch_bounds__(TPB) stats2_kernel(const TensorDesc* __restric
     }
 }
 
-// Select inside the candidates and set both thresholds.
-__global__ void __launch_bounds__(1024) stats2_finish_kernel(const TensorDesc* __restrict__ descs,
-                                                             TensorState* __restrict__ st, Workspace ws,
-                                                             float alpha, float beta) {
+// Histogram path: select inside the bin's keys; the weight threshold.
+__global__ void __launch_bounds__(1024) hist2_finish_kernel(const TensorDesc* __restrict__ descs,
+                                                            TensorState* __restrict__ st, Workspace ws,
+                                                            float alpha) {
     __shared__ u32 hist[512];
     const int t = blockIdx.x, tid = threadIdx.x;
     TensorState& s = st[t];
-    const u64 n = descs[t].numel;
-    if (n == 0) {
-        if (tid == 0) {
-            s.median_bits = 0;
-            s.thr_w = __fmul_rn(alpha, 0.f);
-            s.thr_o = __fmul_rn(beta, 0.f);
-        }
-        return;
-    }
+    if (!s.need_hist) return;
     const u32 c = s.cand_count;
     const u32* cand = reinterpret_cast<const u32*>(ws.surv[0] + (u64)descs[t].tile_begin * TILE);
     u32 k = s.rank_in_bin;
@@ -318,26 +278,276 @@ __global__ void __launch_bounds__(1024) stats2_finish_kernel(const TensorDesc* _
         const u32 bits = (s.bin1 << HIST1_SHIFT) | (a << 9) | b;
         s.median_bits = bits;
         s.thr_w = __fmul_rn(alpha, __uint_as_float(bits));      // alpha * median, Eq. (rw)
-        s.thr_o = __fmul_rn(beta, s.mean_abs_ea);               // beta * mean, Eq. (ro)
         if (c != s.bin_count) s.flags |= FLAG_INTERNAL;
     }
 }
 
+
+// ---------------------------------------------------------------------------
+// The element of rank `rank` (0-based, ascending) among cnt 31-bit keys, by four 8-bit digit
+// passes.  Whole block (at least 256 threads); hist: 256 words of shared memory.
+__device__ static u32 block_select(const u32* __restrict__ keys, u32 cnt, u32 rank, u32* hist) {
+    u32 prefix = 0, mask = 0;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+        __syncthreads();
+        for (u32 i = threadIdx.x; i < cnt; i += blockDim.x) {
+            const u32 key = keys[i];
+            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        u32 bin, rin, c;
+        find_rank_block<256>(hist, rank, bin, rin, c);
+        prefix |= bin << shift;
+        mask |= 255u << shift;
+        rank = rin;
+    }
+    return prefix;
+}
+
+constexpr u32 MEDIAN_SAMPLE = 65536;         // evenly spaced elements that bracket the median
+constexpr u32 MEDIAN_MARGIN = MEDIAN_SAMPLE / 80;   // +-1.25 % of the sample: about six standard deviations
+
+// One block per tensor.  The sample's keys go to the tensor's second survivor segment (free
+// until the mask sweep); a tensor no larger than the sample gets its exact median here.
+__global__ void __launch_bounds__(1024) median_sample_kernel(const TensorDesc* __restrict__ descs,
+                                                             TensorState* __restrict__ st, Workspace ws,
+                                                             int residual_median) {
+    __shared__ u32 hist[256];
+    const int t = blockIdx.x, tid = threadIdx.x;
+    TensorState& s = st[t];
+    const u64 n = descs[t].numel;
+    if (n == 0) {
+        if (tid == 0) { s.med_done = 1; s.median_bits = 0; }
+        return;
+    }
+    const u32 m = (u32)min((u64)MEDIAN_SAMPLE, n);
+    u32* keys = reinterpret_cast<u32*>(ws.surv[1] + (u64)descs[t].tile_begin * TILE);
+    const float* w_t = descs[t].w_t;
+    const float* w_prev = descs[t].w_prev;
+    for (u32 j = tid; j < m; j += 1024) {
+        const u64 i = ((u64)j * n) / m;
+        float a = w_t[i];
+        if (residual_median) a = __fsub_rn(a, w_prev[i]);
+        keys[j] = __float_as_uint(a) & 0x7fffffffu;
+    }
+    __syncthreads();
+    if (n <= MEDIAN_SAMPLE) {
+        const u32 med = block_select(keys, m, (u32)((n - 1) / 2), hist);
+        if (tid == 0) { s.median_bits = med; s.med_done = 1; }
+        return;
+    }
+    const u32 lo = block_select(keys, m, m / 2 - MEDIAN_MARGIN, hist);
+    const u32 hi = block_select(keys, m, m / 2 + MEDIAN_MARGIN, hist);
+    if (tid == 0) { s.lo_key = lo; s.hi_key = hi; }
+}
+
+// ---------------------------------------------------------------------------
+// The statistics sweep.  Every warp walks its own run of tiles; 512-value chunks of the
+// median's source stream(s) and of ea arrive in its ring of stages.
+constexpr int SCH = 512;             // values per stream per staged chunk
+constexpr int SST = 2;               // chunks in flight per warp
+constexpr int SWARPS = TPB / 32;
+
+struct SweepSmem {
+    float buf[SWARPS][SST][3][SCH];
+    unsigned long long bar[SWARPS][SST];
+};
+
+__global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* __restrict__ descs,
+                                                             TensorState* __restrict__ st, int nt, u32 tiles,
+                                                             Workspace ws, int residual_median, CallState* call) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    SweepSmem& sm = *reinterpret_cast<SweepSmem*>(smem_raw);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    WarpRing<3, SCH, SST> ring;
+    ring.init(&sm.buf[warp][0][0][0], sm.bar[warp], lane);
+    const u32 gw = blockIdx.x * SWARPS + warp, nw = gridDim.x * SWARPS;
+    const u32 wlo = (u32)(((u64)tiles * gw) / nw), whi = (u32)(((u64)tiles * (gw + 1)) / nw);
+    TileWalk<SCH> ic, cc;
+    ic.start(wlo); cc.start(wlo);
+    const float* ip[3] = {nullptr, nullptr, nullptr};
+    const float* cp[3] = {nullptr, nullptr, nullptr};
+    u32 lo_key = 0, span = 0;        // bracket [lo_key, lo_key + span]
+    bool want_median = false;
+    u32* cand = nullptr;
+    u32 below = 0;                   // this thread's count of keys under the bracket
+    u64 acc = 0;                     // this thread's share of sum |ea|, unit 2^(ecur-174)
+    int ecur = 1;                    // biased exponent the unit is tied to (warp uniform)
+    int since = 0;
+    int prev = -1;
+
+    auto flush_acc = [&](int t) {
+        const u64 s = warp_sum_u64(acc);
+        if (lane == 0 && s) {
+            atomicAdd(&st[t].sum_lo[ecur], s & 0xffffffffull);
+            atomicAdd(&st[t].sum_hi[ecur], s >> 32);
+        }
+        acc = 0;
+        since = 0;
+    };
+    auto flush_below = [&](int t) {
+        const u32 b = __reduce_add_sync(0xffffffffu, below);
+        if (lane == 0 && b) atomicAdd(&st[t].count_below, b);
+        below = 0;
+    };
+
+    while (cc.tile < whi) {
+        while (ic.tile < whi && ring.can_issue()) {
+            if (ic.chunk == 0 && ic.enter_tile(descs, nt)) {
+                ip[0] = descs[ic.tns].w_t;
+                ip[1] = residual_median ? descs[ic.tns].w_prev : nullptr;
+                ip[2] = descs[ic.tns].ea;
+            }
+            const u64 e0 = ic.elem0();
+            const float* src[3] = {ip[0] + e0, ip[1] ? ip[1] + e0 : nullptr, ip[2] + e0};
+            ring.issue(lane, src, ic.valid() & ~3u);
+            ic.next();
+        }
+        if (cc.chunk == 0 && cc.enter_tile(descs, nt)) {
+            if (prev >= 0) { flush_acc(prev); flush_below(prev); }
+            prev = cc.tns;
+            ecur = 1;
+            cp[0] = descs[cc.tns].w_t; cp[1] = descs[cc.tns].w_prev; cp[2] = descs[cc.tns].ea;
+            want_median = st[cc.tns].med_done == 0;
+            lo_key = st[cc.tns].lo_key;
+            span = st[cc.tns].hi_key - lo_key;
+            cand = reinterpret_cast<u32*>(ws.surv[0] + (u64)cc.tb * TILE);
+        }
+        const u32 valid = cc.valid(), nbulk = valid & ~3u;
+        const u64 e0 = cc.elem0();
+        if (!ring.wait()) {
+            if (lane == 0) atomicOr(&call->flags, FLAG_TIMEOUT);
+            return;
+        }
+        const float* stg = ring.stage();
+        u32 ke[SCH / 32];
+        u32 kmax = 0;
+#pragma unroll
+        for (int r = 0; r < SCH / 128; ++r) {
+            const u32 o = r * 128 + lane * 4;
+            float a[4], b[4], e[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) e[k] = 0.f;
+            if ((u32)r * 128u < valid) {
+                fetch4(stg + 2 * SCH, cp[2] + e0, o, nbulk, valid, e);
+                if (want_median) {
+                    fetch4(stg, cp[0] + e0, o, nbulk, valid, a);
+                    if (residual_median) {
+                        fetch4(stg + SCH, cp[1] + e0, o, nbulk, valid, b);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) a[k] = __fsub_rn(a[k], b[k]);
+                    }
+                    u32 key[4];
+                    int mine = 0;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        key[k] = __float_as_uint(a[k]) & 0x7fffffffu;
+                        const bool real = o + k < valid;
+                        below += real && key[k] < lo_key;
+                        mine += real && key[k] - lo_key <= span;      // unsigned: false below lo_key
+                    }
+                    if (__any_sync(0xffffffffu, mine)) {             // gather the keys inside the bracket
+                        int incl = mine;
+#pragma unroll
+                        for (int w = 1; w < 32; w <<= 1) {
+                            const int v = __shfl_up_sync(0xffffffffu, incl, w);
+                            if (lane >= w) incl += v;
+                        }
+                        u32 start = 0;
+                        if (lane == 31) start = atomicAdd(&st[cc.tns].cand_count, (u32)incl);
+                        start = __shfl_sync(0xffffffffu, start, 31) + incl - mine;
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            if (o + k < valid && key[k] - lo_key <= span) cand[start++] = key[k];
+                    }
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const u32 kk = __float_as_uint(e[k]) & 0x7fffffffu;
+                ke[r * 4 + k] = kk;
+                kmax = max(kmax, kk);
+            }
+        }
+        // exact sum of |ea|: integer mantissas shifted to a common unit tied to the largest
+        // exponent this warp has met in this tensor
+        const int emax = max((int)(__reduce_max_sync(0xffffffffu, kmax) >> 23), 1);
+        if (emax > ecur) { flush_acc(cc.tns); ecur = emax; }
+#pragma unroll
+        for (int j = 0; j < SCH / 32; ++j) {
+            const u32 kk = ke[j];
+            const int e = (int)(kk >> 23);
+            const u32 m = (kk & 0x7fffffu) | (e ? 0x800000u : 0u);
+            const int e1 = max(e, 1);
+            const int sh = e1 - ecur + 24;
+            if (sh >= 0) acc += (u64)m << sh;
+            else if (m) atomicAdd(&st[cc.tns].sum_low[e1], (u64)m);
+        }
+        if (++since >= 32) flush_acc(cc.tns);
+        ring.release();
+        cc.next();
+    }
+    if (prev >= 0) { flush_acc(prev); flush_below(prev); }
+}
+
+// The median among the gathered keys (or the flag for the histogram path), the correctly
+// rounded mean, the thresholds.  One block per tensor.
+__global__ void __launch_bounds__(1024) stats_finish_kernel(const TensorDesc* __restrict__ descs,
+                                                            TensorState* __restrict__ st, Workspace ws,
+                                                            float alpha, float beta) {
+    __shared__ u32 hist[256];
+    __shared__ u64 tab[3][256];
+    const int t = blockIdx.x, tid = threadIdx.x;
+    TensorState& s = st[t];
+    const u64 n = descs[t].numel;
+    if (n == 0) {
+        if (tid == 0) {
+            s.mean_abs_ea = 0.f;
+            s.thr_w = __fmul_rn(alpha, 0.f);
+            s.thr_o = __fmul_rn(beta, 0.f);
+        }
+        return;
+    }
+    if (tid < 256) { tab[0][tid] = s.sum_lo[tid]; tab[1][tid] = s.sum_hi[tid]; tab[2][tid] = s.sum_low[tid]; }
+    __syncthreads();
+    if (tid == 0) {
+        const float mean = exact_mean_from_tables(tab[0], tab[1], tab[2], n);
+        s.mean_abs_ea = mean;
+        s.thr_o = __fmul_rn(beta, mean);                              // beta * mean, Eq. (ro)
+    }
+    u32 med = s.median_bits;
+    if (!s.med_done) {
+        const u32 k = (u32)((n - 1) / 2), below = s.count_below, c = s.cand_count;
+        if (k < below || k - below >= c) {                           // the bracket missed the median
+            if (tid == 0) s.need_hist = 1;
+            return;
+        }
+        const u32* cand = reinterpret_cast<const u32*>(ws.surv[0] + (u64)descs[t].tile_begin * TILE);
+        med = block_select(cand, c, k - below, hist);
+        if (tid == 0) s.median_bits = med;
+    }
+    if (tid == 0) s.thr_w = __fmul_rn(alpha, __uint_as_float(med));  // alpha * median, Eq. (rw)
+}
+
 void launch_stats(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
-                  const Workspace& ws, const Params& p) {
+                  const Workspace& ws, const Params& p, CallState* call) {
     const int resid = p.median_source == 1;
+    median_sample_kernel<<<nt, 1024, 0, cfg.stream>>>(descs, st, ws, resid);
     if (tiles) {
-        const u32 grid = min(tiles, (u32)cfg.sms * 4u);
-        stats1_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, resid);
+        const u32 grid = min((tiles + SWARPS - 1) / SWARPS, (u32)cfg.sms * 2u);
+        cudaFuncSetAttribute(stats_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SweepSmem));
+        stats_sweep_kernel<<<grid, TPB, sizeof(SweepSmem), cfg.stream>>>(descs, st, nt, tiles, ws, resid, call);
     }
-    stats1_finish_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st);
-    prof_mark(cfg, ST_STATS1, tiles ? 2 : 1);
-    if (tiles) {
-        const u32 grid = min(tiles, (u32)cfg.sms * 8u);
-        stats2_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, resid);
+    stats_finish_kernel<<<nt, 1024, 0, cfg.stream>>>(descs, st, ws, p.alpha, p.beta);
+    prof_mark(cfg, ST_STATS1, tiles ? 3 : 2);
+    if (tiles) {          // the histogram path: returns at once unless a bracket missed
+        hist1_kernel<<<min(tiles, (u32)cfg.sms * 4u), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, resid);
+        hist1_finish_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st);
+        hist2_kernel<<<min(tiles, (u32)cfg.sms * 8u), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, resid);
+        hist2_finish_kernel<<<nt, 1024, 0, cfg.stream>>>(descs, st, ws, p.alpha);
+        prof_mark(cfg, ST_STATS2, 4);
     }
-    stats2_finish_kernel<<<nt, 1024, 0, cfg.stream>>>(descs, st, ws, p.alpha, p.beta);
-    prof_mark(cfg, ST_STATS2, tiles ? 2 : 1);
 }
 
 }  // namespace excp

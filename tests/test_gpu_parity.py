@@ -181,6 +181,23 @@ def test_degenerate_value_patterns(handle):
         check_against_oracle(p, cases, blob, offs, stats)
 
 
+def test_median_when_the_sample_misleads(handle):
+    """The median is bracketed from 65536 evenly spaced elements.  Here every 16th element (the
+    ones a 2^20-element tensor's sample takes) is large, so the bracket misses the true median
+    and the histogram path has to find it; a second tensor is exactly as large as the sample."""
+    n = 1 << 20
+    w_t, w_prev, ea, eas = rand_quad_np(n, 450)
+    w_t[::16] = w_prev[::16] + np.float32(0.5)
+    w_prev2 = rand_quad_np(65536, 451)
+    cases = [(w_t, w_prev, ea, eas), w_prev2, rand_quad_np(65537, 452)]
+    for mode in (0, 1):
+        p = binding.Params(median_source=mode, alpha=2e-7 if mode == 0 else 5e-5)
+        if mode == 0:
+            cases[0][0][::16] = np.float32(7.0)
+        blob, offs, stats = gpu_compress(handle, p, to_dev(cases))
+        check_against_oracle(p, cases, blob, offs, stats)
+
+
 def test_zero_kmeans_iterations_and_other_hyperparameters(handle):
     q = [rand_quad_np(60000, 500)]
     for p in (binding.Params(kmeans_iters=0, median_source=1), binding.Params(kmeans_iters=3, median_source=1, seed=99),
@@ -335,7 +352,7 @@ def test_profile_counts_launches_and_times_stages(handle):
     try:
         handle.compress_tensor(binding.Params(median_source=1, kmeans_iters=10), *dq[0], blob)
         ms, launches = handle.profile_read()
-        assert launches == 4 + 1 + 2 + 1 + 2 + 6 + 10 * 2 + 2 + 2 + 1
+        assert launches == 7 + 1 + 2 + 1 + 2 + 6 + 10 * 2 + 2 + 2 + 1
         assert ms["mask_compact"] > 0 and ms["bucket_scan"] > 0 and ms["decode"] == 0
     finally:
         handle.profile_enable(False)
