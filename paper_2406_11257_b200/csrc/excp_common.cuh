@@ -78,6 +78,11 @@ struct TensorState {             // device scratch, zeroed per group
     u32 count_below;             // elements below the bracket
     u32 med_done;                // the sample was the whole tensor: median already known
     u32 need_hist;               // the bracket missed the median: take the histogram path
+    u32 sel_hs;                  // select among the bracket's keys: bits of key - lo_key still open,
+    u32 sel_prefix;              //   the bits above them,
+    u32 sel_rank;                //   the rank wanted among the keys that share those bits
+    u32 sel_done[4];             // blocks that have added their counts, per digit pass
+    u32 sel_hist[4][256];        // digit counts per pass
     u32 pad_;
     u64 blob_off;                // start of this tensor's record in the blob
     u64 blob_bytes;

@@ -284,25 +284,31 @@ __global__ void __launch_bounds__(1024) hist2_finish_kernel(const TensorDesc* __
 
 
 // ---------------------------------------------------------------------------
-// The element of rank `rank` (0-based, ascending) among cnt 31-bit keys, by four 8-bit digit
-// passes.  Whole block (at least 256 threads); hist: 256 words of shared memory.
-__device__ static u32 block_select(const u32* __restrict__ keys, u32 cnt, u32 rank, u32* hist) {
-    u32 prefix = 0, mask = 0;
-    for (int shift = 24; shift >= 0; shift -= 8) {
+// The element of rank `rank` (0-based, ascending) among cnt keys that all lie in
+// [base, base + width], by digit passes of at most 8 bits over key - base, from the top bit of
+// width down: the digits of a narrow range spread over the bins, so the shared-memory atomics
+// do not pile up on one counter.  Whole block (at least 256 threads); hist: 256 words.
+__device__ static u32 block_select(const u32* __restrict__ keys, u32 cnt, u32 rank, u32* hist,
+                                   u32 base, u32 width) {
+    int hs = 32 - __clz(width | 1u);         // bits of key - base above hs equal `prefix`
+    u32 prefix = 0;
+    while (hs > 0) {
+        const int ls = max(hs - 8, 0);
+        const u32 dmask = (1u << (hs - ls)) - 1u;
         if (threadIdx.x < 256) hist[threadIdx.x] = 0;
         __syncthreads();
         for (u32 i = threadIdx.x; i < cnt; i += blockDim.x) {
-            const u32 key = keys[i];
-            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+            const u32 d = keys[i] - base;
+            if ((u32)((u64)d >> hs) == prefix) atomicAdd(&hist[(d >> ls) & dmask], 1u);
         }
         __syncthreads();
         u32 bin, rin, c;
         find_rank_block<256>(hist, rank, bin, rin, c);
-        prefix |= bin << shift;
-        mask |= 255u << shift;
+        prefix = (prefix << (hs - ls)) | bin;
         rank = rin;
+        hs = ls;
     }
-    return prefix;
+    return base + prefix;
 }
 
 constexpr u32 MEDIAN_SAMPLE = 65536;         // evenly spaced elements that bracket the median
@@ -314,6 +320,7 @@ __global__ void __launch_bounds__(1024) median_sample_kernel(const TensorDesc* _
                                                              TensorState* __restrict__ st, Workspace ws,
                                                              int residual_median) {
     __shared__ u32 hist[256];
+    __shared__ u32 range[2];
     const int t = blockIdx.x, tid = threadIdx.x;
     TensorState& s = st[t];
     const u64 n = descs[t].numel;
@@ -321,6 +328,9 @@ __global__ void __launch_bounds__(1024) median_sample_kernel(const TensorDesc* _
         if (tid == 0) { s.med_done = 1; s.median_bits = 0; }
         return;
     }
+    if (tid == 0) { range[0] = 0xffffffffu; range[1] = 0; }
+    __syncthreads();
+    u32 kmin = 0xffffffffu, kmax = 0;
     const u32 m = (u32)min((u64)MEDIAN_SAMPLE, n);
     u32* keys = reinterpret_cast<u32*>(ws.surv[1] + (u64)descs[t].tile_begin * TILE);
     const float* w_t = descs[t].w_t;
@@ -329,16 +339,24 @@ __global__ void __launch_bounds__(1024) median_sample_kernel(const TensorDesc* _
         const u64 i = ((u64)j * n) / m;
         float a = w_t[i];
         if (residual_median) a = __fsub_rn(a, w_prev[i]);
-        keys[j] = __float_as_uint(a) & 0x7fffffffu;
+        const u32 key = __float_as_uint(a) & 0x7fffffffu;
+        keys[j] = key;
+        kmin = min(kmin, key);
+        kmax = max(kmax, key);
     }
+    kmin = __reduce_min_sync(0xffffffffu, kmin);
+    kmax = __reduce_max_sync(0xffffffffu, kmax);
+    if ((tid & 31) == 0) { atomicMin(&range[0], kmin); atomicMax(&range[1], kmax); }
     __syncthreads();
+    kmin = range[0];
+    const u32 width = range[1] - kmin;
     if (n <= MEDIAN_SAMPLE) {
-        const u32 med = block_select(keys, m, (u32)((n - 1) / 2), hist);
+        const u32 med = block_select(keys, m, (u32)((n - 1) / 2), hist, kmin, width);
         if (tid == 0) { s.median_bits = med; s.med_done = 1; }
         return;
     }
-    const u32 lo = block_select(keys, m, m / 2 - MEDIAN_MARGIN, hist);
-    const u32 hi = block_select(keys, m, m / 2 + MEDIAN_MARGIN, hist);
+    const u32 lo = block_select(keys, m, m / 2 - MEDIAN_MARGIN, hist, kmin, width);
+    const u32 hi = block_select(keys, m, m / 2 + MEDIAN_MARGIN, hist, kmin, width);
     if (tid == 0) { s.lo_key = lo; s.hi_key = hi; }
 }
 
@@ -348,10 +366,12 @@ __global__ void __launch_bounds__(1024) median_sample_kernel(const TensorDesc* _
 constexpr int SCH = 512;             // values per stream per staged chunk
 constexpr int SST = 2;               // chunks in flight per warp
 constexpr int SWARPS = TPB / 32;
+constexpr int CAND_STAGE = 512;      // per-warp staging of bracket keys (one atomic per flush)
 
 struct SweepSmem {
     float buf[SWARPS][SST][3][SCH];
     unsigned long long bar[SWARPS][SST];
+    u32 cand[SWARPS][CAND_STAGE];    // bracket keys waiting for their place in the tensor's list
 };
 
 __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* __restrict__ descs,
@@ -371,6 +391,9 @@ __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* _
     u32 lo_key = 0, span = 0;        // bracket [lo_key, lo_key + span]
     bool want_median = false;
     u32* cand = nullptr;
+    u32* stage_keys = sm.cand[warp];
+    u32 nst = 0;                     // keys staged (warp uniform)
+    const u32 lt = (1u << lane) - 1u;
     u32 below = 0;                   // this thread's count of keys under the bracket
     u64 acc = 0;                     // this thread's share of sum |ea|, unit 2^(ecur-174)
     int ecur = 1;                    // biased exponent the unit is tied to (warp uniform)
@@ -392,6 +415,18 @@ __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* _
         below = 0;
     };
 
+    auto flush_cand = [&](int t) {
+        __syncwarp();
+        if (nst) {
+            u32 base = 0;
+            if (lane == 0) base = atomicAdd(&st[t].cand_count, nst);
+            base = __shfl_sync(0xffffffffu, base, 0);
+            for (u32 i = lane; i < nst; i += 32) cand[base + i] = stage_keys[i];
+        }
+        __syncwarp();
+        nst = 0;
+    };
+
     while (cc.tile < whi) {
         while (ic.tile < whi && ring.can_issue()) {
             if (ic.chunk == 0 && ic.enter_tile(descs, nt)) {
@@ -405,7 +440,7 @@ __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* _
             ic.next();
         }
         if (cc.chunk == 0 && cc.enter_tile(descs, nt)) {
-            if (prev >= 0) { flush_acc(prev); flush_below(prev); }
+            if (prev >= 0) { flush_acc(prev); flush_below(prev); flush_cand(prev); }
             prev = cc.tns;
             ecur = 1;
             cp[0] = descs[cc.tns].w_t; cp[1] = descs[cc.tns].w_prev; cp[2] = descs[cc.tns].ea;
@@ -438,28 +473,21 @@ __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* _
 #pragma unroll
                         for (int k = 0; k < 4; ++k) a[k] = __fsub_rn(a[k], b[k]);
                     }
-                    u32 key[4];
-                    int mine = 0;
+                    u32 key[4], bal[4];
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
                         key[k] = __float_as_uint(a[k]) & 0x7fffffffu;
                         const bool real = o + k < valid;
                         below += real && key[k] < lo_key;
-                        mine += real && key[k] - lo_key <= span;      // unsigned: false below lo_key
+                        bal[k] = __ballot_sync(0xffffffffu, real && key[k] - lo_key <= span);   // unsigned: false below lo_key
                     }
-                    if (__any_sync(0xffffffffu, mine)) {             // gather the keys inside the bracket
-                        int incl = mine;
+                    if (bal[0] | bal[1] | bal[2] | bal[3]) {         // stage the keys inside the bracket
 #pragma unroll
-                        for (int w = 1; w < 32; w <<= 1) {
-                            const int v = __shfl_up_sync(0xffffffffu, incl, w);
-                            if (lane >= w) incl += v;
+                        for (int k = 0; k < 4; ++k) {
+                            if ((bal[k] >> lane) & 1u) stage_keys[nst + __popc(bal[k] & lt)] = key[k];
+                            nst += __popc(bal[k]);
                         }
-                        u32 start = 0;
-                        if (lane == 31) start = atomicAdd(&st[cc.tns].cand_count, (u32)incl);
-                        start = __shfl_sync(0xffffffffu, start, 31) + incl - mine;
-#pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            if (o + k < valid && key[k] - lo_key <= span) cand[start++] = key[k];
+                        if (nst > CAND_STAGE - 128) flush_cand(cc.tns);
                     }
                 }
             }
@@ -488,15 +516,14 @@ __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* _
         ring.release();
         cc.next();
     }
-    if (prev >= 0) { flush_acc(prev); flush_below(prev); }
+    if (prev >= 0) { flush_acc(prev); flush_below(prev); flush_cand(prev); }
 }
 
-// The median among the gathered keys (or the flag for the histogram path), the correctly
-// rounded mean, the thresholds.  One block per tensor.
-__global__ void __launch_bounds__(1024) stats_finish_kernel(const TensorDesc* __restrict__ descs,
-                                                            TensorState* __restrict__ st, Workspace ws,
-                                                            float alpha, float beta) {
-    __shared__ u32 hist[256];
+// The correctly rounded mean and its threshold; then, per tensor, either the flag for the
+// histogram path (the bracket missed the median) or the start of the select among the
+// bracket's keys.  One block per tensor.
+__global__ void __launch_bounds__(TPB) stats_finish_kernel(const TensorDesc* __restrict__ descs,
+                                                           TensorState* __restrict__ st, float alpha, float beta) {
     __shared__ u64 tab[3][256];
     const int t = blockIdx.x, tid = threadIdx.x;
     TensorState& s = st[t];
@@ -509,25 +536,83 @@ __global__ void __launch_bounds__(1024) stats_finish_kernel(const TensorDesc* __
         }
         return;
     }
-    if (tid < 256) { tab[0][tid] = s.sum_lo[tid]; tab[1][tid] = s.sum_hi[tid]; tab[2][tid] = s.sum_low[tid]; }
+    tab[0][tid] = s.sum_lo[tid]; tab[1][tid] = s.sum_hi[tid]; tab[2][tid] = s.sum_low[tid];
     __syncthreads();
+    if (tid != 0) return;
+    const float mean = exact_mean_from_tables(tab[0], tab[1], tab[2], n);
+    s.mean_abs_ea = mean;
+    s.thr_o = __fmul_rn(beta, mean);                                  // beta * mean, Eq. (ro)
+    if (s.med_done) {
+        s.thr_w = __fmul_rn(alpha, __uint_as_float(s.median_bits));   // alpha * median, Eq. (rw)
+        return;
+    }
+    const u32 k = (u32)((n - 1) / 2), below = s.count_below, c = s.cand_count;
+    if (k < below || k - below >= c) { s.need_hist = 1; return; }
+    s.sel_hs = 32 - __clz((s.hi_key - s.lo_key) | 1u);
+    s.sel_prefix = 0;
+    s.sel_rank = k - below;
+}
+
+// One digit pass (at most 8 bits, from the top bit of the bracket's width down) of the select
+// among a tensor's bracket keys.  grid = (SEL_SLICES, tensors): every block counts the digits
+// of its slice of the keys that share the bits fixed so far, adds them to the tensor's table,
+// and the block that arrives last picks the digit.  The pass that fixes the lowest bit writes
+// the median and alpha * median (Eq. (rw)).  A tensor whose median is known returns at once.
+constexpr int SEL_SLICES = 64;
+
+__global__ void __launch_bounds__(TPB) median_digit_kernel(TensorState* __restrict__ st,
+                                                           const TensorDesc* __restrict__ descs, Workspace ws,
+                                                           int pass, float alpha) {
+    __shared__ u32 hist[256];
+    __shared__ u32 is_last;
+    const int t = blockIdx.y, tid = threadIdx.x;
+    TensorState& s = st[t];
+    if (s.med_done | s.need_hist) return;
+    const int hs = (int)s.sel_hs;
+    if (hs == 0 || descs[t].numel == 0) return;
+    const int ls = max(hs - 8, 0);
+    const u32 dmask = (1u << (hs - ls)) - 1u;
+    const u32 prefix = s.sel_prefix, base = s.lo_key, c = s.cand_count, rank = s.sel_rank;
+    const u32* __restrict__ cand = reinterpret_cast<const u32*>(ws.surv[0] + (u64)descs[t].tile_begin * TILE);
+    const u32 i0 = (u32)(((u64)c * blockIdx.x) / gridDim.x), i1 = (u32)(((u64)c * (blockIdx.x + 1)) / gridDim.x);
+    hist[tid] = 0;
+    __syncthreads();
+    u32 i = i0 + tid;
+    for (; i + 3 * TPB < i1; i += 4 * TPB) {
+        u32 d[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) d[k] = __ldcg(cand + i + k * TPB) - base;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if ((u32)((u64)d[k] >> hs) == prefix) atomicAdd(&hist[(d[k] >> ls) & dmask], 1u);
+    }
+    for (; i < i1; i += TPB) {
+        const u32 d = __ldcg(cand + i) - base;
+        if ((u32)((u64)d >> hs) == prefix) atomicAdd(&hist[(d >> ls) & dmask], 1u);
+    }
+    __syncthreads();
+    if (hist[tid]) atomicAdd(&s.sel_hist[pass][tid], hist[tid]);
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) is_last = atomicAdd(&s.sel_done[pass], 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    hist[tid] = __ldcg(&s.sel_hist[pass][tid]);
+    __syncthreads();
+    u32 bin, rin, cnt;
+    find_rank_block<256>(hist, rank, bin, rin, cnt);
     if (tid == 0) {
-        const float mean = exact_mean_from_tables(tab[0], tab[1], tab[2], n);
-        s.mean_abs_ea = mean;
-        s.thr_o = __fmul_rn(beta, mean);                              // beta * mean, Eq. (ro)
-    }
-    u32 med = s.median_bits;
-    if (!s.med_done) {
-        const u32 k = (u32)((n - 1) / 2), below = s.count_below, c = s.cand_count;
-        if (k < below || k - below >= c) {                           // the bracket missed the median
-            if (tid == 0) s.need_hist = 1;
-            return;
+        const u32 np = (prefix << (hs - ls)) | bin;
+        s.sel_prefix = np;
+        s.sel_rank = rin;
+        s.sel_hs = (u32)ls;
+        if (ls == 0) {
+            s.median_bits = base + np;
+            s.med_done = 1;
+            s.thr_w = __fmul_rn(alpha, __uint_as_float(base + np));   // alpha * median, Eq. (rw)
         }
-        const u32* cand = reinterpret_cast<const u32*>(ws.surv[0] + (u64)descs[t].tile_begin * TILE);
-        med = block_select(cand, c, k - below, hist);
-        if (tid == 0) s.median_bits = med;
     }
-    if (tid == 0) s.thr_w = __fmul_rn(alpha, __uint_as_float(med));  // alpha * median, Eq. (rw)
 }
 
 void launch_stats(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
@@ -539,8 +624,11 @@ void launch_stats(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st
         cudaFuncSetAttribute(stats_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SweepSmem));
         stats_sweep_kernel<<<grid, TPB, sizeof(SweepSmem), cfg.stream>>>(descs, st, nt, tiles, ws, resid, call);
     }
-    stats_finish_kernel<<<nt, 1024, 0, cfg.stream>>>(descs, st, ws, p.alpha, p.beta);
-    prof_mark(cfg, ST_STATS1, tiles ? 3 : 2);
+    stats_finish_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, p.alpha, p.beta);
+    if (tiles)
+        for (int pass = 0; pass < 4; ++pass)
+            median_digit_kernel<<<dim3(SEL_SLICES, nt), TPB, 0, cfg.stream>>>(st, descs, ws, pass, p.alpha);
+    prof_mark(cfg, ST_STATS1, tiles ? 7 : 2);
     if (tiles) {          // the histogram path: returns at once unless a bracket missed
         hist1_kernel<<<min(tiles, (u32)cfg.sms * 4u), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, resid);
         hist1_finish_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st);
