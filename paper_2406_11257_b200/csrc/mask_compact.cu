@@ -9,6 +9,7 @@
 // from a small scan afterwards and are only needed when the codes are packed.
 #include "excp_common.cuh"
 #include "warp_ring.cuh"
+#include <type_traits>
 
 namespace excp {
 
@@ -91,16 +92,18 @@ __global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc*
         float* seas = ws.surv[2] + (u64)cc.tile * TILE;
         // Lane l takes values l, l+32, l+64, l+96 of each run of 128, so that a ballot IS a
         // bitmap word and the survivors of one ballot go to consecutive addresses.
+        auto sweep_chunk = [&](auto full_tag) {
+        constexpr bool FULL = decltype(full_tag)::value;     // the whole chunk came by bulk copy
 #pragma unroll
         for (int step = 0; step < MCH / 128; ++step) {
-            if ((u32)step * 128u < valid) {
+            if (FULL || (u32)step * 128u < valid) {
                 u32 bw[4], bo[4];
                 float dwv[4], eav[4], easv[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const u32 i = step * 128 + k * 32 + lane;
                     float a, b, e, v;
-                    if (i < nbulk) {
+                    if (FULL || i < nbulk) {
                         a = stg[i]; b = stg[MCH + i]; e = stg[2 * MCH + i]; v = stg[3 * MCH + i];
                     } else if (i < valid) {          // ragged last values of a tensor
                         a = __ldg(cp[0] + e0 + i); b = __ldg(cp[1] + e0 + i);
@@ -144,6 +147,9 @@ __global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc*
                 }
             }
         }
+        };
+        if (valid == (u32)MCH) sweep_chunk(std::true_type{});
+        else sweep_chunk(std::false_type{});
         ring.release();
         if (cc.chunk == TileWalk<MCH>::CHUNKS_PER_TILE - 1 && lane == 0) {
             ws.tile_cnt_w[cc.tile] = rw;
