@@ -18,6 +18,7 @@
 // order in which blocks or warps run.
 #include "excp_common.cuh"
 #include "warp_ring.cuh"
+#include <type_traits>
 
 namespace excp {
 
@@ -366,12 +367,12 @@ __global__ void __launch_bounds__(1024) median_sample_kernel(const TensorDesc* _
 constexpr int SCH = 512;             // values per stream per staged chunk
 constexpr int SST = 2;               // chunks in flight per warp
 constexpr int SWARPS = TPB / 32;
-constexpr int CAND_STAGE = 512;      // per-warp staging of bracket keys (one atomic per flush)
+constexpr int QCAP = 16;             // bracket keys a lane can hold before the warp hands them over
 
 struct SweepSmem {
     float buf[SWARPS][SST][3][SCH];
     unsigned long long bar[SWARPS][SST];
-    u32 cand[SWARPS][CAND_STAGE];    // bracket keys waiting for their place in the tensor's list
+    u32 q[SWARPS][QCAP][32];         // per-lane queues of bracket keys waiting for their place in the tensor's list
 };
 
 __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* __restrict__ descs,
@@ -391,9 +392,8 @@ __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* _
     u32 lo_key = 0, span = 0;        // bracket [lo_key, lo_key + span]
     bool want_median = false;
     u32* cand = nullptr;
-    u32* stage_keys = sm.cand[warp];
-    u32 nst = 0;                     // keys staged (warp uniform)
-    const u32 lt = (1u << lane) - 1u;
+    u32* const q = &sm.q[warp][0][lane];   // this lane's queue: q[32 * j]
+    u32 nq = 0;                      // keys in it
     u32 below = 0;                   // this thread's count of keys under the bracket
     u64 acc = 0;                     // this thread's share of sum |ea|, unit 2^(ecur-174)
     int ecur = 1;                    // biased exponent the unit is tied to (warp uniform)
@@ -415,16 +415,18 @@ __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* _
         below = 0;
     };
 
-    auto flush_cand = [&](int t) {
-        __syncwarp();
-        if (nst) {
-            u32 base = 0;
-            if (lane == 0) base = atomicAdd(&st[t].cand_count, nst);
-            base = __shfl_sync(0xffffffffu, base, 0);
-            for (u32 i = lane; i < nst; i += 32) cand[base + i] = stage_keys[i];
+    auto flush_cand = [&](int t) {   // one atomic for the warp's queued keys
+        u32 incl = nq;
+#pragma unroll
+        for (int w = 1; w < 32; w <<= 1) {
+            const u32 v = __shfl_up_sync(0xffffffffu, incl, w);
+            if (lane >= w) incl += v;
         }
-        __syncwarp();
-        nst = 0;
+        u32 base = 0;
+        if (lane == 31 && incl) base = atomicAdd(&st[t].cand_count, incl);
+        base = __shfl_sync(0xffffffffu, base, 31) + incl - nq;
+        for (u32 j = 0; j < nq; ++j) cand[base + j] = q[32 * j];
+        nq = 0;
     };
 
     while (cc.tile < whi) {
@@ -458,46 +460,61 @@ __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* _
         const float* stg = ring.stage();
         u32 ke[SCH / 32];
         u32 kmax = 0;
+        auto sweep_chunk = [&](auto full_tag) {
+            constexpr bool FULL = decltype(full_tag)::value;     // the whole chunk came by bulk copy
 #pragma unroll
-        for (int r = 0; r < SCH / 128; ++r) {
-            const u32 o = r * 128 + lane * 4;
-            float a[4], b[4], e[4];
+            for (int r = 0; r < SCH / 128; ++r) {
+                const u32 o = r * 128 + lane * 4;
+                float a[4], b[4], e[4];
 #pragma unroll
-            for (int k = 0; k < 4; ++k) e[k] = 0.f;
-            if ((u32)r * 128u < valid) {
-                fetch4(stg + 2 * SCH, cp[2] + e0, o, nbulk, valid, e);
-                if (want_median) {
-                    fetch4(stg, cp[0] + e0, o, nbulk, valid, a);
-                    if (residual_median) {
-                        fetch4(stg + SCH, cp[1] + e0, o, nbulk, valid, b);
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) a[k] = __fsub_rn(a[k], b[k]);
+                for (int k = 0; k < 4; ++k) e[k] = 0.f;
+                if (FULL || (u32)r * 128u < valid) {
+                    if (FULL) {
+                        const float4 t = *reinterpret_cast<const float4*>(stg + 2 * SCH + o);
+                        e[0] = t.x; e[1] = t.y; e[2] = t.z; e[3] = t.w;
+                    } else {
+                        fetch4(stg + 2 * SCH, cp[2] + e0, o, nbulk, valid, e);
                     }
-                    u32 key[4], bal[4];
+                    if (want_median) {
+                        if (FULL) {
+                            const float4 t = *reinterpret_cast<const float4*>(stg + o);
+                            a[0] = t.x; a[1] = t.y; a[2] = t.z; a[3] = t.w;
+                        } else {
+                            fetch4(stg, cp[0] + e0, o, nbulk, valid, a);
+                        }
+                        if (residual_median) {
+                            if (FULL) {
+                                const float4 t = *reinterpret_cast<const float4*>(stg + SCH + o);
+                                b[0] = t.x; b[1] = t.y; b[2] = t.z; b[3] = t.w;
+                            } else {
+                                fetch4(stg + SCH, cp[1] + e0, o, nbulk, valid, b);
+                            }
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        key[k] = __float_as_uint(a[k]) & 0x7fffffffu;
-                        const bool real = o + k < valid;
-                        below += real && key[k] < lo_key;
-                        bal[k] = __ballot_sync(0xffffffffu, real && key[k] - lo_key <= span);   // unsigned: false below lo_key
-                    }
-                    if (bal[0] | bal[1] | bal[2] | bal[3]) {         // stage the keys inside the bracket
+                            for (int k = 0; k < 4; ++k) a[k] = __fsub_rn(a[k], b[k]);
+                        }
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
-                            if ((bal[k] >> lane) & 1u) stage_keys[nst + __popc(bal[k] & lt)] = key[k];
-                            nst += __popc(bal[k]);
+                            const u32 key = __float_as_uint(a[k]) & 0x7fffffffu;
+                            const bool real = FULL || o + k < valid;
+                            below += real && key < lo_key;
+                            if (real && key - lo_key <= span) {      // unsigned: false below lo_key
+                                q[32 * nq] = key;
+                                ++nq;
+                            }
                         }
-                        if (nst > CAND_STAGE - 128) flush_cand(cc.tns);
+                        if (__any_sync(0xffffffffu, nq > (u32)QCAP - 4u)) flush_cand(cc.tns);
                     }
                 }
-            }
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const u32 kk = __float_as_uint(e[k]) & 0x7fffffffu;
-                ke[r * 4 + k] = kk;
-                kmax = max(kmax, kk);
+                for (int k = 0; k < 4; ++k) {
+                    const u32 kk = __float_as_uint(e[k]) & 0x7fffffffu;
+                    ke[r * 4 + k] = kk;
+                    kmax = max(kmax, kk);
+                }
             }
-        }
+        };
+        if (valid == (u32)SCH) sweep_chunk(std::true_type{});
+        else sweep_chunk(std::false_type{});
         // exact sum of |ea|: integer mantissas shifted to a common unit tied to the largest
         // exponent this warp has met in this tensor
         const int emax = max((int)(__reduce_max_sync(0xffffffffu, kmax) >> 23), 1);
@@ -509,7 +526,7 @@ __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* _
             const u32 m = (kk & 0x7fffffu) | (e ? 0x800000u : 0u);
             const int e1 = max(e, 1);
             const int sh = e1 - ecur + 24;
-            if (sh >= 0) acc += (u64)m << sh;
+            if (sh >= 0) acc += (u64)m * (u64)(1u << sh);            // sh <= 24: one wide multiply-add
             else if (m) atomicAdd(&st[cc.tns].sum_low[e1], (u64)m);
         }
         if (++since >= 32) flush_acc(cc.tns);
