@@ -519,15 +519,27 @@ __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* _
         // exponent this warp has met in this tensor
         const int emax = max((int)(__reduce_max_sync(0xffffffffu, kmax) >> 23), 1);
         if (emax > ecur) { flush_acc(cc.tns); ecur = emax; }
+        const int bias = 24 - ecur;
+        u32 lowkey = 0xffffffffu;            // smallest non-zero key, minus one
 #pragma unroll
         for (int j = 0; j < SCH / 32; ++j) {
             const u32 kk = ke[j];
-            const int e = (int)(kk >> 23);
-            const u32 m = (kk & 0x7fffffu) | (e ? 0x800000u : 0u);
-            const int e1 = max(e, 1);
-            const int sh = e1 - ecur + 24;
-            if (sh >= 0) acc += (u64)m * (u64)(1u << sh);            // sh <= 24: one wide multiply-add
-            else if (m) atomicAdd(&st[cc.tns].sum_low[e1], (u64)m);
+            const u32 e1 = max(kk >> 23, 1u);
+            const u32 m = kk - ((e1 - 1u) << 23);                    // mantissa with its implicit bit (none below 2^-126)
+            u32 pow2;                                                // 2^sh, sh = e1 - ecur + 24 <= 24; 0 when sh < 0
+            asm("shl.b32 %0, 1, %1;" : "=r"(pow2) : "r"((u32)((int)e1 + bias)));   // shl clamps: a "negative" amount gives 0
+            acc += (u64)m * (u64)pow2;                               // one wide multiply-add
+            lowkey = min(lowkey, kk - 1u);
+        }
+        // rare: a non-zero value more than 24 binades under the unit goes to the table of small ones
+        const bool has_low = lowkey != 0xffffffffu && (int)max((lowkey + 1u) >> 23, 1u) + bias < 0;
+        if (__any_sync(0xffffffffu, has_low)) {
+#pragma unroll
+            for (int j = 0; j < SCH / 32; ++j) {
+                const u32 kk = ke[j];
+                const u32 e1 = max(kk >> 23, 1u);
+                if (kk && (int)e1 + bias < 0) atomicAdd(&st[cc.tns].sum_low[e1], (u64)(kk - ((e1 - 1u) << 23)));
+            }
         }
         if (++since >= 32) flush_acc(cc.tns);
         ring.release();
