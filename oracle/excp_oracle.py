@@ -44,7 +44,8 @@ readings used here (all of them deterministic, so that the result is unique):
       cannot depend on the order of summation: with E = max(floor(log2(max|x|)),
       -126) over the stream, Q(x) = rint(x * 2^(30-E)) (half-to-even), the sum
       of Q in int64, mean = fp32( fp64(sum) / fp64(count) * 2^(E-30) ).
-  R6  byte layout: see `encode_record`.
+  R6  byte layout: see `encode_record`; the layout the paper prints (an index
+      per element, 0 = pruned) is `encode_dense`, derived from the record.
 
 The paper calls Adam's first moment v_t and its second moment m_t; to stay clear
 of the clash with the usual letters the code below says `ea` (first moment,
@@ -468,6 +469,118 @@ def compress_checkpoint(tensors, p: Params):
 def decompress_checkpoint(blob: bytes, offsets, w_prev_list):
     return [decompress_tensor(blob[offsets[i]:offsets[i + 1]], w_prev_list[i])
             for i in range(len(w_prev_list))]
+
+
+# --------------------------------------------------------------------------
+# The index layout as Sections 3.3 and 4.1 print it: one code per ELEMENT, the
+# pruned ones holding the code of the zero centre (0), no bitmap.  This is the
+# (I, C) pair that Algorithm 1 hands to its archiver.
+# --------------------------------------------------------------------------
+DENSE_MAGIC = 0x44435845  # "EXCD", little endian
+
+
+def dense_section_bytes(numel: int, bits: int) -> int:
+    return _align16((numel * bits + 7) // 8)
+
+
+def dense_bytes(numel: int, bits: int) -> int:
+    return header_bytes((1 << bits) - 1) + 3 * dense_section_bytes(numel, bits)
+
+
+def dense_indices(mask: np.ndarray, codes: np.ndarray) -> np.ndarray:
+    """I(i) = code of element i (1..K) where the mask keeps it, 0 (the zero
+    centre of Section 4.1) where it is pruned."""
+    idx = np.zeros(mask.size, dtype=np.uint8)
+    idx[mask] = codes
+    return idx
+
+
+def encode_dense(numel, bits, nnz_w, nnz_o, c_w, c_ea, c_eas, idx_w, idx_ea, idx_eas) -> bytes:
+    """The dense container.  The header is the record's with magic "EXCD" and
+    the container's size at offset 48; after the centres come the indices of
+    dW, of the first moment and of the second, `bits` per element, element i at
+    bit i*bits of its section (Section 4.1: two int4 per int8), each section
+    padded with zeros to 16 bytes."""
+    k = (1 << bits) - 1
+    hb = header_bytes(k)
+    total = dense_bytes(numel, bits)
+    head = struct.pack("<IIQQQIIIIQQ", DENSE_MAGIC, VERSION, numel, nnz_w, nnz_o, bits, k, hb, 0, total, 0)
+    head += np.asarray(c_w, dtype="<f4").tobytes()
+    head += np.asarray(c_ea, dtype="<f4").tobytes()
+    head += np.asarray(c_eas, dtype="<f4").tobytes()
+    head += b"\0" * (hb - len(head))
+    out = head
+    for idx in (idx_w, idx_ea, idx_eas):
+        raw = pack_codes(np.asarray(idx, dtype=np.uint8), bits)      # padded for `numel` codes
+        out += raw[:dense_section_bytes(numel, bits)]
+    assert len(out) == total
+    return out
+
+
+def record_to_dense(blob: bytes) -> bytes:
+    """Bitmap + compacted codes -> one code per element (0 = pruned)."""
+    r = parse_record(blob)
+    return encode_dense(r["numel"], r["bits"], r["nnz_w"], r["nnz_o"], r["c_w"], r["c_ea"], r["c_eas"],
+                        dense_indices(r["m_w"], r["codes_w"]),
+                        dense_indices(r["m_o"], r["codes_ea"]),
+                        dense_indices(r["m_o"], r["codes_eas"]))
+
+
+def parse_dense(buf: bytes) -> dict:
+    if len(buf) < HEADER_FIXED:
+        raise CorruptBlob("short header")
+    (magic, version, numel, nnz_w, nnz_o, bits, k, hb, z0, total, z1) = struct.unpack_from(
+        "<IIQQQIIIIQQ", buf, 0)
+    if magic != DENSE_MAGIC or version != VERSION:
+        raise CorruptBlob("magic/version")
+    if bits not in (2, 4, 8) or k != (1 << bits) - 1 or hb != header_bytes(k):
+        raise CorruptBlob("bits/K/header size")
+    if nnz_o > nnz_w or nnz_w > numel:
+        raise CorruptBlob("counts")
+    if total != dense_bytes(numel, bits) or len(buf) < total:
+        raise CorruptBlob("container size")
+    cents = np.frombuffer(buf, dtype="<f4", count=3 * k, offset=HEADER_FIXED).reshape(3, k)
+    sb = dense_section_bytes(numel, bits)
+    idx = [unpack_codes(buf[hb + j * sb:hb + (j + 1) * sb], numel, bits) for j in range(3)]
+    if np.count_nonzero(idx[0]) != nnz_w or np.count_nonzero(idx[1]) != nnz_o:
+        raise CorruptBlob("population")
+    if np.any((idx[1] != 0) != (idx[2] != 0)):
+        raise CorruptBlob("the two moments disagree on what is kept")
+    if np.any((idx[1] != 0) & (idx[0] == 0)):
+        raise CorruptBlob("moment kept where the weight is pruned")
+    return dict(numel=numel, nnz_w=nnz_w, nnz_o=nnz_o, bits=bits, k=k, dense_bytes=total,
+                c_w=cents[0].copy(), c_ea=cents[1].copy(), c_eas=cents[2].copy(),
+                idx_w=idx[0], idx_ea=idx[1], idx_eas=idx[2])
+
+
+def decompress_dense(buf: bytes, w_prev):
+    """Algorithm 2 on the dense layout: every element looks its code up;
+    code 0 leaves W^_(t-1) untouched and gives 0 in both moments."""
+    r = parse_dense(buf)
+    w_prev = np.ascontiguousarray(w_prev, dtype=np.float32).ravel()
+    if w_prev.size != r["numel"]:
+        raise ValueError("size mismatch")
+    w_hat = w_prev.copy()
+    kept = r["idx_w"] != 0
+    w_hat[kept] = w_prev[kept] + r["c_w"][r["idx_w"][kept].astype(np.int64) - 1]
+    ea_hat = np.zeros(r["numel"], dtype=np.float32)
+    eas_hat = np.zeros(r["numel"], dtype=np.float32)
+    ko = r["idx_ea"] != 0
+    ea_hat[ko] = r["c_ea"][r["idx_ea"][ko].astype(np.int64) - 1]
+    eas_hat[ko] = r["c_eas"][r["idx_eas"][ko].astype(np.int64) - 1]
+    return w_hat, ea_hat, eas_hat
+
+
+def archive_sizes(parts, preset_extreme: bool = True) -> dict:
+    """The archiver step of Algorithm 1 (its last but one line) on the host: LZMA2 as the xz
+    container of Python's lzma module, preset 9 (extreme), over the concatenated parts."""
+    import lzma
+    raw = b"".join(parts)
+    preset = 9 | (lzma.PRESET_EXTREME if preset_extreme else 0)
+    packed = lzma.compress(raw, format=lzma.FORMAT_XZ, preset=preset)
+    if lzma.decompress(packed) != raw:
+        raise AssertionError("archiver round trip")
+    return dict(raw_bytes=len(raw), archived_bytes=len(packed))
 
 
 # --------------------------------------------------------------------------

@@ -453,3 +453,106 @@ def test_checkpoint_container_offsets():
     # the tensor index enters the K-means start
     b0, _ = orc.compress_tensor(*quads[3], orc.Params(median_source=1, seed=3), tensor_index=3)
     assert b0 == blob[offs[3]:offs[4]]
+
+
+# ------------------------------------------- dense index layout (Sections 3.3 / 4.1) and the archiver
+def rand_quad(n, seed):
+    rng = np.random.default_rng(seed)
+    wp = rng.normal(0, 0.02, n).astype(np.float32)
+    wt = (wp + rng.standard_t(3, n) * 1e-4).astype(np.float32)
+    ea = rng.normal(0, 1e-4, n).astype(np.float32)
+    eas = ((np.abs(rng.normal(0, 1, n)) * 1e-4) ** 2 + 1e-12).astype(np.float32)
+    return wt, wp, ea, eas
+
+
+def test_hand_dense_layout():
+    p = orc.Params(alpha=G["alpha"][0], beta=G["beta"][0], bits=4)
+    blob, info = orc.compress_tensor(f32("w_t"), f32("w_prev"), f32("ea"), f32("eas"), p)
+    dense = orc.record_to_dense(blob)
+    hb = orc.header_bytes(15)
+    assert len(dense) == hb + 3 * 16 == orc.dense_bytes(8, 4)
+    head = struct.unpack_from("<IIQQQIIIIQQ", dense, 0)
+    assert head == (0x44435845, 1, 8, 5, 2, 4, 15, hb, 0, len(dense), 0)
+    assert dense[64:hb] == blob[64:hb]                          # the same centres
+    for j, key in enumerate(("w", "ea", "eas")):
+        sec = dense[hb + 16 * j:hb + 16 * (j + 1)]
+        assert list(sec[:4]) == [int(v) for v in G[f"dense_bytes_{key}_abs_weight"]]
+        assert sec[4:] == b"\0" * 12
+    r = orc.parse_dense(dense)
+    for key in ("w", "ea", "eas"):
+        assert list(r["idx_" + key]) == [int(v) for v in G[f"dense_idx_{key}_abs_weight"]]
+    w, ea, eas = orc.decompress_dense(dense, f32("w_prev"))
+    np.testing.assert_array_equal(w, f32("w_hat_abs_weight"))
+    np.testing.assert_array_equal(ea, f32("ea_hat_abs_weight"))
+    np.testing.assert_array_equal(eas, f32("eas_hat_abs_weight"))
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+@pytest.mark.parametrize("n", [1, 31, 1000, 4099])
+def test_dense_layout_by_independent_unpacking(bits, n):
+    wt, wp, ea, eas = rand_quad(n, 100 + n + bits)
+    p = orc.Params(bits=bits, median_source=orc.MEDIAN_ABS_RESIDUAL, kmeans_iters=3)
+    blob, info = orc.compress_tensor(wt, wp, ea, eas, p)
+    dense = orc.record_to_dense(blob)
+    k = (1 << bits) - 1
+    hb = 16 * ((64 + 12 * k + 15) // 16)
+    sb = 16 * (((n * bits + 7) // 8 + 15) // 16)
+    assert len(dense) == hb + 3 * sb
+    # element i is `bits` bits at bit i*bits of its section; 0 exactly where the mask prunes,
+    # else the code of the survivor with i's rank
+    for j, (mask, codes) in enumerate(((info["m_w"], info["codes_w"]), (info["m_o"], info["codes_ea"]),
+                                       (info["m_o"], info["codes_eas"]))):
+        sec = int.from_bytes(dense[hb + j * sb:hb + (j + 1) * sb], "little")
+        rank = 0
+        for i in range(n):
+            got = (sec >> (i * bits)) & k
+            if mask[i]:
+                assert got == codes[rank]
+                rank += 1
+            else:
+                assert got == 0
+        assert sec >> (n * bits) == 0                         # padding
+    a = orc.decompress_tensor(blob, wp)
+    b = orc.decompress_dense(dense, wp)
+    for x, y in zip(a, b):
+        np.testing.assert_array_equal(x.view(np.uint32), y.view(np.uint32))
+
+
+def test_corrupt_dense_containers_are_refused():
+    wt, wp, ea, eas = rand_quad(500, 7)
+    blob, info = orc.compress_tensor(wt, wp, ea, eas, orc.Params(median_source=orc.MEDIAN_ABS_RESIDUAL))
+    dense = bytearray(orc.record_to_dense(blob))
+    hb = orc.header_bytes(15)
+    sb = orc.dense_section_bytes(500, 4)
+    orc.parse_dense(bytes(dense))
+    for mutate in ("magic", "short", "population", "orphan moment", "moments disagree"):
+        d = bytearray(dense)
+        if mutate == "magic":
+            d[0] ^= 1
+        elif mutate == "short":
+            d = d[:-16]
+        elif mutate == "population":
+            i = int(np.flatnonzero(~info["m_w"])[0])
+            d[hb + i // 2] |= 1 << (4 * (i % 2))
+        elif mutate == "orphan moment":
+            i = int(np.flatnonzero(~info["m_w"])[0])
+            for j in (1, 2):
+                d[hb + j * sb + i // 2] |= 1 << (4 * (i % 2))
+            struct.pack_into("<Q", d, 24, info["nnz_o"] + 1)
+        else:
+            i = int(np.flatnonzero(info["m_w"] & ~info["m_o"])[0])
+            d[hb + sb + i // 2] |= 1 << (4 * (i % 2))
+            struct.pack_into("<Q", d, 24, info["nnz_o"] + 1)
+        with pytest.raises(orc.CorruptBlob):
+            orc.parse_dense(bytes(d))
+
+
+def test_archiver_round_trip_and_sizes():
+    wt, wp, ea, eas = rand_quad(20000, 11)
+    blob, _ = orc.compress_tensor(wt, wp, ea, eas, orc.Params(median_source=orc.MEDIAN_ABS_RESIDUAL))
+    dense = orc.record_to_dense(blob)
+    a, b = orc.archive_sizes([blob]), orc.archive_sizes([dense])
+    assert a["raw_bytes"] == len(blob) and b["raw_bytes"] == len(dense)
+    assert 0 < a["archived_bytes"] <= len(blob) + 128 and 0 < b["archived_bytes"] < len(dense)
+    z = orc.archive_sizes([b"\0" * 100000])
+    assert z["archived_bytes"] < 400                          # LZMA2 collapses a run of zeros
