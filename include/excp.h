@@ -100,7 +100,7 @@ typedef struct {
 } excp_tensor_stats;
 
 /* Creates a handle on CUDA device `device` with a scratch workspace for `workspace_numel`
- * elements (about 12.3 bytes each; tensors are processed in groups whose sizes, each rounded
+ * elements (about 24.3 bytes each; tensors are processed in groups whose sizes, each rounded
  * up to 4096, sum to at most this), so the largest single tensor must not exceed it.
  * Allocates device and pinned host memory.  Returns EXCP_ERR_CUDA if the device or the
  * memory cannot be had. */
@@ -185,6 +185,45 @@ excp_status excp_decompress_checkpoint(excp_handle h, const void* blob, const si
                                        size_t num_tensors, const float* const* w_prev, const size_t* numel,
                                        float* const* w_out, float* const* ea_out, float* const* eas_out,
                                        void* cuda_stream);
+
+/* The index layout as the paper prints it (Section 3.3: the pruned entries stay zero and the
+ * cluster index I_t is saved; Section 4.1: zero occupies one of the 2^n centres, two int4 per
+ * int8): one code per ELEMENT, 0 where the element is pruned, no bitmap.  This is the (I, C) pair
+ * Algorithm 1 hands to its archiver.  Container of one tensor (little endian, sections on 16 bytes,
+ * padding zero):
+ *     the record's 64-byte header with magic "EXCD" and the CONTAINER's size at offset 48,
+ *     f32 centres of dW [K], of ea [K], of eas [K]; header padded to 16 bytes
+ *     codes of dW [numel], of ea [numel], of eas [numel]: `bits` each, element i at bit i * bits
+ * excp_dense_bytes gives its size (0 if bits is not 2, 4 or 8).
+ *
+ * excp_record_to_dense / excp_checkpoint_to_dense rewrite records (device) as dense containers
+ * (device): bitmap rank -> code, per element.
+ *   blob, tensor_offsets  as returned by excp_compress_checkpoint.
+ *   dense_out             device, dense_capacity bytes; containers back to back.
+ *   dense_offsets_out     host [num_tensors + 1] (excp_record_to_dense: dense_bytes_out, host).
+ * Return EXCP_ERR_BUFFER_TOO_SMALL before any launch if the containers do not fit, and
+ * EXCP_ERR_CORRUPT_BLOB like excp_decompress_checkpoint.  Synchronise the stream. */
+size_t excp_dense_bytes(size_t numel, int bits);
+excp_status excp_record_to_dense(excp_handle h, const void* record, size_t record_bytes, size_t numel,
+                                 void* dense_out, size_t dense_capacity, size_t* dense_bytes_out,
+                                 void* cuda_stream);
+excp_status excp_checkpoint_to_dense(excp_handle h, const void* blob, const size_t* tensor_offsets,
+                                     size_t num_tensors, const size_t* numel, void* dense_out,
+                                     size_t dense_capacity, size_t* dense_offsets_out, void* cuda_stream);
+
+/* Algorithm 2 on the dense layout: every element looks its code up; code 0 keeps W^_(t-1) bit for
+ * bit and gives 0 in both moments.  Arguments as for excp_decompress_tensor / _checkpoint, with
+ * dense containers in place of records.  EXCP_ERR_CORRUPT_BLOB if the header disagrees with the
+ * layout, the number of non-zero codes differs from the header's counts, the two moments disagree
+ * on what is kept, a moment is kept where the weight is pruned, or a code lies past the last
+ * element (every read stays inside the container even then).  Synchronise the stream. */
+excp_status excp_decompress_dense_tensor(excp_handle h, const void* dense, size_t dense_bytes,
+                                         const float* w_prev, size_t numel,
+                                         float* w_out, float* ea_out, float* eas_out, void* cuda_stream);
+excp_status excp_decompress_dense_checkpoint(excp_handle h, const void* dense, const size_t* dense_offsets,
+                                             size_t num_tensors, const float* const* w_prev, const size_t* numel,
+                                             float* const* w_out, float* const* ea_out, float* const* eas_out,
+                                             void* cuda_stream);
 
 /* excp_decompress_tensor for callers that cannot allocate memory (the paper has no counterpart:
  * this is a property of the library, not of the method).

@@ -21,7 +21,8 @@ STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED", -3: "BUFFER_TOO_SMALL",
 EXPORTS = ["excp_create", "excp_destroy", "excp_record_bytes", "excp_compress_bound",
            "excp_status_string", "excp_last_cuda_error", "excp_compress_tensor",
            "excp_compress_checkpoint", "excp_compress_checkpoint_host", "excp_decompress_tensor", "excp_decompress_checkpoint",
-           "excp_decompress_tensor_noalloc", "excp_profile_enable", "excp_profile_stage_count", "excp_profile_stage_name", "excp_profile_read"]
+           "excp_decompress_tensor_noalloc", "excp_dense_bytes", "excp_record_to_dense", "excp_checkpoint_to_dense",
+           "excp_decompress_dense_tensor", "excp_decompress_dense_checkpoint", "excp_profile_enable", "excp_profile_stage_count", "excp_profile_stage_name", "excp_profile_read"]
 
 
 class ExcpError(RuntimeError):
@@ -84,6 +85,12 @@ def load_library() -> C.CDLL:
     lib.excp_decompress_checkpoint.argtypes = [vp, vp, C.POINTER(sz), sz, C.POINTER(vp), C.POINTER(sz),
                                                C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), vp]
     lib.excp_decompress_tensor_noalloc.argtypes = [vp, sz, vp, sz, vp, vp, vp, vp]
+    lib.excp_dense_bytes.argtypes = [sz, C.c_int]
+    lib.excp_dense_bytes.restype = sz
+    lib.excp_record_to_dense.argtypes = [vp, vp, sz, sz, vp, sz, C.POINTER(sz), vp]
+    lib.excp_checkpoint_to_dense.argtypes = [vp, vp, C.POINTER(sz), sz, C.POINTER(sz), vp, sz, C.POINTER(sz), vp]
+    lib.excp_decompress_dense_tensor.argtypes = lib.excp_decompress_tensor.argtypes
+    lib.excp_decompress_dense_checkpoint.argtypes = lib.excp_decompress_checkpoint.argtypes
     lib.excp_profile_enable.argtypes = [vp, C.c_int]
     lib.excp_profile_stage_count.argtypes = []
     lib.excp_profile_stage_name.argtypes = [C.c_int]
@@ -112,6 +119,10 @@ def _stream() -> int:
 
 def record_bytes(numel: int, nnz_w: int, nnz_o: int, bits: int = 4) -> int:
     return load_library().excp_record_bytes(numel, nnz_w, nnz_o, bits)
+
+
+def dense_bytes(numel: int, bits: int = 4) -> int:
+    return load_library().excp_dense_bytes(numel, bits)
 
 
 def compress_bound(numel: int, bits: int = 4) -> int:
@@ -234,13 +245,42 @@ class Handle:
         if st != 0:
             raise ExcpError(st, "excp_decompress_tensor")
 
-    def decompress_checkpoint(self, blob: torch.Tensor, offsets, w_prev, w_out, ea_out, eas_out) -> None:
+    def decompress_checkpoint(self, blob: torch.Tensor, offsets, w_prev, w_out, ea_out, eas_out,
+                              dense: bool = False) -> None:
         n = len(w_prev)
         _check_f32_cuda(*w_prev, *w_out, *ea_out, *eas_out)
         arr = lambda ts: (C.c_void_p * n)(*[_ptr(t) for t in ts])
         numel = (C.c_size_t * n)(*[t.numel() for t in w_prev])
         offs = (C.c_size_t * (n + 1))(*offsets)
-        st = self.lib.excp_decompress_checkpoint(self._h, blob.data_ptr(), offs, n, arr(w_prev), numel,
-                                                 arr(w_out), arr(ea_out), arr(eas_out), _stream())
+        fn = self.lib.excp_decompress_dense_checkpoint if dense else self.lib.excp_decompress_checkpoint
+        st = fn(self._h, blob.data_ptr(), offs, n, arr(w_prev), numel, arr(w_out), arr(ea_out), arr(eas_out),
+                _stream())
         if st != 0:
-            raise ExcpError(st, "excp_decompress_checkpoint")
+            raise ExcpError(st, "excp_decompress_dense_checkpoint" if dense else "excp_decompress_checkpoint")
+
+    # ---- the dense index layout (Sections 3.3 / 4.1) ----------------------
+    def record_to_dense(self, record: torch.Tensor, record_bytes: int, numel: int, dense_out: torch.Tensor) -> int:
+        out = C.c_size_t(0)
+        st = self.lib.excp_record_to_dense(self._h, record.data_ptr(), record_bytes, numel, dense_out.data_ptr(),
+                                           dense_out.numel(), C.byref(out), _stream())
+        if st != 0:
+            raise ExcpError(st, "excp_record_to_dense")
+        return out.value
+
+    def checkpoint_to_dense(self, blob: torch.Tensor, offsets, numels, dense_out: torch.Tensor) -> list[int]:
+        n = len(numels)
+        offs = (C.c_size_t * (n + 1))(*offsets)
+        numel = (C.c_size_t * n)(*numels)
+        douts = (C.c_size_t * (n + 1))()
+        st = self.lib.excp_checkpoint_to_dense(self._h, blob.data_ptr(), offs, n, numel, dense_out.data_ptr(),
+                                               dense_out.numel(), douts, _stream())
+        if st != 0:
+            raise ExcpError(st, "excp_checkpoint_to_dense")
+        return list(douts)
+
+    def decompress_dense_tensor(self, dense: torch.Tensor, dense_bytes_: int, w_prev, w_out, ea_out, eas_out) -> None:
+        _check_f32_cuda(w_prev, w_out, ea_out, eas_out)
+        st = self.lib.excp_decompress_dense_tensor(self._h, dense.data_ptr(), dense_bytes_, _ptr(w_prev),
+                                                   w_prev.numel(), _ptr(w_out), _ptr(ea_out), _ptr(eas_out), _stream())
+        if st != 0:
+            raise ExcpError(st, "excp_decompress_dense_tensor")

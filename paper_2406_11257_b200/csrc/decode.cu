@@ -92,6 +92,9 @@ __global__ void __launch_bounds__(TPB) dec_scan_kernel(const DecDesc* __restrict
     }
 }
 
+// DENSE = false: Algorithm 2, fp32 outputs.  DENSE = true: the same walk writes each element's
+// code (0 where pruned) into the three sections of the dense layout instead.
+template <bool DENSE>
 __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__ descs,
                                                      const DecState* __restrict__ st, int nt, u32 tiles,
                                                      Workspace ws, CallState* call) {
@@ -160,8 +163,9 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
             const u32 e0 = r * (TPB * 4) + tid * 4;       // element within the tile
             const u64 i0 = base + e0;
             if (i0 >= n) continue;
-            float wp[4];
-            load4(d.w_prev, i0, n, wp);
+            float wp[4] = {0.f, 0.f, 0.f, 0.f};
+            if (!DENSE) load4(d.w_prev, i0, n, wp);
+            u32 nib[3] = {0, 0, 0};                       // DENSE: four codes per stream
             const u32 word = e0 >> 5, bit = e0 & 31;
             const u32 mw4 = (bw[word] >> bit) & 15u, mo4 = (bo[word] >> bit) & 15u;
             u32 rw = pw[word] + __popc(bw[word] & ((1u << bit) - 1u));
@@ -174,6 +178,7 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
                     const u32 g = offw + rw++;
                     const u32 c = (codes[0][(g >> 1) - (offw >> 1)] >> (4 * (g & 1u))) & 15u;
                     if (c == 0) bad = 1; else ow[k] = __fadd_rn(wp[k], cent[0][c - 1]);
+                    nib[0] |= c << (4 * k);
                 }
                 if ((mo4 >> k) & 1u) {
                     const u32 g = offo + ro++;
@@ -181,9 +186,16 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
                     const u32 c1 = (codes[1][ix] >> sh) & 15u, c2 = (codes[2][ix] >> sh) & 15u;
                     if (c1 == 0 || c2 == 0) bad = 1;
                     else { oa[k] = cent[1][c1 - 1]; os[k] = cent[2][c2 - 1]; }
+                    nib[1] |= c1 << (4 * k);
+                    nib[2] |= c2 << (4 * k);
                 }
             }
-            if (i0 + 4 <= n) {
+            if (DENSE) {                                  // elements i0..i0+3 are bytes i0/2, i0/2+1 of a section
+                const u64 sb = dense_section_bytes(n, BITS);
+                unsigned char* sec = d.dense + header_bytes(KMAX) + i0 / 2;
+#pragma unroll
+                for (int j = 0; j < 3; ++j) *reinterpret_cast<unsigned short*>(sec + j * sb) = (unsigned short)nib[j];
+            } else if (i0 + 4 <= n) {
                 reinterpret_cast<float4*>(d.w_out + i0)[0] = make_float4(ow[0], ow[1], ow[2], ow[3]);
                 reinterpret_cast<float4*>(d.ea_out + i0)[0] = make_float4(oa[0], oa[1], oa[2], oa[3]);
                 reinterpret_cast<float4*>(d.eas_out + i0)[0] = make_float4(os[0], os[1], os[2], os[3]);
@@ -205,8 +217,190 @@ void launch_decode(const LaunchCfg& cfg, const DecDesc* descs, DecState* st, int
     dec_scan_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, ws, call);
     prof_mark(cfg, ST_DEC_PREP, 3);
     const u32 grid = min(tiles, (u32)cfg.sms * 4u);
-    decode_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, call);
+    decode_kernel<false><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, call);
     prof_mark(cfg, ST_DECODE, 1);
+}
+
+// ---------------------------------------------------------------------------
+// The dense layout (Sections 3.3 and 4.1 as printed): header + centres as in the record (magic
+// "EXCD", the container's size at offset 48), then one code per element for dW, ea and eas.
+
+// Header, centres and the zero padding at the end of every section.  One block per tensor.
+__global__ void __launch_bounds__(64) dense_header_kernel(const DecDesc* __restrict__ descs,
+                                                          DecState* __restrict__ st, CallState* call) {
+    const int t = blockIdx.x, tid = threadIdx.x;
+    const DecDesc& d = descs[t];
+    DecState& s = st[t];
+    if (!s.valid) return;
+    const u64 total = dense_bytes(d.numel, BITS);
+    if (total > d.dense_avail) {                          // uniform over the block
+        if (tid == 0) { s.valid = 0; atomicOr(&call->flags, FLAG_BLOB_FULL); }
+        return;
+    }
+    const u32 hb = (u32)header_bytes(KMAX);
+    u32* out = reinterpret_cast<u32*>(d.dense);
+    const u32* in = reinterpret_cast<const u32*>(d.rec);
+    for (u32 w = tid; w < hb / 4; w += 64) {
+        u32 v = in[w];                                    // counts, bits, K, header size, centres, padding
+        if (w == 0) v = DENSE_MAGIC;
+        if (w == 12) v = (u32)total;
+        if (w == 13) v = (u32)(total >> 32);
+        out[w] = v;
+    }
+    const u64 sb = dense_section_bytes(d.numel, BITS);
+    if (sb && tid < 12) {                                 // last 16 bytes of each section
+        const int j = tid / 4;
+        reinterpret_cast<u32*>(d.dense + hb + (j + 1) * sb - 16)[tid % 4] = 0;
+    }
+}
+
+void launch_record_to_dense(const LaunchCfg& cfg, const DecDesc* descs, DecState* st, int nt, u32 tiles,
+                            const Workspace& ws, CallState* call) {
+    dec_validate_kernel<<<nt, 64, 0, cfg.stream>>>(descs, st, call);
+    if (tiles) {
+        dec_popcount_kernel<<<(tiles + TPB / 32 - 1) / (TPB / 32), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws);
+        dec_scan_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, ws, call);
+    }
+    dense_header_kernel<<<nt, 64, 0, cfg.stream>>>(descs, st, call);
+    prof_mark(cfg, ST_DEC_PREP, tiles ? 4 : 2);
+    if (!tiles) return;
+    const u32 grid = min(tiles, (u32)cfg.sms * 4u);
+    decode_kernel<true><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, call);
+    prof_mark(cfg, ST_DENSE, 1);
+}
+
+// Algorithm 2 on the dense layout.  validate: header against the layout; decode: every element
+// looks its code up (no ranks needed), counting the non-zero codes; check: the counts must be the
+// header's.
+__global__ void __launch_bounds__(64) dense_validate_kernel(const DecDesc* __restrict__ descs,
+                                                            DecState* __restrict__ st, CallState* call) {
+    const int t = blockIdx.x, tid = threadIdx.x;
+    const DecDesc& d = descs[t];
+    DecState& s = st[t];
+    __shared__ u32 ok;
+    if (tid == 0) {
+        ok = 0;
+        if (d.rec_avail >= HEADER_FIXED) {
+            const u32* h = reinterpret_cast<const u32*>(d.rec);
+            const u64 numel = h[2] | ((u64)h[3] << 32);
+            const u64 nnz_w = h[4] | ((u64)h[5] << 32);
+            const u64 nnz_o = h[6] | ((u64)h[7] << 32);
+            const u64 total = h[12] | ((u64)h[13] << 32);
+            if (h[0] == DENSE_MAGIC && h[1] == VERSION && numel == d.numel && h[8] == BITS && h[9] == KMAX &&
+                h[10] == header_bytes(KMAX) && nnz_o <= nnz_w && nnz_w <= numel &&
+                total == dense_bytes(numel, BITS) && total <= d.rec_avail) {
+                ok = 1;
+                s.bits = BITS;
+                s.nnz_w = (u32)nnz_w; s.nnz_o = (u32)nnz_o;
+            }
+        }
+        s.valid = ok;
+        s.cnt_w = 0; s.cnt_o = 0;
+        if (!ok) atomicOr(&call->flags, FLAG_CORRUPT);
+    }
+    __syncthreads();
+    if (ok && tid < 3 * KPAD) {
+        const int k = tid / KPAD, j = tid % KPAD;
+        s.cent[k][j] = j < KMAX ? reinterpret_cast<const float*>(d.rec + HEADER_FIXED)[k * KMAX + j] : 0.f;
+    }
+}
+
+// One bit per non-zero 4-bit code of a word of eight.
+__device__ __forceinline__ u32 nonzero_nibbles(u32 w) { return (w | (w >> 1) | (w >> 2) | (w >> 3)) & 0x11111111u; }
+
+__global__ void __launch_bounds__(TPB) dense_decode_kernel(const DecDesc* __restrict__ descs,
+                                                           DecState* __restrict__ st, int nt, u32 tiles,
+                                                           CallState* call) {
+    __shared__ float cent[3][KPAD + 1];                   // [0] = the zero centre of code 0
+    const int tid = threadIdx.x, lane = tid & 31;
+    u32 lo, hi;
+    block_range(tiles, lo, hi);
+    int cur = -1;
+    u32 tb = 0, ntl = 0;
+    u32 bad = 0, cw = 0, co = 0;
+    auto flush = [&](int t) {
+        cw = __reduce_add_sync(0xffffffffu, cw);
+        co = __reduce_add_sync(0xffffffffu, co);
+        if (lane == 0) {
+            if (cw) atomicAdd(&st[t].cnt_w, cw);
+            if (co) atomicAdd(&st[t].cnt_o, co);
+        }
+        cw = co = 0;
+    };
+    for (u32 tile = lo; tile < hi; ++tile) {
+        if (cur < 0 || tile >= tb + ntl) {
+            if (cur >= 0) flush(cur);
+            __syncthreads();
+            cur = find_tensor(descs, nt, tile);
+            tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
+            if (tid < 3 * (KPAD + 1)) {
+                const int k = tid / (KPAD + 1), j = tid % (KPAD + 1);
+                cent[k][j] = j ? st[cur].cent[k][j - 1] : 0.f;
+            }
+            __syncthreads();
+        }
+        if (!st[cur].valid) continue;
+        const DecDesc& d = descs[cur];
+        const u64 n = d.numel;
+        const u64 sb = dense_section_bytes(n, BITS);
+        const unsigned char* sec = d.rec + header_bytes(KMAX);
+        const u64 base = (u64)(tile - tb) * TILE;
+#pragma unroll
+        for (int r = 0; r < TILE / (TPB * 8); ++r) {
+            const u64 i0 = base + r * (TPB * 8) + tid * 8;     // eight elements = one word per stream
+            if (i0 >= n) continue;
+            const u32 ww = *reinterpret_cast<const u32*>(sec + i0 / 2);
+            const u32 wa = *reinterpret_cast<const u32*>(sec + sb + i0 / 2);
+            const u32 we = *reinterpret_cast<const u32*>(sec + 2 * sb + i0 / 2);
+            const u32 zw = nonzero_nibbles(ww), za = nonzero_nibbles(wa), ze = nonzero_nibbles(we);
+            cw += __popc(zw); co += __popc(za);
+            bad |= (za ^ ze) | (za & ~zw);                // moments disagree; a moment kept where the weight is pruned
+            const u32 left = n - i0 >= 8 ? 8u : (u32)(n - i0);
+            if (left < 8 && ((ww | wa | we) >> (4 * left))) bad = 1;   // codes past the last element
+            float wp[8];
+            load4(d.w_prev, i0, n, wp);
+            load4(d.w_prev, i0 + 4, n, wp + 4);
+            float ow[8], oa[8], os[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const u32 c0 = (ww >> (4 * k)) & 15u, c1 = (wa >> (4 * k)) & 15u, c2 = (we >> (4 * k)) & 15u;
+                ow[k] = c0 ? __fadd_rn(wp[k], cent[0][c0]) : wp[k];    // pruned: W^_(t-1) bit for bit
+                oa[k] = cent[1][c1];
+                os[k] = cent[2][c2];
+            }
+            if (i0 + 8 <= n) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    reinterpret_cast<float4*>(d.w_out + i0)[h] = make_float4(ow[4 * h], ow[4 * h + 1], ow[4 * h + 2], ow[4 * h + 3]);
+                    reinterpret_cast<float4*>(d.ea_out + i0)[h] = make_float4(oa[4 * h], oa[4 * h + 1], oa[4 * h + 2], oa[4 * h + 3]);
+                    reinterpret_cast<float4*>(d.eas_out + i0)[h] = make_float4(os[4 * h], os[4 * h + 1], os[4 * h + 2], os[4 * h + 3]);
+                }
+            } else {
+                for (u32 k = 0; k < left; ++k) {
+                    d.w_out[i0 + k] = ow[k]; d.ea_out[i0 + k] = oa[k]; d.eas_out[i0 + k] = os[k];
+                }
+            }
+        }
+    }
+    if (cur >= 0) flush(cur);
+    if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(&call->flags, FLAG_CORRUPT);
+}
+
+__global__ void dense_check_kernel(const DecState* __restrict__ st, int nt, CallState* call) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < nt && st[t].valid && (st[t].cnt_w != st[t].nnz_w || st[t].cnt_o != st[t].nnz_o))
+        atomicOr(&call->flags, FLAG_CORRUPT);
+}
+
+void launch_dense_decode(const LaunchCfg& cfg, const DecDesc* descs, DecState* st, int nt, u32 tiles,
+                         CallState* call) {
+    dense_validate_kernel<<<nt, 64, 0, cfg.stream>>>(descs, st, call);
+    prof_mark(cfg, ST_DEC_PREP, 1);
+    if (!tiles) return;
+    const u32 grid = min(tiles, (u32)cfg.sms * 8u);
+    dense_decode_kernel<<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, call);
+    dense_check_kernel<<<(nt + 127) / 128, 128, 0, cfg.stream>>>(st, nt, call);
+    prof_mark(cfg, ST_DENSE, 2);
 }
 
 }  // namespace excp

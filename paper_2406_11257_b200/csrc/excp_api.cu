@@ -566,7 +566,7 @@ int excp_profile_stage_count(void) { return ST_COUNT; }
 const char* excp_profile_stage_name(int stage) {
     static const char* names[ST_COUNT] = {
         "stats1", "stats2", "mask_compact", "scan_layout", "kmeans_start", "bucket_ids", "bucket_scatter",
-        "bucket_scan", "kmeans_update", "header_edges", "pack_codes", "copy_bitmaps", "dec_prep", "decode", "bucket_sum"};
+        "bucket_scan", "kmeans_update", "header_edges", "pack_codes", "copy_bitmaps", "dec_prep", "decode", "bucket_sum", "dense"};
     return stage >= 0 && stage < ST_COUNT ? names[stage] : "";
 }
 
@@ -582,6 +582,135 @@ excp_status excp_decompress_tensor(excp_handle h, const void* blob, size_t blob_
                                    float* w_out, float* ea_out, float* eas_out, void* cuda_stream) {
     const size_t offs[2] = {0, blob_bytes};
     return excp_decompress_checkpoint(h, blob, offs, 1, &w_prev, &numel, &w_out, &ea_out, &eas_out, cuda_stream);
+}
+
+size_t excp_dense_bytes(size_t numel, int bits) {
+    if (bits != 2 && bits != 4 && bits != 8) return 0;
+    return (size_t)dense_bytes(numel, bits);
+}
+
+excp_status excp_checkpoint_to_dense(excp_handle h, const void* blob, const size_t* tensor_offsets,
+                                     size_t num_tensors, const size_t* numel, void* dense_out,
+                                     size_t dense_capacity, size_t* dense_offsets_out, void* cuda_stream) {
+    if (!h || !blob || !tensor_offsets || !aligned16(blob) || !dense_offsets_out) return EXCP_ERR_INVALID_ARG;
+    dense_offsets_out[0] = 0;
+    if (num_tensors == 0) return EXCP_OK;
+    if (!numel || !dense_out || !aligned16(dense_out)) return EXCP_ERR_INVALID_ARG;
+    for (size_t i = 0; i < num_tensors; ++i) {
+        if (tensor_offsets[i + 1] < tensor_offsets[i] || (tensor_offsets[i] & 15u)) return EXCP_ERR_INVALID_ARG;
+        dense_offsets_out[i + 1] = dense_offsets_out[i] + (size_t)dense_bytes(numel[i], 4);
+    }
+    if (dense_offsets_out[num_tensors] > dense_capacity) return EXCP_ERR_BUFFER_TOO_SMALL;
+    std::vector<Group> groups;
+    if (!make_groups(h, numel, num_tensors, groups)) return EXCP_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return EXCP_ERR_CUDA;
+    if (!ensure_call_arrays(h, num_tensors)) return EXCP_ERR_CUDA;
+
+    DecDesc* hd = static_cast<DecDesc*>(h->h_desc);
+    const unsigned char* base = static_cast<const unsigned char*>(blob);
+    for (const Group& g : groups) {
+        u32 tile = 0;
+        for (size_t i = g.first; i < g.first + g.count; ++i) {
+            DecDesc& d = hd[i];
+            d = DecDesc{};
+            d.rec = base + tensor_offsets[i];
+            d.rec_avail = tensor_offsets[i + 1] - tensor_offsets[i];
+            d.dense = static_cast<unsigned char*>(dense_out) + dense_offsets_out[i];
+            d.dense_avail = dense_offsets_out[i + 1] - dense_offsets_out[i];
+            d.numel = numel[i];
+            d.tile_begin = tile;
+            d.num_tiles = (u32)((numel[i] + TILE - 1) / TILE);
+            tile += d.num_tiles;
+        }
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    LaunchCfg cfg{h->sms, stream, &h->prof};
+    h->prof.begin(stream);
+    DecDesc* dd = static_cast<DecDesc*>(h->d_desc);
+    bool ok = check(h, cudaMemsetAsync(h->d_call, 0, sizeof(CallState), stream));
+    ok = ok && check(h, cudaMemcpyAsync(dd, hd, num_tensors * sizeof(DecDesc), cudaMemcpyHostToDevice, stream));
+    for (size_t gi = 0; ok && gi < groups.size(); ++gi) {
+        const Group& g = groups[gi];
+        launch_record_to_dense(cfg, dd + g.first, h->d_dstate, (int)g.count, g.tiles, h->ws, h->d_call);
+        ok = check(h, cudaGetLastError());
+    }
+    ok = ok && check(h, cudaMemcpyAsync(h->h_call, h->d_call, sizeof(CallState), cudaMemcpyDeviceToHost, stream));
+    if (!check(h, cudaStreamSynchronize(stream)) || !ok) return EXCP_ERR_CUDA;
+    h->prof.finish();
+    return status_from_flags(h->h_call->flags);
+}
+
+excp_status excp_record_to_dense(excp_handle h, const void* record, size_t record_bytes, size_t numel,
+                                 void* dense_out, size_t dense_capacity, size_t* dense_bytes_out,
+                                 void* cuda_stream) {
+    const size_t offs[2] = {0, record_bytes};
+    size_t douts[2] = {0, 0};
+    const excp_status s = excp_checkpoint_to_dense(h, record, offs, 1, &numel, dense_out, dense_capacity, douts,
+                                                   cuda_stream);
+    if (dense_bytes_out) *dense_bytes_out = douts[1];
+    return s;
+}
+
+excp_status excp_decompress_dense_checkpoint(excp_handle h, const void* dense, const size_t* dense_offsets,
+                                             size_t num_tensors, const float* const* w_prev, const size_t* numel,
+                                             float* const* w_out, float* const* ea_out, float* const* eas_out,
+                                             void* cuda_stream) {
+    if (!h || !dense || !dense_offsets || !aligned16(dense)) return EXCP_ERR_INVALID_ARG;
+    if (num_tensors == 0) return EXCP_OK;
+    if (!w_prev || !numel || !w_out || !ea_out || !eas_out) return EXCP_ERR_INVALID_ARG;
+    for (size_t i = 0; i < num_tensors; ++i) {
+        if (dense_offsets[i + 1] < dense_offsets[i] || (dense_offsets[i] & 15u)) return EXCP_ERR_INVALID_ARG;
+        if (numel[i] == 0) continue;
+        if (!w_prev[i] || !w_out[i] || !ea_out[i] || !eas_out[i]) return EXCP_ERR_INVALID_ARG;
+        if (!aligned16(w_prev[i]) || !aligned16(w_out[i]) || !aligned16(ea_out[i]) || !aligned16(eas_out[i]))
+            return EXCP_ERR_INVALID_ARG;
+    }
+    std::vector<Group> groups;
+    if (!make_groups(h, numel, num_tensors, groups)) return EXCP_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return EXCP_ERR_CUDA;
+    if (!ensure_call_arrays(h, num_tensors)) return EXCP_ERR_CUDA;
+
+    DecDesc* hd = static_cast<DecDesc*>(h->h_desc);
+    const unsigned char* base = static_cast<const unsigned char*>(dense);
+    for (const Group& g : groups) {
+        u32 tile = 0;
+        for (size_t i = g.first; i < g.first + g.count; ++i) {
+            DecDesc& d = hd[i];
+            d = DecDesc{};
+            d.rec = base + dense_offsets[i];
+            d.rec_avail = dense_offsets[i + 1] - dense_offsets[i];
+            d.w_prev = w_prev[i]; d.w_out = w_out[i]; d.ea_out = ea_out[i]; d.eas_out = eas_out[i];
+            d.numel = numel[i];
+            d.tile_begin = tile;
+            d.num_tiles = (u32)((numel[i] + TILE - 1) / TILE);
+            tile += d.num_tiles;
+        }
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    LaunchCfg cfg{h->sms, stream, &h->prof};
+    h->prof.begin(stream);
+    DecDesc* dd = static_cast<DecDesc*>(h->d_desc);
+    bool ok = check(h, cudaMemsetAsync(h->d_call, 0, sizeof(CallState), stream));
+    ok = ok && check(h, cudaMemcpyAsync(dd, hd, num_tensors * sizeof(DecDesc), cudaMemcpyHostToDevice, stream));
+    for (size_t gi = 0; ok && gi < groups.size(); ++gi) {
+        const Group& g = groups[gi];
+        launch_dense_decode(cfg, dd + g.first, h->d_dstate, (int)g.count, g.tiles, h->d_call);
+        ok = check(h, cudaGetLastError());
+    }
+    ok = ok && check(h, cudaMemcpyAsync(h->h_call, h->d_call, sizeof(CallState), cudaMemcpyDeviceToHost, stream));
+    if (!check(h, cudaStreamSynchronize(stream)) || !ok) return EXCP_ERR_CUDA;
+    h->prof.finish();
+    return status_from_flags(h->h_call->flags);
+}
+
+excp_status excp_decompress_dense_tensor(excp_handle h, const void* dense, size_t dense_bytes_in,
+                                         const float* w_prev, size_t numel,
+                                         float* w_out, float* ea_out, float* eas_out, void* cuda_stream) {
+    const size_t offs[2] = {0, dense_bytes_in};
+    return excp_decompress_dense_checkpoint(h, dense, offs, 1, &w_prev, &numel, &w_out, &ea_out, &eas_out,
+                                            cuda_stream);
 }
 
 }  // extern "C"

@@ -34,6 +34,7 @@ constexpr u32 FLAG_INTERNAL = 8u;                // a self-check failed (candida
 constexpr u32 FLAG_TIMEOUT = 16u;                // a bounded wait on an asynchronous copy ran out
 
 constexpr u32 MAGIC = 0x50435845u;
+constexpr u32 DENSE_MAGIC = 0x44435845u;         // "EXCD": one code per element, 0 = pruned
 constexpr u32 VERSION = 1u;
 constexpr int HEADER_FIXED = 64;
 
@@ -154,12 +155,15 @@ struct DecDesc {                 // decompress: one per tensor of a group
     u64 numel;
     u32 tile_begin;
     u32 num_tiles;
+    unsigned char* dense;        // record -> dense layout: where the container goes
+    u64 dense_avail;             // and the room there
 };
 
 struct DecState {                // decompress scratch per tensor
     u32 valid;
     u32 bits;
     u32 nnz_w, nnz_o;
+    u32 cnt_w, cnt_o;            // dense layout: non-zero codes met while decoding
     u64 off_bm_w, off_bm_o, off_codes[3];
     float cent[3][KPAD];
 };
@@ -169,6 +173,10 @@ __host__ __device__ inline u64 align16(u64 n) { return (n + 15ull) & ~15ull; }
 __host__ __device__ inline u64 header_bytes(int k) { return align16(HEADER_FIXED + 12ull * k); }
 __host__ __device__ inline u64 bitmap_bytes(u64 numel) { return align16(4ull * ((numel + 31) / 32)); }
 __host__ __device__ inline u64 code_bytes(u64 nnz, int bits) { return align16((nnz * bits + 7) / 8); }
+__host__ __device__ inline u64 dense_section_bytes(u64 numel, int bits) { return align16((numel * bits + 7) / 8); }
+__host__ __device__ inline u64 dense_bytes(u64 numel, int bits) {
+    return header_bytes((1 << bits) - 1) + 3 * dense_section_bytes(numel, bits);
+}
 __host__ __device__ inline u64 record_bytes(u64 numel, u64 nnz_w, u64 nnz_o, int bits) {
     return header_bytes((1 << bits) - 1) + 2 * bitmap_bytes(numel) + code_bytes(nnz_w, bits) +
            2 * code_bytes(nnz_o, bits);
@@ -276,7 +284,7 @@ __device__ inline void scan_tile_counts(u32 tb, u32 ntl, const Workspace& ws, u3
 enum Stage {                       // for the optional per-stage event timing
     ST_STATS1 = 0, ST_STATS2, ST_MASK_COMPACT, ST_SCAN_LAYOUT, ST_KMEANS_START, ST_BUCKET_IDS, ST_BUCKET_SCATTER,
     ST_BUCKET_SCAN, ST_KMEANS_UPDATE, ST_HEADER_EDGES, ST_PACK_CODES, ST_COPY_BITMAPS, ST_DEC_PREP,
-    ST_DECODE, ST_BUCKET_SUM, ST_COUNT
+    ST_DECODE, ST_BUCKET_SUM, ST_DENSE, ST_COUNT
 };
 
 struct Profiler;
@@ -300,5 +308,9 @@ void launch_pack(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int
                  TensorResult* results);
 void launch_decode(const LaunchCfg&, const DecDesc* descs, DecState* st, int nt, u32 tiles,
                    const Workspace& ws, CallState* call);
+void launch_record_to_dense(const LaunchCfg&, const DecDesc* descs, DecState* st, int nt, u32 tiles,
+                            const Workspace& ws, CallState* call);
+void launch_dense_decode(const LaunchCfg&, const DecDesc* descs, DecState* st, int nt, u32 tiles,
+                         CallState* call);
 
 }  // namespace excp

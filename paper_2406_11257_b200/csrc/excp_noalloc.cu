@@ -81,7 +81,7 @@ extern "C" excp_status excp_decompress_tensor_noalloc(const void* blob, size_t b
     }
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    DecDesc d;
+    DecDesc d{};
     d.rec = static_cast<const unsigned char*>(blob);
     d.rec_avail = blob_bytes;
     d.w_prev = w_prev; d.w_out = w_out; d.ea_out = ea_out; d.eas_out = eas_out;
