@@ -49,6 +49,9 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-decompress", action="store_true")
+    ap.add_argument("--no-dense", action="store_true", help="skip the dense-layout and archiver leg")
+    ap.add_argument("--archive-params", type=int, default=17_000_000,
+                    help="largest tensor whose record and dense container go through the host archiver")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--max-tensors", type=int, default=None, help="debug: only the first tensors of the list")
     return ap.parse_args()
@@ -337,6 +340,62 @@ def run_ours(args):
                              "algorithmic_gbs": dec_bytes / (dms * 1e-3) / 1e9,
                              "hbm_frac_of_measured": dec_bytes / (dms * 1e-3) / 1e9 / peak,
                              "calls_per_step": len(chunks)}
+
+        # ---- the dense index layout of Sections 3.3 / 4.1 and the archiver step of Algorithm 1 -------
+        if not args.no_dense:
+            numels = [n for _, n in shapes]
+            dsz = [binding.dense_bytes(n) for n in numels]
+            dense_total = sum(dsz)
+            cap = max(sum(dsz[i] for i, _, _ in ch) for ch in chunks)
+            dense = torch.empty(cap, dtype=torch.uint8, device=dev)          # one chunk of tensors at a time
+            evs = []
+
+            def dense_round(timed):
+                for ch in chunks:
+                    i0, i1 = ch[0][0], ch[-1][0] + 1
+                    wp = [quads[i][1] for i, _, _ in ch]
+                    e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+                    e[0].record()
+                    doffs = h.checkpoint_to_dense(blob[offs[i0]:], [o - offs[i0] for o in offs[i0:i1 + 1]],
+                                                  numels[i0:i1], dense)
+                    e[1].record()
+                    h.decompress_checkpoint(dense, doffs, wp, [out_w[o:o + n] for _, o, n in ch],
+                                            [out_a[o:o + n] for _, o, n in ch], [out_s[o:o + n] for _, o, n in ch],
+                                            dense=True)
+                    e[2].record()
+                    if timed:
+                        evs.append(e)
+            dense_round(False)
+            for _ in range(args.steps):
+                dense_round(True)
+            torch.cuda.synchronize()
+            cms = sum(e[0].elapsed_time(e[1]) for e in evs) / args.steps
+            ddms = sum(e[1].elapsed_time(e[2]) for e in evs) / args.steps
+            conv_bytes = blob_bytes + dense_total                       # the records read, the containers written
+            ddec_bytes = dense_total + 4 * n_tot + 12 * n_tot
+            # the archiver on the host (LZMA2, preset 9 extreme) over a bounded sample of both layouts
+            import lzma
+            pick = next((i for i, n in enumerate(numels) if n <= args.archive_params), 0)
+            rec_raw = blob[offs[pick]:offs[pick + 1]]
+            nb = h.record_to_dense(rec_raw, offs[pick + 1] - offs[pick], numels[pick], dense)
+            ta = time.time()
+            arch = {}
+            for name, t in (("record", rec_raw), ("dense", dense[:nb])):
+                rawb = t.cpu().numpy().tobytes()
+                arch[name + "_bytes"] = len(rawb)
+                arch[name + "_xz_bytes"] = len(lzma.compress(rawb, format=lzma.FORMAT_XZ, preset=9 | lzma.PRESET_EXTREME))
+            out["dense_layout"] = {
+                "to_dense_ms": cms, "to_dense_gbs": conv_bytes / (cms * 1e-3) / 1e9,
+                "to_dense_frac_of_measured": conv_bytes / (cms * 1e-3) / 1e9 / peak,
+                "decode_ms": ddms, "decode_params_per_s": n_tot / (ddms * 1e-3),
+                "decode_gbs": ddec_bytes / (ddms * 1e-3) / 1e9,
+                "decode_frac_of_measured": ddec_bytes / (ddms * 1e-3) / 1e9 / peak,
+                "dense_bytes": dense_total, "ratio_vs_12B_per_param": 12 * n_tot / dense_total,
+                "archive": dict(arch, sample=f"tensor {pick} ({shapes[pick][0]}, {numels[pick]} params) of the workload, "
+                                             f"xz preset 9 extreme, {time.time() - ta:.1f} s on the host",
+                                record_xz_ratio_vs_12B=12 * numels[pick] / arch["record_xz_bytes"],
+                                dense_xz_ratio_vs_12B=12 * numels[pick] / arch["dense_xz_bytes"])}
+            del dense
         del out_w, out_a, out_s
 
     # ---- end to end through the host-buffer entry point ----------------------

@@ -101,7 +101,7 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
     __shared__ u32 bw[TILE_WORDS], bo[TILE_WORDS];
     __shared__ u32 pw[TILE_WORDS], po[TILE_WORDS];        // survivors before each word, within the tile
     __shared__ u32 wsum[2][TILE_WORDS / 32];
-    __shared__ unsigned char codes[3][TILE / 2 + 16];
+    __shared__ u32 codes[3][TILE / 8 + 4];                // the tile's code words (+ alignment slack, + one zero word)
     __shared__ float cent[3][KPAD];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     u32 lo, hi;
@@ -140,15 +140,18 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
             pw[tid] = ia - ca; po[tid] = ib - cb;
             if (lane == 31) { wsum[0][warp] = ia; wsum[1][warp] = ib; }
         }
-        // stage the code bytes of this tile's survivors (ranks [off, off + cnt))
+        // stage the code words of this tile's survivors (ranks [off, off + cnt)): whole aligned
+        // 32-bit words of the sections (a section is padded to 16 bytes, so the last word exists)
+        const u32 fw = offw / 8, fo = offo / 8;           // first staged word of the weight / moment sections
+        const u32 nww = cntw ? (offw + cntw + 7) / 8 - fw : 0;
+        const u32 nwo = cnto ? (offo + cnto + 7) / 8 - fo : 0;
         {
-            const unsigned char* src = d.rec + s.off_codes[0] + offw / 2;
-            const u32 nb = cntw ? (offw + cntw + 1) / 2 - offw / 2 : 0;
-            for (u32 i = tid; i < nb; i += TPB) codes[0][i] = src[i];
-            const unsigned char* s1 = d.rec + s.off_codes[1] + offo / 2;
-            const unsigned char* s2 = d.rec + s.off_codes[2] + offo / 2;
-            const u32 no = cnto ? (offo + cnto + 1) / 2 - offo / 2 : 0;
-            for (u32 i = tid; i < no; i += TPB) { codes[1][i] = s1[i]; codes[2][i] = s2[i]; }
+            const u32* s0 = reinterpret_cast<const u32*>(d.rec + s.off_codes[0]) + fw;
+            const u32* s1 = reinterpret_cast<const u32*>(d.rec + s.off_codes[1]) + fo;
+            const u32* s2 = reinterpret_cast<const u32*>(d.rec + s.off_codes[2]) + fo;
+            for (u32 i = tid; i < nww; i += TPB) codes[0][i] = s0[i];
+            for (u32 i = tid; i < nwo; i += TPB) { codes[1][i] = s1[i]; codes[2][i] = s2[i]; }
+            if (tid == 0) { codes[0][nww] = 0; codes[1][nwo] = 0; codes[2][nwo] = 0; }   // upper half of the last window
         }
         __syncthreads();
         if (tid < TILE_WORDS) {
@@ -158,43 +161,58 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
         }
         __syncthreads();
         const u64 base = (u64)(tile - tb) * TILE;
+        const u32 qw0 = offw - 8 * fw, qo0 = offo - 8 * fo;   // staged nibble index of the tile's first survivor
 #pragma unroll
         for (int r = 0; r < ROUNDS; ++r) {
             const u32 e0 = r * (TPB * 4) + tid * 4;       // element within the tile
             const u64 i0 = base + e0;
-            if (i0 >= n) continue;
+            const bool live = i0 < n;
+            if (!DENSE && !live) continue;
             float wp[4] = {0.f, 0.f, 0.f, 0.f};
             if (!DENSE) load4(d.w_prev, i0, n, wp);
-            u32 nib[3] = {0, 0, 0};                       // DENSE: four codes per stream
             const u32 word = e0 >> 5, bit = e0 & 31;
             const u32 mw4 = (bw[word] >> bit) & 15u, mo4 = (bo[word] >> bit) & 15u;
-            u32 rw = pw[word] + __popc(bw[word] & ((1u << bit) - 1u));
-            u32 ro = po[word] + __popc(bo[word] & ((1u << bit) - 1u));
+            // this thread's survivors have consecutive ranks, so their codes are consecutive
+            // nibbles: one 32-bit window per stream holds all four
+            const u32 qw = qw0 + pw[word] + __popc(bw[word] & ((1u << bit) - 1u));
+            const u32 qo = qo0 + po[word] + __popc(bo[word] & ((1u << bit) - 1u));
+            u32 win0 = __funnelshift_r(codes[0][qw >> 3], codes[0][(qw >> 3) + 1], 4 * (qw & 7u));
+            u32 win1 = __funnelshift_r(codes[1][qo >> 3], codes[1][(qo >> 3) + 1], 4 * (qo & 7u));
+            u32 win2 = __funnelshift_r(codes[2][qo >> 3], codes[2][(qo >> 3) + 1], 4 * (qo & 7u));
             float ow[4], oa[4], os[4];
+            u32 nib0 = 0, nib1 = 0, nib2 = 0;             // DENSE: the four codes per stream
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 ow[k] = wp[k]; oa[k] = 0.f; os[k] = 0.f;
                 if ((mw4 >> k) & 1u) {
-                    const u32 g = offw + rw++;
-                    const u32 c = (codes[0][(g >> 1) - (offw >> 1)] >> (4 * (g & 1u))) & 15u;
+                    const u32 c = win0 & 15u;
+                    win0 >>= 4;
                     if (c == 0) bad = 1; else ow[k] = __fadd_rn(wp[k], cent[0][c - 1]);
-                    nib[0] |= c << (4 * k);
+                    nib0 |= c << (4 * k);
                 }
                 if ((mo4 >> k) & 1u) {
-                    const u32 g = offo + ro++;
-                    const u32 ix = (g >> 1) - (offo >> 1), sh = 4 * (g & 1u);
-                    const u32 c1 = (codes[1][ix] >> sh) & 15u, c2 = (codes[2][ix] >> sh) & 15u;
+                    const u32 c1 = win1 & 15u, c2 = win2 & 15u;
+                    win1 >>= 4; win2 >>= 4;
                     if (c1 == 0 || c2 == 0) bad = 1;
                     else { oa[k] = cent[1][c1 - 1]; os[k] = cent[2][c2 - 1]; }
-                    nib[1] |= c1 << (4 * k);
-                    nib[2] |= c2 << (4 * k);
+                    nib1 |= c1 << (4 * k);
+                    nib2 |= c2 << (4 * k);
                 }
             }
-            if (DENSE) {                                  // elements i0..i0+3 are bytes i0/2, i0/2+1 of a section
+            if (DENSE) {
+                // eight lanes hold 32 consecutive elements = 16 bytes of each section: gather them in
+                // the first of the eight and write them with one store
+                u32 v[3] = {nib0, nib1, nib2};
                 const u64 sb = dense_section_bytes(n, BITS);
                 unsigned char* sec = d.dense + header_bytes(KMAX) + i0 / 2;
 #pragma unroll
-                for (int j = 0; j < 3; ++j) *reinterpret_cast<unsigned short*>(sec + j * sb) = (unsigned short)nib[j];
+                for (int j = 0; j < 3; ++j) {
+                    const u32 pair = v[j] | (__shfl_down_sync(0xffffffffu, v[j], 1) << 16);
+                    const u32 y = __shfl_down_sync(0xffffffffu, pair, 2);
+                    const u32 z = __shfl_down_sync(0xffffffffu, pair, 4);
+                    const u32 w = __shfl_down_sync(0xffffffffu, pair, 6);
+                    if ((lane & 7) == 0 && live) *reinterpret_cast<uint4*>(sec + j * sb) = make_uint4(pair, y, z, w);
+                }
             } else if (i0 + 4 <= n) {
                 reinterpret_cast<float4*>(d.w_out + i0)[0] = make_float4(ow[0], ow[1], ow[2], ow[3]);
                 reinterpret_cast<float4*>(d.ea_out + i0)[0] = make_float4(oa[0], oa[1], oa[2], oa[3]);
