@@ -282,7 +282,7 @@ void launch_record_to_dense(const LaunchCfg& cfg, const DecDesc* descs, DecState
     dense_header_kernel<<<nt, 64, 0, cfg.stream>>>(descs, st, call);
     prof_mark(cfg, ST_DEC_PREP, tiles ? 4 : 2);
     if (!tiles) return;
-    const u32 grid = min(tiles, (u32)cfg.sms * 4u);
+    const u32 grid = min(tiles, (u32)cfg.sms * 8u);
     decode_kernel<true><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, call);
     prof_mark(cfg, ST_DENSE, 1);
 }
@@ -364,35 +364,31 @@ __global__ void __launch_bounds__(TPB) dense_decode_kernel(const DecDesc* __rest
         const unsigned char* sec = d.rec + header_bytes(KMAX);
         const u64 base = (u64)(tile - tb) * TILE;
 #pragma unroll
-        for (int r = 0; r < TILE / (TPB * 8); ++r) {
-            const u64 i0 = base + r * (TPB * 8) + tid * 8;     // eight elements = one word per stream
+        for (int r = 0; r < ROUNDS; ++r) {
+            const u64 i0 = base + r * (TPB * 4) + tid * 4;     // four elements = 16 bits per stream
             if (i0 >= n) continue;
-            const u32 ww = *reinterpret_cast<const u32*>(sec + i0 / 2);
-            const u32 wa = *reinterpret_cast<const u32*>(sec + sb + i0 / 2);
-            const u32 we = *reinterpret_cast<const u32*>(sec + 2 * sb + i0 / 2);
+            const u32 ww = *reinterpret_cast<const unsigned short*>(sec + i0 / 2);
+            const u32 wa = *reinterpret_cast<const unsigned short*>(sec + sb + i0 / 2);
+            const u32 we = *reinterpret_cast<const unsigned short*>(sec + 2 * sb + i0 / 2);
             const u32 zw = nonzero_nibbles(ww), za = nonzero_nibbles(wa), ze = nonzero_nibbles(we);
             cw += __popc(zw); co += __popc(za);
             bad |= (za ^ ze) | (za & ~zw);                // moments disagree; a moment kept where the weight is pruned
-            const u32 left = n - i0 >= 8 ? 8u : (u32)(n - i0);
-            if (left < 8 && ((ww | wa | we) >> (4 * left))) bad = 1;   // codes past the last element
-            float wp[8];
+            const u32 left = n - i0 >= 4 ? 4u : (u32)(n - i0);
+            if (left < 4 && ((ww | wa | we) >> (4 * left))) bad = 1;   // codes past the last element
+            float wp[4];
             load4(d.w_prev, i0, n, wp);
-            load4(d.w_prev, i0 + 4, n, wp + 4);
-            float ow[8], oa[8], os[8];
+            float ow[4], oa[4], os[4];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
+            for (int k = 0; k < 4; ++k) {
                 const u32 c0 = (ww >> (4 * k)) & 15u, c1 = (wa >> (4 * k)) & 15u, c2 = (we >> (4 * k)) & 15u;
                 ow[k] = c0 ? __fadd_rn(wp[k], cent[0][c0]) : wp[k];    // pruned: W^_(t-1) bit for bit
                 oa[k] = cent[1][c1];
                 os[k] = cent[2][c2];
             }
-            if (i0 + 8 <= n) {
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    reinterpret_cast<float4*>(d.w_out + i0)[h] = make_float4(ow[4 * h], ow[4 * h + 1], ow[4 * h + 2], ow[4 * h + 3]);
-                    reinterpret_cast<float4*>(d.ea_out + i0)[h] = make_float4(oa[4 * h], oa[4 * h + 1], oa[4 * h + 2], oa[4 * h + 3]);
-                    reinterpret_cast<float4*>(d.eas_out + i0)[h] = make_float4(os[4 * h], os[4 * h + 1], os[4 * h + 2], os[4 * h + 3]);
-                }
+            if (left == 4) {
+                reinterpret_cast<float4*>(d.w_out + i0)[0] = make_float4(ow[0], ow[1], ow[2], ow[3]);
+                reinterpret_cast<float4*>(d.ea_out + i0)[0] = make_float4(oa[0], oa[1], oa[2], oa[3]);
+                reinterpret_cast<float4*>(d.eas_out + i0)[0] = make_float4(os[0], os[1], os[2], os[3]);
             } else {
                 for (u32 k = 0; k < left; ++k) {
                     d.w_out[i0 + k] = ow[k]; d.ea_out[i0 + k] = oa[k]; d.eas_out[i0 + k] = os[k];
