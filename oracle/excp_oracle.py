@@ -71,6 +71,19 @@ HEADER_FIXED = 64
 MEDIAN_ABS_WEIGHT = 0
 MEDIAN_ABS_RESIDUAL = 1
 
+# Ablation switches (the M2W / W2M columns of the ViT table, the residual / prune / quant columns
+# of the ablation table in Section 4.3).  0 = the full method.
+FLAG_NO_W2M = 1        # M_o(i) = [ |ea(i)| > r_o ] without the conjunction with M_w
+FLAG_NO_M2W = 2        # weights pruned by a set threshold: M_w(i) = [ |dW(i)| > alpha ]
+FLAG_NO_RESIDUAL = 4   # the weights themselves are compressed, not their residual
+FLAG_NO_PRUNE = 8      # every element is kept
+FLAG_NO_QUANT = 16     # the survivors are stored as fp32, no K-means
+FLAGS_ALL = 31
+# What a record says about itself at header offset 44
+REC_MOMENTS_FREE = 1   # M_o need not lie inside M_w
+REC_ABSOLUTE = 2       # the weight stream is W, not dW: Algorithm 2 does not add W^_(t-1)
+REC_RAW = 4            # sections hold fp32 survivors (bits = 32, K = 0)
+
 _M64 = (1 << 64) - 1
 
 
@@ -83,6 +96,7 @@ class Params:
     kmeans_iters: int = 10
     seed: int = 0
     median_source: int = MEDIAN_ABS_WEIGHT
+    flags: int = 0
 
 
 class InvalidInput(ValueError):
@@ -193,6 +207,19 @@ def moment_mask(ea: np.ndarray, m_w: np.ndarray, beta, mean) -> tuple[np.ndarray
     return (np.abs(ea) > thr_o) & m_w, thr_o
 
 
+def weight_mask_set_threshold(dw: np.ndarray, alpha) -> tuple[np.ndarray, np.float32]:
+    """The "no M2W" row of the ViT table: the weights are pruned by a threshold that is set,
+    not derived from the second moment; here alpha itself is that threshold."""
+    thr_w = np.float32(alpha)
+    return np.abs(dw).astype(np.float32) > thr_w, thr_w
+
+
+def moment_mask_alone(ea: np.ndarray, beta, mean) -> tuple[np.ndarray, np.float32]:
+    """The "no W2M" row of the ViT table: M_o(i) = [ |ea(i)| > r_o ], the weight mask ignored."""
+    thr_o = np.float32(np.float32(beta) * np.float32(mean))
+    return np.abs(ea) > thr_o, thr_o
+
+
 # --------------------------------------------------------------------------
 # Section 3.3: non-uniform quantisation (reading R5)
 # --------------------------------------------------------------------------
@@ -281,6 +308,11 @@ def _align16(n: int) -> int:
     return (n + 15) & ~15
 
 
+def centres_of(bits: int) -> int:
+    """K = 2^bits - 1 centres; none when the survivors are stored raw (bits = 32)."""
+    return 0 if bits == 32 else (1 << bits) - 1
+
+
 def header_bytes(k: int) -> int:
     return _align16(HEADER_FIXED + 3 * 4 * k)
 
@@ -294,7 +326,7 @@ def code_bytes(nnz: int, bits: int) -> int:
 
 
 def record_bytes(numel: int, nnz_w: int, nnz_o: int, bits: int) -> int:
-    k = (1 << bits) - 1
+    k = centres_of(bits)
     return (header_bytes(k) + 2 * bitmap_bytes(numel) + code_bytes(nnz_w, bits)
             + 2 * code_bytes(nnz_o, bits))
 
@@ -333,31 +365,40 @@ def unpack_bitmap(raw: bytes, numel: int) -> np.ndarray:
     return np.unpackbits(b, bitorder="little")[:numel].astype(bool)
 
 
-def encode_record(numel, bits, m_w, m_o, c_w, c_ea, c_eas, codes_w, codes_ea, codes_eas) -> bytes:
+def encode_record(numel, bits, m_w, m_o, c_w, c_ea, c_eas, codes_w, codes_ea, codes_eas, rec_flags: int = 0) -> bytes:
     """One tensor's record.  Little endian; every section starts on 16 bytes;
     padding is zero.
 
       0  u32 magic "EXCP"     4  u32 version (1)    8  u64 numel
      16  u64 nnz_w           24  u64 nnz_o         32  u32 bits   36 u32 K
-     40  u32 header bytes    44  u32 zero          48  u64 record bytes
+     40  u32 header bytes    44  u32 record flags  48  u64 record bytes
      56  u64 zero
      64  fp32 centres of dW [K], of the first moment [K], of the second [K]
      ..  bitmap of M_w, bitmap of M_o       (u32 words, LSB = lowest index)
      ..  codes of dW, of the first moment, of the second moment (survivors in
          index order, `bits` each, value 1..K)
+    Record flags (ablation variants; 0 for the full method): REC_MOMENTS_FREE, REC_ABSOLUTE,
+    REC_RAW.  With REC_RAW bits = 32, K = 0, there are no centres and the three sections hold
+    the survivors themselves as fp32 (codes_* are then float32 arrays).
     """
-    k = (1 << bits) - 1
+    k = centres_of(bits)
     nnz_w = int(np.count_nonzero(m_w))
     nnz_o = int(np.count_nonzero(m_o))
     hb = header_bytes(k)
     total = record_bytes(numel, nnz_w, nnz_o, bits)
-    head = struct.pack("<IIQQQIIIIQQ", MAGIC, VERSION, numel, nnz_w, nnz_o, bits, k, hb, 0, total, 0)
-    head += np.asarray(c_w, dtype="<f4").tobytes()
-    head += np.asarray(c_ea, dtype="<f4").tobytes()
-    head += np.asarray(c_eas, dtype="<f4").tobytes()
+    head = struct.pack("<IIQQQIIIIQQ", MAGIC, VERSION, numel, nnz_w, nnz_o, bits, k, hb, rec_flags, total, 0)
+    if k:
+        head += np.asarray(c_w, dtype="<f4").tobytes()
+        head += np.asarray(c_ea, dtype="<f4").tobytes()
+        head += np.asarray(c_eas, dtype="<f4").tobytes()
     head += b"\0" * (hb - len(head))
-    out = (head + pack_bitmap(m_w) + pack_bitmap(m_o) + pack_codes(codes_w, bits)
-           + pack_codes(codes_ea, bits) + pack_codes(codes_eas, bits))
+    out = head + pack_bitmap(m_w) + pack_bitmap(m_o)
+    for c in (codes_w, codes_ea, codes_eas):
+        if bits == 32:
+            raw = np.asarray(c, dtype="<f4").tobytes()
+            out += raw + b"\0" * (code_bytes(len(c), 32) - len(raw))
+        else:
+            out += pack_codes(c, bits)
     assert len(out) == total
     return out
 
@@ -365,13 +406,17 @@ def encode_record(numel, bits, m_w, m_o, c_w, c_ea, c_eas, codes_w, codes_ea, co
 def parse_record(blob: bytes) -> dict:
     if len(blob) < HEADER_FIXED:
         raise CorruptBlob("short header")
-    (magic, version, numel, nnz_w, nnz_o, bits, k, hb, z0, total, z1) = struct.unpack_from(
+    (magic, version, numel, nnz_w, nnz_o, bits, k, hb, rflags, total, z1) = struct.unpack_from(
         "<IIQQQIIIIQQ", blob, 0)
     if magic != MAGIC or version != VERSION:
         raise CorruptBlob("magic/version")
-    if bits not in (2, 4, 8) or k != (1 << bits) - 1 or hb != header_bytes(k):
+    if rflags & ~(REC_MOMENTS_FREE | REC_ABSOLUTE | REC_RAW):
+        raise CorruptBlob("record flags")
+    raw_values = bool(rflags & REC_RAW)
+    if bits not in ((32,) if raw_values else (2, 4, 8)) or k != centres_of(bits) or hb != header_bytes(k):
         raise CorruptBlob("bits/K/header size")
-    if nnz_o > nnz_w or nnz_w > numel:
+    free = bool(rflags & REC_MOMENTS_FREE)
+    if (nnz_o > nnz_w and not free) or nnz_w > numel or nnz_o > numel:
         raise CorruptBlob("counts")
     if total != record_bytes(numel, nnz_w, nnz_o, bits) or len(blob) < total:
         raise CorruptBlob("record size")
@@ -382,17 +427,22 @@ def parse_record(blob: bytes) -> dict:
     m_o = unpack_bitmap(blob[off:off + bb], numel); off += bb
     if np.count_nonzero(m_w) != nnz_w or np.count_nonzero(m_o) != nnz_o:
         raise CorruptBlob("bitmap population")
-    if np.any(m_o & ~m_w):
+    if np.any(m_o & ~m_w) and not free:
         raise CorruptBlob("moment kept where the weight is pruned")
     cw = code_bytes(nnz_w, bits)
     co = code_bytes(nnz_o, bits)
-    codes_w = unpack_codes(blob[off:off + cw], nnz_w, bits); off += cw
-    codes_ea = unpack_codes(blob[off:off + co], nnz_o, bits); off += co
-    codes_eas = unpack_codes(blob[off:off + co], nnz_o, bits); off += co
-    for c in (codes_w, codes_ea, codes_eas):
-        if c.size and (c.min() < 1 or c.max() > k):
-            raise CorruptBlob("code out of range")
-    return dict(numel=numel, nnz_w=nnz_w, nnz_o=nnz_o, bits=bits, k=k, record_bytes=total,
+    if raw_values:
+        codes_w = np.frombuffer(blob, dtype="<f4", count=nnz_w, offset=off).copy(); off += cw
+        codes_ea = np.frombuffer(blob, dtype="<f4", count=nnz_o, offset=off).copy(); off += co
+        codes_eas = np.frombuffer(blob, dtype="<f4", count=nnz_o, offset=off).copy(); off += co
+    else:
+        codes_w = unpack_codes(blob[off:off + cw], nnz_w, bits); off += cw
+        codes_ea = unpack_codes(blob[off:off + co], nnz_o, bits); off += co
+        codes_eas = unpack_codes(blob[off:off + co], nnz_o, bits); off += co
+        for c in (codes_w, codes_ea, codes_eas):
+            if c.size and (c.min() < 1 or c.max() > k):
+                raise CorruptBlob("code out of range")
+    return dict(numel=numel, nnz_w=nnz_w, nnz_o=nnz_o, bits=bits, k=k, record_bytes=total, rec_flags=rflags,
                 c_w=cents[0].copy(), c_ea=cents[1].copy(), c_eas=cents[2].copy(),
                 m_w=m_w, m_o=m_o, codes_w=codes_w, codes_ea=codes_ea, codes_eas=codes_eas)
 
@@ -412,24 +462,45 @@ def compress_tensor(w_t, w_prev, ea, eas, p: Params, tensor_index: int = 0):
         raise ValueError("size mismatch")
     if p.bits not in (2, 4, 8):
         raise ValueError("bits")
+    if p.flags & ~FLAGS_ALL:
+        raise ValueError("flags")
     validate_inputs(w_t, w_prev, ea, eas)
     k = (1 << p.bits) - 1
+    fl = p.flags
 
-    dw = residual(w_t, w_prev)                                        # Algorithm 1, step 1
+    # Algorithm 1, step 1 (ablation "residual" off: the weights themselves go on)
+    dw = w_t.copy() if fl & FLAG_NO_RESIDUAL else residual(w_t, w_prev)
     src = w_t if p.median_source == MEDIAN_ABS_WEIGHT else dw
     med = lower_median_abs(src)
     mean = exact_mean_abs(ea)
-    m_w, thr_w = weight_mask(dw, eas, p.alpha, med)                   # Eq. (rw)
-    m_o, thr_o = moment_mask(ea, m_w, p.beta, mean)                   # Eq. (ro)
+    if fl & FLAG_NO_M2W:
+        m_w, thr_w = weight_mask_set_threshold(dw, p.alpha)
+    else:
+        m_w, thr_w = weight_mask(dw, eas, p.alpha, med)               # Eq. (rw)
+    if fl & FLAG_NO_W2M:
+        m_o, thr_o = moment_mask_alone(ea, p.beta, mean)
+    else:
+        m_o, thr_o = moment_mask(ea, m_w, p.beta, mean)               # Eq. (ro)
+    if fl & FLAG_NO_PRUNE:                                            # ablation "prune" off
+        m_w = np.ones(n, dtype=bool)
+        m_o = np.ones(n, dtype=bool)
     s_w, s_ea, s_eas = dw[m_w], ea[m_o], eas[m_o]                     # joint_prune
 
+    rec_flags = ((REC_MOMENTS_FREE if fl & FLAG_NO_W2M else 0) | (REC_ABSOLUTE if fl & FLAG_NO_RESIDUAL else 0)
+                 | (REC_RAW if fl & FLAG_NO_QUANT else 0))
     cents, codes = [], []
-    for stream, s in enumerate((s_w, s_ea, s_eas)):                   # quantize(.)
-        c0 = kmeans_start(s, k, p.seed, tensor_index, stream)
-        c, idx = lloyd(s, c0, p.kmeans_iters)
-        cents.append(c)
-        codes.append((idx + 1).astype(np.uint8))
-    blob = encode_record(n, p.bits, m_w, m_o, cents[0], cents[1], cents[2], *codes)
+    if fl & FLAG_NO_QUANT:                                            # ablation "quant" off
+        zero = np.zeros(0, dtype=np.float32)
+        cents = [zero, zero, zero]
+        codes = [s_w, s_ea, s_eas]
+        blob = encode_record(n, 32, m_w, m_o, zero, zero, zero, s_w, s_ea, s_eas, rec_flags)
+    else:
+        for stream, s in enumerate((s_w, s_ea, s_eas)):               # quantize(.)
+            c0 = kmeans_start(s, k, p.seed, tensor_index, stream)
+            c, idx = lloyd(s, c0, p.kmeans_iters)
+            cents.append(c)
+            codes.append((idx + 1).astype(np.uint8))
+        blob = encode_record(n, p.bits, m_w, m_o, cents[0], cents[1], cents[2], *codes, rec_flags=rec_flags)
     info = dict(numel=n, dw=dw, median=med, mean_abs_ea=mean, thr_w=thr_w, thr_o=thr_o,
                 m_w=m_w, m_o=m_o, nnz_w=int(m_w.sum()), nnz_o=int(m_o.sum()),
                 s_w=s_w, s_ea=s_ea, s_eas=s_eas, c_w=cents[0], c_ea=cents[1], c_eas=cents[2],
@@ -444,13 +515,19 @@ def decompress_tensor(blob: bytes, w_prev):
     w_prev = np.ascontiguousarray(w_prev, dtype=np.float32).ravel()
     if w_prev.size != r["numel"]:
         raise ValueError("size mismatch")
-    w_hat = w_prev.copy()
+    raw_values = bool(r["rec_flags"] & REC_RAW)
+    val = (lambda c, codes: codes) if raw_values else (lambda c, codes: c[codes.astype(np.int64) - 1])
     kept = r["m_w"]
-    w_hat[kept] = w_prev[kept] + r["c_w"][r["codes_w"].astype(np.int64) - 1]
+    if r["rec_flags"] & REC_ABSOLUTE:            # the stream is W itself: pruned weights are 0
+        w_hat = np.zeros(r["numel"], dtype=np.float32)
+        w_hat[kept] = val(r["c_w"], r["codes_w"])
+    else:
+        w_hat = w_prev.copy()
+        w_hat[kept] = w_prev[kept] + val(r["c_w"], r["codes_w"])
     ea_hat = np.zeros(r["numel"], dtype=np.float32)
     eas_hat = np.zeros(r["numel"], dtype=np.float32)
-    ea_hat[r["m_o"]] = r["c_ea"][r["codes_ea"].astype(np.int64) - 1]
-    eas_hat[r["m_o"]] = r["c_eas"][r["codes_eas"].astype(np.int64) - 1]
+    ea_hat[r["m_o"]] = val(r["c_ea"], r["codes_ea"])
+    eas_hat[r["m_o"]] = val(r["c_eas"], r["codes_eas"])
     return w_hat, ea_hat, eas_hat
 
 
@@ -518,8 +595,11 @@ def encode_dense(numel, bits, nnz_w, nnz_o, c_w, c_ea, c_eas, idx_w, idx_ea, idx
 
 
 def record_to_dense(blob: bytes) -> bytes:
-    """Bitmap + compacted codes -> one code per element (0 = pruned)."""
+    """Bitmap + compacted codes -> one code per element (0 = pruned).  Only records of the
+    method proper (no record flags) have this layout."""
     r = parse_record(blob)
+    if r["rec_flags"]:
+        raise ValueError("ablation variants have no dense layout")
     return encode_dense(r["numel"], r["bits"], r["nnz_w"], r["nnz_o"], r["c_w"], r["c_ea"], r["c_eas"],
                         dense_indices(r["m_w"], r["codes_w"]),
                         dense_indices(r["m_o"], r["codes_ea"]),

@@ -556,3 +556,95 @@ def test_archiver_round_trip_and_sizes():
     assert 0 < a["archived_bytes"] <= len(blob) + 128 and 0 < b["archived_bytes"] < len(dense)
     z = orc.archive_sizes([b"\0" * 100000])
     assert z["archived_bytes"] < 400                          # LZMA2 collapses a run of zeros
+
+
+# ------------------------------------------------ ablation switches (ViT table caption, Section 4.3)
+def hand_params(flags):
+    return orc.Params(alpha=G["alpha"][0], beta=G["beta"][0], bits=4, flags=flags)
+
+
+def test_hand_ablation_masks():
+    q = (f32("w_t"), f32("w_prev"), f32("ea"), f32("eas"))
+    _, a = orc.compress_tensor(*q, hand_params(orc.FLAG_NO_W2M))
+    np.testing.assert_array_equal(a["m_w"].astype(int), np.array(G["m_w_abs_weight"], dtype=int))
+    np.testing.assert_array_equal(a["m_o"].astype(int), np.array(G["m_o_no_w2m"], dtype=int))
+    _, b = orc.compress_tensor(*q, hand_params(orc.FLAG_NO_M2W))
+    assert b["thr_w"] == np.float32(0.25)
+    np.testing.assert_array_equal(b["m_w"].astype(int), np.array(G["m_w_no_m2w"], dtype=int))
+    np.testing.assert_array_equal(b["m_o"].astype(int), np.array(G["m_o_no_m2w"], dtype=int))
+    blob, c = orc.compress_tensor(*q, hand_params(orc.FLAG_NO_RESIDUAL))
+    np.testing.assert_array_equal(c["m_w"].astype(int), np.array(G["m_w_no_residual"], dtype=int))
+    w_hat, _, _ = orc.decompress_tensor(blob, f32("w_prev"))
+    np.testing.assert_array_equal(w_hat, f32("w_hat_no_residual"))
+    _, d = orc.compress_tensor(*q, hand_params(orc.FLAG_NO_PRUNE))
+    assert d["m_w"].all() and d["m_o"].all() and d["nnz_w"] == d["nnz_o"] == 8
+
+
+@pytest.mark.parametrize("flags", [1, 2, 4, 8, 16, 1 | 16, 4 | 8, 2 | 1, 4 | 16, 31])
+def test_ablation_variants_by_independent_parse_and_definitions(flags):
+    n = 3000
+    wt, wp, ea, eas = rand_quad(n, 300 + flags)
+    p = orc.Params(alpha=5e-5 if not flags & orc.FLAG_NO_M2W else 1e-4, median_source=orc.MEDIAN_ABS_RESIDUAL,
+                   kmeans_iters=3, flags=flags)
+    blob, info = orc.compress_tensor(wt, wp, ea, eas, p)
+    dw = wt if flags & 4 else (wt - wp).astype(np.float32)
+    np.testing.assert_array_equal(info["dw"], dw)
+    # the masks, straight from their definitions
+    if flags & 8:
+        m_w = np.ones(n, bool); m_o = np.ones(n, bool)
+    else:
+        if flags & 2:
+            m_w = np.abs(dw) > np.float32(1e-4)
+        else:
+            med = np.sort(np.abs(dw))[(n - 1) // 2]
+            m_w = np.abs(dw) * np.sqrt(eas) > np.float32(np.float32(5e-5) * med)
+        m_o = np.abs(ea) > np.float32(np.float32(2.0) * orc.exact_mean_abs(ea))
+        if not flags & 1:
+            m_o &= m_w
+    np.testing.assert_array_equal(info["m_w"], m_w)
+    np.testing.assert_array_equal(info["m_o"], m_o)
+    # the header's words, read with struct alone
+    head = struct.unpack_from("<IIQQQIIIIQQ", blob, 0)
+    want_flags = (1 if flags & 1 else 0) | (2 if flags & 4 else 0) | (4 if flags & 16 else 0)
+    bits, k = (32, 0) if flags & 16 else (4, 15)
+    hb = 64 if flags & 16 else 256
+    assert head[5:9] == (bits, k, hb, want_flags)
+    nw, no = int(m_w.sum()), int(m_o.sum())
+    a16 = lambda x: (x + 15) // 16 * 16
+    bb = a16(4 * ((n + 31) // 32))
+    assert len(blob) == head[9] == hb + 2 * bb + a16((nw * bits + 7) // 8) + 2 * a16((no * bits + 7) // 8)
+    w_hat, ea_hat, eas_hat = orc.decompress_tensor(blob, wp)
+    if flags & 16:                                       # raw survivors: fp32 straight out of the sections
+        off = hb + 2 * bb
+        np.testing.assert_array_equal(np.frombuffer(blob, "<f4", nw, off), dw[m_w])
+        off += a16(4 * nw)
+        np.testing.assert_array_equal(np.frombuffer(blob, "<f4", no, off), ea[m_o])
+        np.testing.assert_array_equal(np.frombuffer(blob, "<f4", no, off + a16(4 * no)), eas[m_o])
+        base = np.zeros(n, np.float32) if flags & 4 else wp
+        want_w = base.copy(); want_w[m_w] = (base[m_w] + dw[m_w]).astype(np.float32)
+        np.testing.assert_array_equal(w_hat, want_w)
+        np.testing.assert_array_equal(ea_hat, np.where(m_o, ea, 0).astype(np.float32))
+        np.testing.assert_array_equal(eas_hat, np.where(m_o, eas, 0).astype(np.float32))
+    else:
+        base = np.zeros(n, np.float32) if flags & 4 else wp
+        np.testing.assert_array_equal(w_hat[~m_w], base[~m_w])
+        assert np.all(ea_hat[~m_o] == 0) and np.all(eas_hat[~m_o] == 0)
+        r = orc.parse_record(blob)
+        np.testing.assert_array_equal(w_hat[m_w], (base[m_w] + r["c_w"][r["codes_w"].astype(int) - 1]).astype(np.float32))
+    if want_flags:
+        with pytest.raises(ValueError):
+            orc.record_to_dense(blob)
+
+
+def test_flagged_records_keep_their_rules():
+    wt, wp, ea, eas = rand_quad(2000, 41)
+    blob, info = orc.compress_tensor(wt, wp, ea, eas, orc.Params(median_source=1, flags=orc.FLAG_NO_W2M))
+    assert np.any(info["m_o"] & ~info["m_w"])            # moments kept where weights are pruned ...
+    b = bytearray(blob); struct.pack_into("<I", b, 44, 0)
+    with pytest.raises(orc.CorruptBlob):                 # ... which a record of the full method may not hold
+        orc.parse_record(bytes(b))
+    b = bytearray(blob); struct.pack_into("<I", b, 44, 8)
+    with pytest.raises(orc.CorruptBlob):
+        orc.parse_record(bytes(b))
+    with pytest.raises(ValueError):
+        orc.compress_tensor(wt, wp, ea, eas, orc.Params(flags=32))
