@@ -50,6 +50,9 @@ def parse_args():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-decompress", action="store_true")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-layout and archiver leg")
+    ap.add_argument("--no-ablation", action="store_true", help="skip the ablation-table leg")
+    ap.add_argument("--ablation-params", type=int, default=340_000_000,
+                    help="parameters (leading tensors of the workload) the ablation rows are run on")
     ap.add_argument("--archive-params", type=int, default=17_000_000,
                     help="largest tensor whose record and dense container go through the host archiver")
     ap.add_argument("--e2e-steps", type=int, default=2)
@@ -397,6 +400,36 @@ def run_ours(args):
                                 dense_xz_ratio_vs_12B=12 * numels[pick] / arch["dense_xz_bytes"])}
             del dense
         del out_w, out_a, out_s
+
+    # ---- the rows of the ablation table of Section 4.3 (sizes and times; accuracies need training) ----
+    if not args.no_ablation:
+        h.profile_enable(False)
+        sub, acc = [], 0
+        for i, (_, n) in enumerate(shapes):
+            if acc + n > args.ablation_params and sub:
+                break
+            sub.append(i); acc += n
+        cap = sum(binding.record_bytes(shapes[i][1], shapes[i][1], shapes[i][1], 32) for i in sub)
+        ablob = torch.empty(cap, dtype=torch.uint8, device=dev)
+        rows = []
+        for residual, prune, quant in ((0, 0, 0), (1, 0, 0), (0, 1, 0), (0, 0, 1), (1, 1, 0), (1, 0, 1), (1, 1, 1)):
+            fl = ((0 if residual else binding.FLAG_NO_RESIDUAL) | (0 if prune else binding.FLAG_NO_PRUNE)
+                  | (0 if quant else binding.FLAG_NO_QUANT))
+            # without the residual the stream is W_t itself: the same alpha on |W_t| * sqrt(eas) keeps ~all
+            # of it, so the size shows what the paper's table shows (pruning weights directly costs accuracy
+            # there; here it only shows the bytes)
+            pa = binding.Params(alpha=5e-5, beta=2.0, bits=4, kmeans_iters=args.kmeans_iters, seed=0,
+                                median_source=p.median_source, flags=fl)
+            tq = [quads[i] for i in sub]
+            o, _ = h.compress_checkpoint(pa, tq, ablob, want_stats=False)
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record()
+            o, _ = h.compress_checkpoint(pa, tq, ablob, want_stats=False)
+            a1.record(); torch.cuda.synchronize()
+            rows.append({"residual": bool(residual), "prune": bool(prune), "quant": bool(quant),
+                         "bytes": o[-1], "ratio_vs_12B_per_param": 12 * acc / o[-1], "ms": a0.elapsed_time(a1)})
+        out["ablation"] = {"sample": f"tensors 0..{sub[-1]} of the workload ({acc} params)", "rows": rows}
+        del ablob
 
     # ---- end to end through the host-buffer entry point ----------------------
     if not args.no_e2e:

@@ -31,7 +31,8 @@
  * Record layout of one tensor (little endian, every section on a 16-byte boundary, padding zero):
  *     0 u32 magic "EXCP"   4 u32 version = 1     8 u64 numel
  *    16 u64 nnz_w         24 u64 nnz_o          32 u32 bits      36 u32 K = 2^bits - 1
- *    40 u32 header bytes  44 u32 0              48 u64 record bytes   56 u64 0
+ *    40 u32 header bytes  44 u32 record flags   48 u64 record bytes   56 u64 0
+ *       (record flags: 0 for the full method; see excp_flags for the ablation variants)
  *    64 f32 centres of dW [K], of ea [K], of eas [K]; header padded to 16 bytes
  *    .. bitmap of M_w, bitmap of M_o: u32 words, bit k of word w = element 32 w + k
  *    .. codes of dW [nnz_w], of ea [nnz_o], of eas [nnz_o]: survivors in index order, `bits`
@@ -76,6 +77,21 @@ typedef enum {
     EXCP_MEDIAN_ABS_RESIDUAL = 1    /* median(|dW_t|): the quantity the mask prunes */
 } excp_median_source;
 
+/* Ablation switches: the rows of the paper's two ablation tables as variants of the same path.
+ * The ViT table's caption defines the first two ("no check" under M2W: the weights are pruned by a
+ * set threshold instead of alpha / sqrt(m_t); under W2M: M_o(i) = [ v_t(i) > r_o ]); the table of
+ * Section 4.3 toggles residual, prune and quant.  A record written with a switch says so in its
+ * header (offset 44), and excp_decompress_* honour it. */
+typedef enum {
+    EXCP_FLAG_NO_W2M = 1,           /* M_o(i) = [ |ea(i)| > beta * mean ], without "and M_w(i)"; record flag 1 */
+    EXCP_FLAG_NO_M2W = 2,           /* M_w(i) = [ |dW(i)| > alpha ]: alpha itself is the set threshold */
+    EXCP_FLAG_NO_RESIDUAL = 4,      /* W_t is compressed instead of dW; w_prev is not read (may be NULL);
+                                       decompress writes W^ = decoded value, 0 where pruned; record flag 2 */
+    EXCP_FLAG_NO_PRUNE = 8,         /* both masks keep every element */
+    EXCP_FLAG_NO_QUANT = 16         /* no K-means: the sections hold the survivors as fp32 (bits = 32, K = 0,
+                                       64-byte header without centres); record flag 4 */
+} excp_flags;
+
 /* Hyper-parameters.  Section 4.1: alpha = 5e-5, beta = 2.0, bits = 4. */
 typedef struct {
     float alpha;                    /* Eq. (rw) */
@@ -84,7 +100,7 @@ typedef struct {
     int kmeans_iters;               /* Lloyd iterations before the final assignment (>= 0) */
     unsigned long long seed;        /* seed of the K-means start sample */
     int median_source;              /* excp_median_source */
-    unsigned flags;                 /* must be 0 */
+    unsigned flags;                 /* excp_flags, OR-ed; 0 = the full method */
 } excp_params;
 
 /* Per-tensor result, written to host memory. */
@@ -109,7 +125,8 @@ excp_status excp_create(excp_handle* out, int device, size_t workspace_numel);
 /* Frees everything the handle owns.  NULL is accepted. */
 excp_status excp_destroy(excp_handle h);
 
-/* Size in bytes of a record with the given counts (the layout above).  0 if bits is not 2, 4 or 8. */
+/* Size in bytes of a record with the given counts (the layout above).  0 if bits is not 2, 4, 8
+ * or 32 (32 = EXCP_FLAG_NO_QUANT's raw fp32 sections). */
 size_t excp_record_bytes(size_t numel, size_t nnz_w, size_t nnz_o, int bits);
 
 /* Worst-case record size for a tensor of `numel` elements (every element kept). */
@@ -197,7 +214,8 @@ excp_status excp_decompress_checkpoint(excp_handle h, const void* blob, const si
  * excp_dense_bytes gives its size (0 if bits is not 2, 4 or 8).
  *
  * excp_record_to_dense / excp_checkpoint_to_dense rewrite records (device) as dense containers
- * (device): bitmap rank -> code, per element.
+ * (device): bitmap rank -> code, per element.  Records of an ablation variant (non-zero record
+ * flags) have no dense layout: EXCP_ERR_UNSUPPORTED.
  *   blob, tensor_offsets  as returned by excp_compress_checkpoint.
  *   dense_out             device, dense_capacity bytes; containers back to back.
  *   dense_offsets_out     host [num_tensors + 1] (excp_record_to_dense: dense_bytes_out, host).

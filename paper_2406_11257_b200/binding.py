@@ -42,6 +42,9 @@ class CStats(C.Structure):
                 ("thr_w", C.c_float), ("thr_o", C.c_float)]
 
 
+FLAG_NO_W2M, FLAG_NO_M2W, FLAG_NO_RESIDUAL, FLAG_NO_PRUNE, FLAG_NO_QUANT = 1, 2, 4, 8, 16
+
+
 @dataclass
 class Params:
     alpha: float = 5e-5
@@ -50,9 +53,11 @@ class Params:
     kmeans_iters: int = 10
     seed: int = 0
     median_source: int = MEDIAN_ABS_WEIGHT
+    flags: int = 0          # FLAG_NO_*: the ablation switches; 0 = the full method
 
     def to_c(self) -> CParams:
-        return CParams(self.alpha, self.beta, self.bits, self.kmeans_iters, self.seed, self.median_source, 0)
+        return CParams(self.alpha, self.beta, self.bits, self.kmeans_iters, self.seed, self.median_source,
+                       self.flags)
 
 
 _lib = None

@@ -28,17 +28,22 @@ __global__ void __launch_bounds__(64) dec_validate_kernel(const DecDesc* __restr
             const u64 nnz_w = h[4] | ((u64)h[5] << 32);
             const u64 nnz_o = h[6] | ((u64)h[7] << 32);
             const u64 total = h[12] | ((u64)h[13] << 32);
-            if (h[0] == MAGIC && h[1] == VERSION && numel == d.numel && h[8] == BITS && h[9] == KMAX &&
-                h[10] == header_bytes(KMAX) && nnz_o <= nnz_w && nnz_w <= numel &&
-                total == record_bytes(numel, nnz_w, nnz_o, BITS) && total <= d.rec_avail) {
+            const u32 rf = h[11];                         // REC_*: what the record says about itself
+            const int bits = (rf & REC_RAW) ? 32 : BITS;
+            const int kc = centres_of(bits);
+            if (h[0] == MAGIC && h[1] == VERSION && numel == d.numel && !(rf & ~REC_ALL) && h[8] == (u32)bits &&
+                h[9] == (u32)kc && h[10] == header_bytes(kc) && (nnz_o <= nnz_w || (rf & REC_MOMENTS_FREE)) &&
+                nnz_w <= numel && nnz_o <= numel &&
+                total == record_bytes(numel, nnz_w, nnz_o, bits) && total <= d.rec_avail) {
                 ok = 1;
-                s.bits = BITS;
+                s.bits = bits;
+                s.rflags = rf;
                 s.nnz_w = (u32)nnz_w; s.nnz_o = (u32)nnz_o;
-                s.off_bm_w = header_bytes(KMAX);
+                s.off_bm_w = header_bytes(kc);
                 s.off_bm_o = s.off_bm_w + bitmap_bytes(numel);
                 s.off_codes[0] = s.off_bm_o + bitmap_bytes(numel);
-                s.off_codes[1] = s.off_codes[0] + code_bytes(nnz_w, BITS);
-                s.off_codes[2] = s.off_codes[1] + code_bytes(nnz_o, BITS);
+                s.off_codes[1] = s.off_codes[0] + code_bytes(nnz_w, bits);
+                s.off_codes[2] = s.off_codes[1] + code_bytes(nnz_o, bits);
             }
         }
         s.valid = ok;
@@ -47,7 +52,8 @@ __global__ void __launch_bounds__(64) dec_validate_kernel(const DecDesc* __restr
     __syncthreads();
     if (ok && tid < 3 * KPAD) {
         const int k = tid / KPAD, j = tid % KPAD;
-        s.cent[k][j] = j < KMAX ? reinterpret_cast<const float*>(d.rec + HEADER_FIXED)[k * KMAX + j] : 0.f;
+        const bool has = j < KMAX && s.bits != 32;        // a raw record carries no centres
+        s.cent[k][j] = has ? reinterpret_cast<const float*>(d.rec + HEADER_FIXED)[k * KMAX + j] : 0.f;
     }
 }
 
@@ -128,7 +134,7 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
             const u32 a = bm_word(d.rec, s.off_bm_w, nwords, w0 + tid);
             const u32 b = bm_word(d.rec, s.off_bm_o, nwords, w0 + tid);
             bw[tid] = a; bo[tid] = b;
-            bad |= b & ~a;                                // a moment kept where the weight is pruned
+            if (!(s.rflags & REC_MOMENTS_FREE)) bad |= b & ~a;   // a moment kept where the weight is pruned
             u32 ia = __popc(a), ib = __popc(b);
             const u32 ca = ia, cb = ib;
 #pragma unroll
@@ -142,10 +148,12 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
         }
         // stage the code words of this tile's survivors (ranks [off, off + cnt)): whole aligned
         // 32-bit words of the sections (a section is padded to 16 bytes, so the last word exists)
+        const bool raw = s.rflags & REC_RAW;              // sections hold fp32 survivors, read straight from the record
+        const bool absolute = s.rflags & REC_ABSOLUTE;    // the weight stream is W itself
         const u32 fw = offw / 8, fo = offo / 8;           // first staged word of the weight / moment sections
         const u32 nww = cntw ? (offw + cntw + 7) / 8 - fw : 0;
         const u32 nwo = cnto ? (offo + cnto + 7) / 8 - fo : 0;
-        {
+        if (!raw) {
             const u32* s0 = reinterpret_cast<const u32*>(d.rec + s.off_codes[0]) + fw;
             const u32* s1 = reinterpret_cast<const u32*>(d.rec + s.off_codes[1]) + fo;
             const u32* s2 = reinterpret_cast<const u32*>(d.rec + s.off_codes[2]) + fo;
@@ -169,9 +177,23 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
             const bool live = i0 < n;
             if (!DENSE && !live) continue;
             float wp[4] = {0.f, 0.f, 0.f, 0.f};
-            if (!DENSE) load4(d.w_prev, i0, n, wp);
+            if (!DENSE && !absolute) load4(d.w_prev, i0, n, wp);
             const u32 word = e0 >> 5, bit = e0 & 31;
             const u32 mw4 = (bw[word] >> bit) & 15u, mo4 = (bo[word] >> bit) & 15u;
+            if (!DENSE && raw) {
+                u32 gw = offw + pw[word] + __popc(bw[word] & ((1u << bit) - 1u));
+                u32 go = offo + po[word] + __popc(bo[word] & ((1u << bit) - 1u));
+                const float* vw = reinterpret_cast<const float*>(d.rec + s.off_codes[0]);
+                const float* va = reinterpret_cast<const float*>(d.rec + s.off_codes[1]);
+                const float* ve = reinterpret_cast<const float*>(d.rec + s.off_codes[2]);
+                for (int k = 0; k < 4 && i0 + k < n; ++k) {
+                    float w = wp[k], a = 0.f, e = 0.f;
+                    if ((mw4 >> k) & 1u) w = __fadd_rn(wp[k], vw[gw++]);
+                    if ((mo4 >> k) & 1u) { a = va[go]; e = ve[go]; ++go; }
+                    d.w_out[i0 + k] = w; d.ea_out[i0 + k] = a; d.eas_out[i0 + k] = e;
+                }
+                continue;
+            }
             // this thread's survivors have consecutive ranks, so their codes are consecutive
             // nibbles: one 32-bit window per stream holds all four
             const u32 qw = qw0 + pw[word] + __popc(bw[word] & ((1u << bit) - 1u));
@@ -250,6 +272,11 @@ __global__ void __launch_bounds__(64) dense_header_kernel(const DecDesc* __restr
     const DecDesc& d = descs[t];
     DecState& s = st[t];
     if (!s.valid) return;
+    if (s.rflags) {                                       // ablation variants have no dense layout
+        __syncthreads();
+        if (tid == 0) { s.valid = 0; atomicOr(&call->flags, FLAG_UNSUPPORTED); }
+        return;
+    }
     const u64 total = dense_bytes(d.numel, BITS);
     if (total > d.dense_avail) {                          // uniform over the block
         if (tid == 0) { s.valid = 0; atomicOr(&call->flags, FLAG_BLOB_FULL); }

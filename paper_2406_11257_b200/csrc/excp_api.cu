@@ -148,7 +148,7 @@ bool make_groups(excp_handle h, const size_t* numel, size_t n, std::vector<Group
 excp_status validate_params(const excp_params* params) {
     if (!params) return EXCP_ERR_INVALID_ARG;
     if (params->bits == 2 || params->bits == 8) return EXCP_ERR_UNSUPPORTED;
-    if (params->bits != 4 || params->kmeans_iters < 0 || params->flags != 0 ||
+    if (params->bits != 4 || params->kmeans_iters < 0 || (params->flags & ~OPT_ALL) ||
         (params->median_source != 0 && params->median_source != 1) ||
         !(params->alpha >= 0.f) || !(params->beta >= 0.f) || std::isinf(params->alpha) ||
         std::isinf(params->beta))
@@ -160,6 +160,7 @@ Params to_params(const excp_params* params) {
     Params p;
     p.alpha = params->alpha; p.beta = params->beta; p.bits = params->bits;
     p.kmeans_iters = params->kmeans_iters; p.seed = params->seed; p.median_source = params->median_source;
+    p.flags = params->flags;
     return p;
 }
 
@@ -170,7 +171,7 @@ bool run_group(excp_handle h, const LaunchCfg& cfg, const TensorDesc* descs, int
     if (!check(h, cudaMemsetAsync(h->ws.bst, 0, nt * sizeof(BucketState), cfg.stream))) return false;
     launch_stats(cfg, descs, h->d_state, nt, tiles, h->ws, p, h->d_call);
     launch_mask_compact(cfg, descs, h->d_state, nt, tiles, h->ws, p, h->d_call, blob_capacity);
-    launch_kmeans(cfg, descs, h->d_state, nt, tiles, scan_items, h->ws, p, h->d_call);
+    if (!(p.flags & OPT_NO_QUANT)) launch_kmeans(cfg, descs, h->d_state, nt, tiles, scan_items, h->ws, p, h->d_call);
     launch_pack(cfg, descs, h->d_state, nt, tiles, h->ws, p, blob, h->d_call, results);
     return check(h, cudaGetLastError());
 }
@@ -212,6 +213,7 @@ excp_status status_from_flags(u32 flags) {
     if (flags & FLAG_INTERNAL) return EXCP_ERR_CUDA;
     if (flags & FLAG_NONFINITE) return EXCP_ERR_NONFINITE_INPUT;
     if (flags & FLAG_CORRUPT) return EXCP_ERR_CORRUPT_BLOB;
+    if (flags & FLAG_UNSUPPORTED) return EXCP_ERR_UNSUPPORTED;
     if (flags & FLAG_BLOB_FULL) return EXCP_ERR_BUFFER_TOO_SMALL;
     return EXCP_OK;
 }
@@ -293,7 +295,7 @@ excp_status excp_destroy(excp_handle h) {
 }
 
 size_t excp_record_bytes(size_t numel, size_t nnz_w, size_t nnz_o, int bits) {
-    if (bits != 2 && bits != 4 && bits != 8) return 0;
+    if (bits != 2 && bits != 4 && bits != 8 && bits != 32) return 0;
     return (size_t)record_bytes(numel, nnz_w, nnz_o, bits);
 }
 
@@ -332,7 +334,8 @@ excp_status excp_compress_checkpoint(excp_handle h, const excp_params* params, s
     if (ps != EXCP_OK) return ps;
     for (size_t i = 0; i < num_tensors; ++i) {
         if (numel[i] == 0) continue;
-        if (!w_t[i] || !w_prev[i] || !ea[i] || !eas[i]) return EXCP_ERR_INVALID_ARG;
+        const bool need_prev = !(params->flags & OPT_NO_RESIDUAL);     // without the residual W^_(t-1) is not read
+        if (!w_t[i] || (need_prev && !w_prev[i]) || !ea[i] || !eas[i]) return EXCP_ERR_INVALID_ARG;
         if (!aligned16(w_t[i]) || !aligned16(w_prev[i]) || !aligned16(ea[i]) || !aligned16(eas[i]))
             return EXCP_ERR_INVALID_ARG;
     }

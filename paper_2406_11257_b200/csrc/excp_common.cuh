@@ -32,6 +32,20 @@ constexpr u32 FLAG_BLOB_FULL = 2u;               // records do not fit blob_capa
 constexpr u32 FLAG_CORRUPT = 4u;                 // decompress: inconsistent record
 constexpr u32 FLAG_INTERNAL = 8u;                // a self-check failed (candidate count mismatch)
 constexpr u32 FLAG_TIMEOUT = 16u;                // a bounded wait on an asynchronous copy ran out
+constexpr u32 FLAG_UNSUPPORTED = 32u;            // a record variant the called routine does not handle
+
+// Ablation switches of a compress call (ViT table caption; ablation table of Section 4.3)
+constexpr u32 OPT_NO_W2M = 1u;                   // M_o without the conjunction with M_w
+constexpr u32 OPT_NO_M2W = 2u;                   // M_w = [ |dW| > alpha ], alpha the set threshold
+constexpr u32 OPT_NO_RESIDUAL = 4u;              // the weights themselves, not their residual
+constexpr u32 OPT_NO_PRUNE = 8u;                 // every element kept
+constexpr u32 OPT_NO_QUANT = 16u;                // survivors stored as fp32
+constexpr u32 OPT_ALL = 31u;
+// What a record says about itself (header offset 44)
+constexpr u32 REC_MOMENTS_FREE = 1u;             // M_o need not lie inside M_w
+constexpr u32 REC_ABSOLUTE = 2u;                 // the weight stream is W: Algorithm 2 adds nothing
+constexpr u32 REC_RAW = 4u;                      // bits = 32, K = 0: sections hold fp32 survivors
+constexpr u32 REC_ALL = 7u;
 
 constexpr u32 MAGIC = 0x50435845u;
 constexpr u32 DENSE_MAGIC = 0x44435845u;         // "EXCD": one code per element, 0 = pruned
@@ -143,7 +157,13 @@ struct Params {
     int bits, kmeans_iters;
     u64 seed;
     int median_source;
+    u32 flags;                   // OPT_*
 };
+__host__ __device__ inline int stored_bits(const Params& p) { return (p.flags & OPT_NO_QUANT) ? 32 : p.bits; }
+__host__ __device__ inline u32 record_flags(const Params& p) {
+    return ((p.flags & OPT_NO_W2M) ? REC_MOMENTS_FREE : 0u) | ((p.flags & OPT_NO_RESIDUAL) ? REC_ABSOLUTE : 0u) |
+           ((p.flags & OPT_NO_QUANT) ? REC_RAW : 0u);
+}
 
 struct DecDesc {                 // decompress: one per tensor of a group
     const unsigned char* rec;    // start of the record
@@ -164,6 +184,7 @@ struct DecState {                // decompress scratch per tensor
     u32 bits;
     u32 nnz_w, nnz_o;
     u32 cnt_w, cnt_o;            // dense layout: non-zero codes met while decoding
+    u32 rflags, pad_;            // the record's flags (REC_*)
     u64 off_bm_w, off_bm_o, off_codes[3];
     float cent[3][KPAD];
 };
@@ -171,6 +192,7 @@ struct DecState {                // decompress scratch per tensor
 // ---- layout arithmetic (host and device) ----------------------------------
 __host__ __device__ inline u64 align16(u64 n) { return (n + 15ull) & ~15ull; }
 __host__ __device__ inline u64 header_bytes(int k) { return align16(HEADER_FIXED + 12ull * k); }
+__host__ __device__ inline int centres_of(int bits) { return bits == 32 ? 0 : (1 << bits) - 1; }
 __host__ __device__ inline u64 bitmap_bytes(u64 numel) { return align16(4ull * ((numel + 31) / 32)); }
 __host__ __device__ inline u64 code_bytes(u64 nnz, int bits) { return align16((nnz * bits + 7) / 8); }
 __host__ __device__ inline u64 dense_section_bytes(u64 numel, int bits) { return align16((numel * bits + 7) / 8); }
@@ -178,7 +200,7 @@ __host__ __device__ inline u64 dense_bytes(u64 numel, int bits) {
     return header_bytes((1 << bits) - 1) + 3 * dense_section_bytes(numel, bits);
 }
 __host__ __device__ inline u64 record_bytes(u64 numel, u64 nnz_w, u64 nnz_o, int bits) {
-    return header_bytes((1 << bits) - 1) + 2 * bitmap_bytes(numel) + code_bytes(nnz_w, bits) +
+    return header_bytes(centres_of(bits)) + 2 * bitmap_bytes(numel) + code_bytes(nnz_w, bits) +
            2 * code_bytes(nnz_o, bits);
 }
 

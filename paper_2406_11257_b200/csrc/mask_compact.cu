@@ -26,9 +26,12 @@ struct MaskSmem {
 // Every warp owns a contiguous run of tiles and walks it alone: 256-value chunks of the four
 // streams arrive in its ring of stages, a tile's survivor offset is a running count in the
 // warp, and nothing in the sweep synchronises the block.
+// VARIANT = false is the method; VARIANT = true adds the ablation switches `opt` (OPT_*), kept
+// out of the method's own instruction stream.
+template <bool VARIANT>
 __global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc* __restrict__ descs,
                                                               TensorState* __restrict__ st, int nt,
-                                                              u32 tiles, Workspace ws, CallState* call) {
+                                                              u32 tiles, Workspace ws, CallState* call, u32 opt) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     MaskSmem& sm = *reinterpret_cast<MaskSmem*>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -66,9 +69,10 @@ __global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc*
             if (ic.chunk == 0 && ic.enter_tile(descs, nt)) {
                 ip[0] = descs[ic.tns].w_t; ip[1] = descs[ic.tns].w_prev;
                 ip[2] = descs[ic.tns].ea; ip[3] = descs[ic.tns].eas;
+                if (VARIANT && (opt & OPT_NO_RESIDUAL)) ip[1] = nullptr;     // W^_(t-1) is not read
             }
             const u64 e0 = ic.elem0();
-            const float* src[4] = {ip[0] + e0, ip[1] + e0, ip[2] + e0, ip[3] + e0};
+            const float* src[4] = {ip[0] + e0, ip[1] ? ip[1] + e0 : nullptr, ip[2] + e0, ip[3] + e0};
             ring.issue(lane, src, ic.valid() & ~3u);
             ic.next();
         }
@@ -103,10 +107,11 @@ __global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc*
                 for (int k = 0; k < 4; ++k) {
                     const u32 i = step * 128 + k * 32 + lane;
                     float a, b, e, v;
+                    const bool no_prev = VARIANT && (opt & OPT_NO_RESIDUAL);
                     if (FULL || i < nbulk) {
-                        a = stg[i]; b = stg[MCH + i]; e = stg[2 * MCH + i]; v = stg[3 * MCH + i];
+                        a = stg[i]; b = no_prev ? 0.f : stg[MCH + i]; e = stg[2 * MCH + i]; v = stg[3 * MCH + i];
                     } else if (i < valid) {          // ragged last values of a tensor
-                        a = __ldg(cp[0] + e0 + i); b = __ldg(cp[1] + e0 + i);
+                        a = __ldg(cp[0] + e0 + i); b = no_prev ? 0.f : __ldg(cp[1] + e0 + i);
                         e = __ldg(cp[2] + e0 + i); v = __ldg(cp[3] + e0 + i);
                     } else {
                         a = b = e = v = 0.f;
@@ -116,10 +121,18 @@ __global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc*
                     nanacc = __fmaf_rn(e, 0.f, nanacc);
                     nanacc = __fmaf_rn(v, 0.f, nanacc);
                     minv = fminf(minv, v);
-                    const float dw = __fsub_rn(a, b);                            // Eq. (ckpt_res)
-                    const float lhs = __fmul_rn(fabsf(dw), __fsqrt_rn(v));
-                    const bool kw = lhs > thr_w;                                 // Eq. (rw); past numel: 0 > thr is false
-                    const bool ko = kw && (fabsf(e) > thr_o);                    // Eq. (ro)
+                    const float dw = no_prev ? a : __fsub_rn(a, b);              // Eq. (ckpt_res)
+                    bool kw, ko;
+                    if (!VARIANT) {
+                        const float lhs = __fmul_rn(fabsf(dw), __fsqrt_rn(v));
+                        kw = lhs > thr_w;                                        // Eq. (rw); past numel: 0 > thr is false
+                        ko = kw && (fabsf(e) > thr_o);                           // Eq. (ro)
+                    } else {
+                        const bool real = FULL || i < valid;
+                        const float lhs = (opt & OPT_NO_M2W) ? fabsf(dw) : __fmul_rn(fabsf(dw), __fsqrt_rn(v));
+                        kw = real && ((opt & OPT_NO_PRUNE) || lhs > thr_w);
+                        ko = real && ((opt & OPT_NO_PRUNE) || (fabsf(e) > thr_o && ((opt & OPT_NO_W2M) || kw)));
+                    }
                     bw[k] = __ballot_sync(0xffffffffu, kw);
                     bo[k] = __ballot_sync(0xffffffffu, ko);
                     dwv[k] = dw; eav[k] = e; easv[k] = v;
@@ -191,7 +204,7 @@ __global__ void __launch_bounds__(MAX_GROUP_TENSORS) layout_kernel(const TensorD
     __shared__ u64 wtot[32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     u64 bytes = 0;
-    if (tid < nt) bytes = record_bytes(descs[tid].numel, st[tid].nnz_w, st[tid].nnz_o, bits);
+    if (tid < nt) bytes = record_bytes(descs[tid].numel, st[tid].nnz_w, st[tid].nnz_o, bits);   // bits = 32: raw survivors
     u64 incl = bytes;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -221,12 +234,15 @@ void launch_mask_compact(const LaunchCfg& cfg, const TensorDesc* descs, TensorSt
                          const Workspace& ws, const Params& p, CallState* call, u64 blob_capacity) {
     if (tiles) {
         const u32 grid = min((tiles + MWARPS - 1) / MWARPS, (u32)cfg.sms * 2u);
-        cudaFuncSetAttribute(mask_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(MaskSmem));
-        mask_compact_kernel<<<grid, MTPB, sizeof(MaskSmem), cfg.stream>>>(descs, st, nt, tiles, ws, call);
+        const u32 opt = p.flags & (OPT_NO_W2M | OPT_NO_M2W | OPT_NO_RESIDUAL | OPT_NO_PRUNE);
+        cudaFuncSetAttribute(mask_compact_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(MaskSmem));
+        cudaFuncSetAttribute(mask_compact_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(MaskSmem));
+        if (opt) mask_compact_kernel<true><<<grid, MTPB, sizeof(MaskSmem), cfg.stream>>>(descs, st, nt, tiles, ws, call, opt);
+        else mask_compact_kernel<false><<<grid, MTPB, sizeof(MaskSmem), cfg.stream>>>(descs, st, nt, tiles, ws, call, 0u);
         prof_mark(cfg, ST_MASK_COMPACT, 1);
     }
     tile_scan_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, ws);
-    layout_kernel<<<1, MAX_GROUP_TENSORS, 0, cfg.stream>>>(descs, st, nt, p.bits, call, blob_capacity);
+    layout_kernel<<<1, MAX_GROUP_TENSORS, 0, cfg.stream>>>(descs, st, nt, stored_bits(p), call, blob_capacity);
     prof_mark(cfg, ST_SCAN_LAYOUT, 2);
 }
 

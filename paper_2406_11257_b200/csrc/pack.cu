@@ -16,20 +16,20 @@ constexpr int PER_WORD = 32 / BITS;   // 8 codes per 32-bit word
 struct Sections {
     u64 bm_w, bm_o, codes[3];
 };
-__device__ inline Sections sections_of(u64 numel, u64 nnz_w, u64 nnz_o) {
+__device__ inline Sections sections_of(u64 numel, u64 nnz_w, u64 nnz_o, int bits = BITS) {
     Sections s;
-    s.bm_w = header_bytes(KMAX);
+    s.bm_w = header_bytes(centres_of(bits));
     s.bm_o = s.bm_w + bitmap_bytes(numel);
     s.codes[0] = s.bm_o + bitmap_bytes(numel);
-    s.codes[1] = s.codes[0] + code_bytes(nnz_w, BITS);
-    s.codes[2] = s.codes[1] + code_bytes(nnz_o, BITS);
+    s.codes[1] = s.codes[0] + code_bytes(nnz_w, bits);
+    s.codes[2] = s.codes[1] + code_bytes(nnz_o, bits);
     return s;
 }
 
 // Header, zeroed section tails, results for the host.  One block per tensor.
 __global__ void __launch_bounds__(64) header_kernel(const TensorDesc* __restrict__ descs,
                                                     TensorState* __restrict__ st, unsigned char* blob,
-                                                    CallState* call, TensorResult* results) {
+                                                    CallState* call, TensorResult* results, int bits, u32 rflags) {
     const int t = blockIdx.x, tid = threadIdx.x;
     const TensorState& s = st[t];
     if (tid == 0) {
@@ -43,7 +43,8 @@ __global__ void __launch_bounds__(64) header_kernel(const TensorDesc* __restrict
     if (call->flags & FLAG_BLOB_FULL) return;
     unsigned char* rec = blob + s.blob_off;
     const u64 numel = descs[t].numel, nnz_w = s.nnz_w, nnz_o = s.nnz_o;
-    const u32 hb = (u32)header_bytes(KMAX);
+    const int kc = centres_of(bits);                  // 15, or 0 when the survivors are stored raw
+    const u32 hb = (u32)header_bytes(kc);
     u32* h32 = reinterpret_cast<u32*>(rec);
     if (tid < (int)(hb / 4)) {
         u32 v = 0;
@@ -56,13 +57,14 @@ __global__ void __launch_bounds__(64) header_kernel(const TensorDesc* __restrict
             case 5: v = (u32)(nnz_w >> 32); break;
             case 6: v = (u32)nnz_o; break;
             case 7: v = (u32)(nnz_o >> 32); break;
-            case 8: v = BITS; break;
-            case 9: v = KMAX; break;
+            case 8: v = (u32)bits; break;
+            case 9: v = (u32)kc; break;
             case 10: v = hb; break;
+            case 11: v = rflags; break;
             case 12: v = (u32)s.blob_bytes; break;
             case 13: v = (u32)(s.blob_bytes >> 32); break;
             default:
-                if (tid >= 16 && tid < 16 + 3 * KMAX) {
+                if (tid >= 16 && tid < 16 + 3 * kc) {
                     const int i = tid - 16;
                     v = __float_as_uint(s.s[i / KMAX].cent[i % KMAX]);
                 }
@@ -70,10 +72,10 @@ __global__ void __launch_bounds__(64) header_kernel(const TensorDesc* __restrict
         h32[tid] = v;
     }
     // the last 16 bytes of every code section hold the padding: clear them
-    const Sections sec = sections_of(numel, nnz_w, nnz_o);
+    const Sections sec = sections_of(numel, nnz_w, nnz_o, bits);
     if (tid < 12) {
         const int k = tid >> 2;
-        const u64 len = code_bytes(k == 0 ? nnz_w : nnz_o, BITS);
+        const u64 len = code_bytes(k == 0 ? nnz_w : nnz_o, bits);
         if (len) reinterpret_cast<u32*>(rec + sec.codes[k] + len - 16)[tid & 3] = 0u;
     }
 }
@@ -216,7 +218,7 @@ __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __res
 __global__ void __launch_bounds__(TPB) copy_bitmaps_kernel(const TensorDesc* __restrict__ descs,
                                                            const TensorState* __restrict__ st, int nt,
                                                            u32 tiles, Workspace ws, unsigned char* blob,
-                                                           const CallState* call) {
+                                                           const CallState* call, u32 hb) {
     if (call->flags & FLAG_BLOB_FULL) return;
     const u64 g = (u64)blockIdx.x * TPB + threadIdx.x;       // uint4 index over all tiles
     const u32 tile = (u32)(g / (TILE_WORDS / 4));
@@ -228,18 +230,51 @@ __global__ void __launch_bounds__(TPB) copy_bitmaps_kernel(const TensorDesc* __r
     const u64 local = (u64)(tile - descs[t].tile_begin) * (TILE_WORDS / 4) + q;
     if (local >= quads) return;
     unsigned char* rec = blob + st[t].blob_off;
-    const u64 hb = header_bytes(KMAX);
     const uint4 a = reinterpret_cast<const uint4*>(ws.bm_w)[g];
     const uint4 b = reinterpret_cast<const uint4*>(ws.bm_o)[g];
     reinterpret_cast<uint4*>(rec + hb)[local] = a;
     reinterpret_cast<uint4*>(rec + hb + quads * 16)[local] = b;
 }
 
+// Quantisation switched off (ablation table of Section 4.3): the survivors themselves go into the
+// sections, fp32, in index order.  One warp per tile: its segment of each stream is copied to the
+// tile's rank offset in the section.
+__global__ void __launch_bounds__(TPB) pack_raw_kernel(const TensorDesc* __restrict__ descs,
+                                                       const TensorState* __restrict__ st, int nt, u32 tiles,
+                                                       Workspace ws, unsigned char* blob, const CallState* call) {
+    if (call->flags & FLAG_BLOB_FULL) return;
+    const int lane = threadIdx.x & 31;
+    const u32 tile = blockIdx.x * (TPB / 32) + (threadIdx.x >> 5);
+    if (tile >= tiles) return;
+    const int t = find_tensor(descs, nt, tile);
+    const TensorState& s = st[t];
+    const Sections sec = sections_of(descs[t].numel, s.nnz_w, s.nnz_o, 32);
+    unsigned char* rec = blob + s.blob_off;
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+        const u32 cnt = (k == 0 ? ws.tile_cnt_w : ws.tile_cnt_o)[tile];
+        const u32 off = (k == 0 ? ws.tile_off_w : ws.tile_off_o)[tile];
+        const float* src = ws.surv[k] + (u64)tile * TILE;
+        float* dst = reinterpret_cast<float*>(rec + sec.codes[k]) + off;
+        for (u32 i = lane; i < cnt; i += 32) dst[i] = src[i];
+    }
+}
+
 void launch_pack(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                  const Workspace& ws, const Params& p, unsigned char* blob, CallState* call,
                  TensorResult* results) {
-    header_kernel<<<nt, 64, 0, cfg.stream>>>(descs, st, blob, call, results);
+    header_kernel<<<nt, 64, 0, cfg.stream>>>(descs, st, blob, call, results, stored_bits(p), record_flags(p));
     if (!tiles) { prof_mark(cfg, ST_HEADER_EDGES, 1); return; }
+    if (p.flags & OPT_NO_QUANT) {
+        prof_mark(cfg, ST_HEADER_EDGES, 1);
+        pack_raw_kernel<<<(tiles + TPB / 32 - 1) / (TPB / 32), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, blob, call);
+        prof_mark(cfg, ST_PACK_CODES, 1);
+        const u64 quads = (u64)tiles * (TILE_WORDS / 4);
+        copy_bitmaps_kernel<<<(u32)((quads + TPB - 1) / TPB), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, blob, call,
+                                                                                   (u32)header_bytes(0));
+        prof_mark(cfg, ST_COPY_BITMAPS, 1);
+        return;
+    }
     clear_edges_kernel<<<(tiles + TPB - 1) / TPB, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, blob, call);
     prof_mark(cfg, ST_HEADER_EDGES, 2);
     const u32 grid = min((tiles + PWARPS - 1) / PWARPS, (u32)cfg.sms * 4u);
@@ -248,7 +283,7 @@ void launch_pack(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st,
     prof_mark(cfg, ST_PACK_CODES, 2);
     const u64 quads = (u64)tiles * (TILE_WORDS / 4);
     copy_bitmaps_kernel<<<(u32)((quads + TPB - 1) / TPB), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws,
-                                                                               blob, call);
+                                                                               blob, call, (u32)header_bytes(KMAX));
     prof_mark(cfg, ST_COPY_BITMAPS, 1);
 }
 

@@ -22,6 +22,12 @@
 
 namespace excp {
 
+// alpha * median, the right-hand side of Eq. (rw).  A negative alpha is how the launcher passes
+// "the threshold is set": then |alpha| itself is the threshold and the median is not used.
+__device__ __forceinline__ float weight_threshold(float alpha, float median) {
+    return alpha < 0.f || (alpha == 0.f && signbit(alpha)) ? -alpha : __fmul_rn(alpha, median);
+}
+
 // ---------------------------------------------------------------------------
 // Find the bin that holds rank k (0-based) in a histogram in shared memory.
 // Threads 0..255 each own BINS/256 consecutive bins.  All threads of the block
@@ -278,7 +284,7 @@ __global__ void __launch_bounds__(1024) hist2_finish_kernel(const TensorDesc* __
     if (tid == 0) {
         const u32 bits = (s.bin1 << HIST1_SHIFT) | (a << 9) | b;
         s.median_bits = bits;
-        s.thr_w = __fmul_rn(alpha, __uint_as_float(bits));      // alpha * median, Eq. (rw)
+        s.thr_w = weight_threshold(alpha, __uint_as_float(bits));
         if (c != s.bin_count) s.flags |= FLAG_INTERNAL;
     }
 }
@@ -560,7 +566,7 @@ __global__ void __launch_bounds__(TPB) stats_finish_kernel(const TensorDesc* __r
     if (n == 0) {
         if (tid == 0) {
             s.mean_abs_ea = 0.f;
-            s.thr_w = __fmul_rn(alpha, 0.f);
+            s.thr_w = weight_threshold(alpha, 0.f);
             s.thr_o = __fmul_rn(beta, 0.f);
         }
         return;
@@ -572,7 +578,7 @@ __global__ void __launch_bounds__(TPB) stats_finish_kernel(const TensorDesc* __r
     s.mean_abs_ea = mean;
     s.thr_o = __fmul_rn(beta, mean);                                  // beta * mean, Eq. (ro)
     if (s.med_done) {
-        s.thr_w = __fmul_rn(alpha, __uint_as_float(s.median_bits));   // alpha * median, Eq. (rw)
+        s.thr_w = weight_threshold(alpha, __uint_as_float(s.median_bits));
         return;
     }
     const u32 k = (u32)((n - 1) / 2), below = s.count_below, c = s.cand_count;
@@ -639,30 +645,31 @@ __global__ void __launch_bounds__(TPB) median_digit_kernel(TensorState* __restri
         if (ls == 0) {
             s.median_bits = base + np;
             s.med_done = 1;
-            s.thr_w = __fmul_rn(alpha, __uint_as_float(base + np));   // alpha * median, Eq. (rw)
+            s.thr_w = weight_threshold(alpha, __uint_as_float(base + np));
         }
     }
 }
 
 void launch_stats(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                   const Workspace& ws, const Params& p, CallState* call) {
-    const int resid = p.median_source == 1;
+    const int resid = p.median_source == 1 && !(p.flags & OPT_NO_RESIDUAL);   // without the residual dW is W_t
+    const float alpha = (p.flags & OPT_NO_M2W) ? -p.alpha : p.alpha;          // see weight_threshold
     median_sample_kernel<<<nt, 1024, 0, cfg.stream>>>(descs, st, ws, resid);
     if (tiles) {
         const u32 grid = min((tiles + SWARPS - 1) / SWARPS, (u32)cfg.sms * 2u);
         cudaFuncSetAttribute(stats_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SweepSmem));
         stats_sweep_kernel<<<grid, TPB, sizeof(SweepSmem), cfg.stream>>>(descs, st, nt, tiles, ws, resid, call);
     }
-    stats_finish_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, p.alpha, p.beta);
+    stats_finish_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, alpha, p.beta);
     if (tiles)
         for (int pass = 0; pass < 4; ++pass)
-            median_digit_kernel<<<dim3(SEL_SLICES, nt), TPB, 0, cfg.stream>>>(st, descs, ws, pass, p.alpha);
+            median_digit_kernel<<<dim3(SEL_SLICES, nt), TPB, 0, cfg.stream>>>(st, descs, ws, pass, alpha);
     prof_mark(cfg, ST_STATS1, tiles ? 7 : 2);
     if (tiles) {          // the histogram path: returns at once unless a bracket missed
         hist1_kernel<<<min(tiles, (u32)cfg.sms * 4u), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, resid);
         hist1_finish_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st);
         hist2_kernel<<<min(tiles, (u32)cfg.sms * 8u), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, resid);
-        hist2_finish_kernel<<<nt, 1024, 0, cfg.stream>>>(descs, st, ws, p.alpha);
+        hist2_finish_kernel<<<nt, 1024, 0, cfg.stream>>>(descs, st, ws, alpha);
         prof_mark(cfg, ST_STATS2, 4);
     }
 }

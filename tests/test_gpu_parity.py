@@ -33,7 +33,7 @@ def to_np(quads):
 
 def oparams(p: binding.Params) -> orc.Params:
     return orc.Params(alpha=p.alpha, beta=p.beta, bits=p.bits, kmeans_iters=p.kmeans_iters, seed=p.seed,
-                      median_source=p.median_source)
+                      median_source=p.median_source, flags=p.flags)
 
 
 def gpu_compress(h, p, dquads, capacity=None):
