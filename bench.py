@@ -48,6 +48,8 @@ def parse_args():
     ap.add_argument("--workspace-numel", type=int, default=1_200_000_000)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--bits", type=int, default=4, choices=[2, 4, 8],
+                    help="code width (4 is the method's and the headline's; 2 and 8 are the quantisation-bins variants)")
     ap.add_argument("--no-decompress", action="store_true")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-layout and archiver leg")
     ap.add_argument("--no-ablation", action="store_true", help="skip the ablation-table leg")
@@ -214,10 +216,10 @@ def run_ours(args):
     ws_numel = min(args.workspace_numel, n_tot + 4096 * len(shapes))
     ws_numel = max(ws_numel, max(n for _, n in shapes))
     h = binding.Handle(workspace_numel=ws_numel)
-    p = binding.Params(kmeans_iters=args.kmeans_iters,
+    p = binding.Params(kmeans_iters=args.kmeans_iters, bits=args.bits,
                        median_source=binding.MEDIAN_ABS_RESIDUAL if args.median == "residual" else binding.MEDIAN_ABS_WEIGHT)
-    bound = sum(binding.compress_bound(n) for _, n in shapes)
-    cap = min(bound, int(0.80 * n_tot) + 1024 * len(shapes) + (1 << 20))
+    bound = sum(binding.compress_bound(n, args.bits) for _, n in shapes)
+    cap = min(bound, int(0.80 * n_tot * max(args.bits, 4) / 4) + 4096 * len(shapes) + (1 << 20))
     blob = torch.empty(cap, dtype=torch.uint8, device=dev)
 
     h.profile_enable(True)
@@ -262,14 +264,14 @@ def run_ours(args):
         "bucket_ids": 4 * surv,                     # survivors read once to count them per bucket
         "bucket_scatter": 8 * surv,                 # survivors read and written into their buckets
         "bucket_sum": 4 * surv,                     # the bucketed copy read once for the bucket sums
-        "bucket_scan": T * 4 * surv * 14 / 256,     # about 14 of 256 buckets per iteration
-        "pack_codes": 4.5 * surv,
+        "bucket_scan": T * 4 * surv * min(1.0, (2 ** args.bits - 2) / 256),   # about K - 1 of 256 buckets per iteration
+        "pack_codes": (4 + args.bits / 8) * surv,
         "copy_bitmaps": n_tot / 2,
     }
     moved_bytes = sum(stage_bytes.values())         # what these kernels must move by design
     # what the method moves when every Lloyd iteration sweeps the survivors (one statistics sweep,
     # one mask sweep, T + 1 sweeps of the survivors, the codes)
-    algo_bytes = ((src_b + 4) + 16 + 0.25) * n_tot + 4 * surv + (T + 1) * 4 * surv + 0.5 * surv
+    algo_bytes = ((src_b + 4) + 16 + 0.25) * n_tot + 4 * surv + (T + 1) * 4 * surv + args.bits / 8 * surv
     peak, peak_kind = measured_peak()
     per_step = {k: v / args.steps for k, v in stage_ms.items()}
     dom = max((k for k in stage_bytes), key=lambda k: per_step.get(k, 0.0))
@@ -286,7 +288,7 @@ def run_ours(args):
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{shape.name} checkpoint pair ({len(shapes)} tensors, {n_tot} params, fp32 W_t, W_prev, ea, eas), "
                                f"median of |{'dW' if args.median == 'residual' else 'W_t'}|, alpha 5e-5, beta 2.0",
-                   "bits": 4, "kmeans_iters": T, "l2": "inputs larger than L2 (no flush needed)" if 16 * n_tot > 4e8 else "inputs fit L2",
+                   "bits": args.bits, "kmeans_iters": T, "l2": "inputs larger than L2 (no flush needed)" if 16 * n_tot > 4e8 else "inputs fit L2",
                    "workspace_numel": ws_numel, "per_rank": "each rank compresses its own checkpoint; no collective"},
         "input_gbs": 16 * value / 1e9,
         "algorithmic_bytes_per_param": algo_bytes / n_tot,
@@ -338,14 +340,14 @@ def run_ours(args):
             decompress_all()
         d1.record(); torch.cuda.synchronize()
         dms = d0.elapsed_time(d1) / args.steps
-        dec_bytes = n_tot / 4 + 0.5 * (nnz_w + 2 * nnz_o) + 4 * n_tot + 12 * n_tot
+        dec_bytes = n_tot / 4 + args.bits / 8 * (nnz_w + 2 * nnz_o) + 4 * n_tot + 12 * n_tot
         out["decompress"] = {"value": n_tot / (dms * 1e-3), "unit": "params/s", "ms_per_step": dms,
                              "algorithmic_gbs": dec_bytes / (dms * 1e-3) / 1e9,
                              "hbm_frac_of_measured": dec_bytes / (dms * 1e-3) / 1e9 / peak,
                              "calls_per_step": len(chunks)}
 
         # ---- the dense index layout of Sections 3.3 / 4.1 and the archiver step of Algorithm 1 -------
-        if not args.no_dense:
+        if not args.no_dense and args.bits == 4:       # the dense layout is built for the method's 4-bit records
             numels = [n for _, n in shapes]
             dsz = [binding.dense_bytes(n) for n in numels]
             dense_total = sum(dsz)

@@ -64,7 +64,8 @@ typedef struct excp_handle_s* excp_handle;
 typedef enum {
     EXCP_OK = 0,
     EXCP_ERR_INVALID_ARG = -1,      /* null / misaligned pointer, bad parameter, workspace too small for a tensor */
-    EXCP_ERR_UNSUPPORTED = -2,      /* a code width the kernels do not implement */
+    EXCP_ERR_UNSUPPORTED = -2,      /* a record variant the called routine does not handle (dense layout of a
+                                       record that is not the 4-bit method's own) */
     EXCP_ERR_BUFFER_TOO_SMALL = -3, /* blob_capacity below what the records need */
     EXCP_ERR_CUDA = -4,             /* a CUDA runtime call failed; see excp_last_cuda_error */
     EXCP_ERR_CORRUPT_BLOB = -5,     /* decompress: header, sizes, bitmap population or a code is inconsistent */
@@ -96,7 +97,8 @@ typedef enum {
 typedef struct {
     float alpha;                    /* Eq. (rw) */
     float beta;                     /* Eq. (ro) */
-    int bits;                       /* code width n; K = 2^n - 1 centres.  4 is implemented. */
+    int bits;                       /* code width n: 2, 4 or 8; K = 2^n - 1 centres (Section 4.1 uses 4; the
+                                       quantisation-bins table of Section 4.3 also 2 and 8) */
     int kmeans_iters;               /* Lloyd iterations before the final assignment (>= 0) */
     unsigned long long seed;        /* seed of the K-means start sample */
     int median_source;              /* excp_median_source */
@@ -249,7 +251,7 @@ excp_status excp_decompress_dense_checkpoint(excp_handle h, const void* dense, c
  * It takes no handle and calls no allocating routine.  The little scratch memory that decoding
  * needs (survivor counts and offsets per 4096-element tile, the parsed header, an error flag) is
  * a fixed array inside the library's device image, which every GPU that loads the library holds
- * until the process ends (about 65 KB).  It is meant for restore paths that run where memory
+ * until the process ends (about 68 KB).  It is meant for restore paths that run where memory
  * cannot be requested: on a device that the training framework's own allocator has already
  * reserved in full, so that cudaMalloc fails, or where the device-wide synchronisation that
  * cudaMalloc / cudaFree imply must not happen because other streams are busy.

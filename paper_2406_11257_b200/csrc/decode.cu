@@ -29,9 +29,10 @@ __global__ void __launch_bounds__(64) dec_validate_kernel(const DecDesc* __restr
             const u64 nnz_o = h[6] | ((u64)h[7] << 32);
             const u64 total = h[12] | ((u64)h[13] << 32);
             const u32 rf = h[11];                         // REC_*: what the record says about itself
-            const int bits = (rf & REC_RAW) ? 32 : BITS;
-            const int kc = centres_of(bits);
-            if (h[0] == MAGIC && h[1] == VERSION && numel == d.numel && !(rf & ~REC_ALL) && h[8] == (u32)bits &&
+            const int bits = (int)h[8];
+            const bool width_ok = (rf & REC_RAW) ? bits == 32 : (bits == 2 || bits == 4 || bits == 8);
+            const int kc = width_ok ? centres_of(bits) : 0;
+            if (width_ok && h[0] == MAGIC && h[1] == VERSION && numel == d.numel && !(rf & ~REC_ALL) && h[8] == (u32)bits &&
                 h[9] == (u32)kc && h[10] == header_bytes(kc) && (nnz_o <= nnz_w || (rf & REC_MOMENTS_FREE)) &&
                 nnz_w <= numel && nnz_o <= numel &&
                 total == record_bytes(numel, nnz_w, nnz_o, bits) && total <= d.rec_avail) {
@@ -50,10 +51,12 @@ __global__ void __launch_bounds__(64) dec_validate_kernel(const DecDesc* __restr
         if (!ok) atomicOr(&call->flags, FLAG_CORRUPT);
     }
     __syncthreads();
-    if (ok && tid < 3 * KPAD) {
-        const int k = tid / KPAD, j = tid % KPAD;
-        const bool has = j < KMAX && s.bits != 32;        // a raw record carries no centres
-        s.cent[k][j] = has ? reinterpret_cast<const float*>(d.rec + HEADER_FIXED)[k * KMAX + j] : 0.f;
+    if (ok) {
+        const int kc = centres_of((int)s.bits);           // 0: a raw record carries no centres
+        for (int i = tid; i < 3 * KCAP; i += 64) {
+            const int k = i / KCAP, j = i % KCAP;
+            s.cent[k][j] = j < kc ? reinterpret_cast<const float*>(d.rec + HEADER_FIXED)[k * kc + j] : 0.f;
+        }
     }
 }
 
@@ -107,8 +110,8 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
     __shared__ u32 bw[TILE_WORDS], bo[TILE_WORDS];
     __shared__ u32 pw[TILE_WORDS], po[TILE_WORDS];        // survivors before each word, within the tile
     __shared__ u32 wsum[2][TILE_WORDS / 32];
-    __shared__ u32 codes[3][TILE / 8 + 4];                // the tile's code words (+ alignment slack, + one zero word)
-    __shared__ float cent[3][KPAD];
+    __shared__ u32 codes[3][TILE / 4 + 4];                // the tile's code words (8 bits each at most; + slack, + one zero word)
+    __shared__ float cent[3][KCAP];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     u32 lo, hi;
     block_range(tiles, lo, hi);
@@ -120,7 +123,7 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
         if (cur < 0 || tile >= tb + ntl) {
             cur = find_tensor(descs, nt, tile);
             tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
-            if (tid < 3 * KPAD) cent[tid / KPAD][tid % KPAD] = st[cur].cent[tid / KPAD][tid % KPAD];
+            for (int i = tid; i < 3 * KCAP; i += TPB) cent[i / KCAP][i % KCAP] = st[cur].cent[i / KCAP][i % KCAP];
         }
         if (!st[cur].valid) continue;
         const DecDesc& d = descs[cur];
@@ -150,9 +153,11 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
         // 32-bit words of the sections (a section is padded to 16 bytes, so the last word exists)
         const bool raw = s.rflags & REC_RAW;              // sections hold fp32 survivors, read straight from the record
         const bool absolute = s.rflags & REC_ABSOLUTE;    // the weight stream is W itself
-        const u32 fw = offw / 8, fo = offo / 8;           // first staged word of the weight / moment sections
-        const u32 nww = cntw ? (offw + cntw + 7) / 8 - fw : 0;
-        const u32 nwo = cnto ? (offo + cnto + 7) / 8 - fo : 0;
+        const u32 nb = raw ? 4u : s.bits;                 // code width (raw: unused)
+        const u32 cmask = (1u << nb) - 1u;
+        const u32 fw = (u32)(((u64)offw * nb) >> 5), fo = (u32)(((u64)offo * nb) >> 5);   // first staged word of each section
+        const u32 nww = cntw ? (u32)((((u64)offw + cntw) * nb + 31) >> 5) - fw : 0;
+        const u32 nwo = cnto ? (u32)((((u64)offo + cnto) * nb + 31) >> 5) - fo : 0;
         if (!raw) {
             const u32* s0 = reinterpret_cast<const u32*>(d.rec + s.off_codes[0]) + fw;
             const u32* s1 = reinterpret_cast<const u32*>(d.rec + s.off_codes[1]) + fo;
@@ -169,7 +174,7 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
         }
         __syncthreads();
         const u64 base = (u64)(tile - tb) * TILE;
-        const u32 qw0 = offw - 8 * fw, qo0 = offo - 8 * fo;   // staged nibble index of the tile's first survivor
+        const u32 qw0 = (u32)((u64)offw * nb - 32ull * fw), qo0 = (u32)((u64)offo * nb - 32ull * fo);   // staged bit of the tile's first code
 #pragma unroll
         for (int r = 0; r < ROUNDS; ++r) {
             const u32 e0 = r * (TPB * 4) + tid * 4;       // element within the tile
@@ -196,25 +201,25 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
             }
             // this thread's survivors have consecutive ranks, so their codes are consecutive
             // nibbles: one 32-bit window per stream holds all four
-            const u32 qw = qw0 + pw[word] + __popc(bw[word] & ((1u << bit) - 1u));
-            const u32 qo = qo0 + po[word] + __popc(bo[word] & ((1u << bit) - 1u));
-            u32 win0 = __funnelshift_r(codes[0][qw >> 3], codes[0][(qw >> 3) + 1], 4 * (qw & 7u));
-            u32 win1 = __funnelshift_r(codes[1][qo >> 3], codes[1][(qo >> 3) + 1], 4 * (qo & 7u));
-            u32 win2 = __funnelshift_r(codes[2][qo >> 3], codes[2][(qo >> 3) + 1], 4 * (qo & 7u));
+            const u32 qw = qw0 + nb * (pw[word] + __popc(bw[word] & ((1u << bit) - 1u)));
+            const u32 qo = qo0 + nb * (po[word] + __popc(bo[word] & ((1u << bit) - 1u)));
+            u32 win0 = __funnelshift_r(codes[0][qw >> 5], codes[0][(qw >> 5) + 1], qw & 31u);
+            u32 win1 = __funnelshift_r(codes[1][qo >> 5], codes[1][(qo >> 5) + 1], qo & 31u);
+            u32 win2 = __funnelshift_r(codes[2][qo >> 5], codes[2][(qo >> 5) + 1], qo & 31u);
             float ow[4], oa[4], os[4];
             u32 nib0 = 0, nib1 = 0, nib2 = 0;             // DENSE: the four codes per stream
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 ow[k] = wp[k]; oa[k] = 0.f; os[k] = 0.f;
                 if ((mw4 >> k) & 1u) {
-                    const u32 c = win0 & 15u;
-                    win0 >>= 4;
+                    const u32 c = win0 & cmask;
+                    win0 >>= nb;
                     if (c == 0) bad = 1; else ow[k] = __fadd_rn(wp[k], cent[0][c - 1]);
                     nib0 |= c << (4 * k);
                 }
                 if ((mo4 >> k) & 1u) {
-                    const u32 c1 = win1 & 15u, c2 = win2 & 15u;
-                    win1 >>= 4; win2 >>= 4;
+                    const u32 c1 = win1 & cmask, c2 = win2 & cmask;
+                    win1 >>= nb; win2 >>= nb;
                     if (c1 == 0 || c2 == 0) bad = 1;
                     else { oa[k] = cent[1][c1 - 1]; os[k] = cent[2][c2 - 1]; }
                     nib1 |= c1 << (4 * k);
@@ -272,7 +277,7 @@ __global__ void __launch_bounds__(64) dense_header_kernel(const DecDesc* __restr
     const DecDesc& d = descs[t];
     DecState& s = st[t];
     if (!s.valid) return;
-    if (s.rflags) {                                       // ablation variants have no dense layout
+    if (s.rflags || s.bits != BITS) {                     // only 4-bit records of the method proper have a dense layout
         __syncthreads();
         if (tid == 0) { s.valid = 0; atomicOr(&call->flags, FLAG_UNSUPPORTED); }
         return;

@@ -147,8 +147,7 @@ bool make_groups(excp_handle h, const size_t* numel, size_t n, std::vector<Group
 
 excp_status validate_params(const excp_params* params) {
     if (!params) return EXCP_ERR_INVALID_ARG;
-    if (params->bits == 2 || params->bits == 8) return EXCP_ERR_UNSUPPORTED;
-    if (params->bits != 4 || params->kmeans_iters < 0 || (params->flags & ~OPT_ALL) ||
+    if ((params->bits != 2 && params->bits != 4 && params->bits != 8) || params->kmeans_iters < 0 || (params->flags & ~OPT_ALL) ||
         (params->median_source != 0 && params->median_source != 1) ||
         !(params->alpha >= 0.f) || !(params->beta >= 0.f) || std::isinf(params->alpha) ||
         std::isinf(params->beta))

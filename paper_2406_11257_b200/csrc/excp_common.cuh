@@ -24,6 +24,7 @@ constexpr int HIST1_BINS = 1 << HIST1_BITS;
 constexpr int HIST1_SHIFT = 31 - HIST1_BITS;     // 18 bits left for the in-bin select
 constexpr int KMAX = 15;                         // centres at 4 bits
 constexpr int KPAD = 16;
+constexpr int KCAP = 256;                        // room for the centres of the widest code (8 bits: 255)
 constexpr int SAMPLE_MAX = 1024;                 // K-means start sample
 constexpr int MAX_GROUP_TENSORS = 1024;
 
@@ -66,10 +67,8 @@ struct TensorDesc {              // built on the host, one per tensor of a group
 };
 
 struct StreamState {             // K-means state of one stream (0 = dW, 1 = ea, 2 = eas)
-    float cent[KPAD];            // centres, ascending; [15] unused
-    float thr[KPAD];             // thr[j] = largest fp32 <= (c_j + c_j+1)/2; +inf from K-1 on
-    s64 acc_sum[KPAD];           // fixed-point sums of the current pass
-    u64 acc_cnt[KPAD];
+    float cent[KCAP];            // centres, ascending; 0 from K on
+    float thr[KCAP];             // thr[j] = largest fp32 <= (c_j + c_j+1)/2; +inf from K-1 on
     u32 maxkey;                  // max |x| bit pattern over the survivors
     int e;                       // fixed-point exponent E
     float scale1, scale2;        // 2^(30-E) split in two exact factors
@@ -132,9 +131,9 @@ struct BucketStream {            // one stream's buckets
     u32 pad_;
     s64 sumpre[NBKT + 1];        // exclusive prefix of sum
     u32 cursor[NBKT];            // next free slot of each bucket while scattering
-    u32 bstar[KPAD];             // bucket that holds threshold j
-    u64 part_cnt[KPAD];          // survivors <= threshold j inside that bucket
-    s64 part_sum[KPAD];          // and their fixed-point sum
+    u32 bstar[KCAP];             // bucket that holds threshold j
+    u64 part_cnt[KCAP];          // survivors <= threshold j inside that bucket
+    s64 part_sum[KCAP];          // and their fixed-point sum
 };
 struct BucketState {
     BucketStream s[3];
@@ -186,7 +185,7 @@ struct DecState {                // decompress scratch per tensor
     u32 cnt_w, cnt_o;            // dense layout: non-zero codes met while decoding
     u32 rflags, pad_;            // the record's flags (REC_*)
     u64 off_bm_w, off_bm_o, off_codes[3];
-    float cent[3][KPAD];
+    float cent[3][KCAP];
 };
 
 // ---- layout arithmetic (host and device) ----------------------------------

@@ -25,9 +25,9 @@ constexpr u32 NA_MAX_TILES = EXCP_NOALLOC_MAX_NUMEL / TILE;
 constexpr size_t NA_OFF_CALL = 0;                       // CallState
 constexpr size_t NA_OFF_DESC = 256;                     // DecDesc
 constexpr size_t NA_OFF_STATE = 512;                    // DecState
-constexpr size_t NA_OFF_TILES = 1024;                   // 4 arrays of NA_MAX_TILES u32
+constexpr size_t NA_OFF_TILES = 4096;                   // 4 arrays of NA_MAX_TILES u32
 constexpr size_t NA_BYTES = NA_OFF_TILES + 4ull * sizeof(u32) * NA_MAX_TILES;
-static_assert(sizeof(CallState) <= 256 && sizeof(DecDesc) <= 256 && sizeof(DecState) <= 512, "scratch layout");
+static_assert(sizeof(CallState) <= 256 && sizeof(DecDesc) <= 256 && sizeof(DecState) <= 3584, "scratch layout");
 
 // In host code this name is only a handle for cudaGetSymbolAddress, never an address to pass on.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[NA_BYTES];

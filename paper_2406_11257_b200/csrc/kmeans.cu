@@ -1,5 +1,5 @@
 // Non-uniform quantisation of the survivors (Section 3.3): Lloyd's algorithm in
-// one dimension, K = 15 centres, per tensor and per stream.
+// one dimension, K = 2^bits - 1 centres (3, 15 or 255), per tensor and per stream.
 //
 //   start    K equal-mass quantiles of a seeded, index-stratified sample
 //   assign   cluster(x) = #{ j : x > thr_j },  thr_j = largest fp32 not above the
@@ -22,7 +22,7 @@
 //   bucket_offsets  prefix of the counts -> where each bucket starts
 //   bucket_scatter  sweep: survivors into their buckets, bucket sums
 //   bucket_prefix   prefix of the sums; first plan
-//   per iteration:  bucket_scan (the 14 threshold buckets), bucket_update
+//   per iteration:  bucket_scan (the K - 1 threshold buckets), bucket_update
 #include "excp_common.cuh"
 #include "seg_ring.cuh"
 
@@ -35,20 +35,20 @@ __device__ inline u64 mix64(u64 z) {   // SplitMix64 output function
     return z ^ (z >> 31);
 }
 
-__device__ inline void set_thresholds(StreamState& s, int lane) {
-    // lanes 0..15 of one warp; centres already final and sorted
-    if (lane < KPAD) {
+// Thresholds of K sorted, final centres; threads idx, idx + stride, ... of the caller share the work.
+__device__ inline void set_thresholds(StreamState& s, int K, int idx, int stride) {
+    for (int j = idx; j < KCAP; j += stride) {
         float t = __uint_as_float(0x7f800000u);
-        if (lane < KMAX - 1)
-            t = __double2float_rd(((double)s.cent[lane] + (double)s.cent[lane + 1]) * 0.5) + 0.f;   // -0 -> +0
-        s.thr[lane] = t;
+        if (j < K - 1)
+            t = __double2float_rd(((double)s.cent[j] + (double)s.cent[j + 1]) * 0.5) + 0.f;   // -0 -> +0
+        s.thr[j] = t;
     }
 }
 
 // One block per (tensor, stream).
 __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDesc* __restrict__ descs,
                                                                   TensorState* __restrict__ st,
-                                                                  Workspace ws, u64 seed) {
+                                                                  Workspace ws, u64 seed, int K) {
     __shared__ float smp[SAMPLE_MAX];
     __shared__ u32 amin, amax;                        // smallest / largest magnitude pattern in the sample
     const int t = blockIdx.x, stream = blockIdx.y, tid = threadIdx.x;
@@ -59,7 +59,7 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
     const float* data = ws.surv[stream] + (u64)tb * TILE;
     BucketStream& bk = ws.bst[t].s[stream];
     if (nnz == 0) {
-        if (tid < KPAD) { s.cent[tid] = 0.f; s.thr[tid] = __uint_as_float(0x7f800000u); }
+        if (tid < KCAP) { s.cent[tid] = 0.f; s.thr[tid] = __uint_as_float(0x7f800000u); }
         if (tid == 0) { bk.fn.lo = 0; bk.fn.shift = 0; bk.fn.sgn = stream != 2; }
         return;
     }
@@ -96,7 +96,7 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
             __syncthreads();
         }
     }
-    if (tid < KPAD) s.cent[tid] = tid < KMAX ? smp[((2 * tid + 1) * m) / (2 * KMAX)] : 0.f;
+    if (tid < KCAP) s.cent[tid] = tid < K ? smp[((2 * tid + 1) * m) / (2 * K)] : 0.f;
     // bucket function: its steps span the magnitudes seen in the sample (any monotone map
     // would give the same centres; this one spreads these survivors over the 256 buckets)
     if (tid == 0) {
@@ -106,7 +106,7 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
         bk.fn.lo = amin; bk.fn.shift = len > half_bits ? len - half_bits : 0; bk.fn.sgn = stream != 2;
     }
     __syncthreads();
-    if (tid < 32) set_thresholds(s, tid);
+    set_thresholds(s, K, tid, SAMPLE_MAX);
 }
 
 
@@ -327,12 +327,12 @@ __global__ void __launch_bounds__(TPB, 3) bucket_scatter_kernel(const TensorDesc
 }
 
 // The bucket each threshold falls into; the partial sums of the coming scan start at zero.
-// Lanes 0..13 of one warp.
-__device__ inline void plan_scan(const StreamState& s, BucketStream& bk, int lane) {
-    if (lane < KMAX - 1) {
-        bk.bstar[lane] = bucket_of(s.thr[lane], bk.fn);
-        bk.part_cnt[lane] = 0;
-        bk.part_sum[lane] = 0;
+// Threads idx, idx + stride, ... of the caller share the K - 1 thresholds.
+__device__ inline void plan_scan(const StreamState& s, BucketStream& bk, int K, int idx, int stride) {
+    for (int j = idx; j < K - 1; j += stride) {
+        bk.bstar[j] = bucket_of(s.thr[j], bk.fn);
+        bk.part_cnt[j] = 0;
+        bk.part_sum[j] = 0;
     }
 }
 
@@ -370,7 +370,7 @@ __global__ void __launch_bounds__(TPB) bucket_sum_kernel(const TensorDesc* __res
 }
 
 // Exclusive prefix of the bucket sums; plan of the first iteration.  Grid (tensors, 3).
-__global__ void __launch_bounds__(NBKT) bucket_prefix_kernel(const TensorState* __restrict__ st, Workspace ws) {
+__global__ void __launch_bounds__(NBKT) bucket_prefix_kernel(const TensorState* __restrict__ st, Workspace ws, int K) {
     __shared__ s64 wtot[NBKT / 32];
     BucketStream& bk = ws.bst[blockIdx.x].s[blockIdx.y];
     const int b = threadIdx.x, lane = b & 31, warp = b >> 5;
@@ -387,14 +387,14 @@ __global__ void __launch_bounds__(NBKT) bucket_prefix_kernel(const TensorState* 
     for (int w = 0; w < warp; ++w) base += wtot[w];
     bk.sumpre[b] = base + incl - c;
     if (b == NBKT - 1) bk.sumpre[NBKT] = base + incl;
-    if (warp == 0) plan_scan(st[blockIdx.x].s[blockIdx.y], bk, lane);
+    plan_scan(st[blockIdx.x].s[blockIdx.y], bk, K, b, NBKT);
 }
 
 // One iteration's data pass: for threshold j of a stream, the survivors of its bucket that lie
 // at or below it.  Grid (work items, 3 * 14): a tensor has scan_n items that split each bucket.
 __global__ void __launch_bounds__(TPB) bucket_scan_kernel(const TensorDesc* __restrict__ descs,
                                                           const TensorState* __restrict__ st, int nt,
-                                                          Workspace ws) {
+                                                          Workspace ws, int K) {
     __shared__ s64 rsum[TPB / 32];
     __shared__ u32 rcnt[TPB / 32];
     int lo = 0, hi = nt - 1;                       // tensor that owns this work item
@@ -402,7 +402,7 @@ __global__ void __launch_bounds__(TPB) bucket_scan_kernel(const TensorDesc* __re
         const int mid = (lo + hi + 1) >> 1;
         if (descs[mid].scan_first <= blockIdx.x) lo = mid; else hi = mid - 1;
     }
-    const int t = lo, k = blockIdx.y / (KMAX - 1), j = blockIdx.y % (KMAX - 1);
+    const int t = lo, k = blockIdx.y / (K - 1), j = blockIdx.y % (K - 1);
     const u32 split = blockIdx.x - descs[t].scan_first, nsplit = descs[t].scan_n;
     BucketStream& bk = ws.bst[t].s[k];
     const u32 b = bk.bstar[j];
@@ -449,53 +449,59 @@ __global__ void __launch_bounds__(TPB) bucket_scan_kernel(const TensorDesc* __re
     }
 }
 
-// New centres from the finished scan; one block per tensor, one warp per stream.
+// New centres from the finished scan; one block per (tensor, stream), thread j = cluster j.
 // L_j = survivors at or below threshold j = whole buckets below its bucket + the scanned part;
-// cluster k has L_k - L_(k-1) members (L_-1 = 0, L_14 = all), and its sum likewise.
-__global__ void __launch_bounds__(96) bucket_update_kernel(TensorState* __restrict__ st, Workspace ws) {
-    const int t = blockIdx.x, stream = threadIdx.x >> 5, lane = threadIdx.x & 31;
+// cluster k has L_k - L_(k-1) members (L_-1 = 0, L_(K-1) = all), and its sum likewise.
+__global__ void __launch_bounds__(KCAP) bucket_update_kernel(TensorState* __restrict__ st, Workspace ws, int K) {
+    __shared__ u64 Ls[KCAP];
+    __shared__ s64 Ss[KCAP];
+    __shared__ float cs[KCAP];
+    const int t = blockIdx.x, stream = blockIdx.y, j = threadIdx.x;
     StreamState& s = st[t].s[stream];
     BucketStream& bk = ws.bst[t].s[stream];
     u64 L = 0;
     s64 S = 0;
-    if (lane < KMAX - 1) {
-        const u32 b = bk.bstar[lane];
-        L = (u64)bk.off[b] + bk.part_cnt[lane];
-        S = bk.sumpre[b] + bk.part_sum[lane];
-    } else if (lane == KMAX - 1) {
+    if (j < K - 1) {
+        const u32 b = bk.bstar[j];
+        L = (u64)bk.off[b] + bk.part_cnt[j];
+        S = bk.sumpre[b] + bk.part_sum[j];
+    } else if (j == K - 1) {
         L = bk.off[NBKT];
         S = bk.sumpre[NBKT];
     }
-    const u64 Lp = __shfl_up_sync(0xffffffffu, L, 1);
-    const s64 Sp = __shfl_up_sync(0xffffffffu, S, 1);
-    const u64 n = lane == 0 ? L : L - Lp;
-    const s64 sum = lane == 0 ? S : S - Sp;
+    Ls[j] = L; Ss[j] = S;
+    __syncthreads();
     float c = __uint_as_float(0x7f800000u);
-    if (lane < KMAX) {
-        c = s.cent[lane];
+    if (j < K) {
+        const u64 n = j == 0 ? L : L - Ls[j - 1];
+        const s64 sum = j == 0 ? S : S - Ss[j - 1];
+        c = s.cent[j];
         if (n) {
             const double mean = __ll2double_rn(sum) / __ull2double_rn(n);
             const double scale = __longlong_as_double((s64)(s.e - 30 + 1023) << 52);
             c = __double2float_rn(mean * scale);
         }
     }
-    // sort ascending: rank of each centre among the 15 (ties by lane)
-    int rank = 0;
-    for (int j = 0; j < KMAX; ++j) {
-        const float o = __shfl_sync(0xffffffffu, c, j);
-        rank += (o < c) || (o == c && j < lane);
+    cs[j] = c;
+    __syncthreads();
+    if (j < K) {                      // sort ascending: rank of each centre among the K (ties by index)
+        int rank = 0;
+        for (int i = 0; i < K; ++i) {
+            const float o = cs[i];
+            rank += (o < c) || (o == c && i < j);
+        }
+        s.cent[rank] = c;
     }
-    __syncwarp();
-    if (lane < KMAX) s.cent[rank] = c;
-    __syncwarp();
-    set_thresholds(s, lane);
-    __syncwarp();
-    plan_scan(s, bk, lane);
+    __syncthreads();
+    set_thresholds(s, K, j, KCAP);
+    __syncthreads();
+    plan_scan(s, bk, K, j, KCAP);
 }
 
 void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                    u32 scan_items, const Workspace& ws, const Params& p, CallState* call) {
-    kmeans_start_kernel<<<dim3(nt, 3), SAMPLE_MAX, 0, cfg.stream>>>(descs, st, ws, p.seed);
+    const int K = centres_of(p.bits);
+    kmeans_start_kernel<<<dim3(nt, 3), SAMPLE_MAX, 0, cfg.stream>>>(descs, st, ws, p.seed, K);
     prof_mark(cfg, ST_KMEANS_START, 1);
     if (!tiles || p.kmeans_iters == 0) return;
     const u32 grid = min((tiles + BWARPS - 1) / BWARPS, (u32)cfg.sms * 3u);
@@ -516,12 +522,12 @@ void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* s
     }
     prof_mark(cfg, ST_BUCKET_SCATTER, 4);
     bucket_sum_kernel<<<dim3(NBKT, nt * 3), TPB, 0, cfg.stream>>>(descs, st, ws);
-    bucket_prefix_kernel<<<dim3(nt, 3), NBKT, 0, cfg.stream>>>(st, ws);
+    bucket_prefix_kernel<<<dim3(nt, 3), NBKT, 0, cfg.stream>>>(st, ws, K);
     prof_mark(cfg, ST_BUCKET_SUM, 2);
     for (int it = 0; it < p.kmeans_iters; ++it) {
-        bucket_scan_kernel<<<dim3(scan_items, 3 * (KMAX - 1)), TPB, 0, cfg.stream>>>(descs, st, nt, ws);
+        bucket_scan_kernel<<<dim3(scan_items, 3 * (K - 1)), TPB, 0, cfg.stream>>>(descs, st, nt, ws, K);
         prof_mark(cfg, ST_BUCKET_SCAN, 1);
-        bucket_update_kernel<<<nt, 96, 0, cfg.stream>>>(st, ws);
+        bucket_update_kernel<<<dim3(nt, 3), KCAP, 0, cfg.stream>>>(st, ws, K);
         prof_mark(cfg, ST_KMEANS_UPDATE, 1);
     }
 }

@@ -72,7 +72,7 @@ __global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc*
                 if (VARIANT && (opt & OPT_NO_RESIDUAL)) ip[1] = nullptr;     // W^_(t-1) is not read
             }
             const u64 e0 = ic.elem0();
-            const float* src[4] = {ip[0] + e0, ip[1] ? ip[1] + e0 : nullptr, ip[2] + e0, ip[3] + e0};
+            const float* src[4] = {ip[0] + e0, VARIANT && !ip[1] ? nullptr : ip[1] + e0, ip[2] + e0, ip[3] + e0};
             ring.issue(lane, src, ic.valid() & ~3u);
             ic.next();
         }

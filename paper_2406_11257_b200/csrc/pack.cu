@@ -10,8 +10,7 @@
 
 namespace excp {
 
-constexpr int BITS = 4;
-constexpr int PER_WORD = 32 / BITS;   // 8 codes per 32-bit word
+constexpr int BITS = 4;               // the width the method uses (Section 4.1); 2 and 8 are variants
 
 struct Sections {
     u64 bm_w, bm_o, codes[3];
@@ -46,9 +45,9 @@ __global__ void __launch_bounds__(64) header_kernel(const TensorDesc* __restrict
     const int kc = centres_of(bits);                  // 15, or 0 when the survivors are stored raw
     const u32 hb = (u32)header_bytes(kc);
     u32* h32 = reinterpret_cast<u32*>(rec);
-    if (tid < (int)(hb / 4)) {
+    for (int w = tid; w < (int)(hb / 4); w += 64) {
         u32 v = 0;
-        switch (tid) {
+        switch (w) {
             case 0: v = MAGIC; break;
             case 1: v = VERSION; break;
             case 2: v = (u32)numel; break;
@@ -64,12 +63,12 @@ __global__ void __launch_bounds__(64) header_kernel(const TensorDesc* __restrict
             case 12: v = (u32)s.blob_bytes; break;
             case 13: v = (u32)(s.blob_bytes >> 32); break;
             default:
-                if (tid >= 16 && tid < 16 + 3 * kc) {
-                    const int i = tid - 16;
-                    v = __float_as_uint(s.s[i / KMAX].cent[i % KMAX]);
+                if (w >= 16 && w < 16 + 3 * kc) {
+                    const int i = w - 16;
+                    v = __float_as_uint(s.s[i / kc].cent[i % kc]);
                 }
         }
-        h32[tid] = v;
+        h32[w] = v;
     }
     // the last 16 bytes of every code section hold the padding: clear them
     const Sections sec = sections_of(numel, nnz_w, nnz_o, bits);
@@ -84,13 +83,14 @@ __global__ void __launch_bounds__(64) header_kernel(const TensorDesc* __restrict
 __global__ void __launch_bounds__(TPB) clear_edges_kernel(const TensorDesc* __restrict__ descs,
                                                           const TensorState* __restrict__ st, int nt,
                                                           u32 tiles, Workspace ws, unsigned char* blob,
-                                                          const CallState* call) {
+                                                          const CallState* call, int bits) {
     if (call->flags & FLAG_BLOB_FULL) return;
     const u32 tile = blockIdx.x * TPB + threadIdx.x;
     if (tile >= tiles) return;
+    const u32 PER_WORD = 32u / (u32)bits;
     const int t = find_tensor(descs, nt, tile);
     const TensorState& s = st[t];
-    const Sections sec = sections_of(descs[t].numel, s.nnz_w, s.nnz_o);
+    const Sections sec = sections_of(descs[t].numel, s.nnz_w, s.nnz_o, bits);
     unsigned char* rec = blob + s.blob_off;
     for (int k = 0; k < 3; ++k) {
         const u32 cnt = (k == 0 ? ws.tile_cnt_w : ws.tile_cnt_o)[tile];
@@ -110,20 +110,33 @@ __global__ void __launch_bounds__(TPB) clear_edges_kernel(const TensorDesc* __re
 constexpr int PST = 2;
 constexpr int PWARPS = TPB / 32;
 
-template <int NS, int CH>
+template <int NS, int CH, int NB>
 struct PackSmem {
     float buf[PWARPS][PST][NS][CH];
     unsigned long long bar[PWARPS][PST];
-    float thr[PWARPS][NS][KPAD];
-    u32 rows[PWARPS][NS][CH / 8 + 2];   // [0] = last row of the previous chunk, then this chunk's rows
+    float thr[PWARPS][NS][1 << NB];     // the K - 1 thresholds, +inf after them
+    u32 rows[PWARPS][NS][CH * NB / 32 + 2];   // [0] = last row of the previous chunk, then this chunk's rows
 };
 
-template <int NS, int CH>
+// Cluster of x = number of thresholds below it: NB halving steps over the 2^NB - 1 sorted entries
+// (thr[K - 1 ...] = +inf).
+template <int NB>
+__device__ __forceinline__ u32 find_cluster(float x, const float* thr) {
+    u32 p = 0;
+#pragma unroll
+    for (int step = 1 << (NB - 1); step; step >>= 1)
+        if (x > thr[p + step - 1]) p += step;
+    return p;
+}
+
+template <int NS, int CH, int NB>
 __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __restrict__ descs,
                                                          const TensorState* __restrict__ st, int nt,
                                                          u32 tiles, Workspace ws, int stream0,
                                                          unsigned char* blob, CallState* call) {
-    __shared__ __align__(128) PackSmem<NS, CH> sm;
+    constexpr int PER = 32 / NB;                   // codes per 32-bit word = survivors per row
+    constexpr int KTHR = 1 << NB;
+    __shared__ __align__(128) PackSmem<NS, CH, NB> sm;
     if (call->flags & FLAG_BLOB_FULL) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const u32 gw = blockIdx.x * PWARPS + warp, nw = gridDim.x * PWARPS;
@@ -154,17 +167,17 @@ __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __res
                 cur = find_tensor(descs, nt, tile);
                 tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
                 const TensorState& s = st[cur];
-                const Sections sec = sections_of(descs[cur].numel, s.nnz_w, s.nnz_o);
+                const Sections sec = sections_of(descs[cur].numel, s.nnz_w, s.nnz_o, NB);
                 __syncwarp();
 #pragma unroll
                 for (int k = 0; k < NS; ++k) {
                     words[k] = reinterpret_cast<u32*>(blob + s.blob_off + sec.codes[stream0 + k]);
-                    if (lane < KPAD) sm.thr[warp][k][lane] = s.s[stream0 + k].thr[lane];
+                    for (int j = lane; j < KTHR; j += 32) sm.thr[warp][k][j] = s.s[stream0 + k].thr[j];
                 }
                 __syncwarp();
 #pragma unroll
                 for (int k = 0; k < NS; ++k) {
-                    t3[k] = sm.thr[warp][k][3]; t7[k] = sm.thr[warp][k][7]; t11[k] = sm.thr[warp][k][11];
+                    if (NB == 4) { t3[k] = sm.thr[warp][k][3]; t7[k] = sm.thr[warp][k][7]; t11[k] = sm.thr[warp][k][11]; }
                 }
             }
             const u32 cnt = ring.tile_cnt_cur(), off = ring.off(), nel = ring.nel();
@@ -173,9 +186,9 @@ __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __res
                 if (lane == 0) atomicOr(&call->flags, FLAG_TIMEOUT);
                 return;
             }
-            const u32 nrows = (nel + 7) / 8;               // rows of this chunk
-            const u32 sh = (t0 & 7u) * BITS;               // a row's shift inside the tensor's words
-            const u32 wbase = t0 / 8 + off / 8;            // output word of this chunk's first row
+            const u32 nrows = (nel + PER - 1) / PER;       // rows of this chunk
+            const u32 sh = (t0 % PER) * NB;                // a row's shift inside the tensor's words
+            const u32 wbase = t0 / PER + off / PER;        // output word of this chunk's first row
             const bool last_chunk = off + nel == cnt;
 #pragma unroll
             for (int k = 0; k < NS; ++k) {
@@ -184,15 +197,19 @@ __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __res
                 const char* thr_row = reinterpret_cast<const char*>(sm.thr[warp][k]);
                 u32* rows = sm.rows[warp][k];
                 if (lane == 0) rows[0] = carry[k];
-                for (u32 r = lane; r < nrows; r += 32) {   // 8 codes -> one word in the tile's alignment
-                    const float4 u4 = *reinterpret_cast<const float4*>(data + 8 * r);
-                    const float4 v4 = *reinterpret_cast<const float4*>(data + 8 * r + 4);
-                    const float xs[8] = {u4.x, u4.y, u4.z, u4.w, v4.x, v4.y, v4.z, v4.w};
+                for (u32 r = lane; r < nrows; r += 32) {   // PER codes -> one word in the tile's alignment
+                    float xs[PER];
+#pragma unroll
+                    for (int q = 0; q < PER / 4; ++q) {
+                        const float4 u4 = *reinterpret_cast<const float4*>(data + PER * r + 4 * q);
+                        xs[4 * q] = u4.x; xs[4 * q + 1] = u4.y; xs[4 * q + 2] = u4.z; xs[4 * q + 3] = u4.w;
+                    }
                     u32 w = 0;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const u32 code = find_cluster4(xs[i], t3[k], t7[k], t11[k], thr_row) / 4 + 1;
-                        if (8 * r + i < nel) w |= code << (BITS * i);
+                    for (int i = 0; i < PER; ++i) {
+                        const u32 code = NB == 4 ? find_cluster4(xs[i], t3[k], t7[k], t11[k], thr_row) / 4 + 1
+                                                 : find_cluster<NB>(xs[i], sm.thr[warp][k]) + 1;
+                        if (PER * r + i < nel) w |= code << (NB * i);
                     }
                     rows[1 + r] = w;
                 }
@@ -203,8 +220,8 @@ __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __res
                 const u32 nout = nrows + ((last_chunk && sh) ? 1u : 0u);
                 for (u32 m = lane; m < nout; m += 32) {
                     const u32 v = (rows[1 + m] << sh) | (sh ? rows[m] >> (32 - sh) : 0u);
-                    const u64 g0 = (u64)(wbase + m) * 8;   // ranks the word covers: [g0, g0 + 8)
-                    if (g0 >= t0 && g0 + 8 <= (u64)t0 + cnt) words[k][wbase + m] = v;
+                    const u64 g0 = (u64)(wbase + m) * PER; // ranks the word covers: [g0, g0 + PER)
+                    if (g0 >= t0 && g0 + PER <= (u64)t0 + cnt) words[k][wbase + m] = v;
                     else if (v) atomicOr(&words[k][wbase + m], v);
                 }
                 __syncwarp();
@@ -275,15 +292,23 @@ void launch_pack(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st,
         prof_mark(cfg, ST_COPY_BITMAPS, 1);
         return;
     }
-    clear_edges_kernel<<<(tiles + TPB - 1) / TPB, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, blob, call);
+    clear_edges_kernel<<<(tiles + TPB - 1) / TPB, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, blob, call, p.bits);
     prof_mark(cfg, ST_HEADER_EDGES, 2);
     const u32 grid = min((tiles + PWARPS - 1) / PWARPS, (u32)cfg.sms * 4u);
-    pack_codes_kernel<1, 512><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 0, blob, call);
-    pack_codes_kernel<2, 256><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 1, blob, call);
+    if (p.bits == 4) {
+        pack_codes_kernel<1, 512, 4><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 0, blob, call);
+        pack_codes_kernel<2, 256, 4><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 1, blob, call);
+    } else if (p.bits == 2) {
+        pack_codes_kernel<1, 512, 2><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 0, blob, call);
+        pack_codes_kernel<2, 256, 2><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 1, blob, call);
+    } else {
+        pack_codes_kernel<1, 256, 8><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 0, blob, call);
+        pack_codes_kernel<2, 128, 8><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 1, blob, call);
+    }
     prof_mark(cfg, ST_PACK_CODES, 2);
     const u64 quads = (u64)tiles * (TILE_WORDS / 4);
     copy_bitmaps_kernel<<<(u32)((quads + TPB - 1) / TPB), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws,
-                                                                               blob, call, (u32)header_bytes(KMAX));
+                                                                               blob, call, (u32)header_bytes(centres_of(p.bits)));
     prof_mark(cfg, ST_COPY_BITMAPS, 1);
 }
 
