@@ -346,7 +346,7 @@ def run_ours(args):
                              "hbm_frac_of_measured": dec_bytes / (dms * 1e-3) / 1e9 / peak,
                              "calls_per_step": len(chunks)}
 
-        # ---- the dense index layout of Sections 3.3 / 4.1 and the archiver step of Algorithm 1 -------
+        # ---- the dense index layout of Sections 3.3 / 4.2 and the archiver step of Algorithm 1 -------
         if not args.no_dense and args.bits == 4:       # the dense layout is built for the method's 4-bit records
             numels = [n for _, n in shapes]
             dsz = [binding.dense_bytes(n) for n in numels]
@@ -403,7 +403,7 @@ def run_ours(args):
             del dense
         del out_w, out_a, out_s
 
-    # ---- the rows of the ablation table of Section 4.3 (sizes and times; accuracies need training) ----
+    # ---- the rows of the ablation table of Section 4.4 (sizes and times; accuracies need training) ----
     if not args.no_ablation:
         h.profile_enable(False)
         sub, acc = [], 0

@@ -10,7 +10,7 @@
  *                M_o(i) = [ |ea(i)| > beta * mean(|ea|) ] and M_w(i)       (Section 3.2, Eq. ro)
  *                joint application of M_w to dW and of M_o to BOTH moments (Algorithm 1, joint_prune)
  *                K-means of the survivors to 2^bits - 1 centres per stream, codes 1..K,
- *                packed `bits` per code (Section 3.3; Section 4.1: bits = 4, two per byte)
+ *                packed `bits` per code (Section 3.3; Section 4.2: bits = 4, two per byte)
  *   decompress Algorithm 2 without its un-archiver step:
  *                dW^ = C_w[I_w], O^ = C_o[I_o], W^_t = W^_(t-1) + dW^
  *
@@ -81,7 +81,7 @@ typedef enum {
 /* Ablation switches: the rows of the paper's two ablation tables as variants of the same path.
  * The ViT table's caption defines the first two ("no check" under M2W: the weights are pruned by a
  * set threshold instead of alpha / sqrt(m_t); under W2M: M_o(i) = [ v_t(i) > r_o ]); the table of
- * Section 4.3 toggles residual, prune and quant.  A record written with a switch says so in its
+ * Section 4.4 toggles residual, prune and quant.  A record written with a switch says so in its
  * header (offset 44), and excp_decompress_* honour it. */
 typedef enum {
     EXCP_FLAG_NO_W2M = 1,           /* M_o(i) = [ |ea(i)| > beta * mean ], without "and M_w(i)"; record flag 1 */
@@ -93,12 +93,12 @@ typedef enum {
                                        64-byte header without centres); record flag 4 */
 } excp_flags;
 
-/* Hyper-parameters.  Section 4.1: alpha = 5e-5, beta = 2.0, bits = 4. */
+/* Hyper-parameters.  Section 4.2: alpha = 5e-5, beta = 2.0, bits = 4. */
 typedef struct {
     float alpha;                    /* Eq. (rw) */
     float beta;                     /* Eq. (ro) */
-    int bits;                       /* code width n: 2, 4 or 8; K = 2^n - 1 centres (Section 4.1 uses 4; the
-                                       quantisation-bins table of Section 4.3 also 2 and 8) */
+    int bits;                       /* code width n: 2, 4 or 8; K = 2^n - 1 centres (Section 4.2 uses 4; the
+                                       quantisation-bins table of Section 4.4 also 2 and 8) */
     int kmeans_iters;               /* Lloyd iterations before the final assignment (>= 0) */
     unsigned long long seed;        /* seed of the K-means start sample */
     int median_source;              /* excp_median_source */
@@ -206,7 +206,7 @@ excp_status excp_decompress_checkpoint(excp_handle h, const void* blob, const si
                                        void* cuda_stream);
 
 /* The index layout as the paper prints it (Section 3.3: the pruned entries stay zero and the
- * cluster index I_t is saved; Section 4.1: zero occupies one of the 2^n centres, two int4 per
+ * cluster index I_t is saved; Section 4.2: zero occupies one of the 2^n centres, two int4 per
  * int8): one code per ELEMENT, 0 where the element is pruned, no bitmap.  This is the (I, C) pair
  * Algorithm 1 hands to its archiver.  Container of one tensor (little endian, sections on 16 bytes,
  * padding zero):

@@ -12,7 +12,7 @@ What is written from the paper, and where the paper is silent:
   * moment mask  (W2M)       Section 3.2, Eq. (ro)
   * joint application        Algorithm 1, step 2 ("joint_prune")
   * non-uniform quantisation Section 3.3 (K-means to 2^n - 1 centres, zero keeps
-                             one code) and Section 4.1 (n = 4, two codes per byte)
+                             one code) and Section 4.2 (n = 4, two codes per byte)
   * reconstruction           Algorithm 2
 
 The paper does not say how the median, the mean, the K-means start, its
@@ -72,7 +72,7 @@ MEDIAN_ABS_WEIGHT = 0
 MEDIAN_ABS_RESIDUAL = 1
 
 # Ablation switches (the M2W / W2M columns of the ViT table, the residual / prune / quant columns
-# of the ablation table in Section 4.3).  0 = the full method.
+# of the ablation table in Section 4.4).  0 = the full method.
 FLAG_NO_W2M = 1        # M_o(i) = [ |ea(i)| > r_o ] without the conjunction with M_w
 FLAG_NO_M2W = 2        # weights pruned by a set threshold: M_w(i) = [ |dW(i)| > alpha ]
 FLAG_NO_RESIDUAL = 4   # the weights themselves are compressed, not their residual
@@ -87,9 +87,49 @@ REC_RAW = 4            # sections hold fp32 survivors (bits = 32, K = 0)
 _M64 = (1 << 64) - 1
 
 
+# Storage format of the WEIGHT tensors (W_t, W^_(t-1), the reconstructed W^_t).  Section 4.3 notes
+# that the PanGu-pi weights are saved in float16.  The moments stay fp32.
+WEIGHTS_F32 = 0
+WEIGHTS_F16 = 1        # numpy float16 arrays
+WEIGHTS_BF16 = 2       # numpy uint16 arrays holding the upper 16 bits of an fp32 pattern
+
+
+def widen_weights(w: np.ndarray, weight_format: int) -> np.ndarray:
+    """Stored weights -> fp32, exactly (both 16-bit formats are subsets of fp32)."""
+    if weight_format == WEIGHTS_F32:
+        return np.ascontiguousarray(w, dtype=np.float32).ravel()
+    if weight_format == WEIGHTS_F16:
+        w = np.ascontiguousarray(w).ravel()
+        if w.dtype != np.float16:
+            raise TypeError("float16 expected")
+        return w.astype(np.float32)
+    if weight_format == WEIGHTS_BF16:
+        w = np.ascontiguousarray(w).ravel()
+        if w.dtype != np.uint16:
+            raise TypeError("uint16 bit patterns expected")
+        return (w.astype(np.uint32) << np.uint32(16)).view(np.float32)
+    raise ValueError("weight format")
+
+
+def narrow_weights(w32: np.ndarray, weight_format: int) -> np.ndarray:
+    """fp32 -> the stored format, round to nearest, ties to even (finite inputs; a magnitude
+    beyond the format's range becomes infinity, as IEEE rounding has it)."""
+    w32 = np.ascontiguousarray(w32, dtype=np.float32)
+    if weight_format == WEIGHTS_F32:
+        return w32
+    if weight_format == WEIGHTS_F16:
+        with np.errstate(over="ignore"):
+            return w32.astype(np.float16)
+    if weight_format == WEIGHTS_BF16:
+        bits = w32.view(np.uint32).astype(np.uint64)
+        bits = bits + np.uint64(0x7FFF) + ((bits >> np.uint64(16)) & np.uint64(1))
+        return (bits >> np.uint64(16)).astype(np.uint16)
+    raise ValueError("weight format")
+
+
 @dataclass
 class Params:
-    """Hyper-parameters.  alpha, beta, bits: Section 4.1 (5e-5, 2.0, 4)."""
+    """Hyper-parameters.  alpha, beta, bits: Section 4.2 (5e-5, 2.0, 4)."""
     alpha: float = 5e-5
     beta: float = 2.0
     bits: int = 4
@@ -332,7 +372,7 @@ def record_bytes(numel: int, nnz_w: int, nnz_o: int, bits: int) -> int:
 
 
 def pack_codes(codes: np.ndarray, bits: int) -> bytes:
-    """Code r sits at bit r*bits of the stream, low bits first (Section 4.1:
+    """Code r sits at bit r*bits of the stream, low bits first (Section 4.2:
     two 4-bit codes per byte)."""
     per = 8 // bits
     n = codes.size
@@ -450,11 +490,12 @@ def parse_record(blob: bytes) -> dict:
 # --------------------------------------------------------------------------
 # Algorithm 1 (without the archiver) and Algorithm 2
 # --------------------------------------------------------------------------
-def compress_tensor(w_t, w_prev, ea, eas, p: Params, tensor_index: int = 0):
+def compress_tensor(w_t, w_prev, ea, eas, p: Params, tensor_index: int = 0, weight_format: int = WEIGHTS_F32):
     """Algorithm 1 for one tensor, up to (not including) the archiver.
-    Returns (record bytes, dict of every intermediate)."""
-    w_t = np.ascontiguousarray(w_t, dtype=np.float32).ravel()
-    w_prev = np.ascontiguousarray(w_prev, dtype=np.float32).ravel()
+    Returns (record bytes, dict of every intermediate).  Weights stored in a 16-bit format are
+    widened exactly and then take the same path."""
+    w_t = widen_weights(w_t, weight_format)
+    w_prev = widen_weights(w_prev, weight_format)
     ea = np.ascontiguousarray(ea, dtype=np.float32).ravel()
     eas = np.ascontiguousarray(eas, dtype=np.float32).ravel()
     n = w_t.size
@@ -508,11 +549,12 @@ def compress_tensor(w_t, w_prev, ea, eas, p: Params, tensor_index: int = 0):
     return blob, info
 
 
-def decompress_tensor(blob: bytes, w_prev):
+def decompress_tensor(blob: bytes, w_prev, weight_format: int = WEIGHTS_F32):
     """Algorithm 2: codes -> centres, W^_t = W^_(t-1) + dW^Q*; pruned entries
-    keep W^_(t-1) unchanged and decode to 0 in both moments."""
+    keep W^_(t-1) unchanged and decode to 0 in both moments.  With 16-bit weights the sum is
+    taken in fp32 and rounded once to the stored format (a pruned weight keeps its bits)."""
     r = parse_record(blob)
-    w_prev = np.ascontiguousarray(w_prev, dtype=np.float32).ravel()
+    w_prev = widen_weights(w_prev, weight_format)
     if w_prev.size != r["numel"]:
         raise ValueError("size mismatch")
     raw_values = bool(r["rec_flags"] & REC_RAW)
@@ -528,7 +570,7 @@ def decompress_tensor(blob: bytes, w_prev):
     eas_hat = np.zeros(r["numel"], dtype=np.float32)
     ea_hat[r["m_o"]] = val(r["c_ea"], r["codes_ea"])
     eas_hat[r["m_o"]] = val(r["c_eas"], r["codes_eas"])
-    return w_hat, ea_hat, eas_hat
+    return narrow_weights(w_hat, weight_format), ea_hat, eas_hat
 
 
 def compress_checkpoint(tensors, p: Params):
@@ -549,7 +591,7 @@ def decompress_checkpoint(blob: bytes, offsets, w_prev_list):
 
 
 # --------------------------------------------------------------------------
-# The index layout as Sections 3.3 and 4.1 print it: one code per ELEMENT, the
+# The index layout as Sections 3.3 and 4.2 print it: one code per ELEMENT, the
 # pruned ones holding the code of the zero centre (0), no bitmap.  This is the
 # (I, C) pair that Algorithm 1 hands to its archiver.
 # --------------------------------------------------------------------------
@@ -566,7 +608,7 @@ def dense_bytes(numel: int, bits: int) -> int:
 
 def dense_indices(mask: np.ndarray, codes: np.ndarray) -> np.ndarray:
     """I(i) = code of element i (1..K) where the mask keeps it, 0 (the zero
-    centre of Section 4.1) where it is pruned."""
+    centre of Section 4.2) where it is pruned."""
     idx = np.zeros(mask.size, dtype=np.uint8)
     idx[mask] = codes
     return idx
@@ -576,7 +618,7 @@ def encode_dense(numel, bits, nnz_w, nnz_o, c_w, c_ea, c_eas, idx_w, idx_ea, idx
     """The dense container.  The header is the record's with magic "EXCD" and
     the container's size at offset 48; after the centres come the indices of
     dW, of the first moment and of the second, `bits` per element, element i at
-    bit i*bits of its section (Section 4.1: two int4 per int8), each section
+    bit i*bits of its section (Section 4.2: two int4 per int8), each section
     padded with zeros to 16 bytes."""
     k = (1 << bits) - 1
     hb = header_bytes(k)

@@ -263,7 +263,7 @@ class Handle:
         if st != 0:
             raise ExcpError(st, "excp_decompress_dense_checkpoint" if dense else "excp_decompress_checkpoint")
 
-    # ---- the dense index layout (Sections 3.3 / 4.1) ----------------------
+    # ---- the dense index layout (Sections 3.3 / 4.2) ----------------------
     def record_to_dense(self, record: torch.Tensor, record_bytes: int, numel: int, dense_out: torch.Tensor) -> int:
         out = C.c_size_t(0)
         st = self.lib.excp_record_to_dense(self._h, record.data_ptr(), record_bytes, numel, dense_out.data_ptr(),

@@ -267,7 +267,7 @@ void launch_decode(const LaunchCfg& cfg, const DecDesc* descs, DecState* st, int
 }
 
 // ---------------------------------------------------------------------------
-// The dense layout (Sections 3.3 and 4.1 as printed): header + centres as in the record (magic
+// The dense layout (Sections 3.3 and 4.2 as printed): header + centres as in the record (magic
 // "EXCD", the container's size at offset 48), then one code per element for dW, ea and eas.
 
 // Header, centres and the zero padding at the end of every section.  One block per tensor.

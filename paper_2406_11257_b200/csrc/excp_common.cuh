@@ -35,7 +35,7 @@ constexpr u32 FLAG_INTERNAL = 8u;                // a self-check failed (candida
 constexpr u32 FLAG_TIMEOUT = 16u;                // a bounded wait on an asynchronous copy ran out
 constexpr u32 FLAG_UNSUPPORTED = 32u;            // a record variant the called routine does not handle
 
-// Ablation switches of a compress call (ViT table caption; ablation table of Section 4.3)
+// Ablation switches of a compress call (ViT table caption; ablation table of Section 4.4)
 constexpr u32 OPT_NO_W2M = 1u;                   // M_o without the conjunction with M_w
 constexpr u32 OPT_NO_M2W = 2u;                   // M_w = [ |dW| > alpha ], alpha the set threshold
 constexpr u32 OPT_NO_RESIDUAL = 4u;              // the weights themselves, not their residual

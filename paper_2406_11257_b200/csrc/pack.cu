@@ -1,6 +1,6 @@
 // Writing one record per tensor (the layout in include/excp.h): header with
 // the three codebooks, the two bitmaps, and the final K-means assignment packed
-// as 4-bit codes 1..15, two per byte, survivors in index order (Section 4.1).
+// as 4-bit codes 1..15, two per byte, survivors in index order (Section 4.2).
 //
 // A tile's survivors start at an arbitrary rank of the tensor, so the first and
 // last 32-bit code word of a tile may be shared with its neighbours: those words
@@ -10,7 +10,7 @@
 
 namespace excp {
 
-constexpr int BITS = 4;               // the width the method uses (Section 4.1); 2 and 8 are variants
+constexpr int BITS = 4;               // the width the method uses (Section 4.2); 2 and 8 are variants
 
 struct Sections {
     u64 bm_w, bm_o, codes[3];
@@ -253,7 +253,7 @@ __global__ void __launch_bounds__(TPB) copy_bitmaps_kernel(const TensorDesc* __r
     reinterpret_cast<uint4*>(rec + hb + quads * 16)[local] = b;
 }
 
-// Quantisation switched off (ablation table of Section 4.3): the survivors themselves go into the
+// Quantisation switched off (ablation table of Section 4.4): the survivors themselves go into the
 // sections, fp32, in index order.  One warp per tile: its segment of each stream is copied to the
 // tile's rank offset in the section.
 __global__ void __launch_bounds__(TPB) pack_raw_kernel(const TensorDesc* __restrict__ descs,

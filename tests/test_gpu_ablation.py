@@ -1,5 +1,5 @@
 """GPU parity for the ablation switches (ViT table caption: no M2W / no W2M; ablation table of
-Section 4.3: residual / prune / quant off): records byte-identical to the oracle's, Algorithm 2
+Section 4.4: residual / prune / quant off): records byte-identical to the oracle's, Algorithm 2
 bit-identical, for every switch alone and for combinations."""
 import numpy as np
 import pytest

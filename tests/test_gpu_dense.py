@@ -1,4 +1,4 @@
-"""GPU parity for the dense index layout (Sections 3.3 / 4.1: one code per element, 0 = pruned):
+"""GPU parity for the dense index layout (Sections 3.3 / 4.2: one code per element, 0 = pruned):
 record -> dense container and Algorithm 2 on the container, against the oracle, byte for byte."""
 import numpy as np
 import pytest

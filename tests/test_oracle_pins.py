@@ -455,7 +455,7 @@ def test_checkpoint_container_offsets():
     assert b0 == blob[offs[3]:offs[4]]
 
 
-# ------------------------------------------- dense index layout (Sections 3.3 / 4.1) and the archiver
+# ------------------------------------------- dense index layout (Sections 3.3 / 4.2) and the archiver
 def rand_quad(n, seed):
     rng = np.random.default_rng(seed)
     wp = rng.normal(0, 0.02, n).astype(np.float32)
@@ -558,7 +558,7 @@ def test_archiver_round_trip_and_sizes():
     assert z["archived_bytes"] < 400                          # LZMA2 collapses a run of zeros
 
 
-# ------------------------------------------------ ablation switches (ViT table caption, Section 4.3)
+# ------------------------------------------------ ablation switches (ViT table caption, Section 4.4)
 def hand_params(flags):
     return orc.Params(alpha=G["alpha"][0], beta=G["beta"][0], bits=4, flags=flags)
 
@@ -648,3 +648,62 @@ def test_flagged_records_keep_their_rules():
         orc.parse_record(bytes(b))
     with pytest.raises(ValueError):
         orc.compress_tensor(wt, wp, ea, eas, orc.Params(flags=32))
+
+
+# ------------------------------------------------ 16-bit weight storage (Section 4.3: float16 weights)
+def test_widening_is_exact_on_known_patterns():
+    f16 = np.array([0x3C00, 0xBC00, 0x0001, 0x7BFF, 0x0400, 0x8000], dtype=np.uint16).view(np.float16)
+    want = np.array([1.0, -1.0, 2.0 ** -24, 65504.0, 2.0 ** -14, -0.0], dtype=np.float32)
+    got = orc.widen_weights(f16, orc.WEIGHTS_F16)
+    np.testing.assert_array_equal(got.view(np.uint32), want.view(np.uint32))
+    bf = np.array([0x3F80, 0xBF80, 0x0001, 0x7F7F, 0x0080, 0x8000], dtype=np.uint16)
+    want = np.array([1.0, -1.0, 2.0 ** -133, (2 - 2.0 ** -7) * 2.0 ** 127, 2.0 ** -126, -0.0], dtype=np.float32)
+    got = orc.widen_weights(bf, orc.WEIGHTS_BF16)
+    np.testing.assert_array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+def _nearest_even(x: float, candidates):
+    """Nearest of the candidate values (exact rationals), ties to the one with an even index."""
+    fx = Fraction(x)
+    best = min(range(len(candidates)), key=lambda i: (abs(Fraction(candidates[i]) - fx), i % 2))
+    return candidates[best]
+
+
+@pytest.mark.parametrize("fmt", [orc.WEIGHTS_F16, orc.WEIGHTS_BF16])
+def test_narrowing_is_round_to_nearest_even(fmt):
+    rng = np.random.default_rng(5)
+    # all positive values of the format in [2^-3, 2^1], in order: index parity = mantissa parity
+    if fmt == orc.WEIGHTS_F16:
+        pats = np.arange(0x3000, 0x4001, dtype=np.uint16)
+        grid = [float(v) for v in pats.view(np.float16).astype(np.float64)]
+    else:
+        pats = np.arange(0x3E00, 0x4001, dtype=np.uint16)
+        grid = [float(v) for v in (pats.astype(np.uint32) << 16).view(np.float32).astype(np.float64)]
+    xs = rng.uniform(0.125, 2.0, 400).astype(np.float32)
+    ties = np.array([(grid[i] + grid[i + 1]) / 2 for i in range(0, 60)], dtype=np.float32)   # exact mid-points
+    for x in np.concatenate([xs, ties, -ties[:8]]):
+        want = _nearest_even(abs(float(x)), grid) * (1 if x > 0 else -1)
+        got = orc.widen_weights(orc.narrow_weights(np.array([x], np.float32), fmt), fmt)[0]
+        assert float(got) == want, (x, got, want)
+    # stored values survive a round trip bit for bit
+    back = orc.narrow_weights(orc.widen_weights(pats.view(np.float16) if fmt == orc.WEIGHTS_F16 else pats, fmt), fmt)
+    np.testing.assert_array_equal(back.view(np.uint16), pats)
+
+
+@pytest.mark.parametrize("fmt", [orc.WEIGHTS_F16, orc.WEIGHTS_BF16])
+def test_sixteen_bit_weights_take_the_fp32_path_after_widening(fmt):
+    wt, wp, ea, eas = rand_quad(5000, 61)
+    n16 = lambda a: orc.narrow_weights(a, fmt)
+    wp16 = n16(wp)
+    wt16 = n16((orc.widen_weights(wp16, fmt) + (wt - wp) * 30).astype(np.float32))   # residuals a 16-bit format can hold
+    p = orc.Params(median_source=orc.MEDIAN_ABS_RESIDUAL, kmeans_iters=3)
+    blob, info = orc.compress_tensor(wt16, wp16, ea, eas, p, weight_format=fmt)
+    blob32, _ = orc.compress_tensor(orc.widen_weights(wt16, fmt), orc.widen_weights(wp16, fmt), ea, eas, p)
+    assert blob == blob32 and 0 < info["nnz_w"] < 5000
+    w_hat, ea_hat, eas_hat = orc.decompress_tensor(blob, wp16, weight_format=fmt)
+    assert w_hat.dtype == (np.float16 if fmt == orc.WEIGHTS_F16 else np.uint16)
+    w32, ea32, eas32 = orc.decompress_tensor(blob, orc.widen_weights(wp16, fmt))
+    np.testing.assert_array_equal(w_hat.view(np.uint16), n16(w32).view(np.uint16))
+    np.testing.assert_array_equal(ea_hat, ea32)
+    pruned = ~info["m_w"]
+    np.testing.assert_array_equal(w_hat.view(np.uint16)[pruned], wp16.view(np.uint16)[pruned])
