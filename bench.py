@@ -48,6 +48,8 @@ def parse_args():
     ap.add_argument("--workspace-numel", type=int, default=1_200_000_000)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--weights", default="f32", choices=["f32", "f16", "bf16"],
+                    help="storage format of W_t and W^_(t-1) (f32 is the headline's; 16-bit: the paper's float16-weight case)")
     ap.add_argument("--bits", type=int, default=4, choices=[2, 4, 8],
                     help="code width (4 is the method's and the headline's; 2 and 8 are the quantisation-bins variants)")
     ap.add_argument("--no-decompress", action="store_true")
@@ -211,6 +213,17 @@ def run_ours(args):
     n_tot = sum(n for _, n in shapes)
     seed = 1000 + rank                                    # every rank compresses its own checkpoint
     quads = [synth.make_quad(n, seed, i, device=dev) for i, (_, n) in enumerate(shapes)]
+    wfmt = {"f32": binding.WEIGHTS_F32, "f16": binding.WEIGHTS_F16, "bf16": binding.WEIGHTS_BF16}[args.weights]
+    wb = 4 if wfmt == binding.WEIGHTS_F32 else 2            # bytes per stored weight
+    if wb == 2:
+        # 16-bit storage: W^_(t-1) rounded to the format, W_t = that + 30x the synthetic residual (a residual
+        # of 1e-4 is below half's spacing at |w| ~ 0.02), rounded to the format
+        wdt = torch.float16 if wfmt == binding.WEIGHTS_F16 else torch.bfloat16
+        for i, (w_t, w_prev, ea, eas) in enumerate(quads):
+            wp16 = w_prev.to(wdt)
+            w_t.sub_(w_prev).mul_(30.0).add_(wp16.float())
+            quads[i] = (w_t.to(wdt), wp16, ea, eas)
+            del w_t, w_prev
     torch.cuda.synchronize()
 
     ws_numel = min(args.workspace_numel, n_tot + 4096 * len(shapes))
@@ -225,7 +238,7 @@ def run_ours(args):
     h.profile_enable(True)
     offs = stats = None
     for _ in range(max(args.warmup, 0)):
-        offs, stats = h.compress_checkpoint(p, quads, blob)
+        offs, stats = h.compress_checkpoint(p, quads, blob, weight_format=wfmt)
     stage_ms = {}
     launches = 0
     sampler = ClockSampler(local)
@@ -234,7 +247,7 @@ def run_ours(args):
     sampler.start()
     ev0.record()
     for _ in range(args.steps):
-        offs, stats = h.compress_checkpoint(p, quads, blob)
+        offs, stats = h.compress_checkpoint(p, quads, blob, weight_format=wfmt)
         ms, l = h.profile_read()
         launches += l
         for k, v in ms.items():
@@ -255,12 +268,12 @@ def run_ours(args):
     blob_bytes = offs[-1]
     f_w, f_o = nnz_w / n_tot, nnz_o / n_tot
     T = args.kmeans_iters
-    src_b = 8 if args.median == "residual" else 4
+    src_b = 2 * wb if args.median == "residual" else wb
     # bytes each stage must move once (its inputs read once, its outputs written once)
     surv = nnz_w + 2 * nnz_o
     stage_bytes = {
         "stats1": (src_b + 4) * n_tot,
-        "mask_compact": 16 * n_tot + n_tot / 4 + 4 * surv,
+        "mask_compact": (2 * wb + 8) * n_tot + n_tot / 4 + 4 * surv,
         "bucket_ids": 4 * surv,                     # survivors read once to count them per bucket
         "bucket_scatter": 8 * surv,                 # survivors read and written into their buckets
         "bucket_sum": 4 * surv,                     # the bucketed copy read once for the bucket sums
@@ -271,7 +284,7 @@ def run_ours(args):
     moved_bytes = sum(stage_bytes.values())         # what these kernels must move by design
     # what the method moves when every Lloyd iteration sweeps the survivors (one statistics sweep,
     # one mask sweep, T + 1 sweeps of the survivors, the codes)
-    algo_bytes = ((src_b + 4) + 16 + 0.25) * n_tot + 4 * surv + (T + 1) * 4 * surv + args.bits / 8 * surv
+    algo_bytes = ((src_b + 4) + (2 * wb + 8) + 0.25) * n_tot + 4 * surv + (T + 1) * 4 * surv + args.bits / 8 * surv
     peak, peak_kind = measured_peak()
     per_step = {k: v / args.steps for k, v in stage_ms.items()}
     dom = max((k for k in stage_bytes), key=lambda k: per_step.get(k, 0.0))
@@ -286,11 +299,11 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": "params/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{shape.name} checkpoint pair ({len(shapes)} tensors, {n_tot} params, fp32 W_t, W_prev, ea, eas), "
+        "config": {"workload": f"{shape.name} checkpoint pair ({len(shapes)} tensors, {n_tot} params, {args.weights} W_t, W_prev, fp32 ea, eas), "
                                f"median of |{'dW' if args.median == 'residual' else 'W_t'}|, alpha 5e-5, beta 2.0",
                    "bits": args.bits, "kmeans_iters": T, "l2": "inputs larger than L2 (no flush needed)" if 16 * n_tot > 4e8 else "inputs fit L2",
                    "workspace_numel": ws_numel, "per_rank": "each rank compresses its own checkpoint; no collective"},
-        "input_gbs": 16 * value / 1e9,
+        "input_gbs": (2 * wb + 8) * value / 1e9,
         "algorithmic_bytes_per_param": algo_bytes / n_tot,
         "moved_bytes_per_param": moved_bytes / n_tot,
         "moved_gbs": moved_bytes / n_tot * value / world / 1e9,
@@ -299,7 +312,8 @@ def run_ours(args):
         "hbm_frac_of_measured": algo_bytes / n_tot * value / world / 1e9 / peak,
         "hbm_frac_of_nominal_8TBs": algo_bytes / n_tot * value / world / 1e9 / NOMINAL_HBM_GBS,
         "survivors": {"f_w": f_w, "f_o": f_o},
-        "compression": {"blob_bytes": blob_bytes, "ratio_vs_12B_per_param": 12 * n_tot / blob_bytes},
+        "compression": {"blob_bytes": blob_bytes, "ratio_vs_12B_per_param": 12 * n_tot / blob_bytes,
+                        "ratio_vs_stored_state": (wb + 8) * n_tot / blob_bytes},
         "stages": stages,
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
                      "frac": dom_gbs / peak, "peak_kind": peak_kind,
@@ -313,7 +327,7 @@ def run_ours(args):
     if not args.no_decompress:
         h.profile_enable(False)
         chunk_cap = ws_numel
-        out_w = torch.empty(chunk_cap, dtype=torch.float32, device=dev)
+        out_w = torch.empty(chunk_cap, dtype=quads[0][1].dtype, device=dev)
         out_a = torch.empty(chunk_cap, dtype=torch.float32, device=dev)
         out_s = torch.empty(chunk_cap, dtype=torch.float32, device=dev)
         chunks, cur, used = [], [], 0
@@ -331,7 +345,7 @@ def run_ours(args):
                 wp = [quads[i][1] for i, _, _ in ch]
                 h.decompress_checkpoint(blob[offs[i0]:], [o - offs[i0] for o in offs[i0:i1 + 1]], wp,
                                         [out_w[o:o + n] for _, o, n in ch], [out_a[o:o + n] for _, o, n in ch],
-                                        [out_s[o:o + n] for _, o, n in ch])
+                                        [out_s[o:o + n] for _, o, n in ch], weight_format=wfmt)
         decompress_all()
         torch.cuda.synchronize()
         d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -340,14 +354,14 @@ def run_ours(args):
             decompress_all()
         d1.record(); torch.cuda.synchronize()
         dms = d0.elapsed_time(d1) / args.steps
-        dec_bytes = n_tot / 4 + args.bits / 8 * (nnz_w + 2 * nnz_o) + 4 * n_tot + 12 * n_tot
+        dec_bytes = n_tot / 4 + args.bits / 8 * (nnz_w + 2 * nnz_o) + wb * n_tot + (wb + 8) * n_tot
         out["decompress"] = {"value": n_tot / (dms * 1e-3), "unit": "params/s", "ms_per_step": dms,
                              "algorithmic_gbs": dec_bytes / (dms * 1e-3) / 1e9,
                              "hbm_frac_of_measured": dec_bytes / (dms * 1e-3) / 1e9 / peak,
                              "calls_per_step": len(chunks)}
 
         # ---- the dense index layout of Sections 3.3 / 4.2 and the archiver step of Algorithm 1 -------
-        if not args.no_dense and args.bits == 4:       # the dense layout is built for the method's 4-bit records
+        if not args.no_dense and args.bits == 4 and wb == 4:       # the dense layout is built for the method's 4-bit records
             numels = [n for _, n in shapes]
             dsz = [binding.dense_bytes(n) for n in numels]
             dense_total = sum(dsz)
@@ -404,7 +418,7 @@ def run_ours(args):
         del out_w, out_a, out_s
 
     # ---- the rows of the ablation table of Section 4.4 (sizes and times; accuracies need training) ----
-    if not args.no_ablation:
+    if not args.no_ablation and wb == 4:
         h.profile_enable(False)
         sub, acc = [], 0
         for i, (_, n) in enumerate(shapes):
@@ -434,7 +448,7 @@ def run_ours(args):
         del ablob
 
     # ---- end to end through the host-buffer entry point ----------------------
-    if not args.no_e2e:
+    if not args.no_e2e and wb == 4:
         need_gb = 16 * n_tot / 1e9
         sub = list(range(len(shapes)))
         if mem_available_gb() < 1.4 * need_gb + 8:

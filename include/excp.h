@@ -168,6 +168,33 @@ excp_status excp_compress_checkpoint(excp_handle h, const excp_params* params, s
                                      size_t* tensor_offsets_out, excp_tensor_stats* stats_out,
                                      void* cuda_stream);
 
+/* Weights stored in 16 bits (Section 4.3 notes that the PanGu-pi weights are saved in float16).
+ * excp_compress_checkpoint with W_t and W^_(t-1) given as IEEE binary16 (EXCP_WEIGHTS_F16) or
+ * bfloat16 (EXCP_WEIGHTS_BF16) arrays; the moments stay fp32.  Every weight is widened to fp32,
+ * which is exact, and from there the path is the fp32 one: the record is byte for byte the record
+ * of the widened tensors, and carries no trace of the storage format.
+ *   w_t, w_prev           host arrays [num_tensors] of device pointers to numel[i] 16-bit values,
+ *                         16-byte aligned.
+ * Everything else as for excp_compress_checkpoint. */
+typedef enum {
+    EXCP_WEIGHTS_F16 = 1,
+    EXCP_WEIGHTS_BF16 = 2
+} excp_weight_format;
+excp_status excp_compress_checkpoint_w16(excp_handle h, const excp_params* params, size_t num_tensors,
+                                         const void* const* w_t, const void* const* w_prev,
+                                         const float* const* ea, const float* const* eas,
+                                         const size_t* numel, int weight_format, void* blob_out, size_t blob_capacity,
+                                         size_t* tensor_offsets_out, excp_tensor_stats* stats_out,
+                                         void* cuda_stream);
+
+/* excp_decompress_checkpoint for 16-bit weights: w_prev and w_out hold `weight_format` values.
+ * W^_t = W^_(t-1) + dW^ is taken in fp32 and rounded once, to nearest even, to the stored format;
+ * a pruned weight keeps the bits of W^_(t-1).  ea_out, eas_out are fp32. */
+excp_status excp_decompress_checkpoint_w16(excp_handle h, const void* blob, const size_t* tensor_offsets,
+                                           size_t num_tensors, const void* const* w_prev, const size_t* numel,
+                                           int weight_format, void* const* w_out, float* const* ea_out,
+                                           float* const* eas_out, void* cuda_stream);
+
 /* excp_compress_checkpoint for a checkpoint that lives in HOST memory (the usual case: the
  * compression runs beside training, Section 3.4, on a copy of the states).
  *   w_t, w_prev, ea, eas  host arrays [num_tensors] of HOST pointers (fp32[numel[i]]); page-locked

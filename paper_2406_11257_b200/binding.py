@@ -20,7 +20,8 @@ STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED", -3: "BUFFER_TOO_SMALL",
 
 EXPORTS = ["excp_create", "excp_destroy", "excp_record_bytes", "excp_compress_bound",
            "excp_status_string", "excp_last_cuda_error", "excp_compress_tensor",
-           "excp_compress_checkpoint", "excp_compress_checkpoint_host", "excp_decompress_tensor", "excp_decompress_checkpoint",
+           "excp_compress_checkpoint", "excp_compress_checkpoint_w16", "excp_decompress_checkpoint_w16",
+           "excp_compress_checkpoint_host", "excp_decompress_tensor", "excp_decompress_checkpoint",
            "excp_decompress_tensor_noalloc", "excp_dense_bytes", "excp_record_to_dense", "excp_checkpoint_to_dense",
            "excp_decompress_dense_tensor", "excp_decompress_dense_checkpoint", "excp_profile_enable", "excp_profile_stage_count", "excp_profile_stage_name", "excp_profile_read"]
 
@@ -86,6 +87,11 @@ def load_library() -> C.CDLL:
                                              C.POINTER(vp), C.POINTER(vp), C.POINTER(sz), vp, sz,
                                              C.POINTER(sz), C.POINTER(CStats), vp]
     lib.excp_compress_checkpoint_host.argtypes = lib.excp_compress_checkpoint.argtypes
+    lib.excp_compress_checkpoint_w16.argtypes = [vp, C.POINTER(CParams), sz, C.POINTER(vp), C.POINTER(vp),
+                                                 C.POINTER(vp), C.POINTER(vp), C.POINTER(sz), C.c_int, vp, sz,
+                                                 C.POINTER(sz), C.POINTER(CStats), vp]
+    lib.excp_decompress_checkpoint_w16.argtypes = [vp, vp, C.POINTER(sz), sz, C.POINTER(vp), C.POINTER(sz), C.c_int,
+                                                   C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), vp]
     lib.excp_decompress_tensor.argtypes = [vp, vp, sz, vp, sz, vp, vp, vp, vp]
     lib.excp_decompress_checkpoint.argtypes = [vp, vp, C.POINTER(sz), sz, C.POINTER(vp), C.POINTER(sz),
                                                C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), vp]
@@ -116,6 +122,16 @@ def _check_f32_cuda(*ts: torch.Tensor) -> None:
     for t in ts:
         if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
             raise TypeError("expected contiguous float32 CUDA tensors")
+
+
+WEIGHTS_F32, WEIGHTS_F16, WEIGHTS_BF16 = 0, 1, 2
+_WEIGHT_DTYPE = {WEIGHTS_F32: torch.float32, WEIGHTS_F16: torch.float16, WEIGHTS_BF16: torch.bfloat16}
+
+
+def _check_weights(weight_format: int, *ts: torch.Tensor) -> None:
+    for t in ts:
+        if not (t.is_cuda and t.dtype == _WEIGHT_DTYPE[weight_format] and t.is_contiguous()):
+            raise TypeError(f"expected contiguous {_WEIGHT_DTYPE[weight_format]} CUDA tensors")
 
 
 def _stream() -> int:
@@ -202,22 +218,28 @@ class Handle:
             raise ExcpError(st, "excp_compress_tensor")
         return nbytes.value, stats
 
-    def compress_checkpoint(self, p: Params, tensors, blob_out: torch.Tensor, want_stats: bool = True):
-        """excp_compress_checkpoint over a list of (w_t, w_prev, ea, eas).
-        Returns (offsets list of len n+1, list of stats or None)."""
+    def compress_checkpoint(self, p: Params, tensors, blob_out: torch.Tensor, want_stats: bool = True,
+                            weight_format: int = WEIGHTS_F32):
+        """excp_compress_checkpoint (or, for 16-bit weights, excp_compress_checkpoint_w16) over a list of
+        (w_t, w_prev, ea, eas).  Returns (offsets list of len n+1, list of stats or None)."""
         n = len(tensors)
         for q in tensors:
-            _check_f32_cuda(*q)
+            _check_weights(weight_format, q[0], q[1])
+            _check_f32_cuda(q[2], q[3])
         arr = lambda k: (C.c_void_p * n)(*[_ptr(q[k]) for q in tensors])
         numel = (C.c_size_t * n)(*[q[0].numel() for q in tensors])
         offs = (C.c_size_t * (n + 1))()
         stats = (CStats * n)() if want_stats else None
         cp = p.to_c()
-        st = self.lib.excp_compress_checkpoint(self._h, C.byref(cp), n, arr(0), arr(1), arr(2), arr(3), numel,
-                                               blob_out.data_ptr(), blob_out.numel() * blob_out.element_size(),
-                                               offs, stats, _stream())
+        cap = blob_out.numel() * blob_out.element_size()
+        if weight_format == WEIGHTS_F32:
+            st = self.lib.excp_compress_checkpoint(self._h, C.byref(cp), n, arr(0), arr(1), arr(2), arr(3), numel,
+                                                   blob_out.data_ptr(), cap, offs, stats, _stream())
+        else:
+            st = self.lib.excp_compress_checkpoint_w16(self._h, C.byref(cp), n, arr(0), arr(1), arr(2), arr(3), numel,
+                                                       weight_format, blob_out.data_ptr(), cap, offs, stats, _stream())
         if st != 0:
-            raise ExcpError(st, "excp_compress_checkpoint")
+            raise ExcpError(st, "excp_compress_checkpoint" + ("" if weight_format == WEIGHTS_F32 else "_w16"))
         return list(offs), (list(stats) if want_stats else None)
 
     def compress_checkpoint_host(self, p: Params, tensors, blob_out: torch.Tensor, want_stats: bool = True):
@@ -251,12 +273,21 @@ class Handle:
             raise ExcpError(st, "excp_decompress_tensor")
 
     def decompress_checkpoint(self, blob: torch.Tensor, offsets, w_prev, w_out, ea_out, eas_out,
-                              dense: bool = False) -> None:
+                              dense: bool = False, weight_format: int = WEIGHTS_F32) -> None:
         n = len(w_prev)
-        _check_f32_cuda(*w_prev, *w_out, *ea_out, *eas_out)
+        _check_weights(weight_format, *w_prev, *w_out)
+        _check_f32_cuda(*ea_out, *eas_out)
         arr = lambda ts: (C.c_void_p * n)(*[_ptr(t) for t in ts])
         numel = (C.c_size_t * n)(*[t.numel() for t in w_prev])
         offs = (C.c_size_t * (n + 1))(*offsets)
+        if weight_format != WEIGHTS_F32:
+            if dense:
+                raise ValueError("the dense layout decodes to fp32 weights only")
+            st = self.lib.excp_decompress_checkpoint_w16(self._h, blob.data_ptr(), offs, n, arr(w_prev), numel,
+                                                         weight_format, arr(w_out), arr(ea_out), arr(eas_out), _stream())
+            if st != 0:
+                raise ExcpError(st, "excp_decompress_checkpoint_w16")
+            return
         fn = self.lib.excp_decompress_dense_checkpoint if dense else self.lib.excp_decompress_checkpoint
         st = fn(self._h, blob.data_ptr(), offs, n, arr(w_prev), numel, arr(w_out), arr(ea_out), arr(eas_out),
                 _stream())

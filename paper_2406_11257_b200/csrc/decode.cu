@@ -103,7 +103,7 @@ __global__ void __launch_bounds__(TPB) dec_scan_kernel(const DecDesc* __restrict
 
 // DENSE = false: Algorithm 2, fp32 outputs.  DENSE = true: the same walk writes each element's
 // code (0 where pruned) into the three sections of the dense layout instead.
-template <bool DENSE>
+template <bool DENSE, typename WT>
 __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__ descs,
                                                      const DecState* __restrict__ st, int nt, u32 tiles,
                                                      Workspace ws, CallState* call) {
@@ -128,6 +128,8 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
         if (!st[cur].valid) continue;
         const DecDesc& d = descs[cur];
         const DecState& s = st[cur];
+        const WT* w_prev = static_cast<const WT*>(d.w_prev);
+        WT* w_out = static_cast<WT*>(d.w_out);
         const u64 n = d.numel;
         const u64 nwords = bitmap_bytes(n) / 4;
         const u64 w0 = (u64)(tile - tb) * TILE_WORDS;
@@ -182,7 +184,7 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
             const bool live = i0 < n;
             if (!DENSE && !live) continue;
             float wp[4] = {0.f, 0.f, 0.f, 0.f};
-            if (!DENSE && !absolute) load4(d.w_prev, i0, n, wp);
+            if (!DENSE && !absolute) load4(w_prev, i0, n, wp);
             const u32 word = e0 >> 5, bit = e0 & 31;
             const u32 mw4 = (bw[word] >> bit) & 15u, mo4 = (bo[word] >> bit) & 15u;
             if (!DENSE && raw) {
@@ -195,7 +197,7 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
                     float w = wp[k], a = 0.f, e = 0.f;
                     if ((mw4 >> k) & 1u) w = __fadd_rn(wp[k], vw[gw++]);
                     if ((mo4 >> k) & 1u) { a = va[go]; e = ve[go]; ++go; }
-                    d.w_out[i0 + k] = w; d.ea_out[i0 + k] = a; d.eas_out[i0 + k] = e;
+                    wput(w_out, i0 + k, w); d.ea_out[i0 + k] = a; d.eas_out[i0 + k] = e;
                 }
                 continue;
             }
@@ -240,14 +242,10 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
                     const u32 w = __shfl_down_sync(0xffffffffu, pair, 6);
                     if ((lane & 7) == 0 && live) *reinterpret_cast<uint4*>(sec + j * sb) = make_uint4(pair, y, z, w);
                 }
-            } else if (i0 + 4 <= n) {
-                reinterpret_cast<float4*>(d.w_out + i0)[0] = make_float4(ow[0], ow[1], ow[2], ow[3]);
-                reinterpret_cast<float4*>(d.ea_out + i0)[0] = make_float4(oa[0], oa[1], oa[2], oa[3]);
-                reinterpret_cast<float4*>(d.eas_out + i0)[0] = make_float4(os[0], os[1], os[2], os[3]);
             } else {
-                for (int k = 0; k < 4 && i0 + k < n; ++k) {
-                    d.w_out[i0 + k] = ow[k]; d.ea_out[i0 + k] = oa[k]; d.eas_out[i0 + k] = os[k];
-                }
+                store4(w_out, i0, n, ow);
+                store4(d.ea_out, i0, n, oa);
+                store4(d.eas_out, i0, n, os);
             }
         }
     }
@@ -255,14 +253,16 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
 }
 
 void launch_decode(const LaunchCfg& cfg, const DecDesc* descs, DecState* st, int nt, u32 tiles,
-                   const Workspace& ws, CallState* call) {
+                   const Workspace& ws, CallState* call, int wfmt) {
     dec_validate_kernel<<<nt, 64, 0, cfg.stream>>>(descs, st, call);
     if (!tiles) { prof_mark(cfg, ST_DEC_PREP, 1); return; }
     dec_popcount_kernel<<<(tiles + TPB / 32 - 1) / (TPB / 32), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws);
     dec_scan_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, ws, call);
     prof_mark(cfg, ST_DEC_PREP, 3);
     const u32 grid = min(tiles, (u32)cfg.sms * 4u);
-    decode_kernel<false><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, call);
+    if (wfmt == WF_F16) decode_kernel<false, __half><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, call);
+    else if (wfmt == WF_BF16) decode_kernel<false, __nv_bfloat16><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, call);
+    else decode_kernel<false, float><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, call);
     prof_mark(cfg, ST_DECODE, 1);
 }
 
@@ -315,7 +315,7 @@ void launch_record_to_dense(const LaunchCfg& cfg, const DecDesc* descs, DecState
     prof_mark(cfg, ST_DEC_PREP, tiles ? 4 : 2);
     if (!tiles) return;
     const u32 grid = min(tiles, (u32)cfg.sms * 8u);
-    decode_kernel<true><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, call);
+    decode_kernel<true, float><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, call);
     prof_mark(cfg, ST_DENSE, 1);
 }
 
@@ -391,6 +391,8 @@ __global__ void __launch_bounds__(TPB) dense_decode_kernel(const DecDesc* __rest
         }
         if (!st[cur].valid) continue;
         const DecDesc& d = descs[cur];
+        const float* w_prev = static_cast<const float*>(d.w_prev);
+        float* w_out = static_cast<float*>(d.w_out);
         const u64 n = d.numel;
         const u64 sb = dense_section_bytes(n, BITS);
         const unsigned char* sec = d.rec + header_bytes(KMAX);
@@ -408,7 +410,7 @@ __global__ void __launch_bounds__(TPB) dense_decode_kernel(const DecDesc* __rest
             const u32 left = n - i0 >= 4 ? 4u : (u32)(n - i0);
             if (left < 4 && ((ww | wa | we) >> (4 * left))) bad = 1;   // codes past the last element
             float wp[4];
-            load4(d.w_prev, i0, n, wp);
+            load4(w_prev, i0, n, wp);
             float ow[4], oa[4], os[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -417,15 +419,9 @@ __global__ void __launch_bounds__(TPB) dense_decode_kernel(const DecDesc* __rest
                 oa[k] = cent[1][c1];
                 os[k] = cent[2][c2];
             }
-            if (left == 4) {
-                reinterpret_cast<float4*>(d.w_out + i0)[0] = make_float4(ow[0], ow[1], ow[2], ow[3]);
-                reinterpret_cast<float4*>(d.ea_out + i0)[0] = make_float4(oa[0], oa[1], oa[2], oa[3]);
-                reinterpret_cast<float4*>(d.eas_out + i0)[0] = make_float4(os[0], os[1], os[2], os[3]);
-            } else {
-                for (u32 k = 0; k < left; ++k) {
-                    d.w_out[i0 + k] = ow[k]; d.ea_out[i0 + k] = oa[k]; d.eas_out[i0 + k] = os[k];
-                }
-            }
+            store4(w_out, i0, n, ow);
+            store4(d.ea_out, i0, n, oa);
+            store4(d.eas_out, i0, n, os);
         }
     }
     if (cur >= 0) flush(cur);

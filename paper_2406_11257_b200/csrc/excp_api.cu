@@ -160,6 +160,7 @@ Params to_params(const excp_params* params) {
     p.alpha = params->alpha; p.beta = params->beta; p.bits = params->bits;
     p.kmeans_iters = params->kmeans_iters; p.seed = params->seed; p.median_source = params->median_source;
     p.flags = params->flags;
+    p.wfmt = WF_F32;
     return p;
 }
 
@@ -320,13 +321,14 @@ excp_status excp_last_cuda_error(excp_handle h, int* cuda_err) {
     return EXCP_OK;
 }
 
-excp_status excp_compress_checkpoint(excp_handle h, const excp_params* params, size_t num_tensors,
-                                     const float* const* w_t, const float* const* w_prev,
-                                     const float* const* ea, const float* const* eas,
-                                     const size_t* numel, void* blob_out, size_t blob_capacity,
-                                     size_t* tensor_offsets_out, excp_tensor_stats* stats_out,
-                                     void* cuda_stream) {
+static excp_status compress_impl(excp_handle h, const excp_params* params, size_t num_tensors,
+                                 const void* const* w_t, const void* const* w_prev,
+                                 const float* const* ea, const float* const* eas,
+                                 const size_t* numel, int wfmt, void* blob_out, size_t blob_capacity,
+                                 size_t* tensor_offsets_out, excp_tensor_stats* stats_out,
+                                 void* cuda_stream) {
     if (!h || !params || !tensor_offsets_out) return EXCP_ERR_INVALID_ARG;
+    if (wfmt != WF_F32 && wfmt != WF_F16 && wfmt != WF_BF16) return EXCP_ERR_INVALID_ARG;
     if (num_tensors && (!w_t || !w_prev || !ea || !eas || !numel)) return EXCP_ERR_INVALID_ARG;
     if (!blob_out || !aligned16(blob_out)) return EXCP_ERR_INVALID_ARG;
     const excp_status ps = validate_params(params);
@@ -363,7 +365,8 @@ excp_status excp_compress_checkpoint(excp_handle h, const excp_params* params, s
             item += d.scan_n;
         }
     }
-    const Params p = to_params(params);
+    Params p = to_params(params);
+    p.wfmt = wfmt;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     LaunchCfg cfg{h->sms, stream, &h->prof};
     h->prof.begin(stream);
@@ -382,6 +385,28 @@ excp_status excp_compress_checkpoint(excp_handle h, const excp_params* params, s
     h->prof.finish();
     fill_outputs(h, 0, num_tensors, numel, 0, tensor_offsets_out, stats_out);
     return status_from_flags(h->h_call->flags);
+}
+
+excp_status excp_compress_checkpoint(excp_handle h, const excp_params* params, size_t num_tensors,
+                                     const float* const* w_t, const float* const* w_prev,
+                                     const float* const* ea, const float* const* eas,
+                                     const size_t* numel, void* blob_out, size_t blob_capacity,
+                                     size_t* tensor_offsets_out, excp_tensor_stats* stats_out,
+                                     void* cuda_stream) {
+    return compress_impl(h, params, num_tensors, reinterpret_cast<const void* const*>(w_t),
+                         reinterpret_cast<const void* const*>(w_prev), ea, eas, numel, WF_F32, blob_out, blob_capacity,
+                         tensor_offsets_out, stats_out, cuda_stream);
+}
+
+excp_status excp_compress_checkpoint_w16(excp_handle h, const excp_params* params, size_t num_tensors,
+                                         const void* const* w_t, const void* const* w_prev,
+                                         const float* const* ea, const float* const* eas,
+                                         const size_t* numel, int weight_format, void* blob_out, size_t blob_capacity,
+                                         size_t* tensor_offsets_out, excp_tensor_stats* stats_out,
+                                         void* cuda_stream) {
+    if (weight_format != WF_F16 && weight_format != WF_BF16) return EXCP_ERR_INVALID_ARG;
+    return compress_impl(h, params, num_tensors, w_t, w_prev, ea, eas, numel, weight_format, blob_out, blob_capacity,
+                         tensor_offsets_out, stats_out, cuda_stream);
 }
 
 excp_status excp_compress_checkpoint_host(excp_handle h, const excp_params* params, size_t num_tensors,
@@ -498,10 +523,10 @@ excp_status excp_compress_tensor(excp_handle h, const excp_params* params,
     return s;
 }
 
-excp_status excp_decompress_checkpoint(excp_handle h, const void* blob, const size_t* tensor_offsets,
-                                       size_t num_tensors, const float* const* w_prev, const size_t* numel,
-                                       float* const* w_out, float* const* ea_out, float* const* eas_out,
-                                       void* cuda_stream) {
+static excp_status decompress_impl(excp_handle h, const void* blob, const size_t* tensor_offsets,
+                                   size_t num_tensors, const void* const* w_prev, const size_t* numel, int wfmt,
+                                   void* const* w_out, float* const* ea_out, float* const* eas_out,
+                                   void* cuda_stream) {
     if (!h || !blob || !tensor_offsets || !aligned16(blob)) return EXCP_ERR_INVALID_ARG;
     if (num_tensors == 0) return EXCP_OK;
     if (!w_prev || !numel || !w_out || !ea_out || !eas_out) return EXCP_ERR_INVALID_ARG;
@@ -541,13 +566,30 @@ excp_status excp_decompress_checkpoint(excp_handle h, const void* blob, const si
     ok = ok && check(h, cudaMemcpyAsync(dd, hd, num_tensors * sizeof(DecDesc), cudaMemcpyHostToDevice, stream));
     for (size_t gi = 0; ok && gi < groups.size(); ++gi) {
         const Group& g = groups[gi];
-        launch_decode(cfg, dd + g.first, h->d_dstate, (int)g.count, g.tiles, h->ws, h->d_call);
+        launch_decode(cfg, dd + g.first, h->d_dstate, (int)g.count, g.tiles, h->ws, h->d_call, wfmt);
         ok = check(h, cudaGetLastError());
     }
     ok = ok && check(h, cudaMemcpyAsync(h->h_call, h->d_call, sizeof(CallState), cudaMemcpyDeviceToHost, stream));
     if (!check(h, cudaStreamSynchronize(stream)) || !ok) return EXCP_ERR_CUDA;
     h->prof.finish();
     return status_from_flags(h->h_call->flags);
+}
+
+excp_status excp_decompress_checkpoint(excp_handle h, const void* blob, const size_t* tensor_offsets,
+                                       size_t num_tensors, const float* const* w_prev, const size_t* numel,
+                                       float* const* w_out, float* const* ea_out, float* const* eas_out,
+                                       void* cuda_stream) {
+    return decompress_impl(h, blob, tensor_offsets, num_tensors, reinterpret_cast<const void* const*>(w_prev), numel,
+                           WF_F32, reinterpret_cast<void* const*>(w_out), ea_out, eas_out, cuda_stream);
+}
+
+excp_status excp_decompress_checkpoint_w16(excp_handle h, const void* blob, const size_t* tensor_offsets,
+                                           size_t num_tensors, const void* const* w_prev, const size_t* numel,
+                                           int weight_format, void* const* w_out, float* const* ea_out,
+                                           float* const* eas_out, void* cuda_stream) {
+    if (weight_format != WF_F16 && weight_format != WF_BF16) return EXCP_ERR_INVALID_ARG;
+    return decompress_impl(h, blob, tensor_offsets, num_tensors, w_prev, numel, weight_format, w_out, ea_out, eas_out,
+                           cuda_stream);
 }
 
 excp_status excp_profile_enable(excp_handle h, int enable) {

@@ -2,6 +2,8 @@
 // records, small device helpers, and the launch wrappers each .cu file exports.
 #pragma once
 #include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <cuda_bf16.h>
 #include <stdint.h>
 
 namespace excp {
@@ -53,9 +55,12 @@ constexpr u32 DENSE_MAGIC = 0x44435845u;         // "EXCD": one code per element
 constexpr u32 VERSION = 1u;
 constexpr int HEADER_FIXED = 64;
 
+// Storage format of the weight tensors (W_t, W^_(t-1), W^_t); the moments are always fp32.
+enum WeightFormat { WF_F32 = 0, WF_F16 = 1, WF_BF16 = 2 };
+
 struct TensorDesc {              // built on the host, one per tensor of a group
-    const float* w_t;
-    const float* w_prev;
+    const void* w_t;             // fp32, fp16 or bf16 (the call's weight format)
+    const void* w_prev;
     const float* ea;
     const float* eas;
     u64 numel;
@@ -157,6 +162,7 @@ struct Params {
     u64 seed;
     int median_source;
     u32 flags;                   // OPT_*
+    int wfmt;                    // WeightFormat of w_t and w_prev
 };
 __host__ __device__ inline int stored_bits(const Params& p) { return (p.flags & OPT_NO_QUANT) ? 32 : p.bits; }
 __host__ __device__ inline u32 record_flags(const Params& p) {
@@ -167,8 +173,8 @@ __host__ __device__ inline u32 record_flags(const Params& p) {
 struct DecDesc {                 // decompress: one per tensor of a group
     const unsigned char* rec;    // start of the record
     u64 rec_avail;               // bytes the caller says belong to it
-    const float* w_prev;
-    float* w_out;
+    const void* w_prev;          // fp32, fp16 or bf16 (the call's weight format), like w_out
+    void* w_out;
     float* ea_out;
     float* eas_out;
     u64 numel;
@@ -234,6 +240,50 @@ __device__ inline int find_tensor(const DecDesc* __restrict__ descs, int n, u32 
         if (descs[mid].tile_begin <= tile) lo = mid; else hi = mid - 1;
     }
     return lo;
+}
+
+// A stored weight as fp32 (exact: both 16-bit formats are subsets of fp32), and back (round to
+// nearest even).
+__device__ __forceinline__ float wget(const float* p, u64 i) { return p[i]; }
+__device__ __forceinline__ float wget(const __half* p, u64 i) { return __half2float(p[i]); }
+__device__ __forceinline__ float wget(const __nv_bfloat16* p, u64 i) { return __bfloat162float(p[i]); }
+__device__ __forceinline__ void wput(float* p, u64 i, float v) { p[i] = v; }
+__device__ __forceinline__ void wput(__half* p, u64 i, float v) { p[i] = __float2half_rn(v); }
+__device__ __forceinline__ void wput(__nv_bfloat16* p, u64 i, float v) { p[i] = __float2bfloat16_rn(v); }
+
+// Four consecutive 16-bit weights at i0 (a multiple of 4) as fp32; as load4 below.
+template <typename WT>
+__device__ inline int load4(const WT* __restrict__ p, u64 i0, u64 n, float v[4]) {
+    if (i0 + 4 <= n) {
+        const uint2 t = __ldcs(reinterpret_cast<const uint2*>(p + i0));
+        const WT* h = reinterpret_cast<const WT*>(&t);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) v[k] = wget(h, k);
+        return 4;
+    }
+    int c = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        if (i0 + k < n) { v[k] = wget(p, i0 + k); c = k + 1; } else v[k] = 0.f;
+    }
+    return c;
+}
+// Four results to weights i0..i0+3 (those that exist).
+__device__ inline void store4(float* p, u64 i0, u64 n, const float v[4]) {
+    if (i0 + 4 <= n) { *reinterpret_cast<float4*>(p + i0) = make_float4(v[0], v[1], v[2], v[3]); return; }
+    for (int k = 0; k < 4 && i0 + k < n; ++k) p[i0 + k] = v[k];
+}
+template <typename WT>
+__device__ inline void store4(WT* p, u64 i0, u64 n, const float v[4]) {
+    if (i0 + 4 <= n) {
+        uint2 t;
+        WT* h = reinterpret_cast<WT*>(&t);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) wput(h, k, v[k]);
+        *reinterpret_cast<uint2*>(p + i0) = t;
+        return;
+    }
+    for (int k = 0; k < 4 && i0 + k < n; ++k) wput(p, i0 + k, v[k]);
 }
 
 // Four consecutive elements starting at i0 (a multiple of 4).  Elements at or
@@ -328,7 +378,7 @@ void launch_pack(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int
                  const Workspace& ws, const Params& p, unsigned char* blob, CallState* call,
                  TensorResult* results);
 void launch_decode(const LaunchCfg&, const DecDesc* descs, DecState* st, int nt, u32 tiles,
-                   const Workspace& ws, CallState* call);
+                   const Workspace& ws, CallState* call, int wfmt = WF_F32);
 void launch_record_to_dense(const LaunchCfg&, const DecDesc* descs, DecState* st, int nt, u32 tiles,
                             const Workspace& ws, CallState* call);
 void launch_dense_decode(const LaunchCfg&, const DecDesc* descs, DecState* st, int nt, u32 tiles,

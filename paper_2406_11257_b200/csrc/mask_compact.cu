@@ -28,7 +28,7 @@ struct MaskSmem {
 // warp, and nothing in the sweep synchronises the block.
 // VARIANT = false is the method; VARIANT = true adds the ablation switches `opt` (OPT_*), kept
 // out of the method's own instruction stream.
-template <bool VARIANT>
+template <bool VARIANT, typename WT>
 __global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc* __restrict__ descs,
                                                               TensorState* __restrict__ st, int nt,
                                                               u32 tiles, Workspace ws, CallState* call, u32 opt) {
@@ -43,8 +43,11 @@ __global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc*
     const u32 wlo = (u32)(((u64)tiles * gw) / nw), whi = (u32)(((u64)tiles * (gw + 1)) / nw);
     TileWalk<MCH> ic, cc;
     ic.start(wlo); cc.start(wlo);
-    const float* ip[4] = {nullptr, nullptr, nullptr, nullptr};      // issue side: the tensor's streams
+    constexpr u32 BULK_ALIGN = sizeof(WT) == 4 ? 4u : 8u;           // values per bulk-copied unit: 16 bytes of the narrowest stream
+    const float* ip[4] = {nullptr, nullptr, nullptr, nullptr};      // issue side: the tensor's moment streams ([2], [3])
     const float* cp[4] = {nullptr, nullptr, nullptr, nullptr};      // consume side
+    const WT* ipw[2] = {nullptr, nullptr};                          // and its weight streams W_t, W^_(t-1)
+    const WT* cpw[2] = {nullptr, nullptr};
     float thr_w = 0.f, thr_o = 0.f;
     u32 rw = 0, ro = 0;               // survivors of the current tile so far (warp uniform)
     float mk0 = 0.f, mk1 = 0.f, mk2 = 0.f;   // running max magnitudes of the survivors
@@ -67,23 +70,25 @@ __global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc*
     while (cc.tile < whi) {
         while (ic.tile < whi && ring.can_issue()) {
             if (ic.chunk == 0 && ic.enter_tile(descs, nt)) {
-                ip[0] = descs[ic.tns].w_t; ip[1] = descs[ic.tns].w_prev;
+                ipw[0] = static_cast<const WT*>(descs[ic.tns].w_t); ipw[1] = static_cast<const WT*>(descs[ic.tns].w_prev);
                 ip[2] = descs[ic.tns].ea; ip[3] = descs[ic.tns].eas;
-                if (VARIANT && (opt & OPT_NO_RESIDUAL)) ip[1] = nullptr;     // W^_(t-1) is not read
+                if (VARIANT && (opt & OPT_NO_RESIDUAL)) ipw[1] = nullptr;    // W^_(t-1) is not read
             }
             const u64 e0 = ic.elem0();
-            const float* src[4] = {ip[0] + e0, VARIANT && !ip[1] ? nullptr : ip[1] + e0, ip[2] + e0, ip[3] + e0};
-            ring.issue(lane, src, ic.valid() & ~3u);
+            const void* src[4] = {ipw[0] + e0, VARIANT && !ipw[1] ? nullptr : ipw[1] + e0, ip[2] + e0, ip[3] + e0};
+            const u32 nb = ic.valid() & ~(BULK_ALIGN - 1u);
+            const u32 bytes[4] = {nb * (u32)sizeof(WT), nb * (u32)sizeof(WT), nb * 4u, nb * 4u};
+            ring.issue_bytes(lane, src, bytes);
             ic.next();
         }
         if (cc.chunk == 0 && cc.enter_tile(descs, nt)) {
             if (prev >= 0) flush_max(prev);
             prev = cc.tns;
-            cp[0] = descs[cc.tns].w_t; cp[1] = descs[cc.tns].w_prev;
+            cpw[0] = static_cast<const WT*>(descs[cc.tns].w_t); cpw[1] = static_cast<const WT*>(descs[cc.tns].w_prev);
             cp[2] = descs[cc.tns].ea; cp[3] = descs[cc.tns].eas;
             thr_w = st[cc.tns].thr_w; thr_o = st[cc.tns].thr_o;
         }
-        const u32 valid = cc.valid(), nbulk = valid & ~3u;
+        const u32 valid = cc.valid(), nbulk = valid & ~(BULK_ALIGN - 1u);
         const u64 e0 = cc.elem0();
         if (!ring.wait()) {
             if (lane == 0) atomicOr(&call->flags, FLAG_TIMEOUT);
@@ -91,6 +96,8 @@ __global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc*
         }
         if (cc.chunk == 0) { rw = 0; ro = 0; }
         const float* stg = ring.stage();
+        const WT* stw = reinterpret_cast<const WT*>(stg);              // W_t's slot; W^_(t-1)'s starts MCH floats on
+        const WT* stp = reinterpret_cast<const WT*>(stg + MCH);
         float* sw = ws.surv[0] + (u64)cc.tile * TILE;
         float* sea = ws.surv[1] + (u64)cc.tile * TILE;
         float* seas = ws.surv[2] + (u64)cc.tile * TILE;
@@ -109,9 +116,9 @@ __global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc*
                     float a, b, e, v;
                     const bool no_prev = VARIANT && (opt & OPT_NO_RESIDUAL);
                     if (FULL || i < nbulk) {
-                        a = stg[i]; b = no_prev ? 0.f : stg[MCH + i]; e = stg[2 * MCH + i]; v = stg[3 * MCH + i];
+                        a = wget(stw, i); b = no_prev ? 0.f : wget(stp, i); e = stg[2 * MCH + i]; v = stg[3 * MCH + i];
                     } else if (i < valid) {          // ragged last values of a tensor
-                        a = __ldg(cp[0] + e0 + i); b = no_prev ? 0.f : __ldg(cp[1] + e0 + i);
+                        a = wget(cpw[0], e0 + i); b = no_prev ? 0.f : wget(cpw[1], e0 + i);
                         e = __ldg(cp[2] + e0 + i); v = __ldg(cp[3] + e0 + i);
                     } else {
                         a = b = e = v = 0.f;
@@ -235,10 +242,16 @@ void launch_mask_compact(const LaunchCfg& cfg, const TensorDesc* descs, TensorSt
     if (tiles) {
         const u32 grid = min((tiles + MWARPS - 1) / MWARPS, (u32)cfg.sms * 2u);
         const u32 opt = p.flags & (OPT_NO_W2M | OPT_NO_M2W | OPT_NO_RESIDUAL | OPT_NO_PRUNE);
-        cudaFuncSetAttribute(mask_compact_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(MaskSmem));
-        cudaFuncSetAttribute(mask_compact_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(MaskSmem));
-        if (opt) mask_compact_kernel<true><<<grid, MTPB, sizeof(MaskSmem), cfg.stream>>>(descs, st, nt, tiles, ws, call, opt);
-        else mask_compact_kernel<false><<<grid, MTPB, sizeof(MaskSmem), cfg.stream>>>(descs, st, nt, tiles, ws, call, 0u);
+        auto run = [&](auto tag) {
+            using WT = decltype(tag);
+            cudaFuncSetAttribute(mask_compact_kernel<false, WT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(MaskSmem));
+            cudaFuncSetAttribute(mask_compact_kernel<true, WT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(MaskSmem));
+            if (opt) mask_compact_kernel<true, WT><<<grid, MTPB, sizeof(MaskSmem), cfg.stream>>>(descs, st, nt, tiles, ws, call, opt);
+            else mask_compact_kernel<false, WT><<<grid, MTPB, sizeof(MaskSmem), cfg.stream>>>(descs, st, nt, tiles, ws, call, 0u);
+        };
+        if (p.wfmt == WF_F16) run(__half{});
+        else if (p.wfmt == WF_BF16) run(__nv_bfloat16{});
+        else run(float{});
         prof_mark(cfg, ST_MASK_COMPACT, 1);
     }
     tile_scan_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, ws);

@@ -74,6 +74,7 @@ __device__ void find_rank_block(const u32* hist, u32 k, u32& bin, u32& rank_in, 
 // ---------------------------------------------------------------------------
 // Histogram path, sweep 1: top 13 key bits, per block in shared memory, merged with integer
 // atomics.  Only tensors flagged need_hist.
+template <typename WT>
 __global__ void __launch_bounds__(TPB) hist1_kernel(const TensorDesc* __restrict__ descs,
                                                     TensorState* __restrict__ st, int nt, u32 tiles,
                                                     int residual_median) {
@@ -87,7 +88,7 @@ __global__ void __launch_bounds__(TPB) hist1_kernel(const TensorDesc* __restrict
     u32 tb = 0, ntl = 0;
     u64 n = 0;
     bool active = false;
-    const float *w_t = nullptr, *w_prev = nullptr;
+    const WT *w_t = nullptr, *w_prev = nullptr;
     auto flush_hist = [&](int t) {
         __syncthreads();
         for (int i = tid; i < HIST1_BINS; i += TPB) {
@@ -101,7 +102,7 @@ __global__ void __launch_bounds__(TPB) hist1_kernel(const TensorDesc* __restrict
             if (cur >= 0 && active) flush_hist(cur);
             cur = find_tensor(descs, nt, tile);
             tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles; n = descs[cur].numel;
-            w_t = descs[cur].w_t; w_prev = descs[cur].w_prev;
+            w_t = static_cast<const WT*>(descs[cur].w_t); w_prev = static_cast<const WT*>(descs[cur].w_prev);
             active = st[cur].need_hist != 0;
             if (!active) tile = tb + ntl - 1;          // nothing to do for this tensor
         }
@@ -196,6 +197,7 @@ __global__ void __launch_bounds__(TPB) hist1_finish_kernel(const TensorDesc* __r
 // ---------------------------------------------------------------------------
 // Histogram path, sweep 2: keys of the selected bin -> candidate list (kept in the tensor's own
 // survivor segment, which the mask sweep overwrites afterwards).  Only flagged tensors.
+template <typename WT>
 __global__ void __launch_bounds__(TPB) hist2_kernel(const TensorDesc* __restrict__ descs,
                                                      TensorState* __restrict__ st, int nt, u32 tiles,
                                                      Workspace ws, int residual_median) {
@@ -206,13 +208,13 @@ __global__ void __launch_bounds__(TPB) hist2_kernel(const TensorDesc* __restrict
     u32 tb = 0, ntl = 0, bin1 = 0;
     u64 n = 0;
     bool active = false;
-    const float *w_t = nullptr, *w_prev = nullptr;
+    const WT *w_t = nullptr, *w_prev = nullptr;
     u32* cand = nullptr;
     for (u32 tile = lo; tile < hi; ++tile) {
         if (cur < 0 || tile >= tb + ntl) {
             cur = find_tensor(descs, nt, tile);
             tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles; n = descs[cur].numel;
-            w_t = descs[cur].w_t; w_prev = descs[cur].w_prev;
+            w_t = static_cast<const WT*>(descs[cur].w_t); w_prev = static_cast<const WT*>(descs[cur].w_prev);
             bin1 = st[cur].bin1;
             cand = reinterpret_cast<u32*>(ws.surv[0] + (u64)tb * TILE);
             active = st[cur].need_hist != 0;
@@ -323,6 +325,7 @@ constexpr u32 MEDIAN_MARGIN = MEDIAN_SAMPLE / 80;   // +-1.25 % of the sample: a
 
 // One block per tensor.  The sample's keys go to the tensor's second survivor segment (free
 // until the mask sweep); a tensor no larger than the sample gets its exact median here.
+template <typename WT>
 __global__ void __launch_bounds__(1024) median_sample_kernel(const TensorDesc* __restrict__ descs,
                                                              TensorState* __restrict__ st, Workspace ws,
                                                              int residual_median) {
@@ -340,12 +343,12 @@ __global__ void __launch_bounds__(1024) median_sample_kernel(const TensorDesc* _
     u32 kmin = 0xffffffffu, kmax = 0;
     const u32 m = (u32)min((u64)MEDIAN_SAMPLE, n);
     u32* keys = reinterpret_cast<u32*>(ws.surv[1] + (u64)descs[t].tile_begin * TILE);
-    const float* w_t = descs[t].w_t;
-    const float* w_prev = descs[t].w_prev;
+    const WT* w_t = static_cast<const WT*>(descs[t].w_t);
+    const WT* w_prev = static_cast<const WT*>(descs[t].w_prev);
     for (u32 j = tid; j < m; j += 1024) {
         const u64 i = ((u64)j * n) / m;
-        float a = w_t[i];
-        if (residual_median) a = __fsub_rn(a, w_prev[i]);
+        float a = wget(w_t, i);
+        if (residual_median) a = __fsub_rn(a, wget(w_prev, i));
         const u32 key = __float_as_uint(a) & 0x7fffffffu;
         keys[j] = key;
         kmin = min(kmin, key);
@@ -381,6 +384,7 @@ struct SweepSmem {
     u32 q[SWARPS][QCAP][32];         // per-lane queues of bracket keys waiting for their place in the tensor's list
 };
 
+template <typename WT>
 __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* __restrict__ descs,
                                                              TensorState* __restrict__ st, int nt, u32 tiles,
                                                              Workspace ws, int residual_median, CallState* call) {
@@ -393,8 +397,11 @@ __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* _
     const u32 wlo = (u32)(((u64)tiles * gw) / nw), whi = (u32)(((u64)tiles * (gw + 1)) / nw);
     TileWalk<SCH> ic, cc;
     ic.start(wlo); cc.start(wlo);
-    const float* ip[3] = {nullptr, nullptr, nullptr};
-    const float* cp[3] = {nullptr, nullptr, nullptr};
+    constexpr u32 WPER = 16 / sizeof(WT);      // weights per 16 bytes: a bulk copy moves whole 16-byte units
+    const WT* iw[2] = {nullptr, nullptr};      // issue side: the weight streams, and ea
+    const float* iea = nullptr;
+    const WT* cw[2] = {nullptr, nullptr};      // consume side
+    const float* cea = nullptr;
     u32 lo_key = 0, span = 0;        // bracket [lo_key, lo_key + span]
     bool want_median = false;
     u32* cand = nullptr;
@@ -438,32 +445,48 @@ __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* _
     while (cc.tile < whi) {
         while (ic.tile < whi && ring.can_issue()) {
             if (ic.chunk == 0 && ic.enter_tile(descs, nt)) {
-                ip[0] = descs[ic.tns].w_t;
-                ip[1] = residual_median ? descs[ic.tns].w_prev : nullptr;
-                ip[2] = descs[ic.tns].ea;
+                iw[0] = static_cast<const WT*>(descs[ic.tns].w_t);
+                iw[1] = residual_median ? static_cast<const WT*>(descs[ic.tns].w_prev) : nullptr;
+                iea = descs[ic.tns].ea;
             }
             const u64 e0 = ic.elem0();
-            const float* src[3] = {ip[0] + e0, ip[1] ? ip[1] + e0 : nullptr, ip[2] + e0};
-            ring.issue(lane, src, ic.valid() & ~3u);
+            const void* src[3] = {iw[0] + e0, iw[1] ? iw[1] + e0 : nullptr, iea + e0};
+            const u32 v = ic.valid();
+            const u32 wb = (v & ~(WPER - 1u)) * (u32)sizeof(WT);
+            const u32 bytes[3] = {wb, wb, (v & ~3u) * 4u};
+            ring.issue_bytes(lane, src, bytes);
             ic.next();
         }
         if (cc.chunk == 0 && cc.enter_tile(descs, nt)) {
             if (prev >= 0) { flush_acc(prev); flush_below(prev); flush_cand(prev); }
             prev = cc.tns;
             ecur = 1;
-            cp[0] = descs[cc.tns].w_t; cp[1] = descs[cc.tns].w_prev; cp[2] = descs[cc.tns].ea;
+            cw[0] = static_cast<const WT*>(descs[cc.tns].w_t); cw[1] = static_cast<const WT*>(descs[cc.tns].w_prev);
+            cea = descs[cc.tns].ea;
             want_median = st[cc.tns].med_done == 0;
             lo_key = st[cc.tns].lo_key;
             span = st[cc.tns].hi_key - lo_key;
             cand = reinterpret_cast<u32*>(ws.surv[0] + (u64)cc.tb * TILE);
         }
-        const u32 valid = cc.valid(), nbulk = valid & ~3u;
+        const u32 valid = cc.valid(), nbulk = valid & ~3u, nbulk_w = valid & ~(WPER - 1u);
         const u64 e0 = cc.elem0();
         if (!ring.wait()) {
             if (lane == 0) atomicOr(&call->flags, FLAG_TIMEOUT);
             return;
         }
         const float* stg = ring.stage();
+        auto weights4 = [&](int k, u32 o, bool full, float out[4]) {     // four weights of stream k at offset o
+            if constexpr (sizeof(WT) == 4) {
+                if (full) {
+                    const float4 t = *reinterpret_cast<const float4*>(stg + k * SCH + o);
+                    out[0] = t.x; out[1] = t.y; out[2] = t.z; out[3] = t.w;
+                } else {
+                    fetch4(stg + k * SCH, reinterpret_cast<const float*>(cw[k]) + e0, o, nbulk, valid, out);
+                }
+            } else {
+                fetch4w<WT>(stg + k * SCH, cw[k] + e0, o, full ? (u32)SCH : nbulk_w, valid, out);
+            }
+        };
         u32 ke[SCH / 32];
         u32 kmax = 0;
         auto sweep_chunk = [&](auto full_tag) {
@@ -479,22 +502,12 @@ __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* _
                         const float4 t = *reinterpret_cast<const float4*>(stg + 2 * SCH + o);
                         e[0] = t.x; e[1] = t.y; e[2] = t.z; e[3] = t.w;
                     } else {
-                        fetch4(stg + 2 * SCH, cp[2] + e0, o, nbulk, valid, e);
+                        fetch4(stg + 2 * SCH, cea + e0, o, nbulk, valid, e);
                     }
                     if (want_median) {
-                        if (FULL) {
-                            const float4 t = *reinterpret_cast<const float4*>(stg + o);
-                            a[0] = t.x; a[1] = t.y; a[2] = t.z; a[3] = t.w;
-                        } else {
-                            fetch4(stg, cp[0] + e0, o, nbulk, valid, a);
-                        }
+                        weights4(0, o, FULL, a);
                         if (residual_median) {
-                            if (FULL) {
-                                const float4 t = *reinterpret_cast<const float4*>(stg + SCH + o);
-                                b[0] = t.x; b[1] = t.y; b[2] = t.z; b[3] = t.w;
-                            } else {
-                                fetch4(stg + SCH, cp[1] + e0, o, nbulk, valid, b);
-                            }
+                            weights4(1, o, FULL, b);
 #pragma unroll
                             for (int k = 0; k < 4; ++k) a[k] = __fsub_rn(a[k], b[k]);
                         }
@@ -654,24 +667,30 @@ void launch_stats(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st
                   const Workspace& ws, const Params& p, CallState* call) {
     const int resid = p.median_source == 1 && !(p.flags & OPT_NO_RESIDUAL);   // without the residual dW is W_t
     const float alpha = (p.flags & OPT_NO_M2W) ? -p.alpha : p.alpha;          // see weight_threshold
-    median_sample_kernel<<<nt, 1024, 0, cfg.stream>>>(descs, st, ws, resid);
-    if (tiles) {
-        const u32 grid = min((tiles + SWARPS - 1) / SWARPS, (u32)cfg.sms * 2u);
-        cudaFuncSetAttribute(stats_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SweepSmem));
-        stats_sweep_kernel<<<grid, TPB, sizeof(SweepSmem), cfg.stream>>>(descs, st, nt, tiles, ws, resid, call);
-    }
-    stats_finish_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, alpha, p.beta);
-    if (tiles)
-        for (int pass = 0; pass < 4; ++pass)
-            median_digit_kernel<<<dim3(SEL_SLICES, nt), TPB, 0, cfg.stream>>>(st, descs, ws, pass, alpha);
-    prof_mark(cfg, ST_STATS1, tiles ? 7 : 2);
-    if (tiles) {          // the histogram path: returns at once unless a bracket missed
-        hist1_kernel<<<min(tiles, (u32)cfg.sms * 4u), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, resid);
-        hist1_finish_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st);
-        hist2_kernel<<<min(tiles, (u32)cfg.sms * 8u), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, resid);
-        hist2_finish_kernel<<<nt, 1024, 0, cfg.stream>>>(descs, st, ws, alpha);
-        prof_mark(cfg, ST_STATS2, 4);
-    }
+    auto run = [&](auto tag) {
+        using WT = decltype(tag);
+        median_sample_kernel<WT><<<nt, 1024, 0, cfg.stream>>>(descs, st, ws, resid);
+        if (tiles) {
+            const u32 grid = min((tiles + SWARPS - 1) / SWARPS, (u32)cfg.sms * 2u);
+            cudaFuncSetAttribute(stats_sweep_kernel<WT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SweepSmem));
+            stats_sweep_kernel<WT><<<grid, TPB, sizeof(SweepSmem), cfg.stream>>>(descs, st, nt, tiles, ws, resid, call);
+        }
+        stats_finish_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, alpha, p.beta);
+        if (tiles)
+            for (int pass = 0; pass < 4; ++pass)
+                median_digit_kernel<<<dim3(SEL_SLICES, nt), TPB, 0, cfg.stream>>>(st, descs, ws, pass, alpha);
+        prof_mark(cfg, ST_STATS1, tiles ? 7 : 2);
+        if (tiles) {          // the histogram path: returns at once unless a bracket missed
+            hist1_kernel<WT><<<min(tiles, (u32)cfg.sms * 4u), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, resid);
+            hist1_finish_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st);
+            hist2_kernel<WT><<<min(tiles, (u32)cfg.sms * 8u), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, resid);
+            hist2_finish_kernel<<<nt, 1024, 0, cfg.stream>>>(descs, st, ws, alpha);
+            prof_mark(cfg, ST_STATS2, 4);
+        }
+    };
+    if (p.wfmt == WF_F16) run(__half{});
+    else if (p.wfmt == WF_BF16) run(__nv_bfloat16{});
+    else run(float{});
 }
 
 }  // namespace excp

@@ -32,26 +32,35 @@ struct WarpRing {
     }
     __device__ bool can_issue() const { return inflight < (u32)ST; }
 
-    // Starts the copies of one chunk: `nbulk` values (a multiple of 4, possibly 0) from each
-    // non-null source.  Called by the whole warp; lane 0 talks to the copy engine.
-    __device__ void issue(int lane, const float* const (&src)[NS], u32 nbulk) {
+    // Starts the copies of one chunk: bytes[k] bytes (a multiple of 16, possibly 0) from each
+    // non-null source into stream k's slot of the stage.  Called by the whole warp; lane 0 talks
+    // to the copy engine.
+    __device__ void issue_bytes(int lane, const void* const (&src)[NS], const u32 (&bytes)[NS]) {
         if (lane == 0) {
             unsigned long long* b = &bar[i_stage];
             float* dst = buf + i_stage * STAGE_FLOATS;
-            u32 n = 0;
+            u32 total = 0;
 #pragma unroll
-            for (int k = 0; k < NS; ++k) n += src[k] != nullptr;
-            if (nbulk && n) {
-                mbar_arrive_expect_tx(b, n * nbulk * 4u);
+            for (int k = 0; k < NS; ++k) total += src[k] != nullptr ? bytes[k] : 0u;
+            if (total) {
+                mbar_arrive_expect_tx(b, total);
 #pragma unroll
                 for (int k = 0; k < NS; ++k)
-                    if (src[k]) bulk_g2s(dst + k * CH, src[k], nbulk * 4u, b);
+                    if (src[k] && bytes[k]) bulk_g2s(dst + k * CH, src[k], bytes[k], b);
             } else {
                 mbar_arrive(b);
             }
         }
         i_stage = i_stage + 1 == (u32)ST ? 0u : i_stage + 1;
         ++inflight;
+    }
+    // The same for fp32 streams: `nbulk` values (a multiple of 4, possibly 0) from each source.
+    __device__ void issue(int lane, const float* const (&src)[NS], u32 nbulk) {
+        const void* vs[NS];
+        u32 bytes[NS];
+#pragma unroll
+        for (int k = 0; k < NS; ++k) { vs[k] = src[k]; bytes[k] = nbulk * 4u; }
+        issue_bytes(lane, vs, bytes);
     }
     // Blocks (bounded) until the oldest chunk in flight has landed.
     __device__ bool wait() { return mbar_wait_warp(&bar[c_stage], c_phase); }
@@ -99,6 +108,23 @@ struct TileWalk {
 
 // Four consecutive values at offset o (a multiple of 4) of a chunk: from the stage where the
 // bulk copy brought them, from global memory for the ragged last values of a tensor, 0 past it.
+template <typename WT>
+__device__ __forceinline__ void fetch4w(const float* __restrict__ slot, const WT* __restrict__ g, u32 o,
+                                        u32 nbulk, u32 valid, float out[4]) {
+    const WT* st = reinterpret_cast<const WT*>(slot);     // a 16-bit stream fills the first half of its slot
+    if (o + 4 <= nbulk) {
+        const uint2 t = *reinterpret_cast<const uint2*>(st + o);
+        const WT* h = reinterpret_cast<const WT*>(&t);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) out[k] = wget(h, k);
+    } else {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const u32 i = o + k;
+            out[k] = i < nbulk ? wget(st, i) : (i < valid ? wget(g, i) : 0.f);
+        }
+    }
+}
 __device__ __forceinline__ void fetch4(const float* __restrict__ st, const float* __restrict__ g, u32 o,
                                        u32 nbulk, u32 valid, float out[4]) {
     if (o + 4 <= nbulk) {
