@@ -101,29 +101,59 @@ __global__ void __launch_bounds__(TPB) dec_scan_kernel(const DecDesc* __restrict
     }
 }
 
-// DENSE = false: Algorithm 2, fp32 outputs.  DENSE = true: the same walk writes each element's
-// code (0 where pruned) into the three sections of the dense layout instead.
+// DENSE = false: Algorithm 2.  DENSE = true: the same walk writes each element's code (0 where
+// pruned) into the three sections of the dense layout instead.
+//
+// Warps are autonomous: a warp owns a contiguous run of tiles and nothing synchronises the block.
+// Per tile the warp loads the 2 x 128 bitmap words, turns their populations into the rank of
+// every word's first survivor (registers and shuffles), parks words and ranks in its own corner
+// of shared memory, and then walks the tile in 32 rounds of 128 elements, lane l taking four
+// consecutive elements: their survivors have consecutive ranks, so their codes are consecutive
+// bits of the section and one 32-bit window per stream (two aligned words read through the
+// cache) holds all four.
+constexpr int DEC_WARPS = TPB / 32;
+
+struct DecodeSmem {
+    u32 bw[DEC_WARPS][TILE_WORDS], bo[DEC_WARPS][TILE_WORDS];   // the tile's bitmap words
+    u32 pw[DEC_WARPS][TILE_WORDS], po[DEC_WARPS][TILE_WORDS];   // survivors of the tile before each word
+    float cent[DEC_WARPS][3][KCAP];
+};
+
+// The `nb`-bit codes of up to four consecutive survivors starting at rank g of a section:
+// bits [g * nb, g * nb + 32) of it.  Words are read only where codes of these `have` survivors lie.
+__device__ __forceinline__ u32 code_window(const u32* __restrict__ sec, u64 g, u32 nb, u32 have) {
+    if (!have) return 0u;
+    const u64 bit = g * nb;
+    const u32 sh = (u32)bit & 31u;
+    const u32 lo = __ldg(sec + (bit >> 5));
+    const u32 hi = sh + have * nb > 32u ? __ldg(sec + (bit >> 5) + 1) : 0u;
+    return __funnelshift_r(lo, hi, sh);
+}
+
 template <bool DENSE, typename WT>
 __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__ descs,
                                                      const DecState* __restrict__ st, int nt, u32 tiles,
                                                      Workspace ws, CallState* call) {
-    __shared__ u32 bw[TILE_WORDS], bo[TILE_WORDS];
-    __shared__ u32 pw[TILE_WORDS], po[TILE_WORDS];        // survivors before each word, within the tile
-    __shared__ u32 wsum[2][TILE_WORDS / 32];
-    __shared__ u32 codes[3][TILE / 4 + 4];                // the tile's code words (8 bits each at most; + slack, + one zero word)
-    __shared__ float cent[3][KCAP];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    u32 lo, hi;
-    block_range(tiles, lo, hi);
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    DecodeSmem& sm = *reinterpret_cast<DecodeSmem*>(smem_raw);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const u32 gw = blockIdx.x * DEC_WARPS + warp, nw = gridDim.x * DEC_WARPS;
+    const u32 wlo = (u32)(((u64)tiles * gw) / nw), whi = (u32)(((u64)tiles * (gw + 1)) / nw);
+    u32* bw = sm.bw[warp]; u32* bo = sm.bo[warp]; u32* pw = sm.pw[warp]; u32* po = sm.po[warp];
+    float (*cent)[KCAP] = sm.cent[warp];
     int cur = -1;
     u32 tb = 0, ntl = 0;
     u32 bad = 0;
-    for (u32 tile = lo; tile < hi; ++tile) {
-        __syncthreads();                                  // previous tile fully consumed
+    for (u32 tile = wlo; tile < whi; ++tile) {
         if (cur < 0 || tile >= tb + ntl) {
             cur = find_tensor(descs, nt, tile);
             tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
-            for (int i = tid; i < 3 * KCAP; i += TPB) cent[i / KCAP][i % KCAP] = st[cur].cent[i / KCAP][i % KCAP];
+            __syncwarp();
+            if (st[cur].valid) {
+                const int kc = centres_of((int)st[cur].bits);
+                for (int i = lane; i < 3 * kc; i += 32) cent[i / kc][i % kc] = st[cur].cent[i / kc][i % kc];
+            }
+            __syncwarp();
         }
         if (!st[cur].valid) continue;
         const DecDesc& d = descs[cur];
@@ -133,99 +163,83 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
         const u64 n = d.numel;
         const u64 nwords = bitmap_bytes(n) / 4;
         const u64 w0 = (u64)(tile - tb) * TILE_WORDS;
-        const u32 cntw = ws.tile_cnt_w[tile], cnto = ws.tile_cnt_o[tile];
         const u32 offw = ws.tile_off_w[tile], offo = ws.tile_off_o[tile];
-        if (tid < TILE_WORDS) {
-            const u32 a = bm_word(d.rec, s.off_bm_w, nwords, w0 + tid);
-            const u32 b = bm_word(d.rec, s.off_bm_o, nwords, w0 + tid);
-            bw[tid] = a; bo[tid] = b;
-            if (!(s.rflags & REC_MOMENTS_FREE)) bad |= b & ~a;   // a moment kept where the weight is pruned
-            u32 ia = __popc(a), ib = __popc(b);
-            const u32 ca = ia, cb = ib;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                u32 x = __shfl_up_sync(0xffffffffu, ia, o);
-                u32 y = __shfl_up_sync(0xffffffffu, ib, o);
-                if (lane >= o) { ia += x; ib += y; }
-            }
-            pw[tid] = ia - ca; po[tid] = ib - cb;
-            if (lane == 31) { wsum[0][warp] = ia; wsum[1][warp] = ib; }
-        }
-        // stage the code words of this tile's survivors (ranks [off, off + cnt)): whole aligned
-        // 32-bit words of the sections (a section is padded to 16 bytes, so the last word exists)
-        const bool raw = s.rflags & REC_RAW;              // sections hold fp32 survivors, read straight from the record
-        const bool absolute = s.rflags & REC_ABSOLUTE;    // the weight stream is W itself
-        const u32 nb = raw ? 4u : s.bits;                 // code width (raw: unused)
-        const u32 cmask = (1u << nb) - 1u;
-        const u32 fw = (u32)(((u64)offw * nb) >> 5), fo = (u32)(((u64)offo * nb) >> 5);   // first staged word of each section
-        const u32 nww = cntw ? (u32)((((u64)offw + cntw) * nb + 31) >> 5) - fw : 0;
-        const u32 nwo = cnto ? (u32)((((u64)offo + cnto) * nb + 31) >> 5) - fo : 0;
-        if (!raw) {
-            const u32* s0 = reinterpret_cast<const u32*>(d.rec + s.off_codes[0]) + fw;
-            const u32* s1 = reinterpret_cast<const u32*>(d.rec + s.off_codes[1]) + fo;
-            const u32* s2 = reinterpret_cast<const u32*>(d.rec + s.off_codes[2]) + fo;
-            for (u32 i = tid; i < nww; i += TPB) codes[0][i] = s0[i];
-            for (u32 i = tid; i < nwo; i += TPB) { codes[1][i] = s1[i]; codes[2][i] = s2[i]; }
-            if (tid == 0) { codes[0][nww] = 0; codes[1][nwo] = 0; codes[2][nwo] = 0; }   // upper half of the last window
-        }
-        __syncthreads();
-        if (tid < TILE_WORDS) {
-            u32 aw = 0, ao = 0;
-            for (int w = 0; w < warp; ++w) { aw += wsum[0][w]; ao += wsum[1][w]; }
-            pw[tid] += aw; po[tid] += ao;
-        }
-        __syncthreads();
-        const u64 base = (u64)(tile - tb) * TILE;
-        const u32 qw0 = (u32)((u64)offw * nb - 32ull * fw), qo0 = (u32)((u64)offo * nb - 32ull * fo);   // staged bit of the tile's first code
-#pragma unroll
-        for (int r = 0; r < ROUNDS; ++r) {
-            const u32 e0 = r * (TPB * 4) + tid * 4;       // element within the tile
-            const u64 i0 = base + e0;
-            const bool live = i0 < n;
-            if (!DENSE && !live) continue;
-            float wp[4] = {0.f, 0.f, 0.f, 0.f};
-            if (!DENSE && !absolute) load4(w_prev, i0, n, wp);
-            const u32 word = e0 >> 5, bit = e0 & 31;
-            const u32 mw4 = (bw[word] >> bit) & 15u, mo4 = (bo[word] >> bit) & 15u;
-            if (!DENSE && raw) {
-                u32 gw = offw + pw[word] + __popc(bw[word] & ((1u << bit) - 1u));
-                u32 go = offo + po[word] + __popc(bo[word] & ((1u << bit) - 1u));
-                const float* vw = reinterpret_cast<const float*>(d.rec + s.off_codes[0]);
-                const float* va = reinterpret_cast<const float*>(d.rec + s.off_codes[1]);
-                const float* ve = reinterpret_cast<const float*>(d.rec + s.off_codes[2]);
-                for (int k = 0; k < 4 && i0 + k < n; ++k) {
-                    float w = wp[k], a = 0.f, e = 0.f;
-                    if ((mw4 >> k) & 1u) w = __fadd_rn(wp[k], vw[gw++]);
-                    if ((mo4 >> k) & 1u) { a = va[go]; e = ve[go]; ++go; }
-                    wput(w_out, i0 + k, w); d.ea_out[i0 + k] = a; d.eas_out[i0 + k] = e;
-                }
-                continue;
-            }
-            // this thread's survivors have consecutive ranks, so their codes are consecutive
-            // nibbles: one 32-bit window per stream holds all four
-            const u32 qw = qw0 + nb * (pw[word] + __popc(bw[word] & ((1u << bit) - 1u)));
-            const u32 qo = qo0 + nb * (po[word] + __popc(bo[word] & ((1u << bit) - 1u)));
-            u32 win0 = __funnelshift_r(codes[0][qw >> 5], codes[0][(qw >> 5) + 1], qw & 31u);
-            u32 win1 = __funnelshift_r(codes[1][qo >> 5], codes[1][(qo >> 5) + 1], qo & 31u);
-            u32 win2 = __funnelshift_r(codes[2][qo >> 5], codes[2][(qo >> 5) + 1], qo & 31u);
-            float ow[4], oa[4], os[4];
-            u32 nib0 = 0, nib1 = 0, nib2 = 0;             // DENSE: the four codes per stream
+        {   // lane l holds words 4l .. 4l+3 of both bitmaps; ranks by a scan over the lanes
+            u32 a[4], b[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                ow[k] = wp[k]; oa[k] = 0.f; os[k] = 0.f;
-                if ((mw4 >> k) & 1u) {
-                    const u32 c = win0 & cmask;
-                    win0 >>= nb;
-                    if (c == 0) bad = 1; else ow[k] = __fadd_rn(wp[k], cent[0][c - 1]);
-                    nib0 |= c << (4 * k);
+                a[k] = bm_word(d.rec, s.off_bm_w, nwords, w0 + 4 * lane + k);
+                b[k] = bm_word(d.rec, s.off_bm_o, nwords, w0 + 4 * lane + k);
+                if (!(s.rflags & REC_MOMENTS_FREE)) bad |= b[k] & ~a[k];   // a moment kept where the weight is pruned
+            }
+            const u32 ta = __popc(a[0]) + __popc(a[1]) + __popc(a[2]) + __popc(a[3]);
+            const u32 tbm = __popc(b[0]) + __popc(b[1]) + __popc(b[2]) + __popc(b[3]);
+            u32 ia = ta, ib = tbm;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const u32 x = __shfl_up_sync(0xffffffffu, ia, o), y = __shfl_up_sync(0xffffffffu, ib, o);
+                if (lane >= o) { ia += x; ib += y; }
+            }
+            u32 ra = ia - ta, rb = ib - tbm;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                bw[4 * lane + k] = a[k]; bo[4 * lane + k] = b[k];
+                pw[4 * lane + k] = ra; po[4 * lane + k] = rb;
+                ra += __popc(a[k]); rb += __popc(b[k]);
+            }
+        }
+        __syncwarp();
+        const bool raw = s.rflags & REC_RAW;              // sections hold fp32 survivors
+        const bool absolute = s.rflags & REC_ABSOLUTE;    // the weight stream is W itself
+        const u32 nb = raw ? 32u : s.bits;
+        const u32 cmask = raw ? 0xffffffffu : (1u << nb) - 1u;
+        const u32* sec0 = reinterpret_cast<const u32*>(d.rec + s.off_codes[0]);
+        const u32* sec1 = reinterpret_cast<const u32*>(d.rec + s.off_codes[1]);
+        const u32* sec2 = reinterpret_cast<const u32*>(d.rec + s.off_codes[2]);
+        const u64 base = (u64)(tile - tb) * TILE;
+#pragma unroll 2
+        for (int r = 0; r < TILE / 128; ++r) {
+            const u32 e0 = r * 128 + lane * 4;            // element within the tile
+            const u64 i0 = base + e0;
+            const bool live = i0 < n;
+            if (!DENSE && !__any_sync(0xffffffffu, live)) break;
+            float wp[4] = {0.f, 0.f, 0.f, 0.f};
+            if (!DENSE && !absolute && live) load4(w_prev, i0, n, wp);
+            const u32 word = e0 >> 5, bit = e0 & 31;
+            const u32 mw4 = (bw[word] >> bit) & 15u, mo4 = (bo[word] >> bit) & 15u;
+            const u64 gw0 = (u64)offw + pw[word] + __popc(bw[word] & ((1u << bit) - 1u));
+            const u64 go0 = (u64)offo + po[word] + __popc(bo[word] & ((1u << bit) - 1u));
+            float ow[4], oa[4], os[4];
+            u32 nib0 = 0, nib1 = 0, nib2 = 0;             // DENSE: the four codes per stream
+            if (!raw) {
+                u32 win0 = code_window(sec0, gw0, nb, __popc(mw4));
+                u32 win1 = code_window(sec1, go0, nb, __popc(mo4));
+                u32 win2 = code_window(sec2, go0, nb, __popc(mo4));
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    ow[k] = wp[k]; oa[k] = 0.f; os[k] = 0.f;
+                    if ((mw4 >> k) & 1u) {
+                        const u32 c = win0 & cmask;
+                        win0 >>= nb;
+                        if (c == 0) bad = 1; else ow[k] = __fadd_rn(wp[k], cent[0][c - 1]);
+                        nib0 |= c << (4 * k);
+                    }
+                    if ((mo4 >> k) & 1u) {
+                        const u32 c1 = win1 & cmask, c2 = win2 & cmask;
+                        win1 >>= nb; win2 >>= nb;
+                        if (c1 == 0 || c2 == 0) bad = 1;
+                        else { oa[k] = cent[1][c1 - 1]; os[k] = cent[2][c2 - 1]; }
+                        nib1 |= c1 << (4 * k);
+                        nib2 |= c2 << (4 * k);
+                    }
                 }
-                if ((mo4 >> k) & 1u) {
-                    const u32 c1 = win1 & cmask, c2 = win2 & cmask;
-                    win1 >>= nb; win2 >>= nb;
-                    if (c1 == 0 || c2 == 0) bad = 1;
-                    else { oa[k] = cent[1][c1 - 1]; os[k] = cent[2][c2 - 1]; }
-                    nib1 |= c1 << (4 * k);
-                    nib2 |= c2 << (4 * k);
+            } else {
+                u64 gw = gw0, go = go0;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    ow[k] = wp[k]; oa[k] = 0.f; os[k] = 0.f;
+                    if ((mw4 >> k) & 1u) ow[k] = __fadd_rn(wp[k], __uint_as_float(__ldg(sec0 + gw++)));
+                    if ((mo4 >> k) & 1u) { oa[k] = __uint_as_float(__ldg(sec1 + go)); os[k] = __uint_as_float(__ldg(sec2 + go)); ++go; }
                 }
             }
             if (DENSE) {
@@ -242,12 +256,13 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
                     const u32 w = __shfl_down_sync(0xffffffffu, pair, 6);
                     if ((lane & 7) == 0 && live) *reinterpret_cast<uint4*>(sec + j * sb) = make_uint4(pair, y, z, w);
                 }
-            } else {
+            } else if (live) {
                 store4(w_out, i0, n, ow);
                 store4(d.ea_out, i0, n, oa);
                 store4(d.eas_out, i0, n, os);
             }
         }
+        __syncwarp();                                     // the warp's shared-memory corner is free again
     }
     if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(&call->flags, FLAG_CORRUPT);
 }
@@ -259,10 +274,16 @@ void launch_decode(const LaunchCfg& cfg, const DecDesc* descs, DecState* st, int
     dec_popcount_kernel<<<(tiles + TPB / 32 - 1) / (TPB / 32), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws);
     dec_scan_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, ws, call);
     prof_mark(cfg, ST_DEC_PREP, 3);
-    const u32 grid = min(tiles, (u32)cfg.sms * 4u);
-    if (wfmt == WF_F16) decode_kernel<false, __half><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, call);
-    else if (wfmt == WF_BF16) decode_kernel<false, __nv_bfloat16><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, call);
-    else decode_kernel<false, float><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, call);
+    const u32 grid = min((tiles + DEC_WARPS - 1) / DEC_WARPS, (u32)cfg.sms * 4u);
+    const size_t smem = sizeof(DecodeSmem);
+    auto run = [&](auto tag) {
+        using WT = decltype(tag);
+        cudaFuncSetAttribute(decode_kernel<false, WT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        decode_kernel<false, WT><<<grid, TPB, smem, cfg.stream>>>(descs, st, nt, tiles, ws, call);
+    };
+    if (wfmt == WF_F16) run(__half{});
+    else if (wfmt == WF_BF16) run(__nv_bfloat16{});
+    else run(float{});
     prof_mark(cfg, ST_DECODE, 1);
 }
 
@@ -314,8 +335,9 @@ void launch_record_to_dense(const LaunchCfg& cfg, const DecDesc* descs, DecState
     dense_header_kernel<<<nt, 64, 0, cfg.stream>>>(descs, st, call);
     prof_mark(cfg, ST_DEC_PREP, tiles ? 4 : 2);
     if (!tiles) return;
-    const u32 grid = min(tiles, (u32)cfg.sms * 8u);
-    decode_kernel<true, float><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, call);
+    const u32 grid = min((tiles + DEC_WARPS - 1) / DEC_WARPS, (u32)cfg.sms * 4u);
+    cudaFuncSetAttribute(decode_kernel<true, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecodeSmem));
+    decode_kernel<true, float><<<grid, TPB, sizeof(DecodeSmem), cfg.stream>>>(descs, st, nt, tiles, ws, call);
     prof_mark(cfg, ST_DENSE, 1);
 }
 
