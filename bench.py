@@ -32,7 +32,7 @@ METRIC = "compress params/s and GB/s of (W,W_prev,m,v) read at 7B shape; % of HB
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read + dram__bytes_write per parameter from the ncu captures summarised under
 # profiles/ (small case, scaled by parameters); only for kernels unchanged since the capture
-NCU_DRAM_BYTES_PER_PARAM = {"mask_compact": (1.027960e9 + 169.052928e6) / 64108544}
+NCU_DRAM_BYTES_PER_PARAM = {"mask_compact": (1.028104e9 + 169.809664e6) / 64108544}
 FALLBACK_HBM_GBS = 6650.0
 
 
