@@ -190,11 +190,9 @@ def run_reference(args):
 def run_ours(args):
     import torch
     import torch.distributed as dist
-    from paper_2406_11257_b200 import binding, synth
+    from paper_2406_11257_b200 import binding, ranks, synth
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = ranks.rank_info()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the compression path has no CPU fallback")
     torch.cuda.set_device(local)
@@ -203,15 +201,14 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        ranks.barrier(world)
 
     shape = synth.CONFIG_SHAPES[args.config]
     shapes = synth.tensor_list(shape)
     if args.max_tensors:
         shapes = shapes[:args.max_tensors]
     n_tot = sum(n for _, n in shapes)
-    seed = 1000 + rank                                    # every rank compresses its own checkpoint
+    seed = ranks.rank_seed(1000, rank)                    # every rank compresses its own checkpoint
     quads = [synth.make_quad(n, seed, i, device=dev) for i, (_, n) in enumerate(shapes)]
     wfmt = {"f32": binding.WEIGHTS_F32, "f16": binding.WEIGHTS_F16, "bf16": binding.WEIGHTS_BF16}[args.weights]
     wb = 4 if wfmt == binding.WEIGHTS_F32 else 2            # bytes per stored weight
@@ -255,13 +252,9 @@ def run_ours(args):
     ev1.record()
     torch.cuda.synchronize(); barrier()
     clocks = sampler.stop()
-    elapsed_ms = ev0.elapsed_time(ev1)
-    if world > 1:
-        t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = ranks.max_over_ranks(ev0.elapsed_time(ev1), world, dev)
     ms_per_step = elapsed_ms / args.steps
-    value = world * n_tot / (ms_per_step * 1e-3)
+    value = ranks.whole_job_rate(world * n_tot, ms_per_step)
 
     nnz_w = sum(s.nnz_w for s in stats)
     nnz_o = sum(s.nnz_o for s in stats)
@@ -473,12 +466,8 @@ def run_ours(args):
         for _ in range(args.e2e_steps):
             hoffs, _ = h2.compress_checkpoint_host(p, hq, hblob, want_stats=False)
         e1.record(); torch.cuda.synchronize(); barrier()
-        ems = e0.elapsed_time(e1) / args.e2e_steps
-        if world > 1:
-            t = torch.tensor([ems], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ems = float(t.item())
-        out["e2e"] = {"value": world * n_sub / (ems * 1e-3), "unit": "params/s", "h2d_bytes_per_step": 16 * n_sub,
+        ems = ranks.max_over_ranks(e0.elapsed_time(e1) / args.e2e_steps, world, dev)
+        out["e2e"] = {"value": ranks.whole_job_rate(world * n_sub, ems), "unit": "params/s", "h2d_bytes_per_step": 16 * n_sub,
                       "d2h_bytes_per_step": hoffs[-1], "ms_per_step": ems, "steps": args.e2e_steps,
                       "sample": "whole workload" if len(sub) == len(shapes) else f"first {len(sub)} tensors ({n_sub} params): host memory",
                       "h2d_gbs": 16 * n_sub / (ems * 1e-3) / 1e9}
