@@ -209,8 +209,10 @@ __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __res
                     for (int i = 0; i < PER; ++i) {
                         const u32 code = NB == 4 ? find_cluster4(xs[i], t3[k], t7[k], t11[k], thr_row) / 4 + 1
                                                  : find_cluster<NB>(xs[i], sm.thr[warp][k]) + 1;
-                        if (PER * r + i < nel) w |= code << (NB * i);
+                        w |= code << (NB * i);
                     }
+                    const u32 have = nel - PER * r;            // codes of this row that exist (the stage holds stale values after them)
+                    if (have < (u32)PER) w &= (1u << (NB * have)) - 1u;
                     rows[1 + r] = w;
                 }
                 if (lane == 0) rows[1 + nrows] = 0;
