@@ -321,6 +321,7 @@ __device__ static u32 block_select(const u32* __restrict__ keys, u32 cnt, u32 ra
 }
 
 constexpr u32 MEDIAN_SAMPLE = 65536;         // evenly spaced elements that bracket the median
+constexpr int SAMPLE_BINS = 2048;            // steps of the sample's histogram that places the bracket
 constexpr u32 MEDIAN_MARGIN = MEDIAN_SAMPLE / 80;   // +-1.25 % of the sample: about six standard deviations
 
 // One block per tensor.  The sample's keys go to the tensor's second survivor segment (free
@@ -330,6 +331,7 @@ __global__ void __launch_bounds__(1024) median_sample_kernel(const TensorDesc* _
                                                              TensorState* __restrict__ st, Workspace ws,
                                                              int residual_median) {
     __shared__ u32 hist[256];
+    __shared__ u32 fine[SAMPLE_BINS];
     __shared__ u32 range[2];
     const int t = blockIdx.x, tid = threadIdx.x;
     TensorState& s = st[t];
@@ -365,9 +367,21 @@ __global__ void __launch_bounds__(1024) median_sample_kernel(const TensorDesc* _
         if (tid == 0) { s.median_bits = med; s.med_done = 1; }
         return;
     }
-    const u32 lo = block_select(keys, m, m / 2 - MEDIAN_MARGIN, hist, kmin, width);
-    const u32 hi = block_select(keys, m, m / 2 + MEDIAN_MARGIN, hist, kmin, width);
-    if (tid == 0) { s.lo_key = lo; s.hi_key = hi; }
+    // The bracket only has to hold the two sample ranks, not to be them: one histogram of the
+    // sample over 2048 equal steps of its range, and the bracket runs from the lower edge of the
+    // step that holds rank m/2 - margin to the upper edge of the step that holds rank m/2 + margin.
+    const int shift = max(32 - __clz(width | 1u) - 11, 0);
+    for (int i = tid; i < SAMPLE_BINS; i += 1024) fine[i] = 0;
+    __syncthreads();
+    for (u32 j = tid; j < m; j += 1024) atomicAdd(&fine[(keys[j] - kmin) >> shift], 1u);
+    __syncthreads();
+    u32 bin_lo, bin_hi, rin, cnt;
+    find_rank_block<SAMPLE_BINS>(fine, m / 2 - MEDIAN_MARGIN, bin_lo, rin, cnt);
+    find_rank_block<SAMPLE_BINS>(fine, m / 2 + MEDIAN_MARGIN, bin_hi, rin, cnt);
+    if (tid == 0) {
+        s.lo_key = kmin + (bin_lo << shift);
+        s.hi_key = (u32)min((u64)kmin + (((u64)bin_hi + 1) << shift) - 1, (u64)range[1]);
+    }
 }
 
 // ---------------------------------------------------------------------------
