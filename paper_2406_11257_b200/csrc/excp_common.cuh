@@ -224,6 +224,16 @@ __device__ __forceinline__ u32 bucket_of(float x, const BucketFn& f) {
     return min(m, (u32)NBKT - 1);
 }
 
+// The same map, written with min/max and one exclusive-or for the mirror (the counting sweep is
+// bound by its instruction count; the scatter compiles better with the form above).
+__device__ __forceinline__ u32 bucket_index(float x, const BucketFn& f) {
+    const u32 bits = __float_as_uint(x), a = bits & 0x7fffffffu;
+    const u32 m = (max(a, f.lo) - f.lo) >> f.shift;
+    if (f.sgn)      // 128 + m above zero, 127 - m below
+        return (min(m, (u32)NBKT / 2 - 1) | (u32)NBKT / 2) ^ ((u32)((int)bits >> 31) & (u32)(NBKT - 1));
+    return min(m, (u32)NBKT - 1);
+}
+
 // Tensor that owns group tile `tile` (descs are in tile order).
 __device__ inline int find_tensor(const TensorDesc* __restrict__ descs, int n, u32 tile) {
     int lo = 0, hi = n - 1;

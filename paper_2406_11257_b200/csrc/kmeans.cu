@@ -176,13 +176,15 @@ __global__ void __launch_bounds__(TPB) bucket_count_kernel(const TensorDesc* __r
             for (int k = 0; k < NS; ++k) {
                 const float* data = ring.stage() + k * CH;
                 u32* hist = sm.hist[warp][k];
-                for (u32 f = lane; 4 * f < nel; f += 32) {
+                const u32 whole = nel / 4;                             // groups of four that exist entirely
+                for (u32 f = lane; f < whole; f += 32) {
                     const float4 v = *reinterpret_cast<const float4*>(data + 4 * f);
-                    atomicAdd(&hist[bucket_of(v.x, fn[k])], 1u);
-                    if (4 * f + 1 < nel) atomicAdd(&hist[bucket_of(v.y, fn[k])], 1u);
-                    if (4 * f + 2 < nel) atomicAdd(&hist[bucket_of(v.z, fn[k])], 1u);
-                    if (4 * f + 3 < nel) atomicAdd(&hist[bucket_of(v.w, fn[k])], 1u);
+                    atomicAdd(&hist[bucket_index(v.x, fn[k])], 1u);
+                    atomicAdd(&hist[bucket_index(v.y, fn[k])], 1u);
+                    atomicAdd(&hist[bucket_index(v.z, fn[k])], 1u);
+                    atomicAdd(&hist[bucket_index(v.w, fn[k])], 1u);
                 }
+                if (lane < nel - 4 * whole) atomicAdd(&hist[bucket_index(data[4 * whole + lane], fn[k])], 1u);
             }
             ring.advance();
         }
