@@ -234,7 +234,7 @@ struct ScatterSmem {
 // sorts the window by bucket in shared memory and writes each bucket's run with consecutive
 // threads (one 4-byte store per survivor straight to its bucket would be bound by the number
 // of write requests, not by bytes).
-__global__ void __launch_bounds__(TPB, 3) bucket_scatter_kernel(const TensorDesc* __restrict__ descs,
+__global__ void __launch_bounds__(TPB, 4) bucket_scatter_kernel(const TensorDesc* __restrict__ descs,
                                                                 const TensorState* __restrict__ st, int nt,
                                                                 u32 tiles, Workspace ws, int stream) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -286,11 +286,16 @@ __global__ void __launch_bounds__(TPB, 3) bucket_scatter_kernel(const TensorDesc
             }
             u32 bk[SPT / 4];            // the buckets of x[], one byte each
 #pragma unroll
-            for (int k = 0; k < SPT; ++k) {
-                const u32 b = bucket_of(x[k], fn);
-                if ((k & 3) == 0) bk[k / 4] = 0;
-                bk[k / 4] |= b << (8 * (k & 3));
-                if (k * TPB + tid < total) atomicAdd(&sm.cnt[b], 1u);
+            for (int g = 0; g < SPT / 4; ++g) {
+                u32 w = 0;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int k = 4 * g + j;
+                    const u32 b = bucket_of(x[k], fn);
+                    w |= b << (8 * j);
+                    if (k * TPB + tid < total) atomicAdd(&sm.cnt[b], 1u);
+                }
+                bk[g] = w;
             }
             __syncthreads();
             {                          // exclusive prefix of the counts; room in the bucketed copy
@@ -517,7 +522,7 @@ void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* s
     }
     bucket_offsets_kernel<<<dim3(nt, 3), NBKT, 0, cfg.stream>>>(ws);
     {
-        const u32 sgrid = min(tiles, (u32)cfg.sms * 3u);
+        const u32 sgrid = min(tiles, (u32)cfg.sms * 4u);
         cudaFuncSetAttribute(bucket_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ScatterSmem));
         for (int k = 0; k < 3; ++k)
             bucket_scatter_kernel<<<sgrid, TPB, sizeof(ScatterSmem), cfg.stream>>>(descs, st, nt, tiles, ws, k);
