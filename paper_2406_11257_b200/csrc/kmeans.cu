@@ -511,7 +511,7 @@ void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* s
     kmeans_start_kernel<<<dim3(nt, 3), SAMPLE_MAX, 0, cfg.stream>>>(descs, st, ws, p.seed, K);
     prof_mark(cfg, ST_KMEANS_START, 1);
     if (!tiles || p.kmeans_iters == 0) return;
-    const u32 grid = min((tiles + BWARPS - 1) / BWARPS, (u32)cfg.sms * 3u);
+    const u32 grid = min((tiles + BWARPS - 1) / BWARPS, (u32)cfg.sms * 5u);
     {
         const size_t m1 = sizeof(BucketCountSmem<1, 512>), m2 = sizeof(BucketCountSmem<2, 256>);
         cudaFuncSetAttribute(bucket_count_kernel<1, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m1);

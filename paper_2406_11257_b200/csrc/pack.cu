@@ -296,7 +296,7 @@ void launch_pack(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st,
     }
     clear_edges_kernel<<<(tiles + TPB - 1) / TPB, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, blob, call, p.bits);
     prof_mark(cfg, ST_HEADER_EDGES, 2);
-    const u32 grid = min((tiles + PWARPS - 1) / PWARPS, (u32)cfg.sms * 4u);
+    const u32 grid = min((tiles + PWARPS - 1) / PWARPS, (u32)cfg.sms * 6u);
     if (p.bits == 4) {
         pack_codes_kernel<1, 512, 4><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 0, blob, call);
         pack_codes_kernel<2, 256, 4><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 1, blob, call);
