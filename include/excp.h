@@ -64,8 +64,8 @@ typedef struct excp_handle_s* excp_handle;
 typedef enum {
     EXCP_OK = 0,
     EXCP_ERR_INVALID_ARG = -1,      /* null / misaligned pointer, bad parameter, workspace too small for a tensor */
-    EXCP_ERR_UNSUPPORTED = -2,      /* a record variant the called routine does not handle (dense layout of a
-                                       record that is not the 4-bit method's own) */
+    EXCP_ERR_UNSUPPORTED = -2,      /* a variant the called routine does not handle (dense layout of a record that is
+                                       not the 4-bit method's own; raw records through the host-buffer entry point) */
     EXCP_ERR_BUFFER_TOO_SMALL = -3, /* blob_capacity below what the records need */
     EXCP_ERR_CUDA = -4,             /* a CUDA runtime call failed; see excp_last_cuda_error */
     EXCP_ERR_CORRUPT_BLOB = -5,     /* decompress: header, sizes, bitmap population or a code is inconsistent */
@@ -204,7 +204,10 @@ excp_status excp_decompress_checkpoint_w16(excp_handle h, const void* blob, cons
  * of one group run on `cuda_stream`, the inputs of the next are copied to a second device
  * staging slot on a copy stream of the handle and the finished records are copied back on
  * another.  The first call allocates the staging (32 bytes per workspace element plus two record
- * buffers).  Records and offsets are identical to excp_compress_checkpoint's.  Synchronises. */
+ * buffers).  Records and offsets are identical to excp_compress_checkpoint's.  Synchronises.
+ * All four pointers of a tensor are required whatever the flags; EXCP_FLAG_NO_QUANT is not offered here
+ * (EXCP_ERR_UNSUPPORTED: the device-side record staging is sized for coded records; a group whose records
+ * outgrow it returns EXCP_ERR_BUFFER_TOO_SMALL). */
 excp_status excp_compress_checkpoint_host(excp_handle h, const excp_params* params, size_t num_tensors,
                                           const float* const* w_t, const float* const* w_prev,
                                           const float* const* ea, const float* const* eas,

@@ -419,6 +419,7 @@ excp_status excp_compress_checkpoint_host(excp_handle h, const excp_params* para
     if (num_tensors && (!w_t || !w_prev || !ea || !eas || !numel)) return EXCP_ERR_INVALID_ARG;
     const excp_status ps = validate_params(params);
     if (ps != EXCP_OK) return ps;
+    if (params->flags & OPT_NO_QUANT) return EXCP_ERR_UNSUPPORTED;   // the record staging is sized for coded records
     for (size_t i = 0; i < num_tensors; ++i)
         if (numel[i] && (!w_t[i] || !w_prev[i] || !ea[i] || !eas[i])) return EXCP_ERR_INVALID_ARG;
     tensor_offsets_out[0] = 0;

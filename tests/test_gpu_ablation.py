@@ -109,3 +109,19 @@ def test_flag_errors_and_record_flags(handle):
     assert e.value.status == -2
     nbytes, _ = handle.compress_tensor(binding.Params(median_source=1, flags=PRUNE), *dq, blob)
     assert handle.record_to_dense(blob, nbytes, 9000, dense) == binding.dense_bytes(9000)   # no record flag: fine
+
+
+def test_host_buffer_path_with_switches(handle):
+    sizes = [5000, 0, 70000, 4096, 130000]
+    quads = [rand_quad_np(n, 2700 + i) for i, n in enumerate(sizes)]
+    hq = [tuple(torch.as_tensor(a).pin_memory() for a in q) for q in quads]
+    p = binding.Params(median_source=1, kmeans_iters=3, flags=W2M | PRUNE)
+    hblob = torch.empty(sum(binding.compress_bound(n) for n in sizes), dtype=torch.uint8).pin_memory()
+    offs, _ = handle.compress_checkpoint_host(p, hq, hblob)
+    raw = hblob.numpy().tobytes()
+    for i, q in enumerate(quads):
+        want, _ = orc.compress_tensor(*q, orc.Params(median_source=1, kmeans_iters=3, flags=W2M | PRUNE), tensor_index=i)
+        assert raw[offs[i]:offs[i + 1]] == want
+    with pytest.raises(binding.ExcpError) as e:                          # raw records do not go through the staging
+        handle.compress_checkpoint_host(binding.Params(flags=QUANT), hq, hblob)
+    assert e.value.status == -2
