@@ -267,9 +267,8 @@ def run_ours(args):
     stage_bytes = {
         "stats1": (src_b + 4) * n_tot,
         "mask_compact": (2 * wb + 8) * n_tot + n_tot / 4 + 4 * surv,
-        "bucket_ids": 4 * surv,                     # survivors read once to count them per bucket
+        "bucket_ids": 4 * surv,                     # survivors read once: counts and fixed-point sums per bucket
         "bucket_scatter": 8 * surv,                 # survivors read and written into their buckets
-        "bucket_sum": 4 * surv,                     # the bucketed copy read once for the bucket sums
         "bucket_scan": T * 4 * surv * min(1.0, (2 ** args.bits - 2) / 256),   # about K - 1 of 256 buckets per iteration
         "pack_codes": (4 + args.bits / 8) * surv,
         "copy_bitmaps": n_tot / 2,

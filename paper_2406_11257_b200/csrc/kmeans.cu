@@ -18,9 +18,9 @@
 // it count whole, and the one bucket is scanned.  That is a small part of the
 // data per iteration, and the sums are exactly those of a full sweep.
 //
-//   bucket_count    sweep: survivors per bucket
+//   bucket_count    sweep: survivors per bucket and every bucket's fixed-point sum
 //   bucket_offsets  prefix of the counts -> where each bucket starts
-//   bucket_scatter  sweep: survivors into their buckets, bucket sums
+//   bucket_scatter  sweep: survivors into their buckets
 //   bucket_prefix   prefix of the sums; first plan
 //   per iteration:  bucket_scan (the K - 1 threshold buckets), bucket_update
 #include "excp_common.cuh"
@@ -119,11 +119,16 @@ struct BucketCountSmem {
     float buf[BWARPS][BST][NS][CH];
     unsigned long long bar[BWARPS][BST];
     u32 hist[BWARPS][NS][NBKT];      // each warp's counts since its last flush
+    u32 slo[BWARPS][NS][NBKT];       // and fixed-point sums, as sums of the low 16 bits
+    u32 shi[BWARPS][NS][NBKT];       //   and of the (signed) high 16 bits of every value's Q
 };
+constexpr u32 COUNT_FLUSH_CHUNKS = 32768 / 512;   // at most 32768 values per warp between flushes: the 16-bit sums fit
 
-// Sweep 1 of the grouping: survivors per bucket.  NS = 1: dW; NS = 2: both moment streams.
+// Sweep 1 of the grouping: survivors per bucket and their fixed-point sums.  NS = 1: dW; NS = 2:
+// both moment streams.
 template <int NS, int CH>
-__global__ void __launch_bounds__(TPB) bucket_count_kernel(const TensorDesc* __restrict__ descs, int nt, u32 tiles,
+__global__ void __launch_bounds__(TPB) bucket_count_kernel(const TensorDesc* __restrict__ descs,
+                                                           const TensorState* __restrict__ st, int nt, u32 tiles,
                                                            Workspace ws, int stream0, CallState* call) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     BucketCountSmem<NS, CH>& sm = *reinterpret_cast<BucketCountSmem<NS, CH>*>(smem_raw);
@@ -139,11 +144,14 @@ __global__ void __launch_bounds__(TPB) bucket_count_kernel(const TensorDesc* __r
     for (int k = 0; k < NS; ++k) {
         surv[k] = ws.surv[stream0 + k];
         fn[k] = BucketFn{0, 0, 0, 0};
-        for (int b = lane; b < NBKT; b += 32) sm.hist[warp][k][b] = 0;
+        for (int b = lane; b < NBKT; b += 32) { sm.hist[warp][k][b] = 0; sm.slo[warp][k][b] = 0; sm.shi[warp][k][b] = 0; }
     }
     __syncwarp();
     int cur = -1;
-    u32 tb = 0, ntl = 0;
+    u32 tb = 0, ntl = 0, since = 0;
+    float s1[NS], s2[NS];
+#pragma unroll
+    for (int k = 0; k < NS; ++k) { s1[k] = 0.f; s2[k] = 0.f; }
 
     auto flush = [&](int tns) {
         __syncwarp();
@@ -151,8 +159,15 @@ __global__ void __launch_bounds__(TPB) bucket_count_kernel(const TensorDesc* __r
         for (int k = 0; k < NS; ++k)
             for (int b = lane; b < NBKT; b += 32) {
                 const u32 c = sm.hist[warp][k][b];
-                if (c) { atomicAdd(&ws.bst[tns].s[stream0 + k].cnt[b], c); sm.hist[warp][k][b] = 0; }
+                if (c) {
+                    BucketStream& bk = ws.bst[tns].s[stream0 + k];
+                    atomicAdd(&bk.cnt[b], c);
+                    const s64 sum = ((s64)(int)sm.shi[warp][k][b] << 16) + (s64)sm.slo[warp][k][b];
+                    if (sum) atomicAdd(reinterpret_cast<u64*>(&bk.sum[b]), (u64)sum);
+                    sm.hist[warp][k][b] = 0; sm.slo[warp][k][b] = 0; sm.shi[warp][k][b] = 0;
+                }
             }
+        since = 0;
         __syncwarp();
     };
 
@@ -165,7 +180,10 @@ __global__ void __launch_bounds__(TPB) bucket_count_kernel(const TensorDesc* __r
                 cur = find_tensor(descs, nt, tile);
                 tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
 #pragma unroll
-                for (int k = 0; k < NS; ++k) fn[k] = ws.bst[cur].s[stream0 + k].fn;
+                for (int k = 0; k < NS; ++k) {
+                    fn[k] = ws.bst[cur].s[stream0 + k].fn;
+                    s1[k] = st[cur].s[stream0 + k].scale1; s2[k] = st[cur].s[stream0 + k].scale2;
+                }
             }
             const u32 nel = ring.nel();
             if (!ring.wait()) {
@@ -176,16 +194,24 @@ __global__ void __launch_bounds__(TPB) bucket_count_kernel(const TensorDesc* __r
             for (int k = 0; k < NS; ++k) {
                 const float* data = ring.stage() + k * CH;
                 u32* hist = sm.hist[warp][k];
+                u32* slo = sm.slo[warp][k];
+                u32* shi = sm.shi[warp][k];
+                const float a1 = s1[k], a2 = s2[k];
+                auto tally = [&](float x) {
+                    const u32 b = bucket_index(x, fn[k]);
+                    const int q = __float2int_rn(__fmul_rn(__fmul_rn(x, a1), a2));      // Q(x), |Q| < 2^31
+                    atomicAdd(&hist[b], 1u);
+                    atomicAdd(&slo[b], (u32)q & 0xffffu);
+                    atomicAdd(&shi[b], (u32)(q >> 16));
+                };
                 const u32 whole = nel / 4;                             // groups of four that exist entirely
                 for (u32 f = lane; f < whole; f += 32) {
                     const float4 v = *reinterpret_cast<const float4*>(data + 4 * f);
-                    atomicAdd(&hist[bucket_index(v.x, fn[k])], 1u);
-                    atomicAdd(&hist[bucket_index(v.y, fn[k])], 1u);
-                    atomicAdd(&hist[bucket_index(v.z, fn[k])], 1u);
-                    atomicAdd(&hist[bucket_index(v.w, fn[k])], 1u);
+                    tally(v.x); tally(v.y); tally(v.z); tally(v.w);
                 }
-                if (lane < nel - 4 * whole) atomicAdd(&hist[bucket_index(data[4 * whole + lane], fn[k])], 1u);
+                if (lane < nel - 4 * whole) tally(data[4 * whole + lane]);
             }
+            if (++since >= COUNT_FLUSH_CHUNKS * 512u / CH) flush(cur);
             ring.advance();
         }
     }
@@ -343,39 +369,6 @@ __device__ inline void plan_scan(const StreamState& s, BucketStream& bk, int K, 
     }
 }
 
-// Fixed-point sum of every bucket, read off the bucketed copy (each bucket is contiguous there).
-// Grid (NBKT, tensors * 3): one block per bucket.
-__global__ void __launch_bounds__(TPB) bucket_sum_kernel(const TensorDesc* __restrict__ descs,
-                                                         const TensorState* __restrict__ st, Workspace ws) {
-    __shared__ s64 rsum[TPB / 32];
-    const int t = blockIdx.y / 3, k = blockIdx.y % 3, b = blockIdx.x;
-    BucketStream& bk = ws.bst[t].s[k];
-    const u32 r0 = bk.off[b], r1 = bk.off[b + 1];
-    if (r0 == r1) return;
-    const float s1 = st[t].s[k].scale1, s2 = st[t].s[k].scale2;
-    const float* data = ws.bkt[k] + (u64)descs[t].tile_begin * TILE;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    s64 sum = 0;
-    u32 i = r0 + threadIdx.x;
-    for (; i + 7 * TPB < r1; i += 8 * TPB) {               // eight independent loads in flight
-        float x[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) x[j] = __ldcs(data + i + j * TPB);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) sum += __float2int_rn(__fmul_rn(__fmul_rn(x[j], s1), s2));
-    }
-    for (; i < r1; i += TPB) sum += __float2int_rn(__fmul_rn(__fmul_rn(__ldcs(data + i), s1), s2));
-#pragma unroll
-    for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    if (lane == 0) rsum[warp] = sum;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        s64 tot = 0;
-        for (int w = 0; w < TPB / 32; ++w) tot += rsum[w];
-        bk.sum[b] = tot;
-    }
-}
-
 // Exclusive prefix of the bucket sums; plan of the first iteration.  Grid (tensors, 3).
 __global__ void __launch_bounds__(NBKT) bucket_prefix_kernel(const TensorState* __restrict__ st, Workspace ws, int K) {
     __shared__ s64 wtot[NBKT / 32];
@@ -516,8 +509,8 @@ void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* s
         const size_t m1 = sizeof(BucketCountSmem<1, 512>), m2 = sizeof(BucketCountSmem<2, 256>);
         cudaFuncSetAttribute(bucket_count_kernel<1, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m1);
         cudaFuncSetAttribute(bucket_count_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m2);
-        bucket_count_kernel<1, 512><<<grid, TPB, m1, cfg.stream>>>(descs, nt, tiles, ws, 0, call);
-        bucket_count_kernel<2, 256><<<grid, TPB, m2, cfg.stream>>>(descs, nt, tiles, ws, 1, call);
+        bucket_count_kernel<1, 512><<<grid, TPB, m1, cfg.stream>>>(descs, st, nt, tiles, ws, 0, call);
+        bucket_count_kernel<2, 256><<<grid, TPB, m2, cfg.stream>>>(descs, st, nt, tiles, ws, 1, call);
         prof_mark(cfg, ST_BUCKET_IDS, 2);
     }
     bucket_offsets_kernel<<<dim3(nt, 3), NBKT, 0, cfg.stream>>>(ws);
@@ -528,9 +521,8 @@ void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* s
             bucket_scatter_kernel<<<sgrid, TPB, sizeof(ScatterSmem), cfg.stream>>>(descs, st, nt, tiles, ws, k);
     }
     prof_mark(cfg, ST_BUCKET_SCATTER, 4);
-    bucket_sum_kernel<<<dim3(NBKT, nt * 3), TPB, 0, cfg.stream>>>(descs, st, ws);
     bucket_prefix_kernel<<<dim3(nt, 3), NBKT, 0, cfg.stream>>>(st, ws, K);
-    prof_mark(cfg, ST_BUCKET_SUM, 2);
+    prof_mark(cfg, ST_BUCKET_SUM, 1);
     for (int it = 0; it < p.kmeans_iters; ++it) {
         bucket_scan_kernel<<<dim3(scan_items, 3 * (K - 1)), TPB, 0, cfg.stream>>>(descs, st, nt, ws, K);
         prof_mark(cfg, ST_BUCKET_SCAN, 1);

@@ -352,7 +352,7 @@ def test_profile_counts_launches_and_times_stages(handle):
     try:
         handle.compress_tensor(binding.Params(median_source=1, kmeans_iters=10), *dq[0], blob)
         ms, launches = handle.profile_read()
-        assert launches == 11 + 1 + 2 + 1 + 2 + 6 + 10 * 2 + 2 + 2 + 1
+        assert launches == 11 + 1 + 2 + 1 + 2 + 5 + 10 * 2 + 2 + 2 + 1
         assert ms["mask_compact"] > 0 and ms["bucket_scan"] > 0 and ms["decode"] == 0
     finally:
         handle.profile_enable(False)
