@@ -315,6 +315,16 @@ int excp_profile_stage_count(void);
 const char* excp_profile_stage_name(int stage);
 excp_status excp_profile_read(excp_handle h, double* stage_ms_out, unsigned long long* launches_out);
 
+/* Tuning knob of the K-means stage (Section 3.3 leaves the implementation of K-means open; the
+ * centres do not depend on this value).  The iterations need, per threshold between two centres,
+ * the values of one narrow value cell.  The cells that all T iterations will visit are predicted
+ * from per-cell counts and sums, and `margin` further cells on either side of every predicted one
+ * are copied out as well (default 1).  A stream whose exact thresholds leave the copied cells
+ * takes a second, complete round, which costs time but gives the same centres; margin = -1 copies
+ * nothing in the first round, so every stream takes the second one.  margin >= -1, else
+ * EXCP_ERR_INVALID_ARG.  Applies to the handle's later calls. */
+excp_status excp_set_kmeans_margin(excp_handle h, int margin);
+
 #ifdef __cplusplus
 }
 #endif

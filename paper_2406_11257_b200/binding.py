@@ -23,7 +23,8 @@ EXPORTS = ["excp_create", "excp_destroy", "excp_record_bytes", "excp_compress_bo
            "excp_compress_checkpoint", "excp_compress_checkpoint_w16", "excp_decompress_checkpoint_w16",
            "excp_compress_checkpoint_host", "excp_decompress_tensor", "excp_decompress_checkpoint",
            "excp_decompress_tensor_noalloc", "excp_dense_bytes", "excp_record_to_dense", "excp_checkpoint_to_dense",
-           "excp_decompress_dense_tensor", "excp_decompress_dense_checkpoint", "excp_profile_enable", "excp_profile_stage_count", "excp_profile_stage_name", "excp_profile_read"]
+           "excp_decompress_dense_tensor", "excp_decompress_dense_checkpoint", "excp_profile_enable", "excp_profile_stage_count", "excp_profile_stage_name", "excp_profile_read",
+           "excp_set_kmeans_margin"]
 
 
 class ExcpError(RuntimeError):
@@ -103,6 +104,7 @@ def load_library() -> C.CDLL:
     lib.excp_decompress_dense_tensor.argtypes = lib.excp_decompress_tensor.argtypes
     lib.excp_decompress_dense_checkpoint.argtypes = lib.excp_decompress_checkpoint.argtypes
     lib.excp_profile_enable.argtypes = [vp, C.c_int]
+    lib.excp_set_kmeans_margin.argtypes = [vp, C.c_int]
     lib.excp_profile_stage_count.argtypes = []
     lib.excp_profile_stage_name.argtypes = [C.c_int]
     lib.excp_profile_stage_name.restype = C.c_char_p
@@ -192,6 +194,12 @@ class Handle:
         e = C.c_int(0)
         self.lib.excp_last_cuda_error(self._h, C.byref(e))
         return e.value
+
+    def set_kmeans_margin(self, margin: int) -> None:
+        """excp_set_kmeans_margin: a tuning knob; the centres do not depend on it."""
+        st = self.lib.excp_set_kmeans_margin(self._h, int(margin))
+        if st != 0:
+            raise ExcpError(st, "excp_set_kmeans_margin")
 
     def profile_enable(self, on: bool = True) -> None:
         st = self.lib.excp_profile_enable(self._h, int(on))

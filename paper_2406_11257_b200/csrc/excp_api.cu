@@ -1,6 +1,7 @@
 // The C ABI of include/excp.h: handle, argument checks, grouping of the tensor
 // list, and the order of the kernel launches.  No arithmetic of the method
 // lives here.
+#include <algorithm>
 #include <cmath>
 #include <cstring>
 #include <new>
@@ -61,6 +62,7 @@ struct excp_handle_s {
     CallState* h_call = nullptr;         // pinned
     size_t tensor_cap = 0;               // entries the per-call arrays hold
     int last_cuda_error = 0;
+    int km_margin = 1;                   // see excp_set_kmeans_margin
     Profiler prof;
     // host-buffer path: two staging slots (inputs + records), its own copy streams
     float* stage[2][4] = {};
@@ -118,27 +120,20 @@ bool ensure_call_arrays(excp_handle h, size_t n) {
     return true;
 }
 
-struct Group { size_t first, count; u32 tiles; u32 scan_items; };
-
-// Blocks that share the scan of one bucket of a tensor (a bucket holds about 1/256 of it).
-u32 scan_splits(size_t numel) {
-    const size_t s = (numel + (8u << 20) - 1) / (8u << 20);
-    return (u32)(s < 1 ? 1 : (s > 32 ? 32 : s));
-}
+struct Group { size_t first, count; u32 tiles; };
 
 // Consecutive tensors whose tiles fit the workspace (and the per-group state).
 bool make_groups(excp_handle h, const size_t* numel, size_t n, std::vector<Group>& out) {
-    Group g{0, 0, 0, 0};
+    Group g{0, 0, 0};
     for (size_t i = 0; i < n; ++i) {
         if (numel[i] > MAX_NUMEL) return false;
         const size_t t = (numel[i] + TILE - 1) / TILE;
         if (t > h->cap_tiles) return false;
         if (g.count && (g.tiles + t > h->cap_tiles || g.count >= (size_t)MAX_GROUP_TENSORS)) {
             out.push_back(g);
-            g = Group{i, 0, 0, 0};
+            g = Group{i, 0, 0};
         }
         g.tiles += (u32)t;
-        g.scan_items += scan_splits(numel[i]);
         ++g.count;
     }
     if (g.count) out.push_back(g);
@@ -155,8 +150,9 @@ excp_status validate_params(const excp_params* params) {
     return EXCP_OK;
 }
 
-Params to_params(const excp_params* params) {
+Params to_params(excp_handle h, const excp_params* params) {
     Params p;
+    p.km_margin = h->km_margin;
     p.alpha = params->alpha; p.beta = params->beta; p.bits = params->bits;
     p.kmeans_iters = params->kmeans_iters; p.seed = params->seed; p.median_source = params->median_source;
     p.flags = params->flags;
@@ -165,13 +161,13 @@ Params to_params(const excp_params* params) {
 }
 
 // All kernels of one group, in order.
-bool run_group(excp_handle h, const LaunchCfg& cfg, const TensorDesc* descs, int nt, u32 tiles, u32 scan_items,
+bool run_group(excp_handle h, const LaunchCfg& cfg, const TensorDesc* descs, int nt, u32 tiles,
                const Params& p, unsigned char* blob, u64 blob_capacity, TensorResult* results) {
     if (!check(h, cudaMemsetAsync(h->d_state, 0, nt * sizeof(TensorState), cfg.stream))) return false;
-    if (!check(h, cudaMemsetAsync(h->ws.bst, 0, nt * sizeof(BucketState), cfg.stream))) return false;
+    if (!check(h, cudaMemsetAsync(h->ws.cst, 0, nt * sizeof(CellState), cfg.stream))) return false;
     launch_stats(cfg, descs, h->d_state, nt, tiles, h->ws, p, h->d_call);
     launch_mask_compact(cfg, descs, h->d_state, nt, tiles, h->ws, p, h->d_call, blob_capacity);
-    if (!(p.flags & OPT_NO_QUANT)) launch_kmeans(cfg, descs, h->d_state, nt, tiles, scan_items, h->ws, p, h->d_call);
+    if (!(p.flags & OPT_NO_QUANT)) launch_kmeans(cfg, descs, h->d_state, nt, tiles, h->ws, p, h->d_call);
     launch_pack(cfg, descs, h->d_state, nt, tiles, h->ws, p, blob, h->d_call, results);
     return check(h, cudaGetLastError());
 }
@@ -240,7 +236,13 @@ excp_status excp_create(excp_handle* out, int device, size_t workspace_numel) {
             ok = check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.surv[k]), elems * sizeof(float)));
             ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.bkt[k]), elems * sizeof(float)));
         }
-        ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.bst), MAX_GROUP_TENSORS * sizeof(BucketState)));
+        ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.cst), MAX_GROUP_TENSORS * sizeof(CellState)));
+        ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.km_pending), sizeof(u32)));
+        const size_t rows = (size_t)std::min(h->sms * 2, (int)KM_MAX_GRID) + MAX_GROUP_TENSORS;
+        for (int k = 0; k < 3 && ok; ++k) {
+            ok = check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.km_rows[k]), rows * NCELL * sizeof(u32)));
+            ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.km_pos[k]), rows * NCELL * sizeof(u32)));
+        }
         ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.bm_w), elems / 8));
         ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.bm_o), elems / 8));
         ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.tile_cnt_w), h->cap_tiles * 4));
@@ -268,7 +270,12 @@ excp_status excp_destroy(excp_handle h) {
         if (h->ws.surv[k]) cudaFree(h->ws.surv[k]);
         if (h->ws.bkt[k]) cudaFree(h->ws.bkt[k]);
     }
-    if (h->ws.bst) cudaFree(h->ws.bst);
+    if (h->ws.cst) cudaFree(h->ws.cst);
+    if (h->ws.km_pending) cudaFree(h->ws.km_pending);
+    for (int k = 0; k < 3; ++k) {
+        if (h->ws.km_rows[k]) cudaFree(h->ws.km_rows[k]);
+        if (h->ws.km_pos[k]) cudaFree(h->ws.km_pos[k]);
+    }
     if (h->ws.bm_w) cudaFree(h->ws.bm_w);
     if (h->ws.bm_o) cudaFree(h->ws.bm_o);
     if (h->ws.tile_cnt_w) cudaFree(h->ws.tile_cnt_w);
@@ -351,7 +358,7 @@ static excp_status compress_impl(excp_handle h, const excp_params* params, size_
 
     TensorDesc* hd = static_cast<TensorDesc*>(h->h_desc);
     for (const Group& g : groups) {
-        u32 tile = 0, item = 0;
+        u32 tile = 0;
         for (size_t i = g.first; i < g.first + g.count; ++i) {
             TensorDesc& d = hd[i];
             d.w_t = w_t[i]; d.w_prev = w_prev[i]; d.ea = ea[i]; d.eas = eas[i];
@@ -360,12 +367,9 @@ static excp_status compress_impl(excp_handle h, const excp_params* params, size_
             d.tile_begin = tile;
             d.num_tiles = (u32)((numel[i] + TILE - 1) / TILE);
             tile += d.num_tiles;
-            d.scan_first = item;
-            d.scan_n = scan_splits(numel[i]);
-            item += d.scan_n;
         }
     }
-    Params p = to_params(params);
+    Params p = to_params(h, params);
     p.wfmt = wfmt;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     LaunchCfg cfg{h->sms, stream, &h->prof};
@@ -375,7 +379,7 @@ static excp_status compress_impl(excp_handle h, const excp_params* params, size_
     ok = ok && check(h, cudaMemcpyAsync(dd, hd, num_tensors * sizeof(TensorDesc), cudaMemcpyHostToDevice, stream));
     for (size_t gi = 0; ok && gi < groups.size(); ++gi) {
         const Group& g = groups[gi];
-        ok = run_group(h, cfg, dd + g.first, (int)g.count, g.tiles, g.scan_items, p, static_cast<unsigned char*>(blob_out),
+        ok = run_group(h, cfg, dd + g.first, (int)g.count, g.tiles, p, static_cast<unsigned char*>(blob_out),
                        blob_capacity, h->d_results + g.first);
     }
     ok = ok && check(h, cudaMemcpyAsync(h->h_results, h->d_results, num_tensors * sizeof(TensorResult),
@@ -435,7 +439,7 @@ excp_status excp_compress_checkpoint_host(excp_handle h, const excp_params* para
     for (size_t gi = 0; gi < groups.size(); ++gi) {
         const Group& g = groups[gi];
         const int slot = (int)(gi & 1);
-        u32 tile = 0, item = 0;
+        u32 tile = 0;
         for (size_t i = g.first; i < g.first + g.count; ++i) {
             TensorDesc& d = hd[i];
             const size_t off = (size_t)tile * TILE;
@@ -446,12 +450,9 @@ excp_status excp_compress_checkpoint_host(excp_handle h, const excp_params* para
             d.tile_begin = tile;
             d.num_tiles = (u32)((numel[i] + TILE - 1) / TILE);
             tile += d.num_tiles;
-            d.scan_first = item;
-            d.scan_n = scan_splits(numel[i]);
-            item += d.scan_n;
         }
     }
-    const Params p = to_params(params);
+    const Params p = to_params(h, params);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     LaunchCfg cfg{h->sms, stream, &h->prof};
     h->prof.begin(stream);
@@ -486,7 +487,7 @@ excp_status excp_compress_checkpoint_host(excp_handle h, const excp_params* para
         ok = ok && check(h, cudaStreamWaitEvent(stream, h->ev_h2d[slot], 0));
         if (gi >= 2) ok = ok && check(h, cudaStreamWaitEvent(stream, h->ev_d2h[slot], 0));
         ok = ok && check(h, cudaMemsetAsync(&h->d_call->blob_cursor, 0, sizeof(u64), stream));
-        ok = ok && run_group(h, cfg, dd + g.first, (int)g.count, g.tiles, g.scan_items, p, h->stage_blob[slot],
+        ok = ok && run_group(h, cfg, dd + g.first, (int)g.count, g.tiles, p, h->stage_blob[slot],
                              h->stage_blob_bytes, h->d_results + g.first);
         ok = ok && check(h, cudaMemcpyAsync(h->h_results + g.first, h->d_results + g.first,
                                             g.count * sizeof(TensorResult), cudaMemcpyDeviceToHost, stream));
@@ -593,6 +594,12 @@ excp_status excp_decompress_checkpoint_w16(excp_handle h, const void* blob, cons
                            cuda_stream);
 }
 
+excp_status excp_set_kmeans_margin(excp_handle h, int margin) {
+    if (!h || margin < -1) return EXCP_ERR_INVALID_ARG;
+    h->km_margin = margin;
+    return EXCP_OK;
+}
+
 excp_status excp_profile_enable(excp_handle h, int enable) {
     if (!h) return EXCP_ERR_INVALID_ARG;
     DeviceGuard guard(h->device);
@@ -610,8 +617,8 @@ int excp_profile_stage_count(void) { return ST_COUNT; }
 
 const char* excp_profile_stage_name(int stage) {
     static const char* names[ST_COUNT] = {
-        "stats1", "stats2", "mask_compact", "scan_layout", "kmeans_start", "bucket_ids", "bucket_scatter",
-        "bucket_scan", "kmeans_update", "header_edges", "pack_codes", "copy_bitmaps", "dec_prep", "decode", "bucket_sum", "dense"};
+        "stats1", "stats2", "mask_compact", "scan_layout", "kmeans_start", "cell_count", "cell_gather",
+        "kmeans_iterate", "cell_plan", "header_edges", "pack_codes", "copy_bitmaps", "dec_prep", "decode", "kmeans_retry", "dense"};
     return stage >= 0 && stage < ST_COUNT ? names[stage] : "";
 }
 

@@ -29,6 +29,7 @@ constexpr int KPAD = 16;
 constexpr int KCAP = 256;                        // room for the centres of the widest code (8 bits: 255)
 constexpr int SAMPLE_MAX = 1024;                 // K-means start sample
 constexpr int MAX_GROUP_TENSORS = 1024;
+constexpr int KM_MAX_GRID = 1024;                // blocks of a K-means sweep (two per SM)
 
 constexpr u32 FLAG_NONFINITE = 1u;               // NaN/Inf input or negative second moment
 constexpr u32 FLAG_BLOB_FULL = 2u;               // records do not fit blob_capacity
@@ -67,8 +68,6 @@ struct TensorDesc {              // built on the host, one per tensor of a group
     u64 tensor_index;            // position in the checkpoint (enters the start sample)
     u32 tile_begin;              // first tile of this tensor within the group
     u32 num_tiles;
-    u32 scan_first;              // first work item of this tensor in the bucket-scan grid
-    u32 scan_n;                  // work items (splits) this tensor has there
 };
 
 struct StreamState {             // K-means state of one stream (0 = dW, 1 = ea, 2 = eas)
@@ -119,34 +118,36 @@ struct CallState {               // one per handle, device resident
     u32 pad_;
 };
 
-constexpr int NBKT = 256;         // value buckets per tensor and stream for the K-means iterations
+constexpr int NCELL = 4096;       // value cells per tensor and stream for the K-means iterations
+constexpr int NCLASS = 512;       // sign x exponent field of an fp32 value = its top nine bits
 
-struct BucketFn {                // a monotone map of fp32 values to 0..255 (see bucket_of)
-    u32 lo;                      // magnitude bit pattern mapped to the first step
-    u32 shift;                   // magnitude bit patterns per step = 2^shift
-    u32 sgn;                     // 1: 128 steps per sign; 0: 256 steps, non-negative values
-    u32 pad_;
+// K-means working state of one stream of one tensor.  The cells are a monotone map of fp32 values
+// to 0..NCELL-1 (see cell_of): every (sign, exponent) class owns a power-of-two number of equal
+// steps of the mantissa, more of them where a sample of the survivors is dense.
+struct CellStream {
+    u32 tab[NCLASS];             // class -> (anchor cell << 8) | log2(cells of the class); the anchor is the
+                                 //   class's first cell for positive values, its last for negative ones
+    u32 cnt[NCELL];              // survivors per cell
+    u64 mag[NCELL];              // sum of |Q| per cell; once planned: low word = start of the cell in the
+                                 //   gathered copy, high word = values gathered so far
+    u32 cntpre[NCELL + 1];       // exclusive prefix of cnt
+    u32 first_pos;               // first cell of the non-negative values
+    s64 sumpre[NCELL + 1];       // exclusive prefix of the signed fixed-point sums
+    u32 sel[NCELL / 32];         // cells whose values are in the gathered copy
+    u32 it_done;                 // Lloyd iterations completed
+    u32 active;                  // iterations remain: the next round plans and gathers for them
 };
-
-struct BucketStream {            // one stream's buckets
-    BucketFn fn;
-    u32 cnt[NBKT];               // survivors per bucket
-    s64 sum[NBKT];               // their fixed-point sums
-    u32 off[NBKT + 1];           // exclusive prefix of cnt = start of each bucket in the bucketed copy
-    u32 pad_;
-    s64 sumpre[NBKT + 1];        // exclusive prefix of sum
-    u32 cursor[NBKT];            // next free slot of each bucket while scattering
-    u32 bstar[KCAP];             // bucket that holds threshold j
-    u64 part_cnt[KCAP];          // survivors <= threshold j inside that bucket
-    s64 part_sum[KCAP];          // and their fixed-point sum
-};
-struct BucketState {
-    BucketStream s[3];
+struct CellState {
+    CellStream s[3];
 };
 
 struct Workspace {               // device arrays sized for cap_tiles tiles
-    float* bkt[3];               // survivors again, grouped by value bucket (order inside a bucket is arbitrary)
-    BucketState* bst;            // per tensor of the group
+    float* bkt[3];               // gathered copy: the survivors of the selected cells, cell after cell
+    CellState* cst;              // per tensor of the group
+    u32* km_pending;             // streams whose first round of iterations met a cell that was not gathered
+    u32* km_rows[3];             // per stream: survivors per cell of every (block, tensor) share of the counting
+                                 //   sweep, row (block + tensor) of NCELL words
+    u32* km_pos[3];              // the same shape: where each share's values of a cell start in the gathered copy
     float* surv[3];              // survivors, each tile's compacted at the tile's own start
     u32* bm_w;                   // bitmaps, TILE_WORDS words per tile
     u32* bm_o;
@@ -163,6 +164,7 @@ struct Params {
     int median_source;
     u32 flags;                   // OPT_*
     int wfmt;                    // WeightFormat of w_t and w_prev
+    int km_margin;               // cells gathered on either side of every predicted threshold (-1: none)
 };
 __host__ __device__ inline int stored_bits(const Params& p) { return (p.flags & OPT_NO_QUANT) ? 32 : p.bits; }
 __host__ __device__ inline u32 record_flags(const Params& p) {
@@ -211,27 +213,15 @@ __host__ __device__ inline u64 record_bytes(u64 numel, u64 nnz_w, u64 nnz_o, int
 
 // ---- device helpers ---------------------------------------------------------
 #ifdef __CUDACC__
-// Bucket of a value: steps of equal width in the bit pattern of |x| (so roughly logarithmic
-// in |x|), clamped at both ends, negative values mirrored below the positive ones.  All that
-// the K-means iterations need of it is that it never decreases when x grows.
-__device__ __forceinline__ u32 bucket_of(float x, const BucketFn& f) {
-    const u32 bits = __float_as_uint(x), a = bits & 0x7fffffffu;
-    u32 m = a > f.lo ? (a - f.lo) >> f.shift : 0u;
-    if (f.sgn) {
-        m = min(m, (u32)NBKT / 2 - 1);
-        return (bits >> 31) ? NBKT / 2 - 1 - m : NBKT / 2 + m;
-    }
-    return min(m, (u32)NBKT - 1);
-}
-
-// The same map, written with min/max and one exclusive-or for the mirror (the counting sweep is
-// bound by its instruction count; the scatter compiles better with the form above).
-__device__ __forceinline__ u32 bucket_index(float x, const BucketFn& f) {
-    const u32 bits = __float_as_uint(x), a = bits & 0x7fffffffu;
-    const u32 m = (max(a, f.lo) - f.lo) >> f.shift;
-    if (f.sgn)      // 128 + m above zero, 127 - m below
-        return (min(m, (u32)NBKT / 2 - 1) | (u32)NBKT / 2) ^ ((u32)((int)bits >> 31) & (u32)(NBKT - 1));
-    return min(m, (u32)NBKT - 1);
+// Cell of a value.  Monotone: x < y implies cell_of(x) <= cell_of(y) (negative classes run from
+// the largest exponent down, their cells from the largest mantissa down; then the positive ones
+// upwards), which is all the K-means iterations need of it.  Any bit pattern maps inside the table.
+__device__ __forceinline__ u32 cell_of(float x, const u32* __restrict__ tab) {
+    const u32 bits = __float_as_uint(x);
+    const u32 ent = tab[bits >> 23];
+    const u32 sub = (bits & 0x7fffffu) >> (23u - (ent & 31u));
+    const u32 neg = (u32)((int)bits >> 31);            // 0 or all ones
+    return (ent >> 8) + ((sub ^ neg) - neg);           // anchor + sub, or anchor - sub
 }
 
 // Tensor that owns group tile `tile` (descs are in tile order).
@@ -363,9 +353,9 @@ __device__ inline void scan_tile_counts(u32 tb, u32 ntl, const Workspace& ws, u3
 
 // ---- launch wrappers --------------------------------------------------------
 enum Stage {                       // for the optional per-stage event timing
-    ST_STATS1 = 0, ST_STATS2, ST_MASK_COMPACT, ST_SCAN_LAYOUT, ST_KMEANS_START, ST_BUCKET_IDS, ST_BUCKET_SCATTER,
-    ST_BUCKET_SCAN, ST_KMEANS_UPDATE, ST_HEADER_EDGES, ST_PACK_CODES, ST_COPY_BITMAPS, ST_DEC_PREP,
-    ST_DECODE, ST_BUCKET_SUM, ST_DENSE, ST_COUNT
+    ST_STATS1 = 0, ST_STATS2, ST_MASK_COMPACT, ST_SCAN_LAYOUT, ST_KMEANS_START, ST_CELL_COUNT, ST_CELL_GATHER,
+    ST_KMEANS_ITERATE, ST_CELL_PLAN, ST_HEADER_EDGES, ST_PACK_CODES, ST_COPY_BITMAPS, ST_DEC_PREP,
+    ST_DECODE, ST_KMEANS_RETRY, ST_DENSE, ST_COUNT
 };
 
 struct Profiler;
@@ -383,7 +373,7 @@ void launch_stats(const LaunchCfg&, const TensorDesc* descs, TensorState* st, in
 void launch_mask_compact(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                          const Workspace& ws, const Params& p, CallState* call, u64 blob_capacity);
 void launch_kmeans(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
-                   u32 scan_items, const Workspace& ws, const Params& p, CallState* call);
+                   const Workspace& ws, const Params& p, CallState* call);
 void launch_pack(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                  const Workspace& ws, const Params& p, unsigned char* blob, CallState* call,
                  TensorResult* results);

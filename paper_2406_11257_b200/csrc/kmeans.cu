@@ -10,19 +10,25 @@
 //   update   mean = fp32(fp64(sum)/fp64(count) * 2^(E-30)); empty clusters keep
 //            their centre; centres re-sorted; new thresholds
 //
-// The iterations do not sweep the survivors.  Because the clusters are intervals
-// and the sums are integers, the survivors are first grouped ONCE into 256 value
-// buckets (a cheap monotone function of the value, scaled to the range of the
-// start sample) with each bucket's count and sum.  An iteration then
-// needs, per threshold, only the bucket the threshold falls into: buckets below
-// it count whole, and the one bucket is scanned.  That is a small part of the
-// data per iteration, and the sums are exactly those of a full sweep.
+// The iterations do not sweep the survivors.  The clusters are intervals and the sums
+// are integers, so an iteration needs, per threshold, the count and the sum of the
+// survivors at or below it.  One sweep files the survivors into 4096 value cells (a
+// monotone map, fine where the values are dense) with each cell's count and sum; the
+// cells below a threshold then count whole, and only the one cell the threshold falls
+// into has to be looked at value by value.  Which cells those will be over all T
+// iterations is predicted by running the iterations on the cell table alone (a
+// threshold's own cell split by interpolation); a second sweep copies the values of
+// the predicted cells and their neighbours, cell after cell, into a gathered copy (a
+// seventh of the survivors at 4 bits), and the exact iterations run on that copy, one
+// block per tensor and stream.  Should an exact threshold ever leave the gathered
+// cells, the stream stops at that iteration and a second round gathers every cell for
+// it and finishes; the centres are those of full sweeps either way.
 //
-//   bucket_count    sweep: survivors per bucket and every bucket's fixed-point sum
-//   bucket_offsets  prefix of the counts -> where each bucket starts
-//   bucket_scatter  sweep: survivors into their buckets
-//   bucket_prefix   prefix of the sums; first plan
-//   per iteration:  bucket_scan (the K - 1 threshold buckets), bucket_update
+//   kmeans_start    start sample; the cell map
+//   cell_count      sweep: count and fixed-point sum of every cell
+//   cell_plan       prefixes; predicted thresholds -> selected cells -> their places
+//   cell_gather     sweep: values of the selected cells into the gathered copy
+//   kmeans_iterate  the exact iterations
 #include "excp_common.cuh"
 #include "seg_ring.cuh"
 
@@ -35,32 +41,39 @@ __device__ inline u64 mix64(u64 z) {   // SplitMix64 output function
     return z ^ (z >> 31);
 }
 
-// Thresholds of K sorted, final centres; threads idx, idx + stride, ... of the caller share the work.
-__device__ inline void set_thresholds(StreamState& s, int K, int idx, int stride) {
-    for (int j = idx; j < KCAP; j += stride) {
-        float t = __uint_as_float(0x7f800000u);
-        if (j < K - 1)
-            t = __double2float_rd(((double)s.cent[j] + (double)s.cent[j + 1]) * 0.5) + 0.f;   // -0 -> +0
-        s.thr[j] = t;
-    }
+__device__ __forceinline__ float mid_threshold(float a, float b) {
+    return __double2float_rd(((double)a + (double)b) * 0.5) + 0.f;   // -0 -> +0
 }
+
+// Thresholds of K sorted centres; threads idx, idx + stride, ... of the caller share the work.
+__device__ inline void set_thresholds(const float* cent, float* thr, int K, int idx, int stride) {
+    for (int j = idx; j < KCAP; j += stride)
+        thr[j] = j < K - 1 ? mid_threshold(cent[j], cent[j + 1]) : __uint_as_float(0x7f800000u);
+}
+
+constexpr int CELL_SAMPLE = 4096;    // survivors whose classes apportion the cells
+constexpr u32 SMALL_STREAM = 16384;  // at most this many survivors: every cell is gathered
 
 // One block per (tensor, stream).
 __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDesc* __restrict__ descs,
                                                                   TensorState* __restrict__ st,
-                                                                  Workspace ws, u64 seed, int K) {
+                                                                  Workspace ws, u64 seed, int K, int iters) {
     __shared__ float smp[SAMPLE_MAX];
-    __shared__ u32 amin, amax;                        // smallest / largest magnitude pattern in the sample
+    __shared__ u32 chist[NCLASS];                     // sampled survivors per (sign, exponent) class
+    __shared__ u32 wtot[NCLASS / 32];
+    __shared__ u32 cvalid;
     const int t = blockIdx.x, stream = blockIdx.y, tid = threadIdx.x;
     StreamState& s = st[t].s[stream];
+    CellStream& cs = ws.cst[t].s[stream];
     const u32 nnz = stream == 0 ? st[t].nnz_w : st[t].nnz_o;
     const u32 tb = descs[t].tile_begin, ntl = descs[t].num_tiles;
     const u32* toff = (stream == 0 ? ws.tile_off_w : ws.tile_off_o) + tb;
+    const u32* tcnt = (stream == 0 ? ws.tile_cnt_w : ws.tile_cnt_o) + tb;
     const float* data = ws.surv[stream] + (u64)tb * TILE;
-    BucketStream& bk = ws.bst[t].s[stream];
-    if (nnz == 0) {
+    if (t == 0 && stream == 0 && tid == 0) *ws.km_pending = 0;
+    if (nnz == 0) {                                   // the zeroed state is a valid (one-cell) map
         if (tid < KCAP) { s.cent[tid] = 0.f; s.thr[tid] = __uint_as_float(0x7f800000u); }
-        if (tid == 0) { bk.fn.lo = 0; bk.fn.shift = 0; bk.fn.sgn = stream != 2; }
+        if (tid == 0) { cs.it_done = (u32)iters; cs.active = 0; }
         return;
     }
     const u32 m = min(nnz, (u32)SAMPLE_MAX);
@@ -79,11 +92,22 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
         v = data[(u64)a * TILE + (r - toff[a])];
     }
     smp[tid] = v;
-    if (tid == 0) { amin = 0x7fffffffu; amax = 0u; }
+    if (tid < NCLASS) chist[tid] = 0;
+    if (tid == 0) cvalid = 0;
     __syncthreads();
-    if ((u32)tid < m) {
-        atomicMin(&amin, __float_as_uint(v) & 0x7fffffffu);
-        atomicMax(&amax, __float_as_uint(v) & 0x7fffffffu);
+    // The cell map: a second, larger sample (a survivor of each of 4096 evenly spaced tiles) says how
+    // the survivors spread over the (sign, exponent) classes.  Any map that is monotone gives the same
+    // centres; this one makes the cells roughly equally full.
+#pragma unroll
+    for (int r = 0; r < CELL_SAMPLE / SAMPLE_MAX; ++r) {
+        const u32 i = (u32)tid + (u32)r * SAMPLE_MAX;
+        const u32 tile = (u32)(((u64)i * ntl) / CELL_SAMPLE);
+        const u32 c = min(tcnt[tile], (u32)TILE);
+        if (c) {
+            const float x = data[(u64)tile * TILE + ((i * 2654435761u) >> 8) % c];
+            atomicAdd(&chist[__float_as_uint(x) >> 23], 1u);
+            atomicAdd(&cvalid, 1u);
+        }
     }
     for (int k = 2; k <= SAMPLE_MAX; k <<= 1) {       // bitonic sort, ascending
         for (int j = k >> 1; j > 0; j >>= 1) {
@@ -97,437 +121,544 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
         }
     }
     if (tid < KCAP) s.cent[tid] = tid < K ? smp[((2 * tid + 1) * m) / (2 * K)] : 0.f;
-    // bucket function: its steps span the magnitudes seen in the sample (any monotone map
-    // would give the same centres; this one spreads these survivors over the 256 buckets)
-    if (tid == 0) {
-        const u32 d = amax - amin;
-        const int half_bits = stream != 2 ? 7 : 8;            // log2 of the steps per sign
-        const int len = 32 - __clz(d);                        // d < 2^len
-        bk.fn.lo = amin; bk.fn.shift = len > half_bits ? len - half_bits : 0; bk.fn.sgn = stream != 2;
+    // Cells per class: one each, and the rest in proportion to the class's share of the sample,
+    // rounded down to a power of two.  Classes in value order: negative ones from the largest
+    // exponent down (classes 511..256), then the positive ones upwards (0..255).
+    u32 lg = 0, ncell = 0, incl = 0;
+    const int cls = tid < 256 ? 511 - tid : tid - 256;    // class at place `tid` of the value order (tid < 512)
+    if (tid < NCLASS) {
+        const u32 want = cvalid ? (u32)(((u64)chist[cls] * (NCELL - NCLASS)) / cvalid) : 0u;
+        lg = want >= 2 ? 31u - (u32)__clz((int)want) : 0u;
+        ncell = 1u << lg;
+        incl = ncell;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const u32 x = __shfl_up_sync(0xffffffffu, incl, o);
+            if ((tid & 31) >= o) incl += x;
+        }
+        if ((tid & 31) == 31) wtot[tid >> 5] = incl;
     }
     __syncthreads();
-    set_thresholds(s, K, tid, SAMPLE_MAX);
+    if (tid < NCLASS) {
+        u32 base = 0;
+        for (int w = 0; w < (tid >> 5); ++w) base += wtot[w];
+        const u32 f = base + incl - ncell;                // first cell of the class
+        cs.tab[cls] = ((cls >= 256 ? f + ncell - 1 : f) << 8) | lg;
+        if (cls == 0) cs.first_pos = f;
+    }
+    if (tid == 0) { cs.it_done = 0; cs.active = iters > 0 ? 1u : 0u; }
+    __syncthreads();
+    set_thresholds(s.cent, s.thr, K, tid, SAMPLE_MAX);
 }
-
 
 // ---------------------------------------------------------------------------
-constexpr int BWARPS = TPB / 32;
 constexpr int BST = 2;               // stages per warp
+constexpr int KM_GRID_PER_SM_W = 2;  // blocks per SM of the dW sweeps (the moment sweeps run one)
+constexpr int CWARPS = 16;           // warps per block of the counting sweep
 
 template <int NS, int CH>
-struct BucketCountSmem {
-    float buf[BWARPS][BST][NS][CH];
-    unsigned long long bar[BWARPS][BST];
-    u32 hist[BWARPS][NS][NBKT];      // each warp's counts since its last flush
-    u32 slo[BWARPS][NS][NBKT];       // and fixed-point sums, as sums of the low 16 bits
-    u32 shi[BWARPS][NS][NBKT];       //   and of the (signed) high 16 bits of every value's Q
+struct CellCountSmem {
+    float buf[CWARPS][BST][NS][CH];
+    unsigned long long bar[CWARPS][BST];
+    u32 tab[NS][NCLASS];
+    u32 cnt[NS][NCELL];              // the block's counts since its last flush
+    u32 lo[NS][NCELL];               // and sums of |Q|: low word,
+    u32 hi[NS][NCELL];               //   carries out of it
+    u32 abort;
 };
-constexpr u32 COUNT_FLUSH_CHUNKS = 32768 / 512;   // at most 32768 values per warp between flushes: the 16-bit sums fit
 
-// Sweep 1 of the grouping: survivors per bucket and their fixed-point sums.  NS = 1: dW; NS = 2:
-// both moment streams.
+// Sweep 1: survivors per cell and the sum of their |Q| (a cell holds one sign).  A block takes a
+// contiguous share of the tiles and goes through it tensor by tensor; its warps split the tensor's
+// tiles and add into one table in shared memory, flushed to the tensor's own with integer atomics.
+// NS = 1: dW; NS = 2: both moment streams.
 template <int NS, int CH>
-__global__ void __launch_bounds__(TPB) bucket_count_kernel(const TensorDesc* __restrict__ descs,
-                                                           const TensorState* __restrict__ st, int nt, u32 tiles,
-                                                           Workspace ws, int stream0, CallState* call) {
+__global__ void __launch_bounds__(CWARPS * 32) cell_count_kernel(const TensorDesc* __restrict__ descs,
+                                                                 const TensorState* __restrict__ st, int nt, u32 tiles,
+                                                                 Workspace ws, int stream0, CallState* call) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    BucketCountSmem<NS, CH>& sm = *reinterpret_cast<BucketCountSmem<NS, CH>*>(smem_raw);
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const u32 gw = blockIdx.x * BWARPS + warp, nw = gridDim.x * BWARPS;
-    const u32 wlo = (u32)(((u64)tiles * gw) / nw), whi = (u32)(((u64)tiles * (gw + 1)) / nw);
-    SegRing<NS, CH, BST> ring;
-    ring.init(&sm.buf[warp][0][0][0], sm.bar[warp], lane, wlo, whi);
-    const u32* tile_cnt = stream0 == 0 ? ws.tile_cnt_w : ws.tile_cnt_o;
-    const float* surv[NS];
-    BucketFn fn[NS];
-#pragma unroll
-    for (int k = 0; k < NS; ++k) {
-        surv[k] = ws.surv[stream0 + k];
-        fn[k] = BucketFn{0, 0, 0, 0};
-        for (int b = lane; b < NBKT; b += 32) { sm.hist[warp][k][b] = 0; sm.slo[warp][k][b] = 0; sm.shi[warp][k][b] = 0; }
-    }
-    __syncwarp();
-    int cur = -1;
-    u32 tb = 0, ntl = 0, since = 0;
-    float s1[NS], s2[NS];
-#pragma unroll
-    for (int k = 0; k < NS; ++k) { s1[k] = 0.f; s2[k] = 0.f; }
-
-    auto flush = [&](int tns) {
-        __syncwarp();
-#pragma unroll
-        for (int k = 0; k < NS; ++k)
-            for (int b = lane; b < NBKT; b += 32) {
-                const u32 c = sm.hist[warp][k][b];
-                if (c) {
-                    BucketStream& bk = ws.bst[tns].s[stream0 + k];
-                    atomicAdd(&bk.cnt[b], c);
-                    const s64 sum = ((s64)(int)sm.shi[warp][k][b] << 16) + (s64)sm.slo[warp][k][b];
-                    if (sum) atomicAdd(reinterpret_cast<u64*>(&bk.sum[b]), (u64)sum);
-                    sm.hist[warp][k][b] = 0; sm.slo[warp][k][b] = 0; sm.shi[warp][k][b] = 0;
-                }
-            }
-        since = 0;
-        __syncwarp();
-    };
-
-    while (ring.next_window(tile_cnt, lane, whi)) {
-        while (ring.have()) {
-            ring.issue_ahead(lane, surv);
-            const u32 tile = ring.tile();
-            if (cur < 0 || tile >= tb + ntl) {
-                if (cur >= 0) flush(cur);
-                cur = find_tensor(descs, nt, tile);
-                tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
-#pragma unroll
-                for (int k = 0; k < NS; ++k) {
-                    fn[k] = ws.bst[cur].s[stream0 + k].fn;
-                    s1[k] = st[cur].s[stream0 + k].scale1; s2[k] = st[cur].s[stream0 + k].scale2;
-                }
-            }
-            const u32 nel = ring.nel();
-            if (!ring.wait()) {
-                if (lane == 0) atomicOr(&call->flags, FLAG_TIMEOUT);
-                return;
-            }
-#pragma unroll
-            for (int k = 0; k < NS; ++k) {
-                const float* data = ring.stage() + k * CH;
-                u32* hist = sm.hist[warp][k];
-                u32* slo = sm.slo[warp][k];
-                u32* shi = sm.shi[warp][k];
-                const float a1 = s1[k], a2 = s2[k];
-                auto tally = [&](float x) {
-                    const u32 b = bucket_index(x, fn[k]);
-                    const int q = __float2int_rn(__fmul_rn(__fmul_rn(x, a1), a2));      // Q(x), |Q| < 2^31
-                    atomicAdd(&hist[b], 1u);
-                    atomicAdd(&slo[b], (u32)q & 0xffffu);
-                    atomicAdd(&shi[b], (u32)(q >> 16));
-                };
-                const u32 whole = nel / 4;                             // groups of four that exist entirely
-                for (u32 f = lane; f < whole; f += 32) {
-                    const float4 v = *reinterpret_cast<const float4*>(data + 4 * f);
-                    tally(v.x); tally(v.y); tally(v.z); tally(v.w);
-                }
-                if (lane < nel - 4 * whole) tally(data[4 * whole + lane]);
-            }
-            if (++since >= COUNT_FLUSH_CHUNKS * 512u / CH) flush(cur);
-            ring.advance();
-        }
-    }
-    if (cur >= 0) flush(cur);
-}
-
-// Where each bucket starts in the bucketed copy (exclusive prefix of the counts).
-__global__ void __launch_bounds__(NBKT) bucket_offsets_kernel(Workspace ws) {
-    __shared__ u32 wtot[NBKT / 32];
-    BucketStream& bk = ws.bst[blockIdx.x].s[blockIdx.y];
-    const int b = threadIdx.x, lane = b & 31, warp = b >> 5;
-    const u32 c = bk.cnt[b];
-    u32 incl = c;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const u32 v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
-    }
-    if (lane == 31) wtot[warp] = incl;
-    __syncthreads();
-    u32 base = 0;
-    for (int w = 0; w < warp; ++w) base += wtot[w];
-    bk.off[b] = base + incl - c;
-    bk.cursor[b] = base + incl - c;
-    if (b == NBKT - 1) bk.off[NBKT] = base + incl;
-}
-
-constexpr int SPT = 32;               // survivors a thread holds per window
-constexpr int SCAP = SPT * TPB;       // survivors staged per window of tiles (8192)
-
-struct ScatterSmem {
-    float val[SCAP];                 // the window's survivors sorted by bucket
-    unsigned char bid[SCAP];         // and their buckets
-    u32 cnt[NBKT];                   // survivors of the window per bucket
-    u32 lcur[NBKT];                  // next free place of each bucket in val[]
-    u32 delta[NBKT];                 // place in the bucketed copy minus place in val[], per bucket
-    u32 pre[33];                     // survivors before tile i of the window
-    u32 wtot[TPB / 32];
-    u32 wn;                          // tiles in the window
-};
-
-// Sweep 2 of the grouping: survivors into their buckets.
-// A block takes windows of tiles of one tensor holding at most SCAP survivors.  Every thread
-// loads its 32 survivors of the window at once (they stay in registers), the block counts them
-// per bucket, reserves room in every bucket of the bucketed copy with one integer atomic,
-// sorts the window by bucket in shared memory and writes each bucket's run with consecutive
-// threads (one 4-byte store per survivor straight to its bucket would be bound by the number
-// of write requests, not by bytes).
-__global__ void __launch_bounds__(TPB, 4) bucket_scatter_kernel(const TensorDesc* __restrict__ descs,
-                                                                const TensorState* __restrict__ st, int nt,
-                                                                u32 tiles, Workspace ws, int stream) {
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    ScatterSmem& sm = *reinterpret_cast<ScatterSmem*>(smem_raw);
+    CellCountSmem<NS, CH>& sm = *reinterpret_cast<CellCountSmem<NS, CH>*>(smem_raw);
+    if (call->flags & FLAG_TIMEOUT) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     u32 lo, hi;
     block_range(tiles, lo, hi);
-    const u32* tile_cnt = stream == 0 ? ws.tile_cnt_w : ws.tile_cnt_o;
-    const float* surv = ws.surv[stream];
-    int cur = -1;
-    u32 tb = 0, ntl = 0;
-    BucketFn fn = BucketFn{0, 0, 0, 0};
+    SegRing<NS, CH, BST> ring;
+    ring.init(&sm.buf[warp][0][0][0], sm.bar[warp], lane, lo, lo);
+    const u32* tile_cnt = stream0 == 0 ? ws.tile_cnt_w : ws.tile_cnt_o;
+    const float* surv[NS];
+#pragma unroll
+    for (int k = 0; k < NS; ++k) {
+        surv[k] = ws.surv[stream0 + k];
+        for (int c = tid; c < NCELL; c += CWARPS * 32) { sm.cnt[k][c] = 0; sm.lo[k][c] = 0; sm.hi[k][c] = 0; }
+    }
+    if (tid == 0) sm.abort = 0;
     u32 tile = lo;
     while (tile < hi) {
-        if (cur < 0 || tile >= tb + ntl) {
-            cur = find_tensor(descs, nt, tile);
-            tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
-            fn = ws.bst[cur].s[stream].fn;
-        }
-        const u32 wend = min(hi, tb + ntl);
-        if (warp == 0) {              // the window: leading tiles whose survivors fit the stage
-            const u32 c = tile + lane < wend ? tile_cnt[tile + lane] : 0u;
-            u32 incl = c;
+        const int cur = find_tensor(descs, nt, tile);
+        const u32 seg_end = min(hi, descs[cur].tile_begin + descs[cur].num_tiles);
+        float s1[NS], s2[NS];
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const u32 v = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += v;
-            }
-            const u32 ok = __ballot_sync(0xffffffffu, tile + lane < wend && incl <= (u32)SCAP);
-            sm.pre[lane] = incl - c;
-            if (lane == 31) sm.pre[32] = incl;
-            if (lane == 0) sm.wn = ok == 0xffffffffu ? 32u : (u32)__ffs((int)~ok) - 1u;
+        for (int k = 0; k < NS; ++k) {
+            for (int c = tid; c < NCLASS; c += CWARPS * 32) sm.tab[k][c] = ws.cst[cur].s[stream0 + k].tab[c];
+            s1[k] = st[cur].s[stream0 + k].scale1; s2[k] = st[cur].s[stream0 + k].scale2;
         }
-        sm.cnt[tid] = 0;
         __syncthreads();
-        const u32 wn = sm.wn, total = sm.pre[wn];
-        if (total) {
-            // this thread's survivors: window ranks tid, tid + 256, ...  (tile found by walking pre[])
-            float x[SPT];
-            u32 ti = 0;
-#pragma unroll
-            for (int k = 0; k < SPT; ++k) {
-                const u32 idx = k * TPB + tid;
-                x[k] = 0.f;
-                if (idx < total) {
-                    while (idx >= sm.pre[ti + 1]) ++ti;
-                    x[k] = surv[(u64)(tile + ti) * TILE + (idx - sm.pre[ti])];
+        const u32 n = seg_end - tile;
+        const u32 wlo = tile + (u32)(((u64)n * warp) / CWARPS), whi = tile + (u32)(((u64)n * (warp + 1)) / CWARPS);
+        ring.restart(wlo, whi);
+        bool alive = sm.abort == 0;
+        while (alive && ring.next_window(tile_cnt, lane, whi)) {
+            while (alive && ring.have()) {
+                ring.issue_ahead(lane, surv);
+                const u32 nel = ring.nel();
+                if (!ring.wait()) {
+                    if (lane == 0) { atomicOr(&call->flags, FLAG_TIMEOUT); sm.abort = 1; }
+                    alive = false;
+                    break;
                 }
-            }
-            u32 bk[SPT / 4];            // the buckets of x[], one byte each
 #pragma unroll
-            for (int g = 0; g < SPT / 4; ++g) {
-                u32 w = 0;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int k = 4 * g + j;
-                    const u32 b = bucket_of(x[k], fn);
-                    w |= b << (8 * j);
-                    if (k * TPB + tid < total) atomicAdd(&sm.cnt[b], 1u);
+                for (int k = 0; k < NS; ++k) {
+                    const float* data = ring.stage() + k * CH;
+                    const u32* tab = sm.tab[k];
+                    u32* cnt = sm.cnt[k];
+                    u32* slo = sm.lo[k];
+                    u32* shi = sm.hi[k];
+                    const float a1 = s1[k], a2 = s2[k];
+                    auto tally = [&](float x) {
+                        const u32 c = cell_of(x, tab);
+                        const u32 q = (u32)abs(__float2int_rn(__fmul_rn(__fmul_rn(x, a1), a2)));   // |Q(x)| < 2^31
+                        atomicAdd(&cnt[c], 1u);
+                        const u32 old = atomicAdd(&slo[c], q);
+                        if (old + q < old) atomicAdd(&shi[c], 1u);
+                    };
+                    const u32 whole = nel / 4;                             // groups of four that exist entirely
+                    for (u32 f = lane; f < whole; f += 32) {
+                        const float4 v = *reinterpret_cast<const float4*>(data + 4 * f);
+                        tally(v.x); tally(v.y); tally(v.z); tally(v.w);
+                    }
+                    if (lane < nel - 4 * whole) tally(data[4 * whole + lane]);
                 }
-                bk[g] = w;
+                ring.advance();
             }
-            __syncthreads();
-            {                          // exclusive prefix of the counts; room in the bucketed copy
-                const u32 c = sm.cnt[tid];
-                u32 incl = c;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const u32 v = __shfl_up_sync(0xffffffffu, incl, o);
-                    if (lane >= o) incl += v;
-                }
-                if (lane == 31) sm.wtot[warp] = incl;
-                __syncthreads();
-                u32 base = 0;
-                for (int w = 0; w < warp; ++w) base += sm.wtot[w];
-                sm.lcur[tid] = base + incl - c;
-                const u32 g = c ? atomicAdd(&ws.bst[cur].s[stream].cursor[tid], c) : 0u;
-                sm.delta[tid] = g - (base + incl - c);
-            }
-            __syncthreads();
-#pragma unroll
-            for (int k = 0; k < SPT; ++k) {
-                if (k * TPB + tid < total) {
-                    const u32 b = (bk[k / 4] >> (8 * (k & 3))) & 255u;
-                    const u32 r = atomicAdd(&sm.lcur[b], 1u);
-                    sm.val[r] = x[k];
-                    sm.bid[r] = (unsigned char)b;
-                }
-            }
-            __syncthreads();
-            float* dst = ws.bkt[stream] + (u64)tb * TILE;
-            for (u32 i = tid; i < total; i += TPB) dst[i + sm.delta[sm.bid[i]]] = sm.val[i];
         }
-        tile += wn;
         __syncthreads();
+#pragma unroll
+        for (int k = 0; k < NS; ++k) {
+            CellStream& cs = ws.cst[cur].s[stream0 + k];
+            u32* row = ws.km_rows[stream0 + k] + (u64)(blockIdx.x + cur) * NCELL;    // this block's share of the tensor
+            for (int c = tid; c < NCELL; c += CWARPS * 32) {
+                const u32 n_c = sm.cnt[k][c];
+                row[c] = n_c;
+                if (n_c) {
+                    atomicAdd(&cs.cnt[c], n_c);
+                    const u64 mag = ((u64)sm.hi[k][c] << 32) | sm.lo[k][c];
+                    if (mag) atomicAdd(&cs.mag[c], mag);
+                    sm.cnt[k][c] = 0; sm.lo[k][c] = 0; sm.hi[k][c] = 0;
+                }
+            }
+        }
+        __syncthreads();
+        if (sm.abort) return;
+        tile = seg_end;
     }
 }
 
-// The bucket each threshold falls into; the partial sums of the coming scan start at zero.
-// Threads idx, idx + stride, ... of the caller share the K - 1 thresholds.
-__device__ inline void plan_scan(const StreamState& s, BucketStream& bk, int K, int idx, int stride) {
-    for (int j = idx; j < K - 1; j += stride) {
-        bk.bstar[j] = bucket_of(s.thr[j], bk.fn);
-        bk.part_cnt[j] = 0;
-        bk.part_sum[j] = 0;
-    }
-}
-
-// Exclusive prefix of the bucket sums; plan of the first iteration.  Grid (tensors, 3).
-__global__ void __launch_bounds__(NBKT) bucket_prefix_kernel(const TensorState* __restrict__ st, Workspace ws, int K) {
-    __shared__ s64 wtot[NBKT / 32];
-    BucketStream& bk = ws.bst[blockIdx.x].s[blockIdx.y];
-    const int b = threadIdx.x, lane = b & 31, warp = b >> 5;
-    const s64 c = bk.sum[b];
-    s64 incl = c;
+// ---------------------------------------------------------------------------
+// Exclusive prefix over 4 x 1024 items, four consecutive ones per thread; the total to every thread.
+// wt: 32 words of shared memory.  Whole block of 1024 threads.
+template <typename T>
+__device__ inline T block_scan4(T (&v)[4], T* wt) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const T mine = v[0] + v[1] + v[2] + v[3];
+    T incl = mine;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-        const s64 v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
+        const T x = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += x;
     }
-    if (lane == 31) wtot[warp] = incl;
+    __syncthreads();                  // wt may still be read from the previous scan
+    if (lane == 31) wt[warp] = incl;
     __syncthreads();
-    s64 base = 0;
-    for (int w = 0; w < warp; ++w) base += wtot[w];
-    bk.sumpre[b] = base + incl - c;
-    if (b == NBKT - 1) bk.sumpre[NBKT] = base + incl;
-    plan_scan(st[blockIdx.x].s[blockIdx.y], bk, K, b, NBKT);
+    T base = 0, total = 0;
+    for (int w = 0; w < 32; ++w) {
+        if (w < warp) base += wt[w];
+        total += wt[w];
+    }
+    T run = base + incl - mine;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) { const T x = v[k]; v[k] = run; run += x; }
+    return total;
 }
 
-// One iteration's data pass: for threshold j of a stream, the survivors of its bucket that lie
-// at or below it.  Grid (work items, 3 * 14): a tensor has scan_n items that split each bucket.
-__global__ void __launch_bounds__(TPB) bucket_scan_kernel(const TensorDesc* __restrict__ descs,
-                                                          const TensorState* __restrict__ st, int nt,
-                                                          Workspace ws, int K) {
-    __shared__ s64 rsum[TPB / 32];
-    __shared__ u32 rcnt[TPB / 32];
-    int lo = 0, hi = nt - 1;                       // tensor that owns this work item
-    while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (descs[mid].scan_first <= blockIdx.x) lo = mid; else hi = mid - 1;
-    }
-    const int t = lo, k = blockIdx.y / (K - 1), j = blockIdx.y % (K - 1);
-    const u32 split = blockIdx.x - descs[t].scan_first, nsplit = descs[t].scan_n;
-    BucketStream& bk = ws.bst[t].s[k];
-    const u32 b = bk.bstar[j];
-    const u32 b_lo = bk.off[b], n = bk.off[b + 1] - b_lo;
-    if (n == 0) return;
-    const u32 a = b_lo + (u32)(((u64)n * split) / nsplit), e = b_lo + (u32)(((u64)n * (split + 1)) / nsplit);
-    const StreamState& ss = st[t].s[k];
-    const float thr = ss.thr[j], s1 = ss.scale1, s2 = ss.scale2;
-    const float* data = ws.bkt[k] + (u64)descs[t].tile_begin * TILE;
-    u32 cnt = 0;
-    s64 sum = 0;
-    u32 i = a + threadIdx.x;
-    for (; i + 7 * TPB < e; i += 8 * TPB) {                 // eight independent loads in flight
-        float x[8];
+constexpr int PLAN_THREADS = 1024;
+
+// Block of a grid of g blocks whose share [tiles * b / g, tiles * (b + 1) / g) holds tile x (see block_range).
+__device__ inline u32 block_of_tile(u32 x, u32 tiles, u32 g) {
+    u32 b = (u32)(((u64)x * g) / tiles);
+    while ((u32)(((u64)tiles * (b + 1)) / g) <= x) ++b;
+    return b;
+}
+
+// Prefixes of the cell table; the cells the coming iterations will need; their places in the
+// gathered copy.  One block per (tensor, stream).  round 0 predicts; a later round (only for a
+// stream that met a cell it had not gathered) takes every cell.
+__global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDesc* __restrict__ descs,
+                                                                 TensorState* __restrict__ st, Workspace ws, int K,
+                                                                 int iters, int margin, int round, u32 tiles,
+                                                                 u32 grid_w, u32 grid_o) {
+    __shared__ u32 tab[NCLASS];
+    __shared__ u32 selw[NCELL / 32];
+    __shared__ float cent[KCAP], thr[KCAP], cnew[KCAP];
+    __shared__ double Lp[KCAP], Sp[KCAP];
+    __shared__ s64 wt64[32];
+    __shared__ u32 wt32[32];
+    const int t = blockIdx.x, stream = blockIdx.y, tid = threadIdx.x;
+    CellStream& cs = ws.cst[t].s[stream];
+    if (!cs.active) return;
+    const StreamState& s = st[t].s[stream];
+    const u32 nnz = stream == 0 ? st[t].nnz_w : st[t].nnz_o;
+    const u32 c0 = 4u * tid;                           // this thread's cells
+    u32 cnt[4];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) x[j] = __ldcs(data + i + j * TPB);
+    for (int k = 0; k < 4; ++k) cnt[k] = cs.cnt[c0 + k];
+    if (tid < NCELL / 32) selw[tid] = 0xffffffffu;
+    if (round == 0) {
+        const u32 first_pos = cs.first_pos;
+        u32 pc[4];
+        s64 ps[4];
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-            if (!(x[j] > thr)) {
-                ++cnt;
-                sum += __float2int_rn(__fmul_rn(__fmul_rn(x[j], s1), s2));
+        for (int k = 0; k < 4; ++k) {
+            pc[k] = cnt[k];
+            const s64 mag = (s64)cs.mag[c0 + k];
+            ps[k] = c0 + k < first_pos ? -mag : mag;
+        }
+        const u32 tc = block_scan4(pc, wt32);
+        const s64 ts = block_scan4(ps, wt64);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { cs.cntpre[c0 + k] = pc[k]; cs.sumpre[c0 + k] = ps[k]; }
+        if (tid == 0) { cs.cntpre[NCELL] = tc; cs.sumpre[NCELL] = ts; }
+        const bool predict = nnz > SMALL_STREAM && margin < NCELL;
+        if (predict) {
+            if (tid < NCELL / 32) selw[tid] = 0;
+            if (tid < NCLASS) tab[tid] = cs.tab[tid];
+            if (tid < KCAP) { cent[tid] = s.cent[tid]; thr[tid] = s.thr[tid]; }
+        }
+        __syncthreads();                               // also: this block's prefixes are visible to it
+        if (predict && margin >= 0) {
+            const double scale = __longlong_as_double((s64)(s.e - 30 + 1023) << 52);
+            for (int it = (int)cs.it_done; it < iters; ++it) {
+                if (tid < K - 1) {
+                    const float tj = thr[tid];
+                    const u32 c = cell_of(tj, tab);
+                    for (int d = -margin; d <= margin; ++d) {
+                        const int cc = (int)c + d;
+                        if (cc >= 0 && cc < NCELL) atomicOr(&selw[cc >> 5], 1u << (cc & 31));
+                    }
+                    // the share of cell c at or below the threshold, by its place between the cell's edges
+                    const u32 bits = __float_as_uint(tj), sh = 23u - (tab[bits >> 23] & 31u);
+                    const u32 a_lo = (bits & 0x7fffffffu) >> sh << sh;
+                    const u32 a_hi = min(a_lo + (1u << sh), 0x7f7fffffu);
+                    const double v_lo = (double)__uint_as_float(a_lo), v_hi = (double)__uint_as_float(a_hi);
+                    double f = v_hi > v_lo ? (fabs((double)tj) - v_lo) / (v_hi - v_lo) : 1.0;
+                    f = fmin(fmax(f, 0.0), 1.0);
+                    if (bits >> 31) f = 1.0 - f;
+                    Lp[tid] = (double)cs.cntpre[c] + f * (double)(cs.cntpre[c + 1] - cs.cntpre[c]);
+                    Sp[tid] = (double)cs.sumpre[c] + f * (double)(cs.sumpre[c + 1] - cs.sumpre[c]);
+                } else if (tid == K - 1) {
+                    Lp[tid] = (double)tc;
+                    Sp[tid] = (double)ts;
+                }
+                __syncthreads();
+                float c = __uint_as_float(0x7f800000u);
+                if (tid < K) {
+                    const double n = tid == 0 ? Lp[0] : Lp[tid] - Lp[tid - 1];
+                    const double sum = tid == 0 ? Sp[0] : Sp[tid] - Sp[tid - 1];
+                    c = n >= 0.5 ? __double2float_rn(sum / n * scale) : cent[tid];
+                    cnew[tid] = c;
+                }
+                __syncthreads();
+                if (tid < K) {
+                    int rank = 0;
+                    for (int i = 0; i < K; ++i) {
+                        const float o = cnew[i];
+                        rank += (o < c) || (o == c && i < tid);
+                    }
+                    cent[rank] = c;
+                }
+                __syncthreads();
+                set_thresholds(cent, thr, K, tid, PLAN_THREADS);
+                __syncthreads();
             }
+        }
     }
-    for (; i < e; i += TPB) {
-        const float x = __ldcs(data + i);
+    __syncthreads();
+    // places of the selected cells in the gathered copy; the gather cursors start at zero
+    u32 g[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) g[k] = ((selw[(c0 + k) >> 5] >> ((c0 + k) & 31)) & 1u) ? cnt[k] : 0u;
+    block_scan4(g, wt32);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) cs.mag[c0 + k] = (u64)g[k];
+    if (tid < NCELL / 32) cs.sel[tid] = selw[tid];
+    // Where every block of the sweeps puts its values of a cell: the blocks that share the tensor,
+    // in order, each after the ones before it (the counting sweep left their counts in km_rows).
+    const u32 grid = stream == 0 ? grid_w : grid_o;
+    const u32 tb = descs[t].tile_begin, tl = tb + descs[t].num_tiles - 1;
+    const u32 b0 = block_of_tile(tb, tiles, grid), b1 = block_of_tile(tl, tiles, grid);
+    const u32* rows = ws.km_rows[stream];
+    u32* pos = ws.km_pos[stream];
+    for (u32 b = b0; b <= b1; ++b) {
+        const u64 r = (u64)(b + (u32)t) * NCELL + c0;
+        const uint4 n = *reinterpret_cast<const uint4*>(rows + r);
+        *reinterpret_cast<uint4*>(pos + r) = make_uint4(g[0], g[1], g[2], g[3]);
+        g[0] += n.x; g[1] += n.y; g[2] += n.z; g[3] += n.w;
+    }
+}
+
+// ---------------------------------------------------------------------------
+template <int NS, int CH>
+struct CellGatherSmem {
+    float buf[CWARPS][BST][NS][CH];
+    unsigned long long bar[CWARPS][BST];
+    u32 tab[NS][NCLASS];
+    u32 sel[NS][NCELL / 32];
+    u32 cur[NS][NCELL];              // where the block's next value of each selected cell goes
+    u32 abort;
+};
+
+// Sweep 2: the values of the selected cells into the gathered copy, every cell contiguous (the
+// order inside a cell is arbitrary: what is taken from it are integer sums).  Same grid and same
+// shares of the tiles as the counting sweep, so every block owns a reserved run inside every cell
+// (km_pos) and no two blocks ever contend for a place.  A tensor with nothing to gather is skipped.
+template <int NS, int CH>
+__global__ void __launch_bounds__(CWARPS * 32) cell_gather_kernel(const TensorDesc* __restrict__ descs, int nt, u32 tiles,
+                                                                  Workspace ws, int stream0, CallState* call, int round) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    CellGatherSmem<NS, CH>& sm = *reinterpret_cast<CellGatherSmem<NS, CH>*>(smem_raw);
+    if (call->flags & FLAG_TIMEOUT) return;
+    if (round > 0 && *ws.km_pending == 0) return;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    u32 lo, hi;
+    block_range(tiles, lo, hi);
+    SegRing<NS, CH, BST> ring;
+    ring.init(&sm.buf[warp][0][0][0], sm.bar[warp], lane, lo, lo);
+    const u32* tile_cnt = stream0 == 0 ? ws.tile_cnt_w : ws.tile_cnt_o;
+    const float* surv[NS];
+#pragma unroll
+    for (int k = 0; k < NS; ++k) surv[k] = ws.surv[stream0 + k];
+    if (tid == 0) sm.abort = 0;
+    u32 tile = lo;
+    while (tile < hi) {
+        const int cur = find_tensor(descs, nt, tile);
+        const u32 tb = descs[cur].tile_begin;
+        const u32 seg_end = min(hi, tb + descs[cur].num_tiles);
+        bool any = false;
+#pragma unroll
+        for (int k = 0; k < NS; ++k) any |= ws.cst[cur].s[stream0 + k].active != 0;
+        if (!any) { tile = seg_end; continue; }           // the same for the whole block
+#pragma unroll
+        for (int k = 0; k < NS; ++k) {
+            const CellStream& cs = ws.cst[cur].s[stream0 + k];
+            const bool act = cs.active != 0;
+            const u32* pos = ws.km_pos[stream0 + k] + (u64)(blockIdx.x + cur) * NCELL;
+            for (int c = tid; c < NCLASS; c += CWARPS * 32) sm.tab[k][c] = cs.tab[c];
+            for (int c = tid; c < NCELL / 32; c += CWARPS * 32) sm.sel[k][c] = act ? cs.sel[c] : 0u;
+            for (int c = tid; c < NCELL; c += CWARPS * 32) sm.cur[k][c] = pos[c];
+        }
+        __syncthreads();
+        const u32 n = seg_end - tile;
+        const u32 wlo = tile + (u32)(((u64)n * warp) / CWARPS), whi = tile + (u32)(((u64)n * (warp + 1)) / CWARPS);
+        ring.restart(wlo, whi);
+        bool alive = sm.abort == 0;
+        while (alive && ring.next_window(tile_cnt, lane, whi)) {
+            while (alive && ring.have()) {
+                ring.issue_ahead(lane, surv);
+                const u32 nel = ring.nel();
+                if (!ring.wait()) {
+                    if (lane == 0) { atomicOr(&call->flags, FLAG_TIMEOUT); sm.abort = 1; }
+                    alive = false;
+                    break;
+                }
+#pragma unroll
+                for (int k = 0; k < NS; ++k) {
+                    const float* data = ring.stage() + k * CH;
+                    const u32* tab = sm.tab[k];
+                    const u32* sel = sm.sel[k];
+                    u32* cursor = sm.cur[k];
+                    float* out = ws.bkt[stream0 + k] + (u64)tb * TILE;
+                    auto file = [&](float x) {
+                        const u32 c = cell_of(x, tab);
+                        if ((sel[c >> 5] >> (c & 31)) & 1u) out[atomicAdd(&cursor[c], 1u)] = x;
+                    };
+                    const u32 whole = nel / 4;
+                    for (u32 f = lane; f < whole; f += 32) {
+                        const float4 v = *reinterpret_cast<const float4*>(data + 4 * f);
+                        file(v.x); file(v.y); file(v.z); file(v.w);
+                    }
+                    if (lane < nel - 4 * whole) file(data[4 * whole + lane]);
+                }
+                ring.advance();
+            }
+        }
+        __syncthreads();
+        if (sm.abort) return;
+        tile = seg_end;
+    }
+}
+
+// ---------------------------------------------------------------------------
+constexpr int IT_THREADS = 1024;
+constexpr int IT_WARPS = IT_THREADS / 32;
+constexpr int IT_PARTS = 4;          // at most this many warps share one threshold's cell
+
+// Count and fixed-point sum of the values of data[a, e) at or below thr; whole warp.
+__device__ __forceinline__ void scan_range(const float* __restrict__ data, u32 a, u32 e, float thr, float s1,
+                                           float s2, int lane, u32& cnt, s64& sum) {
+    auto test = [&](float x) {
         if (!(x > thr)) {
             ++cnt;
             sum += __float2int_rn(__fmul_rn(__fmul_rn(x, s1), s2));
         }
-    }
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    cnt = __reduce_add_sync(0xffffffffu, cnt);
+    };
+    const u32 h = min(e, (a + 3u) & ~3u);                    // up to three values before a 16-byte boundary
+    if (a + lane < h) test(__ldg(data + a + lane));
+    const u32 be = h + ((e - h) & ~3u);
+    for (u32 i = h + 4u * lane; i < be; i += 512u) {         // four 16-byte loads in flight per lane
+        float4 v[4];
 #pragma unroll
-    for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    if (lane == 0) { rcnt[warp] = cnt; rsum[warp] = sum; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        u64 c = 0; s64 s = 0;
-        for (int w = 0; w < TPB / 32; ++w) { c += rcnt[w]; s += rsum[w]; }
-        if (c) {
-            atomicAdd(&bk.part_cnt[j], c);
-            atomicAdd(reinterpret_cast<u64*>(&bk.part_sum[j]), (u64)s);
-        }
+        for (int k = 0; k < 4; ++k)
+            if (i + 128u * k < be) v[k] = __ldg(reinterpret_cast<const float4*>(data + i + 128u * k));
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (i + 128u * k < be) { test(v[k].x); test(v[k].y); test(v[k].z); test(v[k].w); }
     }
+    if (be + lane < e) test(__ldg(data + be + lane));
 }
 
-// New centres from the finished scan; one block per (tensor, stream), thread j = cluster j.
-// L_j = survivors at or below threshold j = whole buckets below its bucket + the scanned part;
-// cluster k has L_k - L_(k-1) members (L_-1 = 0, L_(K-1) = all), and its sum likewise.
-__global__ void __launch_bounds__(KCAP) bucket_update_kernel(TensorState* __restrict__ st, Workspace ws, int K) {
+// The exact iterations of one stream, from iteration it_done on: one block per (tensor, stream).
+// L_j = survivors at or below threshold j = the cells below its cell, whole, + the part of its own
+// cell found by looking at the gathered values; cluster k has L_k - L_(k-1) members (L_-1 = 0,
+// L_(K-1) = all), and its sum likewise.  If a threshold's cell has values and was not gathered,
+// the stream stops here, stays active and is counted in km_pending.
+__global__ void __launch_bounds__(IT_THREADS) kmeans_iterate_kernel(const TensorDesc* __restrict__ descs,
+                                                                    TensorState* __restrict__ st, Workspace ws, int K,
+                                                                    int iters, const CallState* call) {
+    __shared__ u32 tab[NCLASS];
+    __shared__ u32 selw[NCELL / 32];
+    __shared__ float cent[KCAP], thr[KCAP], cnew[KCAP];
+    __shared__ u32 cellj[KCAP];
+    __shared__ u32 pcnt[KCAP][IT_PARTS];
+    __shared__ s64 psum[KCAP][IT_PARTS];
     __shared__ u64 Ls[KCAP];
     __shared__ s64 Ss[KCAP];
-    __shared__ float cs[KCAP];
-    const int t = blockIdx.x, stream = blockIdx.y, j = threadIdx.x;
+    if (call->flags & FLAG_TIMEOUT) return;
+    const int t = blockIdx.x, stream = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    CellStream& cs = ws.cst[t].s[stream];
+    if (!cs.active) return;
     StreamState& s = st[t].s[stream];
-    BucketStream& bk = ws.bst[t].s[stream];
-    u64 L = 0;
-    s64 S = 0;
-    if (j < K - 1) {
-        const u32 b = bk.bstar[j];
-        L = (u64)bk.off[b] + bk.part_cnt[j];
-        S = bk.sumpre[b] + bk.part_sum[j];
-    } else if (j == K - 1) {
-        L = bk.off[NBKT];
-        S = bk.sumpre[NBKT];
-    }
-    Ls[j] = L; Ss[j] = S;
+    if (tid < NCLASS) tab[tid] = cs.tab[tid];
+    if (tid < NCELL / 32) selw[tid] = cs.sel[tid];
+    if (tid < KCAP) { cent[tid] = s.cent[tid]; thr[tid] = s.thr[tid]; }
+    const float s1 = s.scale1, s2 = s.scale2;
+    const double scale = __longlong_as_double((s64)(s.e - 30 + 1023) << 52);
+    const float* data = ws.bkt[stream] + (u64)descs[t].tile_begin * TILE;
+    const int parts = max(1, min(IT_PARTS, IT_WARPS / max(K - 1, 1)));
     __syncthreads();
-    float c = __uint_as_float(0x7f800000u);
-    if (j < K) {
-        const u64 n = j == 0 ? L : L - Ls[j - 1];
-        const s64 sum = j == 0 ? S : S - Ss[j - 1];
-        c = s.cent[j];
-        if (n) {
-            const double mean = __ll2double_rn(sum) / __ull2double_rn(n);
-            const double scale = __longlong_as_double((s64)(s.e - 30 + 1023) << 52);
-            c = __double2float_rn(mean * scale);
+    int it = (int)cs.it_done;
+    for (; it < iters; ++it) {
+        bool ok = true;
+        if (tid < K - 1) {
+            const u32 c = cell_of(thr[tid], tab);
+            cellj[tid] = c;
+            ok = ((selw[c >> 5] >> (c & 31)) & 1u) || cs.cntpre[c + 1] == cs.cntpre[c];
         }
-    }
-    cs[j] = c;
-    __syncthreads();
-    if (j < K) {                      // sort ascending: rank of each centre among the K (ties by index)
-        int rank = 0;
-        for (int i = 0; i < K; ++i) {
-            const float o = cs[i];
-            rank += (o < c) || (o == c && i < j);
+        if (__syncthreads_or(!ok)) break;
+        for (int item = warp; item < (K - 1) * parts; item += IT_WARPS) {
+            const int j = item / parts, p = item - j * parts;
+            const u32 c = cellj[j];
+            u32 cnt = 0;
+            s64 sum = 0;
+            if ((selw[c >> 5] >> (c & 31)) & 1u) {
+                const u32 b = (u32)cs.mag[c], n = cs.cntpre[c + 1] - cs.cntpre[c];
+                scan_range(data, b + (u32)(((u64)n * p) / parts), b + (u32)(((u64)n * (p + 1)) / parts), thr[j], s1, s2,
+                           lane, cnt, sum);
+            }
+            cnt = __reduce_add_sync(0xffffffffu, cnt);
+#pragma unroll
+            for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            if (lane == 0) { pcnt[j][p] = cnt; psum[j][p] = sum; }
         }
-        s.cent[rank] = c;
+        __syncthreads();
+        u64 L = 0;
+        s64 S = 0;
+        if (tid < K - 1) {
+            const u32 c = cellj[tid];
+            L = cs.cntpre[c];
+            S = cs.sumpre[c];
+            for (int p = 0; p < parts; ++p) { L += pcnt[tid][p]; S += psum[tid][p]; }
+        } else if (tid == K - 1) {
+            L = cs.cntpre[NCELL];
+            S = cs.sumpre[NCELL];
+        }
+        if (tid < KCAP) { Ls[tid] = L; Ss[tid] = S; }
+        __syncthreads();
+        float c = __uint_as_float(0x7f800000u);
+        if (tid < K) {
+            const u64 n = tid == 0 ? L : L - Ls[tid - 1];
+            const s64 sum = tid == 0 ? S : S - Ss[tid - 1];
+            c = cent[tid];
+            if (n) c = __double2float_rn(__ll2double_rn(sum) / __ull2double_rn(n) * scale);
+            cnew[tid] = c;
+        }
+        __syncthreads();
+        if (tid < K) {                    // sort ascending: rank of each centre among the K (ties by index)
+            int rank = 0;
+            for (int i = 0; i < K; ++i) {
+                const float o = cnew[i];
+                rank += (o < c) || (o == c && i < tid);
+            }
+            cent[rank] = c;
+        }
+        __syncthreads();
+        set_thresholds(cent, thr, K, tid, IT_THREADS);
+        __syncthreads();
     }
-    __syncthreads();
-    set_thresholds(s, K, j, KCAP);
-    __syncthreads();
-    plan_scan(s, bk, K, j, KCAP);
+    if (tid < KCAP) { s.cent[tid] = cent[tid]; s.thr[tid] = thr[tid]; }
+    if (tid == 0) {
+        cs.it_done = (u32)it;
+        if (it == iters) cs.active = 0;
+        else atomicAdd(ws.km_pending, 1u);
+    }
 }
 
 void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
-                   u32 scan_items, const Workspace& ws, const Params& p, CallState* call) {
+                   const Workspace& ws, const Params& p, CallState* call) {
     const int K = centres_of(p.bits);
-    kmeans_start_kernel<<<dim3(nt, 3), SAMPLE_MAX, 0, cfg.stream>>>(descs, st, ws, p.seed, K);
+    kmeans_start_kernel<<<dim3(nt, 3), SAMPLE_MAX, 0, cfg.stream>>>(descs, st, ws, p.seed, K, p.kmeans_iters);
     prof_mark(cfg, ST_KMEANS_START, 1);
     if (!tiles || p.kmeans_iters == 0) return;
-    const u32 grid = min((tiles + BWARPS - 1) / BWARPS, (u32)cfg.sms * 5u);
+    // the two sweeps of a stream use one grid: a block's share of the tiles is its share of every cell
+    const u32 grid_w = min(tiles, min((u32)KM_GRID_PER_SM_W * (u32)cfg.sms, (u32)KM_MAX_GRID));
+    const u32 grid_o = min(tiles, min((u32)cfg.sms, (u32)KM_MAX_GRID));
     {
-        const size_t m1 = sizeof(BucketCountSmem<1, 512>), m2 = sizeof(BucketCountSmem<2, 256>);
-        cudaFuncSetAttribute(bucket_count_kernel<1, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m1);
-        cudaFuncSetAttribute(bucket_count_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m2);
-        bucket_count_kernel<1, 512><<<grid, TPB, m1, cfg.stream>>>(descs, st, nt, tiles, ws, 0, call);
-        bucket_count_kernel<2, 256><<<grid, TPB, m2, cfg.stream>>>(descs, st, nt, tiles, ws, 1, call);
-        prof_mark(cfg, ST_BUCKET_IDS, 2);
+        const size_t m1 = sizeof(CellCountSmem<1, 256>), m2 = sizeof(CellCountSmem<2, 256>);
+        cudaFuncSetAttribute(cell_count_kernel<1, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m1);
+        cudaFuncSetAttribute(cell_count_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m2);
+        cell_count_kernel<1, 256><<<grid_w, CWARPS * 32, m1, cfg.stream>>>(descs, st, nt, tiles, ws, 0, call);
+        cell_count_kernel<2, 256><<<grid_o, CWARPS * 32, m2, cfg.stream>>>(descs, st, nt, tiles, ws, 1, call);
+        prof_mark(cfg, ST_CELL_COUNT, 2);
     }
-    bucket_offsets_kernel<<<dim3(nt, 3), NBKT, 0, cfg.stream>>>(ws);
-    {
-        const u32 sgrid = min(tiles, (u32)cfg.sms * 4u);
-        cudaFuncSetAttribute(bucket_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ScatterSmem));
-        for (int k = 0; k < 3; ++k)
-            bucket_scatter_kernel<<<sgrid, TPB, sizeof(ScatterSmem), cfg.stream>>>(descs, st, nt, tiles, ws, k);
-    }
-    prof_mark(cfg, ST_BUCKET_SCATTER, 4);
-    bucket_prefix_kernel<<<dim3(nt, 3), NBKT, 0, cfg.stream>>>(st, ws, K);
-    prof_mark(cfg, ST_BUCKET_SUM, 1);
-    for (int it = 0; it < p.kmeans_iters; ++it) {
-        bucket_scan_kernel<<<dim3(scan_items, 3 * (K - 1)), TPB, 0, cfg.stream>>>(descs, st, nt, ws, K);
-        prof_mark(cfg, ST_BUCKET_SCAN, 1);
-        bucket_update_kernel<<<dim3(nt, 3), KCAP, 0, cfg.stream>>>(st, ws, K);
-        prof_mark(cfg, ST_KMEANS_UPDATE, 1);
+    const size_t g1 = sizeof(CellGatherSmem<1, 256>), g2 = sizeof(CellGatherSmem<2, 256>);
+    cudaFuncSetAttribute(cell_gather_kernel<1, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g1);
+    cudaFuncSetAttribute(cell_gather_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g2);
+    for (int round = 0; round < 2; ++round) {
+        cell_plan_kernel<<<dim3(nt, 3), PLAN_THREADS, 0, cfg.stream>>>(descs, st, ws, K, p.kmeans_iters, p.km_margin, round,
+                                                                     tiles, grid_w, grid_o);
+        if (round == 0) prof_mark(cfg, ST_CELL_PLAN, 1);
+        cell_gather_kernel<1, 256><<<grid_w, CWARPS * 32, g1, cfg.stream>>>(descs, nt, tiles, ws, 0, call, round);
+        cell_gather_kernel<2, 256><<<grid_o, CWARPS * 32, g2, cfg.stream>>>(descs, nt, tiles, ws, 1, call, round);
+        if (round == 0) prof_mark(cfg, ST_CELL_GATHER, 2);
+        kmeans_iterate_kernel<<<dim3(nt, 3), IT_THREADS, 0, cfg.stream>>>(descs, st, ws, K, p.kmeans_iters, call);
+        prof_mark(cfg, round == 0 ? ST_KMEANS_ITERATE : ST_KMEANS_RETRY, round == 0 ? 1 : 4);
     }
 }
 

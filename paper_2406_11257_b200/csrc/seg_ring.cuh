@@ -34,6 +34,12 @@ struct SegRing {
         }
         __syncwarp();
     }
+    // A new run of tiles for the same ring; nothing may be in flight (every issued chunk has been
+    // consumed), so the barriers keep their phases.
+    __device__ void restart(u32 wlo, u32 whi_) {
+        whi = whi_; w0 = wlo; wn = 0;
+        it = ct = 32; i_cnt = c_cnt = ic = cc = 0; mycnt = 0; nz = 0;
+    }
     // first non-empty tile of the window after position i (i = -1: from the start); 32 if none
     __device__ u32 next_tile(int i) const {
         const u32 m = i >= 31 ? 0u : nz & (0xffffffffu << (i + 1));
@@ -47,7 +53,7 @@ struct SegRing {
         w0 += wn;
         if (w0 >= whi) { wn = 0; return false; }
         wn = min(32u, min(limit, whi) - w0);
-        mycnt = (u32)lane < wn ? tile_cnt[w0 + lane] : 0u;
+        mycnt = (u32)lane < wn ? min(tile_cnt[w0 + lane], (u32)TILE) : 0u;   // a count never leads out of its segment
         nz = __ballot_sync(0xffffffffu, mycnt != 0);
         it = ct = next_tile(-1);
         i_cnt = c_cnt = it < 32 ? __shfl_sync(0xffffffffu, mycnt, it) : 0u;
@@ -99,30 +105,12 @@ struct SegRing {
 // Cluster of x = number of thresholds strictly below it.  thr_row: 16 fp32 thresholds
 // (ascending, +inf from the 15th on, none of them -0) in shared memory; t3, t7, t11 are copies
 // in registers.  Returns 4 * cluster.
-// "x > t" is read off the sign of t - x: with gradual underflow the difference of two distinct
-// floats is never rounded to zero, and t - x = +0 when they are equal.  This keeps the search
-// on the floating-point and multiply-add pipes.
-__device__ __forceinline__ u32 gt_bit(float t, float x) { return __float_as_uint(__fsub_rn(t, x)) >> 31; }
-
 __device__ __forceinline__ u32 find_cluster4(float x, float t3, float t7, float t11, const char* thr_row) {
     u32 p = x > t7 ? 32u : 0u;
     p += (x > (p ? t11 : t3)) ? 16u : 0u;
     p += (x > *reinterpret_cast<const float*>(thr_row + p + 4)) ? 8u : 0u;
     p += (x > *reinterpret_cast<const float*>(thr_row + p)) ? 4u : 0u;
     return p;
-}
-
-// cell += q * 2^16 + 1: a 48-bit signed sum above a 16-bit count (at most 65535 additions
-// between two flushes).
-__device__ __forceinline__ void cell_add(u64* cell, int q) {
-    u64 v;
-    asm("mad.wide.s32 %0, %1, 65536, %2;" : "=l"(v) : "r"(q), "l"(*cell));
-    const u32 lo = (u32)v + 1u;            // the count field cannot carry out of the low word
-    *cell = (v & 0xffffffff00000000ull) | lo;
-}
-__device__ __forceinline__ void cell_split(u64 v, s64& sum, s64& cnt) {
-    cnt = (s64)(v & 0xffffull);
-    sum = (s64)v >> 16;
 }
 
 }  // namespace excp

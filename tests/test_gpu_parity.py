@@ -157,6 +157,33 @@ def test_outlier_residuals_and_run_to_run_determinism(handle):
         assert o2 == offs and torch.equal(b2[:offs[-1]], blob[:offs[-1]])
 
 
+def test_centres_do_not_depend_on_which_cells_were_gathered(handle):
+    """The K-means iterations read only the value cells their thresholds fall into.  Whatever the first
+    round gathers (nothing: margin -1, so every stream takes the complete second round; only the
+    predicted cells: 0; more: 1, 5), the records are the oracle's plain Lloyd iterations."""
+    n = 2_000_000
+    dq = [synth.make_quad(n, 21, 0, device=DEV), synth.make_quad(70_000, 21, 1, device=DEV, outlier_frac=0.01)]
+    h = binding.Handle(workspace_numel=n + 80_000)
+    try:
+        for bits in (4, 2):
+            p = binding.Params(median_source=binding.MEDIAN_ABS_RESIDUAL, bits=bits, seed=5)
+            ref = None
+            for margin in (1, -1, 0, 5):
+                h.set_kmeans_margin(margin)
+                bound = sum(binding.compress_bound(q[0].numel(), bits) for q in dq)
+                blob = torch.full((bound,), 0xCD, dtype=torch.uint8, device=DEV)
+                offs, stats = h.compress_checkpoint(p, dq, blob)
+                if ref is None:
+                    check_against_oracle(p, to_np(dq), blob, offs, stats)
+                    ref = (blob[:offs[-1]].clone(), offs)
+                else:
+                    assert offs == ref[1] and torch.equal(blob[:offs[-1]], ref[0]), (bits, margin)
+        with pytest.raises(binding.ExcpError):
+            h.set_kmeans_margin(-2)
+    finally:
+        h.close()
+
+
 def test_degenerate_value_patterns(handle):
     n = 20000
     base = rand_quad_np(n, 400)
@@ -352,7 +379,9 @@ def test_profile_counts_launches_and_times_stages(handle):
     try:
         handle.compress_tensor(binding.Params(median_source=1, kmeans_iters=10), *dq[0], blob)
         ms, launches = handle.profile_read()
-        assert launches == 11 + 1 + 2 + 1 + 2 + 5 + 10 * 2 + 2 + 2 + 1
-        assert ms["mask_compact"] > 0 and ms["bucket_scan"] > 0 and ms["decode"] == 0
+        # statistics, mask sweep, scan + layout, K-means (start, 2 counting sweeps, plan, 2 gathers, iterations,
+        # the second round's 4), header + edges, 2 packing sweeps, bitmaps
+        assert launches == 11 + 1 + 2 + (1 + 2 + 1 + 2 + 1 + 4) + 2 + 2 + 1
+        assert ms["mask_compact"] > 0 and ms["kmeans_iterate"] > 0 and ms["decode"] == 0
     finally:
         handle.profile_enable(False)
