@@ -52,6 +52,7 @@ struct excp_handle_s {
     int sms = 0;
     size_t cap_tiles = 0;
     Workspace ws{};
+    KmArrays km{};
     TensorState* d_state = nullptr;      // MAX_GROUP_TENSORS
     DecState* d_dstate = nullptr;        // MAX_GROUP_TENSORS
     CallState* d_call = nullptr;
@@ -167,7 +168,7 @@ bool run_group(excp_handle h, const LaunchCfg& cfg, const TensorDesc* descs, int
     if (!check(h, cudaMemsetAsync(h->ws.cst, 0, nt * sizeof(CellState), cfg.stream))) return false;
     launch_stats(cfg, descs, h->d_state, nt, tiles, h->ws, p, h->d_call);
     launch_mask_compact(cfg, descs, h->d_state, nt, tiles, h->ws, p, h->d_call, blob_capacity);
-    if (!(p.flags & OPT_NO_QUANT)) launch_kmeans(cfg, descs, h->d_state, nt, tiles, h->ws, p, h->d_call);
+    if (!(p.flags & OPT_NO_QUANT)) launch_kmeans(cfg, descs, h->d_state, nt, tiles, h->ws, h->km, p, h->d_call);
     launch_pack(cfg, descs, h->d_state, nt, tiles, h->ws, p, blob, h->d_call, results);
     return check(h, cudaGetLastError());
 }
@@ -237,11 +238,11 @@ excp_status excp_create(excp_handle* out, int device, size_t workspace_numel) {
             ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.bkt[k]), elems * sizeof(float)));
         }
         ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.cst), MAX_GROUP_TENSORS * sizeof(CellState)));
-        ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.km_pending), sizeof(u32)));
+        ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->km.pending), sizeof(u32)));
         const size_t rows = (size_t)std::min(h->sms * 2, (int)KM_MAX_GRID) + MAX_GROUP_TENSORS;
         for (int k = 0; k < 3 && ok; ++k) {
-            ok = check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.km_rows[k]), rows * NCELL * sizeof(u32)));
-            ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.km_pos[k]), rows * NCELL * sizeof(u32)));
+            ok = check(h, cudaMalloc(reinterpret_cast<void**>(&h->km.rows[k]), rows * NCELL * sizeof(u32)));
+            ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->km.pos[k]), rows * NCELL * sizeof(u32)));
         }
         ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.bm_w), elems / 8));
         ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->ws.bm_o), elems / 8));
@@ -271,10 +272,10 @@ excp_status excp_destroy(excp_handle h) {
         if (h->ws.bkt[k]) cudaFree(h->ws.bkt[k]);
     }
     if (h->ws.cst) cudaFree(h->ws.cst);
-    if (h->ws.km_pending) cudaFree(h->ws.km_pending);
+    if (h->km.pending) cudaFree(h->km.pending);
     for (int k = 0; k < 3; ++k) {
-        if (h->ws.km_rows[k]) cudaFree(h->ws.km_rows[k]);
-        if (h->ws.km_pos[k]) cudaFree(h->ws.km_pos[k]);
+        if (h->km.rows[k]) cudaFree(h->km.rows[k]);
+        if (h->km.pos[k]) cudaFree(h->km.pos[k]);
     }
     if (h->ws.bm_w) cudaFree(h->ws.bm_w);
     if (h->ws.bm_o) cudaFree(h->ws.bm_o);

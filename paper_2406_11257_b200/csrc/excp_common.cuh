@@ -68,6 +68,7 @@ struct TensorDesc {              // built on the host, one per tensor of a group
     u64 tensor_index;            // position in the checkpoint (enters the start sample)
     u32 tile_begin;              // first tile of this tensor within the group
     u32 num_tiles;
+    u32 pad_[2];                 // 64 bytes: indexing the array is a shift
 };
 
 struct StreamState {             // K-means state of one stream (0 = dW, 1 = ea, 2 = eas)
@@ -144,10 +145,6 @@ struct CellState {
 struct Workspace {               // device arrays sized for cap_tiles tiles
     float* bkt[3];               // gathered copy: the survivors of the selected cells, cell after cell
     CellState* cst;              // per tensor of the group
-    u32* km_pending;             // streams whose first round of iterations met a cell that was not gathered
-    u32* km_rows[3];             // per stream: survivors per cell of every (block, tensor) share of the counting
-                                 //   sweep, row (block + tensor) of NCELL words
-    u32* km_pos[3];              // the same shape: where each share's values of a cell start in the gathered copy
     float* surv[3];              // survivors, each tile's compacted at the tile's own start
     u32* bm_w;                   // bitmaps, TILE_WORDS words per tile
     u32* bm_o;
@@ -155,6 +152,13 @@ struct Workspace {               // device arrays sized for cap_tiles tiles
     u32* tile_cnt_o;
     u32* tile_off_w;             // exclusive prefix of the counts within the tensor
     u32* tile_off_o;
+};
+
+struct KmArrays {                // further device arrays of the K-means stage alone
+    u32* pending;                // streams whose first round of iterations met a cell that was not gathered
+    u32* rows[3];                // per stream: survivors per cell of every (block, tensor) share of the counting
+                                 //   sweep, row (block + tensor) of NCELL words
+    u32* pos[3];                 // the same shape: where each share's values of a cell start in the gathered copy
 };
 
 struct Params {
@@ -373,7 +377,7 @@ void launch_stats(const LaunchCfg&, const TensorDesc* descs, TensorState* st, in
 void launch_mask_compact(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                          const Workspace& ws, const Params& p, CallState* call, u64 blob_capacity);
 void launch_kmeans(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
-                   const Workspace& ws, const Params& p, CallState* call);
+                   const Workspace& ws, const KmArrays& km, const Params& p, CallState* call);
 void launch_pack(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                  const Workspace& ws, const Params& p, unsigned char* blob, CallState* call,
                  TensorResult* results);

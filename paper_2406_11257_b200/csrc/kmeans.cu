@@ -57,7 +57,7 @@ constexpr u32 SMALL_STREAM = 16384;  // at most this many survivors: every cell 
 // One block per (tensor, stream).
 __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDesc* __restrict__ descs,
                                                                   TensorState* __restrict__ st,
-                                                                  Workspace ws, u64 seed, int K, int iters) {
+                                                                  Workspace ws, KmArrays km, u64 seed, int K, int iters) {
     __shared__ float smp[SAMPLE_MAX];
     __shared__ u32 chist[NCLASS];                     // sampled survivors per (sign, exponent) class
     __shared__ u32 wtot[NCLASS / 32];
@@ -70,7 +70,7 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
     const u32* toff = (stream == 0 ? ws.tile_off_w : ws.tile_off_o) + tb;
     const u32* tcnt = (stream == 0 ? ws.tile_cnt_w : ws.tile_cnt_o) + tb;
     const float* data = ws.surv[stream] + (u64)tb * TILE;
-    if (t == 0 && stream == 0 && tid == 0) *ws.km_pending = 0;
+    if (t == 0 && stream == 0 && tid == 0) *km.pending = 0;
     if (nnz == 0) {                                   // the zeroed state is a valid (one-cell) map
         if (tid < KCAP) { s.cent[tid] = 0.f; s.thr[tid] = __uint_as_float(0x7f800000u); }
         if (tid == 0) { cs.it_done = (u32)iters; cs.active = 0; }
@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
 }
 
 // ---------------------------------------------------------------------------
-constexpr int BST = 2;               // stages per warp
+constexpr int BST = 3;               // stages per warp
 constexpr int KM_GRID_PER_SM_W = 2;  // blocks per SM of the dW sweeps (the moment sweeps run one)
 constexpr int CWARPS = 16;           // warps per block of the counting sweep
 
@@ -174,7 +174,7 @@ struct CellCountSmem {
 template <int NS, int CH>
 __global__ void __launch_bounds__(CWARPS * 32) cell_count_kernel(const TensorDesc* __restrict__ descs,
                                                                  const TensorState* __restrict__ st, int nt, u32 tiles,
-                                                                 Workspace ws, int stream0, CallState* call) {
+                                                                 Workspace ws, KmArrays km, int stream0, CallState* call) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     CellCountSmem<NS, CH>& sm = *reinterpret_cast<CellCountSmem<NS, CH>*>(smem_raw);
     if (call->flags & FLAG_TIMEOUT) return;
@@ -231,9 +231,26 @@ __global__ void __launch_bounds__(CWARPS * 32) cell_count_kernel(const TensorDes
                         if (old + q < old) atomicAdd(&shi[c], 1u);
                     };
                     const u32 whole = nel / 4;                             // groups of four that exist entirely
-                    for (u32 f = lane; f < whole; f += 32) {
-                        const float4 v = *reinterpret_cast<const float4*>(data + 4 * f);
-                        tally(v.x); tally(v.y); tally(v.z); tally(v.w);
+                    for (u32 f = lane; f < whole; f += 64) {               // two groups per lane: all table look-ups first
+                        const bool two = f + 32 < whole;
+                        const float4 va = *reinterpret_cast<const float4*>(data + 4 * f);
+                        const float4 vb = two ? *reinterpret_cast<const float4*>(data + 4 * (f + 32)) : va;
+                        const float xs[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
+                        u32 c[8], q[8], old[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            c[i] = cell_of(xs[i], tab);
+                            q[i] = (u32)abs(__float2int_rn(__fmul_rn(__fmul_rn(xs[i], a1), a2)));
+                        }
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (i < 4 || two) atomicAdd(&cnt[c[i]], 1u);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (i < 4 || two) old[i] = atomicAdd(&slo[c[i]], q[i]);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if ((i < 4 || two) && old[i] + q[i] < old[i]) atomicAdd(&shi[c[i]], 1u);
                     }
                     if (lane < nel - 4 * whole) tally(data[4 * whole + lane]);
                 }
@@ -244,7 +261,7 @@ __global__ void __launch_bounds__(CWARPS * 32) cell_count_kernel(const TensorDes
 #pragma unroll
         for (int k = 0; k < NS; ++k) {
             CellStream& cs = ws.cst[cur].s[stream0 + k];
-            u32* row = ws.km_rows[stream0 + k] + (u64)(blockIdx.x + cur) * NCELL;    // this block's share of the tensor
+            u32* row = km.rows[stream0 + k] + (u64)(blockIdx.x + cur) * NCELL;    // this block's share of the tensor
             for (int c = tid; c < NCELL; c += CWARPS * 32) {
                 const u32 n_c = sm.cnt[k][c];
                 row[c] = n_c;
@@ -302,7 +319,7 @@ __device__ inline u32 block_of_tile(u32 x, u32 tiles, u32 g) {
 // gathered copy.  One block per (tensor, stream).  round 0 predicts; a later round (only for a
 // stream that met a cell it had not gathered) takes every cell.
 __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDesc* __restrict__ descs,
-                                                                 TensorState* __restrict__ st, Workspace ws, int K,
+                                                                 TensorState* __restrict__ st, Workspace ws, KmArrays km, int K,
                                                                  int iters, int margin, int round, u32 tiles,
                                                                  u32 grid_w, u32 grid_o) {
     __shared__ u32 tab[NCLASS];
@@ -404,8 +421,8 @@ __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDes
     const u32 grid = stream == 0 ? grid_w : grid_o;
     const u32 tb = descs[t].tile_begin, tl = tb + descs[t].num_tiles - 1;
     const u32 b0 = block_of_tile(tb, tiles, grid), b1 = block_of_tile(tl, tiles, grid);
-    const u32* rows = ws.km_rows[stream];
-    u32* pos = ws.km_pos[stream];
+    const u32* rows = km.rows[stream];
+    u32* pos = km.pos[stream];
     for (u32 b = b0; b <= b1; ++b) {
         const u64 r = (u64)(b + (u32)t) * NCELL + c0;
         const uint4 n = *reinterpret_cast<const uint4*>(rows + r);
@@ -431,11 +448,11 @@ struct CellGatherSmem {
 // (km_pos) and no two blocks ever contend for a place.  A tensor with nothing to gather is skipped.
 template <int NS, int CH>
 __global__ void __launch_bounds__(CWARPS * 32) cell_gather_kernel(const TensorDesc* __restrict__ descs, int nt, u32 tiles,
-                                                                  Workspace ws, int stream0, CallState* call, int round) {
+                                                                  Workspace ws, KmArrays km, int stream0, CallState* call, int round) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     CellGatherSmem<NS, CH>& sm = *reinterpret_cast<CellGatherSmem<NS, CH>*>(smem_raw);
     if (call->flags & FLAG_TIMEOUT) return;
-    if (round > 0 && *ws.km_pending == 0) return;
+    if (round > 0 && *km.pending == 0) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     u32 lo, hi;
     block_range(tiles, lo, hi);
@@ -459,7 +476,7 @@ __global__ void __launch_bounds__(CWARPS * 32) cell_gather_kernel(const TensorDe
         for (int k = 0; k < NS; ++k) {
             const CellStream& cs = ws.cst[cur].s[stream0 + k];
             const bool act = cs.active != 0;
-            const u32* pos = ws.km_pos[stream0 + k] + (u64)(blockIdx.x + cur) * NCELL;
+            const u32* pos = km.pos[stream0 + k] + (u64)(blockIdx.x + cur) * NCELL;
             for (int c = tid; c < NCLASS; c += CWARPS * 32) sm.tab[k][c] = cs.tab[c];
             for (int c = tid; c < NCELL / 32; c += CWARPS * 32) sm.sel[k][c] = act ? cs.sel[c] : 0u;
             for (int c = tid; c < NCELL; c += CWARPS * 32) sm.cur[k][c] = pos[c];
@@ -490,9 +507,23 @@ __global__ void __launch_bounds__(CWARPS * 32) cell_gather_kernel(const TensorDe
                         if ((sel[c >> 5] >> (c & 31)) & 1u) out[atomicAdd(&cursor[c], 1u)] = x;
                     };
                     const u32 whole = nel / 4;
-                    for (u32 f = lane; f < whole; f += 32) {
-                        const float4 v = *reinterpret_cast<const float4*>(data + 4 * f);
-                        file(v.x); file(v.y); file(v.z); file(v.w);
+                    for (u32 f = lane; f < whole; f += 64) {               // two groups per lane: all look-ups first
+                        const bool two = f + 32 < whole;
+                        const float4 va = *reinterpret_cast<const float4*>(data + 4 * f);
+                        const float4 vb = two ? *reinterpret_cast<const float4*>(data + 4 * (f + 32)) : va;
+                        const float xs[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
+                        u32 c[8];
+                        u32 hit = 0;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) c[i] = cell_of(xs[i], tab);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) hit |= ((sel[c[i] >> 5] >> (c[i] & 31)) & 1u) << i;
+                        if (!two) hit &= 15u;
+                        if (hit) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                if ((hit >> i) & 1u) out[atomicAdd(&cursor[c[i]], 1u)] = xs[i];
+                        }
                     }
                     if (lane < nel - 4 * whole) file(data[4 * whole + lane]);
                 }
@@ -540,7 +571,7 @@ __device__ __forceinline__ void scan_range(const float* __restrict__ data, u32 a
 // L_(K-1) = all), and its sum likewise.  If a threshold's cell has values and was not gathered,
 // the stream stops here, stays active and is counted in km_pending.
 __global__ void __launch_bounds__(IT_THREADS) kmeans_iterate_kernel(const TensorDesc* __restrict__ descs,
-                                                                    TensorState* __restrict__ st, Workspace ws, int K,
+                                                                    TensorState* __restrict__ st, Workspace ws, KmArrays km, int K,
                                                                     int iters, const CallState* call) {
     __shared__ u32 tab[NCLASS];
     __shared__ u32 selw[NCELL / 32];
@@ -626,14 +657,14 @@ __global__ void __launch_bounds__(IT_THREADS) kmeans_iterate_kernel(const Tensor
     if (tid == 0) {
         cs.it_done = (u32)it;
         if (it == iters) cs.active = 0;
-        else atomicAdd(ws.km_pending, 1u);
+        else atomicAdd(km.pending, 1u);
     }
 }
 
 void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
-                   const Workspace& ws, const Params& p, CallState* call) {
+                   const Workspace& ws, const KmArrays& km, const Params& p, CallState* call) {
     const int K = centres_of(p.bits);
-    kmeans_start_kernel<<<dim3(nt, 3), SAMPLE_MAX, 0, cfg.stream>>>(descs, st, ws, p.seed, K, p.kmeans_iters);
+    kmeans_start_kernel<<<dim3(nt, 3), SAMPLE_MAX, 0, cfg.stream>>>(descs, st, ws, km, p.seed, K, p.kmeans_iters);
     prof_mark(cfg, ST_KMEANS_START, 1);
     if (!tiles || p.kmeans_iters == 0) return;
     // the two sweeps of a stream use one grid: a block's share of the tiles is its share of every cell
@@ -643,21 +674,21 @@ void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* s
         const size_t m1 = sizeof(CellCountSmem<1, 256>), m2 = sizeof(CellCountSmem<2, 256>);
         cudaFuncSetAttribute(cell_count_kernel<1, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m1);
         cudaFuncSetAttribute(cell_count_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m2);
-        cell_count_kernel<1, 256><<<grid_w, CWARPS * 32, m1, cfg.stream>>>(descs, st, nt, tiles, ws, 0, call);
-        cell_count_kernel<2, 256><<<grid_o, CWARPS * 32, m2, cfg.stream>>>(descs, st, nt, tiles, ws, 1, call);
+        cell_count_kernel<1, 256><<<grid_w, CWARPS * 32, m1, cfg.stream>>>(descs, st, nt, tiles, ws, km, 0, call);
+        cell_count_kernel<2, 256><<<grid_o, CWARPS * 32, m2, cfg.stream>>>(descs, st, nt, tiles, ws, km, 1, call);
         prof_mark(cfg, ST_CELL_COUNT, 2);
     }
     const size_t g1 = sizeof(CellGatherSmem<1, 256>), g2 = sizeof(CellGatherSmem<2, 256>);
     cudaFuncSetAttribute(cell_gather_kernel<1, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g1);
     cudaFuncSetAttribute(cell_gather_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g2);
     for (int round = 0; round < 2; ++round) {
-        cell_plan_kernel<<<dim3(nt, 3), PLAN_THREADS, 0, cfg.stream>>>(descs, st, ws, K, p.kmeans_iters, p.km_margin, round,
+        cell_plan_kernel<<<dim3(nt, 3), PLAN_THREADS, 0, cfg.stream>>>(descs, st, ws, km, K, p.kmeans_iters, p.km_margin, round,
                                                                      tiles, grid_w, grid_o);
         if (round == 0) prof_mark(cfg, ST_CELL_PLAN, 1);
-        cell_gather_kernel<1, 256><<<grid_w, CWARPS * 32, g1, cfg.stream>>>(descs, nt, tiles, ws, 0, call, round);
-        cell_gather_kernel<2, 256><<<grid_o, CWARPS * 32, g2, cfg.stream>>>(descs, nt, tiles, ws, 1, call, round);
+        cell_gather_kernel<1, 256><<<grid_w, CWARPS * 32, g1, cfg.stream>>>(descs, nt, tiles, ws, km, 0, call, round);
+        cell_gather_kernel<2, 256><<<grid_o, CWARPS * 32, g2, cfg.stream>>>(descs, nt, tiles, ws, km, 1, call, round);
         if (round == 0) prof_mark(cfg, ST_CELL_GATHER, 2);
-        kmeans_iterate_kernel<<<dim3(nt, 3), IT_THREADS, 0, cfg.stream>>>(descs, st, ws, K, p.kmeans_iters, call);
+        kmeans_iterate_kernel<<<dim3(nt, 3), IT_THREADS, 0, cfg.stream>>>(descs, st, ws, km, K, p.kmeans_iters, call);
         prof_mark(cfg, round == 0 ? ST_KMEANS_ITERATE : ST_KMEANS_RETRY, round == 0 ? 1 : 4);
     }
 }
