@@ -30,7 +30,6 @@
 //   cell_gather     sweep: values of the selected cells into the gathered copy
 //   kmeans_iterate  the exact iterations
 #include "excp_common.cuh"
-#include "seg_ring.cuh"
 
 namespace excp {
 
@@ -152,110 +151,107 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
 }
 
 // ---------------------------------------------------------------------------
-constexpr int BST = 3;               // stages per warp
-constexpr int KM_GRID_PER_SM_W = 2;  // blocks per SM of the dW sweeps (the moment sweeps run one)
-constexpr int CWARPS = 16;           // warps per block of the counting sweep
+constexpr int KM_GRID_PER_SM = 2;    // blocks per SM of the two K-means sweeps
+constexpr int CWARPS = 16;           // warps per block of those sweeps
 
-template <int NS, int CH>
+// A warp's pass over the survivor segments of the tiles [wlo, whi): f8(a, b, two) gets two groups
+// of four values (the second only if `two`), f1(x) the up to three last values of a segment, one per
+// lane.  The counts of 32 tiles are read at a time, one per lane; up to four 16-byte loads per lane
+// are in flight.
+template <typename F8, typename F1>
+__device__ __forceinline__ void sweep_segments(const float* __restrict__ surv, const u32* __restrict__ tile_cnt,
+                                               u32 wlo, u32 whi, int lane, F8&& f8, F1&& f1) {
+    for (u32 t0 = wlo; t0 < whi; t0 += 32) {
+        const u32 nt32 = min(32u, whi - t0);
+        const u32 mycnt = (u32)lane < nt32 ? min(tile_cnt[t0 + lane], (u32)TILE) : 0u;   // a count never leads out of its segment
+        for (u32 i = 0; i < nt32; ++i) {
+            const u32 cnt = __shfl_sync(0xffffffffu, mycnt, i);
+            if (!cnt) continue;
+            const float* seg = surv + (u64)(t0 + i) * TILE;
+            const float4* seg4 = reinterpret_cast<const float4*>(seg);
+            const u32 whole = cnt >> 2;                        // groups of four that exist entirely
+            for (u32 f = lane; f < whole; f += 128) {
+                float4 v[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    v[k] = f + 32u * k < whole ? __ldcs(seg4 + f + 32u * k) : make_float4(0.f, 0.f, 0.f, 0.f);
+                f8(v[0], v[1], f + 32u < whole);
+                if (f + 64u < whole) f8(v[2], v[3], f + 96u < whole);
+            }
+            if ((u32)lane < cnt - 4u * whole) f1(seg[4u * whole + lane]);
+        }
+    }
+}
+
+template <int NS>
 struct CellCountSmem {
-    float buf[CWARPS][BST][NS][CH];
-    unsigned long long bar[CWARPS][BST];
     u32 tab[NS][NCLASS];
-    u32 cnt[NS][NCELL];              // the block's counts since its last flush
+    u32 cnt[NS][NCELL];              // the block's counts of the tensor
     u32 lo[NS][NCELL];               // and sums of |Q|: low word,
     u32 hi[NS][NCELL];               //   carries out of it
-    u32 abort;
 };
 
 // Sweep 1: survivors per cell and the sum of their |Q| (a cell holds one sign).  A block takes a
 // contiguous share of the tiles and goes through it tensor by tensor; its warps split the tensor's
 // tiles and add into one table in shared memory, flushed to the tensor's own with integer atomics.
 // NS = 1: dW; NS = 2: both moment streams.
-template <int NS, int CH>
-__global__ void __launch_bounds__(CWARPS * 32) cell_count_kernel(const TensorDesc* __restrict__ descs,
-                                                                 const TensorState* __restrict__ st, int nt, u32 tiles,
-                                                                 Workspace ws, KmArrays km, int stream0, CallState* call) {
+template <int NS>
+__global__ void __launch_bounds__(CWARPS * 32, 2) cell_count_kernel(const TensorDesc* __restrict__ descs,
+                                                                    const TensorState* __restrict__ st, int nt, u32 tiles,
+                                                                    Workspace ws, KmArrays km, int stream0, CallState* call) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    CellCountSmem<NS, CH>& sm = *reinterpret_cast<CellCountSmem<NS, CH>*>(smem_raw);
+    CellCountSmem<NS>& sm = *reinterpret_cast<CellCountSmem<NS>*>(smem_raw);
     if (call->flags & FLAG_TIMEOUT) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     u32 lo, hi;
     block_range(tiles, lo, hi);
-    SegRing<NS, CH, BST> ring;
-    ring.init(&sm.buf[warp][0][0][0], sm.bar[warp], lane, lo, lo);
     const u32* tile_cnt = stream0 == 0 ? ws.tile_cnt_w : ws.tile_cnt_o;
-    const float* surv[NS];
 #pragma unroll
-    for (int k = 0; k < NS; ++k) {
-        surv[k] = ws.surv[stream0 + k];
+    for (int k = 0; k < NS; ++k)
         for (int c = tid; c < NCELL; c += CWARPS * 32) { sm.cnt[k][c] = 0; sm.lo[k][c] = 0; sm.hi[k][c] = 0; }
-    }
-    if (tid == 0) sm.abort = 0;
     u32 tile = lo;
     while (tile < hi) {
         const int cur = find_tensor(descs, nt, tile);
         const u32 seg_end = min(hi, descs[cur].tile_begin + descs[cur].num_tiles);
-        float s1[NS], s2[NS];
 #pragma unroll
-        for (int k = 0; k < NS; ++k) {
+        for (int k = 0; k < NS; ++k)
             for (int c = tid; c < NCLASS; c += CWARPS * 32) sm.tab[k][c] = ws.cst[cur].s[stream0 + k].tab[c];
-            s1[k] = st[cur].s[stream0 + k].scale1; s2[k] = st[cur].s[stream0 + k].scale2;
-        }
         __syncthreads();
         const u32 n = seg_end - tile;
         const u32 wlo = tile + (u32)(((u64)n * warp) / CWARPS), whi = tile + (u32)(((u64)n * (warp + 1)) / CWARPS);
-        ring.restart(wlo, whi);
-        bool alive = sm.abort == 0;
-        while (alive && ring.next_window(tile_cnt, lane, whi)) {
-            while (alive && ring.have()) {
-                ring.issue_ahead(lane, surv);
-                const u32 nel = ring.nel();
-                if (!ring.wait()) {
-                    if (lane == 0) { atomicOr(&call->flags, FLAG_TIMEOUT); sm.abort = 1; }
-                    alive = false;
-                    break;
+#pragma unroll
+        for (int k = 0; k < NS; ++k) {
+            const u32* tab = sm.tab[k];
+            u32* cnt = sm.cnt[k];
+            u32* slo = sm.lo[k];
+            u32* shi = sm.hi[k];
+            const float a1 = st[cur].s[stream0 + k].scale1, a2 = st[cur].s[stream0 + k].scale2;
+            auto tally = [&](float x) {
+                const u32 c = cell_of(x, tab);
+                const u32 q = (u32)abs(__float2int_rn(__fmul_rn(__fmul_rn(x, a1), a2)));   // |Q(x)| < 2^31
+                atomicAdd(&cnt[c], 1u);
+                const u32 old = atomicAdd(&slo[c], q);
+                if (old + q < old) atomicAdd(&shi[c], 1u);
+            };
+            auto tally8 = [&](const float4& va, const float4& vb, bool two) {      // all table look-ups first
+                const float xs[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
+                u32 c[8], q[8], old[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    c[i] = cell_of(xs[i], tab);
+                    q[i] = (u32)abs(__float2int_rn(__fmul_rn(__fmul_rn(xs[i], a1), a2)));
                 }
 #pragma unroll
-                for (int k = 0; k < NS; ++k) {
-                    const float* data = ring.stage() + k * CH;
-                    const u32* tab = sm.tab[k];
-                    u32* cnt = sm.cnt[k];
-                    u32* slo = sm.lo[k];
-                    u32* shi = sm.hi[k];
-                    const float a1 = s1[k], a2 = s2[k];
-                    auto tally = [&](float x) {
-                        const u32 c = cell_of(x, tab);
-                        const u32 q = (u32)abs(__float2int_rn(__fmul_rn(__fmul_rn(x, a1), a2)));   // |Q(x)| < 2^31
-                        atomicAdd(&cnt[c], 1u);
-                        const u32 old = atomicAdd(&slo[c], q);
-                        if (old + q < old) atomicAdd(&shi[c], 1u);
-                    };
-                    const u32 whole = nel / 4;                             // groups of four that exist entirely
-                    for (u32 f = lane; f < whole; f += 64) {               // two groups per lane: all table look-ups first
-                        const bool two = f + 32 < whole;
-                        const float4 va = *reinterpret_cast<const float4*>(data + 4 * f);
-                        const float4 vb = two ? *reinterpret_cast<const float4*>(data + 4 * (f + 32)) : va;
-                        const float xs[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
-                        u32 c[8], q[8], old[8];
+                for (int i = 0; i < 8; ++i)
+                    if (i < 4 || two) atomicAdd(&cnt[c[i]], 1u);
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            c[i] = cell_of(xs[i], tab);
-                            q[i] = (u32)abs(__float2int_rn(__fmul_rn(__fmul_rn(xs[i], a1), a2)));
-                        }
+                for (int i = 0; i < 8; ++i)
+                    if (i < 4 || two) old[i] = atomicAdd(&slo[c[i]], q[i]);
 #pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            if (i < 4 || two) atomicAdd(&cnt[c[i]], 1u);
-#pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            if (i < 4 || two) old[i] = atomicAdd(&slo[c[i]], q[i]);
-#pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            if ((i < 4 || two) && old[i] + q[i] < old[i]) atomicAdd(&shi[c[i]], 1u);
-                    }
-                    if (lane < nel - 4 * whole) tally(data[4 * whole + lane]);
-                }
-                ring.advance();
-            }
+                for (int i = 0; i < 8; ++i)
+                    if ((i < 4 || two) && old[i] + q[i] < old[i]) atomicAdd(&shi[c[i]], 1u);
+            };
+            sweep_segments(ws.surv[stream0 + k], tile_cnt, wlo, whi, lane, tally8, tally);
         }
         __syncthreads();
 #pragma unroll
@@ -274,7 +270,6 @@ __global__ void __launch_bounds__(CWARPS * 32) cell_count_kernel(const TensorDes
             }
         }
         __syncthreads();
-        if (sm.abort) return;
         tile = seg_end;
     }
 }
@@ -321,7 +316,7 @@ __device__ inline u32 block_of_tile(u32 x, u32 tiles, u32 g) {
 __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDesc* __restrict__ descs,
                                                                  TensorState* __restrict__ st, Workspace ws, KmArrays km, int K,
                                                                  int iters, int margin, int round, u32 tiles,
-                                                                 u32 grid_w, u32 grid_o) {
+                                                                 u32 grid) {
     __shared__ u32 tab[NCLASS];
     __shared__ u32 selw[NCELL / 32];
     __shared__ float cent[KCAP], thr[KCAP], cnew[KCAP];
@@ -418,7 +413,6 @@ __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDes
     if (tid < NCELL / 32) cs.sel[tid] = selw[tid];
     // Where every block of the sweeps puts its values of a cell: the blocks that share the tensor,
     // in order, each after the ones before it (the counting sweep left their counts in km_rows).
-    const u32 grid = stream == 0 ? grid_w : grid_o;
     const u32 tb = descs[t].tile_begin, tl = tb + descs[t].num_tiles - 1;
     const u32 b0 = block_of_tile(tb, tiles, grid), b1 = block_of_tile(tl, tiles, grid);
     const u32* rows = km.rows[stream];
@@ -432,106 +426,79 @@ __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDes
 }
 
 // ---------------------------------------------------------------------------
-template <int NS, int CH>
+template <int NS>
 struct CellGatherSmem {
-    float buf[CWARPS][BST][NS][CH];
-    unsigned long long bar[CWARPS][BST];
     u32 tab[NS][NCLASS];
     u32 sel[NS][NCELL / 32];
     u32 cur[NS][NCELL];              // where the block's next value of each selected cell goes
-    u32 abort;
 };
 
 // Sweep 2: the values of the selected cells into the gathered copy, every cell contiguous (the
 // order inside a cell is arbitrary: what is taken from it are integer sums).  Same grid and same
 // shares of the tiles as the counting sweep, so every block owns a reserved run inside every cell
-// (km_pos) and no two blocks ever contend for a place.  A tensor with nothing to gather is skipped.
-template <int NS, int CH>
-__global__ void __launch_bounds__(CWARPS * 32) cell_gather_kernel(const TensorDesc* __restrict__ descs, int nt, u32 tiles,
-                                                                  Workspace ws, KmArrays km, int stream0, CallState* call, int round) {
+// (km.pos) and no two blocks ever contend for a place.  A tensor with nothing to gather is skipped.
+template <int NS>
+__global__ void __launch_bounds__(CWARPS * 32, 2) cell_gather_kernel(const TensorDesc* __restrict__ descs, int nt, u32 tiles,
+                                                                     Workspace ws, KmArrays km, int stream0, CallState* call,
+                                                                     int round) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    CellGatherSmem<NS, CH>& sm = *reinterpret_cast<CellGatherSmem<NS, CH>*>(smem_raw);
+    CellGatherSmem<NS>& sm = *reinterpret_cast<CellGatherSmem<NS>*>(smem_raw);
     if (call->flags & FLAG_TIMEOUT) return;
     if (round > 0 && *km.pending == 0) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     u32 lo, hi;
     block_range(tiles, lo, hi);
-    SegRing<NS, CH, BST> ring;
-    ring.init(&sm.buf[warp][0][0][0], sm.bar[warp], lane, lo, lo);
     const u32* tile_cnt = stream0 == 0 ? ws.tile_cnt_w : ws.tile_cnt_o;
-    const float* surv[NS];
-#pragma unroll
-    for (int k = 0; k < NS; ++k) surv[k] = ws.surv[stream0 + k];
-    if (tid == 0) sm.abort = 0;
     u32 tile = lo;
     while (tile < hi) {
         const int cur = find_tensor(descs, nt, tile);
         const u32 tb = descs[cur].tile_begin;
         const u32 seg_end = min(hi, tb + descs[cur].num_tiles);
+        bool act[NS];
         bool any = false;
 #pragma unroll
-        for (int k = 0; k < NS; ++k) any |= ws.cst[cur].s[stream0 + k].active != 0;
+        for (int k = 0; k < NS; ++k) { act[k] = ws.cst[cur].s[stream0 + k].active != 0; any |= act[k]; }
         if (!any) { tile = seg_end; continue; }           // the same for the whole block
 #pragma unroll
         for (int k = 0; k < NS; ++k) {
             const CellStream& cs = ws.cst[cur].s[stream0 + k];
-            const bool act = cs.active != 0;
             const u32* pos = km.pos[stream0 + k] + (u64)(blockIdx.x + cur) * NCELL;
             for (int c = tid; c < NCLASS; c += CWARPS * 32) sm.tab[k][c] = cs.tab[c];
-            for (int c = tid; c < NCELL / 32; c += CWARPS * 32) sm.sel[k][c] = act ? cs.sel[c] : 0u;
+            for (int c = tid; c < NCELL / 32; c += CWARPS * 32) sm.sel[k][c] = cs.sel[c];
             for (int c = tid; c < NCELL; c += CWARPS * 32) sm.cur[k][c] = pos[c];
         }
         __syncthreads();
         const u32 n = seg_end - tile;
         const u32 wlo = tile + (u32)(((u64)n * warp) / CWARPS), whi = tile + (u32)(((u64)n * (warp + 1)) / CWARPS);
-        ring.restart(wlo, whi);
-        bool alive = sm.abort == 0;
-        while (alive && ring.next_window(tile_cnt, lane, whi)) {
-            while (alive && ring.have()) {
-                ring.issue_ahead(lane, surv);
-                const u32 nel = ring.nel();
-                if (!ring.wait()) {
-                    if (lane == 0) { atomicOr(&call->flags, FLAG_TIMEOUT); sm.abort = 1; }
-                    alive = false;
-                    break;
+#pragma unroll
+        for (int k = 0; k < NS; ++k) {
+            if (!act[k]) continue;
+            const u32* tab = sm.tab[k];
+            const u32* sel = sm.sel[k];
+            u32* cursor = sm.cur[k];
+            float* out = ws.bkt[stream0 + k] + (u64)tb * TILE;
+            auto file = [&](float x) {
+                const u32 c = cell_of(x, tab);
+                if ((sel[c >> 5] >> (c & 31)) & 1u) out[atomicAdd(&cursor[c], 1u)] = x;
+            };
+            auto file8 = [&](const float4& va, const float4& vb, bool two) {       // all look-ups first
+                const float xs[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
+                u32 c[8];
+                u32 hit = 0;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) c[i] = cell_of(xs[i], tab);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) hit |= ((sel[c[i] >> 5] >> (c[i] & 31)) & 1u) << i;
+                if (!two) hit &= 15u;
+                if (hit) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if ((hit >> i) & 1u) out[atomicAdd(&cursor[c[i]], 1u)] = xs[i];
                 }
-#pragma unroll
-                for (int k = 0; k < NS; ++k) {
-                    const float* data = ring.stage() + k * CH;
-                    const u32* tab = sm.tab[k];
-                    const u32* sel = sm.sel[k];
-                    u32* cursor = sm.cur[k];
-                    float* out = ws.bkt[stream0 + k] + (u64)tb * TILE;
-                    auto file = [&](float x) {
-                        const u32 c = cell_of(x, tab);
-                        if ((sel[c >> 5] >> (c & 31)) & 1u) out[atomicAdd(&cursor[c], 1u)] = x;
-                    };
-                    const u32 whole = nel / 4;
-                    for (u32 f = lane; f < whole; f += 64) {               // two groups per lane: all look-ups first
-                        const bool two = f + 32 < whole;
-                        const float4 va = *reinterpret_cast<const float4*>(data + 4 * f);
-                        const float4 vb = two ? *reinterpret_cast<const float4*>(data + 4 * (f + 32)) : va;
-                        const float xs[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
-                        u32 c[8];
-                        u32 hit = 0;
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) c[i] = cell_of(xs[i], tab);
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) hit |= ((sel[c[i] >> 5] >> (c[i] & 31)) & 1u) << i;
-                        if (!two) hit &= 15u;
-                        if (hit) {
-#pragma unroll
-                            for (int i = 0; i < 8; ++i)
-                                if ((hit >> i) & 1u) out[atomicAdd(&cursor[c[i]], 1u)] = xs[i];
-                        }
-                    }
-                    if (lane < nel - 4 * whole) file(data[4 * whole + lane]);
-                }
-                ring.advance();
-            }
+            };
+            sweep_segments(ws.surv[stream0 + k], tile_cnt, wlo, whi, lane, file8, file);
         }
         __syncthreads();
-        if (sm.abort) return;
         tile = seg_end;
     }
 }
@@ -667,26 +634,25 @@ void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* s
     kmeans_start_kernel<<<dim3(nt, 3), SAMPLE_MAX, 0, cfg.stream>>>(descs, st, ws, km, p.seed, K, p.kmeans_iters);
     prof_mark(cfg, ST_KMEANS_START, 1);
     if (!tiles || p.kmeans_iters == 0) return;
-    // the two sweeps of a stream use one grid: a block's share of the tiles is its share of every cell
-    const u32 grid_w = min(tiles, min((u32)KM_GRID_PER_SM_W * (u32)cfg.sms, (u32)KM_MAX_GRID));
-    const u32 grid_o = min(tiles, min((u32)cfg.sms, (u32)KM_MAX_GRID));
+    // the two sweeps use one grid: a block's share of the tiles is its share of every cell
+    const u32 grid = min(tiles, min((u32)KM_GRID_PER_SM * (u32)cfg.sms, (u32)KM_MAX_GRID));
     {
-        const size_t m1 = sizeof(CellCountSmem<1, 256>), m2 = sizeof(CellCountSmem<2, 256>);
-        cudaFuncSetAttribute(cell_count_kernel<1, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m1);
-        cudaFuncSetAttribute(cell_count_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m2);
-        cell_count_kernel<1, 256><<<grid_w, CWARPS * 32, m1, cfg.stream>>>(descs, st, nt, tiles, ws, km, 0, call);
-        cell_count_kernel<2, 256><<<grid_o, CWARPS * 32, m2, cfg.stream>>>(descs, st, nt, tiles, ws, km, 1, call);
+        const size_t m1 = sizeof(CellCountSmem<1>), m2 = sizeof(CellCountSmem<2>);
+        cudaFuncSetAttribute(cell_count_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m1);
+        cudaFuncSetAttribute(cell_count_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m2);
+        cell_count_kernel<1><<<grid, CWARPS * 32, m1, cfg.stream>>>(descs, st, nt, tiles, ws, km, 0, call);
+        cell_count_kernel<2><<<grid, CWARPS * 32, m2, cfg.stream>>>(descs, st, nt, tiles, ws, km, 1, call);
         prof_mark(cfg, ST_CELL_COUNT, 2);
     }
-    const size_t g1 = sizeof(CellGatherSmem<1, 256>), g2 = sizeof(CellGatherSmem<2, 256>);
-    cudaFuncSetAttribute(cell_gather_kernel<1, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g1);
-    cudaFuncSetAttribute(cell_gather_kernel<2, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g2);
+    const size_t g1 = sizeof(CellGatherSmem<1>), g2 = sizeof(CellGatherSmem<2>);
+    cudaFuncSetAttribute(cell_gather_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g1);
+    cudaFuncSetAttribute(cell_gather_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g2);
     for (int round = 0; round < 2; ++round) {
         cell_plan_kernel<<<dim3(nt, 3), PLAN_THREADS, 0, cfg.stream>>>(descs, st, ws, km, K, p.kmeans_iters, p.km_margin, round,
-                                                                     tiles, grid_w, grid_o);
+                                                                     tiles, grid);
         if (round == 0) prof_mark(cfg, ST_CELL_PLAN, 1);
-        cell_gather_kernel<1, 256><<<grid_w, CWARPS * 32, g1, cfg.stream>>>(descs, nt, tiles, ws, km, 0, call, round);
-        cell_gather_kernel<2, 256><<<grid_o, CWARPS * 32, g2, cfg.stream>>>(descs, nt, tiles, ws, km, 1, call, round);
+        cell_gather_kernel<1><<<grid, CWARPS * 32, g1, cfg.stream>>>(descs, nt, tiles, ws, km, 0, call, round);
+        cell_gather_kernel<2><<<grid, CWARPS * 32, g2, cfg.stream>>>(descs, nt, tiles, ws, km, 1, call, round);
         if (round == 0) prof_mark(cfg, ST_CELL_GATHER, 2);
         kmeans_iterate_kernel<<<dim3(nt, 3), IT_THREADS, 0, cfg.stream>>>(descs, st, ws, km, K, p.kmeans_iters, call);
         prof_mark(cfg, round == 0 ? ST_KMEANS_ITERATE : ST_KMEANS_RETRY, round == 0 ? 1 : 4);
