@@ -401,8 +401,13 @@ def pack_bitmap(mask: np.ndarray) -> bytes:
 
 
 def unpack_bitmap(raw: bytes, numel: int) -> np.ndarray:
+    """The first numel bits.  The layout says that padding is zero: a bit set at or past numel
+    (in the last word or in the words that fill the section up to 16 bytes) makes the record corrupt."""
     b = np.frombuffer(raw, dtype=np.uint8)
-    return np.unpackbits(b, bitorder="little")[:numel].astype(bool)
+    bits = np.unpackbits(b, bitorder="little")
+    if np.any(bits[numel:]):
+        raise CorruptBlob("bitmap bit past the last element")
+    return bits[:numel].astype(bool)
 
 
 def encode_record(numel, bits, m_w, m_o, c_w, c_ea, c_eas, codes_w, codes_ea, codes_eas, rec_flags: int = 0) -> bytes:

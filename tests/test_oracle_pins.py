@@ -415,6 +415,17 @@ def test_corrupt_records_are_refused():
         orc.parse_record(bytes(bad))
     with pytest.raises(orc.CorruptBlob):
         orc.parse_record(blob[:40])
+    # padding is zero by the layout: a bit set past the last element (300 elements: bits 300..319 of the
+    # tenth word, then two whole padding words up to 48 bytes) leaves the first 300 bits and their
+    # population untouched and must still be refused, in either bitmap
+    hb, bb = orc.header_bytes(15), orc.bitmap_bytes(300)
+    assert (hb, bb) == (256, 48)
+    for start in (hb, hb + bb):
+        for bit in (300, 319, 320, 383):
+            bad = bytearray(blob); bad[start + bit // 8] |= 1 << (bit % 8)
+            with pytest.raises(orc.CorruptBlob):
+                orc.parse_record(bytes(bad))
+    assert orc.parse_record(blob)["numel"] == 300                   # the record itself is fine
 
 
 # ---------------------------------------------------------------- chain (Algorithm 3's loop)
