@@ -5,16 +5,20 @@ One "step" = one excp_compress_checkpoint call over the whole tensor list of the
 workload (all stages: statistics, masks + compaction, K-means, packing), inputs
 resident in HBM.  `value` = parameters compressed per second over all ranks.
 Beside it: per-stage CUDA-event times and the roofline of the dominant kernel,
-the decompress rate, the end-to-end rate through the host-buffer entry point
-(host->device and device->host copies inside the timed region), and the CPU
-oracle timed on a bounded sample of the same workload.
+the same step with the median of Eq. (rw) read literally (over |W_t|), the
+decompress rate, the dense layout and the archiver, the ablation rows, the
+compression ratio of the Pythia-410M-shaped checkpoint, the end-to-end rate through
+the host-buffer entry point (host->device and device->host copies inside the timed
+region), and the CPU oracle timed on a bounded sample of the same workload.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
                     [--config llama-7b|pythia-1.4b|pythia-410m|tiny] [--median residual|weight]
+                    [--outlier-frac F] [--chain STEPS] [--scaling weak|strong]
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import statistics
@@ -30,10 +34,9 @@ os.environ.setdefault("PYTORCH_CUDA_ALLOC_CONF", "expandable_segments:True")
 
 METRIC = "compress params/s and GB/s of (W,W_prev,m,v) read at 7B shape; % of HBM peak"
 NOMINAL_HBM_GBS = 8000.0
-# dram__bytes_read + dram__bytes_write per parameter from the ncu captures summarised under
-# profiles/ (small case, scaled by parameters); only for kernels unchanged since the capture
-NCU_DRAM_BYTES_PER_PARAM = {"mask_compact": (1.028104e9 + 169.809664e6) / 64108544}
 FALLBACK_HBM_GBS = 6650.0
+CSRC = os.path.join(ROOT, "paper_2406_11257_b200", "csrc")
+TRAFFIC_JSON = os.path.join(ROOT, "profiles", "ncu_traffic.json")
 
 
 def parse_args():
@@ -46,6 +49,12 @@ def parse_args():
     ap.add_argument("--median", default="residual", choices=["residual", "weight"])
     ap.add_argument("--kmeans-iters", type=int, default=10)
     ap.add_argument("--workspace-numel", type=int, default=1_200_000_000)
+    ap.add_argument("--outlier-frac", type=float, default=0.0,
+                    help="fraction of the residual at 10x scale (0.01 = the threshold-stress configuration)")
+    ap.add_argument("--chain", type=int, default=0,
+                    help="chained run: this many consecutive checkpoints, each residual against the previous reconstruction")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="N > 1: weak = every rank its own checkpoint; strong = one checkpoint's tensors dealt to the ranks")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--weights", default="f32", choices=["f32", "f16", "bf16"],
@@ -55,6 +64,8 @@ def parse_args():
     ap.add_argument("--no-decompress", action="store_true")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-layout and archiver leg")
     ap.add_argument("--no-ablation", action="store_true", help="skip the ablation-table leg")
+    ap.add_argument("--no-literal", action="store_true", help="skip the step with the median over |W_t|")
+    ap.add_argument("--no-410m", action="store_true", help="skip the compression ratio of the Pythia-410M-shaped checkpoint")
     ap.add_argument("--ablation-params", type=int, default=340_000_000,
                     help="parameters (leading tensors of the workload) the ablation rows are run on")
     ap.add_argument("--archive-params", type=int, default=17_000_000,
@@ -71,6 +82,29 @@ def measured_peak():
             return float(json.load(f)["hbm_gbs"]), "measured"
     except Exception:
         return FALLBACK_HBM_GBS, "fallback"
+
+
+def source_digest(files) -> str:
+    """sha256 over the named files of csrc/ (what a kernel is compiled from)."""
+    h = hashlib.sha256()
+    for name in sorted(files):
+        with open(os.path.join(CSRC, name), "rb") as f:
+            h.update(name.encode() + b"\0" + f.read() + b"\0")
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(stage: str, n_tot: int):
+    """DRAM bytes of one launch of the stage's kernel on this workload, from the ncu capture recorded in
+    profiles/ncu_traffic.json (a smaller case, scaled by parameters); None when there is no capture or the
+    kernel's sources have changed since it was taken."""
+    try:
+        with open(TRAFFIC_JSON) as f:
+            rec = json.load(f)[stage]
+        if source_digest(rec["sources"]) != rec["digest"]:
+            return None
+        return (rec["dram_read_bytes"] + rec["dram_write_bytes"]) / rec["params"] * n_tot
+    except Exception:
+        return None
 
 
 class ClockSampler:
@@ -135,39 +169,137 @@ def mem_available_gb() -> float:
     return 0.0
 
 
-def oracle_sample(args, shapes, seed):
-    """The oracle, as it stands, on one mid-sized tensor of the workload.  Returns (params/s, description)."""
+# ---------------------------------------------------------------------------------------------
+# Host-side helpers that run in spawned worker processes (never forked: the parent holds a CUDA
+# context).  They are module-level so that a spawned interpreter can import them.
+def _scratch_dir() -> str:
+    shm = "/dev/shm"
+    return shm if os.path.isdir(shm) and os.access(shm, os.W_OK) else tempfile.gettempdir()
+
+
+def _xz_size(path: str) -> int:
+    import lzma
+    with open(path, "rb") as f:
+        raw = f.read()
+    os.unlink(path)
+    return len(lzma.compress(raw, format=lzma.FORMAT_XZ, preset=9 | lzma.PRESET_EXTREME))
+
+
+def xz_sizes(chunks) -> list[int]:
+    """Size of every byte string after the archiver (LZMA2 in the xz container, preset 9 extreme: the stand-in
+    for Algorithm 1's "7zip" step), each archived on its own, in parallel on the host cores."""
+    import multiprocessing as mp
+    d = tempfile.mkdtemp(prefix="excp_xz_", dir=_scratch_dir())
+    paths = []
+    for i, c in enumerate(chunks):
+        paths.append(os.path.join(d, f"{i}.bin"))
+        with open(paths[-1], "wb") as f:
+            f.write(c)
+    order = sorted(range(len(paths)), key=lambda i: -len(chunks[i]))        # the longest first
+    with mp.get_context("spawn").Pool(min(len(paths), os.cpu_count() or 1)) as pool:
+        sizes = pool.map(_xz_size, [paths[i] for i in order], chunksize=1)
+    os.rmdir(d)
+    out = [0] * len(paths)
+    for i, s in zip(order, sizes):
+        out[i] = s
+    return out
+
+
+def _oracle_worker(paths, params: dict, tensor_index: int, barrier, queue):
+    import numpy as np
+    from oracle import excp_oracle as orc
+    q = [np.load(p) for p in paths]
+    barrier.wait()
+    t0 = time.perf_counter()
+    orc.compress_tensor(*q, orc.Params(**params), tensor_index=tensor_index)
+    queue.put(time.perf_counter() - t0)
+
+
+def oracle_all_cores(q_np, params: dict, tensor_index: int):
+    """The oracle as N independent single-threaded workers (N = the host's cores), each compressing the same
+    tensor at the same time.  Returns (workers, seconds of the slowest)."""
+    import multiprocessing as mp
+    import numpy as np
+    ctx = mp.get_context("spawn")
+    n = os.cpu_count() or 1
+    d = tempfile.mkdtemp(prefix="excp_orc_", dir=_scratch_dir())
+    paths = []
+    for i, a in enumerate(q_np):
+        paths.append(os.path.join(d, f"{i}.npy"))
+        np.save(paths[-1], a)
+    barrier, queue = ctx.Barrier(n + 1), ctx.Queue()
+    procs = [ctx.Process(target=_oracle_worker, args=(paths, params, tensor_index, barrier, queue)) for _ in range(n)]
+    for p in procs:
+        p.start()
+    barrier.wait()
+    times = [queue.get() for _ in procs]
+    for p in procs:
+        p.join()
+    for p in paths:
+        os.unlink(p)
+    os.rmdir(d)
+    return n, max(times)
+
+
+def oracle_sample_tensor(shapes, limit=17_000_000):
+    cand = [(i, n) for i, (_, n) in enumerate(shapes) if n <= limit] or [(0, shapes[0][1])]
+    return max(cand, key=lambda t: t[1])
+
+
+def oracle_params(args) -> dict:
+    return dict(kmeans_iters=args.kmeans_iters, bits=args.bits, median_source=1 if args.median == "residual" else 0)
+
+
+def oracle_sample(args, shapes, seed, all_cores: bool):
+    """The oracle, as it stands, on one mid-sized tensor of the workload: compress on one core, Algorithm 2 on
+    one core, and compress on every core at once."""
     import torch
     from oracle import excp_oracle as orc
     from paper_2406_11257_b200 import synth
-    cand = [(i, n) for i, (_, n) in enumerate(shapes) if n <= 17_000_000]
-    idx, numel = max(cand, key=lambda t: t[1])
+    idx, numel = oracle_sample_tensor(shapes)
     dev = "cuda" if torch.cuda.is_available() else "cpu"
-    q = [t.cpu().numpy() for t in synth.make_quad(numel, seed, idx, device=dev)]
-    p = orc.Params(kmeans_iters=args.kmeans_iters, median_source=1 if args.median == "residual" else 0)
+    q = [t.cpu().numpy() for t in synth.make_quad(numel, seed, idx, device=dev, outlier_frac=args.outlier_frac)]
     torch.set_num_threads(1)
     t0 = time.perf_counter()
-    orc.compress_tensor(*q, p, tensor_index=idx)
+    rec, _ = orc.compress_tensor(*q, orc.Params(**oracle_params(args)), tensor_index=idx)
     dt = time.perf_counter() - t0
-    return numel / dt, f"tensor {idx} ({shapes[idx][0]}, {numel} params) of the workload, {dt:.1f} s", numel, dt
+    t0 = time.perf_counter()
+    orc.decompress_tensor(rec, q[1])
+    ddt = time.perf_counter() - t0
+    out = {"value": numel / dt, "unit": "params/s", "cores": 1, "kind": "oracle",
+           "sample": f"tensor {idx} ({shapes[idx][0]}, {numel} params) of the workload, {dt:.1f} s",
+           "decompress": {"value": numel / ddt, "unit": "params/s", "cores": 1, "seconds": ddt}}
+    if all_cores:
+        n, slow = oracle_all_cores(q, oracle_params(args), idx)
+        out["all_cores"] = {"value": n * numel / slow, "unit": "params/s", "cores": n,
+                            "sample": f"{n} single-threaded workers, the same tensor each, slowest {slow:.1f} s"}
+    return out
+
+
+def workload_name(args) -> str:
+    s = f"{args.config} shaped checkpoint pair, median of |{'dW' if args.median == 'residual' else 'W_t'}|"
+    if args.outlier_frac:
+        s += f", {args.outlier_frac:g} of the residual at 10x"
+    return s
 
 
 def run_reference(args):
-    """The CPU oracle as the reference arm: each step compresses a bounded sample of the workload."""
+    """The CPU oracle as the reference arm: each step compresses a bounded sample of the workload (the tensor the
+    cpu_baseline leg of the other arm times), on one core."""
     from paper_2406_11257_b200 import synth
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     shapes = synth.tensor_list(synth.CONFIG_SHAPES[args.config])
-    cand = [(i, n) for i, (_, n) in enumerate(shapes) if n <= 4_500_000] or [(0, shapes[0][1])]
-    idx, numel = max(cand, key=lambda t: t[1])
+    idx, numel = oracle_sample_tensor(shapes)
     import torch
     from oracle import excp_oracle as orc
     dev = "cuda" if torch.cuda.is_available() else "cpu"
-    q = [t.cpu().numpy() for t in synth.make_quad(numel, 0, idx, device=dev)]
-    p = orc.Params(kmeans_iters=args.kmeans_iters, median_source=1 if args.median == "residual" else 0)
+    q = [t.cpu().numpy() for t in synth.make_quad(numel, 1000, idx, device=dev, outlier_frac=args.outlier_frac)]
+    p = orc.Params(**oracle_params(args))
     torch.set_num_threads(1)
-    for _ in range(args.warmup):
+    warm = min(args.warmup, 1)                               # a step is seconds of CPU work: one warm-up is enough
+    for _ in range(warm):
         orc.compress_tensor(*q, p, tensor_index=idx)
     t0 = time.perf_counter()
     for _ in range(args.steps):
@@ -177,14 +309,117 @@ def run_reference(args):
     sample = f"tensor {idx} ({shapes[idx][0]}, {numel} params) of the workload per step"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": "params/s", "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "steps": args.steps, "warmup": warm, "ms_per_step": 1e3 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{args.config} shaped checkpoint pair, median of |{'dW' if args.median == 'residual' else 'W'}|",
-                   "kmeans_iters": args.kmeans_iters, "bits": 4},
+        "config": {"workload": workload_name(args), "kmeans_iters": args.kmeans_iters, "bits": args.bits},
         "cpu_baseline": {"value": value, "unit": "params/s", "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "params/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }))
+
+
+# ---------------------------------------------------------------------------------------------
+def stage_bytes_of(n_tot, surv, wb, src_b, bits):
+    """Bytes each stage must move once by design (its inputs read once, its outputs written once); the smaller
+    terms (the median's sample and bracket keys, the gathered copy of the K-means cells, per-tile counts) are
+    left out, so the sums understate what the kernels move."""
+    return {
+        "stats1": (src_b + 4) * n_tot,
+        "mask_compact": (2 * wb + 8) * n_tot + n_tot / 4 + 4 * surv,
+        "cell_count": 4 * surv,                     # survivors read once: count and fixed-point sum per value cell
+        "cell_gather": 4 * surv,                    # read again: the cells the iterations visit are copied out
+        "pack_codes": (4 + bits / 8) * surv,
+        "copy_bitmaps": n_tot / 2,
+    }
+
+
+KERNEL_SOURCES = {                                  # what each stage's dominant kernel is compiled from
+    "stats1": ["stats.cu", "warp_ring.cuh", "tma.cuh", "excp_common.cuh"],
+    "mask_compact": ["mask_compact.cu", "warp_ring.cuh", "tma.cuh", "excp_common.cuh"],
+    "cell_count": ["kmeans.cu", "excp_common.cuh"],
+    "cell_gather": ["kmeans.cu", "excp_common.cuh"],
+    "pack_codes": ["pack.cu", "seg_ring.cuh", "tma.cuh", "excp_common.cuh"],
+    "decode": ["decode.cu", "warp_ring.cuh", "tma.cuh", "excp_common.cuh"],
+}
+
+
+def run_chain(args, torch, binding, synth, ranks, dev):
+    """Chained run (Section 3.4, Algorithm 3): `--chain` consecutive checkpoints W_(k+1) = W_k + delta_k with fresh
+    moments; every residual is taken against the previous RECONSTRUCTION, compressed, and decompressed in place;
+    afterwards the whole chain is decompressed again from the initial weights.  One line: per-step times and
+    the drift against the oracle's chain on one tensor of the list."""
+    import numpy as np
+    shape = synth.CONFIG_SHAPES[args.config]
+    shapes = synth.tensor_list(shape)
+    if args.max_tensors:
+        shapes = shapes[:args.max_tensors]
+    nt, n_tot = len(shapes), sum(n for _, n in shapes)
+    h = binding.Handle(workspace_numel=min(args.workspace_numel, n_tot + 4096 * nt))
+    p = binding.Params(kmeans_iters=args.kmeans_iters, bits=args.bits, median_source=binding.MEDIAN_ABS_RESIDUAL)
+    w0 = [synth.make_quad(n, 2000, i, device=dev)[1] for i, (_, n) in enumerate(shapes)]
+    pick, pn = oracle_sample_tensor(shapes, 4_500_000)
+    w_hat = [w.clone() for w in w0]
+    ea_out = [torch.empty_like(w) for w in w0]
+    eas_out = [torch.empty_like(w) for w in w0]
+    cap = int(0.80 * n_tot) + 4096 * nt + (1 << 20)
+    w_true, blobs, cms, dms, ratios, oracle_steps = w0, [], [], [], [], []
+    sampler = ClockSampler(0)
+    sampler.start()
+    for k in range(args.chain):
+        quads = [synth.make_quad(n, 2000, i, device=dev, step=k + 1, w_prev=w_true[i], outlier_frac=args.outlier_frac)
+                 for i, (_, n) in enumerate(shapes)]
+        w_true = [q[0] for q in quads]
+        oracle_steps.append(tuple(quads[pick][j].cpu().numpy() for j in (0, 2, 3)))
+        step_in = [(q[0], w_hat[i], q[2], q[3]) for i, q in enumerate(quads)]
+        blob = torch.empty(cap, dtype=torch.uint8, device=dev)
+        h.compress_checkpoint(p, step_in, blob, want_stats=False)                       # warm-up of this step's shapes
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record()
+        offs, _ = h.compress_checkpoint(p, step_in, blob, want_stats=False)
+        e[1].record()
+        h.decompress_checkpoint(blob, offs, w_hat, w_hat, ea_out, eas_out)
+        e[2].record(); torch.cuda.synchronize()
+        cms.append(e[0].elapsed_time(e[1])); dms.append(e[1].elapsed_time(e[2]))
+        ratios.append(12 * n_tot / offs[-1])
+        blobs.append((blob[:offs[-1]].clone(), offs))
+        del blob, quads, step_in
+    clocks = sampler.stop()
+    w_again = [w.clone() for w in w0]
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a0.record()
+    for blob, offs in blobs:
+        h.decompress_checkpoint(blob, offs, w_again, w_again, ea_out, eas_out)
+    a1.record(); torch.cuda.synchronize()
+    same = all(torch.equal(a, b) for a, b in zip(w_again, w_hat))
+    out = {
+        "metric": METRIC, "value": n_tot / (statistics.mean(cms) * 1e-3), "unit": "params/s", "n_gpus": 1,
+        "steps": args.chain, "warmup": 1, "ms_per_step": statistics.mean(cms), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"chain of {args.chain} {shape.name} checkpoints ({nt} tensors, {n_tot} params each), every residual "
+                               "against the previous reconstruction, median of |dW|, alpha 5e-5, beta 2.0",
+                   "bits": args.bits, "kmeans_iters": args.kmeans_iters,
+                   "l2": "inputs larger than L2 (no flush needed)" if 16 * n_tot > 4e8 else "inputs fit L2"},
+        "chain": {"compress_ms": cms, "decompress_in_place_ms": dms, "ratio_vs_12B_per_param": ratios,
+                  "whole_chain_decompress_ms": a0.elapsed_time(a1), "replay_equals_running_reconstruction": same},
+        "clocks": clocks,
+    }
+    if not args.no_cpu:
+        from oracle import excp_oracle as orc
+        op = orc.Params(kmeans_iters=args.kmeans_iters, bits=args.bits, median_source=1)
+        wh = w0[pick].cpu().numpy()
+        identical, worst = True, 0.0
+        t0 = time.perf_counter()
+        for k, (w_t, ea, eas) in enumerate(oracle_steps):
+            rec, _ = orc.compress_tensor(w_t, wh, ea, eas, op, tensor_index=pick)
+            wh, _, _ = orc.decompress_tensor(rec, wh)
+            blob, offs = blobs[k]
+            identical &= blob[offs[pick]:offs[pick + 1]].cpu().numpy().tobytes() == rec
+        worst = float(np.abs(w_hat[pick].cpu().numpy().astype(np.float64) - wh).max())
+        out["chain"]["drift_vs_oracle_chain"] = {
+            "max_abs_weight_difference_after_last_step": worst, "records_identical_every_step": bool(identical),
+            "sample": f"tensor {pick} ({shapes[pick][0]}, {pn} params), oracle chain {time.perf_counter() - t0:.1f} s on one core"}
+    h.close()
+    print(json.dumps(out))
 
 
 def run_ours(args):
@@ -197,6 +432,10 @@ def run_ours(args):
         raise SystemExit("bench.py needs a CUDA device: the compression path has no CPU fallback")
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
+    if args.chain:
+        if world > 1:
+            raise SystemExit("--chain runs on one GPU")
+        return run_chain(args, torch, binding, synth, ranks, dev)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
@@ -204,12 +443,20 @@ def run_ours(args):
         ranks.barrier(world)
 
     shape = synth.CONFIG_SHAPES[args.config]
-    shapes = synth.tensor_list(shape)
+    all_shapes = synth.tensor_list(shape)
     if args.max_tensors:
-        shapes = shapes[:args.max_tensors]
+        all_shapes = all_shapes[:args.max_tensors]
+    strong = args.scaling == "strong" and world > 1
+    if strong:                                            # one checkpoint, its tensors dealt to the ranks
+        mine = ranks.partition_tensors([n for _, n in all_shapes], world)[rank]
+        seed = 1000
+    else:                                                 # every rank compresses its own checkpoint
+        mine = list(range(len(all_shapes)))
+        seed = ranks.rank_seed(1000, rank)
+    shapes = [all_shapes[i] for i in mine]
     n_tot = sum(n for _, n in shapes)
-    seed = ranks.rank_seed(1000, rank)                    # every rank compresses its own checkpoint
-    quads = [synth.make_quad(n, seed, i, device=dev) for i, (_, n) in enumerate(shapes)]
+    n_job = sum(n for _, n in all_shapes) if strong else world * n_tot
+    quads = [synth.make_quad(n, seed, i, device=dev, outlier_frac=args.outlier_frac) for i, (_, n) in zip(mine, shapes)]
     wfmt = {"f32": binding.WEIGHTS_F32, "f16": binding.WEIGHTS_F16, "bf16": binding.WEIGHTS_BF16}[args.weights]
     wb = 4 if wfmt == binding.WEIGHTS_F32 else 2            # bytes per stored weight
     if wb == 2:
@@ -226,199 +473,195 @@ def run_ours(args):
     ws_numel = min(args.workspace_numel, n_tot + 4096 * len(shapes))
     ws_numel = max(ws_numel, max(n for _, n in shapes))
     h = binding.Handle(workspace_numel=ws_numel)
-    p = binding.Params(kmeans_iters=args.kmeans_iters, bits=args.bits,
-                       median_source=binding.MEDIAN_ABS_RESIDUAL if args.median == "residual" else binding.MEDIAN_ABS_WEIGHT)
+
+    def params(median):
+        return binding.Params(kmeans_iters=args.kmeans_iters, bits=args.bits,
+                              median_source=binding.MEDIAN_ABS_RESIDUAL if median == "residual" else binding.MEDIAN_ABS_WEIGHT)
+    p = params(args.median)
     bound = sum(binding.compress_bound(n, args.bits) for _, n in shapes)
     cap = min(bound, int(0.80 * n_tot * max(args.bits, 4) / 4) + 4096 * len(shapes) + (1 << 20))
     blob = torch.empty(cap, dtype=torch.uint8, device=dev)
+    indices = mine if strong else None
 
-    h.profile_enable(True)
-    offs = stats = None
+    def compress(pp, want_stats=True):
+        return h.compress_checkpoint(pp, quads, blob, weight_format=wfmt, tensor_indices=indices, want_stats=want_stats)
+
+    def timed_steps(pp, steps):
+        """`steps` compress calls between two events; returns (ms per step on the slowest rank, offsets, stats,
+        per-stage ms per step, launches per step, clocks)."""
+        h.profile_enable(True)
+        stage_ms, launches = {}, 0
+        sampler = ClockSampler(local)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier(); torch.cuda.synchronize()
+        sampler.start()
+        ev0.record()
+        for _ in range(steps):
+            offs, stats = compress(pp)
+            ms, l = h.profile_read()
+            launches += l
+            for k, v in ms.items():
+                stage_ms[k] = stage_ms.get(k, 0.0) + v
+        ev1.record()
+        torch.cuda.synchronize(); barrier()
+        clocks = sampler.stop()
+        h.profile_enable(False)
+        elapsed = ranks.max_over_ranks(ev0.elapsed_time(ev1), world, dev)
+        return elapsed / steps, offs, stats, {k: v / steps for k, v in stage_ms.items()}, launches // steps, clocks
+
+    def byte_figures(stats, median, ms_per_step, per_step):
+        nnz_w = sum(s.nnz_w for s in stats)
+        nnz_o = sum(s.nnz_o for s in stats)
+        surv = nnz_w + 2 * nnz_o
+        src_b = 2 * wb if median == "residual" else wb
+        sb = stage_bytes_of(n_tot, surv, wb, src_b, args.bits)
+        moved = sum(sb.values())
+        T = args.kmeans_iters
+        # what a plain implementation moves, every Lloyd iteration sweeping the survivors: one statistics
+        # sweep, the mask sweep and its outputs, T + 1 sweeps of the survivors, the codes
+        sweep = ((src_b + 4) + (2 * wb + 8) + 0.25) * n_tot + 4 * surv + (T + 1) * 4 * surv + args.bits / 8 * surv
+        gbs = lambda b: b / (ms_per_step * 1e-3) / 1e9
+        return sb, {
+            "survivors": {"f_w": nnz_w / n_tot, "f_o": nnz_o / n_tot},
+            "moved_bytes_per_param": moved / n_tot, "moved_gbs": gbs(moved),
+            "hbm_frac_of_nominal_8TBs": gbs(moved) / NOMINAL_HBM_GBS, "hbm_frac_of_measured": gbs(moved) / peak,
+            "sweep_per_iteration_bytes_per_param": sweep / n_tot,
+            "effective_gbs_vs_sweep_per_iteration": gbs(sweep),
+            "effective_frac_of_nominal_8TBs_vs_sweep_per_iteration": gbs(sweep) / NOMINAL_HBM_GBS,
+            "stages": {k: {"ms": round(per_step.get(k, 0.0), 4),
+                           "gbs": round(sb[k] / (per_step[k] * 1e-3) / 1e9, 1) if k in sb else None}
+                       for k in per_step if per_step[k] > 0}}
+
+    peak, peak_kind = measured_peak()
     for _ in range(max(args.warmup, 0)):
-        offs, stats = h.compress_checkpoint(p, quads, blob, weight_format=wfmt)
-    stage_ms = {}
-    launches = 0
-    sampler = ClockSampler(local)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier(); torch.cuda.synchronize()
-    sampler.start()
-    ev0.record()
-    for _ in range(args.steps):
-        offs, stats = h.compress_checkpoint(p, quads, blob, weight_format=wfmt)
-        ms, l = h.profile_read()
-        launches += l
-        for k, v in ms.items():
-            stage_ms[k] = stage_ms.get(k, 0.0) + v
-    ev1.record()
-    torch.cuda.synchronize(); barrier()
-    clocks = sampler.stop()
-    elapsed_ms = ranks.max_over_ranks(ev0.elapsed_time(ev1), world, dev)
-    ms_per_step = elapsed_ms / args.steps
-    value = ranks.whole_job_rate(world * n_tot, ms_per_step)
-
+        compress(p)
+    ms_per_step, offs, stats, per_step, launches, clocks = timed_steps(p, args.steps)
+    value = ranks.whole_job_rate(n_job, ms_per_step)
+    sb, figs = byte_figures(stats, args.median, ms_per_step, per_step)
+    blob_bytes = offs[-1]
     nnz_w = sum(s.nnz_w for s in stats)
     nnz_o = sum(s.nnz_o for s in stats)
-    blob_bytes = offs[-1]
-    f_w, f_o = nnz_w / n_tot, nnz_o / n_tot
-    T = args.kmeans_iters
-    src_b = 2 * wb if args.median == "residual" else wb
-    # bytes each stage must move once (its inputs read once, its outputs written once)
-    surv = nnz_w + 2 * nnz_o
-    stage_bytes = {
-        "stats1": (src_b + 4) * n_tot,
-        "mask_compact": (2 * wb + 8) * n_tot + n_tot / 4 + 4 * surv,
-        "bucket_ids": 4 * surv,                     # survivors read once: counts and fixed-point sums per bucket
-        "bucket_scatter": 8 * surv,                 # survivors read and written into their buckets
-        "bucket_scan": T * 4 * surv * min(1.0, (2 ** args.bits - 2) / 256),   # about K - 1 of 256 buckets per iteration
-        "pack_codes": (4 + args.bits / 8) * surv,
-        "copy_bitmaps": n_tot / 2,
-    }
-    moved_bytes = sum(stage_bytes.values())         # what these kernels must move by design
-    # what the method moves when every Lloyd iteration sweeps the survivors (one statistics sweep,
-    # one mask sweep, T + 1 sweeps of the survivors, the codes)
-    algo_bytes = ((src_b + 4) + (2 * wb + 8) + 0.25) * n_tot + 4 * surv + (T + 1) * 4 * surv + args.bits / 8 * surv
-    peak, peak_kind = measured_peak()
-    per_step = {k: v / args.steps for k, v in stage_ms.items()}
-    dom = max((k for k in stage_bytes), key=lambda k: per_step.get(k, 0.0))
+    dom = max(sb, key=lambda k: per_step.get(k, 0.0))
     dom_ms = per_step[dom]
-    dom_gbs = stage_bytes[dom] / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
-    groups_note = f"{launches // args.steps} launches per step"
-    stages = {k: {"ms": round(per_step.get(k, 0.0), 4),
-                  "gbs": round(stage_bytes[k] / (per_step[k] * 1e-3) / 1e9, 1) if k in stage_bytes and per_step.get(k, 0) > 0 else None}
-              for k in per_step if per_step[k] > 0}
+    dom_gbs = sb[dom] / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
 
     out = {
         "metric": METRIC, "value": value, "unit": "params/s", "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "strong" if strong else "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{shape.name} checkpoint pair ({len(shapes)} tensors, {n_tot} params, {args.weights} W_t, W_prev, fp32 ea, eas), "
-                               f"median of |{'dW' if args.median == 'residual' else 'W_t'}|, alpha 5e-5, beta 2.0",
-                   "bits": args.bits, "kmeans_iters": T, "l2": "inputs larger than L2 (no flush needed)" if 16 * n_tot > 4e8 else "inputs fit L2",
-                   "workspace_numel": ws_numel, "per_rank": "each rank compresses its own checkpoint; no collective"},
+        "config": {"workload": f"{shape.name} checkpoint pair ({len(all_shapes)} tensors, {sum(n for _, n in all_shapes)} params, "
+                               f"{args.weights} W_t, W_prev, fp32 ea, eas), median of |{'dW' if args.median == 'residual' else 'W_t'}|, "
+                               f"alpha 5e-5, beta 2.0" + (f", {args.outlier_frac:g} of the residual at 10x" if args.outlier_frac else ""),
+                   "bits": args.bits, "kmeans_iters": args.kmeans_iters,
+                   "l2": "inputs larger than L2 (no flush needed)" if 16 * n_tot > 4e8 else "inputs fit L2",
+                   "workspace_numel": ws_numel,
+                   "per_rank": ("one checkpoint, its tensors dealt to the ranks by size; only record offsets cross ranks"
+                                if strong else "each rank compresses its own checkpoint; no collective")},
         "input_gbs": (2 * wb + 8) * value / 1e9,
-        "algorithmic_bytes_per_param": algo_bytes / n_tot,
-        "moved_bytes_per_param": moved_bytes / n_tot,
-        "moved_gbs": moved_bytes / n_tot * value / world / 1e9,
-        "moved_frac_of_measured": moved_bytes / n_tot * value / world / 1e9 / peak,
-        "algorithmic_gbs": algo_bytes / n_tot * value / world / 1e9,
-        "hbm_frac_of_measured": algo_bytes / n_tot * value / world / 1e9 / peak,
-        "hbm_frac_of_nominal_8TBs": algo_bytes / n_tot * value / world / 1e9 / NOMINAL_HBM_GBS,
-        "survivors": {"f_w": f_w, "f_o": f_o},
+        **figs,
         "compression": {"blob_bytes": blob_bytes, "ratio_vs_12B_per_param": 12 * n_tot / blob_bytes,
                         "ratio_vs_stored_state": (wb + 8) * n_tot / blob_bytes},
-        "stages": stages,
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": dom_gbs / peak, "peak_kind": peak_kind,
-                     "traffic": NCU_DRAM_BYTES_PER_PARAM[dom] * n_tot if dom in NCU_DRAM_BYTES_PER_PARAM else None,
-                     "algorithmic_bytes_per_step": stage_bytes[dom], "ms_per_step": dom_ms, "note": groups_note},
+                     "frac": dom_gbs / peak, "peak_kind": peak_kind, "traffic": ncu_traffic(dom, n_tot),
+                     "algorithmic_bytes_per_step": sb[dom], "ms_per_step": dom_ms, "note": f"{launches} launches per step"},
         "clocks": clocks,
-        "gpu_launches": launches,
+        "gpu_launches": launches * args.steps,
     }
+    if strong:                                            # the checkpoint-wide offsets, assembled from the ranks' own
+        _, table, goffs = ranks.compress_partitioned(lambda idx: offs, [n for _, n in all_shapes], world, rank)
+        out["compression"] = {"blob_bytes": goffs[-1], "ratio_vs_12B_per_param": 12 * n_job / goffs[-1],
+                              "records_per_rank": [sum(1 for r, _, _ in table if r == k) for k in range(world)]}
 
-    # ---- decompress (Algorithm 2) on the records just written ---------------
-    if not args.no_decompress:
-        h.profile_enable(False)
-        chunk_cap = ws_numel
-        out_w = torch.empty(chunk_cap, dtype=quads[0][1].dtype, device=dev)
-        out_a = torch.empty(chunk_cap, dtype=torch.float32, device=dev)
-        out_s = torch.empty(chunk_cap, dtype=torch.float32, device=dev)
+    # ---- the same step with Eq. (rw)'s median read literally: over |W_t| ----------------------
+    if not args.no_literal and args.median == "residual" and world == 1:
+        pl = params("weight")
+        compress(pl)
+        lms, loffs, lstats, lper, _, _ = timed_steps(pl, args.steps)
+        _, lf = byte_figures(lstats, "weight", lms, lper)
+        out["literal_median"] = {"what": "the same step with median(|W_t|) in Eq. (rw), as printed", "ms_per_step": lms,
+                                 "value": n_tot / (lms * 1e-3), "unit": "params/s", "input_gbs": (2 * wb + 8) * n_tot / (lms * 1e-3) / 1e9,
+                                 "ratio_vs_12B_per_param": 12 * n_tot / loffs[-1], **lf}
+        offs, stats = compress(p, want_stats=True)        # the records of the headline run again, for the legs below
+
+    # ---- the dense index layout of Sections 3.3 / 4.2 and the archiver step of Algorithm 1 -------
+    def chunked(capacity):
         chunks, cur, used = [], [], 0
         for i, (_, n) in enumerate(shapes):
             n4 = (n + 3) // 4 * 4
-            if cur and used + n4 > chunk_cap:
+            if cur and used + n4 > capacity:
                 chunks.append(cur); cur, used = [], 0
             cur.append((i, used, n)); used += n4
         if cur:
             chunks.append(cur)
+        return chunks
 
-        def decompress_all():
+    if not args.no_dense and not args.no_decompress and args.bits == 4 and wb == 4 and world == 1:
+        chunk_cap = ws_numel
+        out_w = torch.empty(chunk_cap, dtype=torch.float32, device=dev)
+        out_a = torch.empty(chunk_cap, dtype=torch.float32, device=dev)
+        out_s = torch.empty(chunk_cap, dtype=torch.float32, device=dev)
+        chunks = chunked(chunk_cap)
+        numels = [n for _, n in shapes]
+        dsz = [binding.dense_bytes(n) for n in numels]
+        dense_total = sum(dsz)
+        dcap = max(sum(dsz[i] for i, _, _ in ch) for ch in chunks)
+        dense = torch.empty(dcap, dtype=torch.uint8, device=dev)          # one chunk of tensors at a time
+        evs = []
+
+        def dense_round(timed):
             for ch in chunks:
                 i0, i1 = ch[0][0], ch[-1][0] + 1
                 wp = [quads[i][1] for i, _, _ in ch]
-                h.decompress_checkpoint(blob[offs[i0]:], [o - offs[i0] for o in offs[i0:i1 + 1]], wp,
-                                        [out_w[o:o + n] for _, o, n in ch], [out_a[o:o + n] for _, o, n in ch],
-                                        [out_s[o:o + n] for _, o, n in ch], weight_format=wfmt)
-        decompress_all()
-        torch.cuda.synchronize()
-        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        d0.record()
+                e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+                e[0].record()
+                doffs = h.checkpoint_to_dense(blob[offs[i0]:], [o - offs[i0] for o in offs[i0:i1 + 1]],
+                                              numels[i0:i1], dense)
+                e[1].record()
+                h.decompress_checkpoint(dense, doffs, wp, [out_w[o:o + n] for _, o, n in ch],
+                                        [out_a[o:o + n] for _, o, n in ch], [out_s[o:o + n] for _, o, n in ch],
+                                        dense=True)
+                e[2].record()
+                if timed:
+                    evs.append(e)
+        dense_round(False)
         for _ in range(args.steps):
-            decompress_all()
-        d1.record(); torch.cuda.synchronize()
-        dms = d0.elapsed_time(d1) / args.steps
-        dec_bytes = n_tot / 4 + args.bits / 8 * (nnz_w + 2 * nnz_o) + wb * n_tot + (wb + 8) * n_tot
-        out["decompress"] = {"value": n_tot / (dms * 1e-3), "unit": "params/s", "ms_per_step": dms,
-                             "algorithmic_gbs": dec_bytes / (dms * 1e-3) / 1e9,
-                             "hbm_frac_of_measured": dec_bytes / (dms * 1e-3) / 1e9 / peak,
-                             "calls_per_step": len(chunks)}
-
-        # ---- the dense index layout of Sections 3.3 / 4.2 and the archiver step of Algorithm 1 -------
-        if not args.no_dense and args.bits == 4 and wb == 4:       # the dense layout is built for the method's 4-bit records
-            numels = [n for _, n in shapes]
-            dsz = [binding.dense_bytes(n) for n in numels]
-            dense_total = sum(dsz)
-            cap = max(sum(dsz[i] for i, _, _ in ch) for ch in chunks)
-            dense = torch.empty(cap, dtype=torch.uint8, device=dev)          # one chunk of tensors at a time
-            evs = []
-
-            def dense_round(timed):
-                for ch in chunks:
-                    i0, i1 = ch[0][0], ch[-1][0] + 1
-                    wp = [quads[i][1] for i, _, _ in ch]
-                    e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
-                    e[0].record()
-                    doffs = h.checkpoint_to_dense(blob[offs[i0]:], [o - offs[i0] for o in offs[i0:i1 + 1]],
-                                                  numels[i0:i1], dense)
-                    e[1].record()
-                    h.decompress_checkpoint(dense, doffs, wp, [out_w[o:o + n] for _, o, n in ch],
-                                            [out_a[o:o + n] for _, o, n in ch], [out_s[o:o + n] for _, o, n in ch],
-                                            dense=True)
-                    e[2].record()
-                    if timed:
-                        evs.append(e)
-            dense_round(False)
-            for _ in range(args.steps):
-                dense_round(True)
-            torch.cuda.synchronize()
-            cms = sum(e[0].elapsed_time(e[1]) for e in evs) / args.steps
-            ddms = sum(e[1].elapsed_time(e[2]) for e in evs) / args.steps
-            conv_bytes = blob_bytes + dense_total                       # the records read, the containers written
-            ddec_bytes = dense_total + 4 * n_tot + 12 * n_tot
-            # the archiver on the host (LZMA2, preset 9 extreme) over a bounded sample of both layouts
-            import lzma
-            pick = next((i for i, n in enumerate(numels) if n <= args.archive_params), 0)
-            rec_raw = blob[offs[pick]:offs[pick + 1]]
-            nb = h.record_to_dense(rec_raw, offs[pick + 1] - offs[pick], numels[pick], dense)
-            ta = time.time()
-            arch = {}
-            for name, t in (("record", rec_raw), ("dense", dense[:nb])):
-                rawb = t.cpu().numpy().tobytes()
-                arch[name + "_bytes"] = len(rawb)
-                arch[name + "_xz_bytes"] = len(lzma.compress(rawb, format=lzma.FORMAT_XZ, preset=9 | lzma.PRESET_EXTREME))
-            out["dense_layout"] = {
-                "to_dense_ms": cms, "to_dense_gbs": conv_bytes / (cms * 1e-3) / 1e9,
-                "to_dense_frac_of_measured": conv_bytes / (cms * 1e-3) / 1e9 / peak,
-                "decode_ms": ddms, "decode_params_per_s": n_tot / (ddms * 1e-3),
-                "decode_gbs": ddec_bytes / (ddms * 1e-3) / 1e9,
-                "decode_frac_of_measured": ddec_bytes / (ddms * 1e-3) / 1e9 / peak,
-                "dense_bytes": dense_total, "ratio_vs_12B_per_param": 12 * n_tot / dense_total,
-                "archive": dict(arch, sample=f"tensor {pick} ({shapes[pick][0]}, {numels[pick]} params) of the workload, "
-                                             f"xz preset 9 extreme, {time.time() - ta:.1f} s on the host",
-                                record_xz_ratio_vs_12B=12 * numels[pick] / arch["record_xz_bytes"],
-                                dense_xz_ratio_vs_12B=12 * numels[pick] / arch["dense_xz_bytes"])}
-            del dense
-        del out_w, out_a, out_s
+            dense_round(True)
+        torch.cuda.synchronize()
+        cms = sum(e[0].elapsed_time(e[1]) for e in evs) / args.steps
+        ddms = sum(e[1].elapsed_time(e[2]) for e in evs) / args.steps
+        conv_bytes = blob_bytes + dense_total                       # the records read, the containers written
+        ddec_bytes = dense_total + 4 * n_tot + 12 * n_tot
+        # the archiver on the host (LZMA2, preset 9 extreme) over a bounded sample of both layouts
+        pick = next((i for i, n in enumerate(numels) if n <= args.archive_params), 0)
+        rec_raw = blob[offs[pick]:offs[pick + 1]]
+        nb = h.record_to_dense(rec_raw, offs[pick + 1] - offs[pick], numels[pick], dense)
+        ta = time.time()
+        raws = [rec_raw.cpu().numpy().tobytes(), dense[:nb].cpu().numpy().tobytes()]
+        xz = xz_sizes(raws)
+        arch = {"record_bytes": len(raws[0]), "record_xz_bytes": xz[0], "dense_bytes": len(raws[1]), "dense_xz_bytes": xz[1]}
+        out["dense_layout"] = {
+            "to_dense_ms": cms, "to_dense_gbs": conv_bytes / (cms * 1e-3) / 1e9,
+            "to_dense_frac_of_measured": conv_bytes / (cms * 1e-3) / 1e9 / peak,
+            "decode_ms": ddms, "decode_params_per_s": n_tot / (ddms * 1e-3),
+            "decode_gbs": ddec_bytes / (ddms * 1e-3) / 1e9,
+            "decode_frac_of_measured": ddec_bytes / (ddms * 1e-3) / 1e9 / peak,
+            "dense_bytes": dense_total, "ratio_vs_12B_per_param": 12 * n_tot / dense_total,
+            "archive": dict(arch, sample=f"tensor {pick} ({shapes[pick][0]}, {numels[pick]} params) of the workload, "
+                                         f"xz preset 9 extreme, {time.time() - ta:.1f} s on the host",
+                            record_xz_ratio_vs_12B=12 * numels[pick] / arch["record_xz_bytes"],
+                            dense_xz_ratio_vs_12B=12 * numels[pick] / arch["dense_xz_bytes"])}
+        del dense, out_w, out_a, out_s
 
     # ---- the rows of the ablation table of Section 4.4 (sizes and times; accuracies need training) ----
-    if not args.no_ablation and wb == 4:
-        h.profile_enable(False)
+    if not args.no_ablation and wb == 4 and world == 1:
         sub, acc = [], 0
         for i, (_, n) in enumerate(shapes):
             if acc + n > args.ablation_params and sub:
                 break
             sub.append(i); acc += n
-        cap = sum(binding.record_bytes(shapes[i][1], shapes[i][1], shapes[i][1], 32) for i in sub)
-        ablob = torch.empty(cap, dtype=torch.uint8, device=dev)
+        acap = sum(binding.record_bytes(shapes[i][1], shapes[i][1], shapes[i][1], 32) for i in sub)
+        ablob = torch.empty(acap, dtype=torch.uint8, device=dev)
         rows = []
         for residual, prune, quant in ((0, 0, 0), (1, 0, 0), (0, 1, 0), (0, 0, 1), (1, 1, 0), (1, 0, 1), (1, 1, 1)):
             fl = ((0 if residual else binding.FLAG_NO_RESIDUAL) | (0 if prune else binding.FLAG_NO_PRUNE)
@@ -440,7 +683,7 @@ def run_ours(args):
         del ablob
 
     # ---- end to end through the host-buffer entry point ----------------------
-    if not args.no_e2e and wb == 4:
+    if not args.no_e2e and wb == 4 and not strong:
         need_gb = 16 * n_tot / 1e9
         sub = list(range(len(shapes)))
         if mem_available_gb() < 1.4 * need_gb + 8:
@@ -475,10 +718,74 @@ def run_ours(args):
 
     # ---- the oracle on the host cores (rank 0, one GPU only) -----------------
     if not args.no_cpu and rank == 0 and world == 1:
-        v, desc, _, _ = oracle_sample(args, shapes, seed)
-        out["cpu_baseline"] = {"value": v, "unit": "params/s", "cores": 1, "kind": "oracle", "sample": desc}
+        out["cpu_baseline"] = oracle_sample(args, shapes, seed, all_cores=True)
 
+    # ---- decompress (Algorithm 2) on the records just written: ONE call over the whole list, in place --------
+    # (W^_t over W^_(t-1), the decoded moments over the input moments, which nothing reads any more: the way a
+    # 108 GB checkpoint is restored on a 180 GB device.)  Last leg that uses the workload's inputs.
+    if not args.no_decompress:
+        wp = [q[1] for q in quads]
+        eo = [q[2] for q in quads]
+        so = [q[3] for q in quads]
+
+        def decompress_all():
+            h.decompress_checkpoint(blob, offs, wp, wp, eo, so, weight_format=wfmt)
+        decompress_all()
+        torch.cuda.synchronize()
+        h.profile_enable(True)
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        dstage = {}
+        d0.record()
+        for _ in range(args.steps):
+            decompress_all()
+            ms, _ = h.profile_read()
+            for k, v in ms.items():
+                dstage[k] = dstage.get(k, 0.0) + v / args.steps
+        d1.record(); torch.cuda.synchronize()
+        h.profile_enable(False)
+        dms = d0.elapsed_time(d1) / args.steps
+        dec_bytes = n_tot / 4 + args.bits / 8 * (nnz_w + 2 * nnz_o) + wb * n_tot + (wb + 8) * n_tot
+        kms = dstage.get("decode", 0.0)
+        out["decompress"] = {"value": n_tot / (dms * 1e-3), "unit": "params/s", "ms_per_step": dms,
+                             "algorithmic_gbs": dec_bytes / (dms * 1e-3) / 1e9,
+                             "hbm_frac_of_measured": dec_bytes / (dms * 1e-3) / 1e9 / peak,
+                             "hbm_frac_of_nominal_8TBs": dec_bytes / (dms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+                             "decode_kernel_ms": kms,
+                             "decode_kernel_frac_of_measured": dec_bytes / (kms * 1e-3) / 1e9 / peak if kms else None,
+                             "traffic": ncu_traffic("decode", n_tot),
+                             "calls_per_step": 1, "in_place": True}
+    del quads, blob
     h.close()
+    torch.cuda.empty_cache()
+
+    # ---- the compression ratio of the Pythia-410M-shaped checkpoint, both readings of the median ----------
+    if not args.no_410m and rank == 0 and world == 1 and args.bits == 4 and wb == 4:
+        s410 = synth.tensor_list(synth.CONFIG_SHAPES["pythia-410m"])
+        n410 = sum(n for _, n in s410)
+        q410 = [synth.make_quad(n, 1000, i, device=dev) for i, (_, n) in enumerate(s410)]
+        h4 = binding.Handle(workspace_numel=n410 + 4096 * len(s410))
+        b410 = torch.empty(sum(binding.compress_bound(n) for _, n in s410), dtype=torch.uint8, device=dev)
+        res = {}
+        for name, mode in (("median_abs_residual", binding.MEDIAN_ABS_RESIDUAL), ("median_abs_weight", binding.MEDIAN_ABS_WEIGHT)):
+            pp = binding.Params(kmeans_iters=args.kmeans_iters, median_source=mode)
+            h4.compress_checkpoint(pp, q410, b410, want_stats=False)
+            c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            c0.record()
+            o4, st4 = h4.compress_checkpoint(pp, q410, b410)
+            c1.record(); torch.cuda.synchronize()
+            raw = b410[:o4[-1]].cpu().numpy().tobytes()
+            ta = time.time()
+            xz = sum(xz_sizes([raw[o4[i]:o4[i + 1]] for i in range(len(s410))]))
+            res[name] = {"record_bytes": o4[-1], "ratio_vs_12B_per_param": 12 * n410 / o4[-1],
+                         "xz_bytes": xz, "ratio_after_xz_vs_12B_per_param": 12 * n410 / xz,
+                         "f_w": sum(s.nnz_w for s in st4) / n410, "f_o": sum(s.nnz_o for s in st4) / n410,
+                         "compress_ms": c0.elapsed_time(c1), "xz_seconds_on_the_host": time.time() - ta}
+        out["pythia_410m_shaped"] = dict(res, params=n410, tensors=len(s410),
+                                         note="synthetic checkpoint pair of the stated distributions; every record archived on "
+                                              "its own with xz preset 9 extreme; the paper's ~70x is on trained weights")
+        h4.close()
+        del q410, b410
+
     if rank == 0:
         print(json.dumps(out))
     if world > 1:

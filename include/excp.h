@@ -168,6 +168,21 @@ excp_status excp_compress_checkpoint(excp_handle h, const excp_params* params, s
                                      size_t* tensor_offsets_out, excp_tensor_stats* stats_out,
                                      void* cuda_stream);
 
+/* excp_compress_checkpoint for a SHARE of a checkpoint: the tensors of one checkpoint dealt to
+ * several processes, one GPU each (Algorithm 1 treats every tensor on its own, so nothing is
+ * exchanged between them).  tensor_index (host [num_tensors]) gives, for every tensor of the call,
+ * its index in the WHOLE checkpoint, which is what seeds its K-means start sample; the records are
+ * then byte for byte the ones a single excp_compress_checkpoint over the whole list writes for
+ * those tensors.  Offsets are relative to this call's blob_out.  Everything else as for
+ * excp_compress_checkpoint. */
+excp_status excp_compress_checkpoint_indexed(excp_handle h, const excp_params* params, size_t num_tensors,
+                                             const float* const* w_t, const float* const* w_prev,
+                                             const float* const* ea, const float* const* eas,
+                                             const size_t* numel, const size_t* tensor_index,
+                                             void* blob_out, size_t blob_capacity,
+                                             size_t* tensor_offsets_out, excp_tensor_stats* stats_out,
+                                             void* cuda_stream);
+
 /* Weights stored in 16 bits (Section 4.3 notes that the PanGu-pi weights are saved in float16).
  * excp_compress_checkpoint with W_t and W^_(t-1) given as IEEE binary16 (EXCP_WEIGHTS_F16) or
  * bfloat16 (EXCP_WEIGHTS_BF16) arrays; the moments stay fp32.  Every weight is widened to fp32,

@@ -20,7 +20,7 @@ STATUS = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED", -3: "BUFFER_TOO_SMALL",
 
 EXPORTS = ["excp_create", "excp_destroy", "excp_record_bytes", "excp_compress_bound",
            "excp_status_string", "excp_last_cuda_error", "excp_compress_tensor",
-           "excp_compress_checkpoint", "excp_compress_checkpoint_w16", "excp_decompress_checkpoint_w16",
+           "excp_compress_checkpoint", "excp_compress_checkpoint_indexed", "excp_compress_checkpoint_w16", "excp_decompress_checkpoint_w16",
            "excp_compress_checkpoint_host", "excp_decompress_tensor", "excp_decompress_checkpoint",
            "excp_decompress_tensor_noalloc", "excp_dense_bytes", "excp_record_to_dense", "excp_checkpoint_to_dense",
            "excp_decompress_dense_tensor", "excp_decompress_dense_checkpoint", "excp_profile_enable", "excp_profile_stage_count", "excp_profile_stage_name", "excp_profile_read",
@@ -88,6 +88,9 @@ def load_library() -> C.CDLL:
                                              C.POINTER(vp), C.POINTER(vp), C.POINTER(sz), vp, sz,
                                              C.POINTER(sz), C.POINTER(CStats), vp]
     lib.excp_compress_checkpoint_host.argtypes = lib.excp_compress_checkpoint.argtypes
+    lib.excp_compress_checkpoint_indexed.argtypes = [vp, C.POINTER(CParams), sz, C.POINTER(vp), C.POINTER(vp),
+                                                     C.POINTER(vp), C.POINTER(vp), C.POINTER(sz), C.POINTER(sz), vp, sz,
+                                                     C.POINTER(sz), C.POINTER(CStats), vp]
     lib.excp_compress_checkpoint_w16.argtypes = [vp, C.POINTER(CParams), sz, C.POINTER(vp), C.POINTER(vp),
                                                  C.POINTER(vp), C.POINTER(vp), C.POINTER(sz), C.c_int, vp, sz,
                                                  C.POINTER(sz), C.POINTER(CStats), vp]
@@ -227,9 +230,11 @@ class Handle:
         return nbytes.value, stats
 
     def compress_checkpoint(self, p: Params, tensors, blob_out: torch.Tensor, want_stats: bool = True,
-                            weight_format: int = WEIGHTS_F32):
+                            weight_format: int = WEIGHTS_F32, tensor_indices=None):
         """excp_compress_checkpoint (or, for 16-bit weights, excp_compress_checkpoint_w16) over a list of
-        (w_t, w_prev, ea, eas).  Returns (offsets list of len n+1, list of stats or None)."""
+        (w_t, w_prev, ea, eas).  Returns (offsets list of len n+1, list of stats or None).  With
+        `tensor_indices` (the tensors' places in the whole checkpoint, for a rank that compresses a share of
+        it) the call is excp_compress_checkpoint_indexed."""
         n = len(tensors)
         for q in tensors:
             _check_weights(weight_format, q[0], q[1])
@@ -240,7 +245,13 @@ class Handle:
         stats = (CStats * n)() if want_stats else None
         cp = p.to_c()
         cap = blob_out.numel() * blob_out.element_size()
-        if weight_format == WEIGHTS_F32:
+        if tensor_indices is not None:
+            if weight_format != WEIGHTS_F32 or len(tensor_indices) != n:
+                raise ValueError("tensor_indices: one per tensor, fp32 weights only")
+            idx = (C.c_size_t * n)(*[int(i) for i in tensor_indices])
+            st = self.lib.excp_compress_checkpoint_indexed(self._h, C.byref(cp), n, arr(0), arr(1), arr(2), arr(3), numel, idx,
+                                                           blob_out.data_ptr(), cap, offs, stats, _stream())
+        elif weight_format == WEIGHTS_F32:
             st = self.lib.excp_compress_checkpoint(self._h, C.byref(cp), n, arr(0), arr(1), arr(2), arr(3), numel,
                                                    blob_out.data_ptr(), cap, offs, stats, _stream())
         else:

@@ -172,6 +172,14 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
                 b[k] = bm_word(d.rec, s.off_bm_o, nwords, w0 + 4 * lane + k);
                 if (!(s.rflags & REC_MOMENTS_FREE)) bad |= b[k] & ~a[k];   // a moment kept where the weight is pruned
             }
+            if ((u64)(tile - tb + 1) * TILE > n) {        // the tensor ends in this tile: no bit at or past its last element
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const u64 e = (w0 + 4 * lane + k) * 32;                 // first element of the word
+                    const u32 stray = e >= n ? 0xffffffffu : (n - e >= 32 ? 0u : 0xffffffffu << (u32)(n - e));
+                    bad |= (a[k] | b[k]) & stray;
+                }
+            }
             const u32 ta = __popc(a[0]) + __popc(a[1]) + __popc(a[2]) + __popc(a[3]);
             const u32 tbm = __popc(b[0]) + __popc(b[1]) + __popc(b[2]) + __popc(b[3]);
             u32 ia = ta, ib = tbm;

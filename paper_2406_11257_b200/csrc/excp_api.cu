@@ -69,6 +69,7 @@ struct excp_handle_s {
     float* stage[2][4] = {};
     unsigned char* stage_blob[2] = {};
     size_t stage_blob_bytes = 0;
+    int stage_bits = 0;                  // code width the record staging is sized for
     cudaStream_t s_h2d = nullptr, s_d2h = nullptr;
     cudaEvent_t ev_h2d[2] = {}, ev_compute[2] = {}, ev_d2h[2] = {};
 };
@@ -187,21 +188,35 @@ void fill_outputs(excp_handle h, size_t first, size_t count, const size_t* numel
     }
 }
 
-bool ensure_host_path(excp_handle h) {
-    if (h->s_h2d) return true;
+// Staging of the host-buffer path.  The record staging holds the largest records a group can
+// produce at `bits` (every element a survivor); a call with wider codes than any before it on this
+// handle gets a larger one.
+bool ensure_host_path(excp_handle h, int bits) {
     const size_t elems = h->cap_tiles * (size_t)TILE;
-    h->stage_blob_bytes = (size_t)record_bytes(elems, elems, elems, 4) + (size_t)MAX_GROUP_TENSORS * 512;
+    if (bits > h->stage_bits) {
+        if (h->s_d2h && !check(h, cudaStreamSynchronize(h->s_d2h))) return false;
+        h->stage_blob_bytes = (size_t)record_bytes(elems, elems, elems, bits) + (size_t)MAX_GROUP_TENSORS * 512;
+        for (int k = 0; k < 2; ++k) {
+            if (h->stage_blob[k]) cudaFree(h->stage_blob[k]);
+            h->stage_blob[k] = nullptr;
+            if (!check(h, cudaMalloc(reinterpret_cast<void**>(&h->stage_blob[k]), h->stage_blob_bytes))) {
+                h->stage_bits = 0;
+                return false;
+            }
+        }
+        h->stage_bits = bits;
+    }
+    if (h->s_h2d) return true;
     bool ok = true;
     for (int k = 0; k < 2 && ok; ++k) {
         for (int j = 0; j < 4 && ok; ++j)
-            ok = check(h, cudaMalloc(reinterpret_cast<void**>(&h->stage[k][j]), elems * sizeof(float)));
-        ok = ok && check(h, cudaMalloc(reinterpret_cast<void**>(&h->stage_blob[k]), h->stage_blob_bytes));
-        ok = ok && check(h, cudaEventCreateWithFlags(&h->ev_h2d[k], cudaEventDisableTiming));
-        ok = ok && check(h, cudaEventCreateWithFlags(&h->ev_compute[k], cudaEventDisableTiming));
-        ok = ok && check(h, cudaEventCreateWithFlags(&h->ev_d2h[k], cudaEventDisableTiming));
+            if (!h->stage[k][j]) ok = check(h, cudaMalloc(reinterpret_cast<void**>(&h->stage[k][j]), elems * sizeof(float)));
+        if (!h->ev_h2d[k]) ok = ok && check(h, cudaEventCreateWithFlags(&h->ev_h2d[k], cudaEventDisableTiming));
+        if (!h->ev_compute[k]) ok = ok && check(h, cudaEventCreateWithFlags(&h->ev_compute[k], cudaEventDisableTiming));
+        if (!h->ev_d2h[k]) ok = ok && check(h, cudaEventCreateWithFlags(&h->ev_d2h[k], cudaEventDisableTiming));
     }
-    ok = ok && check(h, cudaStreamCreateWithFlags(&h->s_d2h, cudaStreamNonBlocking));
-    ok = ok && check(h, cudaStreamCreateWithFlags(&h->s_h2d, cudaStreamNonBlocking));
+    if (!h->s_d2h) ok = ok && check(h, cudaStreamCreateWithFlags(&h->s_d2h, cudaStreamNonBlocking));
+    ok = ok && check(h, cudaStreamCreateWithFlags(&h->s_h2d, cudaStreamNonBlocking));   // last: marks the path as ready
     return ok;
 }
 
@@ -334,7 +349,7 @@ static excp_status compress_impl(excp_handle h, const excp_params* params, size_
                                  const float* const* ea, const float* const* eas,
                                  const size_t* numel, int wfmt, void* blob_out, size_t blob_capacity,
                                  size_t* tensor_offsets_out, excp_tensor_stats* stats_out,
-                                 void* cuda_stream) {
+                                 void* cuda_stream, const size_t* tensor_index = nullptr) {
     if (!h || !params || !tensor_offsets_out) return EXCP_ERR_INVALID_ARG;
     if (wfmt != WF_F32 && wfmt != WF_F16 && wfmt != WF_BF16) return EXCP_ERR_INVALID_ARG;
     if (num_tensors && (!w_t || !w_prev || !ea || !eas || !numel)) return EXCP_ERR_INVALID_ARG;
@@ -364,7 +379,7 @@ static excp_status compress_impl(excp_handle h, const excp_params* params, size_
             TensorDesc& d = hd[i];
             d.w_t = w_t[i]; d.w_prev = w_prev[i]; d.ea = ea[i]; d.eas = eas[i];
             d.numel = numel[i];
-            d.tensor_index = i;
+            d.tensor_index = tensor_index ? tensor_index[i] : i;
             d.tile_begin = tile;
             d.num_tiles = (u32)((numel[i] + TILE - 1) / TILE);
             tile += d.num_tiles;
@@ -403,6 +418,19 @@ excp_status excp_compress_checkpoint(excp_handle h, const excp_params* params, s
                          tensor_offsets_out, stats_out, cuda_stream);
 }
 
+excp_status excp_compress_checkpoint_indexed(excp_handle h, const excp_params* params, size_t num_tensors,
+                                             const float* const* w_t, const float* const* w_prev,
+                                             const float* const* ea, const float* const* eas,
+                                             const size_t* numel, const size_t* tensor_index,
+                                             void* blob_out, size_t blob_capacity,
+                                             size_t* tensor_offsets_out, excp_tensor_stats* stats_out,
+                                             void* cuda_stream) {
+    if (num_tensors && !tensor_index) return EXCP_ERR_INVALID_ARG;
+    return compress_impl(h, params, num_tensors, reinterpret_cast<const void* const*>(w_t),
+                         reinterpret_cast<const void* const*>(w_prev), ea, eas, numel, WF_F32, blob_out, blob_capacity,
+                         tensor_offsets_out, stats_out, cuda_stream, tensor_index);
+}
+
 excp_status excp_compress_checkpoint_w16(excp_handle h, const excp_params* params, size_t num_tensors,
                                          const void* const* w_t, const void* const* w_prev,
                                          const float* const* ea, const float* const* eas,
@@ -434,7 +462,7 @@ excp_status excp_compress_checkpoint_host(excp_handle h, const excp_params* para
     if (!make_groups(h, numel, num_tensors, groups)) return EXCP_ERR_INVALID_ARG;
     DeviceGuard guard(h->device);
     if (!guard.ok) return EXCP_ERR_CUDA;
-    if (!ensure_call_arrays(h, num_tensors) || !ensure_host_path(h)) return EXCP_ERR_CUDA;
+    if (!ensure_call_arrays(h, num_tensors) || !ensure_host_path(h, params->bits)) return EXCP_ERR_CUDA;
 
     TensorDesc* hd = static_cast<TensorDesc*>(h->h_desc);
     for (size_t gi = 0; gi < groups.size(); ++gi) {
@@ -498,6 +526,8 @@ excp_status excp_compress_checkpoint_host(excp_handle h, const excp_params* para
         if (!ok) break;
         const size_t bytes = (size_t)h->h_call->blob_cursor;
         flags |= h->h_call->flags;
+        // a group whose records outgrew the staging wrote none of them: nothing to copy
+        if ((flags & FLAG_BLOB_FULL) || bytes > h->stage_blob_bytes) { flags |= FLAG_BLOB_FULL; break; }
         if (host_off + bytes > blob_capacity) { flags |= FLAG_BLOB_FULL; break; }
         ok = check(h, cudaStreamWaitEvent(h->s_d2h, h->ev_compute[slot], 0));
         ok = ok && check(h, cudaMemcpyAsync(static_cast<unsigned char*>(blob_out) + host_off, h->stage_blob[slot],

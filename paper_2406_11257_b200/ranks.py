@@ -66,3 +66,58 @@ def sum_over_ranks(value: float, world: int, device="cpu") -> float:
 def whole_job_rate(units_all_ranks: float, ms_slowest: float) -> float:
     """Units per second of the whole job: everything all ranks processed over the slowest rank's time."""
     return units_all_ranks / (ms_slowest * 1e-3)
+
+
+def gather_objects(obj, world: int) -> list:
+    """Every rank's `obj`, in rank order, on every rank (host-side bookkeeping; not on the data path)."""
+    if world == 1:
+        return [obj]
+    out = [None] * world
+    dist.all_gather_object(out, obj)
+    return out
+
+
+def assemble_offsets(numels, shares, local_offsets_by_rank):
+    """The checkpoint-wide table of one partitioned checkpoint.
+
+    shares[r] = tensor indices rank r compressed (ascending); local_offsets_by_rank[r] = that rank's
+    offsets list (len(shares[r]) + 1) into its own blob.  Returns (table, offsets): table[i] =
+    (owner rank, offset in the owner's blob, record bytes) for tensor i of the checkpoint; offsets =
+    where record i starts if the records are laid back to back in checkpoint order (len n + 1), i.e.
+    the tensor_offsets a single-process compress of the whole list returns."""
+    n = len(numels)
+    table = [None] * n
+    for r, (idx, offs) in enumerate(zip(shares, local_offsets_by_rank)):
+        if len(offs) != len(idx) + 1:
+            raise ValueError(f"rank {r}: {len(idx)} tensors but {len(offs)} offsets")
+        for k, i in enumerate(idx):
+            if table[i] is not None:
+                raise ValueError(f"tensor {i} compressed twice")
+            table[i] = (r, int(offs[k]), int(offs[k + 1] - offs[k]))
+    if any(t is None for t in table):
+        raise ValueError("a tensor was compressed by no rank")
+    offsets = [0]
+    for _, _, nbytes in table:
+        offsets.append(offsets[-1] + nbytes)
+    return table, offsets
+
+
+def compress_partitioned(compress_share, numels, world: int, rank: int):
+    """One checkpoint compressed by `world` ranks, each on its own GPU (strong scaling).
+
+    The tensor list is dealt by partition_tensors; this rank calls compress_share(indices), which
+    compresses those tensors into the rank's own blob with their checkpoint-wide indices (so the
+    records are the ones a single process writes) and returns the offsets into that blob.  The ranks
+    then exchange only those offsets (host objects) and every rank assembles the same table.  No
+    tensor data, record or statistic crosses ranks.  Returns (my indices, table, offsets) as in
+    assemble_offsets."""
+    shares = partition_tensors(numels, world)
+    mine = shares[rank]
+    local = [int(o) for o in compress_share(mine)]
+    table, offsets = assemble_offsets(numels, shares, gather_objects(local, world))
+    return mine, table, offsets
+
+
+def assemble_blob(table, blobs_by_rank) -> bytes:
+    """The single checkpoint blob (records in checkpoint order) from the ranks' blobs; host bytes."""
+    return b"".join(bytes(blobs_by_rank[r][off:off + nbytes]) for r, off, nbytes in table)

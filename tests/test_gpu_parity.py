@@ -347,6 +347,21 @@ def test_corrupt_records_are_refused_without_faulting(handle):
         handle.decompress_tensor(blob, nbytes - 16, dq[1], *outs)
     assert e.value.status == -5
     handle.decompress_tensor(blob, nbytes, dq[1], *outs)     # the intact record still decodes
+    # A bit set past the last element, with the populations kept equal to the header's counts (a kept weight whose
+    # moments are pruned is cleared in exchange): only the rule "no bit at or past numel" catches it; the oracle
+    # refuses the same bytes.
+    raw = bytearray(blob[:nbytes].cpu().numpy().tobytes())
+    r = orc.parse_record(bytes(raw))
+    victim = int(np.flatnonzero(r["m_w"] & ~r["m_o"])[-1])
+    raw[256 + victim // 8] ^= 1 << (victim % 8)
+    stray = 9000 + 5                                          # 9000 = 281 * 32 + 8: bit 13 of the last word
+    raw[256 + stray // 8] |= 1 << (stray % 8)
+    with pytest.raises(orc.CorruptBlob):
+        orc.parse_record(bytes(raw))
+    bad = torch.frombuffer(raw, dtype=torch.uint8).to(DEV)
+    with pytest.raises(binding.ExcpError) as e:
+        handle.decompress_tensor(bad, nbytes, dq[1], *outs)
+    assert e.value.status == -5
 
 
 # ----------------------------------------------------------------- host path
@@ -370,6 +385,60 @@ def test_host_buffer_path_gives_the_same_records(handle):
         assert e.value.status == -3
     finally:
         small.close()
+
+
+def test_host_buffer_path_with_wide_codes_and_every_element_kept():
+    """Records far larger than 4-bit ones (8-bit codes, nothing pruned) through the host-buffer entry point: the
+    device staging grows with the code width, the records equal the device path's, and a host buffer that is too
+    small is refused with status -3 before anything is copied past the staging."""
+    sizes = [70000, 4096, 130000, 33, 64000]
+    quads = [rand_quad_np(n, 1100 + i) for i, n in enumerate(sizes)]
+    dquads = to_dev(quads)
+    small = binding.Handle(workspace_numel=140_000)
+    try:
+        hquads = [tuple(torch.as_tensor(a).pin_memory() for a in q) for q in quads]
+        p4 = binding.Params(median_source=binding.MEDIAN_ABS_RESIDUAL, seed=8)
+        cap4 = sum(binding.compress_bound(n) for n in sizes)
+        small.compress_checkpoint_host(p4, hquads, torch.empty(cap4, dtype=torch.uint8).pin_memory())   # staging sized for 4 bits
+        p = binding.Params(median_source=binding.MEDIAN_ABS_RESIDUAL, seed=8, bits=8, kmeans_iters=3,
+                           flags=binding.FLAG_NO_PRUNE)
+        cap = sum(binding.compress_bound(n, 8) for n in sizes)
+        blob = torch.full((cap,), 0xAB, dtype=torch.uint8, device=DEV)
+        offs, stats = small.compress_checkpoint(p, dquads, blob)
+        assert [s.nnz_w for s in stats] == sizes and offs[-1] > cap4
+        hblob = torch.full((cap,), 0xCD, dtype=torch.uint8).pin_memory()
+        hoffs, hstats = small.compress_checkpoint_host(p, hquads, hblob)
+        assert hoffs == offs
+        assert bytes(hblob[:offs[-1]].numpy()) == blob[:offs[-1]].cpu().numpy().tobytes()
+        with pytest.raises(binding.ExcpError) as e:
+            small.compress_checkpoint_host(p, hquads, hblob[:offs[-1] - 16])
+        assert e.value.status == -3
+        hoffs, _ = small.compress_checkpoint_host(p, hquads, hblob)              # the handle is still usable
+        assert hoffs == offs
+    finally:
+        small.close()
+
+
+def test_a_share_of_a_checkpoint_gives_the_whole_lists_records(handle):
+    """excp_compress_checkpoint_indexed: the tensors dealt to two ranks, each share compressed on its own with the
+    tensors' checkpoint-wide indices, give together exactly the records (and, assembled, the blob and the offsets)
+    of one call over the whole list."""
+    from paper_2406_11257_b200 import ranks
+    sizes = [30000, 5000, 70000, 0, 4096, 130000, 33, 8192, 99999]
+    dquads = to_dev([rand_quad_np(n, 1300 + i) for i, n in enumerate(sizes)])
+    p = binding.Params(median_source=binding.MEDIAN_ABS_RESIDUAL, seed=21)
+    blob, offs, _ = gpu_compress(handle, p, dquads)
+    whole = blob[:offs[-1]].cpu().numpy().tobytes()
+    shares = ranks.partition_tensors(sizes, 2)
+    blobs, local = [], []
+    for idx in shares:
+        b = torch.empty(sum(binding.compress_bound(sizes[i]) for i in idx) + 16, dtype=torch.uint8, device=DEV)
+        o, _ = handle.compress_checkpoint(p, [dquads[i] for i in idx], b, tensor_indices=idx)
+        blobs.append(b[:o[-1]].cpu().numpy().tobytes())
+        local.append(o)
+    table, goffs = ranks.assemble_offsets(sizes, shares, local)
+    assert goffs == offs
+    assert ranks.assemble_blob(table, blobs) == whole
 
 
 def test_profile_counts_launches_and_times_stages(handle):

@@ -93,3 +93,58 @@ def test_two_gloo_ranks_shard_by_tensor_and_agree_on_the_timing():
     for d in res[0]["sizes"]:
         sizes.update(d)
     assert sizes == {i: len(b) for i, b in merged.items()}
+
+
+def _part_worker(rank, world, port, out):
+    os.environ.update(RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        numels = [n for _, n in synth.tensor_list(synth.CONFIG_SHAPES["tiny"])]
+        blob = bytearray()
+
+        def compress_share(indices):                               # stub records: the tensor's index and size, repeated
+            offs = [0]
+            for i in indices:
+                blob.extend(_stub_record(i, numels[i]))
+                offs.append(len(blob))
+            return offs
+
+        mine, table, offsets = ranks.compress_partitioned(compress_share, numels, world, rank)
+        out[rank] = dict(mine=mine, table=table, offsets=offsets, blob=bytes(blob))
+    finally:
+        dist.destroy_process_group()
+
+
+def _stub_record(i, numel):
+    return (i.to_bytes(4, "little") + numel.to_bytes(8, "little")) * (1 + numel % 7) + bytes(4)   # 16-byte multiples
+
+
+def test_two_gloo_ranks_compress_one_partitioned_checkpoint():
+    world, port = 2, _free_port()
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_part_worker, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    numels = [n for _, n in synth.tensor_list(synth.CONFIG_SHAPES["tiny"])]
+    assert res[0]["table"] == res[1]["table"] and res[0]["offsets"] == res[1]["offsets"]
+    assert sorted(res[0]["mine"] + res[1]["mine"]) == list(range(len(numels)))
+    whole = b"".join(_stub_record(i, n) for i, n in enumerate(numels))          # what one process writes
+    assert ranks.assemble_blob(res[0]["table"], [res[0]["blob"], res[1]["blob"]]) == whole
+    offs = res[0]["offsets"]
+    assert offs[-1] == len(whole)
+    for i, n in enumerate(numels):
+        assert whole[offs[i]:offs[i + 1]] == _stub_record(i, n)
+        r, off, nbytes = res[0]["table"][i]
+        assert i in res[r]["mine"] and res[r]["blob"][off:off + nbytes] == _stub_record(i, n)
+
+
+def test_assemble_offsets_refuses_inconsistent_shares():
+    with pytest.raises(ValueError):
+        ranks.assemble_offsets([4, 4], [[0], [0]], [[0, 16], [0, 16]])          # tensor 0 twice, tensor 1 never
+    with pytest.raises(ValueError):
+        ranks.assemble_offsets([4, 4], [[0], []], [[0, 16], [0]])               # tensor 1 by nobody
+    with pytest.raises(ValueError):
+        ranks.assemble_offsets([4], [[0]], [[0]])                               # offsets too short
+    table, offs = ranks.assemble_offsets([4, 8, 4], [[1], [0, 2]], [[0, 32], [0, 16, 48]])
+    assert table == [(1, 0, 16), (0, 0, 32), (1, 16, 32)] and offs == [0, 16, 48, 80]
