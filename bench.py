@@ -750,7 +750,7 @@ def run_ours(args):
                              "algorithmic_gbs": dec_bytes / (dms * 1e-3) / 1e9,
                              "hbm_frac_of_measured": dec_bytes / (dms * 1e-3) / 1e9 / peak,
                              "hbm_frac_of_nominal_8TBs": dec_bytes / (dms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
-                             "decode_kernel_ms": kms,
+                             "decode_kernel_ms": kms, "prep_kernels_ms": dstage.get("dec_prep", 0.0),
                              "decode_kernel_frac_of_measured": dec_bytes / (kms * 1e-3) / 1e9 / peak if kms else None,
                              "traffic": ncu_traffic("decode", n_tot),
                              "calls_per_step": 1, "in_place": True}

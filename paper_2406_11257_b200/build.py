@@ -13,8 +13,24 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
               "-fmad=false", "-Xcompiler", "-fPIC", "-cudart", "static"]
 
 
+STAMP = os.path.join(HERE, "libexcp.flags")          # the extra flags the library was last built with
+
+
+def extra_flags() -> list[str]:
+    """Extra nvcc flags from the environment (EXCP_NVCC_FLAGS), e.g. -DEXCP_DEBUG_BOUNDS for the build whose
+    kernels check every index they form and report through the call's status instead of faulting."""
+    return os.environ.get("EXCP_NVCC_FLAGS", "").split()
+
+
 def _stale() -> bool:
     if not os.path.exists(LIB):
+        return True
+    try:
+        with open(STAMP) as f:
+            built_with = f.read().split()
+    except OSError:
+        built_with = []
+    if built_with != extra_flags():
         return True
     t = os.path.getmtime(LIB)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)]
@@ -31,7 +47,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     procs = []
     for src in SOURCES:
         obj = os.path.join(CSRC, src[:-3] + ".o")
-        cmd = [nvcc, *NVCC_FLAGS, "-c", os.path.join(CSRC, src), "-o", obj]
+        cmd = [nvcc, *NVCC_FLAGS, *extra_flags(), "-c", os.path.join(CSRC, src), "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas=-v")
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
@@ -45,6 +61,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if failed:
         raise RuntimeError("nvcc failed")
     subprocess.check_call([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-cudart", "static", "-o", LIB, *objs, "-lrt", "-ldl", "-lpthread"])
+    with open(STAMP, "w") as f:
+        f.write(" ".join(extra_flags()))
     return LIB
 
 

@@ -6,8 +6,8 @@
 //            below reads a record that failed (so no read leaves the record)
 // popcount   survivors per tile from the bitmaps
 // scan       tensor-wide offsets; totals must equal the header's counts
-// decode     per tile: word prefix in shared memory, codes staged in shared
-//            memory, dense outputs
+// decode     per block of 1024 elements: ranks by a warp scan of the bitmap words, codes dealt
+//            out to the set positions, then the dense outputs
 #include "excp_common.cuh"
 
 namespace excp {
@@ -105,42 +105,255 @@ __global__ void __launch_bounds__(TPB) dec_scan_kernel(const DecDesc* __restrict
 // pruned) into the three sections of the dense layout instead.
 //
 // Warps are autonomous: a warp owns a contiguous run of tiles and nothing synchronises the block.
-// Per tile the warp loads the 2 x 128 bitmap words, turns their populations into the rank of
-// every word's first survivor (registers and shuffles), parks words and ranks in its own corner
-// of shared memory, and then walks the tile in 32 rounds of 128 elements, lane l taking four
-// consecutive elements: their survivors have consecutive ranks, so their codes are consecutive
-// bits of the section and one 32-bit window per stream (two aligned words read through the
-// cache) holds all four.
+// A tile is walked in four blocks of 1024 elements, each in two phases.
+//   A  lane l owns bitmap word l of the block (32 consecutive elements).  A warp scan of the
+//      words' populations gives the rank of every word's first survivor; the word's codes are then
+//      consecutive bits of the section, fetched as one window and dealt out to the word's set
+//      positions four elements at a time (a byte permute with a selector looked up by the 4 mask
+//      bits).  The result, one byte per element, goes to the warp's rows in shared memory (or, for
+//      the dense layout, straight to the container as 16 bytes per lane).
+//   B  eight rounds of 128 elements, lane l taking four consecutive ones: codes from the rows,
+//      centres from the table, 16-byte loads of W^_(t-1) and 16-byte stores of the three outputs,
+//      all rounds independent of one another.
+#ifndef EXCP_DEC_MIN_BLOCKS
+#define EXCP_DEC_MIN_BLOCKS 3                // resident blocks per SM the decoder's registers are held to
+#endif
+#ifndef EXCP_DEC_RB
+#define EXCP_DEC_RB 4                        // rounds of phase B whose loads are issued together
+#endif
 constexpr int DEC_WARPS = TPB / 32;
+constexpr int ROW_BYTES = 48;                // 32 codes + padding: 16-byte aligned, rows spread over the banks
+constexpr int CENT_SMEM = 16;                // centres kept in shared memory per stream (codes of at most 4 bits)
 
 struct DecodeSmem {
-    u32 bw[DEC_WARPS][TILE_WORDS], bo[DEC_WARPS][TILE_WORDS];   // the tile's bitmap words
-    u32 pw[DEC_WARPS][TILE_WORDS], po[DEC_WARPS][TILE_WORDS];   // survivors of the tile before each word
-    float cent[DEC_WARPS][3][KCAP];
+    unsigned char rows[DEC_WARPS][3][32 * ROW_BYTES];   // codes of the block in flight, one byte per element
+    float cent[DEC_WARPS][3][CENT_SMEM];
+    u32 sel[16];                             // 4 mask bits -> byte-permute selector (see expand_word)
+    u32 spread[16];                          // 4 mask bits -> 0x01 in every byte whose bit is set
 };
 
-// The `nb`-bit codes of up to four consecutive survivors starting at rank g of a section:
-// bits [g * nb, g * nb + 32) of it.  Words are read only where codes of these `have` survivors lie.
-__device__ __forceinline__ u32 code_window(const u32* __restrict__ sec, u64 g, u32 nb, u32 have) {
-    if (!have) return 0u;
-    const u64 bit = g * nb;
+// Code windows: the NB-bit codes of `cnt` consecutive survivors starting at rank g of a section, as
+// NB 32-bit words with the first code at bit 0.  Only words that hold such codes are read.
+template <int NB>
+__device__ __forceinline__ void load_window(const u32* __restrict__ sec, u64 g, u32 cnt, u32 (&c)[NB]) {
+    const u64 bit = g * NB;
     const u32 sh = (u32)bit & 31u;
-    const u32 lo = __ldg(sec + (bit >> 5));
-    const u32 hi = sh + have * nb > 32u ? __ldg(sec + (bit >> 5) + 1) : 0u;
-    return __funnelshift_r(lo, hi, sh);
+    const u32* p = sec + (bit >> 5);
+    const u32 nw = cnt ? (sh + cnt * NB + 31u) >> 5 : 0u;   // words that hold the codes
+    u32 w[NB + 1];
+#pragma unroll
+    for (int k = 0; k <= NB; ++k) w[k] = (u32)k < nw ? __ldg(p + k) : 0u;
+#pragma unroll
+    for (int k = 0; k < NB; ++k) c[k] = __funnelshift_r(w[k], w[k + 1], sh);
+}
+
+// The next four codes of a window as four bytes (code k in byte k).
+template <int NB>
+__device__ __forceinline__ u32 four_codes(u32 low) {
+    if (NB == 8) return low;
+    if (NB == 4) {
+        const u32 x = (low & 0x00ffu) | ((low & 0xff00u) << 8);
+        return (x | (x << 4)) & 0x0f0f0f0fu;
+    }
+    low &= 0xffu;                                        // NB == 2: two codes per half
+    const u32 x = (low | (low << 12)) & 0x000f000fu;
+    return (x | (x << 6)) & 0x03030303u;
+}
+
+// Deals the codes of window c to the set positions of bitmap word `m`: out[j] holds elements
+// 4j .. 4j+3 of the word, one byte each, 0 where the bit is clear.  Returns non-zero if a
+// survivor's code is 0 (no record written by the compressor has one).
+template <int NB>
+__device__ __forceinline__ u32 expand_word(u32 m, u32 (&c)[NB], const u32* __restrict__ sel,
+                                           const u32* __restrict__ spread, u32 (&out)[8]) {
+    u32 bad = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const u32 m4 = (m >> (4 * j)) & 15u;
+        const u32 o = __byte_perm(four_codes<NB>(c[0]), 0u, sel[m4]);
+        u32 any = o | (o >> 1);                          // bit 0 of every byte: the byte's code is not 0
+        if (NB >= 4) any |= (o >> 2) | (o >> 3);
+        if (NB == 8) any |= (o >> 4) | (o >> 5) | (o >> 6) | (o >> 7);
+        const u32 nz = any & 0x01010101u;
+        bad |= nz ^ spread[m4];
+        out[j] = o;
+        const u32 s = (u32)__popc(m4) * NB;              // bits used: at most 32
+        if (NB == 8 && s == 32u) {
+#pragma unroll
+            for (int k = 0; k + 1 < NB; ++k) c[k] = c[k + 1];
+            c[NB - 1] = 0u;
+        } else {
+#pragma unroll
+            for (int k = 0; k + 1 < NB; ++k) c[k] = __funnelshift_r(c[k], c[k + 1], s);
+            c[NB - 1] >>= s;
+        }
+    }
+    return bad;
+}
+
+// Eight bytes-per-element words -> four nibbles-per-element words (the dense layout's 16 bytes).
+__device__ __forceinline__ uint4 pack_nibbles(const u32 (&o)[8]) {
+    u32 d[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        u32 lo = o[2 * q], hi = o[2 * q + 1];
+        lo = (lo | (lo >> 4)) & 0x00ff00ffu; lo = (lo | (lo >> 8)) & 0xffffu;
+        hi = (hi | (hi >> 4)) & 0x00ff00ffu; hi = (hi | (hi >> 8)) & 0xffffu;
+        d[q] = lo | (hi << 16);
+    }
+    return make_uint4(d[0], d[1], d[2], d[3]);
+}
+
+struct DecTile {                 // what the phases need to know about the tile in hand
+    const unsigned char* rec;
+    const u32 *sec0, *sec1, *sec2;
+    u64 n, base;                 // elements of the tensor; first element of the tile
+    u32 rflags;
+    int tensor;
+};
+
+// One block of 1024 elements whose codes are NB bits wide.  a, b: this lane's words of the two
+// bitmaps; gw, go: ranks of their first survivors.
+template <bool DENSE, int NB, typename WT>
+__device__ __forceinline__ u32 decode_block(const DecTile& t, const DecDesc& d, const DecState& s, DecodeSmem& sm, int warp,
+                                            int lane, u32 blk, u32 a, u32 b, u64 gw, u64 go) {
+    u32 bad = 0;
+    u32 ow8[8], oa8[8], os8[8];
+    {
+        u32 c[NB];
+        load_window<NB>(t.sec0, gw, (u32)__popc(a), c);
+        bad |= expand_word<NB>(a, c, sm.sel, sm.spread, ow8);
+    }
+    {
+        u32 c1[NB], c2[NB];
+        load_window<NB>(t.sec1, go, (u32)__popc(b), c1);
+        load_window<NB>(t.sec2, go, (u32)__popc(b), c2);
+        bad |= expand_word<NB>(b, c1, sm.sel, sm.spread, oa8);
+        bad |= expand_word<NB>(b, c2, sm.sel, sm.spread, os8);
+    }
+    const u64 e0 = t.base + (u64)blk * 1024u;            // first element of the block
+    if (DENSE) {                                         // NB == 4: 32 codes = 16 bytes per lane and section
+        const u64 i = e0 + 32u * lane;
+        if (i < t.n) {
+            const u64 sb = dense_section_bytes(t.n, BITS);
+            unsigned char* out = d.dense + header_bytes(KMAX) + i / 2;
+            *reinterpret_cast<uint4*>(out) = pack_nibbles(ow8);
+            *reinterpret_cast<uint4*>(out + sb) = pack_nibbles(oa8);
+            *reinterpret_cast<uint4*>(out + 2 * sb) = pack_nibbles(os8);
+        }
+        return bad;
+    }
+    unsigned char* rw = sm.rows[warp][0] + lane * ROW_BYTES;
+    unsigned char* ra = sm.rows[warp][1] + lane * ROW_BYTES;
+    unsigned char* rs = sm.rows[warp][2] + lane * ROW_BYTES;
+    reinterpret_cast<uint4*>(rw)[0] = make_uint4(ow8[0], ow8[1], ow8[2], ow8[3]);
+    reinterpret_cast<uint4*>(rw)[1] = make_uint4(ow8[4], ow8[5], ow8[6], ow8[7]);
+    reinterpret_cast<uint4*>(ra)[0] = make_uint4(oa8[0], oa8[1], oa8[2], oa8[3]);
+    reinterpret_cast<uint4*>(ra)[1] = make_uint4(oa8[4], oa8[5], oa8[6], oa8[7]);
+    reinterpret_cast<uint4*>(rs)[0] = make_uint4(os8[0], os8[1], os8[2], os8[3]);
+    reinterpret_cast<uint4*>(rs)[1] = make_uint4(os8[4], os8[5], os8[6], os8[7]);
+    __syncwarp();
+    const WT* w_prev = static_cast<const WT*>(d.w_prev);
+    WT* w_out = static_cast<WT*>(d.w_out);
+    const bool absolute = t.rflags & REC_ABSOLUTE;       // the weight stream is W itself
+    const float* cw = NB <= 4 ? sm.cent[warp][0] : s.cent[0];   // wide codes: the table stays in global memory (cached)
+    const float* ca = NB <= 4 ? sm.cent[warp][1] : s.cent[1];
+    const float* cs = NB <= 4 ? sm.cent[warp][2] : s.cent[2];
+    constexpr int RB = EXCP_DEC_RB;
+#pragma unroll
+    for (int r0 = 0; r0 < 8; r0 += RB) {
+        float wp[RB][4];
+#pragma unroll
+        for (int r = 0; r < RB; ++r) {
+            const u64 i0 = e0 + (u32)(r0 + r) * 128u + 4u * lane;
+            wp[r][0] = wp[r][1] = wp[r][2] = wp[r][3] = 0.f;
+            if (!absolute && i0 < t.n) load4(w_prev, i0, t.n, wp[r]);
+        }
+#pragma unroll
+        for (int r = 0; r < RB; ++r) {
+            const u32 e = (u32)(r0 + r) * 128u + 4u * lane;             // element within the block
+            const u64 i0 = e0 + e;
+            if (i0 >= t.n) continue;
+            const u32 ro = (e >> 5) * ROW_BYTES + (e & 31u);
+            const u32 kw = *reinterpret_cast<const u32*>(sm.rows[warp][0] + ro);
+            const u32 ka = *reinterpret_cast<const u32*>(sm.rows[warp][1] + ro);
+            const u32 ks = *reinterpret_cast<const u32*>(sm.rows[warp][2] + ro);
+            float ow[4], oa[4], os[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const u32 c0 = (kw >> (8 * k)) & 255u, c1 = (ka >> (8 * k)) & 255u, c2 = (ks >> (8 * k)) & 255u;
+                ow[k] = c0 ? __fadd_rn(wp[r][k], cw[c0 - 1]) : wp[r][k];   // pruned: W^_(t-1) bit for bit
+                oa[k] = c1 ? ca[c1 - 1] : 0.f;
+                os[k] = c2 ? cs[c2 - 1] : 0.f;
+            }
+            store4(w_out, i0, t.n, ow);
+            store4(d.ea_out, i0, t.n, oa);
+            store4(d.eas_out, i0, t.n, os);
+        }
+    }
+    __syncwarp();                                        // the rows are free again
+    return bad;
+}
+
+// A block of a record whose sections hold the survivors themselves (fp32, no codes): every element
+// first gets its pruned value, then every lane puts the survivors of its word in place.
+template <typename WT>
+__device__ __forceinline__ void decode_block_raw(const DecTile& t, const DecDesc& d, int lane, u32 blk, u32 a, u32 b,
+                                                 u64 gw, u64 go) {
+    const WT* w_prev = static_cast<const WT*>(d.w_prev);
+    WT* w_out = static_cast<WT*>(d.w_out);
+    const bool absolute = t.rflags & REC_ABSOLUTE;
+    const u64 e0 = t.base + (u64)blk * 1024u;
+    const float zero[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 2
+    for (int r = 0; r < 8; ++r) {
+        const u64 i0 = e0 + (u32)r * 128u + 4u * lane;
+        if (i0 >= t.n) continue;
+        float wp[4] = {0.f, 0.f, 0.f, 0.f};
+        if (!absolute) load4(w_prev, i0, t.n, wp);
+        store4(w_out, i0, t.n, wp);
+        store4(d.ea_out, i0, t.n, zero);
+        store4(d.eas_out, i0, t.n, zero);
+    }
+    __syncwarp();                                        // the warp's stores above are ordered before the ones below
+    const u64 i = e0 + 32u * lane;
+    for (u32 m = a; m; m &= m - 1u) {
+        const u64 el = i + (u32)__ffs((int)m) - 1u;
+        const float v = __uint_as_float(__ldg(t.sec0 + gw++));
+        wput(w_out, el, absolute ? v : __fadd_rn(wget(w_out, el), v));
+    }
+    for (u32 m = b; m; m &= m - 1u) {
+        const u64 el = i + (u32)__ffs((int)m) - 1u;
+        d.ea_out[el] = __uint_as_float(__ldg(t.sec1 + go));
+        d.eas_out[el] = __uint_as_float(__ldg(t.sec2 + go));
+        ++go;
+    }
+    __syncwarp();
 }
 
 template <bool DENSE, typename WT>
-__global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__ descs,
+__global__ void __launch_bounds__(TPB, EXCP_DEC_MIN_BLOCKS) decode_kernel(const DecDesc* __restrict__ descs,
                                                      const DecState* __restrict__ st, int nt, u32 tiles,
                                                      Workspace ws, CallState* call) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     DecodeSmem& sm = *reinterpret_cast<DecodeSmem*>(smem_raw);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x < 16) {
+        // selector: byte p of the output takes the next unused code if bit p of the mask is set, else
+        // byte 4 of the permute's operand pair (a zero)
+        u32 sel = 0, spread = 0, next = 0;
+        for (u32 p = 0; p < 4; ++p) {
+            const bool on = (threadIdx.x >> p) & 1u;
+            sel |= (on ? next : 4u) << (4 * p);
+            spread |= (on ? 1u : 0u) << (8 * p);
+            next += on;
+        }
+        sm.sel[threadIdx.x] = sel;
+        sm.spread[threadIdx.x] = spread;
+    }
+    __syncthreads();
     const u32 gw = blockIdx.x * DEC_WARPS + warp, nw = gridDim.x * DEC_WARPS;
     const u32 wlo = (u32)(((u64)tiles * gw) / nw), whi = (u32)(((u64)tiles * (gw + 1)) / nw);
-    u32* bw = sm.bw[warp]; u32* bo = sm.bo[warp]; u32* pw = sm.pw[warp]; u32* po = sm.po[warp];
-    float (*cent)[KCAP] = sm.cent[warp];
     int cur = -1;
     u32 tb = 0, ntl = 0;
     u32 bad = 0;
@@ -149,128 +362,62 @@ __global__ void __launch_bounds__(TPB) decode_kernel(const DecDesc* __restrict__
             cur = find_tensor(descs, nt, tile);
             tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
             __syncwarp();
-            if (st[cur].valid) {
+            if (!DENSE && st[cur].valid && st[cur].bits <= 4) {
                 const int kc = centres_of((int)st[cur].bits);
-                for (int i = lane; i < 3 * kc; i += 32) cent[i / kc][i % kc] = st[cur].cent[i / kc][i % kc];
+                for (int i = lane; i < 3 * CENT_SMEM; i += 32)
+                    sm.cent[warp][i / CENT_SMEM][i % CENT_SMEM] = i % CENT_SMEM < kc ? st[cur].cent[i / CENT_SMEM][i % CENT_SMEM] : 0.f;
             }
             __syncwarp();
         }
         if (!st[cur].valid) continue;
         const DecDesc& d = descs[cur];
         const DecState& s = st[cur];
-        const WT* w_prev = static_cast<const WT*>(d.w_prev);
-        WT* w_out = static_cast<WT*>(d.w_out);
-        const u64 n = d.numel;
-        const u64 nwords = bitmap_bytes(n) / 4;
+        DecTile t;
+        t.rec = d.rec; t.n = d.numel; t.rflags = s.rflags; t.tensor = cur;
+        t.base = (u64)(tile - tb) * TILE;
+        t.sec0 = reinterpret_cast<const u32*>(d.rec + s.off_codes[0]);
+        t.sec1 = reinterpret_cast<const u32*>(d.rec + s.off_codes[1]);
+        t.sec2 = reinterpret_cast<const u32*>(d.rec + s.off_codes[2]);
+        const u64 nwords = bitmap_bytes(t.n) / 4;
         const u64 w0 = (u64)(tile - tb) * TILE_WORDS;
-        const u32 offw = ws.tile_off_w[tile], offo = ws.tile_off_o[tile];
-        {   // lane l holds words 4l .. 4l+3 of both bitmaps; ranks by a scan over the lanes
-            u32 a[4], b[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                a[k] = bm_word(d.rec, s.off_bm_w, nwords, w0 + 4 * lane + k);
-                b[k] = bm_word(d.rec, s.off_bm_o, nwords, w0 + 4 * lane + k);
-                if (!(s.rflags & REC_MOMENTS_FREE)) bad |= b[k] & ~a[k];   // a moment kept where the weight is pruned
+        const bool last_tile = t.base + TILE > t.n;      // the tensor ends in this tile
+        u64 rank_w = ws.tile_off_w[tile], rank_o = ws.tile_off_o[tile];
+        const bool raw = s.rflags & REC_RAW;
+        const u32 bits = s.bits;
+#pragma unroll 1
+        for (u32 blk = 0; blk < TILE / 1024; ++blk) {
+            if (w0 + blk * 32u >= nwords) break;          // past the stored bitmap: nothing left in this tile
+            const u64 wi = w0 + blk * 32u + lane;
+            const u32 a = bm_word(d.rec, s.off_bm_w, nwords, wi);
+            const u32 b = bm_word(d.rec, s.off_bm_o, nwords, wi);
+            if (!(s.rflags & REC_MOMENTS_FREE)) bad |= b & ~a;       // a moment kept where the weight is pruned
+            if (last_tile) {                             // no bit at or past the last element
+                const u64 e = wi * 32;
+                const u32 stray = e >= t.n ? 0xffffffffu : (t.n - e >= 32 ? 0u : 0xffffffffu << (u32)(t.n - e));
+                bad |= (a | b) & stray;
             }
-            if ((u64)(tile - tb + 1) * TILE > n) {        // the tensor ends in this tile: no bit at or past its last element
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const u64 e = (w0 + 4 * lane + k) * 32;                 // first element of the word
-                    const u32 stray = e >= n ? 0xffffffffu : (n - e >= 32 ? 0u : 0xffffffffu << (u32)(n - e));
-                    bad |= (a[k] | b[k]) & stray;
-                }
-            }
-            const u32 ta = __popc(a[0]) + __popc(a[1]) + __popc(a[2]) + __popc(a[3]);
-            const u32 tbm = __popc(b[0]) + __popc(b[1]) + __popc(b[2]) + __popc(b[3]);
-            u32 ia = ta, ib = tbm;
+            const u32 pa = (u32)__popc(a), pb = (u32)__popc(b);
+            u32 ia = pa, ib = pb;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const u32 x = __shfl_up_sync(0xffffffffu, ia, o), y = __shfl_up_sync(0xffffffffu, ib, o);
                 if (lane >= o) { ia += x; ib += y; }
             }
-            u32 ra = ia - ta, rb = ib - tbm;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                bw[4 * lane + k] = a[k]; bo[4 * lane + k] = b[k];
-                pw[4 * lane + k] = ra; po[4 * lane + k] = rb;
-                ra += __popc(a[k]); rb += __popc(b[k]);
-            }
-        }
-        __syncwarp();
-        const bool raw = s.rflags & REC_RAW;              // sections hold fp32 survivors
-        const bool absolute = s.rflags & REC_ABSOLUTE;    // the weight stream is W itself
-        const u32 nb = raw ? 32u : s.bits;
-        const u32 cmask = raw ? 0xffffffffu : (1u << nb) - 1u;
-        const u32* sec0 = reinterpret_cast<const u32*>(d.rec + s.off_codes[0]);
-        const u32* sec1 = reinterpret_cast<const u32*>(d.rec + s.off_codes[1]);
-        const u32* sec2 = reinterpret_cast<const u32*>(d.rec + s.off_codes[2]);
-        const u64 base = (u64)(tile - tb) * TILE;
-#pragma unroll 2
-        for (int r = 0; r < TILE / 128; ++r) {
-            const u32 e0 = r * 128 + lane * 4;            // element within the tile
-            const u64 i0 = base + e0;
-            const bool live = i0 < n;
-            if (!DENSE && !__any_sync(0xffffffffu, live)) break;
-            float wp[4] = {0.f, 0.f, 0.f, 0.f};
-            if (!DENSE && !absolute && live) load4(w_prev, i0, n, wp);
-            const u32 word = e0 >> 5, bit = e0 & 31;
-            const u32 mw4 = (bw[word] >> bit) & 15u, mo4 = (bo[word] >> bit) & 15u;
-            const u64 gw0 = (u64)offw + pw[word] + __popc(bw[word] & ((1u << bit) - 1u));
-            const u64 go0 = (u64)offo + po[word] + __popc(bo[word] & ((1u << bit) - 1u));
-            float ow[4], oa[4], os[4];
-            u32 nib0 = 0, nib1 = 0, nib2 = 0;             // DENSE: the four codes per stream
-            if (!raw) {
-                u32 win0 = code_window(sec0, gw0, nb, __popc(mw4));
-                u32 win1 = code_window(sec1, go0, nb, __popc(mo4));
-                u32 win2 = code_window(sec2, go0, nb, __popc(mo4));
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    ow[k] = wp[k]; oa[k] = 0.f; os[k] = 0.f;
-                    if ((mw4 >> k) & 1u) {
-                        const u32 c = win0 & cmask;
-                        win0 >>= nb;
-                        if (c == 0) bad = 1; else ow[k] = __fadd_rn(wp[k], cent[0][c - 1]);
-                        nib0 |= c << (4 * k);
-                    }
-                    if ((mo4 >> k) & 1u) {
-                        const u32 c1 = win1 & cmask, c2 = win2 & cmask;
-                        win1 >>= nb; win2 >>= nb;
-                        if (c1 == 0 || c2 == 0) bad = 1;
-                        else { oa[k] = cent[1][c1 - 1]; os[k] = cent[2][c2 - 1]; }
-                        nib1 |= c1 << (4 * k);
-                        nib2 |= c2 << (4 * k);
-                    }
-                }
+            const u64 gwl = rank_w + ia - pa, gol = rank_o + ib - pb;
+            rank_w += __shfl_sync(0xffffffffu, ia, 31);
+            rank_o += __shfl_sync(0xffffffffu, ib, 31);
+            if (__any_sync(0xffffffffu, bad)) break;     // nothing is decoded past an inconsistency
+            if (raw) {
+                if (!DENSE) decode_block_raw<WT>(t, d, lane, blk, a, b, gwl, gol);
+            } else if (DENSE || bits == 4) {
+                bad |= decode_block<DENSE, 4, WT>(t, d, s, sm, warp, lane, blk, a, b, gwl, gol);
+            } else if (bits == 2) {
+                bad |= decode_block<false, 2, WT>(t, d, s, sm, warp, lane, blk, a, b, gwl, gol);
             } else {
-                u64 gw = gw0, go = go0;
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    ow[k] = wp[k]; oa[k] = 0.f; os[k] = 0.f;
-                    if ((mw4 >> k) & 1u) ow[k] = __fadd_rn(wp[k], __uint_as_float(__ldg(sec0 + gw++)));
-                    if ((mo4 >> k) & 1u) { oa[k] = __uint_as_float(__ldg(sec1 + go)); os[k] = __uint_as_float(__ldg(sec2 + go)); ++go; }
-                }
-            }
-            if (DENSE) {
-                // eight lanes hold 32 consecutive elements = 16 bytes of each section: gather them in
-                // the first of the eight and write them with one store
-                u32 v[3] = {nib0, nib1, nib2};
-                const u64 sb = dense_section_bytes(n, BITS);
-                unsigned char* sec = d.dense + header_bytes(KMAX) + i0 / 2;
-#pragma unroll
-                for (int j = 0; j < 3; ++j) {
-                    const u32 pair = v[j] | (__shfl_down_sync(0xffffffffu, v[j], 1) << 16);
-                    const u32 y = __shfl_down_sync(0xffffffffu, pair, 2);
-                    const u32 z = __shfl_down_sync(0xffffffffu, pair, 4);
-                    const u32 w = __shfl_down_sync(0xffffffffu, pair, 6);
-                    if ((lane & 7) == 0 && live) *reinterpret_cast<uint4*>(sec + j * sb) = make_uint4(pair, y, z, w);
-                }
-            } else if (live) {
-                store4(w_out, i0, n, ow);
-                store4(d.ea_out, i0, n, oa);
-                store4(d.eas_out, i0, n, os);
+                bad |= decode_block<false, 8, WT>(t, d, s, sm, warp, lane, blk, a, b, gwl, gol);
             }
         }
-        __syncwarp();                                     // the warp's shared-memory corner is free again
+        if (__any_sync(0xffffffffu, bad)) break;
     }
     if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(&call->flags, FLAG_CORRUPT);
 }
@@ -282,7 +429,7 @@ void launch_decode(const LaunchCfg& cfg, const DecDesc* descs, DecState* st, int
     dec_popcount_kernel<<<(tiles + TPB / 32 - 1) / (TPB / 32), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws);
     dec_scan_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, ws, call);
     prof_mark(cfg, ST_DEC_PREP, 3);
-    const u32 grid = min((tiles + DEC_WARPS - 1) / DEC_WARPS, (u32)cfg.sms * 4u);
+    const u32 grid = min((tiles + DEC_WARPS - 1) / DEC_WARPS, (u32)cfg.sms * (u32)EXCP_DEC_MIN_BLOCKS);
     const size_t smem = sizeof(DecodeSmem);
     auto run = [&](auto tag) {
         using WT = decltype(tag);
@@ -343,7 +490,7 @@ void launch_record_to_dense(const LaunchCfg& cfg, const DecDesc* descs, DecState
     dense_header_kernel<<<nt, 64, 0, cfg.stream>>>(descs, st, call);
     prof_mark(cfg, ST_DEC_PREP, tiles ? 4 : 2);
     if (!tiles) return;
-    const u32 grid = min((tiles + DEC_WARPS - 1) / DEC_WARPS, (u32)cfg.sms * 4u);
+    const u32 grid = min((tiles + DEC_WARPS - 1) / DEC_WARPS, (u32)cfg.sms * (u32)EXCP_DEC_MIN_BLOCKS);
     cudaFuncSetAttribute(decode_kernel<true, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecodeSmem));
     decode_kernel<true, float><<<grid, TPB, sizeof(DecodeSmem), cfg.stream>>>(descs, st, nt, tiles, ws, call);
     prof_mark(cfg, ST_DENSE, 1);
