@@ -13,10 +13,38 @@
 
 namespace excp {
 
-constexpr int MCH = 512;             // values per stream per staged chunk
-constexpr int MST = 2;               // chunks in flight per warp
-constexpr int MWARPS = 7;            // 7 warps x 16 KB of stages: two blocks per SM
+#ifndef EXCP_MC_CH
+#define EXCP_MC_CH 512
+#endif
+#ifndef EXCP_MC_ST
+#define EXCP_MC_ST 2
+#endif
+#ifndef EXCP_MC_WARPS
+#define EXCP_MC_WARPS 7
+#endif
+#ifndef EXCP_MC_BLOCKS
+#define EXCP_MC_BLOCKS 2
+#endif
+constexpr int MCH = EXCP_MC_CH;      // values per stream per staged chunk
+constexpr int MST = EXCP_MC_ST;      // chunks in flight per warp
+constexpr int MWARPS = EXCP_MC_WARPS;   // 7 warps x 16 KB of stages: two blocks per SM
+constexpr int MBLOCKS = EXCP_MC_BLOCKS; // resident blocks per SM
 constexpr int MTPB = MWARPS * 32;
+
+// sqrt(x) to within a few units in the last place (the hardware's approximation; its documented
+// relative error is 2^-23).  Used only to decide the elements that are far from the threshold.
+__device__ __forceinline__ float sqrt_fast(float x) {
+    float r;
+    asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
+// Eq. (rw) is decided on lhs = |dW| (x) sqrt_rn(eas) in fp32.  With the approximate root the product
+// differs from lhs by well under 2^-20 of its value (plus a subnormal's spacing), so outside the band
+// [lo, hi] around the threshold the approximate product decides exactly as lhs would; inside it the
+// warp recomputes with the correctly rounded root.
+constexpr float BAND = 1.f / 262144.f;        // 2^-18
+constexpr float TINY = 7.174648e-43f;         // 2^-140
 
 struct MaskSmem {
     float buf[MWARPS][MST][4][MCH];
@@ -29,7 +57,7 @@ struct MaskSmem {
 // VARIANT = false is the method; VARIANT = true adds the ablation switches `opt` (OPT_*), kept
 // out of the method's own instruction stream.
 template <bool VARIANT, typename WT>
-__global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc* __restrict__ descs,
+__global__ void __launch_bounds__(MTPB, MBLOCKS) mask_compact_kernel(const TensorDesc* __restrict__ descs,
                                                               TensorState* __restrict__ st, int nt,
                                                               u32 tiles, Workspace ws, CallState* call, u32 opt) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -49,6 +77,7 @@ __global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc*
     const WT* ipw[2] = {nullptr, nullptr};                          // and its weight streams W_t, W^_(t-1)
     const WT* cpw[2] = {nullptr, nullptr};
     float thr_w = 0.f, thr_o = 0.f;
+    float thr_lo = 0.f, thr_hi = 0.f;        // the band around thr_w (non-variant path)
     u32 rw = 0, ro = 0;               // survivors of the current tile so far (warp uniform)
     float mk0 = 0.f, mk1 = 0.f, mk2 = 0.f;   // running max magnitudes of the survivors
     float nanacc = 0.f;                      // turns NaN once any input is NaN or infinite
@@ -87,6 +116,8 @@ __global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc*
             cpw[0] = static_cast<const WT*>(descs[cc.tns].w_t); cpw[1] = static_cast<const WT*>(descs[cc.tns].w_prev);
             cp[2] = descs[cc.tns].ea; cp[3] = descs[cc.tns].eas;
             thr_w = st[cc.tns].thr_w; thr_o = st[cc.tns].thr_o;
+            thr_lo = __fsub_rd(__fmul_rd(thr_w, 1.f - BAND), TINY);
+            thr_hi = __fadd_ru(__fmul_ru(thr_w, 1.f + BAND), TINY);
         }
         const u32 valid = cc.valid(), nbulk = valid & ~(BULK_ALIGN - 1u);
         const u64 e0 = cc.elem0();
@@ -110,6 +141,8 @@ __global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc*
             if (FULL || (u32)step * 128u < valid) {
                 u32 bw[4], bo[4];
                 float dwv[4], eav[4], easv[4];
+                bool kwv[4], kov[4];
+                bool amb = false;
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const u32 i = step * 128 + k * 32 + lane;
@@ -123,26 +156,43 @@ __global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc*
                     } else {
                         a = b = e = v = 0.f;
                     }
-                    nanacc = __fmaf_rn(a, 0.f, nanacc);       // inf * 0 and NaN * 0 are NaN
-                    nanacc = __fmaf_rn(b, 0.f, nanacc);
-                    nanacc = __fmaf_rn(e, 0.f, nanacc);
-                    nanacc = __fmaf_rn(v, 0.f, nanacc);
-                    minv = fminf(minv, v);
                     const float dw = no_prev ? a : __fsub_rn(a, b);              // Eq. (ckpt_res)
                     bool kw, ko;
                     if (!VARIANT) {
-                        const float lhs = __fmul_rn(fabsf(dw), __fsqrt_rn(v));
-                        kw = lhs > thr_w;                                        // Eq. (rw); past numel: 0 > thr is false
-                        ko = kw && (fabsf(e) > thr_o);                           // Eq. (ro)
+                        // a NaN, an infinity or a negative second moment anywhere makes the product NaN or
+                        // infinite; so can finite values that overflow, which the exact check at the end tells apart
+                        const float lhs = __fmul_rn(fabsf(dw), sqrt_fast(v));
+                        nanacc = __fmaf_rn(lhs, 0.f, nanacc);     // inf * 0 and NaN * 0 are NaN
+                        nanacc = __fmaf_rn(e, 0.f, nanacc);
+                        kw = lhs > thr_hi;                                       // Eq. (rw); past numel: 0 > thr is false
+                        amb |= kw != (lhs >= thr_lo);
+                        ko = fabsf(e) > thr_o;                                   // Eq. (ro), before the conjunction
                     } else {
+                        nanacc = __fmaf_rn(a, 0.f, nanacc);
+                        nanacc = __fmaf_rn(b, 0.f, nanacc);
+                        nanacc = __fmaf_rn(e, 0.f, nanacc);
+                        nanacc = __fmaf_rn(v, 0.f, nanacc);
+                        minv = fminf(minv, v);
                         const bool real = FULL || i < valid;
                         const float lhs = (opt & OPT_NO_M2W) ? fabsf(dw) : __fmul_rn(fabsf(dw), __fsqrt_rn(v));
                         kw = real && ((opt & OPT_NO_PRUNE) || lhs > thr_w);
                         ko = real && ((opt & OPT_NO_PRUNE) || (fabsf(e) > thr_o && ((opt & OPT_NO_W2M) || kw)));
                     }
-                    bw[k] = __ballot_sync(0xffffffffu, kw);
-                    bo[k] = __ballot_sync(0xffffffffu, ko);
+                    kwv[k] = kw; kov[k] = ko;
                     dwv[k] = dw; eav[k] = e; easv[k] = v;
+                }
+                if (!VARIANT) {
+                    if (__any_sync(0xffffffffu, amb)) {          // rare: some product lies next to the threshold
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) kwv[k] = __fmul_rn(fabsf(dwv[k]), __fsqrt_rn(easv[k])) > thr_w;
+                    }
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) kov[k] = kov[k] && kwv[k];       // the joint rule
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    bw[k] = __ballot_sync(0xffffffffu, kwv[k]);
+                    bo[k] = __ballot_sync(0xffffffffu, kov[k]);
                 }
                 if (lane < 4) {
                     const u64 wi = (u64)cc.tile * TILE_WORDS + cc.chunk * (MCH / 32) + step * 4 + lane;
@@ -178,7 +228,27 @@ __global__ void __launch_bounds__(MTPB, 2) mask_compact_kernel(const TensorDesc*
         cc.next();
     }
     if (prev >= 0) flush_max(prev);
-    const bool bad = (nanacc != nanacc) || (minv < 0.f);
+    bool bad = (nanacc != nanacc) || (minv < 0.f);
+    if (!VARIANT && __any_sync(0xffffffffu, bad)) {
+        // The products went NaN or infinite somewhere in this warp's run.  Tell an invalid input from
+        // finite values that overflowed: look at the inputs themselves (plain loads; this path is cold).
+        bad = false;
+        TileWalk<MCH> rc;
+        rc.start(wlo);
+        while (rc.tile < whi) {
+            rc.enter_tile(descs, nt);
+            const TensorDesc& d = descs[rc.tns];
+            const WT* wt = static_cast<const WT*>(d.w_t);
+            const WT* wp = static_cast<const WT*>(d.w_prev);
+            for (u32 i = lane; i < rc.tv; i += 32) {
+                const u64 el = rc.toff + i;
+                const float a = wget(wt, el), b = wget(wp, el), e = d.ea[el], v = d.eas[el];
+                const float z = __fmaf_rn(a, 0.f, __fmaf_rn(b, 0.f, __fmaf_rn(e, 0.f, __fmul_rn(v, 0.f))));
+                bad |= (z != z) || (v < 0.f);
+            }
+            ++rc.tile;
+        }
+    }
     if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(&call->flags, FLAG_NONFINITE);
 }
 
@@ -240,7 +310,7 @@ __global__ void __launch_bounds__(MAX_GROUP_TENSORS) layout_kernel(const TensorD
 void launch_mask_compact(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                          const Workspace& ws, const Params& p, CallState* call, u64 blob_capacity) {
     if (tiles) {
-        const u32 grid = min((tiles + MWARPS - 1) / MWARPS, (u32)cfg.sms * 2u);
+        const u32 grid = min((tiles + MWARPS - 1) / MWARPS, (u32)cfg.sms * (u32)MBLOCKS);
         const u32 opt = p.flags & (OPT_NO_W2M | OPT_NO_M2W | OPT_NO_RESIDUAL | OPT_NO_PRUNE);
         auto run = [&](auto tag) {
             using WT = decltype(tag);
