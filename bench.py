@@ -338,7 +338,7 @@ KERNEL_SOURCES = {                                  # what each stage's dominant
     "mask_compact": ["mask_compact.cu", "warp_ring.cuh", "tma.cuh", "excp_common.cuh"],
     "cell_count": ["kmeans.cu", "excp_common.cuh"],
     "cell_gather": ["kmeans.cu", "excp_common.cuh"],
-    "pack_codes": ["pack.cu", "seg_ring.cuh", "tma.cuh", "excp_common.cuh"],
+    "pack_codes": ["pack.cu", "excp_common.cuh"],
     "decode": ["decode.cu", "warp_ring.cuh", "tma.cuh", "excp_common.cuh"],
 }
 

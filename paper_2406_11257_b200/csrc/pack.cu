@@ -6,7 +6,6 @@
 // last 32-bit code word of a tile may be shared with its neighbours: those words
 // are cleared beforehand and OR-ed into; interior words are stored whole.
 #include "excp_common.cuh"
-#include "seg_ring.cuh"
 
 namespace excp {
 
@@ -102,21 +101,29 @@ __global__ void __launch_bounds__(TPB) clear_edges_kernel(const TensorDesc* __re
     }
 }
 
-// Final assignment + packing: NS = 1 for dW, NS = 2 for the two moment streams together.
-// A warp owns a run of tiles and streams their survivor segments through its ring of stages
-// (see seg_ring.cuh).  Within a tile the survivors form rows of 8 (one 32-bit word of codes in
-// the tile's own alignment); the tile starts at an arbitrary rank of the tensor, so every
-// output word is two neighbouring rows funnel-shifted by the rank's offset in its word.
-constexpr int PST = 2;
+// Final assignment + packing: NS = 1 for dW, NS = 2 for the two moment streams together (they
+// share their counts).  A warp owns a run of tiles and reads their survivor segments with plain
+// 16-byte loads.  Within a tile the survivors form rows of 32 / NB (one 32-bit word of codes in the
+// tile's own alignment), one row per lane; the tile starts at an arbitrary rank of the tensor, so
+// every output word is two neighbouring rows funnel-shifted by the rank's offset in its word: the
+// neighbour's row comes by a shuffle, the last row of the previous 32 through a register.
 constexpr int PWARPS = TPB / 32;
 
-template <int NS, int CH, int NB>
+template <int NS, int NB>
 struct PackSmem {
-    float buf[PWARPS][PST][NS][CH];
-    unsigned long long bar[PWARPS][PST];
     float thr[PWARPS][NS][1 << NB];     // the K - 1 thresholds, +inf after them
-    u32 rows[PWARPS][NS][CH * NB / 32 + 2];   // [0] = last row of the previous chunk, then this chunk's rows
 };
+
+// Cluster of x = number of thresholds strictly below it.  thr_row: 16 fp32 thresholds
+// (ascending, +inf from the 15th on, none of them -0) in shared memory; t3, t7, t11 are copies
+// in registers.  Returns 4 * cluster.
+__device__ __forceinline__ u32 find_cluster4(float x, float t3, float t7, float t11, const char* thr_row) {
+    u32 p = x > t7 ? 32u : 0u;
+    p += (x > (p ? t11 : t3)) ? 16u : 0u;
+    p += (x > *reinterpret_cast<const float*>(thr_row + p + 4)) ? 8u : 0u;
+    p += (x > *reinterpret_cast<const float*>(thr_row + p)) ? 4u : 0u;
+    return p;
+}
 
 // Cluster of x = number of thresholds below it: NB halving steps over the 2^NB - 1 sorted entries
 // (thr[K - 1 ...] = +inf).
@@ -129,25 +136,21 @@ __device__ __forceinline__ u32 find_cluster(float x, const float* thr) {
     return p;
 }
 
-template <int NS, int CH, int NB>
+template <int NS, int NB>
 __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __restrict__ descs,
                                                          const TensorState* __restrict__ st, int nt,
                                                          u32 tiles, Workspace ws, int stream0,
                                                          unsigned char* blob, CallState* call) {
     constexpr int PER = 32 / NB;                   // codes per 32-bit word = survivors per row
     constexpr int KTHR = 1 << NB;
-    __shared__ __align__(128) PackSmem<NS, CH, NB> sm;
-    if (call->flags & FLAG_BLOB_FULL) return;
+    constexpr int U = NS == 1 ? 2 : 1;             // rows a lane has in flight per stream
+    __shared__ __align__(16) PackSmem<NS, NB> sm;
+    if (call->flags & (FLAG_BLOB_FULL | FLAG_TIMEOUT)) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const u32 gw = blockIdx.x * PWARPS + warp, nw = gridDim.x * PWARPS;
     const u32 wlo = (u32)(((u64)tiles * gw) / nw), whi = (u32)(((u64)tiles * (gw + 1)) / nw);
-    SegRing<NS, CH, PST> ring;
-    ring.init(&sm.buf[warp][0][0][0], sm.bar[warp], lane, wlo, whi);
     const u32* tile_cnt = stream0 == 0 ? ws.tile_cnt_w : ws.tile_cnt_o;
     const u32* tile_off = stream0 == 0 ? ws.tile_off_w : ws.tile_off_o;
-    const float* surv[NS];
-#pragma unroll
-    for (int k = 0; k < NS; ++k) surv[k] = ws.surv[stream0 + k];
 
     int cur = -1;
     u32 tb = 0, ntl = 0;
@@ -155,14 +158,16 @@ __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __res
     float t3[NS], t7[NS], t11[NS];
 #pragma unroll
     for (int k = 0; k < NS; ++k) { words[k] = nullptr; t3[k] = t7[k] = t11[k] = 0.f; }
-    u32 carry[NS];                       // last row of the previous chunk of the same tile
-#pragma unroll
-    for (int k = 0; k < NS; ++k) carry[k] = 0;
 
-    while (ring.next_window(tile_cnt, lane, whi)) {
-        while (ring.have()) {
-            ring.issue_ahead(lane, surv);
-            const u32 tile = ring.tile();
+    for (u32 w0 = wlo; w0 < whi; w0 += 32) {
+        const u32 nt32 = min(32u, whi - w0);
+        const u32 mycnt = (u32)lane < nt32 ? min(tile_cnt[w0 + lane], (u32)TILE) : 0u;   // a count never leads out of its segment
+        const u32 myoff = (u32)lane < nt32 ? tile_off[w0 + lane] : 0u;
+        for (u32 ti = 0; ti < nt32; ++ti) {
+            const u32 cnt = __shfl_sync(0xffffffffu, mycnt, ti);
+            const u32 t0 = __shfl_sync(0xffffffffu, myoff, ti);    // tensor-wide rank of the tile's first survivor
+            if (!cnt) continue;
+            const u32 tile = w0 + ti;
             if (cur < 0 || tile >= tb + ntl) {
                 cur = find_tensor(descs, nt, tile);
                 tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
@@ -180,55 +185,61 @@ __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __res
                     if (NB == 4) { t3[k] = sm.thr[warp][k][3]; t7[k] = sm.thr[warp][k][7]; t11[k] = sm.thr[warp][k][11]; }
                 }
             }
-            const u32 cnt = ring.tile_cnt_cur(), off = ring.off(), nel = ring.nel();
-            const u32 t0 = tile_off[tile];                 // tensor-wide rank of the tile's first survivor
-            if (!ring.wait()) {
-                if (lane == 0) atomicOr(&call->flags, FLAG_TIMEOUT);
-                return;
-            }
-            const u32 nrows = (nel + PER - 1) / PER;       // rows of this chunk
-            const u32 sh = (t0 % PER) * NB;                // a row's shift inside the tensor's words
-            const u32 wbase = t0 / PER + off / PER;        // output word of this chunk's first row
-            const bool last_chunk = off + nel == cnt;
+            const u32 nrows = (cnt + PER - 1) / PER;
+            const u32 sh = (t0 % PER) * NB;                 // a row's shift inside the tensor's words
+            const u32 wbase = t0 / PER;                     // output word of the tile's first row
+            const u32 nout = nrows + (sh ? 1u : 0u);        // the last row spills into one more word
+            u32 carry[NS];
 #pragma unroll
-            for (int k = 0; k < NS; ++k) {
-                if (off == 0) carry[k] = 0;
-                const float* data = ring.stage() + k * CH;
-                const char* thr_row = reinterpret_cast<const char*>(sm.thr[warp][k]);
-                u32* rows = sm.rows[warp][k];
-                if (lane == 0) rows[0] = carry[k];
-                for (u32 r = lane; r < nrows; r += 32) {   // PER codes -> one word in the tile's alignment
-                    float xs[PER];
+            for (int k = 0; k < NS; ++k) carry[k] = 0;
+            for (u32 r0 = 0; r0 < nout; r0 += 32 * U) {
+                float xs[U][NS][PER];
 #pragma unroll
-                    for (int q = 0; q < PER / 4; ++q) {
-                        const float4 u4 = *reinterpret_cast<const float4*>(data + PER * r + 4 * q);
-                        xs[4 * q] = u4.x; xs[4 * q + 1] = u4.y; xs[4 * q + 2] = u4.z; xs[4 * q + 3] = u4.w;
+                for (int u = 0; u < U; ++u) {
+                    const u32 r = r0 + 32 * u + lane;
+                    if (r < nrows) {
+#pragma unroll
+                        for (int k = 0; k < NS; ++k) {
+                            const float4* src = reinterpret_cast<const float4*>(ws.surv[stream0 + k] + (u64)tile * TILE + PER * r);
+#pragma unroll
+                            for (int q = 0; q < PER / 4; ++q) {
+                                const float4 v = __ldcs(src + q);
+                                xs[u][k][4 * q] = v.x; xs[u][k][4 * q + 1] = v.y; xs[u][k][4 * q + 2] = v.z; xs[u][k][4 * q + 3] = v.w;
+                            }
+                        }
                     }
-                    u32 w = 0;
+                }
 #pragma unroll
-                    for (int i = 0; i < PER; ++i) {
-                        const u32 code = NB == 4 ? find_cluster4(xs[i], t3[k], t7[k], t11[k], thr_row) / 4 + 1
-                                                 : find_cluster<NB>(xs[i], sm.thr[warp][k]) + 1;
-                        w |= code << (NB * i);
+                for (int u = 0; u < U; ++u) {
+                    const u32 m = r0 + 32 * u + lane;               // this lane's row = its output word within the tile
+                    if (r0 + 32 * u >= nout) break;                 // warp uniform
+#pragma unroll
+                    for (int k = 0; k < NS; ++k) {
+                        u32 w = 0;
+                        if (m < nrows) {
+                            const char* thr_row = reinterpret_cast<const char*>(sm.thr[warp][k]);
+#pragma unroll
+                            for (int i = 0; i < PER; ++i) {
+                                const u32 code = NB == 4 ? find_cluster4(xs[u][k][i], t3[k], t7[k], t11[k], thr_row) / 4 + 1
+                                                         : find_cluster<NB>(xs[u][k][i], sm.thr[warp][k]) + 1;
+                                w |= code << (NB * i);
+                            }
+                            const u32 have = cnt - PER * m;         // codes of this row that exist (the segment holds stale values after them)
+                            if (have < (u32)PER) w &= (1u << (NB * have)) - 1u;
+                        }
+                        u32 prev = __shfl_up_sync(0xffffffffu, w, 1);
+                        if (lane == 0) prev = carry[k];
+                        carry[k] = __shfl_sync(0xffffffffu, w, 31);
+                        // output word m of the tile = row m shifted up | row m-1 shifted down
+                        const u32 v = (w << sh) | (sh ? prev >> (32 - sh) : 0u);
+                        if (m < nout) {
+                            const u64 g0 = (u64)(wbase + m) * PER;  // ranks the word covers: [g0, g0 + PER)
+                            if (g0 >= t0 && g0 + PER <= (u64)t0 + cnt) words[k][wbase + m] = v;
+                            else if (v) atomicOr(&words[k][wbase + m], v);
+                        }
                     }
-                    const u32 have = nel - PER * r;            // codes of this row that exist (the stage holds stale values after them)
-                    if (have < (u32)PER) w &= (1u << (NB * have)) - 1u;
-                    rows[1 + r] = w;
                 }
-                if (lane == 0) rows[1 + nrows] = 0;
-                __syncwarp();
-                carry[k] = rows[nrows];                    // the chunk's last row (for the next chunk)
-                // output word m of the chunk = row m shifted up | row m-1 shifted down
-                const u32 nout = nrows + ((last_chunk && sh) ? 1u : 0u);
-                for (u32 m = lane; m < nout; m += 32) {
-                    const u32 v = (rows[1 + m] << sh) | (sh ? rows[m] >> (32 - sh) : 0u);
-                    const u64 g0 = (u64)(wbase + m) * PER; // ranks the word covers: [g0, g0 + PER)
-                    if (g0 >= t0 && g0 + PER <= (u64)t0 + cnt) words[k][wbase + m] = v;
-                    else if (v) atomicOr(&words[k][wbase + m], v);
-                }
-                __syncwarp();
             }
-            ring.advance();
         }
     }
 }
@@ -298,14 +309,14 @@ void launch_pack(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st,
     prof_mark(cfg, ST_HEADER_EDGES, 2);
     const u32 grid = min((tiles + PWARPS - 1) / PWARPS, (u32)cfg.sms * 6u);
     if (p.bits == 4) {
-        pack_codes_kernel<1, 512, 4><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 0, blob, call);
-        pack_codes_kernel<2, 256, 4><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 1, blob, call);
+        pack_codes_kernel<1, 4><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 0, blob, call);
+        pack_codes_kernel<2, 4><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 1, blob, call);
     } else if (p.bits == 2) {
-        pack_codes_kernel<1, 512, 2><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 0, blob, call);
-        pack_codes_kernel<2, 256, 2><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 1, blob, call);
+        pack_codes_kernel<1, 2><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 0, blob, call);
+        pack_codes_kernel<2, 2><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 1, blob, call);
     } else {
-        pack_codes_kernel<1, 256, 8><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 0, blob, call);
-        pack_codes_kernel<2, 128, 8><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 1, blob, call);
+        pack_codes_kernel<1, 8><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 0, blob, call);
+        pack_codes_kernel<2, 8><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 1, blob, call);
     }
     prof_mark(cfg, ST_PACK_CODES, 2);
     const u64 quads = (u64)tiles * (TILE_WORDS / 4);
