@@ -330,6 +330,19 @@ int excp_profile_stage_count(void);
 const char* excp_profile_stage_name(int stage);
 excp_status excp_profile_read(excp_handle h, double* stage_ms_out, unsigned long long* launches_out);
 
+/* The bounded waits (no counterpart in the paper).  The dense sweeps stage their inputs in shared memory with
+ * asynchronous bulk copies; a warp waits for a copy at most `nanoseconds` (default 2 s; a healthy copy lands
+ * within microseconds).  When a wait runs out the warp raises the call's time-out flag, lets its other
+ * copies land and leaves; every later kernel of the call then returns at once and the call returns
+ * EXCP_ERR_TIMEOUT with the output buffers unspecified.  The handle stays usable.
+ *   excp_set_wait_limit          sets the limit for the handle's later calls.
+ *   excp_selftest_wait_timeout   exercises the error path on its own: one warp waits `nanoseconds` (at most
+ *                                1e9) on a barrier that nothing will ever complete, so the wait always runs
+ *                                out and the call returns EXCP_ERR_TIMEOUT; no copy is in flight at any
+ *                                point.  Synchronises the stream. */
+excp_status excp_set_wait_limit(excp_handle h, unsigned long long nanoseconds);
+excp_status excp_selftest_wait_timeout(excp_handle h, unsigned long long nanoseconds, void* cuda_stream);
+
 /* Tuning knob of the K-means stage (Section 3.3 leaves the implementation of K-means open; the
  * centres do not depend on this value).  The iterations need, per threshold between two centres,
  * the values of one narrow value cell.  The cells that all T iterations will visit are predicted

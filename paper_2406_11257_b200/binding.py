@@ -24,7 +24,7 @@ EXPORTS = ["excp_create", "excp_destroy", "excp_record_bytes", "excp_compress_bo
            "excp_compress_checkpoint_host", "excp_decompress_tensor", "excp_decompress_checkpoint",
            "excp_decompress_tensor_noalloc", "excp_dense_bytes", "excp_record_to_dense", "excp_checkpoint_to_dense",
            "excp_decompress_dense_tensor", "excp_decompress_dense_checkpoint", "excp_profile_enable", "excp_profile_stage_count", "excp_profile_stage_name", "excp_profile_read",
-           "excp_set_kmeans_margin"]
+           "excp_set_kmeans_margin", "excp_set_wait_limit", "excp_selftest_wait_timeout"]
 
 
 class ExcpError(RuntimeError):
@@ -108,6 +108,8 @@ def load_library() -> C.CDLL:
     lib.excp_decompress_dense_checkpoint.argtypes = lib.excp_decompress_checkpoint.argtypes
     lib.excp_profile_enable.argtypes = [vp, C.c_int]
     lib.excp_set_kmeans_margin.argtypes = [vp, C.c_int]
+    lib.excp_set_wait_limit.argtypes = [vp, C.c_ulonglong]
+    lib.excp_selftest_wait_timeout.argtypes = [vp, C.c_ulonglong, vp]
     lib.excp_profile_stage_count.argtypes = []
     lib.excp_profile_stage_name.argtypes = [C.c_int]
     lib.excp_profile_stage_name.restype = C.c_char_p
@@ -203,6 +205,16 @@ class Handle:
         st = self.lib.excp_set_kmeans_margin(self._h, int(margin))
         if st != 0:
             raise ExcpError(st, "excp_set_kmeans_margin")
+
+    def set_wait_limit(self, nanoseconds: int) -> None:
+        """excp_set_wait_limit: how long a warp waits for an asynchronous copy before the call gives up."""
+        st = self.lib.excp_set_wait_limit(self._h, int(nanoseconds))
+        if st != 0:
+            raise ExcpError(st, "excp_set_wait_limit")
+
+    def selftest_wait_timeout(self, nanoseconds: int) -> int:
+        """excp_selftest_wait_timeout: returns the status (EXCP_ERR_TIMEOUT = -7 is the expected one)."""
+        return self.lib.excp_selftest_wait_timeout(self._h, int(nanoseconds), _stream())
 
     def profile_enable(self, on: bool = True) -> None:
         st = self.lib.excp_profile_enable(self._h, int(on))

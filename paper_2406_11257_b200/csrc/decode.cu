@@ -135,7 +135,9 @@ struct DecodeSmem {
 // Code windows: the NB-bit codes of `cnt` consecutive survivors starting at rank g of a section, as
 // NB 32-bit words with the first code at bit 0.  Only words that hold such codes are read.
 template <int NB>
-__device__ __forceinline__ void load_window(const u32* __restrict__ sec, u64 g, u32 cnt, u32 (&c)[NB]) {
+__device__ __forceinline__ void load_window(const u32* __restrict__ sec, u64 g, u32 cnt, u32 (&c)[NB],
+                                            const CallState* call, u64 nnz) {
+    if (!EXCP_IN_BOUNDS(call, g + cnt <= nnz)) cnt = 0;      // the codes asked for lie inside the section
     const u64 bit = g * NB;
     const u32 sh = (u32)bit & 31u;
     const u32* p = sec + (bit >> 5);
@@ -216,18 +218,18 @@ struct DecTile {                 // what the phases need to know about the tile 
 // bitmaps; gw, go: ranks of their first survivors.
 template <bool DENSE, int NB, typename WT>
 __device__ __forceinline__ u32 decode_block(const DecTile& t, const DecDesc& d, const DecState& s, DecodeSmem& sm, int warp,
-                                            int lane, u32 blk, u32 a, u32 b, u64 gw, u64 go) {
+                                            int lane, u32 blk, u32 a, u32 b, u64 gw, u64 go, const CallState* call) {
     u32 bad = 0;
     u32 ow8[8], oa8[8], os8[8];
     {
         u32 c[NB];
-        load_window<NB>(t.sec0, gw, (u32)__popc(a), c);
+        load_window<NB>(t.sec0, gw, (u32)__popc(a), c, call, s.nnz_w);
         bad |= expand_word<NB>(a, c, sm.sel, sm.spread, ow8);
     }
     {
         u32 c1[NB], c2[NB];
-        load_window<NB>(t.sec1, go, (u32)__popc(b), c1);
-        load_window<NB>(t.sec2, go, (u32)__popc(b), c2);
+        load_window<NB>(t.sec1, go, (u32)__popc(b), c1, call, s.nnz_o);
+        load_window<NB>(t.sec2, go, (u32)__popc(b), c2, call, s.nnz_o);
         bad |= expand_word<NB>(b, c1, sm.sel, sm.spread, oa8);
         bad |= expand_word<NB>(b, c2, sm.sel, sm.spread, os8);
     }
@@ -410,11 +412,11 @@ __global__ void __launch_bounds__(TPB, EXCP_DEC_MIN_BLOCKS) decode_kernel(const 
             if (raw) {
                 if (!DENSE) decode_block_raw<WT>(t, d, lane, blk, a, b, gwl, gol);
             } else if (DENSE || bits == 4) {
-                bad |= decode_block<DENSE, 4, WT>(t, d, s, sm, warp, lane, blk, a, b, gwl, gol);
+                bad |= decode_block<DENSE, 4, WT>(t, d, s, sm, warp, lane, blk, a, b, gwl, gol, call);
             } else if (bits == 2) {
-                bad |= decode_block<false, 2, WT>(t, d, s, sm, warp, lane, blk, a, b, gwl, gol);
+                bad |= decode_block<false, 2, WT>(t, d, s, sm, warp, lane, blk, a, b, gwl, gol, call);
             } else {
-                bad |= decode_block<false, 8, WT>(t, d, s, sm, warp, lane, blk, a, b, gwl, gol);
+                bad |= decode_block<false, 8, WT>(t, d, s, sm, warp, lane, blk, a, b, gwl, gol, call);
             }
         }
         if (__any_sync(0xffffffffu, bad)) break;

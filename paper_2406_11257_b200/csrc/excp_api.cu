@@ -64,6 +64,7 @@ struct excp_handle_s {
     size_t tensor_cap = 0;               // entries the per-call arrays hold
     int last_cuda_error = 0;
     int km_margin = 1;                   // see excp_set_kmeans_margin
+    unsigned long long wait_limit_ns = 2000000000ull;   // see excp_set_wait_limit
     Profiler prof;
     // host-buffer path: two staging slots (inputs + records), its own copy streams
     float* stage[2][4] = {};
@@ -155,6 +156,7 @@ excp_status validate_params(const excp_params* params) {
 Params to_params(excp_handle h, const excp_params* params) {
     Params p;
     p.km_margin = h->km_margin;
+    p.wait_ns = h->wait_limit_ns;
     p.alpha = params->alpha; p.beta = params->beta; p.bits = params->bits;
     p.kmeans_iters = params->kmeans_iters; p.seed = params->seed; p.median_source = params->median_source;
     p.flags = params->flags;
@@ -167,6 +169,10 @@ bool run_group(excp_handle h, const LaunchCfg& cfg, const TensorDesc* descs, int
                const Params& p, unsigned char* blob, u64 blob_capacity, TensorResult* results) {
     if (!check(h, cudaMemsetAsync(h->d_state, 0, nt * sizeof(TensorState), cfg.stream))) return false;
     if (!check(h, cudaMemsetAsync(h->ws.cst, 0, nt * sizeof(CellState), cfg.stream))) return false;
+    // the per-tile survivor counts start at zero, so that no kernel can meet a stale count where a sweep gave up
+    if (tiles && (!check(h, cudaMemsetAsync(h->ws.tile_cnt_w, 0, (size_t)tiles * sizeof(u32), cfg.stream)) ||
+                  !check(h, cudaMemsetAsync(h->ws.tile_cnt_o, 0, (size_t)tiles * sizeof(u32), cfg.stream))))
+        return false;
     launch_stats(cfg, descs, h->d_state, nt, tiles, h->ws, p, h->d_call);
     launch_mask_compact(cfg, descs, h->d_state, nt, tiles, h->ws, p, h->d_call, blob_capacity);
     if (!(p.flags & OPT_NO_QUANT)) launch_kmeans(cfg, descs, h->d_state, nt, tiles, h->ws, h->km, p, h->d_call);
@@ -629,6 +635,26 @@ excp_status excp_set_kmeans_margin(excp_handle h, int margin) {
     if (!h || margin < -1) return EXCP_ERR_INVALID_ARG;
     h->km_margin = margin;
     return EXCP_OK;
+}
+
+excp_status excp_set_wait_limit(excp_handle h, unsigned long long nanoseconds) {
+    if (!h) return EXCP_ERR_INVALID_ARG;
+    h->wait_limit_ns = nanoseconds;
+    return EXCP_OK;
+}
+
+excp_status excp_selftest_wait_timeout(excp_handle h, unsigned long long nanoseconds, void* cuda_stream) {
+    if (!h || nanoseconds > 1000000000ull) return EXCP_ERR_INVALID_ARG;      // at most a second: this wait always runs out
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return EXCP_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    LaunchCfg cfg{h->sms, stream, nullptr};
+    bool ok = check(h, cudaMemsetAsync(h->d_call, 0, sizeof(CallState), stream));
+    if (ok) launch_wait_selftest(cfg, h->d_call, nanoseconds);
+    ok = ok && check(h, cudaGetLastError());
+    ok = ok && check(h, cudaMemcpyAsync(h->h_call, h->d_call, sizeof(CallState), cudaMemcpyDeviceToHost, stream));
+    if (!check(h, cudaStreamSynchronize(stream)) || !ok) return EXCP_ERR_CUDA;
+    return status_from_flags(h->h_call->flags);
 }
 
 excp_status excp_profile_enable(excp_handle h, int enable) {

@@ -169,6 +169,7 @@ struct Params {
     u32 flags;                   // OPT_*
     int wfmt;                    // WeightFormat of w_t and w_prev
     int km_margin;               // cells gathered on either side of every predicted threshold (-1: none)
+    u64 wait_ns;                 // how long a warp waits for an asynchronous copy before it gives up
 };
 __host__ __device__ inline int stored_bits(const Params& p) { return (p.flags & OPT_NO_QUANT) ? 32 : p.bits; }
 __host__ __device__ inline u32 record_flags(const Params& p) {
@@ -227,6 +228,23 @@ __device__ __forceinline__ u32 cell_of(float x, const u32* __restrict__ tab) {
     const u32 neg = (u32)((int)bits >> 31);            // 0 or all ones
     return (ent >> 8) + ((sub ^ neg) - neg);           // anchor + sub, or anchor - sub
 }
+
+// A warp gave up waiting for a copy somewhere in this call: every later kernel returns at once, so
+// nothing is computed from arrays that were only partly written.
+__device__ __forceinline__ bool call_aborted(const CallState* call) { return (call->flags & FLAG_TIMEOUT) != 0u; }
+
+// The checked build (-DEXCP_DEBUG_BOUNDS): every index that depends on data is tested before it is
+// used; a violation raises FLAG_INTERNAL (the call returns EXCP_ERR_CUDA) and the access is skipped.
+// Nothing traps.  In the normal build the test is the constant `true`.
+#ifdef EXCP_DEBUG_BOUNDS
+__device__ __forceinline__ bool bounds_ok(const CallState* call, bool in_bounds) {
+    if (!in_bounds) atomicOr(const_cast<u32*>(&call->flags), FLAG_INTERNAL);
+    return in_bounds;
+}
+#define EXCP_IN_BOUNDS(call, cond) bounds_ok((call), (cond))
+#else
+#define EXCP_IN_BOUNDS(call, cond) (true)
+#endif
 
 // Tensor that owns group tile `tile` (descs are in tile order).
 __device__ inline int find_tensor(const TensorDesc* __restrict__ descs, int n, u32 tile) {
@@ -387,5 +405,6 @@ void launch_record_to_dense(const LaunchCfg&, const DecDesc* descs, DecState* st
                             const Workspace& ws, CallState* call);
 void launch_dense_decode(const LaunchCfg&, const DecDesc* descs, DecState* st, int nt, u32 tiles,
                          CallState* call);
+void launch_wait_selftest(const LaunchCfg&, CallState* call, u64 limit_ns);
 
 }  // namespace excp

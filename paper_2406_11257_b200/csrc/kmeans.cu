@@ -56,11 +56,13 @@ constexpr u32 SMALL_STREAM = 16384;  // at most this many survivors: every cell 
 // One block per (tensor, stream).
 __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDesc* __restrict__ descs,
                                                                   TensorState* __restrict__ st,
-                                                                  Workspace ws, KmArrays km, u64 seed, int K, int iters) {
+                                                                  Workspace ws, KmArrays km, u64 seed, int K, int iters,
+                                                                  const CallState* call) {
     __shared__ float smp[SAMPLE_MAX];
     __shared__ u32 chist[NCLASS];                     // sampled survivors per (sign, exponent) class
     __shared__ u32 wtot[NCLASS / 32];
     __shared__ u32 cvalid;
+    if (call_aborted(call)) return;
     const int t = blockIdx.x, stream = blockIdx.y, tid = threadIdx.x;
     StreamState& s = st[t].s[stream];
     CellStream& cs = ws.cst[t].s[stream];
@@ -88,7 +90,7 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
             const u32 mid = (a + b + 1) >> 1;
             if (toff[mid] <= r) a = mid; else b = mid - 1;
         }
-        v = data[(u64)a * TILE + (r - toff[a])];
+        if (EXCP_IN_BOUNDS(call, r - toff[a] < (u32)TILE)) v = data[(u64)a * TILE + (r - toff[a])];
     }
     smp[tid] = v;
     if (tid < NCLASS) chist[tid] = 0;
@@ -201,7 +203,7 @@ __global__ void __launch_bounds__(CWARPS * 32, 2) cell_count_kernel(const Tensor
                                                                     Workspace ws, KmArrays km, int stream0, CallState* call) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     CellCountSmem<NS>& sm = *reinterpret_cast<CellCountSmem<NS>*>(smem_raw);
-    if (call->flags & FLAG_TIMEOUT) return;
+    if (call_aborted(call)) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     u32 lo, hi;
     block_range(tiles, lo, hi);
@@ -228,6 +230,7 @@ __global__ void __launch_bounds__(CWARPS * 32, 2) cell_count_kernel(const Tensor
             const float a1 = st[cur].s[stream0 + k].scale1, a2 = st[cur].s[stream0 + k].scale2;
             auto tally = [&](float x) {
                 const u32 c = cell_of(x, tab);
+                if (!EXCP_IN_BOUNDS(call, c < (u32)NCELL)) return;
                 const u32 q = (u32)abs(__float2int_rn(__fmul_rn(__fmul_rn(x, a1), a2)));   // |Q(x)| < 2^31
                 atomicAdd(&cnt[c], 1u);
                 const u32 old = atomicAdd(&slo[c], q);
@@ -239,6 +242,7 @@ __global__ void __launch_bounds__(CWARPS * 32, 2) cell_count_kernel(const Tensor
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     c[i] = cell_of(xs[i], tab);
+                    if (!EXCP_IN_BOUNDS(call, c[i] < (u32)NCELL)) c[i] = 0;
                     q[i] = (u32)abs(__float2int_rn(__fmul_rn(__fmul_rn(xs[i], a1), a2)));
                 }
 #pragma unroll
@@ -316,13 +320,14 @@ __device__ inline u32 block_of_tile(u32 x, u32 tiles, u32 g) {
 __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDesc* __restrict__ descs,
                                                                  TensorState* __restrict__ st, Workspace ws, KmArrays km, int K,
                                                                  int iters, int margin, int round, u32 tiles,
-                                                                 u32 grid) {
+                                                                 u32 grid, const CallState* call) {
     __shared__ u32 tab[NCLASS];
     __shared__ u32 selw[NCELL / 32];
     __shared__ float cent[KCAP], thr[KCAP], cnew[KCAP];
     __shared__ double Lp[KCAP], Sp[KCAP];
     __shared__ s64 wt64[32];
     __shared__ u32 wt32[32];
+    if (call_aborted(call)) return;
     const int t = blockIdx.x, stream = blockIdx.y, tid = threadIdx.x;
     CellStream& cs = ws.cst[t].s[stream];
     if (!cs.active) return;
@@ -348,7 +353,9 @@ __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDes
 #pragma unroll
         for (int k = 0; k < 4; ++k) { cs.cntpre[c0 + k] = pc[k]; cs.sumpre[c0 + k] = ps[k]; }
         if (tid == 0) { cs.cntpre[NCELL] = tc; cs.sumpre[NCELL] = ts; }
-        const bool predict = nnz > SMALL_STREAM && margin < NCELL;
+        // With 255 centres nearly every cell holds or neighbours a threshold at some iteration, and ten iterations
+        // on the cell table alone drift further than a cell: every cell is taken, so that no second round is needed.
+        const bool predict = nnz > SMALL_STREAM && margin < NCELL && K <= KMAX;
         if (predict) {
             if (tid < NCELL / 32) selw[tid] = 0;
             if (tid < NCLASS) tab[tid] = cs.tab[tid];
@@ -443,7 +450,7 @@ __global__ void __launch_bounds__(CWARPS * 32, 2) cell_gather_kernel(const Tenso
                                                                      int round) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     CellGatherSmem<NS>& sm = *reinterpret_cast<CellGatherSmem<NS>*>(smem_raw);
-    if (call->flags & FLAG_TIMEOUT) return;
+    if (call_aborted(call)) return;
     if (round > 0 && *km.pending == 0) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     u32 lo, hi;
@@ -477,23 +484,32 @@ __global__ void __launch_bounds__(CWARPS * 32, 2) cell_gather_kernel(const Tenso
             const u32* sel = sm.sel[k];
             u32* cursor = sm.cur[k];
             float* out = ws.bkt[stream0 + k] + (u64)tb * TILE;
+            const u64 room = (u64)descs[cur].num_tiles * TILE;               // the tensor's share of the gathered copy
+            auto put = [&](u32 c, float x) {
+                const u32 at = atomicAdd(&cursor[c], 1u);
+                if (EXCP_IN_BOUNDS(call, at < room)) out[at] = x;
+            };
             auto file = [&](float x) {
                 const u32 c = cell_of(x, tab);
-                if ((sel[c >> 5] >> (c & 31)) & 1u) out[atomicAdd(&cursor[c], 1u)] = x;
+                if (!EXCP_IN_BOUNDS(call, c < (u32)NCELL)) return;
+                if ((sel[c >> 5] >> (c & 31)) & 1u) put(c, x);
             };
             auto file8 = [&](const float4& va, const float4& vb, bool two) {       // all look-ups first
                 const float xs[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
                 u32 c[8];
                 u32 hit = 0;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) c[i] = cell_of(xs[i], tab);
+                for (int i = 0; i < 8; ++i) {
+                    c[i] = cell_of(xs[i], tab);
+                    if (!EXCP_IN_BOUNDS(call, c[i] < (u32)NCELL)) c[i] = 0;
+                }
 #pragma unroll
                 for (int i = 0; i < 8; ++i) hit |= ((sel[c[i] >> 5] >> (c[i] & 31)) & 1u) << i;
                 if (!two) hit &= 15u;
                 if (hit) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
-                        if ((hit >> i) & 1u) out[atomicAdd(&cursor[c[i]], 1u)] = xs[i];
+                        if ((hit >> i) & 1u) put(c[i], xs[i]);
                 }
             };
             sweep_segments(ws.surv[stream0 + k], tile_cnt, wlo, whi, lane, file8, file);
@@ -548,7 +564,7 @@ __global__ void __launch_bounds__(IT_THREADS) kmeans_iterate_kernel(const Tensor
     __shared__ s64 psum[KCAP][IT_PARTS];
     __shared__ u64 Ls[KCAP];
     __shared__ s64 Ss[KCAP];
-    if (call->flags & FLAG_TIMEOUT) return;
+    if (call_aborted(call)) return;
     const int t = blockIdx.x, stream = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     CellStream& cs = ws.cst[t].s[stream];
     if (!cs.active) return;
@@ -577,6 +593,7 @@ __global__ void __launch_bounds__(IT_THREADS) kmeans_iterate_kernel(const Tensor
             s64 sum = 0;
             if ((selw[c >> 5] >> (c & 31)) & 1u) {
                 const u32 b = (u32)cs.mag[c], n = cs.cntpre[c + 1] - cs.cntpre[c];
+                if (EXCP_IN_BOUNDS(call, (u64)b + n <= (u64)descs[t].num_tiles * TILE))
                 scan_range(data, b + (u32)(((u64)n * p) / parts), b + (u32)(((u64)n * (p + 1)) / parts), thr[j], s1, s2,
                            lane, cnt, sum);
             }
@@ -631,7 +648,7 @@ __global__ void __launch_bounds__(IT_THREADS) kmeans_iterate_kernel(const Tensor
 void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                    const Workspace& ws, const KmArrays& km, const Params& p, CallState* call) {
     const int K = centres_of(p.bits);
-    kmeans_start_kernel<<<dim3(nt, 3), SAMPLE_MAX, 0, cfg.stream>>>(descs, st, ws, km, p.seed, K, p.kmeans_iters);
+    kmeans_start_kernel<<<dim3(nt, 3), SAMPLE_MAX, 0, cfg.stream>>>(descs, st, ws, km, p.seed, K, p.kmeans_iters, call);
     prof_mark(cfg, ST_KMEANS_START, 1);
     if (!tiles || p.kmeans_iters == 0) return;
     // the two sweeps use one grid: a block's share of the tiles is its share of every cell
@@ -649,7 +666,7 @@ void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* s
     cudaFuncSetAttribute(cell_gather_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g2);
     for (int round = 0; round < 2; ++round) {
         cell_plan_kernel<<<dim3(nt, 3), PLAN_THREADS, 0, cfg.stream>>>(descs, st, ws, km, K, p.kmeans_iters, p.km_margin, round,
-                                                                     tiles, grid);
+                                                                     tiles, grid, call);
         if (round == 0) prof_mark(cfg, ST_CELL_PLAN, 1);
         cell_gather_kernel<1><<<grid, CWARPS * 32, g1, cfg.stream>>>(descs, nt, tiles, ws, km, 0, call, round);
         cell_gather_kernel<2><<<grid, CWARPS * 32, g2, cfg.stream>>>(descs, nt, tiles, ws, km, 1, call, round);

@@ -59,13 +59,14 @@ struct MaskSmem {
 template <bool VARIANT, typename WT>
 __global__ void __launch_bounds__(MTPB, MBLOCKS) mask_compact_kernel(const TensorDesc* __restrict__ descs,
                                                               TensorState* __restrict__ st, int nt,
-                                                              u32 tiles, Workspace ws, CallState* call, u32 opt) {
+                                                              u32 tiles, Workspace ws, CallState* call, u32 opt, u64 wait_ns) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     MaskSmem& sm = *reinterpret_cast<MaskSmem*>(smem_raw);
+    if (call_aborted(call)) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const u32 lt = (1u << lane) - 1u;
     WarpRing<4, MCH, MST> ring;
-    ring.init(&sm.buf[warp][0][0][0], sm.bar[warp], lane);
+    ring.init(&sm.buf[warp][0][0][0], sm.bar[warp], lane, wait_ns);
 
     const u32 gw = blockIdx.x * MWARPS + warp, nw = gridDim.x * MWARPS;
     const u32 wlo = (u32)(((u64)tiles * gw) / nw), whi = (u32)(((u64)tiles * (gw + 1)) / nw);
@@ -123,6 +124,7 @@ __global__ void __launch_bounds__(MTPB, MBLOCKS) mask_compact_kernel(const Tenso
         const u64 e0 = cc.elem0();
         if (!ring.wait()) {
             if (lane == 0) atomicOr(&call->flags, FLAG_TIMEOUT);
+            ring.drain();
             return;
         }
         if (cc.chunk == 0) { rw = 0; ro = 0; }
@@ -196,16 +198,18 @@ __global__ void __launch_bounds__(MTPB, MBLOCKS) mask_compact_kernel(const Tenso
                 }
                 if (lane < 4) {
                     const u64 wi = (u64)cc.tile * TILE_WORDS + cc.chunk * (MCH / 32) + step * 4 + lane;
-                    ws.bm_w[wi] = lane == 0 ? bw[0] : lane == 1 ? bw[1] : lane == 2 ? bw[2] : bw[3];
-                    ws.bm_o[wi] = lane == 0 ? bo[0] : lane == 1 ? bo[1] : lane == 2 ? bo[2] : bo[3];
+                    if (EXCP_IN_BOUNDS(call, wi < (u64)tiles * TILE_WORDS)) {
+                        ws.bm_w[wi] = lane == 0 ? bw[0] : lane == 1 ? bw[1] : lane == 2 ? bw[2] : bw[3];
+                        ws.bm_o[wi] = lane == 0 ? bo[0] : lane == 1 ? bo[1] : lane == 2 ? bo[2] : bo[3];
+                    }
                 }
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    if ((bw[k] >> lane) & 1u) {
+                    if (((bw[k] >> lane) & 1u) && EXCP_IN_BOUNDS(call, rw + __popc(bw[k] & lt) < (u32)TILE)) {
                         sw[rw + __popc(bw[k] & lt)] = dwv[k];
                         mk0 = fmaxf(mk0, fabsf(dwv[k]));
                     }
-                    if ((bo[k] >> lane) & 1u) {
+                    if (((bo[k] >> lane) & 1u) && EXCP_IN_BOUNDS(call, ro + __popc(bo[k] & lt) < (u32)TILE)) {
                         const u32 po = ro + __popc(bo[k] & lt);
                         sea[po] = eav[k];
                         seas[po] = easv[k];
@@ -255,7 +259,9 @@ __global__ void __launch_bounds__(MTPB, MBLOCKS) mask_compact_kernel(const Tenso
 // Exclusive prefix of the tile counts inside each tensor; totals; the
 // fixed-point scale of each stream's sums.
 __global__ void __launch_bounds__(TPB) tile_scan_kernel(const TensorDesc* __restrict__ descs,
-                                                        TensorState* __restrict__ st, Workspace ws) {
+                                                        TensorState* __restrict__ st, Workspace ws,
+                                                        const CallState* call) {
+    if (call_aborted(call)) return;
     const int t = blockIdx.x, tid = threadIdx.x;
     u32 carry_w, carry_o;
     scan_tile_counts(descs[t].tile_begin, descs[t].num_tiles, ws, carry_w, carry_o);
@@ -279,6 +285,7 @@ __global__ void __launch_bounds__(MAX_GROUP_TENSORS) layout_kernel(const TensorD
                                                                    int bits, CallState* call,
                                                                    u64 blob_capacity) {
     __shared__ u64 wtot[32];
+    if (call_aborted(call)) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     u64 bytes = 0;
     if (tid < nt) bytes = record_bytes(descs[tid].numel, st[tid].nnz_w, st[tid].nnz_o, bits);   // bits = 32: raw survivors
@@ -316,15 +323,15 @@ void launch_mask_compact(const LaunchCfg& cfg, const TensorDesc* descs, TensorSt
             using WT = decltype(tag);
             cudaFuncSetAttribute(mask_compact_kernel<false, WT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(MaskSmem));
             cudaFuncSetAttribute(mask_compact_kernel<true, WT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(MaskSmem));
-            if (opt) mask_compact_kernel<true, WT><<<grid, MTPB, sizeof(MaskSmem), cfg.stream>>>(descs, st, nt, tiles, ws, call, opt);
-            else mask_compact_kernel<false, WT><<<grid, MTPB, sizeof(MaskSmem), cfg.stream>>>(descs, st, nt, tiles, ws, call, 0u);
+            if (opt) mask_compact_kernel<true, WT><<<grid, MTPB, sizeof(MaskSmem), cfg.stream>>>(descs, st, nt, tiles, ws, call, opt, p.wait_ns);
+            else mask_compact_kernel<false, WT><<<grid, MTPB, sizeof(MaskSmem), cfg.stream>>>(descs, st, nt, tiles, ws, call, 0u, p.wait_ns);
         };
         if (p.wfmt == WF_F16) run(__half{});
         else if (p.wfmt == WF_BF16) run(__nv_bfloat16{});
         else run(float{});
         prof_mark(cfg, ST_MASK_COMPACT, 1);
     }
-    tile_scan_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, ws);
+    tile_scan_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, ws, call);
     layout_kernel<<<1, MAX_GROUP_TENSORS, 0, cfg.stream>>>(descs, st, nt, stored_bits(p), call, blob_capacity);
     prof_mark(cfg, ST_SCAN_LAYOUT, 2);
 }

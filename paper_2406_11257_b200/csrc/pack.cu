@@ -38,7 +38,7 @@ __global__ void __launch_bounds__(64) header_kernel(const TensorDesc* __restrict
         results[t] = r;
         if (s.flags) atomicOr(&call->flags, s.flags);
     }
-    if (call->flags & FLAG_BLOB_FULL) return;
+    if (call->flags & (FLAG_BLOB_FULL | FLAG_TIMEOUT)) return;
     unsigned char* rec = blob + s.blob_off;
     const u64 numel = descs[t].numel, nnz_w = s.nnz_w, nnz_o = s.nnz_o;
     const int kc = centres_of(bits);                  // 15, or 0 when the survivors are stored raw
@@ -83,7 +83,7 @@ __global__ void __launch_bounds__(TPB) clear_edges_kernel(const TensorDesc* __re
                                                           const TensorState* __restrict__ st, int nt,
                                                           u32 tiles, Workspace ws, unsigned char* blob,
                                                           const CallState* call, int bits) {
-    if (call->flags & FLAG_BLOB_FULL) return;
+    if (call->flags & (FLAG_BLOB_FULL | FLAG_TIMEOUT)) return;
     const u32 tile = blockIdx.x * TPB + threadIdx.x;
     if (tile >= tiles) return;
     const u32 PER_WORD = 32u / (u32)bits;
@@ -234,8 +234,11 @@ __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __res
                         const u32 v = (w << sh) | (sh ? prev >> (32 - sh) : 0u);
                         if (m < nout) {
                             const u64 g0 = (u64)(wbase + m) * PER;  // ranks the word covers: [g0, g0 + PER)
-                            if (g0 >= t0 && g0 + PER <= (u64)t0 + cnt) words[k][wbase + m] = v;
-                            else if (v) atomicOr(&words[k][wbase + m], v);
+                            const bool whole = g0 >= t0 && g0 + PER <= (u64)t0 + cnt;
+                            if ((whole || v) && EXCP_IN_BOUNDS(call, (u64)(wbase + m) * 4 < code_bytes(stream0 + k == 0 ? st[cur].nnz_w : st[cur].nnz_o, NB))) {
+                                if (whole) words[k][wbase + m] = v;
+                                else atomicOr(&words[k][wbase + m], v);
+                            }
                         }
                     }
                 }
@@ -249,7 +252,7 @@ __global__ void __launch_bounds__(TPB) copy_bitmaps_kernel(const TensorDesc* __r
                                                            const TensorState* __restrict__ st, int nt,
                                                            u32 tiles, Workspace ws, unsigned char* blob,
                                                            const CallState* call, u32 hb) {
-    if (call->flags & FLAG_BLOB_FULL) return;
+    if (call->flags & (FLAG_BLOB_FULL | FLAG_TIMEOUT)) return;
     const u64 g = (u64)blockIdx.x * TPB + threadIdx.x;       // uint4 index over all tiles
     const u32 tile = (u32)(g / (TILE_WORDS / 4));
     if (tile >= tiles) return;
@@ -272,7 +275,7 @@ __global__ void __launch_bounds__(TPB) copy_bitmaps_kernel(const TensorDesc* __r
 __global__ void __launch_bounds__(TPB) pack_raw_kernel(const TensorDesc* __restrict__ descs,
                                                        const TensorState* __restrict__ st, int nt, u32 tiles,
                                                        Workspace ws, unsigned char* blob, const CallState* call) {
-    if (call->flags & FLAG_BLOB_FULL) return;
+    if (call->flags & (FLAG_BLOB_FULL | FLAG_TIMEOUT)) return;
     const int lane = threadIdx.x & 31;
     const u32 tile = blockIdx.x * (TPB / 32) + (threadIdx.x >> 5);
     if (tile >= tiles) return;

@@ -401,12 +401,12 @@ struct SweepSmem {
 template <typename WT>
 __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* __restrict__ descs,
                                                              TensorState* __restrict__ st, int nt, u32 tiles,
-                                                             Workspace ws, int residual_median, CallState* call) {
+                                                             Workspace ws, int residual_median, CallState* call, u64 wait_ns) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     SweepSmem& sm = *reinterpret_cast<SweepSmem*>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     WarpRing<3, SCH, SST> ring;
-    ring.init(&sm.buf[warp][0][0][0], sm.bar[warp], lane);
+    ring.init(&sm.buf[warp][0][0][0], sm.bar[warp], lane, wait_ns);
     const u32 gw = blockIdx.x * SWARPS + warp, nw = gridDim.x * SWARPS;
     const u32 wlo = (u32)(((u64)tiles * gw) / nw), whi = (u32)(((u64)tiles * (gw + 1)) / nw);
     TileWalk<SCH> ic, cc;
@@ -452,7 +452,8 @@ __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* _
         u32 base = 0;
         if (lane == 31 && incl) base = atomicAdd(&st[t].cand_count, incl);
         base = __shfl_sync(0xffffffffu, base, 31) + incl - nq;
-        for (u32 j = 0; j < nq; ++j) cand[base + j] = q[32 * j];
+        for (u32 j = 0; j < nq; ++j)
+            if (EXCP_IN_BOUNDS(call, (u64)base + j < (u64)descs[t].num_tiles * TILE)) cand[base + j] = q[32 * j];
         nq = 0;
     };
 
@@ -486,6 +487,7 @@ __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* _
         const u64 e0 = cc.elem0();
         if (!ring.wait()) {
             if (lane == 0) atomicOr(&call->flags, FLAG_TIMEOUT);
+            ring.drain();
             return;
         }
         const float* stg = ring.stage();
@@ -585,8 +587,10 @@ __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* _
 // histogram path (the bracket missed the median) or the start of the select among the
 // bracket's keys.  One block per tensor.
 __global__ void __launch_bounds__(TPB) stats_finish_kernel(const TensorDesc* __restrict__ descs,
-                                                           TensorState* __restrict__ st, float alpha, float beta) {
+                                                           TensorState* __restrict__ st, float alpha, float beta,
+                                                           const CallState* call) {
     __shared__ u64 tab[3][256];
+    if (call_aborted(call)) return;
     const int t = blockIdx.x, tid = threadIdx.x;
     TensorState& s = st[t];
     const u64 n = descs[t].numel;
@@ -624,9 +628,10 @@ constexpr int SEL_SLICES = 64;
 
 __global__ void __launch_bounds__(TPB) median_digit_kernel(TensorState* __restrict__ st,
                                                            const TensorDesc* __restrict__ descs, Workspace ws,
-                                                           int pass, float alpha) {
+                                                           int pass, float alpha, const CallState* call) {
     __shared__ u32 hist[256];
     __shared__ u32 is_last;
+    if (call_aborted(call)) return;
     const int t = blockIdx.y, tid = threadIdx.x;
     TensorState& s = st[t];
     if (s.med_done | s.need_hist) return;
@@ -687,12 +692,12 @@ void launch_stats(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st
         if (tiles) {
             const u32 grid = min((tiles + SWARPS - 1) / SWARPS, (u32)cfg.sms * 2u);
             cudaFuncSetAttribute(stats_sweep_kernel<WT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SweepSmem));
-            stats_sweep_kernel<WT><<<grid, TPB, sizeof(SweepSmem), cfg.stream>>>(descs, st, nt, tiles, ws, resid, call);
+            stats_sweep_kernel<WT><<<grid, TPB, sizeof(SweepSmem), cfg.stream>>>(descs, st, nt, tiles, ws, resid, call, p.wait_ns);
         }
-        stats_finish_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, alpha, p.beta);
+        stats_finish_kernel<<<nt, TPB, 0, cfg.stream>>>(descs, st, alpha, p.beta, call);
         if (tiles)
             for (int pass = 0; pass < 4; ++pass)
-                median_digit_kernel<<<dim3(SEL_SLICES, nt), TPB, 0, cfg.stream>>>(st, descs, ws, pass, alpha);
+                median_digit_kernel<<<dim3(SEL_SLICES, nt), TPB, 0, cfg.stream>>>(st, descs, ws, pass, alpha, call);
         prof_mark(cfg, ST_STATS1, tiles ? 7 : 2);
         if (tiles) {          // the histogram path: returns at once unless a bracket missed
             hist1_kernel<WT><<<min(tiles, (u32)cfg.sms * 4u), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, resid);

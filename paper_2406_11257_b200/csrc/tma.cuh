@@ -3,7 +3,7 @@
 // copy lands in the issuing CTA's own shared memory.
 //
 // Rules the callers keep: source and destination 16-byte aligned, size a
-// multiple of 16 bytes; a waiting warp polls with a bound and gives up as a whole
+// multiple of 16 bytes; a waiting warp polls until a deadline and gives up as a whole
 // (so that no thread is left behind at a later barrier), reporting through a flag.
 #pragma once
 #include <cuda_runtime.h>
@@ -49,15 +49,26 @@ __device__ __forceinline__ uint32_t mbar_try_wait(unsigned long long* bar, uint3
     return ok;
 }
 
-// Whole-warp wait for phase `parity`; false if the bound ran out (the caller
-// sets an error flag and leaves as a warp).  A healthy copy completes within
-// microseconds; the bound is far above a second.
-__device__ __forceinline__ bool mbar_wait_warp(unsigned long long* bar, uint32_t parity) {
-    for (uint32_t i = 0; i < (1u << 22); ++i) {
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Whole-warp wait for phase `parity`; false once `limit_ns` nanoseconds have passed without it
+// (the caller sets an error flag, lets its other copies land and leaves as a warp).  A healthy
+// copy completes within microseconds.
+__device__ __forceinline__ bool mbar_wait_warp(unsigned long long* bar, uint32_t parity, unsigned long long limit_ns) {
+    if (limit_ns == 0) return false;                             // no time at all: every wait fails (exercises the error path)
+    for (uint32_t i = 0; i < 16; ++i)
         if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
-        if (i > 16) __nanosleep(200);
+    const unsigned long long t0 = global_ns();
+    for (;;) {
+        if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+        const bool late = global_ns() - t0 > limit_ns;
+        if (__any_sync(0xffffffffu, late)) return false;         // one clock reading decides for the warp
+        __nanosleep(200);
     }
-    return false;
 }
 
 }  // namespace excp

@@ -21,9 +21,10 @@ struct WarpRing {
     float* buf;                    // ST stages of NS streams of CH values
     unsigned long long* bar;       // one barrier per stage
     u32 i_stage, c_stage, c_phase, inflight;
+    u64 limit_ns;                  // how long a wait may last
 
-    __device__ void init(float* b, unsigned long long* r, int lane) {
-        buf = b; bar = r; i_stage = 0; c_stage = 0; c_phase = 0; inflight = 0;
+    __device__ void init(float* b, unsigned long long* r, int lane, u64 wait_limit_ns) {
+        buf = b; bar = r; i_stage = 0; c_stage = 0; c_phase = 0; inflight = 0; limit_ns = wait_limit_ns;
         if (lane == 0) {
             for (int s = 0; s < ST; ++s) mbar_init(&bar[s], 1);
             mbar_fence_init();
@@ -63,7 +64,17 @@ struct WarpRing {
         issue_bytes(lane, vs, bytes);
     }
     // Blocks (bounded) until the oldest chunk in flight has landed.
-    __device__ bool wait() { return mbar_wait_warp(&bar[c_stage], c_phase); }
+    __device__ bool wait() { return mbar_wait_warp(&bar[c_stage], c_phase, limit_ns); }
+    // After a wait that ran out: lets every copy still in flight land (each wait bounded by DRAIN_NS,
+    // far above what a copy needs), so that the warp leaves with nothing writing into its stages.
+    static constexpr u64 DRAIN_NS = 2000000000ull;
+    __device__ void drain() {
+        while (inflight) {
+            mbar_wait_warp(&bar[c_stage], c_phase, DRAIN_NS);
+            if (++c_stage == (u32)ST) { c_stage = 0; c_phase ^= 1u; }
+            --inflight;
+        }
+    }
     __device__ const float* stage() const { return buf + c_stage * STAGE_FLOATS; }
     // Every lane is done reading the stage: it may be refilled.
     __device__ void release() {

@@ -441,6 +441,30 @@ def test_a_share_of_a_checkpoint_gives_the_whole_lists_records(handle):
     assert ranks.assemble_blob(table, blobs) == whole
 
 
+def test_a_wait_that_runs_out_comes_back_as_status_minus_7(handle):
+    """The bounded waits: a barrier that nothing completes makes the wait run out after the given time (no copy is
+    in flight, nothing faults); a whole compress call whose waits are given no time at all returns -7 after every
+    warp has let its own copies land, the later kernels of the call do nothing, and the handle works afterwards."""
+    import time
+    t0 = time.time()
+    assert handle.selftest_wait_timeout(5_000_000) == -7          # 5 ms
+    assert time.time() - t0 < 10
+    assert handle.selftest_wait_timeout(0) == -7
+    q = rand_quad_np(300_000, 1400)
+    dq = to_dev([q])
+    p = binding.Params(median_source=binding.MEDIAN_ABS_RESIDUAL, seed=2)
+    blob = torch.empty(binding.compress_bound(300_000), dtype=torch.uint8, device=DEV)
+    handle.set_wait_limit(0)
+    try:
+        with pytest.raises(binding.ExcpError) as e:
+            handle.compress_tensor(p, *dq[0], blob)
+        assert e.value.status == -7
+    finally:
+        handle.set_wait_limit(2_000_000_000)
+    blob2, offs, stats = gpu_compress(handle, p, dq)
+    check_against_oracle(p, [q], blob2, offs, stats)
+
+
 def test_profile_counts_launches_and_times_stages(handle):
     dq = [synth.make_quad(200_000, 3, 0, device=DEV)]
     blob = torch.empty(binding.compress_bound(200_000), dtype=torch.uint8, device=DEV)
