@@ -115,6 +115,14 @@ typedef struct {
     float mean_abs_ea;              /* the mean entering Eq. (ro) */
     float thr_w;                    /* alpha * median */
     float thr_o;                    /* beta * mean */
+    /* The K-means objective (Section 3.3) after the final assignment, per stream: the sum over the
+     * survivors of (value - its centre)^2.  A diagnostic: squares and sums of up to 16 of them in fp32, those
+     * added in fp64 in no fixed order, so it agrees with the plain fp64 sum to about 1e-6 relative and its
+     * last bits can differ from run to run.  0 where the sections hold raw fp32 survivors, and 0 unless
+     * excp_set_report_sse has switched it on (it costs the packing sweep about a quarter more time). */
+    double sse_w;
+    double sse_ea;
+    double sse_eas;
 } excp_tensor_stats;
 
 /* Creates a handle on CUDA device `device` with a scratch workspace for `workspace_numel`
@@ -329,6 +337,10 @@ excp_status excp_profile_enable(excp_handle h, int enable);
 int excp_profile_stage_count(void);
 const char* excp_profile_stage_name(int stage);
 excp_status excp_profile_read(excp_handle h, double* stage_ms_out, unsigned long long* launches_out);
+
+/* Switches the K-means objective in excp_tensor_stats (sse_w, sse_ea, sse_eas) on (non-zero) or off (the
+ * default) for the handle's later compress calls. */
+excp_status excp_set_report_sse(excp_handle h, int enable);
 
 /* The bounded waits (no counterpart in the paper).  The dense sweeps stage their inputs in shared memory with
  * asynchronous bulk copies; a warp waits for a copy at most `nanoseconds` (default 2 s; a healthy copy lands

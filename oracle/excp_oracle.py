@@ -341,6 +341,15 @@ def lloyd(s: np.ndarray, c0: np.ndarray, iters: int) -> tuple[np.ndarray, np.nda
     return c, assign(s, c)
 
 
+def quantisation_sse(s: np.ndarray, c: np.ndarray, idx: np.ndarray) -> float:
+    """Sum of squared distances of the values to their assigned centres (the K-means objective of
+    Section 3.3), in fp64.  A diagnostic: nothing in the record depends on it."""
+    if s.size == 0:
+        return 0.0
+    d = s.astype(np.float64) - c.astype(np.float64)[idx]
+    return float(np.sum(d * d))
+
+
 # --------------------------------------------------------------------------
 # Byte layout (reading R6)
 # --------------------------------------------------------------------------
@@ -534,11 +543,12 @@ def compress_tensor(w_t, w_prev, ea, eas, p: Params, tensor_index: int = 0, weig
 
     rec_flags = ((REC_MOMENTS_FREE if fl & FLAG_NO_W2M else 0) | (REC_ABSOLUTE if fl & FLAG_NO_RESIDUAL else 0)
                  | (REC_RAW if fl & FLAG_NO_QUANT else 0))
-    cents, codes = [], []
+    cents, codes, sse = [], [], []
     if fl & FLAG_NO_QUANT:                                            # ablation "quant" off
         zero = np.zeros(0, dtype=np.float32)
         cents = [zero, zero, zero]
         codes = [s_w, s_ea, s_eas]
+        sse = [0.0, 0.0, 0.0]
         blob = encode_record(n, 32, m_w, m_o, zero, zero, zero, s_w, s_ea, s_eas, rec_flags)
     else:
         for stream, s in enumerate((s_w, s_ea, s_eas)):               # quantize(.)
@@ -546,11 +556,13 @@ def compress_tensor(w_t, w_prev, ea, eas, p: Params, tensor_index: int = 0, weig
             c, idx = lloyd(s, c0, p.kmeans_iters)
             cents.append(c)
             codes.append((idx + 1).astype(np.uint8))
+            sse.append(quantisation_sse(s, c, idx))
         blob = encode_record(n, p.bits, m_w, m_o, cents[0], cents[1], cents[2], *codes, rec_flags=rec_flags)
     info = dict(numel=n, dw=dw, median=med, mean_abs_ea=mean, thr_w=thr_w, thr_o=thr_o,
                 m_w=m_w, m_o=m_o, nnz_w=int(m_w.sum()), nnz_o=int(m_o.sum()),
                 s_w=s_w, s_ea=s_ea, s_eas=s_eas, c_w=cents[0], c_ea=cents[1], c_eas=cents[2],
-                codes_w=codes[0], codes_ea=codes[1], codes_eas=codes[2])
+                codes_w=codes[0], codes_ea=codes[1], codes_eas=codes[2],
+                sse_w=sse[0], sse_ea=sse[1], sse_eas=sse[2])
     return blob, info
 
 

@@ -24,7 +24,7 @@ EXPORTS = ["excp_create", "excp_destroy", "excp_record_bytes", "excp_compress_bo
            "excp_compress_checkpoint_host", "excp_decompress_tensor", "excp_decompress_checkpoint",
            "excp_decompress_tensor_noalloc", "excp_dense_bytes", "excp_record_to_dense", "excp_checkpoint_to_dense",
            "excp_decompress_dense_tensor", "excp_decompress_dense_checkpoint", "excp_profile_enable", "excp_profile_stage_count", "excp_profile_stage_name", "excp_profile_read",
-           "excp_set_kmeans_margin", "excp_set_wait_limit", "excp_selftest_wait_timeout"]
+           "excp_set_kmeans_margin", "excp_set_wait_limit", "excp_selftest_wait_timeout", "excp_set_report_sse"]
 
 
 class ExcpError(RuntimeError):
@@ -41,7 +41,8 @@ class CParams(C.Structure):
 class CStats(C.Structure):
     _fields_ = [("numel", C.c_ulonglong), ("nnz_w", C.c_ulonglong), ("nnz_o", C.c_ulonglong),
                 ("blob_bytes", C.c_ulonglong), ("median", C.c_float), ("mean_abs_ea", C.c_float),
-                ("thr_w", C.c_float), ("thr_o", C.c_float)]
+                ("thr_w", C.c_float), ("thr_o", C.c_float),
+                ("sse_w", C.c_double), ("sse_ea", C.c_double), ("sse_eas", C.c_double)]
 
 
 FLAG_NO_W2M, FLAG_NO_M2W, FLAG_NO_RESIDUAL, FLAG_NO_PRUNE, FLAG_NO_QUANT = 1, 2, 4, 8, 16
@@ -109,6 +110,7 @@ def load_library() -> C.CDLL:
     lib.excp_profile_enable.argtypes = [vp, C.c_int]
     lib.excp_set_kmeans_margin.argtypes = [vp, C.c_int]
     lib.excp_set_wait_limit.argtypes = [vp, C.c_ulonglong]
+    lib.excp_set_report_sse.argtypes = [vp, C.c_int]
     lib.excp_selftest_wait_timeout.argtypes = [vp, C.c_ulonglong, vp]
     lib.excp_profile_stage_count.argtypes = []
     lib.excp_profile_stage_name.argtypes = [C.c_int]
@@ -205,6 +207,12 @@ class Handle:
         st = self.lib.excp_set_kmeans_margin(self._h, int(margin))
         if st != 0:
             raise ExcpError(st, "excp_set_kmeans_margin")
+
+    def set_report_sse(self, on: bool = True) -> None:
+        """excp_set_report_sse: fill sse_w, sse_ea, sse_eas of the statistics (off by default)."""
+        st = self.lib.excp_set_report_sse(self._h, int(on))
+        if st != 0:
+            raise ExcpError(st, "excp_set_report_sse")
 
     def set_wait_limit(self, nanoseconds: int) -> None:
         """excp_set_wait_limit: how long a warp waits for an asynchronous copy before the call gives up."""

@@ -65,6 +65,7 @@ struct excp_handle_s {
     int last_cuda_error = 0;
     int km_margin = 1;                   // see excp_set_kmeans_margin
     unsigned long long wait_limit_ns = 2000000000ull;   // see excp_set_wait_limit
+    bool report_sse = false;             // see excp_set_report_sse
     Profiler prof;
     // host-buffer path: two staging slots (inputs + records), its own copy streams
     float* stage[2][4] = {};
@@ -166,7 +167,7 @@ Params to_params(excp_handle h, const excp_params* params) {
 
 // All kernels of one group, in order.
 bool run_group(excp_handle h, const LaunchCfg& cfg, const TensorDesc* descs, int nt, u32 tiles,
-               const Params& p, unsigned char* blob, u64 blob_capacity, TensorResult* results) {
+               const Params& p, unsigned char* blob, u64 blob_capacity, TensorResult* results, bool want_sse) {
     if (!check(h, cudaMemsetAsync(h->d_state, 0, nt * sizeof(TensorState), cfg.stream))) return false;
     if (!check(h, cudaMemsetAsync(h->ws.cst, 0, nt * sizeof(CellState), cfg.stream))) return false;
     // the per-tile survivor counts start at zero, so that no kernel can meet a stale count where a sweep gave up
@@ -176,7 +177,7 @@ bool run_group(excp_handle h, const LaunchCfg& cfg, const TensorDesc* descs, int
     launch_stats(cfg, descs, h->d_state, nt, tiles, h->ws, p, h->d_call);
     launch_mask_compact(cfg, descs, h->d_state, nt, tiles, h->ws, p, h->d_call, blob_capacity);
     if (!(p.flags & OPT_NO_QUANT)) launch_kmeans(cfg, descs, h->d_state, nt, tiles, h->ws, h->km, p, h->d_call);
-    launch_pack(cfg, descs, h->d_state, nt, tiles, h->ws, p, blob, h->d_call, results);
+    launch_pack(cfg, descs, h->d_state, nt, tiles, h->ws, p, blob, h->d_call, results, want_sse);
     return check(h, cudaGetLastError());
 }
 
@@ -190,6 +191,7 @@ void fill_outputs(excp_handle h, size_t first, size_t count, const size_t* numel
             excp_tensor_stats& s = stats_out[i];
             s.numel = numel[i]; s.nnz_w = r.nnz_w; s.nnz_o = r.nnz_o; s.blob_bytes = r.blob_bytes;
             s.median = r.median; s.mean_abs_ea = r.mean_abs_ea; s.thr_w = r.thr_w; s.thr_o = r.thr_o;
+            s.sse_w = r.sse[0]; s.sse_ea = r.sse[1]; s.sse_eas = r.sse[2];
         }
     }
 }
@@ -402,7 +404,7 @@ static excp_status compress_impl(excp_handle h, const excp_params* params, size_
     for (size_t gi = 0; ok && gi < groups.size(); ++gi) {
         const Group& g = groups[gi];
         ok = run_group(h, cfg, dd + g.first, (int)g.count, g.tiles, p, static_cast<unsigned char*>(blob_out),
-                       blob_capacity, h->d_results + g.first);
+                       blob_capacity, h->d_results + g.first, stats_out != nullptr && h->report_sse);
     }
     ok = ok && check(h, cudaMemcpyAsync(h->h_results, h->d_results, num_tensors * sizeof(TensorResult),
                                         cudaMemcpyDeviceToHost, stream));
@@ -523,7 +525,7 @@ excp_status excp_compress_checkpoint_host(excp_handle h, const excp_params* para
         if (gi >= 2) ok = ok && check(h, cudaStreamWaitEvent(stream, h->ev_d2h[slot], 0));
         ok = ok && check(h, cudaMemsetAsync(&h->d_call->blob_cursor, 0, sizeof(u64), stream));
         ok = ok && run_group(h, cfg, dd + g.first, (int)g.count, g.tiles, p, h->stage_blob[slot],
-                             h->stage_blob_bytes, h->d_results + g.first);
+                             h->stage_blob_bytes, h->d_results + g.first, stats_out != nullptr && h->report_sse);
         ok = ok && check(h, cudaMemcpyAsync(h->h_results + g.first, h->d_results + g.first,
                                             g.count * sizeof(TensorResult), cudaMemcpyDeviceToHost, stream));
         ok = ok && check(h, cudaMemcpyAsync(h->h_call, h->d_call, sizeof(CallState), cudaMemcpyDeviceToHost, stream));
@@ -634,6 +636,12 @@ excp_status excp_decompress_checkpoint_w16(excp_handle h, const void* blob, cons
 excp_status excp_set_kmeans_margin(excp_handle h, int margin) {
     if (!h || margin < -1) return EXCP_ERR_INVALID_ARG;
     h->km_margin = margin;
+    return EXCP_OK;
+}
+
+excp_status excp_set_report_sse(excp_handle h, int enable) {
+    if (!h) return EXCP_ERR_INVALID_ARG;
+    h->report_sse = enable != 0;
     return EXCP_OK;
 }
 

@@ -111,6 +111,7 @@ struct TensorState {             // device scratch, zeroed per group
 struct TensorResult {            // copied back to the host at the end of a call
     u64 nnz_w, nnz_o, blob_off, blob_bytes;
     float median, mean_abs_ea, thr_w, thr_o;
+    double sse[3];               // sum of squared distances to the assigned centre, per stream (when asked for)
 };
 
 struct CallState {               // one per handle, device resident
@@ -398,7 +399,7 @@ void launch_kmeans(const LaunchCfg&, const TensorDesc* descs, TensorState* st, i
                    const Workspace& ws, const KmArrays& km, const Params& p, CallState* call);
 void launch_pack(const LaunchCfg&, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                  const Workspace& ws, const Params& p, unsigned char* blob, CallState* call,
-                 TensorResult* results);
+                 TensorResult* results, bool want_sse);
 void launch_decode(const LaunchCfg&, const DecDesc* descs, DecState* st, int nt, u32 tiles,
                    const Workspace& ws, CallState* call, int wfmt = WF_F32);
 void launch_record_to_dense(const LaunchCfg&, const DecDesc* descs, DecState* st, int nt, u32 tiles,

@@ -189,8 +189,12 @@ template <int NS>
 struct CellCountSmem {
     u32 tab[NS][NCLASS];
     u32 cnt[NS][NCELL];              // the block's counts of the tensor
+#ifdef EXCP_CC_U64
+    u64 mag[NS][NCELL];              // and sums of |Q|
+#else
     u32 lo[NS][NCELL];               // and sums of |Q|: low word,
     u32 hi[NS][NCELL];               //   carries out of it
+#endif
 };
 
 // Sweep 1: survivors per cell and the sum of their |Q| (a cell holds one sign).  A block takes a
@@ -210,7 +214,14 @@ __global__ void __launch_bounds__(CWARPS * 32, 2) cell_count_kernel(const Tensor
     const u32* tile_cnt = stream0 == 0 ? ws.tile_cnt_w : ws.tile_cnt_o;
 #pragma unroll
     for (int k = 0; k < NS; ++k)
-        for (int c = tid; c < NCELL; c += CWARPS * 32) { sm.cnt[k][c] = 0; sm.lo[k][c] = 0; sm.hi[k][c] = 0; }
+        for (int c = tid; c < NCELL; c += CWARPS * 32) {
+            sm.cnt[k][c] = 0;
+#ifdef EXCP_CC_U64
+            sm.mag[k][c] = 0;
+#else
+            sm.lo[k][c] = 0; sm.hi[k][c] = 0;
+#endif
+        }
     u32 tile = lo;
     while (tile < hi) {
         const int cur = find_tensor(descs, nt, tile);
@@ -225,16 +236,24 @@ __global__ void __launch_bounds__(CWARPS * 32, 2) cell_count_kernel(const Tensor
         for (int k = 0; k < NS; ++k) {
             const u32* tab = sm.tab[k];
             u32* cnt = sm.cnt[k];
+#ifdef EXCP_CC_U64
+            u64* smag = sm.mag[k];
+#else
             u32* slo = sm.lo[k];
             u32* shi = sm.hi[k];
+#endif
             const float a1 = st[cur].s[stream0 + k].scale1, a2 = st[cur].s[stream0 + k].scale2;
             auto tally = [&](float x) {
                 const u32 c = cell_of(x, tab);
                 if (!EXCP_IN_BOUNDS(call, c < (u32)NCELL)) return;
                 const u32 q = (u32)abs(__float2int_rn(__fmul_rn(__fmul_rn(x, a1), a2)));   // |Q(x)| < 2^31
                 atomicAdd(&cnt[c], 1u);
+#ifdef EXCP_CC_U64
+                atomicAdd(&smag[c], (u64)q);
+#else
                 const u32 old = atomicAdd(&slo[c], q);
                 if (old + q < old) atomicAdd(&shi[c], 1u);
+#endif
             };
             auto tally8 = [&](const float4& va, const float4& vb, bool two) {      // all table look-ups first
                 const float xs[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
@@ -248,12 +267,19 @@ __global__ void __launch_bounds__(CWARPS * 32, 2) cell_count_kernel(const Tensor
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
                     if (i < 4 || two) atomicAdd(&cnt[c[i]], 1u);
+#ifdef EXCP_CC_U64
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (i < 4 || two) atomicAdd(&smag[c[i]], (u64)q[i]);
+                (void)old;
+#else
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
                     if (i < 4 || two) old[i] = atomicAdd(&slo[c[i]], q[i]);
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
                     if ((i < 4 || two) && old[i] + q[i] < old[i]) atomicAdd(&shi[c[i]], 1u);
+#endif
             };
             sweep_segments(ws.surv[stream0 + k], tile_cnt, wlo, whi, lane, tally8, tally);
         }
@@ -267,9 +293,15 @@ __global__ void __launch_bounds__(CWARPS * 32, 2) cell_count_kernel(const Tensor
                 row[c] = n_c;
                 if (n_c) {
                     atomicAdd(&cs.cnt[c], n_c);
+#ifdef EXCP_CC_U64
+                    const u64 mag = sm.mag[k][c];
+                    sm.mag[k][c] = 0;
+#else
                     const u64 mag = ((u64)sm.hi[k][c] << 32) | sm.lo[k][c];
+                    sm.lo[k][c] = 0; sm.hi[k][c] = 0;
+#endif
                     if (mag) atomicAdd(&cs.mag[c], mag);
-                    sm.cnt[k][c] = 0; sm.lo[k][c] = 0; sm.hi[k][c] = 0;
+                    sm.cnt[k][c] = 0;
                 }
             }
         }
@@ -353,9 +385,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDes
 #pragma unroll
         for (int k = 0; k < 4; ++k) { cs.cntpre[c0 + k] = pc[k]; cs.sumpre[c0 + k] = ps[k]; }
         if (tid == 0) { cs.cntpre[NCELL] = tc; cs.sumpre[NCELL] = ts; }
-        // With 255 centres nearly every cell holds or neighbours a threshold at some iteration, and ten iterations
-        // on the cell table alone drift further than a cell: every cell is taken, so that no second round is needed.
-        const bool predict = nnz > SMALL_STREAM && margin < NCELL && K <= KMAX;
+        const bool predict = nnz > SMALL_STREAM && margin < NCELL;
         if (predict) {
             if (tid < NCELL / 32) selw[tid] = 0;
             if (tid < NCLASS) tab[tid] = cs.tab[tid];
@@ -436,9 +466,9 @@ __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDes
 template <int NS>
 struct CellGatherSmem {
     u32 tab[NS][NCLASS];
-    u32 sel[NS][NCELL / 32];
-    u32 cur[NS][NCELL];              // where the block's next value of each selected cell goes
+    u32 cur[NS][NCELL];              // where the block's next value of each selected cell goes; NOT_TAKEN for the others
 };
+constexpr u32 NOT_TAKEN = 0xffffffffu;
 
 // Sweep 2: the values of the selected cells into the gathered copy, every cell contiguous (the
 // order inside a cell is arbitrary: what is taken from it are integer sums).  Same grid and same
@@ -471,8 +501,8 @@ __global__ void __launch_bounds__(CWARPS * 32, 2) cell_gather_kernel(const Tenso
             const CellStream& cs = ws.cst[cur].s[stream0 + k];
             const u32* pos = km.pos[stream0 + k] + (u64)(blockIdx.x + cur) * NCELL;
             for (int c = tid; c < NCLASS; c += CWARPS * 32) sm.tab[k][c] = cs.tab[c];
-            for (int c = tid; c < NCELL / 32; c += CWARPS * 32) sm.sel[k][c] = cs.sel[c];
-            for (int c = tid; c < NCELL; c += CWARPS * 32) sm.cur[k][c] = pos[c];
+            for (int c = tid; c < NCELL; c += CWARPS * 32)
+                sm.cur[k][c] = ((cs.sel[c >> 5] >> (c & 31)) & 1u) ? pos[c] : NOT_TAKEN;
         }
         __syncthreads();
         const u32 n = seg_end - tile;
@@ -481,7 +511,6 @@ __global__ void __launch_bounds__(CWARPS * 32, 2) cell_gather_kernel(const Tenso
         for (int k = 0; k < NS; ++k) {
             if (!act[k]) continue;
             const u32* tab = sm.tab[k];
-            const u32* sel = sm.sel[k];
             u32* cursor = sm.cur[k];
             float* out = ws.bkt[stream0 + k] + (u64)tb * TILE;
             const u64 room = (u64)descs[cur].num_tiles * TILE;               // the tensor's share of the gathered copy
@@ -492,7 +521,7 @@ __global__ void __launch_bounds__(CWARPS * 32, 2) cell_gather_kernel(const Tenso
             auto file = [&](float x) {
                 const u32 c = cell_of(x, tab);
                 if (!EXCP_IN_BOUNDS(call, c < (u32)NCELL)) return;
-                if ((sel[c >> 5] >> (c & 31)) & 1u) put(c, x);
+                if (cursor[c] != NOT_TAKEN) put(c, x);
             };
             auto file8 = [&](const float4& va, const float4& vb, bool two) {       // all look-ups first
                 const float xs[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
@@ -504,7 +533,7 @@ __global__ void __launch_bounds__(CWARPS * 32, 2) cell_gather_kernel(const Tenso
                     if (!EXCP_IN_BOUNDS(call, c[i] < (u32)NCELL)) c[i] = 0;
                 }
 #pragma unroll
-                for (int i = 0; i < 8; ++i) hit |= ((sel[c[i] >> 5] >> (c[i] & 31)) & 1u) << i;
+                for (int i = 0; i < 8; ++i) hit |= (cursor[c[i]] != NOT_TAKEN ? 1u : 0u) << i;
                 if (!two) hit &= 15u;
                 if (hit) {
 #pragma unroll

@@ -6,6 +6,7 @@
 // last 32-bit code word of a tile may be shared with its neighbours: those words
 // are cleared beforehand and OR-ed into; interior words are stored whole.
 #include "excp_common.cuh"
+#include <type_traits>
 
 namespace excp {
 
@@ -35,6 +36,7 @@ __global__ void __launch_bounds__(64) header_kernel(const TensorDesc* __restrict
         r.nnz_w = s.nnz_w; r.nnz_o = s.nnz_o; r.blob_off = s.blob_off; r.blob_bytes = s.blob_bytes;
         r.median = __uint_as_float(s.median_bits); r.mean_abs_ea = s.mean_abs_ea;
         r.thr_w = s.thr_w; r.thr_o = s.thr_o;
+        r.sse[0] = r.sse[1] = r.sse[2] = 0.0;             // the packing kernels add to these
         results[t] = r;
         if (s.flags) atomicOr(&call->flags, s.flags);
     }
@@ -109,9 +111,10 @@ __global__ void __launch_bounds__(TPB) clear_edges_kernel(const TensorDesc* __re
 // neighbour's row comes by a shuffle, the last row of the previous 32 through a register.
 constexpr int PWARPS = TPB / 32;
 
-template <int NS, int NB>
+template <int NS, int NB, bool SSE>
 struct PackSmem {
     float thr[PWARPS][NS][1 << NB];     // the K - 1 thresholds, +inf after them
+    float cent[PWARPS][NS][SSE ? (1 << NB) : 1];   // the K centres (only when the quantisation error is wanted)
 };
 
 // Cluster of x = number of thresholds strictly below it.  thr_row: 16 fp32 thresholds
@@ -136,15 +139,17 @@ __device__ __forceinline__ u32 find_cluster(float x, const float* thr) {
     return p;
 }
 
-template <int NS, int NB>
+// SSE: also add up the squared distances to the assigned centres (the statistics' sse_* fields).
+template <int NS, int NB, bool SSE>
 __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __restrict__ descs,
                                                          const TensorState* __restrict__ st, int nt,
                                                          u32 tiles, Workspace ws, int stream0,
-                                                         unsigned char* blob, CallState* call) {
+                                                         unsigned char* blob, CallState* call,
+                                                         TensorResult* results) {
     constexpr int PER = 32 / NB;                   // codes per 32-bit word = survivors per row
     constexpr int KTHR = 1 << NB;
     constexpr int U = NS == 1 ? 2 : 1;             // rows a lane has in flight per stream
-    __shared__ __align__(16) PackSmem<NS, NB> sm;
+    __shared__ __align__(16) PackSmem<NS, NB, SSE> sm;
     if (call->flags & (FLAG_BLOB_FULL | FLAG_TIMEOUT)) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const u32 gw = blockIdx.x * PWARPS + warp, nw = gridDim.x * PWARPS;
@@ -158,6 +163,19 @@ __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __res
     float t3[NS], t7[NS], t11[NS];
 #pragma unroll
     for (int k = 0; k < NS; ++k) { words[k] = nullptr; t3[k] = t7[k] = t11[k] = 0.f; }
+    double sse[NS];                      // this lane's share of sum (x - centre)^2 in the tensor in hand
+#pragma unroll
+    for (int k = 0; k < NS; ++k) sse[k] = 0.0;
+    auto flush_sse = [&](int t) {        // floating-point atomics: the last bits depend on the order of arrival
+#pragma unroll
+        for (int k = 0; k < NS; ++k) {
+            double v = sse[k];
+#pragma unroll
+            for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            if (lane == 0 && v != 0.0) atomicAdd(&results[t].sse[stream0 + k], v);
+            sse[k] = 0.0;
+        }
+    };
 
     for (u32 w0 = wlo; w0 < whi; w0 += 32) {
         const u32 nt32 = min(32u, whi - w0);
@@ -169,6 +187,7 @@ __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __res
             if (!cnt) continue;
             const u32 tile = w0 + ti;
             if (cur < 0 || tile >= tb + ntl) {
+                if (SSE && cur >= 0) flush_sse(cur);
                 cur = find_tensor(descs, nt, tile);
                 tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
                 const TensorState& s = st[cur];
@@ -177,7 +196,10 @@ __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __res
 #pragma unroll
                 for (int k = 0; k < NS; ++k) {
                     words[k] = reinterpret_cast<u32*>(blob + s.blob_off + sec.codes[stream0 + k]);
-                    for (int j = lane; j < KTHR; j += 32) sm.thr[warp][k][j] = s.s[stream0 + k].thr[j];
+                    for (int j = lane; j < KTHR; j += 32) {
+                        sm.thr[warp][k][j] = s.s[stream0 + k].thr[j];
+                        if (SSE) sm.cent[warp][k][j] = s.s[stream0 + k].cent[j];
+                    }
                 }
                 __syncwarp();
 #pragma unroll
@@ -226,6 +248,16 @@ __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __res
                             }
                             const u32 have = cnt - PER * m;         // codes of this row that exist (the segment holds stale values after them)
                             if (have < (u32)PER) w &= (1u << (NB * have)) - 1u;
+                            if (SSE) {                            // the row's squared distances in fp32, rows added in fp64
+                                float acc = 0.f;
+#pragma unroll
+                                for (int i = 0; i < PER; ++i) {
+                                    const u32 code = (w >> (NB * i)) & ((1u << NB) - 1u);
+                                    const float d = __fsub_rn(xs[u][k][i], sm.cent[warp][k][code ? code - 1 : 0]);
+                                    acc = code ? __fmaf_rn(d, d, acc) : acc;
+                                }
+                                sse[k] += (double)acc;
+                            }
                         }
                         u32 prev = __shfl_up_sync(0xffffffffu, w, 1);
                         if (lane == 0) prev = carry[k];
@@ -245,6 +277,7 @@ __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __res
             }
         }
     }
+    if (SSE && cur >= 0) flush_sse(cur);
 }
 
 // Bitmaps: scratch -> record.  One thread per 16 bytes.
@@ -295,7 +328,7 @@ __global__ void __launch_bounds__(TPB) pack_raw_kernel(const TensorDesc* __restr
 
 void launch_pack(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
                  const Workspace& ws, const Params& p, unsigned char* blob, CallState* call,
-                 TensorResult* results) {
+                 TensorResult* results, bool want_sse) {
     header_kernel<<<nt, 64, 0, cfg.stream>>>(descs, st, blob, call, results, stored_bits(p), record_flags(p));
     if (!tiles) { prof_mark(cfg, ST_HEADER_EDGES, 1); return; }
     if (p.flags & OPT_NO_QUANT) {
@@ -311,16 +344,19 @@ void launch_pack(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st,
     clear_edges_kernel<<<(tiles + TPB - 1) / TPB, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, blob, call, p.bits);
     prof_mark(cfg, ST_HEADER_EDGES, 2);
     const u32 grid = min((tiles + PWARPS - 1) / PWARPS, (u32)cfg.sms * 6u);
-    if (p.bits == 4) {
-        pack_codes_kernel<1, 4><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 0, blob, call);
-        pack_codes_kernel<2, 4><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 1, blob, call);
-    } else if (p.bits == 2) {
-        pack_codes_kernel<1, 2><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 0, blob, call);
-        pack_codes_kernel<2, 2><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 1, blob, call);
-    } else {
-        pack_codes_kernel<1, 8><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 0, blob, call);
-        pack_codes_kernel<2, 8><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 1, blob, call);
-    }
+    auto run = [&](auto nb_tag, auto sse_tag) {
+        constexpr int NB = decltype(nb_tag)::value;
+        constexpr bool SSE = decltype(sse_tag)::value;
+        pack_codes_kernel<1, NB, SSE><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 0, blob, call, results);
+        pack_codes_kernel<2, NB, SSE><<<grid, TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws, 1, blob, call, results);
+    };
+    auto run_width = [&](auto sse_tag) {
+        if (p.bits == 4) run(std::integral_constant<int, 4>{}, sse_tag);
+        else if (p.bits == 2) run(std::integral_constant<int, 2>{}, sse_tag);
+        else run(std::integral_constant<int, 8>{}, sse_tag);
+    };
+    if (want_sse) run_width(std::true_type{});
+    else run_width(std::false_type{});
     prof_mark(cfg, ST_PACK_CODES, 2);
     const u64 quads = (u64)tiles * (TILE_WORDS / 4);
     copy_bitmaps_kernel<<<(u32)((quads + TPB - 1) / TPB), TPB, 0, cfg.stream>>>(descs, st, nt, tiles, ws,

@@ -18,6 +18,7 @@ W2M, M2W, RES, PRUNE, QUANT = (binding.FLAG_NO_W2M, binding.FLAG_NO_M2W, binding
 @pytest.fixture(scope="module")
 def handle():
     h = binding.Handle(workspace_numel=700_000)
+    h.set_report_sse(True)
     yield h
     h.close()
 

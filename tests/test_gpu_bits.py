@@ -14,6 +14,7 @@ pytestmark = pytest.mark.gpu
 @pytest.fixture(scope="module")
 def handle():
     h = binding.Handle(workspace_numel=700_000)
+    h.set_report_sse(True)
     yield h
     h.close()
 

@@ -19,6 +19,7 @@ DEV = "cuda:0"
 @pytest.fixture(scope="module")
 def handle():
     h = binding.Handle(workspace_numel=6_000_000)
+    h.set_report_sse(True)
     yield h
     h.close()
 
@@ -53,6 +54,8 @@ def check_against_oracle(p, quads_np, blob_t, offs, stats, first_index=0):
         assert np.float32(st.mean_abs_ea).view(np.uint32) == np.float32(info["mean_abs_ea"]).view(np.uint32), tag
         assert st.thr_w == info["thr_w"] and st.thr_o == info["thr_o"], tag
         assert (st.nnz_w, st.nnz_o) == (info["nnz_w"], info["nnz_o"]), tag
+        for got_sse, want_sse in ((st.sse_w, info["sse_w"]), (st.sse_ea, info["sse_ea"]), (st.sse_eas, info["sse_eas"])):
+            assert math.isclose(got_sse, want_sse, rel_tol=1e-5, abs_tol=0.0), tag    # a diagnostic: fp32 squares, sums in another order
         got = raw[offs[i]:offs[i + 1]]
         assert len(got) == len(want) == st.blob_bytes, tag
         rec = orc.parse_record(got)
@@ -137,6 +140,7 @@ def test_many_groups_and_tensor_index(handle):
     dquads = to_dev(quads)
     p = binding.Params(median_source=binding.MEDIAN_ABS_RESIDUAL, seed=5)
     small = binding.Handle(workspace_numel=140_000)
+    small.set_report_sse(True)
     try:
         blob, offs, stats = gpu_compress(small, p, dquads)
         check_against_oracle(p, quads, blob, offs, stats)
@@ -164,6 +168,7 @@ def test_centres_do_not_depend_on_which_cells_were_gathered(handle):
     n = 2_000_000
     dq = [synth.make_quad(n, 21, 0, device=DEV), synth.make_quad(70_000, 21, 1, device=DEV, outlier_frac=0.01)]
     h = binding.Handle(workspace_numel=n + 80_000)
+    h.set_report_sse(True)
     try:
         for bits in (4, 2):
             p = binding.Params(median_source=binding.MEDIAN_ABS_RESIDUAL, bits=bits, seed=5)

@@ -72,6 +72,7 @@ def test_hand_two_bit_kmeans_reaches_the_optimal_partition():
     s = info["s_w"].astype(np.float64)
     sse = float(np.sum((s - info["c_w"].astype(np.float64)[info["codes_w"] - 1]) ** 2))
     assert sse == G["sse_2bit"][0]
+    assert info["sse_w"] == G["sse_2bit"][0]                  # the reported objective is that sum
     assert orc.optimal_kmeans_1d_sse(info["s_w"], 3) == Fraction(G["sse_2bit"][0])
 
 
