@@ -48,7 +48,8 @@ def parse_args():
     ap.add_argument("--config", default="llama-7b")
     ap.add_argument("--median", default="residual", choices=["residual", "weight"])
     ap.add_argument("--kmeans-iters", type=int, default=10)
-    ap.add_argument("--workspace-numel", type=int, default=1_200_000_000)
+    ap.add_argument("--workspace-numel", type=int, default=1_700_000_000,
+                    help="elements of a group of tensors (the handle's scratch: about 24.3 bytes each)")
     ap.add_argument("--outlier-frac", type=float, default=0.0,
                     help="fraction of the residual at 10x scale (0.01 = the threshold-stress configuration)")
     ap.add_argument("--chain", type=int, default=0,
@@ -72,6 +73,14 @@ def parse_args():
                     help="largest tensor whose record and dense container go through the host archiver")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--max-tensors", type=int, default=None, help="debug: only the first tensors of the list")
+    ap.add_argument("--ncu-summary", default=None, metavar="REPORT",
+                    help="no benchmark: read an .ncu-rep of ONE kernel launch and write its text summary under profiles/ "
+                         "(and, with --ncu-stage, the DRAM byte counts `roofline.traffic` is derived from)")
+    ap.add_argument("--ncu-stage", default=None, help="stage whose dominant kernel the report captured (a key of KERNEL_SOURCES)")
+    ap.add_argument("--ncu-params", type=int, default=0, help="parameters of the captured workload")
+    ap.add_argument("--ncu-workload", default="", help="short tag of the captured workload for the file name, e.g. 410m14")
+    ap.add_argument("--ncu-command", default="", help="the command line that made the report (recorded in the summary)")
+    ap.add_argument("--ncu-note", default="", help="a sentence of reading recorded in the summary")
     return ap.parse_args()
 
 
@@ -343,6 +352,73 @@ KERNEL_SOURCES = {                                  # what each stage's dominant
 }
 
 
+NCU_KEEP = ("gpu__time_duration.sum", "dram__bytes_read.sum", "dram__bytes_write.sum", "gpu__dram_throughput.avg.pct_of_peak_sustained_elapsed",
+            "sm__throughput.avg.pct_of_peak_sustained_elapsed", "l1tex__throughput.avg.pct_of_peak_sustained_active",
+            "lts__throughput.avg.pct_of_peak_sustained_elapsed", "smsp__inst_executed.sum",
+            "smsp__issue_active.avg.pct_of_peak_sustained_active", "sm__warps_active.avg.pct_of_peak_sustained_active",
+            "launch__registers_per_thread", "launch__grid_size", "launch__block_size", "launch__occupancy_limit_registers",
+            "launch__occupancy_limit_shared_mem", "launch__occupancy_limit_warps",
+            "l1tex__data_pipe_lsu_wavefronts_mem_shared.sum", "l1tex__data_bank_conflicts_pipe_lsu_mem_shared.sum",
+            "smsp__inst_executed_op_shared_ld.sum", "smsp__inst_executed_op_shared_st.sum", "smsp__inst_executed_op_shared_atom.sum",
+            "lts__t_sectors_srcunit_tex_op_write.sum", "lts__t_sectors_srcunit_tex_op_read.sum")
+UNIT_SCALE = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9, "Tbyte": 1e12}
+
+
+def ncu_summary(args):
+    """Turns the .ncu-rep of one kernel launch (read with `ncu -i REPORT --page raw --csv`) into the short text
+    summary kept under profiles/, and records the launch's DRAM bytes in profiles/ncu_traffic.json together with a
+    digest of the kernel's sources, so that bench.py can tell when the counters have gone stale."""
+    import csv
+    raw = subprocess.run(["ncu", "-i", args.ncu_summary, "--page", "raw", "--csv"], capture_output=True, text=True, check=True).stdout
+    rows = list(csv.reader(raw.splitlines()))
+    hdr, units, vals = rows[0], rows[1], rows[2]
+    kernel = vals[hdr.index("Kernel Name")]
+    base = kernel.split("(")[0].replace("void ", "").split("<")[0].strip()
+    lines, got = [], {}
+    for h, u, v in zip(hdr, units, vals):
+        stall = h.startswith("smsp__average_warps_issue_stalled") and h.endswith("per_issue_active.ratio")
+        if h in NCU_KEEP or stall:
+            try:
+                if stall and float(v) < 0.3:
+                    continue
+            except ValueError:
+                pass
+            lines.append(f"{h} [{u}] = {v}")
+            got[h] = (u, v)
+    dram = {}
+    for key in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
+        u, v = got[key]
+        dram[key] = float(v.replace(",", "")) * UNIT_SCALE[u]
+    head = [f"ncu counters of one launch of {kernel[:150]}",
+            f"workload: {args.ncu_workload} ({args.ncu_params} parameters)" if args.ncu_params else f"workload: {args.ncu_workload}",
+            f"capture: {args.ncu_command}", f"read with: ncu -i {os.path.basename(args.ncu_summary)} --page raw --csv"]
+    if args.ncu_params:
+        per = (dram["dram__bytes_read.sum"] + dram["dram__bytes_write.sum"]) / args.ncu_params
+        us = float(got["gpu__time_duration.sum"][1].replace(",", "")) * {"us": 1.0, "ms": 1e3, "ns": 1e-3, "s": 1e6}[got["gpu__time_duration.sum"][0]]
+        inst = float(got["smsp__inst_executed.sum"][1].replace(",", "")) * 32 / args.ncu_params
+        head.append(f"derived: DRAM traffic {per:.2f} B/param, {(dram['dram__bytes_read.sum'] + dram['dram__bytes_write.sum']) / us / 1e3:.0f} GB/s "
+                    f"under the profiler, {inst:.1f} thread-instructions per parameter")
+    if args.ncu_note:
+        head.append("reading: " + args.ncu_note)
+    os.makedirs(os.path.join(ROOT, "profiles"), exist_ok=True)
+    out_path = os.path.join(ROOT, "profiles", f"ncu_{base}_{args.ncu_workload or 'case'}.txt")
+    with open(out_path, "w") as f:
+        f.write("\n".join(head + sorted(lines)) + "\n")
+    if args.ncu_stage:
+        try:
+            with open(TRAFFIC_JSON) as f:
+                table = json.load(f)
+        except Exception:
+            table = {}
+        table[args.ncu_stage] = {"kernel": base, "params": args.ncu_params, "dram_read_bytes": dram["dram__bytes_read.sum"],
+                                 "dram_write_bytes": dram["dram__bytes_write.sum"], "sources": KERNEL_SOURCES[args.ncu_stage],
+                                 "digest": source_digest(KERNEL_SOURCES[args.ncu_stage]), "summary": os.path.basename(out_path)}
+        with open(TRAFFIC_JSON, "w") as f:
+            json.dump(table, f, indent=1, sort_keys=True)
+            f.write("\n")
+    print(out_path)
+
+
 def run_chain(args, torch, binding, synth, ranks, dev):
     """Chained run (Section 3.4, Algorithm 3): `--chain` consecutive checkpoints W_(k+1) = W_k + delta_k with fresh
     moments; every residual is taken against the previous RECONSTRUCTION, compressed, and decompressed in place;
@@ -597,7 +673,7 @@ def run_ours(args):
         return chunks
 
     if not args.no_dense and not args.no_decompress and args.bits == 4 and wb == 4 and world == 1:
-        chunk_cap = ws_numel
+        chunk_cap = max(min(ws_numel, 1_200_000_000), max(n for _, n in shapes))   # outputs of one chunk of tensors
         out_w = torch.empty(chunk_cap, dtype=torch.float32, device=dev)
         out_a = torch.empty(chunk_cap, dtype=torch.float32, device=dev)
         out_s = torch.empty(chunk_cap, dtype=torch.float32, device=dev)
@@ -794,6 +870,8 @@ def run_ours(args):
 
 def main():
     args = parse_args()
+    if args.ncu_summary:
+        return ncu_summary(args)
     if args.impl == "reference":
         run_reference(args)
     else:

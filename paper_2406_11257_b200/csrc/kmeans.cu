@@ -189,12 +189,8 @@ template <int NS>
 struct CellCountSmem {
     u32 tab[NS][NCLASS];
     u32 cnt[NS][NCELL];              // the block's counts of the tensor
-#ifdef EXCP_CC_U64
-    u64 mag[NS][NCELL];              // and sums of |Q|
-#else
     u32 lo[NS][NCELL];               // and sums of |Q|: low word,
     u32 hi[NS][NCELL];               //   carries out of it
-#endif
 };
 
 // Sweep 1: survivors per cell and the sum of their |Q| (a cell holds one sign).  A block takes a
@@ -216,11 +212,7 @@ __global__ void __launch_bounds__(CWARPS * 32, 2) cell_count_kernel(const Tensor
     for (int k = 0; k < NS; ++k)
         for (int c = tid; c < NCELL; c += CWARPS * 32) {
             sm.cnt[k][c] = 0;
-#ifdef EXCP_CC_U64
-            sm.mag[k][c] = 0;
-#else
             sm.lo[k][c] = 0; sm.hi[k][c] = 0;
-#endif
         }
     u32 tile = lo;
     while (tile < hi) {
@@ -236,24 +228,16 @@ __global__ void __launch_bounds__(CWARPS * 32, 2) cell_count_kernel(const Tensor
         for (int k = 0; k < NS; ++k) {
             const u32* tab = sm.tab[k];
             u32* cnt = sm.cnt[k];
-#ifdef EXCP_CC_U64
-            u64* smag = sm.mag[k];
-#else
             u32* slo = sm.lo[k];
             u32* shi = sm.hi[k];
-#endif
             const float a1 = st[cur].s[stream0 + k].scale1, a2 = st[cur].s[stream0 + k].scale2;
             auto tally = [&](float x) {
                 const u32 c = cell_of(x, tab);
                 if (!EXCP_IN_BOUNDS(call, c < (u32)NCELL)) return;
                 const u32 q = (u32)abs(__float2int_rn(__fmul_rn(__fmul_rn(x, a1), a2)));   // |Q(x)| < 2^31
                 atomicAdd(&cnt[c], 1u);
-#ifdef EXCP_CC_U64
-                atomicAdd(&smag[c], (u64)q);
-#else
                 const u32 old = atomicAdd(&slo[c], q);
                 if (old + q < old) atomicAdd(&shi[c], 1u);
-#endif
             };
             auto tally8 = [&](const float4& va, const float4& vb, bool two) {      // all table look-ups first
                 const float xs[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
@@ -267,19 +251,12 @@ __global__ void __launch_bounds__(CWARPS * 32, 2) cell_count_kernel(const Tensor
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
                     if (i < 4 || two) atomicAdd(&cnt[c[i]], 1u);
-#ifdef EXCP_CC_U64
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    if (i < 4 || two) atomicAdd(&smag[c[i]], (u64)q[i]);
-                (void)old;
-#else
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
                     if (i < 4 || two) old[i] = atomicAdd(&slo[c[i]], q[i]);
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
                     if ((i < 4 || two) && old[i] + q[i] < old[i]) atomicAdd(&shi[c[i]], 1u);
-#endif
             };
             sweep_segments(ws.surv[stream0 + k], tile_cnt, wlo, whi, lane, tally8, tally);
         }
@@ -293,13 +270,8 @@ __global__ void __launch_bounds__(CWARPS * 32, 2) cell_count_kernel(const Tensor
                 row[c] = n_c;
                 if (n_c) {
                     atomicAdd(&cs.cnt[c], n_c);
-#ifdef EXCP_CC_U64
-                    const u64 mag = sm.mag[k][c];
-                    sm.mag[k][c] = 0;
-#else
                     const u64 mag = ((u64)sm.hi[k][c] << 32) | sm.lo[k][c];
                     sm.lo[k][c] = 0; sm.hi[k][c] = 0;
-#endif
                     if (mag) atomicAdd(&cs.mag[c], mag);
                     sm.cnt[k][c] = 0;
                 }

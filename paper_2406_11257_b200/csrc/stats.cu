@@ -503,8 +503,12 @@ __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* _
                 fetch4w<WT>(stg + k * SCH, cw[k] + e0, o, full ? (u32)SCH : nbulk_w, valid, out);
             }
         };
-        u32 ke[SCH / 32];
+        // exact sum of |ea|: every lane adds its 16 values of the chunk in fp64 (exact: they span at most
+        // 52 bits, see below), and the chunk's sums join a 64-bit integer whose unit 2^(ecur-174) is tied to
+        // the largest exponent this warp has met in this tensor
+        double dsum = 0.0;
         u32 kmax = 0;
+        u32 lowkey = 0xffffffffu;            // smallest non-zero key, minus one
         auto sweep_chunk = [&](auto full_tag) {
             constexpr bool FULL = decltype(full_tag)::value;     // the whole chunk came by bulk copy
 #pragma unroll
@@ -543,37 +547,32 @@ __global__ void __launch_bounds__(TPB, 2) stats_sweep_kernel(const TensorDesc* _
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const u32 kk = __float_as_uint(e[k]) & 0x7fffffffu;
-                    ke[r * 4 + k] = kk;
                     kmax = max(kmax, kk);
+                    lowkey = min(lowkey, kk - 1u);
+                    dsum += (double)__uint_as_float(kk);
                 }
             }
         };
         if (valid == (u32)SCH) sweep_chunk(std::true_type{});
         else sweep_chunk(std::false_type{});
-        // exact sum of |ea|: integer mantissas shifted to a common unit tied to the largest
-        // exponent this warp has met in this tensor
         const int emax = max((int)(__reduce_max_sync(0xffffffffu, kmax) >> 23), 1);
         if (emax > ecur) { flush_acc(cc.tns); ecur = emax; }
         const int bias = 24 - ecur;
-        u32 lowkey = 0xffffffffu;            // smallest non-zero key, minus one
-#pragma unroll
-        for (int j = 0; j < SCH / 32; ++j) {
-            const u32 kk = ke[j];
-            const u32 e1 = max(kk >> 23, 1u);
-            const u32 m = kk - ((e1 - 1u) << 23);                    // mantissa with its implicit bit (none below 2^-126)
-            u32 pow2;                                                // 2^sh, sh = e1 - ecur + 24 <= 24; 0 when sh < 0
-            asm("shl.b32 %0, 1, %1;" : "=r"(pow2) : "r"((u32)((int)e1 + bias)));   // shl clamps: a "negative" amount gives 0
-            acc += (u64)m * (u64)pow2;                               // one wide multiply-add
-            lowkey = min(lowkey, kk - 1u);
-        }
-        // rare: a non-zero value more than 24 binades under the unit goes to the table of small ones
+        // A value is a whole number of units iff its exponent is within 24 binades of ecur; then a lane's 16
+        // values (each below 2^(ecur-126), the unit 2^(ecur-174)) add up to less than 2^52 units: exact in fp64.
         const bool has_low = lowkey != 0xffffffffu && (int)max((lowkey + 1u) >> 23, 1u) + bias < 0;
-        if (__any_sync(0xffffffffu, has_low)) {
-#pragma unroll
-            for (int j = 0; j < SCH / 32; ++j) {
-                const u32 kk = ke[j];
+        if (!__any_sync(0xffffffffu, has_low)) {
+            const double unit_inv = __longlong_as_double((s64)(1197 - ecur) << 52);          // 2^(174-ecur)
+            acc += (u64)__double2ull_rz(dsum * unit_inv);
+        } else {
+            // rare: some non-zero value lies more than 24 binades under the unit.  Redo the chunk in integers:
+            // mantissas shifted to the unit, the small ones into the table of their own
+            for (u32 o = lane; o < valid; o += 32) {
+                const u32 kk = __float_as_uint(o < nbulk ? stg[2 * SCH + o] : __ldg(cea + e0 + o)) & 0x7fffffffu;
                 const u32 e1 = max(kk >> 23, 1u);
-                if (kk && (int)e1 + bias < 0) atomicAdd(&st[cc.tns].sum_low[e1], (u64)(kk - ((e1 - 1u) << 23)));
+                const u32 m = kk - ((e1 - 1u) << 23);                    // mantissa with its implicit bit (none below 2^-126)
+                if ((int)e1 + bias >= 0) acc += (u64)m << (e1 + bias);
+                else if (kk) atomicAdd(&st[cc.tns].sum_low[e1], (u64)m);
             }
         }
         if (++since >= 32) flush_acc(cc.tns);
