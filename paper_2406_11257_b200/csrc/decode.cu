@@ -193,6 +193,47 @@ __device__ __forceinline__ u32 expand_word(u32 m, u32 (&c)[NB], const u32* __res
     return bad;
 }
 
+// The sparse form of expand_word for the two moment streams, which share their bitmap word `m` and keep
+// few elements: one step per set bit (the caller makes sure that no lane of the warp has more than
+// SPARSE_MAX of them, so that a stream's codes fit the first two words of its window).  TO_ROWS: the codes
+// go to the lane's (zeroed) rows in shared memory, a byte each; otherwise they are returned as the dense
+// layout's 16 bytes, a nibble each (NB = 4).
+constexpr u32 SPARSE_MAX = 8;
+
+template <int NB, bool TO_ROWS>
+__device__ __forceinline__ u32 expand_sparse2(u32 m, const u32 (&c1)[NB], const u32 (&c2)[NB], unsigned char* row1,
+                                              unsigned char* row2, uint4& d1, uint4& d2) {
+    u64 w1 = c1[0], w2 = c2[0];
+    if (NB > 1) { w1 |= (u64)c1[NB > 1 ? 1 : 0] << 32; w2 |= (u64)c2[NB > 1 ? 1 : 0] << 32; }
+    u64 lo1 = 0, hi1 = 0, lo2 = 0, hi2 = 0;
+    u32 bad = 0;
+    constexpr u32 CMASK = (1u << NB) - 1u;
+    if (TO_ROWS) {
+        reinterpret_cast<uint4*>(row1)[0] = make_uint4(0, 0, 0, 0); reinterpret_cast<uint4*>(row1)[1] = make_uint4(0, 0, 0, 0);
+        reinterpret_cast<uint4*>(row2)[0] = make_uint4(0, 0, 0, 0); reinterpret_cast<uint4*>(row2)[1] = make_uint4(0, 0, 0, 0);
+    }
+    while (m) {
+        const u32 pos = (u32)__ffs((int)m) - 1u;
+        m &= m - 1u;
+        const u32 k1 = (u32)w1 & CMASK, k2 = (u32)w2 & CMASK;
+        w1 >>= NB; w2 >>= NB;
+        bad |= (k1 == 0u) | (k2 == 0u);
+        if (TO_ROWS) {
+            row1[pos] = (unsigned char)k1;
+            row2[pos] = (unsigned char)k2;
+        } else {
+            const u32 sh = 4u * (pos & 15u);
+            const u64 v1 = (u64)k1 << sh, v2 = (u64)k2 << sh;
+            if (pos < 16u) { lo1 |= v1; lo2 |= v2; } else { hi1 |= v1; hi2 |= v2; }
+        }
+    }
+    if (!TO_ROWS) {
+        d1 = make_uint4((u32)lo1, (u32)(lo1 >> 32), (u32)hi1, (u32)(hi1 >> 32));
+        d2 = make_uint4((u32)lo2, (u32)(lo2 >> 32), (u32)hi2, (u32)(hi2 >> 32));
+    }
+    return bad;
+}
+
 // Eight bytes-per-element words -> four nibbles-per-element words (the dense layout's 16 bytes).
 __device__ __forceinline__ uint4 pack_nibbles(const u32 (&o)[8]) {
     u32 d[4];
@@ -220,40 +261,54 @@ template <bool DENSE, int NB, typename WT>
 __device__ __forceinline__ u32 decode_block(const DecTile& t, const DecDesc& d, const DecState& s, DecodeSmem& sm, int warp,
                                             int lane, u32 blk, u32 a, u32 b, u64 gw, u64 go, const CallState* call) {
     u32 bad = 0;
-    u32 ow8[8], oa8[8], os8[8];
-    {
-        u32 c[NB];
-        load_window<NB>(t.sec0, gw, (u32)__popc(a), c, call, s.nnz_w);
-        bad |= expand_word<NB>(a, c, sm.sel, sm.spread, ow8);
-    }
-    {
-        u32 c1[NB], c2[NB];
-        load_window<NB>(t.sec1, go, (u32)__popc(b), c1, call, s.nnz_o);
-        load_window<NB>(t.sec2, go, (u32)__popc(b), c2, call, s.nnz_o);
-        bad |= expand_word<NB>(b, c1, sm.sel, sm.spread, oa8);
-        bad |= expand_word<NB>(b, c2, sm.sel, sm.spread, os8);
-    }
-    const u64 e0 = t.base + (u64)blk * 1024u;            // first element of the block
-    if (DENSE) {                                         // NB == 4: 32 codes = 16 bytes per lane and section
-        const u64 i = e0 + 32u * lane;
-        if (i < t.n) {
-            const u64 sb = dense_section_bytes(t.n, BITS);
-            unsigned char* out = d.dense + header_bytes(KMAX) + i / 2;
-            *reinterpret_cast<uint4*>(out) = pack_nibbles(ow8);
-            *reinterpret_cast<uint4*>(out + sb) = pack_nibbles(oa8);
-            *reinterpret_cast<uint4*>(out + 2 * sb) = pack_nibbles(os8);
-        }
-        return bad;
-    }
     unsigned char* rw = sm.rows[warp][0] + lane * ROW_BYTES;
     unsigned char* ra = sm.rows[warp][1] + lane * ROW_BYTES;
     unsigned char* rs = sm.rows[warp][2] + lane * ROW_BYTES;
-    reinterpret_cast<uint4*>(rw)[0] = make_uint4(ow8[0], ow8[1], ow8[2], ow8[3]);
-    reinterpret_cast<uint4*>(rw)[1] = make_uint4(ow8[4], ow8[5], ow8[6], ow8[7]);
-    reinterpret_cast<uint4*>(ra)[0] = make_uint4(oa8[0], oa8[1], oa8[2], oa8[3]);
-    reinterpret_cast<uint4*>(ra)[1] = make_uint4(oa8[4], oa8[5], oa8[6], oa8[7]);
-    reinterpret_cast<uint4*>(rs)[0] = make_uint4(os8[0], os8[1], os8[2], os8[3]);
-    reinterpret_cast<uint4*>(rs)[1] = make_uint4(os8[4], os8[5], os8[6], os8[7]);
+    const u64 e0 = t.base + (u64)blk * 1024u;            // first element of the block
+    const u64 sb = DENSE ? dense_section_bytes(t.n, BITS) : 0;
+    unsigned char* dout = DENSE ? d.dense + header_bytes(KMAX) + (e0 + 32u * lane) / 2 : nullptr;
+    const bool dlive = e0 + 32u * lane < t.n;            // DENSE: 32 codes = 16 bytes per lane and section (NB == 4)
+    {
+        u32 c[NB], ow8[8];
+        load_window<NB>(t.sec0, gw, (u32)__popc(a), c, call, s.nnz_w);
+        bad |= expand_word<NB>(a, c, sm.sel, sm.spread, ow8);
+        if (DENSE) {
+            if (dlive) *reinterpret_cast<uint4*>(dout) = pack_nibbles(ow8);
+        } else {
+            reinterpret_cast<uint4*>(rw)[0] = make_uint4(ow8[0], ow8[1], ow8[2], ow8[3]);
+            reinterpret_cast<uint4*>(rw)[1] = make_uint4(ow8[4], ow8[5], ow8[6], ow8[7]);
+        }
+    }
+    {
+        u32 c1[NB], c2[NB];
+        const u32 pb = (u32)__popc(b);
+        load_window<NB>(t.sec1, go, pb, c1, call, s.nnz_o);
+        load_window<NB>(t.sec2, go, pb, c2, call, s.nnz_o);
+        if (__reduce_max_sync(0xffffffffu, pb) <= SPARSE_MAX) {      // the usual case: few moments survive
+            uint4 d1, d2;
+            bad |= expand_sparse2<NB, !DENSE>(b, c1, c2, ra, rs, d1, d2);
+            if (DENSE && dlive) {
+                *reinterpret_cast<uint4*>(dout + sb) = d1;
+                *reinterpret_cast<uint4*>(dout + 2 * sb) = d2;
+            }
+        } else {
+            u32 oa8[8], os8[8];
+            bad |= expand_word<NB>(b, c1, sm.sel, sm.spread, oa8);
+            bad |= expand_word<NB>(b, c2, sm.sel, sm.spread, os8);
+            if (DENSE) {
+                if (dlive) {
+                    *reinterpret_cast<uint4*>(dout + sb) = pack_nibbles(oa8);
+                    *reinterpret_cast<uint4*>(dout + 2 * sb) = pack_nibbles(os8);
+                }
+            } else {
+                reinterpret_cast<uint4*>(ra)[0] = make_uint4(oa8[0], oa8[1], oa8[2], oa8[3]);
+                reinterpret_cast<uint4*>(ra)[1] = make_uint4(oa8[4], oa8[5], oa8[6], oa8[7]);
+                reinterpret_cast<uint4*>(rs)[0] = make_uint4(os8[0], os8[1], os8[2], os8[3]);
+                reinterpret_cast<uint4*>(rs)[1] = make_uint4(os8[4], os8[5], os8[6], os8[7]);
+            }
+        }
+    }
+    if (DENSE) return bad;
     __syncwarp();
     const WT* w_prev = static_cast<const WT*>(d.w_prev);
     WT* w_out = static_cast<WT*>(d.w_out);
@@ -333,8 +388,11 @@ __device__ __forceinline__ void decode_block_raw(const DecTile& t, const DecDesc
     __syncwarp();
 }
 
+#ifndef EXCP_DENSE_MIN_BLOCKS
+#define EXCP_DENSE_MIN_BLOCKS 3
+#endif
 template <bool DENSE, typename WT>
-__global__ void __launch_bounds__(TPB, EXCP_DEC_MIN_BLOCKS) decode_kernel(const DecDesc* __restrict__ descs,
+__global__ void __launch_bounds__(TPB, DENSE ? EXCP_DENSE_MIN_BLOCKS : EXCP_DEC_MIN_BLOCKS) decode_kernel(const DecDesc* __restrict__ descs,
                                                      const DecState* __restrict__ st, int nt, u32 tiles,
                                                      Workspace ws, CallState* call) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -492,7 +550,7 @@ void launch_record_to_dense(const LaunchCfg& cfg, const DecDesc* descs, DecState
     dense_header_kernel<<<nt, 64, 0, cfg.stream>>>(descs, st, call);
     prof_mark(cfg, ST_DEC_PREP, tiles ? 4 : 2);
     if (!tiles) return;
-    const u32 grid = min((tiles + DEC_WARPS - 1) / DEC_WARPS, (u32)cfg.sms * (u32)EXCP_DEC_MIN_BLOCKS);
+    const u32 grid = min((tiles + DEC_WARPS - 1) / DEC_WARPS, (u32)cfg.sms * (u32)EXCP_DENSE_MIN_BLOCKS);
     cudaFuncSetAttribute(decode_kernel<true, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecodeSmem));
     decode_kernel<true, float><<<grid, TPB, sizeof(DecodeSmem), cfg.stream>>>(descs, st, nt, tiles, ws, call);
     prof_mark(cfg, ST_DENSE, 1);
@@ -576,25 +634,35 @@ __global__ void __launch_bounds__(TPB) dense_decode_kernel(const DecDesc* __rest
         const u64 sb = dense_section_bytes(n, BITS);
         const unsigned char* sec = d.rec + header_bytes(KMAX);
         const u64 base = (u64)(tile - tb) * TILE;
+        // all loads of the tile's four rounds first, then the arithmetic and the stores
+        u32 ww[ROUNDS], wa[ROUNDS], we[ROUNDS];
+        float wp[ROUNDS][4];
 #pragma unroll
         for (int r = 0; r < ROUNDS; ++r) {
             const u64 i0 = base + r * (TPB * 4) + tid * 4;     // four elements = 16 bits per stream
+            ww[r] = wa[r] = we[r] = 0;
+            wp[r][0] = wp[r][1] = wp[r][2] = wp[r][3] = 0.f;
+            if (i0 < n) {
+                ww[r] = *reinterpret_cast<const unsigned short*>(sec + i0 / 2);
+                wa[r] = *reinterpret_cast<const unsigned short*>(sec + sb + i0 / 2);
+                we[r] = *reinterpret_cast<const unsigned short*>(sec + 2 * sb + i0 / 2);
+                load4(w_prev, i0, n, wp[r]);
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < ROUNDS; ++r) {
+            const u64 i0 = base + r * (TPB * 4) + tid * 4;
             if (i0 >= n) continue;
-            const u32 ww = *reinterpret_cast<const unsigned short*>(sec + i0 / 2);
-            const u32 wa = *reinterpret_cast<const unsigned short*>(sec + sb + i0 / 2);
-            const u32 we = *reinterpret_cast<const unsigned short*>(sec + 2 * sb + i0 / 2);
-            const u32 zw = nonzero_nibbles(ww), za = nonzero_nibbles(wa), ze = nonzero_nibbles(we);
+            const u32 zw = nonzero_nibbles(ww[r]), za = nonzero_nibbles(wa[r]), ze = nonzero_nibbles(we[r]);
             cw += __popc(zw); co += __popc(za);
             bad |= (za ^ ze) | (za & ~zw);                // moments disagree; a moment kept where the weight is pruned
             const u32 left = n - i0 >= 4 ? 4u : (u32)(n - i0);
-            if (left < 4 && ((ww | wa | we) >> (4 * left))) bad = 1;   // codes past the last element
-            float wp[4];
-            load4(w_prev, i0, n, wp);
+            if (left < 4 && ((ww[r] | wa[r] | we[r]) >> (4 * left))) bad = 1;   // codes past the last element
             float ow[4], oa[4], os[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const u32 c0 = (ww >> (4 * k)) & 15u, c1 = (wa >> (4 * k)) & 15u, c2 = (we >> (4 * k)) & 15u;
-                ow[k] = c0 ? __fadd_rn(wp[k], cent[0][c0]) : wp[k];    // pruned: W^_(t-1) bit for bit
+                const u32 c0 = (ww[r] >> (4 * k)) & 15u, c1 = (wa[r] >> (4 * k)) & 15u, c2 = (we[r] >> (4 * k)) & 15u;
+                ow[k] = c0 ? __fadd_rn(wp[r][k], cent[0][c0]) : wp[r][k];    // pruned: W^_(t-1) bit for bit
                 oa[k] = cent[1][c1];
                 os[k] = cent[2][c2];
             }

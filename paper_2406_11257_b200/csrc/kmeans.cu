@@ -537,13 +537,14 @@ __device__ __forceinline__ void scan_range(const float* __restrict__ data, u32 a
     const u32 h = min(e, (a + 3u) & ~3u);                    // up to three values before a 16-byte boundary
     if (a + lane < h) test(__ldg(data + a + lane));
     const u32 be = h + ((e - h) & ~3u);
-    for (u32 i = h + 4u * lane; i < be; i += 512u) {         // four 16-byte loads in flight per lane
-        float4 v[4];
+    constexpr int INFL = 8;                                  // 16-byte loads in flight per lane
+    for (u32 i = h + 4u * lane; i < be; i += 128u * INFL) {
+        float4 v[INFL];
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
+        for (int k = 0; k < INFL; ++k)
             if (i + 128u * k < be) v[k] = __ldg(reinterpret_cast<const float4*>(data + i + 128u * k));
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
+        for (int k = 0; k < INFL; ++k)
             if (i + 128u * k < be) { test(v[k].x); test(v[k].y); test(v[k].z); test(v[k].w); }
     }
     if (be + lane < e) test(__ldg(data + be + lane));
