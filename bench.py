@@ -73,6 +73,7 @@ def parse_args():
                     help="largest tensor whose record and dense container go through the host archiver")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--max-tensors", type=int, default=None, help="debug: only the first tensors of the list")
+    ap.add_argument("--km-margin", type=int, default=None, help="tuning: excp_set_kmeans_margin (the records do not depend on it)")
     ap.add_argument("--ncu-summary", default=None, metavar="REPORT",
                     help="no benchmark: read an .ncu-rep of ONE kernel launch and write its text summary under profiles/ "
                          "(and, with --ncu-stage, the DRAM byte counts `roofline.traffic` is derived from)")
@@ -549,6 +550,8 @@ def run_ours(args):
     ws_numel = min(args.workspace_numel, n_tot + 4096 * len(shapes))
     ws_numel = max(ws_numel, max(n for _, n in shapes))
     h = binding.Handle(workspace_numel=ws_numel)
+    if args.km_margin is not None:
+        h.set_kmeans_margin(args.km_margin)
 
     def params(median):
         return binding.Params(kmeans_iters=args.kmeans_iters, bits=args.bits,
