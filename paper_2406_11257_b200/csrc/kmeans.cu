@@ -30,6 +30,7 @@
 //   cell_gather     sweep: values of the selected cells into the gathered copy
 //   kmeans_iterate  the exact iterations
 #include "excp_common.cuh"
+#include <cstdio>
 
 namespace excp {
 
@@ -379,11 +380,22 @@ __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDes
                     const u32 a_lo = (bits & 0x7fffffffu) >> sh << sh;
                     const u32 a_hi = min(a_lo + (1u << sh), 0x7f7fffffu);
                     const double v_lo = (double)__uint_as_float(a_lo), v_hi = (double)__uint_as_float(a_hi);
-                    double f = v_hi > v_lo ? (fabs((double)tj) - v_lo) / (v_hi - v_lo) : 1.0;
-                    f = fmin(fmax(f, 0.0), 1.0);
+                    const double n_c = (double)(cs.cntpre[c + 1] - cs.cntpre[c]);
+                    const double s_c = (double)(cs.sumpre[c + 1] - cs.sumpre[c]);
+                    // The cell's values are taken as spread evenly over the widest interval inside the cell
+                    // that is centred on their mean: the whole cell when the mean is its middle, a point when
+                    // the mean sits on an edge.
+                    double f = 1.0;
+                    if (n_c > 0.0) {
+                        const double mean = fmin(fmax(fabs(s_c / n_c * scale), v_lo), v_hi);
+                        const double half = fmin(mean - v_lo, v_hi - mean);
+                        const double x = fabs((double)tj);
+                        f = half > 0.0 ? (x - (mean - half)) / (2.0 * half) : (x >= mean ? 1.0 : 0.0);
+                        f = fmin(fmax(f, 0.0), 1.0);
+                    }
                     if (bits >> 31) f = 1.0 - f;
-                    Lp[tid] = (double)cs.cntpre[c] + f * (double)(cs.cntpre[c + 1] - cs.cntpre[c]);
-                    Sp[tid] = (double)cs.sumpre[c] + f * (double)(cs.sumpre[c + 1] - cs.sumpre[c]);
+                    Lp[tid] = (double)cs.cntpre[c] + f * n_c;
+                    Sp[tid] = (double)cs.sumpre[c] + f * s_c;
                 } else if (tid == K - 1) {
                     Lp[tid] = (double)tc;
                     Sp[tid] = (double)ts;
@@ -644,6 +656,9 @@ __global__ void __launch_bounds__(IT_THREADS) kmeans_iterate_kernel(const Tensor
         cs.it_done = (u32)it;
         if (it == iters) cs.active = 0;
         else atomicAdd(km.pending, 1u);
+#ifdef EXCP_TRACE_KMEANS
+        if (it != iters) printf("kmeans miss: tensor %d stream %d numel %llu stopped at iteration %d\n", t, stream, descs[t].numel, it);
+#endif
     }
 }
 
