@@ -21,8 +21,8 @@
 // the predicted cells and their neighbours, cell after cell, into a gathered copy (a
 // seventh of the survivors at 4 bits), and the exact iterations run on that copy, one
 // block per tensor and stream.  Should an exact threshold ever leave the gathered
-// cells, the stream stops at that iteration and a second round gathers every cell for
-// it and finishes; the centres are those of full sweeps either way.
+// cells, the stream stops at that iteration; a second round predicts again from there with a
+// wider neighbourhood, a third gathers every cell; the centres are those of full sweeps either way.
 //
 //   kmeans_start    start sample; the cell map
 //   cell_count      sweep: count and fixed-point sum of every cell
@@ -320,8 +320,9 @@ __device__ inline u32 block_of_tile(u32 x, u32 tiles, u32 g) {
 }
 
 // Prefixes of the cell table; the cells the coming iterations will need; their places in the
-// gathered copy.  One block per (tensor, stream).  round 0 predicts; a later round (only for a
-// stream that met a cell it had not gathered) takes every cell.
+// gathered copy.  One block per (tensor, stream).  Round 0 predicts; the later rounds are only for
+// streams that met a cell they had not gathered: one more prediction, then every cell.
+constexpr int KM_ROUNDS = 3;
 __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDesc* __restrict__ descs,
                                                                  TensorState* __restrict__ st, Workspace ws, KmArrays km, int K,
                                                                  int iters, int margin, int round, u32 tiles,
@@ -332,6 +333,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDes
     __shared__ double Lp[KCAP], Sp[KCAP];
     __shared__ s64 wt64[32];
     __shared__ u32 wt32[32];
+    __shared__ u32 smax;
     if (call_aborted(call)) return;
     const int t = blockIdx.x, stream = blockIdx.y, tid = threadIdx.x;
     CellStream& cs = ws.cst[t].s[stream];
@@ -343,6 +345,18 @@ __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDes
 #pragma unroll
     for (int k = 0; k < 4; ++k) cnt[k] = cs.cnt[c0 + k];
     if (tid < NCELL / 32) selw[tid] = 0xffffffffu;
+    if (tid == 0) smax = 0;
+    __syncthreads();
+    atomicMax(&smax, max(max(cnt[0], cnt[1]), max(cnt[2], cnt[3])));
+    __syncthreads();
+    // Where single cells hold far more than their share (values on a coarse grid, as with weights stored in 16
+    // bits), the iterations on the cell table drift further from the exact ones: a wider neighbourhood is copied.
+    if (margin >= 0 && (u64)smax * NCELL > 16ull * nnz) margin = max(margin, 8);
+    // A stream whose first round met a cell it had not copied predicts again from where it stopped (its centres
+    // are exact up to there), with a wider neighbourhood; the last round takes every cell.
+    if (round > 0 && margin >= 0) margin = max(8 * margin, 8);
+    u32 tc = 0;
+    s64 ts = 0;
     if (round == 0) {
         const u32 first_pos = cs.first_pos;
         u32 pc[4];
@@ -353,11 +367,16 @@ __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDes
             const s64 mag = (s64)cs.mag[c0 + k];
             ps[k] = c0 + k < first_pos ? -mag : mag;
         }
-        const u32 tc = block_scan4(pc, wt32);
-        const s64 ts = block_scan4(ps, wt64);
+        tc = block_scan4(pc, wt32);
+        ts = block_scan4(ps, wt64);
 #pragma unroll
         for (int k = 0; k < 4; ++k) { cs.cntpre[c0 + k] = pc[k]; cs.sumpre[c0 + k] = ps[k]; }
         if (tid == 0) { cs.cntpre[NCELL] = tc; cs.sumpre[NCELL] = ts; }
+    } else {
+        tc = cs.cntpre[NCELL];
+        ts = cs.sumpre[NCELL];
+    }
+    if (round < KM_ROUNDS - 1) {
         const bool predict = nnz > SMALL_STREAM && margin < NCELL;
         if (predict) {
             if (tid < NCELL / 32) selw[tid] = 0;
@@ -681,7 +700,7 @@ void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* s
     const size_t g1 = sizeof(CellGatherSmem<1>), g2 = sizeof(CellGatherSmem<2>);
     cudaFuncSetAttribute(cell_gather_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g1);
     cudaFuncSetAttribute(cell_gather_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g2);
-    for (int round = 0; round < 2; ++round) {
+    for (int round = 0; round < KM_ROUNDS; ++round) {
         cell_plan_kernel<<<dim3(nt, 3), PLAN_THREADS, 0, cfg.stream>>>(descs, st, ws, km, K, p.kmeans_iters, p.km_margin, round,
                                                                      tiles, grid, call);
         if (round == 0) prof_mark(cfg, ST_CELL_PLAN, 1);

@@ -478,8 +478,8 @@ def test_profile_counts_launches_and_times_stages(handle):
         handle.compress_tensor(binding.Params(median_source=1, kmeans_iters=10), *dq[0], blob)
         ms, launches = handle.profile_read()
         # statistics, mask sweep, scan + layout, K-means (start, 2 counting sweeps, plan, 2 gathers, iterations,
-        # the second round's 4), header + edges, 2 packing sweeps, bitmaps
-        assert launches == 11 + 1 + 2 + (1 + 2 + 1 + 2 + 1 + 4) + 2 + 2 + 1
+        # the second and third rounds' 4 each), header + edges, 2 packing sweeps, bitmaps
+        assert launches == 11 + 1 + 2 + (1 + 2 + 1 + 2 + 1 + 4 + 4) + 2 + 2 + 1
         assert ms["mask_compact"] > 0 and ms["kmeans_iterate"] > 0 and ms["decode"] == 0
     finally:
         handle.profile_enable(False)
