@@ -765,8 +765,9 @@ def run_ours(args):
     if not args.no_e2e and wb == 4 and not strong:
         need_gb = 16 * n_tot / 1e9
         sub = list(range(len(shapes)))
-        if mem_available_gb() < 1.4 * need_gb + 8:
-            budget, acc, sub = 0.45 * mem_available_gb() * 1e9, 0, []
+        avail_gb = mem_available_gb() / world              # the ranks of one node share its host memory
+        if avail_gb < 1.4 * need_gb + 8:
+            budget, acc, sub = 0.45 * avail_gb * 1e9, 0, []
             for i, (_, n) in enumerate(shapes):
                 if acc + 16 * n > budget:
                     break
