@@ -642,7 +642,8 @@ def run_ours(args):
         "compression": {"blob_bytes": blob_bytes, "ratio_vs_12B_per_param": 12 * n_tot / blob_bytes,
                         "ratio_vs_stored_state": (wb + 8) * n_tot / blob_bytes},
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": dom_gbs / peak, "peak_kind": peak_kind, "traffic": ncu_traffic(dom, n_tot),
+                     "frac": dom_gbs / peak, "peak_kind": peak_kind,
+                     "traffic": ncu_traffic(dom, n_tot) if wb == 4 and args.median == "residual" else None,
                      "algorithmic_bytes_per_step": sb[dom], "ms_per_step": dom_ms, "note": f"{launches} launches per step"},
         "clocks": clocks,
         "gpu_launches": launches * args.steps,
@@ -832,7 +833,7 @@ def run_ours(args):
                              "hbm_frac_of_nominal_8TBs": dec_bytes / (dms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
                              "decode_kernel_ms": kms, "prep_kernels_ms": dstage.get("dec_prep", 0.0),
                              "decode_kernel_frac_of_measured": dec_bytes / (kms * 1e-3) / 1e9 / peak if kms else None,
-                             "traffic": ncu_traffic("decode", n_tot),
+                             "traffic": ncu_traffic("decode", n_tot) if wb == 4 and args.bits == 4 else None,   # the capture is of fp32 weights, 4-bit codes
                              "calls_per_step": 1, "in_place": True}
     del quads, blob
     h.close()
