@@ -48,7 +48,7 @@ def parse_args():
     ap.add_argument("--config", default="llama-7b")
     ap.add_argument("--median", default="residual", choices=["residual", "weight"])
     ap.add_argument("--kmeans-iters", type=int, default=10)
-    ap.add_argument("--workspace-numel", type=int, default=1_700_000_000,
+    ap.add_argument("--workspace-numel", type=int, default=1_800_000_000,
                     help="elements of a group of tensors (the handle's scratch: about 24.3 bytes each)")
     ap.add_argument("--outlier-frac", type=float, default=0.0,
                     help="fraction of the residual at 10x scale (0.01 = the threshold-stress configuration)")

@@ -35,7 +35,7 @@ def test_llama7b_checkpoint_in_the_benchmark_configuration():
     oparams = dict(kmeans_iters=10, median_source=orc.MEDIAN_ABS_RESIDUAL)
     jobs = {i: oracle_pool.submit_compress(tuple(t.cpu().numpy() for t in quads[i]), oparams, i, want_decode=i in (big, mlp))
             for i in (big, mlp, attn, small)}                      # the longest first
-    h = binding.Handle(workspace_numel=1_700_000_000)
+    h = binding.Handle(workspace_numel=1_800_000_000)
     try:
         p = binding.Params(kmeans_iters=10, median_source=binding.MEDIAN_ABS_RESIDUAL)
         blob = torch.empty(int(0.80 * n_tot) + 4096 * len(shapes) + (1 << 20), dtype=torch.uint8, device=DEV)
