@@ -313,8 +313,11 @@ excp_status excp_decompress_dense_checkpoint(excp_handle h, const void* dense, c
  *     Arguments and results are those of excp_decompress_tensor (w_out may be w_prev).
  *   - numel may not exceed EXCP_NOALLOC_MAX_NUMEL; larger tensors return EXCP_ERR_INVALID_ARG
  *     before anything is launched (use a handle for those).
- *   - The first call on a device looks up the array's device address; make that first call
- *     before any stream capture begins.
+ *   - The first call on a device looks up the array's device address, and the first launch of each
+ *     of its kernels makes the CUDA runtime load that kernel's code, which takes a little device
+ *     memory once and may synchronise.  So make one warm-up call per device, with a non-empty
+ *     tensor (every kernel then runs), while memory is still to be had and before any stream capture
+ *     begins; the calls after it do nothing but launch.
  *   - All calls on a device share the one array, which keeps the previous call's contents; each
  *     call clears what it needs cleared.  Calls that overlap on the GPU (two streams, two
  *     threads) race on it: issue them one after the other.
