@@ -127,8 +127,7 @@ constexpr int NCLASS = 512;       // sign x exponent field of an fp32 value = it
 // to 0..NCELL-1 (see cell_of): every (sign, exponent) class owns a power-of-two number of equal
 // steps of the mantissa, more of them where a sample of the survivors is dense.
 struct CellStream {
-    u32 tab[NCLASS];             // class -> (anchor cell << 8) | log2(cells of the class); the anchor is the
-                                 //   class's first cell for positive values, its last for negative ones
+    u32 tab[NCLASS];             // class of the value key (see cell_of) -> (first cell << 8) | mantissa shift
     u32 cnt[NCELL];              // survivors per cell
     u64 mag[NCELL];              // sum of |Q| per cell; once planned: low word = start of the cell in the
                                  //   gathered copy, high word = values gathered so far
@@ -219,15 +218,20 @@ __host__ __device__ inline u64 record_bytes(u64 numel, u64 nnz_w, u64 nnz_o, int
 
 // ---- device helpers ---------------------------------------------------------
 #ifdef __CUDACC__
-// Cell of a value.  Monotone: x < y implies cell_of(x) <= cell_of(y) (negative classes run from
-// the largest exponent down, their cells from the largest mantissa down; then the positive ones
-// upwards), which is all the K-means iterations need of it.  Any bit pattern maps inside the table.
-__device__ __forceinline__ u32 cell_of(float x, const u32* __restrict__ tab) {
+// Cell of a value.  Monotone: x < y implies cell_of(x) <= cell_of(y), which is all the K-means
+// iterations need of it.  The value's bit pattern is first turned into a key that orders like the
+// values (negative: all bits flipped; non-negative: sign bit set); the key's top nine bits are its
+// (sign, exponent) class in value order, and the class's table entry gives its first cell and how far
+// the 23 mantissa bits are shifted down to number the class's cells.  Any bit pattern maps inside
+// the table.
+__device__ __forceinline__ u32 value_key(float x) {
     const u32 bits = __float_as_uint(x);
-    const u32 ent = tab[bits >> 23];
-    const u32 sub = (bits & 0x7fffffu) >> (23u - (ent & 31u));
-    const u32 neg = (u32)((int)bits >> 31);            // 0 or all ones
-    return (ent >> 8) + ((sub ^ neg) - neg);           // anchor + sub, or anchor - sub
+    return bits ^ ((u32)((int)bits >> 31) | 0x80000000u);
+}
+__device__ __forceinline__ u32 cell_of(float x, const u32* __restrict__ tab) {
+    const u32 key = value_key(x);
+    const u32 ent = tab[key >> 23];                    // (first cell << 8) | shift
+    return (ent >> 8) + __funnelshift_r(key & 0x7fffffu, 0u, ent);   // the shift is the entry's low five bits
 }
 
 // A warp gave up waiting for a copy somewhere in this call: every later kernel returns at once, so

@@ -124,8 +124,9 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
     }
     if (tid < KCAP) s.cent[tid] = tid < K ? smp[((2 * tid + 1) * m) / (2 * K)] : 0.f;
     // Cells per class: one each, and the rest in proportion to the class's share of the sample,
-    // rounded down to a power of two.  Classes in value order: negative ones from the largest
-    // exponent down (classes 511..256), then the positive ones upwards (0..255).
+    // rounded down to a power of two.  Classes in value order (the order of the value key's top nine
+    // bits): negative ones from the largest exponent down (sign-and-exponent fields 511..256), then the
+    // positive ones upwards (0..255).
     u32 lg = 0, ncell = 0, incl = 0;
     const int cls = tid < 256 ? 511 - tid : tid - 256;    // class at place `tid` of the value order (tid < 512)
     if (tid < NCLASS) {
@@ -145,7 +146,7 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
         u32 base = 0;
         for (int w = 0; w < (tid >> 5); ++w) base += wtot[w];
         const u32 f = base + incl - ncell;                // first cell of the class
-        cs.tab[cls] = ((cls >= 256 ? f + ncell - 1 : f) << 8) | lg;
+        cs.tab[tid] = (f << 8) | (23u - lg);              // place `tid` of the value order = class of the value key
         if (cls == 0) cs.first_pos = f;
     }
     if (tid == 0) { cs.it_done = 0; cs.active = iters > 0 ? 1u : 0u; }
@@ -395,7 +396,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDes
                         if (cc >= 0 && cc < NCELL) atomicOr(&selw[cc >> 5], 1u << (cc & 31));
                     }
                     // the share of cell c at or below the threshold, by its place between the cell's edges
-                    const u32 bits = __float_as_uint(tj), sh = 23u - (tab[bits >> 23] & 31u);
+                    const u32 bits = __float_as_uint(tj), sh = tab[value_key(tj) >> 23] & 31u;
                     const u32 a_lo = (bits & 0x7fffffffu) >> sh << sh;
                     const u32 a_hi = min(a_lo + (1u << sh), 0x7f7fffffu);
                     const double v_lo = (double)__uint_as_float(a_lo), v_hi = (double)__uint_as_float(a_hi);
