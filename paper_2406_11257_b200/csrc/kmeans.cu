@@ -34,6 +34,22 @@
 
 namespace excp {
 
+// Cell of a value.  Monotone: x < y implies cell_of(x) <= cell_of(y), which is all the K-means
+// iterations need of it.  The value's bit pattern is first turned into a key that orders like the
+// values (negative: all bits flipped; non-negative: sign bit set); the key's top nine bits are its
+// (sign, exponent) class in value order, and the class's table entry gives its first cell and how far
+// the 23 mantissa bits are shifted down to number the class's cells.  Any bit pattern maps inside
+// the table.
+__device__ __forceinline__ u32 value_key(float x) {
+    const u32 bits = __float_as_uint(x);
+    return bits ^ ((u32)((int)bits >> 31) | 0x80000000u);
+}
+__device__ __forceinline__ u32 cell_of(float x, const u32* __restrict__ tab) {
+    const u32 key = value_key(x);
+    const u32 ent = tab[key >> 23];                    // (first cell << 8) | shift
+    return (ent >> 8) + __funnelshift_r(key & 0x7fffffu, 0u, ent);   // the shift is the entry's low five bits
+}
+
 __device__ inline u64 mix64(u64 z) {   // SplitMix64 output function
     z += 0x9E3779B97F4A7C15ull;
     z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
