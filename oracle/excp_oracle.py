@@ -277,6 +277,14 @@ def sample_hash(seed: int, tensor_index: int, stream: int, i: int) -> int:
     return mix64((h + i) & _M64)
 
 
+def sort_values(x: np.ndarray) -> np.ndarray:
+    """x in ascending order; of two zeros the negative one comes first.  Without the second rule
+    the order of -0 and +0 (equal as numbers, different as stored centres) would be whatever the
+    sorting routine happens to do.  They only meet when pruning is switched off: a kept value is
+    never zero otherwise."""
+    return x[np.lexsort((~np.signbit(x), x))]
+
+
 def kmeans_start(s: np.ndarray, k: int, seed: int, tensor_index: int, stream: int) -> np.ndarray:
     """K equal-mass quantiles of a seeded, index-stratified sample of s."""
     nnz = s.size
@@ -289,7 +297,7 @@ def kmeans_start(s: np.ndarray, k: int, seed: int, tensor_index: int, stream: in
         lo = (i * nnz) // m
         hi = ((i + 1) * nnz) // m
         picks[i] = s[lo + sample_hash(seed, tensor_index, stream, i) % (hi - lo)]
-    picks.sort()
+    picks = sort_values(picks)
     for j in range(k):
         c[j] = picks[((2 * j + 1) * m) // (2 * k)]
     return c
@@ -337,7 +345,7 @@ def lloyd(s: np.ndarray, c0: np.ndarray, iters: int) -> tuple[np.ndarray, np.nda
             cnt = int(np.count_nonzero(members))
             if cnt:
                 c[j] = rsum_mean(int(q[members].sum(dtype=np.int64)), cnt, e)
-        c.sort()
+        c = sort_values(c)
     return c, assign(s, c)
 
 

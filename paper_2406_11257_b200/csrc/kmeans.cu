@@ -127,13 +127,13 @@ __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDe
             atomicAdd(&cvalid, 1u);
         }
     }
-    for (int k = 2; k <= SAMPLE_MAX; k <<= 1) {       // bitonic sort, ascending
+    for (int k = 2; k <= SAMPLE_MAX; k <<= 1) {       // bitonic sort, ascending, -0 before +0 (the order of the keys)
         for (int j = k >> 1; j > 0; j >>= 1) {
             const int p = tid ^ j;
             if (p > tid) {
                 const float x = smp[tid], y = smp[p];
                 const bool up = (tid & k) == 0;
-                if ((x > y) == up) { smp[tid] = y; smp[p] = x; }
+                if ((value_key(x) > value_key(y)) == up) { smp[tid] = y; smp[p] = x; }
             }
             __syncthreads();
         }
@@ -675,11 +675,12 @@ __global__ void __launch_bounds__(IT_THREADS) kmeans_iterate_kernel(const Tensor
             cnew[tid] = c;
         }
         __syncthreads();
-        if (tid < K) {                    // sort ascending: rank of each centre among the K (ties by index)
+        if (tid < K) {                    // sort ascending, -0 before +0: rank of each centre among the K (equal bits by index)
             int rank = 0;
+            const u32 kc = value_key(c);
             for (int i = 0; i < K; ++i) {
-                const float o = cnew[i];
-                rank += (o < c) || (o == c && i < tid);
+                const u32 ko = value_key(cnew[i]);
+                rank += (ko < kc) || (ko == kc && i < tid);
             }
             cent[rank] = c;
         }

@@ -353,6 +353,30 @@ def test_kmeans_start_small_sets_and_constant_values():
     assert not orc.kmeans_start(np.zeros(0, np.float32), 15, 0, 0, 0).any()
 
 
+def test_zeros_of_either_sign_among_the_kept_values_have_one_order():
+    """-0 and +0 are equal as numbers but not as stored centres; they can only be kept when pruning is off.
+    The order is fixed (-0 first), so the centres do not depend on the sorting routine or on the order
+    in which equal values arrive."""
+    x = np.array([0.0, 2.0, -0.0, -3.0, 0.0, -0.0, 1e-45, -1e-45], np.float32)
+    for perm in (np.arange(8), np.arange(8)[::-1], np.array([2, 0, 5, 4, 1, 3, 7, 6])):
+        got = orc.sort_values(x[perm])
+        want = sorted(x[perm].tolist(), key=lambda v: (v, not math.copysign(1.0, v) < 0))     # python's sort: by value, then the sign
+        assert got.tolist() == want and np.signbit(got).tolist() == [True, True, True, True, False, False, False, False]
+    # a stream of zeros of both signs and a few values: the first centres are -0, then +0, whatever the order of the input
+    rng = np.random.default_rng(3)
+    s = np.zeros(4000, np.float32)
+    s[rng.random(4000) < 0.5] = -0.0
+    s[::400] = rng.standard_normal(10).astype(np.float32)
+    c0 = orc.kmeans_start(s, 15, 1, 0, 1)
+    zeros = c0[c0 == 0]
+    assert zeros.size >= 10 and np.signbit(zeros).any() and not np.signbit(zeros).all()
+    assert (np.diff(np.signbit(zeros).astype(int)) <= 0).all()      # all -0 before all +0
+    c, idx = orc.lloyd(s, c0, 5)
+    zeros = c[c == 0]
+    assert (np.diff(c) >= 0).all() and (np.diff(np.signbit(zeros).astype(int)) <= 0).all()
+    assert (c[idx][s == 0] == 0).all()
+
+
 def test_kmeans_start_sample_is_stratified():
     s = np.arange(10240, dtype=np.float32)
     c = orc.kmeans_start(s, 15, 123, 4, 1)
