@@ -113,7 +113,7 @@ constexpr int PWARPS = TPB / 32;
 
 template <int NS, int NB, bool SSE>
 struct PackSmem {
-    float thr[PWARPS][NS][1 << NB];     // the K - 1 thresholds, +inf after them
+    float thr[PWARPS][NS][1 << NB];     // the K - 1 thresholds, +inf after them: sorted (4 bits) or as find_cluster's tree
     float cent[PWARPS][NS][SSE ? (1 << NB) : 1];   // the K centres (only when the quantisation error is wanted)
 };
 
@@ -128,15 +128,22 @@ __device__ __forceinline__ u32 find_cluster4(float x, float t3, float t7, float 
     return p;
 }
 
-// Cluster of x = number of thresholds below it: NB halving steps over the 2^NB - 1 sorted entries
-// (thr[K - 1 ...] = +inf).
+// Cluster of x = number of thresholds below it, for the widths other than 4: NB steps down the
+// search tree of the 2^NB - 1 sorted entries (the last ones +inf), stored level by level: node i
+// (the root is 1) has the children 2i and 2i + 1.  With the sorted array itself the probes of one
+// level lie a power of two apart, all in one shared-memory bank; level by level they are neighbours.
 template <int NB>
-__device__ __forceinline__ u32 find_cluster(float x, const float* thr) {
-    u32 p = 0;
+__device__ __forceinline__ u32 find_cluster(float x, const float* tree) {
+    u32 i = 1;
 #pragma unroll
-    for (int step = 1 << (NB - 1); step; step >>= 1)
-        if (x > thr[p + step - 1]) p += step;
-    return p;
+    for (int step = 0; step < NB; ++step) i = 2u * i + (x > tree[i] ? 1u : 0u);
+    return i - (1u << NB);
+}
+// Place in the sorted array of node i of that tree.
+template <int NB>
+__device__ __forceinline__ u32 tree_source(u32 i) {
+    const u32 level = 31u - (u32)__clz((int)i);
+    return ((2u * (i - (1u << level)) + 1u) << (NB - 1 - level)) - 1u;
 }
 
 // SSE: also add up the squared distances to the assigned centres (the statistics' sse_* fields).
@@ -197,7 +204,8 @@ __global__ void __launch_bounds__(TPB) pack_codes_kernel(const TensorDesc* __res
                 for (int k = 0; k < NS; ++k) {
                     words[k] = reinterpret_cast<u32*>(blob + s.blob_off + sec.codes[stream0 + k]);
                     for (int j = lane; j < KTHR; j += 32) {
-                        sm.thr[warp][k][j] = s.s[stream0 + k].thr[j];
+                        if (NB == 4) sm.thr[warp][k][j] = s.s[stream0 + k].thr[j];
+                        else if (j) sm.thr[warp][k][j] = s.s[stream0 + k].thr[tree_source<NB>((u32)j)];
                         if (SSE) sm.cent[warp][k][j] = s.s[stream0 + k].cent[j];
                     }
                 }
