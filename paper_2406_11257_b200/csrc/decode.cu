@@ -313,7 +313,11 @@ __device__ __forceinline__ u32 decode_block(const DecTile& t, const DecDesc& d, 
     const WT* w_prev = static_cast<const WT*>(d.w_prev);
     WT* w_out = static_cast<WT*>(d.w_out);
     const bool absolute = t.rflags & REC_ABSOLUTE;       // the weight stream is W itself
-    const float* cw = NB <= 4 ? sm.cent[warp][0] : s.cent[0];   // wide codes: the table stays in global memory (cached)
+    // Codes of at most 4 bits: the tables in shared memory are indexed by the code itself, and code 0 (pruned)
+    // finds 0 for the moments and -0 for the weights: x + (-0) = x for every x, so a pruned weight keeps
+    // W^_(t-1) bit for bit (and an absolute one becomes 0 + (-0) = +0) with no test of the code.
+    // Wide codes: the tables stay in global memory (cached), entry code - 1.
+    const float* cw = NB <= 4 ? sm.cent[warp][0] : s.cent[0];
     const float* ca = NB <= 4 ? sm.cent[warp][1] : s.cent[1];
     const float* cs = NB <= 4 ? sm.cent[warp][2] : s.cent[2];
     constexpr int RB = EXCP_DEC_RB;
@@ -339,9 +343,15 @@ __device__ __forceinline__ u32 decode_block(const DecTile& t, const DecDesc& d, 
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 const u32 c0 = (kw >> (8 * k)) & 255u, c1 = (ka >> (8 * k)) & 255u, c2 = (ks >> (8 * k)) & 255u;
-                ow[k] = c0 ? __fadd_rn(wp[r][k], cw[c0 - 1]) : wp[r][k];   // pruned: W^_(t-1) bit for bit
-                oa[k] = c1 ? ca[c1 - 1] : 0.f;
-                os[k] = c2 ? cs[c2 - 1] : 0.f;
+                if (NB <= 4) {
+                    ow[k] = __fadd_rn(wp[r][k], cw[c0]);
+                    oa[k] = ca[c1];
+                    os[k] = cs[c2];
+                } else {
+                    ow[k] = c0 ? __fadd_rn(wp[r][k], cw[c0 - 1]) : wp[r][k];   // pruned: W^_(t-1) bit for bit
+                    oa[k] = c1 ? ca[c1 - 1] : 0.f;
+                    os[k] = c2 ? cs[c2 - 1] : 0.f;
+                }
             }
             store4(w_out, i0, t.n, ow);
             store4(d.ea_out, i0, t.n, oa);
@@ -424,8 +434,10 @@ __global__ void __launch_bounds__(TPB, DENSE ? EXCP_DENSE_MIN_BLOCKS : EXCP_DEC_
             __syncwarp();
             if (!DENSE && st[cur].valid && st[cur].bits <= 4) {
                 const int kc = centres_of((int)st[cur].bits);
-                for (int i = lane; i < 3 * CENT_SMEM; i += 32)
-                    sm.cent[warp][i / CENT_SMEM][i % CENT_SMEM] = i % CENT_SMEM < kc ? st[cur].cent[i / CENT_SMEM][i % CENT_SMEM] : 0.f;
+                for (int i = lane; i < 3 * CENT_SMEM; i += 32) {       // entry c = centre of code c; entry 0: see decode_block
+                    const int k = i / CENT_SMEM, c = i % CENT_SMEM;
+                    sm.cent[warp][k][c] = c == 0 ? (k == 0 ? -0.f : 0.f) : c <= kc ? st[cur].cent[k][c - 1] : 0.f;
+                }
             }
             __syncwarp();
         }
@@ -622,7 +634,7 @@ __global__ void __launch_bounds__(TPB) dense_decode_kernel(const DecDesc* __rest
             tb = descs[cur].tile_begin; ntl = descs[cur].num_tiles;
             if (tid < 3 * (KPAD + 1)) {
                 const int k = tid / (KPAD + 1), j = tid % (KPAD + 1);
-                cent[k][j] = j ? st[cur].cent[k][j - 1] : 0.f;
+                cent[k][j] = j ? st[cur].cent[k][j - 1] : k == 0 ? -0.f : 0.f;   // x + (-0) = x: a pruned weight keeps its bits
             }
             __syncthreads();
         }
@@ -634,41 +646,61 @@ __global__ void __launch_bounds__(TPB) dense_decode_kernel(const DecDesc* __rest
         const u64 sb = dense_section_bytes(n, BITS);
         const unsigned char* sec = d.rec + header_bytes(KMAX);
         const u64 base = (u64)(tile - tb) * TILE;
-        // all loads of the tile's four rounds first, then the arithmetic and the stores
-        u32 ww[ROUNDS], wa[ROUNDS], we[ROUNDS];
-        float wp[ROUNDS][4];
+        // All loads of the tile first, then the arithmetic and the stores.  In a round a warp has 256
+        // elements: every lane loads one 32-bit word of codes per stream (its eight elements) and, twice, four
+        // weights in the order that keeps a warp's 16-byte accesses contiguous (lane l: elements 4l.. of each
+        // half); the codes of those four come from lane l/2 of that half by a shuffle.
+        constexpr int R8 = TILE / (TPB * 8);
+        u32 ww[R8], wa[R8], we[R8];
+        float wp[R8][2][4];
 #pragma unroll
-        for (int r = 0; r < ROUNDS; ++r) {
-            const u64 i0 = base + r * (TPB * 4) + tid * 4;     // four elements = 16 bits per stream
+        for (int r = 0; r < R8; ++r) {
+            const u64 w0 = base + (u64)r * (TPB * 8) + (u64)(tid >> 5) * 256u;     // the warp's first element
+            const u64 e0 = w0 + 8u * lane;                 // a section is padded to whole 16-byte units: the word exists
             ww[r] = wa[r] = we[r] = 0;
-            wp[r][0] = wp[r][1] = wp[r][2] = wp[r][3] = 0.f;
-            if (i0 < n) {
-                ww[r] = *reinterpret_cast<const unsigned short*>(sec + i0 / 2);
-                wa[r] = *reinterpret_cast<const unsigned short*>(sec + sb + i0 / 2);
-                we[r] = *reinterpret_cast<const unsigned short*>(sec + 2 * sb + i0 / 2);
-                load4(w_prev, i0, n, wp[r]);
+            if (e0 < n) {
+                ww[r] = *reinterpret_cast<const u32*>(sec + e0 / 2);
+                wa[r] = *reinterpret_cast<const u32*>(sec + sb + e0 / 2);
+                we[r] = *reinterpret_cast<const u32*>(sec + 2 * sb + e0 / 2);
+            }
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const u64 i0 = w0 + 128u * h + 4u * lane;
+                wp[r][h][0] = wp[r][h][1] = wp[r][h][2] = wp[r][h][3] = 0.f;
+                if (i0 < n) load4(w_prev, i0, n, wp[r][h]);
             }
         }
 #pragma unroll
-        for (int r = 0; r < ROUNDS; ++r) {
-            const u64 i0 = base + r * (TPB * 4) + tid * 4;
-            if (i0 >= n) continue;
-            const u32 zw = nonzero_nibbles(ww[r]), za = nonzero_nibbles(wa[r]), ze = nonzero_nibbles(we[r]);
-            cw += __popc(zw); co += __popc(za);
-            bad |= (za ^ ze) | (za & ~zw);                // moments disagree; a moment kept where the weight is pruned
-            const u32 left = n - i0 >= 4 ? 4u : (u32)(n - i0);
-            if (left < 4 && ((ww[r] | wa[r] | we[r]) >> (4 * left))) bad = 1;   // codes past the last element
-            float ow[4], oa[4], os[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const u32 c0 = (ww[r] >> (4 * k)) & 15u, c1 = (wa[r] >> (4 * k)) & 15u, c2 = (we[r] >> (4 * k)) & 15u;
-                ow[k] = c0 ? __fadd_rn(wp[r][k], cent[0][c0]) : wp[r][k];    // pruned: W^_(t-1) bit for bit
-                oa[k] = cent[1][c1];
-                os[k] = cent[2][c2];
+        for (int r = 0; r < R8; ++r) {
+            const u64 w0 = base + (u64)r * (TPB * 8) + (u64)(tid >> 5) * 256u;
+            const u64 e0 = w0 + 8u * lane;
+            if (e0 < n) {                                   // the checks, on the lane's own eight elements
+                const u32 zw = nonzero_nibbles(ww[r]), za = nonzero_nibbles(wa[r]), ze = nonzero_nibbles(we[r]);
+                cw += __popc(zw); co += __popc(za);
+                bad |= (za ^ ze) | (za & ~zw);            // moments disagree; a moment kept where the weight is pruned
+                const u32 left = n - e0 >= 8 ? 8u : (u32)(n - e0);
+                if (left < 8 && ((ww[r] | wa[r] | we[r]) >> (4 * left))) bad = 1;   // codes past the last element
             }
-            store4(w_out, i0, n, ow);
-            store4(d.ea_out, i0, n, oa);
-            store4(d.eas_out, i0, n, os);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int src = 16 * h + (lane >> 1), sh = 16 * (lane & 1);
+                const u32 kw = __shfl_sync(0xffffffffu, ww[r], src) >> sh;
+                const u32 ka = __shfl_sync(0xffffffffu, wa[r], src) >> sh;
+                const u32 ke = __shfl_sync(0xffffffffu, we[r], src) >> sh;
+                const u64 i0 = w0 + 128u * h + 4u * lane;
+                if (i0 >= n) continue;
+                float ow[4], oa[4], os[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const u32 c0 = (kw >> (4 * k)) & 15u, c1 = (ka >> (4 * k)) & 15u, c2 = (ke >> (4 * k)) & 15u;
+                    ow[k] = __fadd_rn(wp[r][h][k], cent[0][c0]);      // code 0: + (-0), W^_(t-1) bit for bit
+                    oa[k] = cent[1][c1];
+                    os[k] = cent[2][c2];
+                }
+                store4(w_out, i0, n, ow);
+                store4(d.ea_out, i0, n, oa);
+                store4(d.eas_out, i0, n, os);
+            }
         }
     }
     if (cur >= 0) flush(cur);
