@@ -26,7 +26,9 @@
  *     = number of mid-points (c_j + c_j+1)/2, taken in fp64, lying strictly below x; update =
  *     fixed-point mean (values scaled by 2^(30-E), E = exponent of the stream's largest
  *     magnitude, rounded half-to-even, summed in int64); empty clusters keep their centre;
- *     centres re-sorted; `kmeans_iters` iterations, then the final assignment.
+ *     centres kept in ascending order, -0 before +0 (they can only meet with pruning switched
+ *     off: a kept value is never zero otherwise); `kmeans_iters` iterations, then the final
+ *     assignment.
  *
  * Record layout of one tensor (little endian, every section on a 16-byte boundary, padding zero):
  *     0 u32 magic "EXCP"   4 u32 version = 1     8 u64 numel
