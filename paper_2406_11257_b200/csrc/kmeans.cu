@@ -371,7 +371,9 @@ __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDes
     if (margin >= 0 && (u64)smax * NCELL > 16ull * nnz) margin = max(margin, 8);
     // A stream whose first round met a cell it had not copied predicts again from where it stopped (its centres
     // are exact up to there), with a wider neighbourhood; the last round takes every cell.
-    if (round > 0 && margin >= 0) margin = max(8 * margin, 8);
+    // (With 255 centres a cluster is about 16 cells wide and eight cells either side would be every cell already:
+    // there the second round widens to two.)
+    if (round > 0 && margin >= 0) margin = K > 15 ? max(2 * margin, 2) : max(8 * margin, 8);
     u32 tc = 0;
     s64 ts = 0;
     if (round == 0) {
