@@ -30,6 +30,7 @@
 //   cell_gather     sweep: values of the selected cells into the gathered copy
 //   kmeans_iterate  the exact iterations
 #include "excp_common.cuh"
+#include <cooperative_groups.h>
 #include <cstdio>
 
 namespace excp {
@@ -573,7 +574,9 @@ __global__ void __launch_bounds__(CWARPS * 32, 2) cell_gather_kernel(const Tenso
 // ---------------------------------------------------------------------------
 constexpr int IT_THREADS = 1024;
 constexpr int IT_WARPS = IT_THREADS / 32;
-constexpr int IT_PARTS = 4;          // at most this many warps share one threshold's cell
+constexpr int IT_PARTS = 4;          // at most this many warps of a block share one threshold's cell
+constexpr int IT_CLUSTER = 4;        // blocks (one thread-block cluster) that share a large stream's iterations at wide codes
+constexpr u32 IT_LARGE = 2u << 20;   // survivors from which a stream counts as large (measured: 4 x 2 M best of 2..8 x 1..24 M)
 
 // Count and fixed-point sum of the values of data[a, e) at or below thr; whole warp.
 __device__ __forceinline__ void scan_range(const float* __restrict__ data, u32 a, u32 e, float thr, float s1,
@@ -600,26 +603,47 @@ __device__ __forceinline__ void scan_range(const float* __restrict__ data, u32 a
     if (be + lane < e) test(__ldg(data + be + lane));
 }
 
-// The exact iterations of one stream, from iteration it_done on: one block per (tensor, stream).
-// L_j = survivors at or below threshold j = the cells below its cell, whole, + the part of its own
-// cell found by looking at the gathered values; cluster k has L_k - L_(k-1) members (L_-1 = 0,
-// L_(K-1) = all), and its sum likewise.  If a threshold's cell has values and was not gathered,
-// the stream stops here, stays active and is counted in km_pending.
+// The exact iterations of one stream, from iteration it_done on: one block, or one thread-block
+// cluster, per (tensor, stream); streams whose number of survivors is outside [nnz_lo, nnz_hi) are
+// left to another launch.  L_j = survivors at or below threshold j = the cells below its cell,
+// whole, + the part of its own cell found by looking at the gathered values; cluster k has
+// L_k - L_(k-1) members (L_-1 = 0, L_(K-1) = all), and its sum likewise.  If a threshold's cell has
+// values and was not gathered, the stream stops here, stays active and is counted in km_pending.
+// Launched as clusters, the blocks split every threshold's cell between them (with 255 centres a large
+// tensor's ten iterations read hundreds of MB, and one block's load bandwidth would set the time of the
+// launch), leave their counts and integer sums in their own shared memory, and after the cluster's
+// barrier every block reads all of them through distributed shared memory and computes the same new
+// centres, so nothing is sent back.  The shares are double-buffered: one barrier per iteration.
+// Every block of a cluster takes the same way through the kernel (what decides it: the call's time-out
+// flag, which no K-means kernel sets; the stream's state, which only block 0 writes, after the last
+// barrier; thresholds that are the same in every block), so every barrier is reached by all of them
+// and none leaves while another may still read its shared memory.
+// CL: launched as clusters (otherwise the kernel is the plain one-block form: a block barrier, one buffer).
+template <bool CL>
 __global__ void __launch_bounds__(IT_THREADS) kmeans_iterate_kernel(const TensorDesc* __restrict__ descs,
                                                                     TensorState* __restrict__ st, Workspace ws, KmArrays km, int K,
-                                                                    int iters, const CallState* call) {
+                                                                    int iters, const CallState* call, u32 nnz_lo, u32 nnz_hi) {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
     __shared__ u32 tab[NCLASS];
     __shared__ u32 selw[NCELL / 32];
     __shared__ float cent[KCAP], thr[KCAP], cnew[KCAP];
     __shared__ u32 cellj[KCAP];
-    __shared__ u32 pcnt[KCAP][IT_PARTS];
-    __shared__ s64 psum[KCAP][IT_PARTS];
+    __shared__ u32 pcnt[CL ? 2 : 1][KCAP][IT_PARTS];
+    __shared__ s64 psum[CL ? 2 : 1][KCAP][IT_PARTS];
     __shared__ u64 Ls[KCAP];
     __shared__ s64 Ss[KCAP];
     if (call_aborted(call)) return;
-    const int t = blockIdx.x, stream = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const u32 crank = CL ? cluster.block_rank() : 0u, csize = CL ? cluster.num_blocks() : 1u;
+    const u32 unit = blockIdx.x / csize;                 // a cluster's blocks are neighbours in x
+    const u32 nt = gridDim.x / (3u * csize);             // all dW streams first: they are the long ones
+    const int t = (int)(unit % nt), stream = (int)(unit / nt), tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     CellStream& cs = ws.cst[t].s[stream];
     if (!cs.active) return;
+    {
+        const u64 nnz = stream == 0 ? st[t].nnz_w : st[t].nnz_o;
+        if (nnz < nnz_lo || nnz >= nnz_hi) return;
+    }
     StreamState& s = st[t].s[stream];
     if (tid < NCLASS) tab[tid] = cs.tab[tid];
     if (tid < NCELL / 32) selw[tid] = cs.sel[tid];
@@ -630,7 +654,9 @@ __global__ void __launch_bounds__(IT_THREADS) kmeans_iterate_kernel(const Tensor
     const int parts = max(1, min(IT_PARTS, IT_WARPS / max(K - 1, 1)));
     __syncthreads();
     int it = (int)cs.it_done;
-    for (; it < iters; ++it) {
+    const u32 allparts = (u32)parts * csize;             // shares of a threshold's cell over the whole cluster
+    int buf = 0;
+    for (; it < iters; ++it, buf ^= CL ? 1 : 0) {
         bool ok = true;
         if (tid < K - 1) {
             const u32 c = cell_of(thr[tid], tab);
@@ -645,23 +671,33 @@ __global__ void __launch_bounds__(IT_THREADS) kmeans_iterate_kernel(const Tensor
             s64 sum = 0;
             if ((selw[c >> 5] >> (c & 31)) & 1u) {
                 const u32 b = (u32)cs.mag[c], n = cs.cntpre[c + 1] - cs.cntpre[c];
+                const u32 gp = crank * (u32)parts + (u32)p;              // this warp's share among the cluster's
                 if (EXCP_IN_BOUNDS(call, (u64)b + n <= (u64)descs[t].num_tiles * TILE))
-                scan_range(data, b + (u32)(((u64)n * p) / parts), b + (u32)(((u64)n * (p + 1)) / parts), thr[j], s1, s2,
+                scan_range(data, b + (u32)(((u64)n * gp) / allparts), b + (u32)(((u64)n * (gp + 1)) / allparts), thr[j], s1, s2,
                            lane, cnt, sum);
             }
             cnt = __reduce_add_sync(0xffffffffu, cnt);
 #pragma unroll
             for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-            if (lane == 0) { pcnt[j][p] = cnt; psum[j][p] = sum; }
+            if (lane == 0) { pcnt[buf][j][p] = cnt; psum[buf][j][p] = sum; }
         }
-        __syncthreads();
+        if (CL) cluster.sync();                          // every block's shares are in its shared memory
+        else __syncthreads();
         u64 L = 0;
         s64 S = 0;
         if (tid < K - 1) {
             const u32 c = cellj[tid];
             L = cs.cntpre[c];
             S = cs.sumpre[c];
-            for (int p = 0; p < parts; ++p) { L += pcnt[tid][p]; S += psum[tid][p]; }
+            if (CL) {
+                for (u32 r = 0; r < csize; ++r) {
+                    const u32* rc = cluster.map_shared_rank(&pcnt[buf][tid][0], r);
+                    const s64* rs = cluster.map_shared_rank(&psum[buf][tid][0], r);
+                    for (int p = 0; p < parts; ++p) { L += rc[p]; S += rs[p]; }
+                }
+            } else {
+                for (int p = 0; p < parts; ++p) { L += pcnt[0][tid][p]; S += psum[0][tid][p]; }
+            }
         } else if (tid == K - 1) {
             L = cs.cntpre[NCELL];
             S = cs.sumpre[NCELL];
@@ -690,6 +726,10 @@ __global__ void __launch_bounds__(IT_THREADS) kmeans_iterate_kernel(const Tensor
         set_thresholds(cent, thr, K, tid, IT_THREADS);
         __syncthreads();
     }
+    if (CL) {
+        cluster.sync();                                  // nobody still reads this block's shares
+        if (crank != 0) return;
+    }
     if (tid < KCAP) { s.cent[tid] = cent[tid]; s.thr[tid] = thr[tid]; }
     if (tid == 0) {
         cs.it_done = (u32)it;
@@ -699,6 +739,30 @@ __global__ void __launch_bounds__(IT_THREADS) kmeans_iterate_kernel(const Tensor
         if (it != iters) printf("kmeans miss: tensor %d stream %d numel %llu stopped at iteration %d\n", t, stream, descs[t].numel, it);
 #endif
     }
+}
+
+// With up to 15 centres: one block per (tensor, stream).  With more, the large streams go to a second
+// launch as clusters of IT_CLUSTER blocks, side by side in x (a block of either launch whose stream
+// belongs to the other returns at once).
+static void launch_iterate(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st, int nt, const Workspace& ws,
+                           const KmArrays& km, int K, int iters, const CallState* call) {
+    const bool split = K > 15;
+    kmeans_iterate_kernel<false><<<(unsigned)nt * 3u, IT_THREADS, 0, cfg.stream>>>(descs, st, ws, km, K, iters, call, 0u,
+                                                                           split ? IT_LARGE : 0xffffffffu);
+    if (!split) return;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3((unsigned)nt * 3u * (unsigned)IT_CLUSTER, 1, 1);
+    lc.blockDim = dim3(IT_THREADS, 1, 1);
+    lc.dynamicSmemBytes = 0;
+    lc.stream = cfg.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = IT_CLUSTER;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    cudaLaunchKernelEx(&lc, kmeans_iterate_kernel<true>, descs, st, ws, km, K, iters, call, (u32)IT_LARGE, 0xffffffffu);
 }
 
 void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* st, int nt, u32 tiles,
@@ -727,8 +791,8 @@ void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* s
         cell_gather_kernel<1><<<grid, CWARPS * 32, g1, cfg.stream>>>(descs, nt, tiles, ws, km, 0, call, round);
         cell_gather_kernel<2><<<grid, CWARPS * 32, g2, cfg.stream>>>(descs, nt, tiles, ws, km, 1, call, round);
         if (round == 0) prof_mark(cfg, ST_CELL_GATHER, 2);
-        kmeans_iterate_kernel<<<dim3(nt, 3), IT_THREADS, 0, cfg.stream>>>(descs, st, ws, km, K, p.kmeans_iters, call);
-        prof_mark(cfg, round == 0 ? ST_KMEANS_ITERATE : ST_KMEANS_RETRY, round == 0 ? 1 : 4);
+        launch_iterate(cfg, descs, st, nt, ws, km, K, p.kmeans_iters, call);
+        prof_mark(cfg, round == 0 ? ST_KMEANS_ITERATE : ST_KMEANS_RETRY, (round == 0 ? 0 : 3) + (K > 15 ? 2 : 1));   // launches since the last mark
     }
 }
 
