@@ -70,6 +70,8 @@ __device__ inline void set_thresholds(const float* cent, float* thr, int K, int 
 
 constexpr int CELL_SAMPLE = 4096;    // survivors whose classes apportion the cells
 constexpr u32 SMALL_STREAM = 16384;  // at most this many survivors: every cell is gathered
+constexpr u32 SMALL_STREAM_WIDE = 1u << 20;   // the same with 255 centres: a cluster then has few values per cell, the prediction
+                                              // of such a stream fails four times in ten, and its whole copy costs less than the second round
 
 // One block per (tensor, stream).
 __global__ void __launch_bounds__(SAMPLE_MAX) kmeans_start_kernel(const TensorDesc* __restrict__ descs,
@@ -397,7 +399,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDes
         ts = cs.sumpre[NCELL];
     }
     if (round < KM_ROUNDS - 1) {
-        const bool predict = nnz > SMALL_STREAM && margin < NCELL;
+        const bool predict = nnz > (K > 15 ? SMALL_STREAM_WIDE : SMALL_STREAM) && margin < NCELL;
         if (predict) {
             if (tid < NCELL / 32) selw[tid] = 0;
             if (tid < NCLASS) tab[tid] = cs.tab[tid];
