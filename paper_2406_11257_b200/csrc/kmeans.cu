@@ -433,6 +433,11 @@ __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDes
                         const double x = fabs((double)tj);
                         f = half > 0.0 ? (x - (mean - half)) / (2.0 * half) : (x >= mean ? 1.0 : 0.0);
                         f = fmin(fmax(f, 0.0), 1.0);
+                        // A threshold exactly on the cell's lower edge (the first thresholds are mid-points of sampled values,
+                        // and values on a grid, such as residuals of 16-bit weights, sit on cell edges): the values equal to it
+                        // count as at or below it.  If the cell is a point mass on that edge plus an even spread, its mean
+                        // says how much the point holds.  (Below zero the equal values count already: 1 - f.)
+                        if (!(bits >> 31) && x == v_lo && v_hi > v_lo) f = fmax(f, fmax(0.0, 1.0 - 2.0 * (mean - v_lo) / (v_hi - v_lo)));
                     }
                     if (bits >> 31) f = 1.0 - f;
                     Lp[tid] = (double)cs.cntpre[c] + f * n_c;
