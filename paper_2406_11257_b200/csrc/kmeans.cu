@@ -345,7 +345,7 @@ __device__ inline u32 block_of_tile(u32 x, u32 tiles, u32 g) {
 constexpr int KM_ROUNDS = 3;
 __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDesc* __restrict__ descs,
                                                                  TensorState* __restrict__ st, Workspace ws, KmArrays km, int K,
-                                                                 int iters, int margin, int round, u32 tiles,
+                                                                 int iters, int margin, int w16, int round, u32 tiles,
                                                                  u32 grid, const CallState* call) {
     __shared__ u32 tab[NCLASS];
     __shared__ u32 selw[NCELL / 32];
@@ -360,6 +360,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDes
     if (!cs.active) return;
     const StreamState& s = st[t].s[stream];
     const u32 nnz = stream == 0 ? st[t].nnz_w : st[t].nnz_o;
+    const bool gridded = w16 && stream == 0;           // dW of weights stored in 16 bits
     const u32 c0 = 4u * tid;                           // this thread's cells
     u32 cnt[4];
 #pragma unroll
@@ -431,6 +432,13 @@ __global__ void __launch_bounds__(PLAN_THREADS) cell_plan_kernel(const TensorDes
                         const double mean = fmin(fmax(fabs(s_c / n_c * scale), v_lo), v_hi);
                         const double half = fmin(mean - v_lo, v_hi - mean);
                         const double x = fabs((double)tj);
+                        if (gridded && mean - v_lo <= v_hi - mean && v_hi > v_lo) {
+                            // Values known to lie on a grid (residuals of 16-bit weights): grid points are cell edges, so
+                            // the cell is taken as a point mass on its lower edge plus an even spread, with the cell's mean.
+                            // f is the share of magnitudes at or below x above zero, strictly below x under it.
+                            const double w = v_hi - v_lo, pm = 1.0 - 2.0 * (mean - v_lo) / w;
+                            f = (!(bits >> 31) || x > v_lo ? pm : 0.0) + (1.0 - pm) * (x - v_lo) / w;
+                        } else
                         f = half > 0.0 ? (x - (mean - half)) / (2.0 * half) : (x >= mean ? 1.0 : 0.0);
                         f = fmin(fmax(f, 0.0), 1.0);
                         // A threshold exactly on the cell's lower edge (the first thresholds are mid-points of sampled values,
@@ -792,7 +800,7 @@ void launch_kmeans(const LaunchCfg& cfg, const TensorDesc* descs, TensorState* s
     cudaFuncSetAttribute(cell_gather_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g1);
     cudaFuncSetAttribute(cell_gather_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g2);
     for (int round = 0; round < KM_ROUNDS; ++round) {
-        cell_plan_kernel<<<dim3(nt, 3), PLAN_THREADS, 0, cfg.stream>>>(descs, st, ws, km, K, p.kmeans_iters, p.km_margin, round,
+        cell_plan_kernel<<<dim3(nt, 3), PLAN_THREADS, 0, cfg.stream>>>(descs, st, ws, km, K, p.kmeans_iters, p.km_margin, p.wfmt != WF_F32, round,
                                                                      tiles, grid, call);
         if (round == 0) prof_mark(cfg, ST_CELL_PLAN, 1);
         cell_gather_kernel<1><<<grid, CWARPS * 32, g1, cfg.stream>>>(descs, nt, tiles, ws, km, 0, call, round);
